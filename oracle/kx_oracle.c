@@ -1,0 +1,191 @@
+/*
+ * CPU ORACLE — TEST INFRASTRUCTURE, NOT PART OF THE PRODUCT.
+ *
+ * A plain, slow, obviously-correct definition of the BF16 attention output
+ * projection with residual addition,
+ *
+ *     ref[m,n] = sum_{k=0..K-1} X[m,k] * W[n,k]  (+ bias[n])  (+ R[m,n]),
+ *
+ * which is the row-major form of the paper's residual GEMM epilogue
+ * D = alpha * W^T A + beta * C with C = D, alpha = beta = 1 (Appendix A,
+ * "L1-030: attention output projection with residual", Algorithm 3, last two
+ * steps: the output is aliased onto the residual and O <- W^T A + O), and,
+ * with bias = R = NULL, the plain BF16 matrix product of the paper's
+ * fixed-shape GEMM study (Section 4.1).
+ *
+ * Arithmetic: every BF16 input is widened exactly to double; each product of
+ * two BF16 values is exact in double (8 x 8 significant bits); the sum runs
+ * over k in increasing order, one output element at a time; bias and residual
+ * are added last, in that order; the result is kept as an unrounded double.
+ * The four outputs handled per inner loop are independent elements: nothing
+ * is blocked, fused or reordered inside one element's sum.
+ *
+ * Only tests, the smoke check and the benchmark's CPU-baseline leg may call
+ * this.  It shares no code, header, table or helper with the CUDA path.
+ *
+ * Pins (tests that run without a GPU): exact rational brute force on tiny
+ * shapes, agreement with a float64 library matmul, closed forms (constant
+ * operands, one-hot selectors), the invariants W=0, W=I and linearity in X,
+ * and a hand-computed fixture.  The paper prints no worked numerical example
+ * for this operation, so no fixture carries paper-printed values.
+ */
+#include <fenv.h>
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+/* BF16 bit pattern -> double (exact): BF16 is the upper half of an FP32. */
+static inline double bf16_widen(uint16_t b) {
+    uint32_t u = (uint32_t)b << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+int kx_oracle_max_threads(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+void kx_oracle_widen_bf16(const uint16_t* in, double* out, int64_t n) {
+    for (int64_t i = 0; i < n; ++i) out[i] = bf16_widen(in[i]);
+}
+
+/*
+ * double -> BF16 bits, ONE round-to-nearest-even from the exact value.
+ * BF16 has 8 significant bits (1 implicit + 7 stored) and FP32's exponent
+ * range: normal binades 2^-126 .. 2^127, subnormal quantum 2^-133.
+ * For |x| in [2^e, 2^(e+1)) the representable grid has spacing q = 2^(e-7);
+ * x/q is exact (q is a power of two) and nearbyint() under the default
+ * rounding mode rounds half-way cases to the even integer, i.e. to the BF16
+ * value whose last stored bit is zero.
+ */
+static uint16_t bf16_round_one(double x) {
+    if (isnan(x)) return 0x7FC0;
+    uint16_t sign = signbit(x) ? 0x8000 : 0;
+    double a = fabs(x);
+    if (isinf(a)) return (uint16_t)(sign | 0x7F80);
+    if (a == 0.0) return sign;
+    int ex;
+    (void)frexp(a, &ex);           /* a = f * 2^ex, f in [0.5,1)  => 2^(ex-1) <= a */
+    int e = ex - 1;
+    if (e < -126) e = -126;        /* subnormal range shares the 2^-126 binade's grid */
+    double q = ldexp(1.0, e - 7);
+    double r = nearbyint(a / q) * q;   /* exact: integer < 2^9 times a power of two */
+    if (r >= ldexp(1.0, 128)) return (uint16_t)(sign | 0x7F80);
+    float f = (float)r;            /* exact: r has <= 8 significant bits */
+    uint32_t u;
+    memcpy(&u, &f, sizeof u);
+    return (uint16_t)(sign | (uint16_t)(u >> 16));
+}
+
+void kx_oracle_round_bf16(const double* in, uint16_t* out, int64_t n) {
+    fesetround(FE_TONEAREST);
+    for (int64_t i = 0; i < n; ++i) out[i] = bf16_round_one(in[i]);
+}
+
+/*
+ * Reference for a set of rows.
+ *   X    [M,K]  BF16 bits, row-major (host)
+ *   W    [N,K]  BF16 bits, row-major (host)
+ *   bias [N]    BF16 bits or NULL
+ *   R    [M,N]  BF16 bits or NULL
+ *   rows [nrows] row indices into X / R, or NULL meaning rows 0..nrows-1
+ *   ref    [nrows,N] out: unrounded double
+ *   absref [nrows,N] out or NULL: sum_k |X||W| + |bias| + |R|
+ * Returns 0, or -1 on a bad argument / failed allocation.
+ */
+int kx_oracle_outproj_rows(const uint16_t* X, const uint16_t* W, const uint16_t* bias,
+                           const uint16_t* R, const int64_t* rows, int64_t nrows,
+                           double* ref, double* absref,
+                           int64_t M, int64_t N, int64_t K, int threads) {
+    if (M < 0 || N < 0 || K < 0 || nrows < 0) return -1;
+    if (nrows == 0 || N == 0) return 0;
+    if (!ref || (K > 0 && (!X || !W))) return -1;
+    for (int64_t i = 0; rows && i < nrows; ++i)
+        if (rows[i] < 0 || rows[i] >= M) return -1;
+    if (!rows && nrows > M) return -1;
+
+    double* Wd = (double*)malloc(sizeof(double) * (size_t)(N * K > 0 ? N * K : 1));
+    double* Xd = (double*)malloc(sizeof(double) * (size_t)(nrows * K > 0 ? nrows * K : 1));
+    if (!Wd || !Xd) { free(Wd); free(Xd); return -1; }
+#ifdef _OPENMP
+    if (threads <= 0) threads = omp_get_max_threads();
+#else
+    threads = 1;
+#endif
+
+#pragma omp parallel for schedule(static) num_threads(threads)
+    for (int64_t n = 0; n < N; ++n)
+        for (int64_t k = 0; k < K; ++k) Wd[n * K + k] = bf16_widen(W[n * K + k]);
+#pragma omp parallel for schedule(static) num_threads(threads)
+    for (int64_t i = 0; i < nrows; ++i) {
+        int64_t m = rows ? rows[i] : i;
+        for (int64_t k = 0; k < K; ++k) Xd[i * K + k] = bf16_widen(X[m * K + k]);
+    }
+
+    const int64_t nblk = (N + 3) / 4;
+#pragma omp parallel for collapse(2) schedule(static) num_threads(threads)
+    for (int64_t i = 0; i < nrows; ++i) {
+        for (int64_t nb = 0; nb < nblk; ++nb) {
+            const int64_t m = rows ? rows[i] : i;
+            const int64_t n0 = nb * 4;
+            const int cnt = (int)((N - n0) < 4 ? (N - n0) : 4);
+            const double* x = Xd + i * K;
+            const double* w[4];
+            for (int j = 0; j < 4; ++j) w[j] = Wd + (n0 + (j < cnt ? j : 0)) * K;
+            /* four independent output elements; each sums k = 0,1,2,... in order */
+            double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
+            for (int64_t k = 0; k < K; ++k) {
+                const double xv = x[k];
+                s0 += xv * w[0][k];
+                s1 += xv * w[1][k];
+                s2 += xv * w[2][k];
+                s3 += xv * w[3][k];
+            }
+            double s[4] = {s0, s1, s2, s3};
+            for (int j = 0; j < cnt; ++j) {
+                double v = s[j];
+                if (bias) v += bf16_widen(bias[n0 + j]);
+                if (R) v += bf16_widen(R[m * N + n0 + j]);
+                ref[i * N + n0 + j] = v;
+            }
+            if (absref) {
+                for (int j = 0; j < cnt; ++j) {
+                    double a = 0.0;
+                    for (int64_t k = 0; k < K; ++k) a += fabs(x[k]) * fabs(w[j][k]);
+                    if (bias) a += fabs(bf16_widen(bias[n0 + j]));
+                    if (R) a += fabs(bf16_widen(R[m * N + n0 + j]));
+                    absref[i * N + n0 + j] = a;
+                }
+            }
+        }
+    }
+    free(Wd);
+    free(Xd);
+    return 0;
+}
+
+/* Reference for the whole [M,N] output. */
+int kx_oracle_outproj(const uint16_t* X, const uint16_t* W, const uint16_t* bias,
+                      const uint16_t* R, double* ref, double* absref,
+                      int64_t M, int64_t N, int64_t K, int threads) {
+    return kx_oracle_outproj_rows(X, W, bias, R, NULL, M, ref, absref, M, N, K, threads);
+}
+
+/* Reference for one output element (used for spot checks at full sizes). */
+double kx_oracle_element(const uint16_t* X, const uint16_t* W, const uint16_t* bias,
+                         const uint16_t* R, int64_t m, int64_t n, int64_t N, int64_t K) {
+    double s = 0.0;
+    for (int64_t k = 0; k < K; ++k) s += bf16_widen(X[m * K + k]) * bf16_widen(W[n * K + k]);
+    if (bias) s += bf16_widen(bias[n]);
+    if (R) s += bf16_widen(R[m * N + n]);
+    return s;
+}

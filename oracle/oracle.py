@@ -1,0 +1,118 @@
+"""ctypes wrapper around the plain-C oracle (test infrastructure, CPU only).
+
+All tensors are numpy ``uint16`` arrays holding BF16 bit patterns, row-major:
+X [M,K], W [N,K], bias [N] or None, R [M,N] or None.  Results are unrounded
+float64.  The definition implemented is the paper's residual GEMM epilogue
+(Appendix A, Algorithm 3: O <- W^T A + O with alpha = beta = 1) in row-major
+form, plus an optional bias; with bias = R = None it is the plain product of
+the paper's fixed-shape GEMM study (Section 4.1).
+"""
+from __future__ import annotations
+
+import ctypes
+from typing import Optional, Tuple
+
+import numpy as np
+
+from . import build as _build
+
+_lib = None
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(_build.build())
+        p = ctypes.c_void_p
+        i64 = ctypes.c_int64
+        lib.kx_oracle_outproj_rows.argtypes = [p, p, p, p, p, i64, p, p, i64, i64, i64, ctypes.c_int]
+        lib.kx_oracle_outproj_rows.restype = ctypes.c_int
+        lib.kx_oracle_element.argtypes = [p, p, p, p, i64, i64, i64, i64]
+        lib.kx_oracle_element.restype = ctypes.c_double
+        lib.kx_oracle_round_bf16.argtypes = [p, p, i64]
+        lib.kx_oracle_round_bf16.restype = None
+        lib.kx_oracle_widen_bf16.argtypes = [p, p, i64]
+        lib.kx_oracle_widen_bf16.restype = None
+        lib.kx_oracle_max_threads.argtypes = []
+        lib.kx_oracle_max_threads.restype = ctypes.c_int
+        _lib = lib
+    return _lib
+
+
+def _bits(a: Optional[np.ndarray], shape, name: str) -> Optional[np.ndarray]:
+    if a is None:
+        return None
+    if a.dtype != np.uint16:
+        raise TypeError(f"{name} must be uint16 BF16 bits, got {a.dtype}")
+    if tuple(a.shape) != tuple(shape):
+        raise ValueError(f"{name} has shape {a.shape}, expected {tuple(shape)}")
+    return np.ascontiguousarray(a)
+
+
+def _ptr(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def max_threads() -> int:
+    return int(_load().kx_oracle_max_threads())
+
+
+def outproj_rows(X, W, bias, R, rows, want_abs: bool = False, threads: int = 0
+                 ) -> Tuple[np.ndarray, Optional[np.ndarray]]:
+    """Reference for the given rows (None = all rows): returns (ref, absref)."""
+    lib = _load()
+    M, K = X.shape
+    N = W.shape[0]
+    X = _bits(X, (M, K), "X")
+    W = _bits(W, (N, K), "W")
+    bias = _bits(bias, (N,), "bias")
+    R = _bits(R, (M, N), "R")
+    if rows is None:
+        rows_arr = None
+        nrows = M
+    else:
+        rows_arr = np.ascontiguousarray(rows, dtype=np.int64)
+        nrows = int(rows_arr.size)
+    ref = np.empty((nrows, N), dtype=np.float64)
+    absref = np.empty((nrows, N), dtype=np.float64) if want_abs else None
+    rc = lib.kx_oracle_outproj_rows(_ptr(X), _ptr(W), _ptr(bias), _ptr(R), _ptr(rows_arr), nrows,
+                                    _ptr(ref), _ptr(absref), M, N, K, int(threads))
+    if rc != 0:
+        raise RuntimeError(f"kx_oracle_outproj_rows failed ({rc})")
+    return ref, absref
+
+
+def outproj(X, W, bias=None, R=None, want_abs: bool = False, threads: int = 0):
+    """Reference for the whole output: ref[M,N] float64 (and absref if asked)."""
+    ref, absref = outproj_rows(X, W, bias, R, None, want_abs, threads)
+    return (ref, absref) if want_abs else ref
+
+
+def element(X, W, bias, R, m: int, n: int) -> float:
+    """Reference for one output element."""
+    lib = _load()
+    M, K = X.shape
+    N = W.shape[0]
+    X = _bits(X, (M, K), "X")
+    W = _bits(W, (N, K), "W")
+    bias = _bits(bias, (N,), "bias")
+    R = _bits(R, (M, N), "R")
+    if not (0 <= m < M and 0 <= n < N):
+        raise IndexError((m, n))
+    return float(lib.kx_oracle_element(_ptr(X), _ptr(W), _ptr(bias), _ptr(R), m, n, N, K))
+
+
+def round_bf16(a: np.ndarray) -> np.ndarray:
+    """float64 -> BF16 bits with a single round-to-nearest-even."""
+    a = np.ascontiguousarray(a, dtype=np.float64)
+    out = np.empty(a.shape, dtype=np.uint16)
+    _load().kx_oracle_round_bf16(_ptr(a), _ptr(out), a.size)
+    return out
+
+
+def widen_bf16(bits: np.ndarray) -> np.ndarray:
+    """BF16 bits -> float64 (exact)."""
+    bits = np.ascontiguousarray(bits, dtype=np.uint16)
+    out = np.empty(bits.shape, dtype=np.float64)
+    _load().kx_oracle_widen_bf16(_ptr(bits), _ptr(out), bits.size)
+    return out
