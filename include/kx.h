@@ -1,0 +1,175 @@
+/*
+ * kx — BF16 attention output projection with residual addition on B200 (sm_100a).
+ *
+ *     Y[M,N] = X[M,K] . W[N,K]^T  (+ bias[N])  + R[M,N]        (kx_outproj_residual)
+ *     Y[M,N] = X[M,K] . W[N,K]^T                                (kx_gemm_bf16)
+ *
+ * Operation: the residual GEMM epilogue of the paper's Appendix A ("L1-030:
+ * attention output projection with residual", Algorithm 3: the destination is
+ * aliased onto the residual and O <- W^T A + O with alpha = beta = 1), written
+ * row-major; the optional bias is an extension of this library.  The plain
+ * product is the operation of the paper's fixed-shape GEMM study (Section 4.1).
+ *
+ * All tensors are dense row-major BF16 (leading dimension = row length):
+ *   X [M,K], W [N,K] (the nn.Linear layout, K contiguous), bias [N] or NULL,
+ *   R [M,N], Y [M,N].  Products are accumulated in FP32; bias and residual are
+ *   added in FP32 and the sum is rounded to BF16 once (round-to-nearest-even).
+ *
+ * Pointers are DEVICE pointers unless an entry point's name ends in `_host`.
+ * The caller owns every tensor before, during and after the call; the library
+ * never frees, reallocates or keeps a reference to tensor contents (it keeps
+ * only encoded TMA descriptors keyed on address and shape).  Calls enqueue
+ * work on the caller's stream and return without synchronising.
+ *
+ * Preconditions (checked; a violated one returns an error and enqueues nothing):
+ *   - X, W, R, Y non-NULL (unless the matching extent is zero) and 16-byte aligned;
+ *     bias NULL or 16-byte aligned;
+ *   - M, N, K >= 0; N % 8 == 0 and K % 8 == 0 (16-byte row pitch for TMA);
+ *   - Y may be exactly R (in place, the paper's aliasing); any other overlap of
+ *     Y with X, W, bias or R is rejected;
+ *   - the current device has compute capability 10.x.
+ *   M == 0 or N == 0 is a successful no-op.  K == 0 gives Y = R (+ bias).
+ *
+ * There is no CPU fallback and no vendor-library GEMM behind these calls.
+ */
+#ifndef KX_H_
+#define KX_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define KX_VERSION 100
+
+typedef enum kx_status {
+    KX_OK = 0,
+    KX_ERR_NULL = 1,            /* a required pointer is NULL                         */
+    KX_ERR_SHAPE = 2,           /* negative extent, N or K not a multiple of 8, ...   */
+    KX_ERR_ALIGN = 3,           /* a pointer is not 16-byte aligned                   */
+    KX_ERR_OVERLAP = 4,         /* Y overlaps an input other than Y == R              */
+    KX_ERR_ARCH = 5,            /* current device is not sm_100                       */
+    KX_ERR_CUDA = 6,            /* a CUDA runtime/driver call failed                  */
+    KX_ERR_WORKSPACE = 7,       /* split-K workspace too small / allocation failed    */
+    KX_ERR_DEVICE_TIMEOUT = 8,  /* a bounded device-side wait gave up (see below)     */
+    KX_ERR_PLAN = 9             /* plan override names an unsupported configuration   */
+} kx_status;
+
+/* Execution paths (Section 3.3's scheduling strategy names split-K and
+ * persistent kernels; the per-M specialisation follows Algorithm 3's per-M plan). */
+enum { KX_PATH_AUTO = 0, KX_PATH_TILE = 1, KX_PATH_SWAP = 2 };
+
+/*
+ * Plan override for tests, profiling and tuning.  Zero-initialise for "auto".
+ *   path          KX_PATH_AUTO / KX_PATH_TILE (128-row output tiles, persistent,
+ *                 TMA-store epilogue) / KX_PATH_SWAP (small M: W rows on the MMA
+ *                 M axis, split-K, W streamed once)
+ *   block_n       tile path: 64, 128 or 256 output columns per tile;
+ *                 swap path: 16, 32, 64 or 128 (>= M)
+ *   cta_pair      0 auto, 1 = one CTA per tile, 2 = CTA pair per 256-row tile
+ *   split_k       swap path only: number of K splits (1..64)
+ *   raster_group  tile path: number of 128-row tile rows that share a raster group
+ *   max_ctas      cap on the persistent grid (0 = number of SMs)
+ *   spin_limit_us bound on every device-side wait (0 = 2 000 000 us)
+ *   debug_drop_kblocks  test hook: the TMA producer issues this many fewer
+ *                 k-blocks than the MMA consumer expects, so the consumer's
+ *                 bounded wait expires and the call reports
+ *                 KX_ERR_DEVICE_TIMEOUT through kx_last_device_status.  The
+ *                 kernel still exits cleanly.  Never set in production.
+ */
+typedef struct kx_plan_override {
+    int32_t path;
+    int32_t block_n;
+    int32_t cta_pair;
+    int32_t split_k;
+    int32_t raster_group;
+    int32_t max_ctas;
+    int32_t spin_limit_us;
+    int32_t debug_drop_kblocks;
+    int32_t reserved[8];
+} kx_plan_override;
+
+/* What the planner chose for a shape (kx_plan_query). */
+typedef struct kx_plan_info {
+    int32_t path;          /* KX_PATH_TILE or KX_PATH_SWAP                         */
+    int32_t block_n;
+    int32_t cta_pair;      /* 1 or 2                                               */
+    int32_t stages;        /* depth of the TMA -> MMA shared-memory ring           */
+    int32_t split_k;
+    int32_t raster_group;
+    int32_t grid;          /* CTAs launched                                        */
+    int32_t tiles;         /* work units (tiles x splits)                          */
+    int32_t launches;      /* kernels enqueued per call                            */
+    int32_t smem_bytes;    /* dynamic shared memory per CTA                        */
+    int64_t workspace_bytes; /* FP32 split-K scratch this plan uses (0 if none)    */
+    int32_t reserved[4];
+} kx_plan_info;
+
+/*
+ * Optional.  Creates the per-device state for `device` (SM count, kernel
+ * attributes, the split-K workspace and its counters) so that later calls do
+ * no allocation.  Idempotent, thread-safe.  Without it, the first kx_* call on
+ * a device does the same lazily (so make that first call outside stream capture).
+ */
+int kx_init(int device);
+
+/* Frees library-owned memory on every initialised device.  Never touches caller tensors. */
+int kx_shutdown(void);
+
+/*
+ * Y = X W^T (+ bias) + R.   Appendix A, Algorithm 3 (alpha = beta = 1, C = D).
+ *   X [M,K], W [N,K], bias_or_null [N], R [M,N] (may equal Y), Y [M,N]: device, BF16.
+ *   stream: a cudaStream_t passed as void* (NULL = the legacy default stream).
+ * Returns a kx_status.  Asynchronous: errors raised by the kernel itself are
+ * visible through kx_last_device_status after the stream has drained.
+ */
+int kx_outproj_residual(const void* X, const void* W, const void* bias_or_null, const void* R,
+                        void* Y, int64_t M, int64_t N, int64_t K, void* stream);
+
+/* Y = X W^T.   Section 4.1's BF16 matrix product (FLOPs counted as 2 M N K). */
+int kx_gemm_bf16(const void* X, const void* W, void* Y, int64_t M, int64_t N, int64_t K, void* stream);
+
+/*
+ * Same as kx_outproj_residual (R and bias may both be NULL: plain GEMM) with an
+ * explicit plan.  `ov` may be NULL (= auto).  Unsupported combinations return
+ * KX_ERR_PLAN.
+ */
+int kx_outproj_residual_ex(const void* X, const void* W, const void* bias_or_null, const void* R,
+                           void* Y, int64_t M, int64_t N, int64_t K, void* stream,
+                           const kx_plan_override* ov);
+
+/*
+ * Host-buffer convenience form of kx_outproj_residual: every tensor pointer is a
+ * HOST pointer (pinned memory gives the best copy rate; pageable works).  The
+ * call copies X, W, bias, R to library-owned device staging buffers (grown on
+ * demand, kept until kx_shutdown), runs the kernel, copies Y back into Y_host
+ * and synchronises `stream` before returning.  R_host and bias_host may be NULL.
+ * Not for use under stream capture (it may allocate and it synchronises).
+ */
+int kx_outproj_residual_host(const void* X_host, const void* W_host, const void* bias_host_or_null,
+                             const void* R_host_or_null, void* Y_host,
+                             int64_t M, int64_t N, int64_t K, void* stream);
+
+/* Fills `out` with the plan the library would use for this shape on the current
+ * device (has_residual / has_bias as 0 or 1).  No work is enqueued. */
+int kx_plan_query(int64_t M, int64_t N, int64_t K, int has_bias, int has_residual,
+                  const kx_plan_override* ov_or_null, kx_plan_info* out);
+
+/*
+ * Synchronises `stream`, then reads and clears the current device's kernel
+ * status word.  *code_out is KX_OK or KX_ERR_DEVICE_TIMEOUT; *detail_out (may be
+ * NULL) identifies which wait gave up.  Debug/test use: it blocks the host.
+ */
+int kx_last_device_status(void* stream, int* code_out, int* detail_out);
+
+/* Static string for a kx_status value. */
+const char* kx_status_string(int status);
+
+/* KX_VERSION the library was built from. */
+int kx_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KX_H_ */

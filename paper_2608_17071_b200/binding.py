@@ -1,0 +1,213 @@
+"""Thin ctypes binding over libkx.so — argument marshalling only.
+
+Every function has the name of the C entry point it calls (see ``include/kx.h``);
+all arithmetic runs in the CUDA kernels behind the C ABI.  Tensors may be
+``torch`` CUDA tensors of dtype bfloat16 (contiguous) or raw integer device
+addresses.  If the shared library is missing this module raises: there is no
+fallback path.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libkx.so")
+
+KX_OK = 0
+KX_ERR_NULL, KX_ERR_SHAPE, KX_ERR_ALIGN, KX_ERR_OVERLAP = 1, 2, 3, 4
+KX_ERR_ARCH, KX_ERR_CUDA, KX_ERR_WORKSPACE, KX_ERR_DEVICE_TIMEOUT, KX_ERR_PLAN = 5, 6, 7, 8, 9
+KX_PATH_AUTO, KX_PATH_TILE, KX_PATH_SWAP = 0, 1, 2
+
+EXPORTS = (
+    "kx_init", "kx_shutdown", "kx_outproj_residual", "kx_gemm_bf16", "kx_outproj_residual_ex",
+    "kx_outproj_residual_host", "kx_plan_query", "kx_last_device_status", "kx_status_string",
+    "kx_version",
+)
+
+
+class PlanOverride(ctypes.Structure):
+    _fields_ = [
+        ("path", ctypes.c_int32), ("block_n", ctypes.c_int32), ("cta_pair", ctypes.c_int32),
+        ("split_k", ctypes.c_int32), ("raster_group", ctypes.c_int32), ("max_ctas", ctypes.c_int32),
+        ("spin_limit_us", ctypes.c_int32), ("debug_drop_kblocks", ctypes.c_int32),
+        ("reserved", ctypes.c_int32 * 8),
+    ]
+
+
+class PlanInfo(ctypes.Structure):
+    _fields_ = [
+        ("path", ctypes.c_int32), ("block_n", ctypes.c_int32), ("cta_pair", ctypes.c_int32),
+        ("stages", ctypes.c_int32), ("split_k", ctypes.c_int32), ("raster_group", ctypes.c_int32),
+        ("grid", ctypes.c_int32), ("tiles", ctypes.c_int32), ("launches", ctypes.c_int32),
+        ("smem_bytes", ctypes.c_int32), ("workspace_bytes", ctypes.c_int64),
+        ("reserved", ctypes.c_int32 * 4),
+    ]
+
+
+class KxError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {kx_status_string(status)}")
+
+
+_lib = None
+
+
+def load():
+    """Load libkx.so.  Raises if it has not been built: no fallback exists."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2608_17071_b200.build` "
+            "(the CUDA library is the only implementation; there is no fallback)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i64, ci = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int
+    lib.kx_init.argtypes = [ci]
+    lib.kx_shutdown.argtypes = []
+    lib.kx_outproj_residual.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, vp]
+    lib.kx_gemm_bf16.argtypes = [vp, vp, vp, i64, i64, i64, vp]
+    lib.kx_outproj_residual_ex.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, vp, ctypes.POINTER(PlanOverride)]
+    lib.kx_outproj_residual_host.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, vp]
+    lib.kx_plan_query.argtypes = [i64, i64, i64, ci, ci, ctypes.POINTER(PlanOverride), ctypes.POINTER(PlanInfo)]
+    lib.kx_last_device_status.argtypes = [vp, ctypes.POINTER(ci), ctypes.POINTER(ci)]
+    lib.kx_status_string.argtypes = [ci]
+    lib.kx_status_string.restype = ctypes.c_char_p
+    lib.kx_version.argtypes = []
+    for name in EXPORTS:
+        if name != "kx_status_string":
+            getattr(lib, name).restype = ci
+    _lib = lib
+    return lib
+
+
+def _addr(t) -> Optional[int]:
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    return int(t.data_ptr())
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+        return int(torch.cuda.current_stream().cuda_stream) or None
+    if isinstance(stream, int):
+        return stream or None
+    return int(stream.cuda_stream) or None
+
+
+def _check_bf16(name, t, shape):
+    import torch
+    if t is None or isinstance(t, int):
+        return
+    if t.dtype != torch.bfloat16 or not t.is_contiguous() or tuple(t.shape) != tuple(shape):
+        raise ValueError(f"{name}: need a contiguous bfloat16 tensor of shape {tuple(shape)}, "
+                         f"got {t.dtype} {tuple(t.shape)} contiguous={t.is_contiguous()}")
+
+
+def make_override(**kw) -> PlanOverride:
+    ov = PlanOverride()
+    for k, v in kw.items():
+        if not hasattr(ov, k):
+            raise TypeError(f"unknown plan override field {k!r}")
+        setattr(ov, k, int(v))
+    return ov
+
+
+def kx_version() -> int:
+    return int(load().kx_version())
+
+
+def kx_status_string(status: int) -> str:
+    return load().kx_status_string(int(status)).decode()
+
+
+def kx_init(device: int = 0) -> None:
+    rc = load().kx_init(int(device))
+    if rc != KX_OK:
+        raise KxError(rc, "kx_init")
+
+
+def kx_shutdown() -> None:
+    load().kx_shutdown()
+
+
+def kx_outproj_residual(X, W, bias, R, Y, stream=None, M=None, N=None, K=None, check=True) -> int:
+    """Y = X W^T (+ bias) + R on the current stream.  Shapes come from the tensors
+    unless M, N, K are given (raw-pointer use)."""
+    if M is None:
+        M, K = X.shape
+        N = W.shape[0]
+        _check_bf16("X", X, (M, K)); _check_bf16("W", W, (N, K)); _check_bf16("bias", bias, (N,))
+        _check_bf16("R", R, (M, N)); _check_bf16("Y", Y, (M, N))
+    rc = load().kx_outproj_residual(_addr(X), _addr(W), _addr(bias), _addr(R), _addr(Y), M, N, K, _stream(stream))
+    if check and rc != KX_OK:
+        raise KxError(rc, "kx_outproj_residual")
+    return rc
+
+
+def kx_gemm_bf16(X, W, Y, stream=None, M=None, N=None, K=None, check=True) -> int:
+    """Y = X W^T on the current stream."""
+    if M is None:
+        M, K = X.shape
+        N = W.shape[0]
+        _check_bf16("X", X, (M, K)); _check_bf16("W", W, (N, K)); _check_bf16("Y", Y, (M, N))
+    rc = load().kx_gemm_bf16(_addr(X), _addr(W), _addr(Y), M, N, K, _stream(stream))
+    if check and rc != KX_OK:
+        raise KxError(rc, "kx_gemm_bf16")
+    return rc
+
+
+def kx_outproj_residual_ex(X, W, bias, R, Y, ov: Optional[PlanOverride] = None, stream=None,
+                           M=None, N=None, K=None, check=True) -> int:
+    """As kx_outproj_residual (bias and R optional) with an explicit plan override."""
+    if M is None:
+        M, K = X.shape
+        N = W.shape[0]
+        _check_bf16("X", X, (M, K)); _check_bf16("W", W, (N, K)); _check_bf16("bias", bias, (N,))
+        _check_bf16("R", R, (M, N)); _check_bf16("Y", Y, (M, N))
+    rc = load().kx_outproj_residual_ex(_addr(X), _addr(W), _addr(bias), _addr(R), _addr(Y), M, N, K,
+                                       _stream(stream), ctypes.byref(ov) if ov is not None else None)
+    if check and rc != KX_OK:
+        raise KxError(rc, "kx_outproj_residual_ex")
+    return rc
+
+
+def kx_outproj_residual_host(X, W, bias, R, Y, M: int, N: int, K: int, stream=None, check=True) -> int:
+    """Host-buffer form: X, W, bias, R, Y are HOST addresses (ints) or CPU tensors /
+    numpy arrays holding BF16 bits; copies in, runs, copies Y back, synchronises."""
+    def host_addr(a):
+        if a is None or isinstance(a, int):
+            return a
+        if hasattr(a, "data_ptr"):
+            return int(a.data_ptr())
+        return int(a.ctypes.data)
+    rc = load().kx_outproj_residual_host(host_addr(X), host_addr(W), host_addr(bias), host_addr(R),
+                                         host_addr(Y), M, N, K, _stream(stream))
+    if check and rc != KX_OK:
+        raise KxError(rc, "kx_outproj_residual_host")
+    return rc
+
+
+def kx_plan_query(M: int, N: int, K: int, has_bias: bool = True, has_residual: bool = True,
+                  ov: Optional[PlanOverride] = None) -> PlanInfo:
+    info = PlanInfo()
+    rc = load().kx_plan_query(M, N, K, int(has_bias), int(has_residual),
+                              ctypes.byref(ov) if ov is not None else None, ctypes.byref(info))
+    if rc != KX_OK:
+        raise KxError(rc, "kx_plan_query")
+    return info
+
+
+def kx_last_device_status(stream=None):
+    """(code, detail) after synchronising the stream; clears the status word."""
+    code, detail = ctypes.c_int(0), ctypes.c_int(0)
+    rc = load().kx_last_device_status(_stream(stream), ctypes.byref(code), ctypes.byref(detail))
+    if rc != KX_OK:
+        raise KxError(rc, "kx_last_device_status")
+    return code.value, detail.value

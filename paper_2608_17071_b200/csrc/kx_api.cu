@@ -1,0 +1,626 @@
+// C-ABI of the kx library: argument validation, plan selection, TMA descriptor
+// cache, kernel launches.  See include/kx.h for the contract of every entry point.
+#include "../../include/kx.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <mutex>
+
+#include "kx_kernels.cuh"
+
+namespace {
+
+using namespace kx;
+
+constexpr int kMaxDevices = 16;
+constexpr size_t kWorkspaceBytes = size_t(64) << 20;   // FP32 split-K partials
+constexpr int kMaxCounters = 1 << 16;
+
+// Kernel status words: [0] = kx_status code, [1] = which wait gave up.
+__device__ unsigned int g_kx_status[4];
+
+struct DeviceCtx {
+    bool ready = false;
+    int sm_count = 0;
+    float* ws = nullptr;
+    unsigned int* counters = nullptr;
+    unsigned int* status = nullptr;
+    // staging for the *_host entry point
+    void* stage = nullptr;
+    size_t stage_bytes = 0;
+};
+DeviceCtx g_ctx[kMaxDevices];
+std::mutex g_mu;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+
+bool log_enabled() {
+    static const bool on = [] {
+        const char* e = std::getenv("KX_LOG");
+        return e && e[0] && e[0] != '0';
+    }();
+    return on;
+}
+
+// ------------------------------------------------------------------ kernel table
+struct TileVariant {
+    int bn, ctas, stages, nb, smem;
+    const void* fn;
+};
+struct SwapVariant {
+    int bn, stages, smem;
+    const void* fn;
+};
+
+#define KX_TILE(BN, CTAS, ST, NB)                                                             \
+    TileVariant {                                                                             \
+        BN, CTAS, ST, NB, TileCfg<BN, CTAS, ST, NB>::SMEM_BYTES,                              \
+            reinterpret_cast<const void*>(&kx_tile_kernel<BN, CTAS, ST, NB>)                  \
+    }
+#define KX_SWAP(BN, ST)                                                                       \
+    SwapVariant { BN, ST, SwapCfg<BN, ST>::SMEM_BYTES, reinterpret_cast<const void*>(&kx_swap_kernel<BN, ST>) }
+
+const TileVariant kTileVariants[] = {
+    KX_TILE(256, 1, 4, 2), KX_TILE(128, 1, 6, 2), KX_TILE(64, 1, 8, 2), KX_TILE(256, 2, 5, 4),
+    KX_TILE(128, 2, 7, 2),
+};
+const SwapVariant kSwapVariants[] = {
+    KX_SWAP(16, 12), KX_SWAP(32, 11), KX_SWAP(64, 9), KX_SWAP(128, 7), KX_SWAP(256, 4),
+};
+
+const TileVariant* find_tile(int bn, int ctas) {
+    for (const auto& v : kTileVariants)
+        if (v.bn == bn && v.ctas == ctas) return &v;
+    return nullptr;
+}
+const SwapVariant* find_swap(int bn) {
+    for (const auto& v : kSwapVariants)
+        if (v.bn == bn) return &v;
+    return nullptr;
+}
+
+// ------------------------------------------------------------------ device state
+int ensure_device(int dev, DeviceCtx** out) {
+    if (dev < 0 || dev >= kMaxDevices) return KX_ERR_CUDA;
+    DeviceCtx& c = g_ctx[dev];
+    if (c.ready) {
+        *out = &c;
+        return KX_OK;
+    }
+    std::lock_guard<std::mutex> lk(g_mu);
+    if (c.ready) {
+        *out = &c;
+        return KX_OK;
+    }
+    int prev = 0;
+    if (cudaGetDevice(&prev) != cudaSuccess) return KX_ERR_CUDA;
+    if (prev != dev && cudaSetDevice(dev) != cudaSuccess) return KX_ERR_CUDA;
+    int rc = KX_OK;
+    do {
+        int major = 0, sms = 0;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+            rc = KX_ERR_CUDA;
+            break;
+        }
+        if (major != 10) {
+            rc = KX_ERR_ARCH;
+            break;
+        }
+        c.sm_count = sms;
+        if (!g_encode) {
+            void* fn = nullptr;
+            cudaDriverEntryPointQueryResult qres;
+            if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) !=
+                    cudaSuccess ||
+                qres != cudaDriverEntryPointSuccess || !fn) {
+                rc = KX_ERR_CUDA;
+                break;
+            }
+            g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+        }
+        bool ok = true;
+        for (const auto& v : kTileVariants)
+            ok = ok && cudaFuncSetAttribute(v.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, v.smem) ==
+                           cudaSuccess;
+        for (const auto& v : kSwapVariants)
+            ok = ok && cudaFuncSetAttribute(v.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, v.smem) ==
+                           cudaSuccess;
+        if (!ok) {
+            rc = KX_ERR_CUDA;
+            break;
+        }
+        if (cudaMalloc(&c.ws, kWorkspaceBytes) != cudaSuccess ||
+            cudaMalloc(&c.counters, kMaxCounters * sizeof(unsigned int)) != cudaSuccess) {
+            rc = KX_ERR_WORKSPACE;
+            break;
+        }
+        if (cudaMemset(c.counters, 0, kMaxCounters * sizeof(unsigned int)) != cudaSuccess ||
+            cudaGetSymbolAddress(reinterpret_cast<void**>(&c.status), g_kx_status) != cudaSuccess ||
+            cudaMemset(c.status, 0, sizeof(unsigned int) * 4) != cudaSuccess ||
+            cudaDeviceSynchronize() != cudaSuccess) {
+            rc = KX_ERR_CUDA;
+            break;
+        }
+        c.ready = true;
+    } while (false);
+    if (rc != KX_OK) {
+        cudaGetLastError();
+        if (c.ws) cudaFree(c.ws);
+        if (c.counters) cudaFree(c.counters);
+        c.ws = nullptr;
+        c.counters = nullptr;
+    }
+    if (prev != dev) cudaSetDevice(prev);
+    *out = &c;
+    return rc;
+}
+
+// ------------------------------------------------------------------ TMA descriptors
+// Cache of encoded descriptors keyed on (address, extents, box).  It holds no tensor
+// contents, so rewriting a tensor in place between calls is always seen.
+struct TmapKey {
+    const void* ptr;
+    uint64_t rows, cols;
+    uint32_t box_rows;
+    bool operator==(const TmapKey& o) const {
+        return ptr == o.ptr && rows == o.rows && cols == o.cols && box_rows == o.box_rows;
+    }
+};
+struct TmapEntry {
+    TmapKey key;
+    bool valid;
+    alignas(64) CUtensorMap map;
+};
+constexpr int kTmapSlots = 64;
+thread_local TmapEntry t_tmaps[kTmapSlots];
+
+// Row-major BF16 matrix [rows, cols]; box = box_rows x 64 columns; 128-byte swizzle;
+// 256-byte L2 promotion; out-of-bounds elements read as zero and are not written.
+int get_tmap(const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows, CUtensorMap* out) {
+    TmapKey key{ptr, rows, cols, box_rows};
+    uint64_t h = reinterpret_cast<uint64_t>(ptr) >> 4;
+    h ^= rows * 0x9E3779B97F4A7C15ull;
+    h ^= (cols + 0x7F4A7C15ull) * 0xC2B2AE3D27D4EB4Full;
+    h ^= box_rows * 0x165667B19E3779F9ull;
+    h ^= h >> 29;
+    TmapEntry& e = t_tmaps[h % kTmapSlots];
+    if (e.valid && e.key == key) {
+        *out = e.map;
+        return KX_OK;
+    }
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols * 2};
+    cuuint32_t box[2] = {64, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = g_encode(&e.map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides,
+                          box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        e.valid = false;
+        if (log_enabled()) std::fprintf(stderr, "[kx] cuTensorMapEncodeTiled failed: %d\n", static_cast<int>(r));
+        return KX_ERR_CUDA;
+    }
+    e.key = key;
+    e.valid = true;
+    *out = e.map;
+    return KX_OK;
+}
+
+// ------------------------------------------------------------------ planning
+struct Plan {
+    int path = 0;
+    int bn = 0, ctas = 1, stages = 0, nb = 0;
+    int splits = 1;
+    int raster_group = 8;
+    int grid = 0, units = 0;
+    int tiles_m = 0, tiles_n = 0;   // tile path: tile grid; swap path: m_tiles / n_tiles
+    int smem = 0;
+    size_t ws_bytes = 0;
+    const void* fn = nullptr;
+    int launches = 1;
+};
+
+int ceil_div(long long a, long long b) { return static_cast<int>((a + b - 1) / b); }
+
+int pick_splits(int n_units, int nkb, int sms, long long M, long long N) {
+    int best = 1;
+    double best_eff = -1.0;
+    const int max_s = std::min(nkb, 64);
+    for (int s = 1; s <= max_s; ++s) {
+        if (s > 1 && nkb / s < 4) break;
+        if (static_cast<size_t>(s) * M * N * 4 > kWorkspaceBytes) break;
+        const long long units = static_cast<long long>(n_units) * s;
+        const long long waves = (units + sms - 1) / sms;
+        const double eff = static_cast<double>(units) / static_cast<double>(waves * sms);
+        if (eff > best_eff + 0.03) {
+            best = s;
+            best_eff = eff;
+        }
+    }
+    return best;
+}
+
+int make_plan(long long M, long long N, long long K, const kx_plan_override* ov, int sms, Plan* pl) {
+    const int nkb = ceil_div(K, 64);
+    int path = ov ? ov->path : KX_PATH_AUTO;
+    if (path == KX_PATH_AUTO) path = (M <= 128) ? KX_PATH_SWAP : KX_PATH_TILE;
+    if (path != KX_PATH_TILE && path != KX_PATH_SWAP) return KX_ERR_PLAN;
+    const int max_ctas = (ov && ov->max_ctas > 0) ? std::min(ov->max_ctas, sms) : sms;
+    pl->path = path;
+    if (path == KX_PATH_TILE) {
+        int ctas = (ov && ov->cta_pair) ? ov->cta_pair : 1;
+        if (ctas != 1 && ctas != 2) return KX_ERR_PLAN;
+        int bn = ov ? ov->block_n : 0;
+        if (bn == 0) {
+            // widest tile that still gives every SM work
+            bn = 64;
+            for (int cand : {256, 128}) {
+                const long long tiles = static_cast<long long>(ceil_div(M, 128)) * ceil_div(N, cand);
+                if (tiles >= (max_ctas * 4) / 5) {
+                    bn = cand;
+                    break;
+                }
+            }
+        }
+        const TileVariant* v = find_tile(bn, ctas);
+        if (!v) return KX_ERR_PLAN;
+        if (ov && ov->split_k > 1) return KX_ERR_PLAN;
+        pl->bn = bn;
+        pl->ctas = ctas;
+        pl->stages = v->stages;
+        pl->nb = v->nb;
+        pl->smem = v->smem;
+        pl->fn = v->fn;
+        pl->tiles_m = ceil_div(M, 128 * ctas);
+        pl->tiles_n = ceil_div(N, bn);
+        pl->units = pl->tiles_m * pl->tiles_n;
+        pl->raster_group = (ov && ov->raster_group > 0) ? ov->raster_group : 8;
+        const int slots = std::max(1, max_ctas / ctas);
+        pl->grid = std::min(pl->units, slots) * ctas;
+        pl->splits = 1;
+        pl->ws_bytes = 0;
+    } else {
+        int bn = ov ? ov->block_n : 0;
+        if (bn == 0) bn = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : M <= 128 ? 128 : 256;
+        const SwapVariant* v = find_swap(bn);
+        if (!v) return KX_ERR_PLAN;
+        if (ov && ov->cta_pair > 1) return KX_ERR_PLAN;
+        pl->bn = bn;
+        pl->ctas = 1;
+        pl->stages = v->stages;
+        pl->smem = v->smem;
+        pl->fn = v->fn;
+        pl->tiles_n = ceil_div(N, 128);
+        pl->tiles_m = ceil_div(M, bn);
+        const long long tiles = static_cast<long long>(pl->tiles_n) * pl->tiles_m;
+        if (tiles > kMaxCounters) return KX_ERR_WORKSPACE;
+        int splits = (ov && ov->split_k > 0) ? ov->split_k : pick_splits(static_cast<int>(tiles), nkb, max_ctas, M, N);
+        splits = std::max(1, std::min(splits, std::max(1, nkb)));
+        if (splits > 64) return KX_ERR_PLAN;
+        pl->splits = splits;
+        pl->ws_bytes = splits > 1 ? static_cast<size_t>(splits) * M * N * 4 : 0;
+        if (pl->ws_bytes > kWorkspaceBytes) return KX_ERR_WORKSPACE;
+        pl->units = static_cast<int>(tiles * splits);
+        pl->grid = std::min(pl->units, max_ctas);
+    }
+    return KX_OK;
+}
+
+// ------------------------------------------------------------------ validation
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+bool overlaps(const void* a, size_t abytes, const void* b, size_t bbytes) {
+    if (!a || !b || abytes == 0 || bbytes == 0) return false;
+    const uintptr_t a0 = reinterpret_cast<uintptr_t>(a), b0 = reinterpret_cast<uintptr_t>(b);
+    return a0 < b0 + bbytes && b0 < a0 + abytes;
+}
+
+int validate(const void* X, const void* W, const void* bias, const void* R, const void* Y, long long M,
+             long long N, long long K, bool need_r) {
+    if (M < 0 || N < 0 || K < 0) return KX_ERR_SHAPE;
+    if (M > 0x7FFFFFFFll / 2 || N > 0x7FFFFFFFll / 2 || K > 0x7FFFFFFFll / 2) return KX_ERR_SHAPE;
+    if (M == 0 || N == 0) return KX_OK;
+    if ((N % 8) != 0 || (K % 8) != 0) return KX_ERR_SHAPE;
+    if (!Y) return KX_ERR_NULL;
+    if (K > 0 && (!X || !W)) return KX_ERR_NULL;
+    if (need_r && !R) return KX_ERR_NULL;
+    if (!aligned16(Y) || (K > 0 && (!aligned16(X) || !aligned16(W))) || (R && !aligned16(R)) ||
+        (bias && !aligned16(bias)))
+        return KX_ERR_ALIGN;
+    const size_t yb = static_cast<size_t>(M) * N * 2;
+    if (overlaps(Y, yb, X, static_cast<size_t>(M) * K * 2) || overlaps(Y, yb, W, static_cast<size_t>(N) * K * 2) ||
+        overlaps(Y, yb, bias, static_cast<size_t>(N) * 2))
+        return KX_ERR_OVERLAP;
+    if (R && R != Y && overlaps(Y, yb, R, yb)) return KX_ERR_OVERLAP;
+    return KX_OK;
+}
+
+// ------------------------------------------------------------------ launch
+int run(const void* X, const void* W, const void* bias, const void* R, void* Y, long long M, long long N,
+        long long K, void* stream_v, const kx_plan_override* ov, bool need_r) {
+    int rc = validate(X, W, bias, R, Y, M, N, K, need_r);
+    if (rc != KX_OK) return rc;
+    if (M == 0 || N == 0) return KX_OK;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return KX_ERR_CUDA;
+    DeviceCtx* ctx = nullptr;
+    rc = ensure_device(dev, &ctx);
+    if (rc != KX_OK) return rc;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+
+    if (K == 0) {
+        const long long total = M * N;
+        const int blocks = static_cast<int>(std::min<long long>((total + 255) / 256, ctx->sm_count * 8));
+        kx_k0_kernel<<<blocks, 256, 0, stream>>>(static_cast<const uint16_t*>(bias),
+                                                 static_cast<const uint16_t*>(R), static_cast<uint16_t*>(Y), M, N);
+        return cudaGetLastError() == cudaSuccess ? KX_OK : KX_ERR_CUDA;
+    }
+
+    Plan pl;
+    rc = make_plan(M, N, K, ov, ctx->sm_count, &pl);
+    if (rc != KX_OK) return rc;
+    const unsigned long long spin_ns =
+        (ov && ov->spin_limit_us > 0) ? static_cast<unsigned long long>(ov->spin_limit_us) * 1000ull
+                                      : 2000000000ull;
+    const int drop = ov ? std::max(0, ov->debug_drop_kblocks) : 0;
+    if (log_enabled())
+        std::fprintf(stderr, "[kx] M=%lld N=%lld K=%lld path=%d bn=%d ctas=%d stages=%d splits=%d grid=%d units=%d\n",
+                     M, N, K, pl.path, pl.bn, pl.ctas, pl.stages, pl.splits, pl.grid, pl.units);
+
+    cudaLaunchConfig_t cfg;
+    std::memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3(pl.grid, 1, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = pl.smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    if (pl.ctas == 2) {
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+    }
+
+    if (pl.path == KX_PATH_TILE) {
+        CUtensorMap tmA, tmB, tmY, tmR;
+        if ((rc = get_tmap(X, M, K, 128, &tmA)) != KX_OK) return rc;
+        if ((rc = get_tmap(W, N, K, pl.bn / pl.ctas, &tmB)) != KX_OK) return rc;
+        if ((rc = get_tmap(Y, M, N, 32, &tmY)) != KX_OK) return rc;
+        if (R) {
+            if ((rc = get_tmap(R, M, N, 32, &tmR)) != KX_OK) return rc;
+        } else {
+            tmR = tmY;
+        }
+        TileParams p;
+        p.M = static_cast<int>(M);
+        p.N = static_cast<int>(N);
+        p.K = static_cast<int>(K);
+        p.tiles_m = pl.tiles_m;
+        p.tiles_n = pl.tiles_n;
+        p.num_tiles = pl.units;
+        p.raster_group = pl.raster_group;
+        p.has_bias = bias ? 1 : 0;
+        p.has_r = R ? 1 : 0;
+        p.drop_kblocks = drop;
+        p.spin_limit_ns = spin_ns;
+        p.status = ctx->status;
+        const uint16_t* bias_p = static_cast<const uint16_t*>(bias);
+        void* args[] = {&tmA, &tmB, &tmY, &tmR, &bias_p, &p};
+        if (cudaLaunchKernelExC(&cfg, pl.fn, args) != cudaSuccess) {
+            cudaGetLastError();
+            return KX_ERR_CUDA;
+        }
+    } else {
+        CUtensorMap tmW, tmX;
+        if ((rc = get_tmap(W, N, K, 128, &tmW)) != KX_OK) return rc;
+        if ((rc = get_tmap(X, M, K, pl.bn, &tmX)) != KX_OK) return rc;
+        SwapParams p;
+        p.M = static_cast<int>(M);
+        p.N = static_cast<int>(N);
+        p.K = static_cast<int>(K);
+        p.n_tiles = pl.tiles_n;
+        p.m_tiles = pl.tiles_m;
+        p.splits = pl.splits;
+        p.num_units = pl.units;
+        p.has_bias = bias ? 1 : 0;
+        p.has_r = R ? 1 : 0;
+        p.drop_kblocks = drop;
+        p.spin_limit_ns = spin_ns;
+        p.status = ctx->status;
+        p.ws = ctx->ws;
+        p.counters = ctx->counters;
+        p.bias = static_cast<const uint16_t*>(bias);
+        p.R = static_cast<const uint16_t*>(R);
+        p.Y = static_cast<uint16_t*>(Y);
+        void* args[] = {&tmW, &tmX, &p};
+        if (cudaLaunchKernelExC(&cfg, pl.fn, args) != cudaSuccess) {
+            cudaGetLastError();
+            return KX_ERR_CUDA;
+        }
+    }
+    return KX_OK;
+}
+
+}  // namespace
+
+// ====================================================================== C ABI
+extern "C" {
+#pragma GCC visibility push(default)
+
+int kx_version(void) { return KX_VERSION; }
+
+const char* kx_status_string(int s) {
+    switch (s) {
+        case KX_OK: return "KX_OK";
+        case KX_ERR_NULL: return "KX_ERR_NULL: a required pointer is NULL";
+        case KX_ERR_SHAPE: return "KX_ERR_SHAPE: bad extent (negative, too large, or N/K not a multiple of 8)";
+        case KX_ERR_ALIGN: return "KX_ERR_ALIGN: a pointer is not 16-byte aligned";
+        case KX_ERR_OVERLAP: return "KX_ERR_OVERLAP: Y overlaps an input (only Y == R is allowed)";
+        case KX_ERR_ARCH: return "KX_ERR_ARCH: device is not compute capability 10.x";
+        case KX_ERR_CUDA: return "KX_ERR_CUDA: a CUDA call failed";
+        case KX_ERR_WORKSPACE: return "KX_ERR_WORKSPACE: split-K workspace too small or not allocated";
+        case KX_ERR_DEVICE_TIMEOUT: return "KX_ERR_DEVICE_TIMEOUT: a bounded device-side wait gave up";
+        case KX_ERR_PLAN: return "KX_ERR_PLAN: unsupported plan override";
+        default: return "KX_ERR_UNKNOWN";
+    }
+}
+
+int kx_init(int device) {
+    DeviceCtx* ctx = nullptr;
+    return ensure_device(device, &ctx);
+}
+
+int kx_shutdown(void) {
+    std::lock_guard<std::mutex> lk(g_mu);
+    int prev = 0;
+    cudaGetDevice(&prev);
+    for (int d = 0; d < kMaxDevices; ++d) {
+        DeviceCtx& c = g_ctx[d];
+        if (!c.ready && !c.stage) continue;
+        cudaSetDevice(d);
+        cudaDeviceSynchronize();
+        if (c.ws) cudaFree(c.ws);
+        if (c.counters) cudaFree(c.counters);
+        if (c.stage) cudaFree(c.stage);
+        c = DeviceCtx();
+    }
+    cudaSetDevice(prev);
+    return KX_OK;
+}
+
+int kx_outproj_residual(const void* X, const void* W, const void* bias, const void* R, void* Y, int64_t M,
+                        int64_t N, int64_t K, void* stream) {
+    return run(X, W, bias, R, Y, M, N, K, stream, nullptr, true);
+}
+
+int kx_gemm_bf16(const void* X, const void* W, void* Y, int64_t M, int64_t N, int64_t K, void* stream) {
+    return run(X, W, nullptr, nullptr, Y, M, N, K, stream, nullptr, false);
+}
+
+int kx_outproj_residual_ex(const void* X, const void* W, const void* bias, const void* R, void* Y, int64_t M,
+                           int64_t N, int64_t K, void* stream, const kx_plan_override* ov) {
+    return run(X, W, bias, R, Y, M, N, K, stream, ov, false);
+}
+
+int kx_plan_query(int64_t M, int64_t N, int64_t K, int has_bias, int has_residual,
+                  const kx_plan_override* ov, kx_plan_info* out) {
+    (void)has_bias;
+    (void)has_residual;
+    if (!out) return KX_ERR_NULL;
+    if (M <= 0 || N <= 0 || K <= 0 || (N % 8) || (K % 8)) return KX_ERR_SHAPE;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return KX_ERR_CUDA;
+    DeviceCtx* ctx = nullptr;
+    int rc = ensure_device(dev, &ctx);
+    if (rc != KX_OK) return rc;
+    Plan pl;
+    rc = make_plan(M, N, K, ov, ctx->sm_count, &pl);
+    if (rc != KX_OK) return rc;
+    std::memset(out, 0, sizeof *out);
+    out->path = pl.path;
+    out->block_n = pl.bn;
+    out->cta_pair = pl.ctas;
+    out->stages = pl.stages;
+    out->split_k = pl.splits;
+    out->raster_group = pl.raster_group;
+    out->grid = pl.grid;
+    out->tiles = pl.units;
+    out->launches = pl.launches;
+    out->smem_bytes = pl.smem;
+    out->workspace_bytes = static_cast<int64_t>(pl.ws_bytes);
+    return KX_OK;
+}
+
+int kx_last_device_status(void* stream, int* code_out, int* detail_out) {
+    if (!code_out) return KX_ERR_NULL;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return KX_ERR_CUDA;
+    DeviceCtx* ctx = nullptr;
+    int rc = ensure_device(dev, &ctx);
+    if (rc != KX_OK) return rc;
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return KX_ERR_CUDA;
+    unsigned int h[4] = {0, 0, 0, 0};
+    if (cudaMemcpy(h, ctx->status, sizeof h, cudaMemcpyDeviceToHost) != cudaSuccess) return KX_ERR_CUDA;
+    *code_out = static_cast<int>(h[0]);
+    if (detail_out) *detail_out = static_cast<int>(h[1]);
+    if (h[0] != 0) {
+        // a kernel that gave up may have left split-K tile counters part-way
+        if (cudaMemset(ctx->status, 0, sizeof h) != cudaSuccess ||
+            cudaMemset(ctx->counters, 0, kMaxCounters * sizeof(unsigned int)) != cudaSuccess)
+            return KX_ERR_CUDA;
+    }
+    return KX_OK;
+}
+
+int kx_outproj_residual_host(const void* Xh, const void* Wh, const void* bh, const void* Rh, void* Yh,
+                             int64_t M, int64_t N, int64_t K, void* stream_v) {
+    if (M < 0 || N < 0 || K < 0) return KX_ERR_SHAPE;
+    if (M == 0 || N == 0) return KX_OK;
+    if (!Yh || (K > 0 && (!Xh || !Wh))) return KX_ERR_NULL;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return KX_ERR_CUDA;
+    DeviceCtx* ctx = nullptr;
+    int rc = ensure_device(dev, &ctx);
+    if (rc != KX_OK) return rc;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    auto up = [](size_t b) { return (b + 255) & ~size_t(255); };
+    const size_t xb = up(static_cast<size_t>(M) * K * 2), wb = up(static_cast<size_t>(N) * K * 2);
+    const size_t bb = up(static_cast<size_t>(N) * 2), yb = up(static_cast<size_t>(M) * N * 2);
+    const size_t need = xb + wb + bb + yb;   // R is staged in Y's buffer (in-place form)
+    {
+        std::lock_guard<std::mutex> lk(g_mu);
+        if (ctx->stage_bytes < need) {
+            if (ctx->stage) {
+                cudaDeviceSynchronize();
+                cudaFree(ctx->stage);
+                ctx->stage = nullptr;
+                ctx->stage_bytes = 0;
+            }
+            if (cudaMalloc(&ctx->stage, need) != cudaSuccess) {
+                cudaGetLastError();
+                return KX_ERR_WORKSPACE;
+            }
+            ctx->stage_bytes = need;
+        }
+    }
+    char* base = static_cast<char*>(ctx->stage);
+    void* Xd = base;
+    void* Wd = base + xb;
+    void* bd = base + xb + wb;
+    void* Yd = base + xb + wb + bb;
+    bool ok = true;
+    if (K > 0) {
+        ok = ok && cudaMemcpyAsync(Xd, Xh, static_cast<size_t>(M) * K * 2, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+        ok = ok && cudaMemcpyAsync(Wd, Wh, static_cast<size_t>(N) * K * 2, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    }
+    if (bh) ok = ok && cudaMemcpyAsync(bd, bh, static_cast<size_t>(N) * 2, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    // the residual is copied straight into the output buffer: the kernel then runs in place (Y == R)
+    if (Rh) ok = ok && cudaMemcpyAsync(Yd, Rh, static_cast<size_t>(M) * N * 2, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    if (!ok) {
+        cudaGetLastError();
+        return KX_ERR_CUDA;
+    }
+    rc = run(Xd, Wd, bh ? bd : nullptr, Rh ? Yd : nullptr, Yd, M, N, K, stream, nullptr, false);
+    if (rc != KX_OK) return rc;
+    if (cudaMemcpyAsync(Yh, Yd, static_cast<size_t>(M) * N * 2, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+        cudaStreamSynchronize(stream) != cudaSuccess) {
+        cudaGetLastError();
+        return KX_ERR_CUDA;
+    }
+    return KX_OK;
+}
+
+#pragma GCC visibility pop
+}  // extern "C"

@@ -1,0 +1,649 @@
+// sm_100a kernels for Y = X W^T (+ bias) + R  (BF16 in/out, FP32 accumulate).
+//
+// Two kernels share one mainloop design (TMA -> swizzled shared-memory ring ->
+// tcgen05.mma into TMEM, warp-specialised, mbarrier hand-offs, double-buffered
+// accumulators so the epilogue of unit i overlaps the mainloop of unit i+1):
+//
+//   kx_tile_kernel  large M.  Output tile = 128 rows of X (x2 for a CTA pair)
+//                   by BN rows of W.  Persistent over a rastered tile list.
+//                   Epilogue per warp: R slab by TMA into swizzled staging,
+//                   tcgen05.ld, + bias + R in FP32, one BF16 rounding, written
+//                   back in place, TMA store to Y.
+//   kx_swap_kernel  small / medium M.  W rows sit on the MMA M axis (128 per
+//                   unit), X rows on the MMA N axis (BN per unit), K may be
+//                   split across CTAs.  W is streamed exactly once through a
+//                   deep ring.  Partials go to an FP32 workspace; the last CTA
+//                   to finish a tile sums the splits in fixed order and applies
+//                   bias + R once.
+//
+// The operation is the paper's residual GEMM epilogue (Appendix A, Algorithm 3:
+// O <- W^T A + O, alpha = beta = 1, output aliased onto the residual) and the
+// plain GEMM of Section 4.1.  The warp roles follow the curriculum of Table 2
+// (tensor-core pipeline, producer/consumer specialisation, persistent CTAs with
+// raw mbarriers, chunked TMA epilogue, tile scheduling) re-expressed for
+// Blackwell: tcgen05 + TMEM replace WGMMA, and a CTA pair (cta_group::2)
+// replaces the cluster multicast tier.
+//
+// Every wait on an mbarrier is bounded: after `spin_limit_ns` the waiting thread
+// records where it gave up, raises a CTA-wide abort flag and every role falls
+// through to the common teardown (TMEM is always freed).
+#pragma once
+#include "kx_ptx.cuh"
+
+namespace kx {
+
+constexpr int kThreads = 192;         // warps 0-3 epilogue, 4 TMA producer, 5 MMA issuer
+constexpr int kBlockK = 64;           // BF16 elements per k-block = one 128-byte swizzle row
+constexpr int kABytes = 128 * 128;    // 128 operand rows x 128 bytes
+
+constexpr uint32_t kWhereEmpty = 1, kWhereFull = 2, kWhereAccEmpty = 3, kWhereAccFull = 4,
+                   kWhereRFull = 5, kWhereDrain = 6;
+
+struct Waiter {
+    volatile uint32_t* abort_flag;   // this CTA's shared abort word
+    uint32_t peer_abort;             // shared::cluster address of the peer's abort word (0 = none)
+    unsigned long long limit_ns;
+
+    __device__ __forceinline__ void raise(uint32_t where) const {
+        atomicCAS(const_cast<uint32_t*>(abort_flag), 0u, where);
+        if (peer_abort) st_cluster_u32(peer_abort, where);
+    }
+    __device__ __forceinline__ bool aborted() const { return *abort_flag != 0; }
+    // true = barrier phase completed; false = gave up (abort raised)
+    __device__ __forceinline__ bool wait(uint32_t bar, uint32_t parity, uint32_t where) const {
+        if (mbar_try_wait(bar, parity)) return true;
+        const unsigned long long t0 = globaltimer_ns();
+        uint32_t it = 0;
+        for (;;) {
+            if (mbar_try_wait(bar, parity)) return true;
+            if ((++it & 15u) == 0u) {
+                if (*abort_flag != 0) return false;
+                if (globaltimer_ns() - t0 > limit_ns) {
+                    raise(where);
+                    return false;
+                }
+            }
+        }
+    }
+};
+
+__host__ __device__ constexpr int tmem_cols_for(int n) {
+    return n <= 32 ? 32 : n <= 64 ? 64 : n <= 128 ? 128 : n <= 256 ? 256 : 512;
+}
+
+// Rastered tile order: tile rows are taken in groups of `group`; inside a group the
+// row index runs fastest, so the tiles resident at one time cover a compact block of
+// tile rows and tile columns and share their X and W panels in L2.
+__device__ __forceinline__ void tile_coords(int t, int tiles_m, int tiles_n, int group, int& tm, int& tn) {
+    const int per_group = group * tiles_n;
+    const int g = t / per_group;
+    const int r = t - g * per_group;
+    const int m0 = g * group;
+    const int gsize = min(group, tiles_m - m0);
+    tn = r / gsize;
+    tm = m0 + (r - tn * gsize);
+}
+
+// ===========================================================================
+// kx_tile_kernel
+// ===========================================================================
+struct TileParams {
+    int M, N, K;
+    int tiles_m, tiles_n, num_tiles;
+    int raster_group;
+    int has_bias, has_r;
+    int drop_kblocks;
+    unsigned long long spin_limit_ns;
+    unsigned int* status;
+};
+
+template <int BN, int CTAS, int STAGES, int NB>
+struct TileCfg {
+    static constexpr int BN_LOAD = BN / CTAS;               // W rows this CTA loads per k-block
+    static constexpr int B_BYTES = BN_LOAD * 128;
+    static constexpr int STAGE_BYTES = kABytes + B_BYTES;
+    static constexpr int SLAB_BYTES = 32 * 128;             // 32 rows x 64 BF16 per warp per chunk
+    static constexpr int EPI_BYTES = 4 * NB * SLAB_BYTES;
+    static constexpr int NUM_BARS = 2 * STAGES + 4 + 4 * NB + 1;
+    static constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + EPI_BYTES + 1024;
+    static constexpr int TMEM_COLS = tmem_cols_for(2 * BN);
+    static constexpr int CHUNKS = BN / 64;                  // 64-column epilogue chunks per tile
+    static_assert(BN % 64 == 0 && BN <= 256, "BN");
+    static_assert(NUM_BARS * 8 + 16 <= 1024, "barrier area");
+    static_assert(STAGE_BYTES % 1024 == 0, "stage alignment");
+};
+
+template <int BN, int CTAS, int STAGES, int NB>
+__global__ void __launch_bounds__(kThreads, 1)
+kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const __grid_constant__ CUtensorMap tmY, const __grid_constant__ CUtensorMap tmR,
+               const uint16_t* __restrict__ bias, const TileParams p) {
+    using C = TileCfg<BN, CTAS, STAGES, NB>;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t* const gbase = smem_raw + (base - raw);
+    const uint32_t s_stage = base;
+    const uint32_t s_epi = base + STAGES * C::STAGE_BYTES;
+    const uint32_t s_bar = s_epi + C::EPI_BYTES;
+    auto full = [&](int s) { return s_bar + 8u * s; };
+    auto empty = [&](int s) { return s_bar + 8u * (STAGES + s); };
+    auto acc_full = [&](int b) { return s_bar + 8u * (2 * STAGES + b); };
+    auto acc_empty = [&](int b) { return s_bar + 8u * (2 * STAGES + 2 + b); };
+    auto r_full = [&](int w, int j) { return s_bar + 8u * (2 * STAGES + 4 + w * NB + j); };
+    const uint32_t drain_bar = s_bar + 8u * (2 * STAGES + 4 + 4 * NB);
+    volatile uint32_t* const s_tmem =
+        reinterpret_cast<volatile uint32_t*>(gbase + (s_bar - base) + 8 * C::NUM_BARS);
+    volatile uint32_t* const s_abort = s_tmem + 1;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const uint32_t cta_rank = (CTAS == 2) ? cluster_ctarank() : 0u;
+    const bool leader = (cta_rank == 0);
+    const int nkb = (p.K + kBlockK - 1) / kBlockK;
+    const int unit0 = blockIdx.x / CTAS;
+    const int ustride = gridDim.x / CTAS;
+
+    if (threadIdx.x == 0) *s_abort = 0;
+    if (warp == 4 && lane == 0) {
+        prefetch_tmap(&tmA);
+        prefetch_tmap(&tmB);
+        prefetch_tmap(&tmY);
+        if (p.has_r) prefetch_tmap(&tmR);
+    }
+    if (warp == 5) {
+        if (lane == 0) {
+            for (int s = 0; s < STAGES; ++s) {
+                mbar_init(full(s), 1);
+                mbar_init(empty(s), 1);
+            }
+            for (int b = 0; b < 2; ++b) {
+                mbar_init(acc_full(b), 1);
+                mbar_init(acc_empty(b), 4 * CTAS);
+            }
+            for (int w = 0; w < 4; ++w)
+                for (int j = 0; j < NB; ++j) mbar_init(r_full(w, j), 1);
+            mbar_init(drain_bar, 1);
+            fence_mbar_init();
+        }
+        __syncwarp();
+        tmem_alloc<CTAS>(smem_u32(const_cast<uint32_t*>(s_tmem)), C::TMEM_COLS);
+        tmem_relinquish<CTAS>();
+    }
+    tc_fence_before();
+    __syncthreads();
+    if constexpr (CTAS == 2) {
+        cluster_arrive();
+        cluster_wait();
+    }
+    tc_fence_after();
+    const uint32_t tmem_base = *s_tmem;
+
+    Waiter wt;
+    wt.abort_flag = s_abort;
+    wt.peer_abort = (CTAS == 2) ? map_to_cta(smem_u32(const_cast<uint32_t*>(s_abort)), cta_rank ^ 1u) : 0u;
+    wt.limit_ns = p.spin_limit_ns;
+
+    if (warp == 4) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t s = 0, ph = 0;
+            bool ok = true;
+            const int nkb_issue = nkb - p.drop_kblocks;
+            for (int t = unit0; t < p.num_tiles && ok; t += ustride) {
+                int tm, tn;
+                tile_coords(t, p.tiles_m, p.tiles_n, p.raster_group, tm, tn);
+                const int a_row = tm * (128 * CTAS) + static_cast<int>(cta_rank) * 128;
+                const int b_row = tn * BN + static_cast<int>(cta_rank) * C::BN_LOAD;
+                for (int kb = 0; kb < nkb_issue; ++kb) {
+                    if (!wt.wait(empty(s), ph ^ 1u, kWhereEmpty)) { ok = false; break; }
+                    const uint32_t sa = s_stage + s * C::STAGE_BYTES;
+                    const uint32_t sb = sa + kABytes;
+                    if constexpr (CTAS == 1) {
+                        mbar_arrive_expect_tx(full(s), C::STAGE_BYTES);
+                        tma_load_2d(sa, &tmA, kb * kBlockK, a_row, full(s));
+                        tma_load_2d(sb, &tmB, kb * kBlockK, b_row, full(s));
+                    } else {
+                        // both CTAs' copies complete on the leader's barrier
+                        if (leader) mbar_arrive_expect_tx(full(s), 2 * C::STAGE_BYTES);
+                        const uint32_t fb = map_to_cta(full(s), 0);
+                        tma_load_2d_pair(sa, &tmA, kb * kBlockK, a_row, fb);
+                        tma_load_2d_pair(sb, &tmB, kb * kBlockK, b_row, fb);
+                    }
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+                }
+            }
+        }
+    } else if (warp == 5) {
+        // ------------------------------------------------------------ MMA issuer
+        if (leader && lane == 0) {
+            constexpr uint32_t idesc = idesc_bf16_f32(128 * CTAS, BN);
+            uint32_t s = 0, ph = 0, tcount = 0;
+            bool ok = true;
+            for (int t = unit0; t < p.num_tiles && ok; t += ustride, ++tcount) {
+                const uint32_t b = tcount & 1u, aph = (tcount >> 1) & 1u;
+                if (!wt.wait(acc_empty(b), aph ^ 1u, kWhereAccEmpty)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d = tmem_base + b * BN;
+                for (int kb = 0; kb < nkb; ++kb) {
+                    if (!wt.wait(full(s), ph, kWhereFull)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t sa = s_stage + s * C::STAGE_BYTES;
+                    const uint32_t sb = sa + kABytes;
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        mma_bf16<CTAS>(d, smem_desc_sw128(sa + k * 32), smem_desc_sw128(sb + k * 32), idesc,
+                                       static_cast<uint32_t>(kb | k));
+                    if constexpr (CTAS == 1) {
+                        mma_commit<1>(empty(s));
+                    } else {
+                        mma_commit<2>(map_to_cta(empty(s), 0));
+                        mma_commit<2>(map_to_cta(empty(s), 1));
+                    }
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+                }
+                if (!ok) break;
+                if constexpr (CTAS == 1) {
+                    mma_commit<1>(acc_full(b));
+                } else {
+                    mma_commit<2>(map_to_cta(acc_full(b), 0));
+                    mma_commit<2>(map_to_cta(acc_full(b), 1));
+                }
+            }
+            if (!ok) {  // let every MMA issued so far retire before TMEM is freed
+                mma_commit<CTAS>(CTAS == 1 ? drain_bar : map_to_cta(drain_bar, 0));
+                uint32_t spins = 0;
+                while (!mbar_try_wait(drain_bar, 0) && ++spins < (1u << 20)) {}
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue warps
+        const int q = warp;                                // TMEM lanes 32q .. 32q+31
+        const uint32_t my_epi = s_epi + q * NB * C::SLAB_BYTES;
+        const int my_tiles = (unit0 < p.num_tiles) ? (p.num_tiles - unit0 + ustride - 1) / ustride : 0;
+        const uint32_t total_chunks = static_cast<uint32_t>(my_tiles) * C::CHUNKS;
+        const bool has_r = p.has_r != 0, has_bias = p.has_bias != 0;
+
+        // position of this warp's slab for chunk number x of this CTA's chunk sequence
+        auto chunk_pos = [&](uint32_t x, int& row0, int& col0) {
+            const int seq = static_cast<int>(x / C::CHUNKS);
+            const int c = static_cast<int>(x % C::CHUNKS);
+            int tm, tn;
+            tile_coords(unit0 + seq * ustride, p.tiles_m, p.tiles_n, p.raster_group, tm, tn);
+            row0 = tm * (128 * CTAS) + static_cast<int>(cta_rank) * 128 + q * 32;
+            col0 = tn * BN + c * 64;
+        };
+        auto issue_r = [&](uint32_t x) {                   // lane 0 only
+            int row0, col0;
+            chunk_pos(x, row0, col0);
+            if (row0 < p.M && col0 < p.N) {
+                const int j = static_cast<int>(x % NB);
+                mbar_arrive_expect_tx(r_full(q, j), C::SLAB_BYTES);
+                tma_load_2d(my_epi + j * C::SLAB_BYTES, &tmR, col0, row0, r_full(q, j));
+            }
+        };
+        if (has_r && lane == 0)
+            for (uint32_t x = 0; x + 1 < static_cast<uint32_t>(NB) && x < total_chunks; ++x) issue_r(x);
+
+        uint32_t cc = 0, tcount = 0, rphase = 0;
+        bool ok = true;
+        for (int t = unit0; t < p.num_tiles && ok; t += ustride, ++tcount) {
+            const uint32_t b = tcount & 1u, aph = (tcount >> 1) & 1u;
+            int tm, tn;
+            tile_coords(t, p.tiles_m, p.tiles_n, p.raster_group, tm, tn);
+            const int row0 = tm * (128 * CTAS) + static_cast<int>(cta_rank) * 128 + q * 32;
+            if (!__all_sync(0xffffffffu, wt.wait(acc_full(b), aph, kWhereAccFull))) { ok = false; break; }
+            tc_fence_after();
+#pragma unroll 1
+            for (int c = 0; c < C::CHUNKS; ++c, ++cc) {
+                const int j = static_cast<int>(cc % NB);
+                const int col0 = tn * BN + c * 64;
+                const bool valid = (row0 < p.M) && (col0 < p.N);
+                const uint32_t buf = my_epi + j * C::SLAB_BYTES;
+                uint32_t acc[2][32];
+                if (valid) {
+                    const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + b * BN + c * 64;
+                    tmem_ld_32x32(taddr, acc[0]);
+                    tmem_ld_32x32(taddr + 32, acc[1]);
+                    tmem_ld_wait();
+                }
+                if (c == C::CHUNKS - 1) {                  // accumulator buffer b is drained
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) {
+                        if constexpr (CTAS == 1) mbar_arrive(acc_empty(b));
+                        else mbar_arrive_cluster(map_to_cta(acc_empty(b), 0));
+                    }
+                }
+                if (valid) {
+                    if (has_r) {
+                        if (!__all_sync(0xffffffffu, wt.wait(r_full(q, j), (rphase >> j) & 1u, kWhereRFull))) {
+                            ok = false;
+                            break;
+                        }
+                        rphase ^= (1u << j);
+                    }
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+#pragma unroll
+                        for (int g = 0; g < 4; ++g) {
+                            const int c16 = h * 4 + g;     // 16-byte group inside the 128-byte row
+                            const uint32_t addr = buf + lane * 128 + ((c16 ^ (lane & 7)) << 4);
+                            float v[8];
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(acc[h][g * 8 + i]);
+                            if (has_bias) {
+                                const int n = col0 + c16 * 8;
+                                if (n + 8 <= p.N) {
+                                    const uint4 bb = __ldg(reinterpret_cast<const uint4*>(bias + n));
+                                    v[0] += bf16_lo(bb.x); v[1] += bf16_hi(bb.x);
+                                    v[2] += bf16_lo(bb.y); v[3] += bf16_hi(bb.y);
+                                    v[4] += bf16_lo(bb.z); v[5] += bf16_hi(bb.z);
+                                    v[6] += bf16_lo(bb.w); v[7] += bf16_hi(bb.w);
+                                }
+                            }
+                            if (has_r) {
+                                uint4 rr;
+                                asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+                                             : "=r"(rr.x), "=r"(rr.y), "=r"(rr.z), "=r"(rr.w)
+                                             : "r"(addr));
+                                v[0] += bf16_lo(rr.x); v[1] += bf16_hi(rr.x);
+                                v[2] += bf16_lo(rr.y); v[3] += bf16_hi(rr.y);
+                                v[4] += bf16_lo(rr.z); v[5] += bf16_hi(rr.z);
+                                v[6] += bf16_lo(rr.w); v[7] += bf16_hi(rr.w);
+                            }
+                            const uint32_t o0 = pack_bf16x2(v[0], v[1]), o1 = pack_bf16x2(v[2], v[3]);
+                            const uint32_t o2 = pack_bf16x2(v[4], v[5]), o3 = pack_bf16x2(v[6], v[7]);
+                            asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(o0),
+                                         "r"(o1), "r"(o2), "r"(o3)
+                                         : "memory");
+                        }
+                    }
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        tma_store_2d(&tmY, col0, row0, buf);
+                        tma_store_commit();
+                        tma_store_wait_read<1>();          // the store before this one has left its buffer
+                    }
+                }
+                // refill the buffer released by the previous chunk with the R slab NB-1 chunks ahead
+                if (has_r && lane == 0 && cc + NB - 1 < total_chunks) {
+                    if (!valid) tma_store_wait_read<0>();  // no store was issued above: drain the last one
+                    issue_r(cc + NB - 1);
+                }
+                __syncwarp();
+            }
+        }
+        if (lane == 0) tma_store_wait_all<0>();
+    }
+
+    // ---------------------------------------------------------------- teardown
+    __syncwarp();
+    tc_fence_before();
+    __syncthreads();
+    if constexpr (CTAS == 2) {
+        cluster_arrive();
+        cluster_wait();
+    }
+    if (warp == 5) tmem_dealloc<CTAS>(tmem_base, C::TMEM_COLS);
+    if (threadIdx.x == 0 && *s_abort != 0) {
+        if (atomicCAS(p.status, 0u, 8u) == 0u) p.status[1] = *s_abort;
+    }
+}
+
+// ===========================================================================
+// kx_swap_kernel
+// ===========================================================================
+struct SwapParams {
+    int M, N, K;
+    int n_tiles, m_tiles, splits, num_units;
+    int has_bias, has_r;
+    int drop_kblocks;
+    unsigned long long spin_limit_ns;
+    unsigned int* status;
+    float* ws;                 // [splits][M][N] FP32 partials (splits > 1)
+    unsigned int* counters;    // [n_tiles * m_tiles], zero between launches
+    const uint16_t* bias;
+    const uint16_t* R;
+    uint16_t* Y;
+};
+
+template <int BN, int STAGES>
+struct SwapCfg {
+    static constexpr int B_BYTES = BN * 128;
+    static constexpr int STAGE_BYTES = kABytes + B_BYTES;
+    static constexpr int NUM_BARS = 2 * STAGES + 4 + 2;
+    static constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + 1024;
+    static constexpr int TMEM_COLS = tmem_cols_for(2 * BN);
+    static_assert(BN % 16 == 0 && BN >= 16 && BN <= 256, "BN");
+    static_assert(NUM_BARS * 8 + 16 <= 1024, "barrier area");
+    static_assert(STAGE_BYTES % 1024 == 0, "stage alignment");
+};
+
+template <int BN, int STAGES>
+__global__ void __launch_bounds__(kThreads, 1)
+kx_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
+               const SwapParams p) {
+    using C = SwapCfg<BN, STAGES>;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t* const gbase = smem_raw + (base - raw);
+    const uint32_t s_stage = base;
+    const uint32_t s_bar = base + STAGES * C::STAGE_BYTES;
+    auto full = [&](int s) { return s_bar + 8u * s; };
+    auto empty = [&](int s) { return s_bar + 8u * (STAGES + s); };
+    auto acc_full = [&](int b) { return s_bar + 8u * (2 * STAGES + b); };
+    auto acc_empty = [&](int b) { return s_bar + 8u * (2 * STAGES + 2 + b); };
+    const uint32_t drain_bar = s_bar + 8u * (2 * STAGES + 4);
+    const uint32_t epi_bar = s_bar + 8u * (2 * STAGES + 5);   // the four epilogue warps meet here
+    volatile uint32_t* const s_tmem =
+        reinterpret_cast<volatile uint32_t*>(gbase + (s_bar - base) + 8 * C::NUM_BARS);
+    volatile uint32_t* const s_abort = s_tmem + 1;
+    volatile uint32_t* const s_last = s_tmem + 2;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int nkb = (p.K + kBlockK - 1) / kBlockK;
+
+    if (threadIdx.x == 0) *s_abort = 0;
+    if (warp == 4 && lane == 0) {
+        prefetch_tmap(&tmW);
+        prefetch_tmap(&tmX);
+    }
+    if (warp == 5) {
+        if (lane == 0) {
+            for (int s = 0; s < STAGES; ++s) {
+                mbar_init(full(s), 1);
+                mbar_init(empty(s), 1);
+            }
+            for (int b = 0; b < 2; ++b) {
+                mbar_init(acc_full(b), 1);
+                mbar_init(acc_empty(b), 4);
+            }
+            mbar_init(drain_bar, 1);
+            mbar_init(epi_bar, 4);
+            fence_mbar_init();
+        }
+        __syncwarp();
+        tmem_alloc<1>(smem_u32(const_cast<uint32_t*>(s_tmem)), C::TMEM_COLS);
+        tmem_relinquish<1>();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *s_tmem;
+
+    Waiter wt;
+    wt.abort_flag = s_abort;
+    wt.peer_abort = 0;
+    wt.limit_ns = p.spin_limit_ns;
+
+    // unit u -> (n_tile, m_tile, split); the splits of one tile are adjacent units
+    auto unit_coords = [&](int u, int& nt, int& mt, int& sp, int& kb0, int& kb1) {
+        sp = u % p.splits;
+        const int tile = u / p.splits;
+        mt = tile % p.m_tiles;
+        nt = tile / p.m_tiles;
+        kb0 = static_cast<int>((static_cast<long long>(sp) * nkb) / p.splits);
+        kb1 = static_cast<int>((static_cast<long long>(sp + 1) * nkb) / p.splits);
+    };
+
+    if (warp == 4) {
+        if (lane == 0) {
+            uint32_t s = 0, ph = 0;
+            bool ok = true;
+            for (int u = blockIdx.x; u < p.num_units && ok; u += gridDim.x) {
+                int nt, mt, sp, kb0, kb1;
+                unit_coords(u, nt, mt, sp, kb0, kb1);
+                kb1 -= p.drop_kblocks;
+                for (int kb = kb0; kb < kb1; ++kb) {
+                    if (!wt.wait(empty(s), ph ^ 1u, kWhereEmpty)) { ok = false; break; }
+                    const uint32_t sa = s_stage + s * C::STAGE_BYTES;
+                    mbar_arrive_expect_tx(full(s), C::STAGE_BYTES);
+                    tma_load_2d(sa, &tmW, kb * kBlockK, nt * 128, full(s));
+                    tma_load_2d(sa + kABytes, &tmX, kb * kBlockK, mt * BN, full(s));
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+                }
+            }
+        }
+    } else if (warp == 5) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = idesc_bf16_f32(128, BN);
+            uint32_t s = 0, ph = 0, ucount = 0;
+            bool ok = true;
+            for (int u = blockIdx.x; u < p.num_units && ok; u += gridDim.x, ++ucount) {
+                int nt, mt, sp, kb0, kb1;
+                unit_coords(u, nt, mt, sp, kb0, kb1);
+                const uint32_t b = ucount & 1u, aph = (ucount >> 1) & 1u;
+                if (!wt.wait(acc_empty(b), aph ^ 1u, kWhereAccEmpty)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d = tmem_base + b * BN;
+                for (int kb = kb0; kb < kb1; ++kb) {
+                    if (!wt.wait(full(s), ph, kWhereFull)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t sa = s_stage + s * C::STAGE_BYTES;
+                    const uint32_t sb = sa + kABytes;
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        mma_bf16<1>(d, smem_desc_sw128(sa + k * 32), smem_desc_sw128(sb + k * 32), idesc,
+                                    static_cast<uint32_t>((kb - kb0) | k));
+                    mma_commit<1>(empty(s));
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+                }
+                if (!ok) break;
+                mma_commit<1>(acc_full(b));
+            }
+            if (!ok) {
+                mma_commit<1>(drain_bar);
+                uint32_t spins = 0;
+                while (!mbar_try_wait(drain_bar, 0) && ++spins < (1u << 20)) {}
+            }
+        }
+    } else {
+        // epilogue: lane <-> one W row (output column n); TMEM columns <-> output rows m
+        const int q = warp;
+        const int etid = threadIdx.x;                      // 0..127
+        const bool has_r = p.has_r != 0, has_bias = p.has_bias != 0;
+        uint32_t ucount = 0, epi_phase = 0;
+        bool ok = true;
+        // bounded meeting point of the 128 epilogue threads (an mbarrier, so a wait can give up)
+        auto epi_sync = [&]() -> bool {
+            __syncwarp();
+            if (lane == 0) mbar_arrive(epi_bar);
+            const bool w = __all_sync(0xffffffffu, wt.wait(epi_bar, epi_phase, kWhereDrain));
+            epi_phase ^= 1u;
+            return w;
+        };
+        for (int u = blockIdx.x; u < p.num_units && ok; u += gridDim.x, ++ucount) {
+            int nt, mt, sp, kb0, kb1;
+            unit_coords(u, nt, mt, sp, kb0, kb1);
+            const uint32_t b = ucount & 1u, aph = (ucount >> 1) & 1u;
+            const int n = nt * 128 + q * 32 + lane;
+            const bool n_ok = n < p.N;
+            const int m0 = mt * BN;
+            const int m_cnt = min(BN, p.M - m0);
+            float bias_v = 0.f;
+            if (has_bias && n_ok) bias_v = __uint_as_float(static_cast<uint32_t>(__ldg(p.bias + n)) << 16);
+            if (!__all_sync(0xffffffffu, wt.wait(acc_full(b), aph, kWhereAccFull))) { ok = false; break; }
+            tc_fence_after();
+#pragma unroll 1
+            for (int c0 = 0; c0 < m_cnt; c0 += 16) {
+                uint32_t a[16];
+                tmem_ld_32x16(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + b * BN + c0, a);
+                tmem_ld_wait();
+                if (n_ok) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const int m = m0 + c0 + i;
+                        if (c0 + i < m_cnt) {
+                            const size_t off = static_cast<size_t>(m) * p.N + n;
+                            if (p.splits == 1) {
+                                float v = __uint_as_float(a[i]) + bias_v;
+                                if (has_r) v += __uint_as_float(static_cast<uint32_t>(p.R[off]) << 16);
+                                p.Y[off] = static_cast<uint16_t>(pack_bf16x2(v, 0.f) & 0xFFFFu);
+                            } else {
+                                p.ws[static_cast<size_t>(sp) * p.M * p.N + off] = __uint_as_float(a[i]);
+                            }
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acc_empty(b));
+            if (p.splits > 1) {
+                // last CTA to finish this tile sums the splits in fixed order (deterministic)
+                __threadfence();
+                if (!epi_sync()) { ok = false; break; }
+                if (etid == 0) {
+                    const int tile = nt * p.m_tiles + mt;
+                    const unsigned int old = atomicAdd(p.counters + tile, 1u);
+                    const bool last = (old == static_cast<unsigned int>(p.splits - 1));
+                    if (last) p.counters[tile] = 0u;       // self-resetting for the next launch
+                    *s_last = last ? 1u : 0u;
+                }
+                if (!epi_sync()) { ok = false; break; }
+                if (*s_last) {
+                    __threadfence();
+                    if (n_ok) {
+                        const size_t plane = static_cast<size_t>(p.M) * p.N;
+#pragma unroll 1
+                        for (int i = 0; i < m_cnt; ++i) {
+                            const size_t off = static_cast<size_t>(m0 + i) * p.N + n;
+                            float v = 0.f;
+                            for (int s2 = 0; s2 < p.splits; ++s2) v += __ldcg(p.ws + s2 * plane + off);
+                            v += bias_v;
+                            if (has_r) v += __uint_as_float(static_cast<uint32_t>(p.R[off]) << 16);
+                            p.Y[off] = static_cast<uint16_t>(pack_bf16x2(v, 0.f) & 0xFFFFu);
+                        }
+                    }
+                }
+            }
+        }
+    }
+
+    __syncwarp();
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 5) tmem_dealloc<1>(tmem_base, C::TMEM_COLS);
+    if (threadIdx.x == 0 && *s_abort != 0) {
+        if (atomicCAS(p.status, 0u, 8u) == 0u) p.status[1] = *s_abort;
+    }
+}
+
+// K == 0: the sum over k is empty, Y = R (+ bias) or zero.
+__global__ void kx_k0_kernel(const uint16_t* __restrict__ bias, const uint16_t* R, uint16_t* Y, long long M,
+                             long long N) {
+    const long long total = M * N;
+    for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < total;
+         i += static_cast<long long>(gridDim.x) * blockDim.x) {
+        float v = 0.f;
+        if (bias) v += __uint_as_float(static_cast<uint32_t>(bias[i % N]) << 16);
+        if (R) v += __uint_as_float(static_cast<uint32_t>(R[i]) << 16);
+        Y[i] = static_cast<uint16_t>(pack_bf16x2(v, 0.f) & 0xFFFFu);
+    }
+}
+
+}  // namespace kx
