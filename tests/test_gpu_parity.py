@@ -1,0 +1,322 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle, element by
+element, on sizes the oracle finishes in seconds: every kernel variant, several
+tiles plus ragged tails, exact pins and the tolerance gates."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2608_17071_b200 import binding as kx
+from paper_2608_17071_b200 import inputs
+
+import kxtest as kt
+
+pytestmark = pytest.mark.gpu
+
+T, S = kx.KX_PATH_TILE, kx.KX_PATH_SWAP
+TILE_VARIANTS = [
+    dict(path=T, block_n=256, cta_pair=1), dict(path=T, block_n=128, cta_pair=1),
+    dict(path=T, block_n=64, cta_pair=1), dict(path=T, block_n=256, cta_pair=2),
+    dict(path=T, block_n=128, cta_pair=2),
+]
+SWAP_VARIANTS = [
+    dict(path=S, block_n=16, split_k=1), dict(path=S, block_n=16, split_k=4),
+    dict(path=S, block_n=32, split_k=3), dict(path=S, block_n=64, split_k=2),
+    dict(path=S, block_n=128, split_k=5), dict(path=S, block_n=256, split_k=1),
+    dict(path=S, block_n=256, split_k=4),
+]
+
+
+def vid(v):
+    return "-".join(f"{k}{val}" for k, val in v.items())
+
+
+def run(X, W, b, R, ov=None, inplace=False, entry="ex"):
+    M, K = X.shape
+    N = W.shape[0]
+    Xd, Wd, bd = kt.to_dev(X), kt.to_dev(W), kt.to_dev(b)
+    if inplace:
+        Y = kt.to_dev(R)
+        Rd = Y
+    else:
+        Y = kt.nan_filled(M, N)
+        Rd = kt.to_dev(R)
+    o = kx.make_override(**ov) if ov else None
+    if entry == "ex":
+        kx.kx_outproj_residual_ex(Xd, Wd, bd, Rd, Y, o)
+    elif entry == "fused":
+        kx.kx_outproj_residual(Xd, Wd, bd, Rd, Y)
+    else:
+        kx.kx_gemm_bf16(Xd, Wd, Y)
+    code, detail = kx.kx_last_device_status()
+    assert code == kx.KX_OK, f"device status {code} (wait {detail})"
+    return kt.from_dev(Y)
+
+
+def ternary_case(M, N, K, seed=1, bias=True, res=True):
+    X = inputs.ternary_bf16(seed, "X", (M, K))
+    W = inputs.ternary_bf16(seed, "W", (N, K))
+    b = inputs.small_int_bf16(seed, "bias", (N,), -4, 4) if bias else None
+    R = inputs.small_int_bf16(seed, "R", (M, N), -8, 8) if res else None
+    return X, W, b, R
+
+
+# ------------------------------------------------------------------ exact pins
+@pytest.mark.parametrize("ov", TILE_VARIANTS, ids=vid)
+@pytest.mark.parametrize("M,N,K", [(128, 256, 64), (640, 1024, 512), (300, 520, 264), (1000, 776, 1096)])
+def test_tile_exact_integer_arithmetic(ov, M, N, K):
+    """X, W in {-1,0,1}, small-integer bias and residual: every partial sum is an
+    integer below 2^24, FP32 accumulation is exact in any order, so the output
+    must equal the once-rounded exact result bit for bit."""
+    X, W, b, R = ternary_case(M, N, K)
+    y = run(X, W, b, R, ov)
+    ok, msg = kt.gate_exact(y, oracle.outproj(X, W, b, R))
+    assert ok, msg
+
+
+@pytest.mark.parametrize("ov", SWAP_VARIANTS, ids=vid)
+@pytest.mark.parametrize("N,K", [(256, 512), (1000, 1096), (2048, 4096)])
+def test_swap_exact_integer_arithmetic(ov, N, K):
+    bn = ov["block_n"]
+    for M in sorted({1, bn // 2 + 1, bn, (2 * bn + 3) if bn >= 128 else bn}):
+        X, W, b, R = ternary_case(M, N, K, seed=2)
+        y = run(X, W, b, R, ov)
+        ok, msg = kt.gate_exact(y, oracle.outproj(X, W, b, R))
+        assert ok, f"M={M}: {msg}"
+
+
+@pytest.mark.parametrize("ov", [TILE_VARIANTS[0], TILE_VARIANTS[3], SWAP_VARIANTS[1], SWAP_VARIANTS[6]], ids=vid)
+def test_exact_large_k(ov):
+    """K = 14336 (the longest reduction of the workloads): any dropped or repeated
+    k-block, or a ring-phase slip after many wraps, shows as a bit mismatch."""
+    M = 16 if ov["path"] == S and ov["block_n"] == 16 else 256
+    X, W, b, R = ternary_case(M, 512, 14336, seed=3)
+    y = run(X, W, b, R, ov)
+    ok, msg = kt.gate_exact(y, oracle.outproj(X, W, b, R))
+    assert ok, msg
+
+
+@pytest.mark.parametrize("ov", [None] + TILE_VARIANTS[:1] + TILE_VARIANTS[3:4] + SWAP_VARIANTS[3:4], ids=lambda v: "auto" if v is None else vid(v))
+def test_zero_weight_returns_residual_plus_bias(ov):
+    """W = 0: Y == R bit for bit without bias; with bias Y == rne(R + bias)."""
+    M, N, K = (48 if ov and ov["path"] == S else 384), 520, 320
+    d = inputs.make_inputs(inputs.Workload("t", M, N, K, 31, True, True), stress=True)
+    W0 = np.zeros((N, K), dtype=np.uint16)
+    y = run(d["X"], W0, None, d["R"], ov)
+    assert np.array_equal(y, d["R"])
+    y = run(d["X"], W0, d["bias"], d["R"], ov)
+    f = lambda a: oracle.widen_bf16(a)
+    assert np.array_equal(y, oracle.round_bf16(f(d["R"]) + f(d["bias"])[None, :]))
+
+
+@pytest.mark.parametrize("ov", [TILE_VARIANTS[0], TILE_VARIANTS[2], TILE_VARIANTS[3], SWAP_VARIANTS[2], SWAP_VARIANTS[6]], ids=vid)
+def test_selectors(ov):
+    """W a permutation matrix picks columns of X; one-hot X picks columns of W."""
+    M = 24 if ov["path"] == S and ov["block_n"] < 128 else 260
+    N, K = 392, 448
+    W, pi = inputs.permutation_matrix_bf16(5, N, K)
+    X = inputs.normal_bf16(5, "X", (M, K), 1.0)
+    y = run(X, W, None, None, ov)
+    assert np.array_equal(y, X[:, pi])
+    X1 = inputs.one_hot_rows_bf16(M, K)
+    Wr = inputs.normal_bf16(6, "W", (N, K), 1.0)
+    y = run(X1, Wr, None, None, ov)
+    assert np.array_equal(y, Wr[:, np.arange(M) % K].T)
+
+
+@pytest.mark.parametrize("ov", [TILE_VARIANTS[1], TILE_VARIANTS[3], SWAP_VARIANTS[4]], ids=vid)
+def test_power_of_two_scaling_is_bitwise(ov):
+    M = 100 if ov["path"] == S else 512
+    d = inputs.make_inputs(inputs.Workload("t", M, 512, 1024, 41, False, False), stress=True)
+    y1 = run(d["X"], d["W"], None, None, ov)
+    X2 = inputs.f32_to_bf16_bits(2.0 * inputs.bf16_bits_to_f32(d["X"]))
+    y2 = run(X2, d["W"], None, None, ov)
+    want = inputs.f32_to_bf16_bits(2.0 * inputs.bf16_bits_to_f32(y1))
+    assert np.array_equal(y2, want)
+
+
+@pytest.mark.parametrize("ov", [None, TILE_VARIANTS[0], TILE_VARIANTS[2], TILE_VARIANTS[3], TILE_VARIANTS[4],
+                                SWAP_VARIANTS[1], SWAP_VARIANTS[5], SWAP_VARIANTS[6]],
+                         ids=lambda v: "auto" if v is None else vid(v))
+def test_in_place_matches_out_of_place(ov):
+    """Y aliased onto R (the paper's destination/residual aliasing) gives the same bits."""
+    M = 20 if ov and ov["path"] == S and ov["block_n"] < 128 else 700
+    d = inputs.make_inputs(inputs.Workload("t", M, 1032, 512, 51, True, True), stress=True)
+    y_out = run(d["X"], d["W"], d["bias"], d["R"], ov)
+    y_in = run(d["X"], d["W"], d["bias"], d["R"].copy(), ov, inplace=True)
+    assert np.array_equal(y_out, y_in)
+    ok, msg = kt.gate_a(y_in, oracle.outproj(d["X"], d["W"], d["bias"], d["R"]))
+    assert ok, msg
+
+
+def test_weight_rewritten_in_place_is_seen():
+    """Same pointers, new contents: nothing derived from tensor contents may be cached."""
+    M, N, K = 256, 512, 512
+    X, W, b, R = ternary_case(M, N, K, seed=7)
+    Xd, Wd, bd, Rd = kt.to_dev(X), kt.to_dev(W), kt.to_dev(b), kt.to_dev(R)
+    Y = kt.nan_filled(M, N)
+    for ov in (None, dict(path=S, block_n=256, split_k=2)):
+        o = kx.make_override(**ov) if ov else None
+        kx.kx_outproj_residual_ex(Xd, Wd, bd, Rd, Y, o)
+        assert kt.gate_exact(kt.from_dev(Y), oracle.outproj(X, W, b, R))[0]
+        W2 = inputs.ternary_bf16(8, "W", (N, K))
+        Wd.copy_(kt.to_dev(W2))
+        kx.kx_outproj_residual_ex(Xd, Wd, bd, Rd, Y, o)
+        ok, msg = kt.gate_exact(kt.from_dev(Y), oracle.outproj(X, W2, b, R))
+        assert ok, msg
+        Wd.copy_(kt.to_dev(W))
+
+
+def test_repeated_calls_are_deterministic():
+    d = inputs.make_inputs(inputs.Workload("t", 77, 2048, 2048, 61, True, True))
+    ys = [run(d["X"], d["W"], d["bias"], d["R"], dict(path=S, block_n=128, split_k=8)) for _ in range(3)]
+    assert np.array_equal(ys[0], ys[1]) and np.array_equal(ys[0], ys[2])
+    d = inputs.make_inputs(inputs.Workload("t", 1024, 1024, 1024, 62, True, True))
+    ys = [run(d["X"], d["W"], d["bias"], d["R"]) for _ in range(3)]
+    assert np.array_equal(ys[0], ys[1]) and np.array_equal(ys[0], ys[2])
+
+
+# ------------------------------------------------------------------ tolerance gates on random data
+CASES = [
+    # (name of recipe, M, N, K) — the workloads' recipes at sizes the oracle finishes in seconds
+    ("cfg1", 128, 1024, 1024),      # the small workload at full size
+    ("cfg2", 520, 1024, 4096),
+    ("cfg5", 384, 512, 14336),
+    ("sweep_M1_H2048", 1, 2048, 2048),
+    ("sweep_M32_H5120", 32, 5120, 5120),
+    ("sweep_M512_H2048", 512, 2048, 2048),
+    ("sweep_M8192_H4096", 1100, 1304, 4096),
+]
+
+
+@pytest.mark.parametrize("name,M,N,K", CASES)
+@pytest.mark.parametrize("stress", [False, True], ids=["literal", "stress"])
+def test_random_workloads_all_gates(name, M, N, K, stress):
+    """Gate A (the formal tolerance) and the sharp gate on the workloads' own
+    distributions, through the public entry point with the automatic plan.
+    `stress` rescales X to N(0,1) so the GEMM term itself is O(1)."""
+    wl = inputs.all_workloads()[name]
+    d = inputs.make_inputs(wl, stress=stress, M=M, N=N, K=K)
+    ref, absref = oracle.outproj(d["X"], d["W"], d["bias"], d["R"], want_abs=True)
+    y = run(d["X"], d["W"], d["bias"], d["R"], None, entry="fused")
+    ok, msg = kt.gate_a(y, ref)
+    assert ok, msg
+    ok, msg = kt.gate_c(y, ref, absref, K, rate_limit=3e-2 if stress else 5e-3)
+    assert ok, msg
+
+
+@pytest.mark.parametrize("ov", TILE_VARIANTS + SWAP_VARIANTS[4:], ids=vid)
+def test_plain_gemm_relative_error(ov):
+    """Plain GEMM on uniform data: relative Frobenius error <= 2^-8 (BF16 rounding
+    alone gives ~1.7e-3; a dropped 64-wide k-block would give several percent)."""
+    M = 128 if ov["path"] == S and ov["block_n"] == 128 else 600
+    wl = inputs.all_workloads()["cfg4"]
+    d = inputs.make_inputs(wl, M=M, N=1040, K=2048)
+    ref, absref = oracle.outproj(d["X"], d["W"], want_abs=True)
+    y = run(d["X"], d["W"], None, None, ov)
+    assert kt.rel_fro(y, ref) <= 2.0 ** -8
+    ok, msg = kt.gate_c(y, ref, absref, 2048, rate_limit=3e-2)   # no residual: GEMM term is the output
+    assert ok, msg
+    y2 = run(d["X"], d["W"], None, None, None, entry="gemm")
+    assert kt.rel_fro(y2, ref) <= 2.0 ** -8
+
+
+# ------------------------------------------------------------------ edge cases
+@pytest.mark.parametrize("M,N,K", [(1, 8, 8), (1, 8, 64), (3, 16, 8), (129, 8, 72), (257, 264, 8),
+                                   (127, 1016, 136), (255, 24, 4096)])
+@pytest.mark.parametrize("path", [0, T, S])
+def test_small_and_ragged_shapes(M, N, K, path):
+    X, W, b, R = ternary_case(M, N, K, seed=9)
+    ov = dict(path=path) if path else None
+    y = run(X, W, b, R, ov)
+    ok, msg = kt.gate_exact(y, oracle.outproj(X, W, b, R))
+    assert ok, msg
+
+
+def test_empty_sum_and_empty_output():
+    M, N = 37, 264
+    _, _, b, R = ternary_case(M, N, 8, seed=10)
+    X0 = np.zeros((M, 0), dtype=np.uint16)
+    W0 = np.zeros((N, 0), dtype=np.uint16)
+    Rd, bd = kt.to_dev(R), kt.to_dev(b)
+    Y = kt.nan_filled(M, N)
+    assert kx.kx_outproj_residual(0, 0, bd, Rd, Y, M=M, N=N, K=0) == kx.KX_OK
+    f = oracle.widen_bf16
+    assert np.array_equal(kt.from_dev(Y), oracle.round_bf16(f(R) + f(b)[None, :]))
+    assert np.array_equal(oracle.outproj(X0, W0, b, R), f(R) + f(b)[None, :])
+    Y = kt.nan_filled(M, N)
+    assert kx.kx_gemm_bf16(0, 0, Y, M=M, N=N, K=0) == kx.KX_OK
+    assert not kt.from_dev(Y).any()
+    # M == 0 / N == 0: nothing is written, nothing is launched
+    Y = kt.nan_filled(4, 8)
+    assert kx.kx_gemm_bf16(0, 0, Y, M=0, N=8, K=8) == kx.KX_OK
+    assert np.isnan(oracle.widen_bf16(kt.from_dev(Y))).all()
+
+
+def test_special_values_propagate_only_where_they_should():
+    M, N, K = 130, 264, 192
+    X, W, b, R = ternary_case(M, N, K, seed=11)
+    X = X.copy(); R = R.copy()
+    X[5, 70] = 0x7F80          # +inf in one row of X
+    X[100, 3] = 0x7FC0         # NaN in another
+    R[17, 200] = 0xFF80        # -inf in one residual element
+    for ov in (None, dict(path=S, block_n=256, split_k=2)):
+        y = oracle.widen_bf16(run(X, W, b, R, ov))
+        ref = oracle.outproj(X, W, b, R)
+        assert np.array_equal(np.isnan(y), np.isnan(ref))
+        fin = np.isfinite(ref)
+        assert np.array_equal(y[~np.isnan(ref) & ~fin], ref[~np.isnan(ref) & ~fin])
+        assert np.array_equal(oracle.round_bf16(ref[fin]), oracle.round_bf16(y[fin]))
+        assert np.isnan(y[100]).all() and y[17, 200] == -np.inf
+
+
+def test_guard_regions_are_untouched():
+    """Canaries before and after Y: the TMA stores and the split-K epilogue must
+    not write outside [Y, Y + M*N)."""
+    import torch
+    M, N, K = 300, 520, 264
+    X, W, b, R = ternary_case(M, N, K, seed=12)
+    pad = 4096
+    for ov in (None, dict(path=T, block_n=256, cta_pair=2), dict(path=S, block_n=256, split_k=3)):
+        buf = torch.full((pad + M * N + pad,), -7.0, dtype=torch.bfloat16, device="cuda")
+        Y = buf[pad:pad + M * N].view(M, N)
+        o = kx.make_override(**ov) if ov else None
+        kx.kx_outproj_residual_ex(kt.to_dev(X), kt.to_dev(W), kt.to_dev(b), kt.to_dev(R), Y, o)
+        torch.cuda.synchronize()
+        assert (buf[:pad] == -7.0).all() and (buf[pad + M * N:] == -7.0).all()
+        assert kt.gate_exact(kt.from_dev(Y.contiguous()), oracle.outproj(X, W, b, R))[0]
+
+
+def test_host_buffer_entry_point():
+    import torch
+    M, N, K = 200, 520, 1032
+    d = inputs.make_inputs(inputs.Workload("t", M, N, K, 71, True, True), stress=True)
+    pin = lambda a: torch.from_numpy(a.view(np.int16)).pin_memory()
+    Xh, Wh, bh, Rh = pin(d["X"]), pin(d["W"]), pin(d["bias"]), pin(d["R"])
+    Yh = torch.empty(M, N, dtype=torch.int16).pin_memory()
+    kx.kx_outproj_residual_host(Xh, Wh, bh, Rh, Yh, M, N, K)
+    y = Yh.numpy().view(np.uint16)
+    assert np.array_equal(y, run(d["X"], d["W"], d["bias"], d["R"]))
+    ok, msg = kt.gate_a(y, oracle.outproj(d["X"], d["W"], d["bias"], d["R"]))
+    assert ok, msg
+    # a larger problem afterwards grows the staging buffer
+    M2 = 900
+    d2 = inputs.make_inputs(inputs.Workload("t", M2, N, K, 72, False, False), stress=True)
+    Y2 = np.empty((M2, N), dtype=np.uint16)
+    kx.kx_outproj_residual_host(np.ascontiguousarray(d2["X"]), np.ascontiguousarray(d2["W"]), None, None, Y2, M2, N, K)
+    assert kt.rel_fro(Y2, oracle.outproj(d2["X"], d2["W"])) <= 2.0 ** -8
+
+
+def test_non_default_stream_and_plan_query():
+    import torch
+    info = kx.kx_plan_query(4096, 4096, 4096)
+    assert info.path == T and info.grid >= 1 and info.launches == 1 and info.tiles >= info.grid // 2
+    info = kx.kx_plan_query(32, 4096, 4096)
+    assert info.path == S and info.block_n == 32 and info.split_k >= 1
+    assert info.workspace_bytes == (info.split_k * 32 * 4096 * 4 if info.split_k > 1 else 0)
+    with pytest.raises(kx.KxError):
+        kx.kx_plan_query(4096, 4096, 4096, ov=kx.make_override(path=T, block_n=96))
+    X, W, b, R = ternary_case(256, 512, 256, seed=13)
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        y = run(X, W, b, R)
+    assert kt.gate_exact(y, oracle.outproj(X, W, b, R))[0]
