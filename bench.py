@@ -1,0 +1,443 @@
+#!/usr/bin/env python
+"""Benchmark of the BF16 output projection with residual (kx library) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+A step is one pass of the whole hot path (one C-ABI call = one kernel launch)
+over one batch of synthetic input.  The headline workload is the 4096^3
+out-projection + residual (no bias); the JSON line also carries every other
+measured workload under "shapes" (TFLOP/s, GB/s and roofline fraction per shape,
+geometric mean over the 16-shape sweep).
+
+`--impl reference` times the CPU oracle (the plain, slow definition the tests
+check against) on the host cores: a reported baseline, not a target.
+
+With N > 1 (under torchrun) every rank runs the same per-GPU workload on its own
+rows of a N-times-taller problem (rows of X, R, Y are independent; W is
+replicated), so there is no collective on the data path: weak scaling.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+L2_BYTES = 126 * (1 << 20)
+METRIC = "bf16_tflops"
+UNIT = "TFLOP/s"
+HEADLINE = "cfg2"
+# DRAM traffic per launch of the dominant kernel from the ncu capture summarised in
+# profiles/ (dram__bytes_read.sum + dram__bytes_write.sum); None until captured.
+NCU_TRAFFIC_BYTES = {"cfg2": 150873856}   # profiles/kx_tile_kernel_pair_cfg2.md
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            p = json.load(open(path))
+            return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                    "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                    "source": "measured"}
+        except Exception:
+            pass
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ---------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU through NVML while the
+    timed region runs (read-only)."""
+
+    def __init__(self, index: int, period_s: float = 0.004):
+        self.index, self.period = index, period_s
+        self.samples, self.reasons = [], set()
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+
+    def _reason_names(self, mask):
+        nv = self.nv
+        table = [("hw_slowdown", "nvmlClocksThrottleReasonHwSlowdown"),
+                 ("hw_thermal_slowdown", "nvmlClocksThrottleReasonHwThermalSlowdown"),
+                 ("sw_thermal_slowdown", "nvmlClocksThrottleReasonSwThermalSlowdown"),
+                 ("sw_power_cap", "nvmlClocksThrottleReasonSwPowerCap"),
+                 ("hw_power_brake", "nvmlClocksThrottleReasonHwPowerBrakeSlowdown"),
+                 ("applications_clocks", "nvmlClocksThrottleReasonApplicationsClocksSetting"),
+                 ("sync_boost", "nvmlClocksThrottleReasonSyncBoost")]
+        out = []
+        for name, attr in table:
+            bit = getattr(nv, attr, None)
+            if bit is not None and (mask & bit):
+                out.append(name)
+        return out
+
+    def _run(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                self.reasons.update(self._reason_names(int(mask)))
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join(timeout=2)
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": 0}
+        return {"sm_mhz": int(statistics.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# ---------------------------------------------------------------------------- helpers
+def roof(wl, seconds, peaks, sustained):
+    """Roofline line for one launch of `wl` that took `seconds`."""
+    tf_peak = peaks["bf16_tflops_sustained"] if sustained else peaks["bf16_tflops"]
+    t_tensor = wl.flops / (tf_peak * 1e12)
+    t_hbm = wl.algorithmic_bytes / (peaks["hbm_gbs"] * 1e9)
+    if t_tensor >= t_hbm:
+        ach = wl.flops / seconds / 1e12
+        return {"bound": "tensor", "achieved": ach, "peak": tf_peak, "unit": "TFLOP/s", "frac": ach / tf_peak}
+    ach = wl.algorithmic_bytes / seconds / 1e9
+    return {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"]}
+
+
+def device_sets(torch, wl, nsets, seed_bits=None):
+    """`nsets` independent operand sets for one workload on the current device.
+    Set 0 holds the workload's own seeded bits when given; further sets are
+    row-rotated copies (still random data, different addresses)."""
+    dev = torch.device("cuda")
+    sets = []
+    if seed_bits is not None:
+        def up(a):
+            return None if a is None else torch.from_numpy(a.view(np.int16)).to(dev).view(torch.bfloat16)
+        base = (up(seed_bits["X"]), up(seed_bits["W"]), up(seed_bits["bias"]), up(seed_bits["R"]))
+    else:
+        g = torch.Generator(device=dev)
+        g.manual_seed(wl.seed)
+        inv = 1.0 / math.sqrt(wl.K)
+        if wl.dist == "uniform":
+            X = ((torch.rand(wl.M, wl.K, device=dev, generator=g) * 2 - 1) * inv).bfloat16()
+            W = ((torch.rand(wl.N, wl.K, device=dev, generator=g) * 2 - 1) * inv).bfloat16()
+        else:
+            X = (torch.randn(wl.M, wl.K, device=dev, generator=g) * inv).bfloat16()
+            W = (torch.randn(wl.N, wl.K, device=dev, generator=g) * inv).bfloat16()
+        b = (torch.randn(wl.N, device=dev, generator=g) * 0.1).bfloat16() if wl.has_bias else None
+        R = torch.randn(wl.M, wl.N, device=dev, generator=g).bfloat16() if wl.has_residual else None
+        base = (X, W, b, R)
+    for j in range(nsets):
+        if j == 0:
+            X, W, b, R = base
+        else:
+            X = base[0].roll(j, 0).contiguous() if wl.M > 1 else base[0].roll(j, 1).contiguous()
+            W = base[1].roll(j, 0).contiguous()
+            b = None if base[2] is None else base[2].roll(j, 0).contiguous()
+            R = None if base[3] is None else base[3].roll(j, 1).contiguous()
+        Y = torch.empty(wl.M, wl.N, dtype=torch.bfloat16, device=dev)
+        sets.append((X, W, b, R, Y))
+    return sets
+
+
+def shard_workload(wl, rank):
+    """Rank r's slab of the N-times-taller problem: same shape per GPU, its own rows
+    of X and R (a different seed), the same W and bias (replicated)."""
+    import dataclasses
+    return wl if rank == 0 else dataclasses.replace(wl, seed=wl.seed + 1000 * rank)
+
+
+def shard_inputs(inputs, wl, rank):
+    bits = inputs.make_inputs(shard_workload(wl, rank))
+    if rank != 0:
+        base = inputs.make_inputs(wl)
+        bits["W"], bits["bias"] = base["W"], base["bias"]
+    return bits
+
+
+def max_over_ranks(dist, seconds, device):
+    """Whole-job time of a step = the slowest rank's device time."""
+    if dist is None:
+        return seconds
+    import torch
+    t = torch.tensor([seconds], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def sets_needed(wl, factor=2.0, cap=24):
+    per = wl.algorithmic_bytes
+    return int(max(2, min(cap, math.ceil(factor * L2_BYTES / per))))
+
+
+def bind_sets(kx, wl, sets):
+    """One pre-marshalled C-ABI call per operand set (on the current stream)."""
+    return [kx.bound_call(X, W, b, R, Y, plain=not wl.has_residual) for (X, W, b, R, Y) in sets]
+
+
+def call(kx, wl, s):
+    s()
+
+
+def time_steps(torch, kx, wl, sets, steps, warmup):
+    """CUDA-event time of `steps` back-to-back calls on the current stream (seconds per step)."""
+    for i in range(warmup):
+        call(kx, wl, sets[i % len(sets)])
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(steps):
+        call(kx, wl, sets[i % len(sets)])
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) * 1e-3 / steps
+
+
+# ---------------------------------------------------------------------------- reference arm
+def oracle_sample_rate(wl, bits, rows, repeats=1):
+    """Times the CPU oracle, as it stands, on `rows` rows of the workload."""
+    import oracle
+    t0 = time.perf_counter()
+    for _ in range(repeats):
+        oracle.outproj_rows(bits["X"], bits["W"], bits["bias"], bits["R"], rows)
+    dt = (time.perf_counter() - t0) / repeats
+    flops = 2.0 * len(rows) * wl.N * wl.K
+    return flops / dt / 1e12, dt
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    import oracle
+    from paper_2608_17071_b200 import inputs
+    wl = inputs.all_workloads()[HEADLINE]
+    bits = inputs.make_inputs(wl)
+    rows = np.arange(0, min(wl.M, 256), dtype=np.int64)
+    for _ in range(max(0, args.warmup)):
+        oracle.outproj_rows(bits["X"], bits["W"], bits["bias"], bits["R"], rows)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.outproj_rows(bits["X"], bits["W"], bits["bias"], bits["R"], rows)
+    dt = (time.perf_counter() - t0) / args.steps
+    val = 2.0 * len(rows) * wl.N * wl.K / dt / 1e12
+    cores = oracle.max_threads()
+    sample = f"{len(rows)} of {wl.M} rows of {HEADLINE} per step (all {wl.N} columns, K={wl.K})"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{HEADLINE}: out-proj + residual, M=K=N=4096, BF16 inputs, no bias", "sample": sample},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+# ---------------------------------------------------------------------------- our arm
+def run_ours(args):
+    import torch
+    from paper_2608_17071_b200 import binding as kx
+    from paper_2608_17071_b200 import inputs
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the kx library has no CPU fallback")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    kx.kx_init(local)
+    peaks = load_peaks()
+    wls = inputs.all_workloads()
+    headline = args.workload
+    wl = wls[headline]
+
+    # ---- headline workload: seeded bits (rank r draws its own rows: seed offset by rank)
+    bits = shard_inputs(inputs, wl, rank)
+    nsets = sets_needed(wl)
+    sets = bind_sets(kx, wl, device_sets(torch, wl, nsets, bits))
+    info = kx.kx_plan_query(wl.M, wl.N, wl.K, wl.has_bias, wl.has_residual)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(max(3, args.warmup)):
+        call(kx, wl, sets[i % nsets])
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local) as clk:
+        e0.record()
+        for i in range(args.steps):
+            call(kx, wl, sets[i % nsets])
+        e1.record()
+        torch.cuda.synchronize()
+    barrier()
+    sec = e0.elapsed_time(e1) * 1e-3
+    code, detail = kx.kx_last_device_status()
+    if code != 0:
+        raise SystemExit(f"kernel reported status {code} (wait {detail})")
+    sec = max_over_ranks(dist, sec, "cuda")
+    per_step = sec / args.steps
+    value = world * wl.flops / per_step / 1e12
+    sustained = sec > 1.0
+    rl = roof(wl, per_step, peaks, sustained)
+    rl["traffic"] = NCU_TRAFFIC_BYTES.get(headline)
+    rl["peak_source"] = f"of {peaks['source']} ({'sustained' if sustained else 'burst'} bf16 GEMM figure)"
+    rl["frac_of_nominal_2250"] = rl["achieved"] / 2250.0 if rl["bound"] == "tensor" else None
+
+    # ---- end to end through the host-buffer entry point (pinned host memory)
+    e2e = None
+    launches_e2e = 0
+    if not args.no_e2e:
+        pin = lambda a: None if a is None else torch.from_numpy(a.view(np.int16)).pin_memory()
+        Xh, Wh, bh, Rh = pin(bits["X"]), pin(bits["W"]), pin(bits["bias"]), pin(bits["R"])
+        Yh = torch.empty(wl.M, wl.N, dtype=torch.int16).pin_memory()
+        e2e_steps = max(3, min(args.steps, 20))
+        for _ in range(3):
+            kx.kx_outproj_residual_host(Xh, Wh, bh, Rh, Yh, wl.M, wl.N, wl.K)
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            kx.kx_outproj_residual_host(Xh, Wh, bh, Rh, Yh, wl.M, wl.N, wl.K)
+        torch.cuda.synchronize()
+        dt = time.perf_counter() - t0
+        dt = max_over_ranks(dist, dt, "cuda")
+        h2d = 2 * (wl.M * wl.K + wl.N * wl.K + (wl.M * wl.N if wl.has_residual else 0) + (wl.N if wl.has_bias else 0))
+        e2e = {"value": world * wl.flops / (dt / e2e_steps) / 1e12, "unit": UNIT,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": 2 * wl.M * wl.N, "steps": e2e_steps,
+               "ms_per_step": dt / e2e_steps * 1e3,
+               "api": "kx_outproj_residual_host (pinned host buffers in, Y copied back, stream synchronised)"}
+        launches_e2e = (3 + e2e_steps) * info.launches
+
+    # ---- every other workload (rank 0, N = 1 only): per-shape roofline lines
+    shapes = []
+    if rank == 0 and world == 1 and not args.no_sweep:
+        order = ["cfg1", "cfg2", "cfg4", "cfg5", "gemm4096"] + [w.name for w in inputs.sweep_workloads()]
+        for name in order:
+            w = wls[name]
+            ns = sets_needed(w)
+            ss = sets if name == headline else bind_sets(kx, w, device_sets(torch, w, ns))
+            iters = 200 if w.flops < 5e11 else 30
+            t = time_steps(torch, kx, w, ss, iters, 5)
+            pi = kx.kx_plan_query(w.M, w.N, w.K, w.has_bias, w.has_residual)
+            r = roof(w, t, peaks, False)
+            shapes.append({"name": name, "M": w.M, "N": w.N, "K": w.K, "us": t * 1e6,
+                           "tflops": w.flops / t / 1e12, "gbs": w.algorithmic_bytes / t / 1e9,
+                           "bound": r["bound"], "frac": r["frac"],
+                           "frac_nominal": (w.flops / t / 1e12 / 2250.0) if r["bound"] == "tensor"
+                           else (w.algorithmic_bytes / t / 1e9 / 8000.0),
+                           "plan": {"path": "tile" if pi.path == 1 else "swap", "block_n": pi.block_n,
+                                    "cta_pair": pi.cta_pair, "split_k": pi.split_k, "grid": pi.grid},
+                           "operand_sets": len(ss)})
+            del ss
+            torch.cuda.empty_cache()
+            print(f"[bench] {name:>18s} M={w.M:<6d} N={w.N:<5d} K={w.K:<6d} {t*1e6:9.1f} us "
+                  f"{w.flops/t/1e12:8.1f} TF {w.algorithmic_bytes/t/1e9:7.0f} GB/s  {r['bound']:6s} "
+                  f"{r['frac']*100:5.1f}% of {peaks['source']}", file=sys.stderr, flush=True)
+
+    # ---- the oracle on the host cores, bounded sample (rank 0, N = 1 only)
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        rows = np.arange(0, min(wl.M, 1024), dtype=np.int64)
+        v, dt = oracle_sample_rate(wl, bits, rows)
+        cpu = {"value": v, "unit": UNIT, "cores": oracle.max_threads(), "kind": "oracle",
+               "sample": f"rows 0..{len(rows) - 1} of {headline} ({len(rows)} of {wl.M} rows, all columns), {dt:.2f} s"}
+
+    if rank == 0:
+        sweep = [s for s in shapes if s["name"].startswith("sweep_")]
+        geo = lambda xs: math.exp(sum(math.log(x) for x in xs) / len(xs)) if xs else None
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(3, args.warmup), "ms_per_step": per_step * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"{headline}: {'out-proj + residual' if wl.has_residual else 'plain GEMM'}"
+                                   f"{' + bias' if wl.has_bias else ''}, M={wl.M} N={wl.N} K={wl.K} per GPU, BF16, "
+                                   f"{'X,W ~ U(-1,1)/sqrt(K)' if wl.dist == 'uniform' else 'X,W ~ N(0,1)/sqrt(K), R ~ N(0,1)'}, "
+                                   f"seed {wl.seed}",
+                       "l2": f"rotating {nsets} operand sets ({nsets * wl.algorithmic_bytes / 1e6:.0f} MB) > L2",
+                       "plan": {"path": "tile" if info.path == 1 else "swap", "block_n": info.block_n,
+                                "cta_pair": info.cta_pair, "stages": info.stages, "grid": info.grid,
+                                "tiles": info.tiles, "smem_bytes": info.smem_bytes},
+                       "parallelism": "none" if world == 1 else f"{world} independent row shards, W replicated, no collective"},
+            "roofline": rl,
+            "cpu_baseline": cpu,
+            "e2e": e2e,
+            "gpu_launches": args.steps * info.launches,
+            "gpu_launches_all_legs": (max(3, args.warmup) + args.steps) * info.launches + launches_e2e,
+            "clocks": clk.summary(),
+            "shapes": shapes,
+            "sweep_geomean": {"tflops": geo([s["tflops"] for s in sweep]), "roofline_frac": geo([s["frac"] for s in sweep]),
+                              "roofline_frac_nominal": geo([s["frac_nominal"] for s in sweep])},
+            "paper_context": "766 TFLOP/s BF16 on one 4096x4096 GEMM, H100 SXM (Section 4.1): other hardware, context only",
+        }
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--no-sweep", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--workload", default=HEADLINE, help="headline workload name (default: the 4096^3 out-projection)")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        args.steps = 5 if args.steps is None else args.steps
+        args.warmup = 1 if args.warmup is None else args.warmup
+        return run_reference(args)
+    args.steps = 500 if args.steps is None else args.steps
+    args.warmup = 10 if args.warmup is None else args.warmup
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -56,7 +56,7 @@ typedef enum kx_status {
     KX_ERR_PLAN = 9             /* plan override names an unsupported configuration   */
 } kx_status;
 
-/* Execution paths (Section 3.3's scheduling strategy names split-K and
+/* Execution paths (the scheduling strategy of Table 1 names split-K and
  * persistent kernels; the per-M specialisation follows Algorithm 3's per-M plan). */
 enum { KX_PATH_AUTO = 0, KX_PATH_TILE = 1, KX_PATH_SWAP = 2 };
 
@@ -65,13 +65,14 @@ enum { KX_PATH_AUTO = 0, KX_PATH_TILE = 1, KX_PATH_SWAP = 2 };
  *   path          KX_PATH_AUTO / KX_PATH_TILE (128-row output tiles, persistent,
  *                 TMA-store epilogue) / KX_PATH_SWAP (small M: W rows on the MMA
  *                 M axis, split-K, W streamed once)
- *   block_n       tile path: 64, 128 or 256 output columns per tile;
- *                 swap path: 16, 32, 64 or 128 (>= M)
+ *   block_n       tile path: 64, 128, 192 or 256 output columns per tile;
+ *                 swap path: 16, 32, 64, 128 or 256 X rows per unit
  *   cta_pair      0 auto, 1 = one CTA per tile, 2 = CTA pair per 256-row tile
  *   split_k       swap path only: number of K splits (1..64)
  *   raster_group  tile path: number of 128-row tile rows that share a raster group
  *   max_ctas      cap on the persistent grid (0 = number of SMs)
  *   spin_limit_us bound on every device-side wait (0 = 2 000 000 us)
+ *   stages        tile path: pick the variant with this ring depth (0 = default)
  *   debug_drop_kblocks  test hook: the TMA producer issues this many fewer
  *                 k-blocks than the MMA consumer expects, so the consumer's
  *                 bounded wait expires and the call reports
@@ -87,7 +88,8 @@ typedef struct kx_plan_override {
     int32_t max_ctas;
     int32_t spin_limit_us;
     int32_t debug_drop_kblocks;
-    int32_t reserved[8];
+    int32_t stages;
+    int32_t reserved[7];
 } kx_plan_override;
 
 /* What the planner chose for a shape (kx_plan_query). */

@@ -32,7 +32,7 @@ class PlanOverride(ctypes.Structure):
         ("path", ctypes.c_int32), ("block_n", ctypes.c_int32), ("cta_pair", ctypes.c_int32),
         ("split_k", ctypes.c_int32), ("raster_group", ctypes.c_int32), ("max_ctas", ctypes.c_int32),
         ("spin_limit_us", ctypes.c_int32), ("debug_drop_kblocks", ctypes.c_int32),
-        ("reserved", ctypes.c_int32 * 8),
+        ("stages", ctypes.c_int32), ("reserved", ctypes.c_int32 * 7),
     ]
 
 
@@ -176,6 +176,37 @@ def kx_outproj_residual_ex(X, W, bias, R, Y, ov: Optional[PlanOverride] = None, 
     if check and rc != KX_OK:
         raise KxError(rc, "kx_outproj_residual_ex")
     return rc
+
+
+def bound_call(X, W, bias, R, Y, stream=None, plain: bool = False):
+    """Marshal the arguments of kx_outproj_residual (or kx_gemm_bf16 when `plain`)
+    once and return a zero-argument callable that enqueues that same C call.
+    For callers that repeat one call many times (the Python-side checks and pointer
+    extraction cost more than a small kernel runs).  The callable holds references to
+    the tensors, so their memory stays allocated for as long as it is alive."""
+    M, K = X.shape
+    N = W.shape[0]
+    _check_bf16("X", X, (M, K)); _check_bf16("W", W, (N, K)); _check_bf16("Y", Y, (M, N))
+    lib = load()
+    vp = ctypes.c_void_p
+    st = vp(_stream(stream))
+    if plain:
+        args = (vp(_addr(X)), vp(_addr(W)), vp(_addr(Y)), ctypes.c_int64(M), ctypes.c_int64(N), ctypes.c_int64(K), st)
+        fn = lib.kx_gemm_bf16
+    else:
+        _check_bf16("bias", bias, (N,)); _check_bf16("R", R, (M, N))
+        args = (vp(_addr(X)), vp(_addr(W)), vp(_addr(bias)), vp(_addr(R)), vp(_addr(Y)),
+                ctypes.c_int64(M), ctypes.c_int64(N), ctypes.c_int64(K), st)
+        fn = lib.kx_outproj_residual
+
+    keep = (X, W, bias, R, Y, stream)
+
+    def run(_keep=keep):
+        rc = fn(*args)
+        if rc != KX_OK:
+            raise KxError(rc, fn.__name__)
+    run.tensors = keep
+    return run
 
 
 def kx_outproj_residual_host(X, W, bias, R, Y, M: int, N: int, K: int, stream=None, check=True) -> int:

@@ -70,16 +70,17 @@ struct SwapVariant {
     SwapVariant { BN, ST, SwapCfg<BN, ST>::SMEM_BYTES, reinterpret_cast<const void*>(&kx_swap_kernel<BN, ST>) }
 
 const TileVariant kTileVariants[] = {
-    KX_TILE(256, 1, 4, 2), KX_TILE(128, 1, 6, 2), KX_TILE(64, 1, 8, 2), KX_TILE(256, 2, 5, 4),
-    KX_TILE(128, 2, 7, 2),
+    KX_TILE(256, 1, 4, 2), KX_TILE(192, 1, 4, 3), KX_TILE(128, 1, 6, 2), KX_TILE(64, 1, 8, 2),
+    KX_TILE(256, 2, 6, 2), KX_TILE(256, 2, 5, 4), KX_TILE(192, 2, 6, 3), KX_TILE(128, 2, 7, 2),
 };
 const SwapVariant kSwapVariants[] = {
     KX_SWAP(16, 12), KX_SWAP(32, 11), KX_SWAP(64, 9), KX_SWAP(128, 7), KX_SWAP(256, 4),
 };
 
-const TileVariant* find_tile(int bn, int ctas) {
+// first variant in table order that matches; stages == 0 matches any depth
+const TileVariant* find_tile(int bn, int ctas, int stages) {
     for (const auto& v : kTileVariants)
-        if (v.bn == bn && v.ctas == ctas) return &v;
+        if (v.bn == bn && v.ctas == ctas && (stages == 0 || v.stages == stages)) return &v;
     return nullptr;
 }
 const SwapVariant* find_swap(int bn) {
@@ -232,19 +233,38 @@ struct Plan {
 
 int ceil_div(long long a, long long b) { return static_cast<int>((a + b - 1) / b); }
 
+// Split-K factor of the small-M path: enough units to give every SM one (a single
+// wave: the reduction tail of a second wave costs more than it buys), each split at
+// least four k-blocks long, partials inside the workspace.
 int pick_splits(int n_units, int nkb, int sms, long long M, long long N) {
-    int best = 1;
-    double best_eff = -1.0;
-    const int max_s = std::min(nkb, 64);
-    for (int s = 1; s <= max_s; ++s) {
-        if (s > 1 && nkb / s < 4) break;
-        if (static_cast<size_t>(s) * M * N * 4 > kWorkspaceBytes) break;
-        const long long units = static_cast<long long>(n_units) * s;
-        const long long waves = (units + sms - 1) / sms;
-        const double eff = static_cast<double>(units) / static_cast<double>(waves * sms);
-        if (eff > best_eff + 0.03) {
-            best = s;
-            best_eff = eff;
+    int s = std::max(1, sms / std::max(1, n_units));
+    s = std::min(s, std::max(1, nkb / 4));
+    s = std::min(s, 64);
+    while (s > 1 && static_cast<size_t>(s) * M * N * 4 > kWorkspaceBytes) --s;
+    return s;
+}
+
+// Relative mainloop efficiency of a tile width, measured on B200 with one CTA per
+// tile: operand bytes per flop grow as the tile narrows and the L2 -> SM feed
+// (about 128 B/clk/SM) becomes the limit (128x256 needs 94 B/clk, 128x192 104).
+double tile_width_eff(int bn) { return bn >= 256 ? 1.0 : bn >= 192 ? 0.85 : bn >= 128 ? 0.66 : 0.45; }
+
+// Tile width for the large-M path: the candidate with the best modelled throughput
+// = useful work / (waves x slots x tile area) x width efficiency.  On 148 SMs a
+// 4096 x 4096 output is 3.46 waves of 128x256 tiles (86 %) but 4.76 waves of
+// 128x192 tiles (92 % of five waves).
+int pick_block_n(long long M, long long N, int ctas, int slots) {
+    int best = 256;
+    double best_score = -1.0;
+    for (int bn : {256, 192, 128, 64}) {
+        const long long tiles = static_cast<long long>(ceil_div(M, 128 * ctas)) * ceil_div(N, bn);
+        const long long waves = (tiles + slots - 1) / slots;
+        const double useful = static_cast<double>(M) * static_cast<double>(N);
+        const double paid = static_cast<double>(waves) * slots * (128.0 * ctas) * bn;
+        const double score = useful / paid * tile_width_eff(bn);
+        if (score > best_score * 1.005) {
+            best_score = score;
+            best = bn;
         }
     }
     return best;
@@ -253,26 +273,22 @@ int pick_splits(int n_units, int nkb, int sms, long long M, long long N) {
 int make_plan(long long M, long long N, long long K, const kx_plan_override* ov, int sms, Plan* pl) {
     const int nkb = ceil_div(K, 64);
     int path = ov ? ov->path : KX_PATH_AUTO;
-    if (path == KX_PATH_AUTO) path = (M <= 128) ? KX_PATH_SWAP : KX_PATH_TILE;
+    if (path == KX_PATH_AUTO) path = (M <= 64) ? KX_PATH_SWAP : KX_PATH_TILE;
     if (path != KX_PATH_TILE && path != KX_PATH_SWAP) return KX_ERR_PLAN;
     const int max_ctas = (ov && ov->max_ctas > 0) ? std::min(ov->max_ctas, sms) : sms;
     pl->path = path;
     if (path == KX_PATH_TILE) {
-        int ctas = (ov && ov->cta_pair) ? ov->cta_pair : 1;
+        // A CTA pair (256 x BN tile, each CTA loading half of the W rows) halves the
+        // L2 -> SM operand traffic per flop; used whenever there are enough 256-row
+        // tiles to fill every pair slot.
+        int ctas = (ov && ov->cta_pair) ? ov->cta_pair : 0;
+        if (ctas == 0)
+            ctas = (static_cast<long long>(ceil_div(M, 256)) * ceil_div(N, 256) >= max_ctas / 2 && max_ctas >= 2) ? 2 : 1;
         if (ctas != 1 && ctas != 2) return KX_ERR_PLAN;
+        const int slots = std::max(1, max_ctas / ctas);
         int bn = ov ? ov->block_n : 0;
-        if (bn == 0) {
-            // widest tile that still gives every SM work
-            bn = 64;
-            for (int cand : {256, 128}) {
-                const long long tiles = static_cast<long long>(ceil_div(M, 128)) * ceil_div(N, cand);
-                if (tiles >= (max_ctas * 4) / 5) {
-                    bn = cand;
-                    break;
-                }
-            }
-        }
-        const TileVariant* v = find_tile(bn, ctas);
+        if (bn == 0) bn = pick_block_n(M, N, ctas, slots);
+        const TileVariant* v = find_tile(bn, ctas, ov ? ov->stages : 0);
         if (!v) return KX_ERR_PLAN;
         if (ov && ov->split_k > 1) return KX_ERR_PLAN;
         pl->bn = bn;
@@ -285,7 +301,6 @@ int make_plan(long long M, long long N, long long K, const kx_plan_override* ov,
         pl->tiles_n = ceil_div(N, bn);
         pl->units = pl->tiles_m * pl->tiles_n;
         pl->raster_group = (ov && ov->raster_group > 0) ? ov->raster_group : 8;
-        const int slots = std::max(1, max_ctas / ctas);
         pl->grid = std::min(pl->units, slots) * ctas;
         pl->splits = 1;
         pl->ws_bytes = 0;

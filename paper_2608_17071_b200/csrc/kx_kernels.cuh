@@ -607,16 +607,60 @@ kx_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
                 if (!epi_sync()) { ok = false; break; }
                 if (*s_last) {
                     __threadfence();
-                    if (n_ok) {
-                        const size_t plane = static_cast<size_t>(p.M) * p.N;
+                    // Re-mapped for memory-level parallelism: a warp covers one output row of the
+                    // tile (32 lanes x 4 columns, 16-byte loads), the four warps take rows
+                    // round-robin, and the loads of up to 8 splits x 2 rows are in flight before
+                    // any is consumed.  The sum still runs over splits 0,1,2,... in that order.
+                    const size_t plane = static_cast<size_t>(p.M) * p.N;
+                    const int nq = nt * 128 + lane * 4;
+                    if (nq < p.N) {
+                        float b4[4] = {0.f, 0.f, 0.f, 0.f};
+                        if (has_bias) {
+                            const uint2 bb = __ldg(reinterpret_cast<const uint2*>(p.bias + nq));
+                            b4[0] = bf16_lo(bb.x); b4[1] = bf16_hi(bb.x);
+                            b4[2] = bf16_lo(bb.y); b4[3] = bf16_hi(bb.y);
+                        }
 #pragma unroll 1
-                        for (int i = 0; i < m_cnt; ++i) {
-                            const size_t off = static_cast<size_t>(m0 + i) * p.N + n;
-                            float v = 0.f;
-                            for (int s2 = 0; s2 < p.splits; ++s2) v += __ldcg(p.ws + s2 * plane + off);
-                            v += bias_v;
-                            if (has_r) v += __uint_as_float(static_cast<uint32_t>(p.R[off]) << 16);
-                            p.Y[off] = static_cast<uint16_t>(pack_bf16x2(v, 0.f) & 0xFFFFu);
+                        for (int i0 = q; i0 < m_cnt; i0 += 8) {
+                            const int i1 = i0 + 4;
+                            const bool two = i1 < m_cnt;
+                            const size_t off0 = static_cast<size_t>(m0 + i0) * p.N + nq;
+                            const size_t off1 = static_cast<size_t>(m0 + (two ? i1 : i0)) * p.N + nq;
+                            float4 a0 = make_float4(0.f, 0.f, 0.f, 0.f), a1 = a0;
+                            uint2 r0 = make_uint2(0u, 0u), r1 = r0;
+                            if (has_r) {
+                                r0 = *reinterpret_cast<const uint2*>(p.R + off0);
+                                if (two) r1 = *reinterpret_cast<const uint2*>(p.R + off1);
+                            }
+#pragma unroll 1
+                            for (int s0 = 0; s0 < p.splits; s0 += 8) {
+                                float4 t0[8], t1[8];
+#pragma unroll
+                                for (int j = 0; j < 8; ++j) {
+                                    if (s0 + j < p.splits) {
+                                        const float* src = p.ws + static_cast<size_t>(s0 + j) * plane;
+                                        t0[j] = __ldcg(reinterpret_cast<const float4*>(src + off0));
+                                        t1[j] = __ldcg(reinterpret_cast<const float4*>(src + off1));
+                                    }
+                                }
+#pragma unroll
+                                for (int j = 0; j < 8; ++j) {
+                                    if (s0 + j < p.splits) {
+                                        a0.x += t0[j].x; a0.y += t0[j].y; a0.z += t0[j].z; a0.w += t0[j].w;
+                                        a1.x += t1[j].x; a1.y += t1[j].y; a1.z += t1[j].z; a1.w += t1[j].w;
+                                    }
+                                }
+                            }
+                            {
+                                const float v0 = a0.x + b4[0] + bf16_lo(r0.x), v1 = a0.y + b4[1] + bf16_hi(r0.x);
+                                const float v2 = a0.z + b4[2] + bf16_lo(r0.y), v3 = a0.w + b4[3] + bf16_hi(r0.y);
+                                *reinterpret_cast<uint2*>(p.Y + off0) = make_uint2(pack_bf16x2(v0, v1), pack_bf16x2(v2, v3));
+                            }
+                            if (two) {
+                                const float v0 = a1.x + b4[0] + bf16_lo(r1.x), v1 = a1.y + b4[1] + bf16_hi(r1.x);
+                                const float v2 = a1.z + b4[2] + bf16_lo(r1.y), v3 = a1.w + b4[3] + bf16_hi(r1.y);
+                                *reinterpret_cast<uint2*>(p.Y + off1) = make_uint2(pack_bf16x2(v0, v1), pack_bf16x2(v2, v3));
+                            }
                         }
                     }
                 }

@@ -103,3 +103,24 @@ def test_product_does_not_import_oracle():
                 text = open(os.path.join(dirpath, fn)).read()
                 assert not re.search(r"^\s*(from|import)\s+oracle\b", text, flags=re.M), fn
                 assert "kx_oracle" not in text, fn
+
+
+def test_bound_call_keeps_its_tensors_alive(lib):
+    """The pre-marshalled callable stores raw addresses, so it must own references
+    to the tensors: otherwise their memory could be released while calls remain."""
+    import gc
+    import weakref
+    import torch
+    X = torch.zeros(4, 8, dtype=torch.bfloat16)
+    W = torch.zeros(8, 8, dtype=torch.bfloat16)
+    R = torch.zeros(4, 8, dtype=torch.bfloat16)
+    Y = torch.zeros(4, 8, dtype=torch.bfloat16)
+    refs = [weakref.ref(t) for t in (X, W, R, Y)]
+    f = kx.bound_call(X, W, None, R, Y, stream=0)
+    del X, W, R, Y
+    gc.collect()
+    assert all(r() is not None for r in refs)
+    assert len(f.tensors) == 6
+    del f
+    gc.collect()
+    assert all(r() is None for r in refs)

@@ -16,7 +16,8 @@ T, S = kx.KX_PATH_TILE, kx.KX_PATH_SWAP
 TILE_VARIANTS = [
     dict(path=T, block_n=256, cta_pair=1), dict(path=T, block_n=128, cta_pair=1),
     dict(path=T, block_n=64, cta_pair=1), dict(path=T, block_n=256, cta_pair=2),
-    dict(path=T, block_n=128, cta_pair=2),
+    dict(path=T, block_n=128, cta_pair=2), dict(path=T, block_n=192, cta_pair=1),
+    dict(path=T, block_n=192, cta_pair=2),
 ]
 SWAP_VARIANTS = [
     dict(path=S, block_n=16, split_k=1), dict(path=S, block_n=16, split_k=4),
