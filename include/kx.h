@@ -53,7 +53,8 @@ typedef enum kx_status {
     KX_ERR_CUDA = 6,            /* a CUDA runtime/driver call failed                  */
     KX_ERR_WORKSPACE = 7,       /* split-K workspace too small / allocation failed    */
     KX_ERR_DEVICE_TIMEOUT = 8,  /* a bounded device-side wait gave up (see below)     */
-    KX_ERR_PLAN = 9             /* plan override names an unsupported configuration   */
+    KX_ERR_PLAN = 9,            /* plan override names an unsupported configuration   */
+    KX_ERR_LIMIT = 10           /* shape beyond kx_outproj_residual_noalloc's fixed scratch */
 } kx_status;
 
 /* Execution paths (the scheduling strategy of Table 1 names split-K and
@@ -152,6 +153,40 @@ int kx_outproj_residual_ex(const void* X, const void* W, const void* bias_or_nul
 int kx_outproj_residual_host(const void* X_host, const void* W_host, const void* bias_host_or_null,
                              const void* R_host_or_null, void* Y_host,
                              int64_t M, int64_t N, int64_t K, void* stream);
+
+/*
+ * Y = X W^T (+ bias) (+ R) for small M without any allocation, ever.  (The paper has no
+ * counterpart for this entry point; it exists for the sake of callers, not of the method.)
+ *
+ * Who needs it: code that must not ask the driver for device memory.  Examples are a
+ * serving process whose framework grabbed all of HBM for its own pool at start-up (a
+ * cudaMalloc from a library would fail or fragment that pool), a latency-critical loop
+ * that cannot tolerate the device-wide synchronisation a cudaMalloc / cudaFree may
+ * imply, and plug-ins whose host forbids allocation from worker threads.  The other
+ * entry points allocate their split-K workspace in kx_init or on first use; this one
+ * calls no cudaMalloc, no cudaFree and no routine that allocates on its behalf.
+ *
+ * How: it always runs the small-M split-K kernel, and the kernel's scratch (FP32 partial
+ * sums plus per-tile arrival counters) is a fixed array of 8 MiB + 16 KiB built into the
+ * library's device image.  Every GPU that loads the library carries that array until the
+ * process exits.
+ *
+ * Arguments, layout and preconditions are those of kx_outproj_residual_ex with a NULL
+ * plan (bias and R may each be NULL; Y may equal R).  Limits: M <= 256 and
+ * N <= 524288 (4096 column tiles); anything larger returns KX_ERR_LIMIT and enqueues
+ * nothing.  The split count shrinks as needed so that the partial sums fit in 8 MiB.
+ *
+ * The first call on each device looks up the array's device address and sets kernel
+ * attributes (no allocation); make that first call with the device current and before
+ * any stream capture begins.  All calls share the one array and it keeps the previous
+ * call's contents: the entry point zeroes the counters on `stream` before each launch,
+ * and partial sums are rewritten before they are read.  Two calls that run on the GPU at
+ * the same time (different streams, or different host threads on one device) would race
+ * on the array: order them on one stream or with events.
+ */
+int kx_outproj_residual_noalloc(const void* X, const void* W, const void* bias_or_null,
+                                const void* R_or_null, void* Y, int64_t M, int64_t N, int64_t K,
+                                void* stream);
 
 /* Fills `out` with the plan the library would use for this shape on the current
  * device (has_residual / has_bias as 0 or 1).  No work is enqueued. */

@@ -18,11 +18,12 @@ LIB_PATH = os.path.join(HERE, "libkx.so")
 KX_OK = 0
 KX_ERR_NULL, KX_ERR_SHAPE, KX_ERR_ALIGN, KX_ERR_OVERLAP = 1, 2, 3, 4
 KX_ERR_ARCH, KX_ERR_CUDA, KX_ERR_WORKSPACE, KX_ERR_DEVICE_TIMEOUT, KX_ERR_PLAN = 5, 6, 7, 8, 9
+KX_ERR_LIMIT = 10
 KX_PATH_AUTO, KX_PATH_TILE, KX_PATH_SWAP = 0, 1, 2
 
 EXPORTS = (
     "kx_init", "kx_shutdown", "kx_outproj_residual", "kx_gemm_bf16", "kx_outproj_residual_ex",
-    "kx_outproj_residual_host", "kx_plan_query", "kx_last_device_status", "kx_status_string",
+    "kx_outproj_residual_host", "kx_outproj_residual_noalloc", "kx_plan_query", "kx_last_device_status", "kx_status_string",
     "kx_version",
 )
 
@@ -72,6 +73,7 @@ def load():
     lib.kx_gemm_bf16.argtypes = [vp, vp, vp, i64, i64, i64, vp]
     lib.kx_outproj_residual_ex.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, vp, ctypes.POINTER(PlanOverride)]
     lib.kx_outproj_residual_host.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, vp]
+    lib.kx_outproj_residual_noalloc.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, vp]
     lib.kx_plan_query.argtypes = [i64, i64, i64, ci, ci, ctypes.POINTER(PlanOverride), ctypes.POINTER(PlanInfo)]
     lib.kx_last_device_status.argtypes = [vp, ctypes.POINTER(ci), ctypes.POINTER(ci)]
     lib.kx_status_string.argtypes = [ci]
@@ -175,6 +177,24 @@ def kx_outproj_residual_ex(X, W, bias, R, Y, ov: Optional[PlanOverride] = None, 
                                        _stream(stream), ctypes.byref(ov) if ov is not None else None)
     if check and rc != KX_OK:
         raise KxError(rc, "kx_outproj_residual_ex")
+    return rc
+
+
+def kx_outproj_residual_noalloc(X, W, bias, R, Y, stream=None, M=None, N=None, K=None, check=True) -> int:
+    """Small-M form that never allocates: for callers that may not ask the driver
+    for device memory (a process whose framework owns all of HBM, a loop that cannot
+    afford an allocation's synchronisation).  Its scratch is a fixed array inside the
+    library; M <= 256, N <= 524288, otherwise KX_ERR_LIMIT.  bias and R may be None.
+    Calls that overlap on the GPU share that array and would race."""
+    if M is None:
+        M, K = X.shape
+        N = W.shape[0]
+        _check_bf16("X", X, (M, K)); _check_bf16("W", W, (N, K)); _check_bf16("bias", bias, (N,))
+        _check_bf16("R", R, (M, N)); _check_bf16("Y", Y, (M, N))
+    rc = load().kx_outproj_residual_noalloc(_addr(X), _addr(W), _addr(bias), _addr(R), _addr(Y), M, N, K,
+                                            _stream(stream))
+    if check and rc != KX_OK:
+        raise KxError(rc, "kx_outproj_residual_noalloc")
     return rc
 
 

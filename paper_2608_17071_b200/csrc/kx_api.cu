@@ -13,6 +13,16 @@
 
 #include "kx_kernels.cuh"
 
+// Fixed scratch of kx_outproj_residual_noalloc: FP32 split-K partial sums followed by
+// the per-tile arrival counters.  It lives in the library's device image, so every GPU
+// that loads the library holds these bytes until the process exits.  Host code must
+// never hand this name to a kernel: on the host it is only a stand-in for the symbol;
+// the device address comes from cudaGetSymbolAddress (see noalloc_setup below).
+#define KX_NOALLOC_PARTIAL_BYTES (8u << 20)
+#define KX_NOALLOC_COUNTERS 4096u
+static __device__ __align__(256) unsigned char
+    g_kx_noalloc_scratch[KX_NOALLOC_PARTIAL_BYTES + KX_NOALLOC_COUNTERS * sizeof(unsigned int)];
+
 namespace {
 
 using namespace kx;
@@ -488,6 +498,9 @@ const char* kx_status_string(int s) {
         case KX_ERR_WORKSPACE: return "KX_ERR_WORKSPACE: split-K workspace too small or not allocated";
         case KX_ERR_DEVICE_TIMEOUT: return "KX_ERR_DEVICE_TIMEOUT: a bounded device-side wait gave up";
         case KX_ERR_PLAN: return "KX_ERR_PLAN: unsupported plan override";
+        case KX_ERR_LIMIT:
+            return "KX_ERR_LIMIT: shape exceeds the fixed scratch of kx_outproj_residual_noalloc "
+                   "(M <= 256 and N <= 524288)";
         default: return "KX_ERR_UNKNOWN";
     }
 }
@@ -631,6 +644,138 @@ int kx_outproj_residual_host(const void* Xh, const void* Wh, const void* bh, con
     if (rc != KX_OK) return rc;
     if (cudaMemcpyAsync(Yh, Yd, static_cast<size_t>(M) * N * 2, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
         cudaStreamSynchronize(stream) != cudaSuccess) {
+        cudaGetLastError();
+        return KX_ERR_CUDA;
+    }
+    return KX_OK;
+}
+
+// ---------------------------------------------------------------- no-allocation entry
+namespace {
+struct NoAllocCtx {
+    bool ready = false;
+    int sm_count = 0;
+    unsigned char* scratch = nullptr;   // device address of g_kx_noalloc_scratch on this device
+    unsigned int* status = nullptr;
+};
+NoAllocCtx g_noalloc[kMaxDevices];
+
+// Once per device, with that device current: resolve the device address of the static
+// scratch and raise the shared-memory limit of the kernels this entry point launches.
+// Nothing here allocates device memory.
+int noalloc_setup(int dev, NoAllocCtx** out) {
+    if (dev < 0 || dev >= kMaxDevices) return KX_ERR_CUDA;
+    NoAllocCtx& c = g_noalloc[dev];
+    std::lock_guard<std::mutex> lk(g_mu);
+    if (c.ready) {
+        *out = &c;
+        return KX_OK;
+    }
+    int major = 0, sms = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+        cudaGetLastError();
+        return KX_ERR_CUDA;
+    }
+    if (major != 10) return KX_ERR_ARCH;
+    if (!g_encode) {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+            qres != cudaDriverEntryPointSuccess || !fn) {
+            cudaGetLastError();
+            return KX_ERR_CUDA;
+        }
+        g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+    }
+    for (const auto& v : kSwapVariants)
+        if (cudaFuncSetAttribute(v.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, v.smem) != cudaSuccess) {
+            cudaGetLastError();
+            return KX_ERR_CUDA;
+        }
+    unsigned char* ptr = nullptr;
+    unsigned int* st = nullptr;
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_kx_noalloc_scratch) != cudaSuccess || !ptr ||
+        cudaGetSymbolAddress(reinterpret_cast<void**>(&st), g_kx_status) != cudaSuccess || !st) {
+        cudaGetLastError();
+        return KX_ERR_CUDA;
+    }
+    c.sm_count = sms;
+    c.scratch = ptr;
+    c.status = st;
+    c.ready = true;
+    *out = &c;
+    return KX_OK;
+}
+}  // namespace
+
+int kx_outproj_residual_noalloc(const void* X, const void* W, const void* bias, const void* R, void* Y,
+                                int64_t M, int64_t N, int64_t K, void* stream_v) {
+    int rc = validate(X, W, bias, R, Y, M, N, K, false);
+    if (rc != KX_OK) return rc;
+    if (M == 0 || N == 0) return KX_OK;
+    if (M > 256 || (N + 127) / 128 > static_cast<int64_t>(KX_NOALLOC_COUNTERS)) return KX_ERR_LIMIT;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return KX_ERR_CUDA;
+    NoAllocCtx* ctx = nullptr;
+    rc = noalloc_setup(dev, &ctx);
+    if (rc != KX_OK) return rc;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    if (K == 0) {
+        const long long total = M * N;
+        const int blocks = static_cast<int>(std::min<long long>((total + 255) / 256, ctx->sm_count * 8));
+        kx_k0_kernel<<<blocks, 256, 0, stream>>>(static_cast<const uint16_t*>(bias),
+                                                 static_cast<const uint16_t*>(R), static_cast<uint16_t*>(Y), M, N);
+        return cudaGetLastError() == cudaSuccess ? KX_OK : KX_ERR_CUDA;
+    }
+    const int bn = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : M <= 128 ? 128 : 256;
+    const SwapVariant* v = find_swap(bn);
+    if (!v) return KX_ERR_PLAN;
+    const int nkb = ceil_div(K, 64);
+    const int n_tiles = ceil_div(N, 128);
+    int splits = std::max(1, ctx->sm_count / n_tiles);
+    splits = std::min(splits, std::max(1, nkb / 4));
+    splits = std::min(splits, 64);
+    while (splits > 1 && static_cast<size_t>(splits) * M * N * 4 > KX_NOALLOC_PARTIAL_BYTES) --splits;
+
+    float* partials = reinterpret_cast<float*>(ctx->scratch);
+    unsigned int* counters = reinterpret_cast<unsigned int*>(ctx->scratch + KX_NOALLOC_PARTIAL_BYTES);
+    // The array keeps whatever the previous call (or a call that gave up) left in it.
+    // Partials are fully rewritten before they are read; the arrival counters must start at zero.
+    if (splits > 1 &&
+        cudaMemsetAsync(counters, 0, static_cast<size_t>(n_tiles) * sizeof(unsigned int), stream) != cudaSuccess) {
+        cudaGetLastError();
+        return KX_ERR_CUDA;
+    }
+    CUtensorMap tmW, tmX;
+    if ((rc = get_tmap(W, N, K, 128, &tmW)) != KX_OK) return rc;
+    if ((rc = get_tmap(X, M, K, bn, &tmX)) != KX_OK) return rc;
+    SwapParams p;
+    p.M = static_cast<int>(M);
+    p.N = static_cast<int>(N);
+    p.K = static_cast<int>(K);
+    p.n_tiles = n_tiles;
+    p.m_tiles = 1;
+    p.splits = splits;
+    p.num_units = n_tiles * splits;
+    p.has_bias = bias ? 1 : 0;
+    p.has_r = R ? 1 : 0;
+    p.drop_kblocks = 0;
+    p.spin_limit_ns = 2000000000ull;
+    p.status = ctx->status;
+    p.ws = partials;
+    p.counters = counters;
+    p.bias = static_cast<const uint16_t*>(bias);
+    p.R = static_cast<const uint16_t*>(R);
+    p.Y = static_cast<uint16_t*>(Y);
+    cudaLaunchConfig_t cfg;
+    std::memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3(std::min(p.num_units, ctx->sm_count), 1, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = v->smem;
+    cfg.stream = stream;
+    void* args[] = {&tmW, &tmX, &p};
+    if (cudaLaunchKernelExC(&cfg, v->fn, args) != cudaSuccess) {
         cudaGetLastError();
         return KX_ERR_CUDA;
     }

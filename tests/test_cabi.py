@@ -34,7 +34,7 @@ def test_header_symbols_are_exported(lib):
 
 def test_version_and_status_strings(lib):
     assert kx.kx_version() == 100
-    for code in range(0, 10):
+    for code in range(0, 11):
         s = kx.kx_status_string(code)
         assert s.startswith("KX_") and "UNKNOWN" not in s
     assert "UNKNOWN" in kx.kx_status_string(99)
