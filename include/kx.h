@@ -74,6 +74,11 @@ enum { KX_PATH_AUTO = 0, KX_PATH_TILE = 1, KX_PATH_SWAP = 2 };
  *   max_ctas      cap on the persistent grid (0 = number of SMs)
  *   spin_limit_us bound on every device-side wait (0 = 2 000 000 us)
  *   stages        tile path: pick the variant with this ring depth (0 = default)
+ *   stream_k      tile path: 0 auto, 1 = whole tiles per CTA (round-robin), 2 = stream-K
+ *                 (every CTA gets an equal contiguous range of (tile, k-block) units;
+ *                 split tiles are summed in the FP32 workspace in a fixed order)
+ *   narrow_tail   tile path: 0 auto, 1 off, 2 = run the tiles left over after the full
+ *                 waves as half-width tiles when they then fit in one extra wave
  *   debug_drop_kblocks  test hook: the TMA producer issues this many fewer
  *                 k-blocks than the MMA consumer expects, so the consumer's
  *                 bounded wait expires and the call reports
@@ -90,7 +95,9 @@ typedef struct kx_plan_override {
     int32_t spin_limit_us;
     int32_t debug_drop_kblocks;
     int32_t stages;
-    int32_t reserved[7];
+    int32_t stream_k;
+    int32_t narrow_tail;
+    int32_t reserved[5];
 } kx_plan_override;
 
 /* What the planner chose for a shape (kx_plan_query). */
@@ -105,8 +112,10 @@ typedef struct kx_plan_info {
     int32_t tiles;         /* work units (tiles x splits)                          */
     int32_t launches;      /* kernels enqueued per call                            */
     int32_t smem_bytes;    /* dynamic shared memory per CTA                        */
-    int64_t workspace_bytes; /* FP32 split-K scratch this plan uses (0 if none)    */
-    int32_t reserved[4];
+    int64_t workspace_bytes; /* FP32 split-K / stream-K scratch this plan uses (0 if none) */
+    int32_t stream_k;      /* 1 if the tile path runs with stream-K scheduling     */
+    int32_t narrow_tiles;  /* number of half-width tail tiles (0 if none)          */
+    int32_t reserved[2];
 } kx_plan_info;
 
 /*

@@ -45,6 +45,9 @@ struct DeviceCtx {
     size_t stage_bytes = 0;
 };
 DeviceCtx g_ctx[kMaxDevices];
+#ifdef KX_TRACE
+unsigned long long* g_kx_trace = nullptr;   // development builds: timeline buffer, 64 words per slot
+#endif
 std::mutex g_mu;
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -232,6 +235,10 @@ struct Plan {
     int path = 0;
     int bn = 0, ctas = 1, stages = 0, nb = 0;
     int splits = 1;
+    int stream_k = 0;
+    int sk_tile0 = 0;
+    int narrow_tile0 = 0;   // first half-width tail tile id (== units: none)
+    int wide_units = 0;     // number of full-width tile positions
     int raster_group = 8;
     int grid = 0, units = 0;
     int tiles_m = 0, tiles_n = 0;   // tile path: tile grid; swap path: m_tiles / n_tiles
@@ -311,9 +318,48 @@ int make_plan(long long M, long long N, long long K, const kx_plan_override* ov,
         pl->tiles_n = ceil_div(N, bn);
         pl->units = pl->tiles_m * pl->tiles_n;
         pl->raster_group = (ov && ov->raster_group > 0) ? ov->raster_group : 8;
-        pl->grid = std::min(pl->units, slots) * ctas;
         pl->splits = 1;
-        pl->ws_bytes = 0;
+        // Stream-K on the tail: when whole tiles would leave part of the last wave idle, the
+        // full waves but one stay whole-tile work and the remaining (slots + r) tiles are cut
+        // into equal contiguous ranges of (tile, k-block) units, one per slot; a tile that
+        // straddles two slots is finished by whichever holder arrives last.
+        const int full_waves = pl->units / slots, rem = pl->units % slots;
+        const int sk_tile0 = (full_waves >= 1) ? (full_waves - 1) * slots : 0;
+        const long long sk_units = static_cast<long long>(pl->units - sk_tile0) * nkb;
+        const int sk_slots = static_cast<int>(std::min<long long>(slots, sk_units));
+        const size_t sk_ws = static_cast<size_t>(sk_slots) * 2 * ctas * 128 * bn * sizeof(float);
+        const bool sk_fits = sk_ws <= kWorkspaceBytes &&
+                             static_cast<long long>(pl->units) * ctas * 4 <= kMaxCounters;
+        const long long waves = (pl->units + slots - 1) / slots;
+        const double dp_eff = static_cast<double>(pl->units) / static_cast<double>(waves * slots);
+        int sk = ov ? ov->stream_k : 0;                       // 0 auto, 1 off, 2 on
+        // Measured on B200: the fix-up of split tiles sits exposed at the kernel's tail and the
+        // part is power-limited (idle tail SMs leave headroom to the busy ones), so stream-K
+        // bought nothing on the measured shapes.  It stays available by explicit request only.
+        (void)dp_eff;
+        if (sk == 0) sk = 1;
+        if (sk == 2 && !sk_fits) return KX_ERR_WORKSPACE;
+        if (sk != 1 && sk != 2) return KX_ERR_PLAN;
+        pl->stream_k = (sk == 2) ? 1 : 0;
+        pl->sk_tile0 = pl->stream_k ? sk_tile0 : pl->units;
+        pl->grid = (pl->stream_k ? (sk_tile0 > 0 ? slots : sk_slots) : std::min(pl->units, slots)) * ctas;
+        pl->ws_bytes = pl->stream_k ? sk_ws : 0;
+        // Half-width tail: when the tiles left over after the full waves fit, cut in two, into
+        // one more (half as long) wave, run them as 128*ctas x BN/2 tiles.  No reduction, no
+        // workspace; 4096 x 4096 on 74 pair slots becomes 3 + 1/2 wave-times instead of 4.
+        pl->wide_units = pl->units;
+        pl->narrow_tile0 = pl->units;
+        int nt = ov ? ov->narrow_tail : 0;                    // 0 auto, 1 off, 2 on
+        const bool nt_ok = !pl->stream_k && (bn == 256 || bn == 128) && rem > 0 && full_waves >= 1 &&
+                           2 * rem <= slots;
+        if (nt == 0) nt = nt_ok ? 2 : 1;
+        if (nt == 2 && !nt_ok) nt = 1;
+        if (nt == 2) {
+            pl->narrow_tile0 = full_waves * slots;
+            pl->units = pl->narrow_tile0 + 2 * rem;
+            pl->sk_tile0 = pl->units;
+            pl->grid = slots * ctas;
+        }
     } else {
         int bn = ov ? ov->block_n : 0;
         if (bn == 0) bn = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : M <= 128 ? 128 : 256;
@@ -399,8 +445,8 @@ int run(const void* X, const void* W, const void* bias, const void* R, void* Y, 
                                       : 2000000000ull;
     const int drop = ov ? std::max(0, ov->debug_drop_kblocks) : 0;
     if (log_enabled())
-        std::fprintf(stderr, "[kx] M=%lld N=%lld K=%lld path=%d bn=%d ctas=%d stages=%d splits=%d grid=%d units=%d\n",
-                     M, N, K, pl.path, pl.bn, pl.ctas, pl.stages, pl.splits, pl.grid, pl.units);
+        std::fprintf(stderr, "[kx] M=%lld N=%lld K=%lld path=%d bn=%d ctas=%d stages=%d splits=%d streamk=%d grid=%d units=%d\n",
+                     M, N, K, pl.path, pl.bn, pl.ctas, pl.stages, pl.splits, pl.stream_k, pl.grid, pl.units);
 
     cudaLaunchConfig_t cfg;
     std::memset(&cfg, 0, sizeof cfg);
@@ -419,9 +465,14 @@ int run(const void* X, const void* W, const void* bias, const void* R, void* Y, 
     }
 
     if (pl.path == KX_PATH_TILE) {
-        CUtensorMap tmA, tmB, tmY, tmR;
+        CUtensorMap tmA, tmB, tmB2, tmY, tmR;
         if ((rc = get_tmap(X, M, K, 128, &tmA)) != KX_OK) return rc;
         if ((rc = get_tmap(W, N, K, pl.bn / pl.ctas, &tmB)) != KX_OK) return rc;
+        if (pl.narrow_tile0 < pl.units) {
+            if ((rc = get_tmap(W, N, K, pl.bn / 2 / pl.ctas, &tmB2)) != KX_OK) return rc;
+        } else {
+            tmB2 = tmB;
+        }
         if ((rc = get_tmap(Y, M, N, 32, &tmY)) != KX_OK) return rc;
         if (R) {
             if ((rc = get_tmap(R, M, N, 32, &tmR)) != KX_OK) return rc;
@@ -439,10 +490,17 @@ int run(const void* X, const void* W, const void* bias, const void* R, void* Y, 
         p.has_bias = bias ? 1 : 0;
         p.has_r = R ? 1 : 0;
         p.drop_kblocks = drop;
+        p.sk_tile0 = pl.sk_tile0;
+        p.narrow_tile0 = pl.narrow_tile0;
         p.spin_limit_ns = spin_ns;
         p.status = ctx->status;
+        p.ws = ctx->ws;
+        p.counters = ctx->counters;
+#ifdef KX_TRACE
+        p.trace = g_kx_trace;
+#endif
         const uint16_t* bias_p = static_cast<const uint16_t*>(bias);
-        void* args[] = {&tmA, &tmB, &tmY, &tmR, &bias_p, &p};
+        void* args[] = {&tmA, &tmB, &tmB2, &tmY, &tmR, &bias_p, &p};
         if (cudaLaunchKernelExC(&cfg, pl.fn, args) != cudaSuccess) {
             cudaGetLastError();
             return KX_ERR_CUDA;
@@ -485,6 +543,13 @@ extern "C" {
 #pragma GCC visibility push(default)
 
 int kx_version(void) { return KX_VERSION; }
+
+#ifdef KX_TRACE
+int kx_debug_set_trace(void* device_buffer) {
+    g_kx_trace = static_cast<unsigned long long*>(device_buffer);
+    return KX_OK;
+}
+#endif
 
 const char* kx_status_string(int s) {
     switch (s) {
@@ -562,6 +627,8 @@ int kx_plan_query(int64_t M, int64_t N, int64_t K, int has_bias, int has_residua
     out->cta_pair = pl.ctas;
     out->stages = pl.stages;
     out->split_k = pl.splits;
+    out->stream_k = pl.stream_k;
+    out->narrow_tiles = (pl.path == KX_PATH_TILE) ? pl.units - pl.narrow_tile0 : 0;
     out->raster_group = pl.raster_group;
     out->grid = pl.grid;
     out->tiles = pl.units;

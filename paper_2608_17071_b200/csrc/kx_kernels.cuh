@@ -30,6 +30,19 @@
 #pragma once
 #include "kx_ptx.cuh"
 
+// Optional timeline instrumentation (development builds only: -DKX_TRACE).  Each slot
+// records %globaltimer at up to 64 points; compiled out otherwise.
+#ifdef KX_TRACE
+#define KX_TRACE_DECL unsigned long long* trace;
+#define KX_TRACE_POINT(p, slot, idx)                                                        \
+    do {                                                                                     \
+        if ((p).trace && (idx) < 64) (p).trace[static_cast<size_t>(slot) * 64 + (idx)] = globaltimer_ns(); \
+    } while (0)
+#else
+#define KX_TRACE_DECL
+#define KX_TRACE_POINT(p, slot, idx) do { } while (0)
+#endif
+
 namespace kx {
 
 constexpr int kThreads = 192;         // warps 0-3 epilogue, 4 TMA producer, 5 MMA issuer
@@ -93,8 +106,16 @@ struct TileParams {
     int raster_group;
     int has_bias, has_r;
     int drop_kblocks;
+    int sk_tile0;                 // tiles [0, sk_tile0) are taken whole, round-robin over the slots;
+                                  // tiles [sk_tile0, num_tiles) are stream-K'd (== num_tiles: none)
+    int narrow_tile0;             // tile ids >= narrow_tile0 are half-width tiles: id = narrow_tile0 + 2 * j + half
+                                  // covers columns [half * BN/2, +BN/2) of full-width position narrow_tile0 + j
+                                  // (== num_tiles: none; never combined with stream-K)
     unsigned long long spin_limit_ns;
     unsigned int* status;
+    float* ws;                    // stream-K partials: [slot][head|tail][cta rank][chunk][warp][16-byte group][lane]
+    unsigned int* counters;       // stream-K arrivals: one word per (tile, cta rank, epilogue warp), zero between launches
+    KX_TRACE_DECL
 };
 
 template <int BN, int CTAS, int STAGES, int NB>
@@ -108,16 +129,67 @@ struct TileCfg {
     static constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + EPI_BYTES + 1024;
     static constexpr int TMEM_COLS = tmem_cols_for(2 * BN);
     static constexpr int CHUNKS = BN / 64;                  // 64-column epilogue chunks per tile
+    static constexpr int PART_FLOATS = 128 * BN;            // one CTA's FP32 partial of one tile
+    static constexpr bool HAS_NARROW = (BN % 128 == 0) && ((BN / 2 / CTAS) % 8 == 0);   // half-width tail tiles
     static_assert(BN % 64 == 0 && BN <= 256, "BN");
     static_assert(NUM_BARS * 8 + 16 <= 1024, "barrier area");
     static_assert(STAGE_BYTES % 1024 == 0, "stage alignment");
 };
 
+// Stream-K bookkeeping.  The stream-K region is the last (num_tiles - sk_tile0) tiles; its
+// iteration space is U = tiles x k-blocks units and slot s of G owns units
+// [s U / G, (s+1) U / G).  Earlier tiles are whole-tile work in round-robin order, which keeps
+// the tiles resident at one time adjacent in the raster (they share X and W panels in L2).
+__device__ __forceinline__ long long sk_begin(long long U, int G, int s) {
+    return (static_cast<long long>(s) * U) / G;
+}
+__device__ __forceinline__ int sk_slot_of(long long U, int G, long long u) {
+    return static_cast<int>(((u + 1) * G - 1) / U);
+}
+
+// The work of one slot (a CTA or a CTA pair) as a sequence of segments (tile, kb0, kb1).
+struct SegIter {
+    int nkb, sk_tile0, t, tstride;
+    long long u, u1;
+    __device__ __forceinline__ void init(const TileParams& p, int nkb_, int slot, int slots) {
+        nkb = nkb_;
+        sk_tile0 = p.sk_tile0;
+        t = slot;
+        tstride = slots;
+        const long long U = static_cast<long long>(p.num_tiles - p.sk_tile0) * nkb_;
+        u = sk_begin(U, slots, slot);
+        u1 = sk_begin(U, slots, slot + 1);
+    }
+    __device__ __forceinline__ bool next(int& tile, int& kb0, int& kb1) {
+        if (t < sk_tile0) {
+            tile = t;
+            kb0 = 0;
+            kb1 = nkb;
+            t += tstride;
+            return true;
+        }
+        if (u >= u1) return false;
+        const int st = static_cast<int>(u / nkb);
+        tile = sk_tile0 + st;
+        kb0 = static_cast<int>(u - static_cast<long long>(st) * nkb);
+        const long long len = min(static_cast<long long>(nkb - kb0), u1 - u);
+        kb1 = kb0 + static_cast<int>(len);
+        u += len;
+        return true;
+    }
+};
+
+__device__ __forceinline__ uint32_t ld_acquire_gpu_u32(const unsigned int* p) {
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
 template <int BN, int CTAS, int STAGES, int NB>
 __global__ void __launch_bounds__(kThreads, 1)
 kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-               const __grid_constant__ CUtensorMap tmY, const __grid_constant__ CUtensorMap tmR,
-               const uint16_t* __restrict__ bias, const TileParams p) {
+               const __grid_constant__ CUtensorMap tmB2, const __grid_constant__ CUtensorMap tmY,
+               const __grid_constant__ CUtensorMap tmR, const uint16_t* __restrict__ bias, const TileParams p) {
     using C = TileCfg<BN, CTAS, STAGES, NB>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -141,13 +213,14 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const uint32_t cta_rank = (CTAS == 2) ? cluster_ctarank() : 0u;
     const bool leader = (cta_rank == 0);
     const int nkb = (p.K + kBlockK - 1) / kBlockK;
-    const int unit0 = blockIdx.x / CTAS;
-    const int ustride = gridDim.x / CTAS;
+    const int slot = blockIdx.x / CTAS;
+    const int slots = gridDim.x / CTAS;
 
     if (threadIdx.x == 0) *s_abort = 0;
     if (warp == 4 && lane == 0) {
         prefetch_tmap(&tmA);
         prefetch_tmap(&tmB);
+        if (p.narrow_tile0 < p.num_tiles) prefetch_tmap(&tmB2);
         prefetch_tmap(&tmY);
         if (p.has_r) prefetch_tmap(&tmR);
     }
@@ -184,31 +257,51 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     wt.peer_abort = (CTAS == 2) ? map_to_cta(smem_u32(const_cast<uint32_t*>(s_abort)), cta_rank ^ 1u) : 0u;
     wt.limit_ns = p.spin_limit_ns;
 
+    SegIter it;
+    it.init(p, nkb, slot, slots);
+    int tile, kb0, kb1;
+    // tile id -> tile row, first output column, width class
+    auto decode_tile = [&](int t, int& tm, int& col, bool& narrow) {
+        narrow = t >= p.narrow_tile0;
+        int pos = t, half = 0;
+        if (narrow) {
+            const int j = t - p.narrow_tile0;
+            pos = p.narrow_tile0 + (j >> 1);
+            half = j & 1;
+        }
+        int tn;
+        tile_coords(pos, p.tiles_m, p.tiles_n, p.raster_group, tm, tn);
+        col = tn * BN + half * (BN / 2);
+    };
+
     if (warp == 4) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
             uint32_t s = 0, ph = 0;
             bool ok = true;
-            const int nkb_issue = nkb - p.drop_kblocks;
-            for (int t = unit0; t < p.num_tiles && ok; t += ustride) {
-                int tm, tn;
-                tile_coords(t, p.tiles_m, p.tiles_n, p.raster_group, tm, tn);
+            while (ok && it.next(tile, kb0, kb1)) {
+                int tm, col;
+                bool narrow;
+                decode_tile(tile, tm, col, narrow);
                 const int a_row = tm * (128 * CTAS) + static_cast<int>(cta_rank) * 128;
-                const int b_row = tn * BN + static_cast<int>(cta_rank) * C::BN_LOAD;
-                for (int kb = 0; kb < nkb_issue; ++kb) {
+                const int b_row = col + static_cast<int>(cta_rank) * (narrow ? C::BN_LOAD / 2 : C::BN_LOAD);
+                const CUtensorMap* const mapB = narrow ? &tmB2 : &tmB;
+                const uint32_t stage_tx = kABytes + (narrow ? C::B_BYTES / 2 : C::B_BYTES);
+                const int kb_end = kb1 - p.drop_kblocks;
+                for (int kb = kb0; kb < kb_end; ++kb) {
                     if (!wt.wait(empty(s), ph ^ 1u, kWhereEmpty)) { ok = false; break; }
                     const uint32_t sa = s_stage + s * C::STAGE_BYTES;
                     const uint32_t sb = sa + kABytes;
                     if constexpr (CTAS == 1) {
-                        mbar_arrive_expect_tx(full(s), C::STAGE_BYTES);
+                        mbar_arrive_expect_tx(full(s), stage_tx);
                         tma_load_2d(sa, &tmA, kb * kBlockK, a_row, full(s));
-                        tma_load_2d(sb, &tmB, kb * kBlockK, b_row, full(s));
+                        tma_load_2d(sb, mapB, kb * kBlockK, b_row, full(s));
                     } else {
                         // both CTAs' copies complete on the leader's barrier
-                        if (leader) mbar_arrive_expect_tx(full(s), 2 * C::STAGE_BYTES);
+                        if (leader) mbar_arrive_expect_tx(full(s), 2 * stage_tx);
                         const uint32_t fb = map_to_cta(full(s), 0);
                         tma_load_2d_pair(sa, &tmA, kb * kBlockK, a_row, fb);
-                        tma_load_2d_pair(sb, &tmB, kb * kBlockK, b_row, fb);
+                        tma_load_2d_pair(sb, mapB, kb * kBlockK, b_row, fb);
                     }
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
@@ -217,15 +310,20 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     } else if (warp == 5) {
         // ------------------------------------------------------------ MMA issuer
         if (leader && lane == 0) {
-            constexpr uint32_t idesc = idesc_bf16_f32(128 * CTAS, BN);
-            uint32_t s = 0, ph = 0, tcount = 0;
+            constexpr uint32_t idesc_wide = idesc_bf16_f32(128 * CTAS, BN);
+            constexpr uint32_t idesc_narrow = idesc_bf16_f32(128 * CTAS, BN / 2);
+            uint32_t s = 0, ph = 0, scount = 0;
             bool ok = true;
-            for (int t = unit0; t < p.num_tiles && ok; t += ustride, ++tcount) {
-                const uint32_t b = tcount & 1u, aph = (tcount >> 1) & 1u;
+            while (ok && it.next(tile, kb0, kb1)) {
+                const uint32_t b = scount & 1u, aph = (scount >> 1) & 1u;
+                const uint32_t idesc = (tile >= p.narrow_tile0) ? idesc_narrow : idesc_wide;
+                ++scount;
+                KX_TRACE_POINT(p, slot, (scount - 1) * 4 + 0);
                 if (!wt.wait(acc_empty(b), aph ^ 1u, kWhereAccEmpty)) { ok = false; break; }
                 tc_fence_after();
+                KX_TRACE_POINT(p, slot, (scount - 1) * 4 + 1);
                 const uint32_t d = tmem_base + b * BN;
-                for (int kb = 0; kb < nkb; ++kb) {
+                for (int kb = kb0; kb < kb1; ++kb) {
                     if (!wt.wait(full(s), ph, kWhereFull)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t sa = s_stage + s * C::STAGE_BYTES;
@@ -233,7 +331,7 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
                     for (int k = 0; k < 4; ++k)
                         mma_bf16<CTAS>(d, smem_desc_sw128(sa + k * 32), smem_desc_sw128(sb + k * 32), idesc,
-                                       static_cast<uint32_t>(kb | k));
+                                       static_cast<uint32_t>((kb - kb0) | k));
                     if constexpr (CTAS == 1) {
                         mma_commit<1>(empty(s));
                     } else {
@@ -258,63 +356,219 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
     } else {
         // ------------------------------------------------------------ epilogue warps
-        const int q = warp;                                // TMEM lanes 32q .. 32q+31
+        // Warp q owns TMEM lanes / tile rows 32q..32q+31 and is independent of the other
+        // three: its own staging buffers, R barriers, stores and stream-K counter.
+        const int q = warp;
         const uint32_t my_epi = s_epi + q * NB * C::SLAB_BYTES;
-        const int my_tiles = (unit0 < p.num_tiles) ? (p.num_tiles - unit0 + ustride - 1) / ustride : 0;
-        const uint32_t total_chunks = static_cast<uint32_t>(my_tiles) * C::CHUNKS;
         const bool has_r = p.has_r != 0, has_bias = p.has_bias != 0;
-
-        // position of this warp's slab for chunk number x of this CTA's chunk sequence
-        auto chunk_pos = [&](uint32_t x, int& row0, int& col0) {
-            const int seq = static_cast<int>(x / C::CHUNKS);
-            const int c = static_cast<int>(x % C::CHUNKS);
-            int tm, tn;
-            tile_coords(unit0 + seq * ustride, p.tiles_m, p.tiles_n, p.raster_group, tm, tn);
-            row0 = tm * (128 * CTAS) + static_cast<int>(cta_rank) * 128 + q * 32;
-            col0 = tn * BN + c * 64;
+        const long long U = static_cast<long long>(p.num_tiles - p.sk_tile0) * nkb;   // stream-K units
+        // Inside a partial, the 64 FP32 values a thread holds for chunk c live at float4 index
+        // ((c*4 + q)*16 + g)*32 + lane, g = 0..15: every warp-wide access is 512 contiguous bytes.
+        auto slab4 = [&](float* part, int c) {
+            return reinterpret_cast<float4*>(part) + (static_cast<size_t>(c) * 4 + q) * 16 * 32 + lane;
         };
-        auto issue_r = [&](uint32_t x) {                   // lane 0 only
-            int row0, col0;
-            chunk_pos(x, row0, col0);
-            if (row0 < p.M && col0 < p.N) {
-                const int j = static_cast<int>(x % NB);
-                mbar_arrive_expect_tx(r_full(q, j), C::SLAB_BYTES);
-                tma_load_2d(my_epi + j * C::SLAB_BYTES, &tmR, col0, row0, r_full(q, j));
-            }
-        };
-        if (has_r && lane == 0)
-            for (uint32_t x = 0; x + 1 < static_cast<uint32_t>(NB) && x < total_chunks; ++x) issue_r(x);
-
-        uint32_t cc = 0, tcount = 0, rphase = 0;
+        enum { kWhole = 0, kFast = 1, kWriter = 2, kSlow = 3, kNone = 4 };
+        uint32_t scount = 0, rphase = 0;
         bool ok = true;
-        for (int t = unit0; t < p.num_tiles && ok; t += ustride, ++tcount) {
-            const uint32_t b = tcount & 1u, aph = (tcount >> 1) & 1u;
-            int tm, tn;
-            tile_coords(t, p.tiles_m, p.tiles_n, p.raster_group, tm, tn);
+
+        // partial of (slot sl, tile tl) for this CTA rank: "head" if tl is the first tile the slot touches
+        auto part_ptr = [&](int sl, int tl) -> float* {
+            const int first_tile = p.sk_tile0 + static_cast<int>(sk_begin(U, slots, sl) / nkb);
+            const size_t idx = (static_cast<size_t>(sl) * 2 + (tl == first_tile ? 0 : 1)) * CTAS + cta_rank;
+            return p.ws + idx * C::PART_FLOATS;
+        };
+
+        while (ok && it.next(tile, kb0, kb1)) {
+            const uint32_t b = scount & 1u, aph = (scount >> 1) & 1u;
+            ++scount;
+            int tm, colbase;
+            bool narrow;
+            decode_tile(tile, tm, colbase, narrow);
             const int row0 = tm * (128 * CTAS) + static_cast<int>(cta_rank) * 128 + q * 32;
-            if (!__all_sync(0xffffffffu, wt.wait(acc_full(b), aph, kWhereAccFull))) { ok = false; break; }
-            tc_fence_after();
-#pragma unroll 1
-            for (int c = 0; c < C::CHUNKS; ++c, ++cc) {
-                const int j = static_cast<int>(cc % NB);
-                const int col0 = tn * BN + c * 64;
-                const bool valid = (row0 < p.M) && (col0 < p.N);
-                const uint32_t buf = my_epi + j * C::SLAB_BYTES;
-                uint32_t acc[2][32];
-                if (valid) {
-                    const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + b * BN + c * 64;
-                    tmem_ld_32x32(taddr, acc[0]);
-                    tmem_ld_32x32(taddr + 32, acc[1]);
-                    tmem_ld_wait();
+            const int nchunks = narrow ? C::CHUNKS / 2 : C::CHUNKS;
+            const bool whole = (kb0 == 0) && (kb1 == nkb);
+            auto chunk_valid = [&](int c) { return (row0 < p.M) && (colbase + c * 64 < p.N); };
+            auto issue_r = [&](int c) {                    // lane 0 only
+                if (chunk_valid(c)) {
+                    const int j = c % NB;
+                    mbar_arrive_expect_tx(r_full(q, j), C::SLAB_BYTES);
+                    tma_load_2d(my_epi + j * C::SLAB_BYTES, &tmR, colbase + c * 64, row0, r_full(q, j));
                 }
-                if (c == C::CHUNKS - 1) {                  // accumulator buffer b is drained
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) {
-                        if constexpr (CTAS == 1) mbar_arrive(acc_empty(b));
-                        else mbar_arrive_cluster(map_to_cta(acc_empty(b), 0));
+            };
+            // R slabs are requested in chunk order, up to NB-1 chunks ahead.  They are requested
+            // before the accumulator is ready whenever this warp will (whole tile) or is expected
+            // to (the slot's last segment: its partners ran at the start of their ranges) produce
+            // the output.
+            const bool last_seg = (it.t >= it.sk_tile0) && (it.u >= it.u1);
+            const bool spec_r = has_r && (whole || last_seg);
+            int n_iss = 0;                                 // R chunks requested so far (warp-uniform)
+            if (lane == 0) tma_store_wait_read<0>();       // staging buffers of the previous tile are free
+            if (spec_r) {
+                const int pre = (NB - 1 < nchunks) ? NB - 1 : nchunks;
+                for (; n_iss < pre; ++n_iss)
+                    if (lane == 0) issue_r(n_iss);
+            }
+            __syncwarp();
+
+            const uint32_t tbase = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + b * BN;
+            const uint32_t tother = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + (b ^ 1u) * BN;
+            int role = kWhole, s_first = 0, s_last = 0;
+            unsigned int* ctr = nullptr;
+            bool staged = false;   // the partner's partial already sits in the other accumulator buffer
+            if (!whole) {
+                const long long ut = static_cast<long long>(tile - p.sk_tile0) * nkb;
+                s_first = sk_slot_of(U, slots, ut);
+                s_last = sk_slot_of(U, slots, ut + nkb - 1);
+                ctr = p.counters + (static_cast<size_t>(tile) * CTAS + cta_rank) * 4 + q;
+                // Two-segment tile, last segment of this slot: no later segment needs the second
+                // accumulator buffer, and the partner usually finished long ago.  Copy its partial
+                // into that idle TMEM buffer while this segment's MMAs are still running.  (a + b is
+                // commutative, so taking this route or not gives the same bits.)
+                if (last_seg && s_last - s_first == 1) {
+                    uint32_t arrived = 0;
+                    if (lane == 0) arrived = ld_acquire_gpu_u32(ctr);
+                    arrived = __shfl_sync(0xffffffffu, arrived, 0);
+                    if (arrived == 1u) {
+                        float* src = part_ptr(s_first == slot ? s_last : s_first, tile);
+#pragma unroll 1
+                        for (int c = 0; c < C::CHUNKS; ++c) {
+                            if (!chunk_valid(c)) continue;
+                            const float4* s4 = slab4(src, c);
+                            float4 t[16];
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) t[i] = __ldcg(s4 + i * 32);
+                            uint32_t a[2][32];
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) {
+                                a[i >> 3][(i & 7) * 4 + 0] = __float_as_uint(t[i].x);
+                                a[i >> 3][(i & 7) * 4 + 1] = __float_as_uint(t[i].y);
+                                a[i >> 3][(i & 7) * 4 + 2] = __float_as_uint(t[i].z);
+                                a[i >> 3][(i & 7) * 4 + 3] = __float_as_uint(t[i].w);
+                            }
+                            tmem_st_32x32(tother + c * 64, a[0]);
+                            tmem_st_32x32(tother + c * 64 + 32, a[1]);
+                        }
+                        tmem_st_wait();
+                        staged = true;
                     }
                 }
+            }
+            if (!__all_sync(0xffffffffu, wt.wait(acc_full(b), aph, kWhereAccFull))) { ok = false; break; }
+            tc_fence_after();
+            if (q == 0 && lane == 0 && leader) KX_TRACE_POINT(p, slot, (scount - 1) * 4 + 2);
+
+            auto release_acc = [&]() {                     // accumulator buffer b is drained
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) {
+                    if constexpr (CTAS == 1) mbar_arrive(acc_empty(b));
+                    else mbar_arrive_cluster(map_to_cta(acc_empty(b), 0));
+                }
+            };
+            if (!whole) {
+                if (staged) {
+                    role = kFast;
+                } else {
+                    uint32_t arrived = 0;
+                    if (lane == 0) arrived = ld_acquire_gpu_u32(ctr);
+                    arrived = __shfl_sync(0xffffffffu, arrived, 0);
+                    role = (arrived == static_cast<uint32_t>(s_last - s_first)) ? kFast : kWriter;
+                }
+            }
+            if (role == kWriter) {
+                // not (yet) the last segment of this tile to arrive: park the partial in the workspace
+                float* dst = part_ptr(slot, tile);
+#pragma unroll 1
+                for (int c = 0; c < C::CHUNKS; ++c) {
+                    if (!chunk_valid(c)) continue;
+                    uint32_t a[2][32];
+                    tmem_ld_32x32(tbase + c * 64, a[0]);
+                    tmem_ld_32x32(tbase + c * 64 + 32, a[1]);
+                    tmem_ld_wait();
+                    float4* d4 = slab4(dst, c);
+#pragma unroll
+                    for (int i = 0; i < 16; ++i)
+                        d4[i * 32] = make_float4(__uint_as_float(a[i >> 3][(i & 7) * 4 + 0]),
+                                                 __uint_as_float(a[i >> 3][(i & 7) * 4 + 1]),
+                                                 __uint_as_float(a[i >> 3][(i & 7) * 4 + 2]),
+                                                 __uint_as_float(a[i >> 3][(i & 7) * 4 + 3]));
+                }
+                release_acc();
+                __threadfence();
+                __syncwarp();
+                uint32_t old = 0;
+                if (lane == 0) old = atomicAdd(ctr, 1u);
+                old = __shfl_sync(0xffffffffu, old, 0);
+                role = (old == static_cast<uint32_t>(s_last - s_first)) ? kSlow : kNone;
+                if (role == kSlow) __threadfence();
+            }
+            if (role == kNone) {
+                // another segment holder finishes this tile; consume the R slabs requested on spec
+                if (spec_r) {
+                    bool w = true;
+                    for (int c = 0; c < n_iss && w; ++c) {
+                        if (!chunk_valid(c)) continue;
+                        const int j = c % NB;
+                        w = __all_sync(0xffffffffu, wt.wait(r_full(q, j), (rphase >> j) & 1u, kWhereRFull));
+                        rphase ^= (1u << j);
+                    }
+                    if (!w) { ok = false; break; }
+                }
+                continue;
+            }
+
+            // kWhole / kFast / kSlow: this warp writes the tile's output rows
+#pragma unroll 1
+            for (int c = 0; c < nchunks; ++c) {
+                const int j = c % NB;
+                const int col0 = colbase + c * 64;
+                const bool valid = chunk_valid(c);
+                const uint32_t buf = my_epi + j * C::SLAB_BYTES;
+                if (has_r)
+                    for (; n_iss <= c; ++n_iss)
+                        if (lane == 0) issue_r(n_iss);
+                uint32_t acc[2][32];
+                if (valid && role == kWhole) {
+                    tmem_ld_32x32(tbase + c * 64, acc[0]);
+                    tmem_ld_32x32(tbase + c * 64 + 32, acc[1]);
+                    tmem_ld_wait();
+                }
+                if (valid && role != kWhole) {
+                    // split tile: sum the segments in slot order (own accumulator in its place);
+                    // all 16 loads of a segment are in flight before the first is consumed
+                    float sum[64];
+#pragma unroll
+                    for (int i = 0; i < 64; ++i) sum[i] = 0.f;
+#pragma unroll 1
+                    for (int sl = s_first; sl <= s_last; ++sl) {
+                        if (role == kFast && sl == slot) {
+                            tmem_ld_32x32(tbase + c * 64, acc[0]);
+                            tmem_ld_32x32(tbase + c * 64 + 32, acc[1]);
+                            tmem_ld_wait();
+#pragma unroll
+                            for (int i = 0; i < 64; ++i) sum[i] += __uint_as_float(acc[i >> 5][i & 31]);
+                        } else if (staged) {
+                            tmem_ld_32x32(tother + c * 64, acc[0]);
+                            tmem_ld_32x32(tother + c * 64 + 32, acc[1]);
+                            tmem_ld_wait();
+#pragma unroll
+                            for (int i = 0; i < 64; ++i) sum[i] += __uint_as_float(acc[i >> 5][i & 31]);
+                        } else {
+                            const float4* s4 = slab4(part_ptr(sl, tile), c);
+                            float4 t[16];
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) t[i] = __ldcg(s4 + i * 32);
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) {
+                                sum[i * 4 + 0] += t[i].x; sum[i * 4 + 1] += t[i].y;
+                                sum[i * 4 + 2] += t[i].z; sum[i * 4 + 3] += t[i].w;
+                            }
+                        }
+                    }
+#pragma unroll
+                    for (int i = 0; i < 64; ++i) acc[i >> 5][i & 31] = __float_as_uint(sum[i]);
+                }
+                if (c == nchunks - 1 && role != kSlow) release_acc();
                 if (valid) {
                     if (has_r) {
                         if (!__all_sync(0xffffffffu, wt.wait(r_full(q, j), (rphase >> j) & 1u, kWhereRFull))) {
@@ -366,14 +620,19 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         tma_store_commit();
                         tma_store_wait_read<1>();          // the store before this one has left its buffer
                     }
+                } else if (lane == 0) {
+                    tma_store_wait_read<0>();              // nothing stored for this chunk: drain the last store
                 }
-                // refill the buffer released by the previous chunk with the R slab NB-1 chunks ahead
-                if (has_r && lane == 0 && cc + NB - 1 < total_chunks) {
-                    if (!valid) tma_store_wait_read<0>();  // no store was issued above: drain the last one
-                    issue_r(cc + NB - 1);
+                // request the R slabs up to NB-1 chunks ahead; their buffers were just released
+                if (has_r) {
+                    const int target = (c + NB < nchunks) ? c + NB : nchunks;
+                    for (; n_iss < target; ++n_iss)
+                        if (lane == 0) issue_r(n_iss);
                 }
                 __syncwarp();
             }
+            if (role != kWhole && lane == 0) *ctr = 0u;    // every segment has arrived: reset for the next launch
+            if (q == 0 && lane == 0 && leader) KX_TRACE_POINT(p, slot, (scount - 1) * 4 + 3);
         }
         if (lane == 0) tma_store_wait_all<0>();
     }

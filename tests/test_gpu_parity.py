@@ -85,6 +85,71 @@ def test_swap_exact_integer_arithmetic(ov, N, K):
         assert ok, f"M={M}: {msg}"
 
 
+STREAMK_VARIANTS = [
+    dict(path=T, block_n=256, cta_pair=1, stream_k=2), dict(path=T, block_n=256, cta_pair=2, stream_k=2),
+    dict(path=T, block_n=128, cta_pair=1, stream_k=2), dict(path=T, block_n=192, cta_pair=2, stream_k=2),
+    dict(path=T, block_n=64, cta_pair=1, stream_k=2),
+]
+
+
+@pytest.mark.parametrize("ov", STREAMK_VARIANTS, ids=vid)
+@pytest.mark.parametrize("max_ctas", [0, 6, 37])
+@pytest.mark.parametrize("M,N,K", [(640, 1024, 512), (300, 520, 264), (512, 2048, 2048), (1000, 776, 4096)])
+def test_stream_k_exact_integer_arithmetic(ov, max_ctas, M, N, K):
+    """Stream-K scheduling: every CTA takes an equal contiguous range of (tile, k-block)
+    units, so tiles are split between CTAs at arbitrary k positions and summed through
+    the workspace.  With integer-valued data the result must still be bit-exact, and
+    the same bits must come out in place and on a second run (fixed summation order)."""
+    X, W, b, R = ternary_case(M, N, K, seed=21)
+    o = dict(ov, max_ctas=max_ctas)
+    ref = oracle.outproj(X, W, b, R)
+    y = run(X, W, b, R, o)
+    ok, msg = kt.gate_exact(y, ref)
+    assert ok, msg
+    y2 = run(X, W, b, R.copy(), o, inplace=True)
+    assert np.array_equal(y, y2)
+
+
+@pytest.mark.parametrize("ov,max_ctas,M,N", [
+    (dict(path=T, block_n=256, cta_pair=2), 12, 640, 1280),    # 15 pair tiles on 6 slots: 12 wide + 6 narrow
+    (dict(path=T, block_n=256, cta_pair=1), 10, 640, 1280),    # 25 tiles on 10 slots: 20 wide + 10 narrow
+    (dict(path=T, block_n=128, cta_pair=2), 12, 700, 520),     # 15 pair tiles on 6 slots, ragged rows and columns
+    (dict(path=T, block_n=128, cta_pair=1), 9, 300, 776),
+], ids=["pair256", "single256", "pair128-ragged", "single128-ragged"])
+def test_half_width_tail_tiles_exact(ov, max_ctas, M, N):
+    """Tiles left over after the full waves run as half-width tiles (second W tensor map,
+    narrower MMA, half the epilogue chunks).  Must be bit-exact, also in place."""
+    K = 520
+    o = dict(ov, max_ctas=max_ctas, narrow_tail=2)
+    info = kx.kx_plan_query(M, N, K, ov=kx.make_override(**o))
+    assert info.narrow_tiles > 0 and info.narrow_tiles % 2 == 0 and info.stream_k == 0
+    X, W, b, R = ternary_case(M, N, K, seed=23)
+    ref = oracle.outproj(X, W, b, R)
+    y = run(X, W, b, R, o)
+    ok, msg = kt.gate_exact(y, ref)
+    assert ok, msg
+    assert np.array_equal(run(X, W, b, R.copy(), o, inplace=True), y)
+    off = dict(ov, max_ctas=max_ctas, narrow_tail=1)
+    assert kx.kx_plan_query(M, N, K, ov=kx.make_override(**off)).narrow_tiles == 0
+    assert np.array_equal(run(X, W, b, R, off), y)
+
+
+@pytest.mark.parametrize("ov", STREAMK_VARIANTS[:2], ids=vid)
+def test_stream_k_random_data_is_deterministic_and_within_gates(ov):
+    wl = inputs.all_workloads()["cfg2"]
+    d = inputs.make_inputs(wl, stress=True, M=1100, N=1304, K=4096)
+    ref, absref = oracle.outproj(d["X"], d["W"], None, d["R"], want_abs=True)
+    ys = [run(d["X"], d["W"], None, d["R"], ov) for _ in range(3)]
+    assert np.array_equal(ys[0], ys[1]) and np.array_equal(ys[0], ys[2])
+    ok, msg = kt.gate_a(ys[0], ref)
+    assert ok, msg
+    ok, msg = kt.gate_c(ys[0], ref, absref, 4096, rate_limit=3e-2)
+    assert ok, msg
+    # plain GEMM through stream-K
+    y = run(d["X"], d["W"], None, None, ov)
+    assert kt.rel_fro(y, oracle.outproj(d["X"], d["W"])) <= 2.0 ** -8
+
+
 @pytest.mark.parametrize("ov", [TILE_VARIANTS[0], TILE_VARIANTS[3], SWAP_VARIANTS[1], SWAP_VARIANTS[6]], ids=vid)
 def test_exact_large_k(ov):
     """K = 14336 (the longest reduction of the workloads): any dropped or repeated
