@@ -225,6 +225,21 @@ def time_steps(torch, kx, wl, sets, steps, warmup):
     return e0.elapsed_time(e1) * 1e-3 / steps
 
 
+def time_shape(torch, kx, wl, sets, repeats=5, block_s=0.03, idle_s=0.25):
+    """Per-shape protocol of the sweep: `repeats` timed blocks of at most ~block_s seconds of
+    back-to-back calls, each after a short idle and 3 warm-up calls, so that every shape is
+    measured from a comparable power/thermal state (the part throttles under sustained tensor
+    load).  Returns (median, best) seconds per call."""
+    est = time_steps(torch, kx, wl, sets, 3, 3)
+    steps = int(max(5, min(300, block_s / max(est, 1e-7))))
+    ts = []
+    for _ in range(repeats):
+        time.sleep(idle_s)
+        ts.append(time_steps(torch, kx, wl, sets, steps, 3))
+    ts.sort()
+    return ts[len(ts) // 2], ts[0], steps
+
+
 # ---------------------------------------------------------------------------- reference arm
 def oracle_sample_rate(wl, bits, rows, repeats=1):
     """Times the CPU oracle, as it stands, on `rows` rows of the workload."""
@@ -358,21 +373,22 @@ def run_ours(args):
             w = wls[name]
             ns = sets_needed(w)
             ss = sets if name == headline else bind_sets(kx, w, device_sets(torch, w, ns))
-            iters = 200 if w.flops < 5e11 else 30
-            t = time_steps(torch, kx, w, ss, iters, 5)
+            t, tbest, iters = time_shape(torch, kx, w, ss)
             pi = kx.kx_plan_query(w.M, w.N, w.K, w.has_bias, w.has_residual)
             r = roof(w, t, peaks, False)
-            shapes.append({"name": name, "M": w.M, "N": w.N, "K": w.K, "us": t * 1e6,
+            shapes.append({"name": name, "M": w.M, "N": w.N, "K": w.K, "us": t * 1e6, "us_best": tbest * 1e6,
+                           "calls_per_block": iters,
                            "tflops": w.flops / t / 1e12, "gbs": w.algorithmic_bytes / t / 1e9,
-                           "bound": r["bound"], "frac": r["frac"],
+                           "bound": r["bound"], "frac": r["frac"], "frac_best": roof(w, tbest, peaks, False)["frac"],
                            "frac_nominal": (w.flops / t / 1e12 / 2250.0) if r["bound"] == "tensor"
                            else (w.algorithmic_bytes / t / 1e9 / 8000.0),
                            "plan": {"path": "tile" if pi.path == 1 else "swap", "block_n": pi.block_n,
-                                    "cta_pair": pi.cta_pair, "split_k": pi.split_k, "grid": pi.grid},
+                                    "cta_pair": pi.cta_pair, "split_k": pi.split_k, "grid": pi.grid,
+                                    "narrow_tiles": pi.narrow_tiles},
                            "operand_sets": len(ss)})
             del ss
             torch.cuda.empty_cache()
-            print(f"[bench] {name:>18s} M={w.M:<6d} N={w.N:<5d} K={w.K:<6d} {t*1e6:9.1f} us "
+            print(f"[bench] {name:>18s} M={w.M:<6d} N={w.N:<5d} K={w.K:<6d} {t*1e6:9.1f} us (best {tbest*1e6:7.1f}) "
                   f"{w.flops/t/1e12:8.1f} TF {w.algorithmic_bytes/t/1e9:7.0f} GB/s  {r['bound']:6s} "
                   f"{r['frac']*100:5.1f}% of {peaks['source']}", file=sys.stderr, flush=True)
 

@@ -79,6 +79,9 @@ enum { KX_PATH_AUTO = 0, KX_PATH_TILE = 1, KX_PATH_SWAP = 2 };
  *                 split tiles are summed in the FP32 workspace in a fixed order)
  *   narrow_tail   tile path: 0 auto, 1 off, 2 = run the tiles left over after the full
  *                 waves as half-width tiles when they then fit in one extra wave
+ *   no_pdl        1 = launch without programmatic stream serialization (by default the
+ *                 kernel's prologue may overlap the tail of the previous kernel in the
+ *                 stream; it waits for that kernel before its first global access)
  *   debug_drop_kblocks  test hook: the TMA producer issues this many fewer
  *                 k-blocks than the MMA consumer expects, so the consumer's
  *                 bounded wait expires and the call reports
@@ -97,7 +100,8 @@ typedef struct kx_plan_override {
     int32_t stages;
     int32_t stream_k;
     int32_t narrow_tail;
-    int32_t reserved[5];
+    int32_t no_pdl;
+    int32_t reserved[4];
 } kx_plan_override;
 
 /* What the planner chose for a shape (kx_plan_query). */

@@ -454,15 +454,24 @@ int run(const void* X, const void* W, const void* bias, const void* R, void* Y, 
     cfg.blockDim = dim3(kThreads, 1, 1);
     cfg.dynamicSmemBytes = pl.smem;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    if (pl.ctas == 2) {
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = 2;
-        attr[0].val.clusterDim.y = 1;
-        attr[0].val.clusterDim.z = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;
+    // Programmatic dependent launch: this kernel may be scheduled while its predecessor in the
+    // stream drains; it waits (griddepcontrol.wait) before its first global access.
+    cudaLaunchAttribute attr[2];
+    int nattr = 0;
+    if (!(ov && ov->no_pdl)) {
+        attr[nattr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[nattr].val.programmaticStreamSerializationAllowed = 1;
+        ++nattr;
     }
+    if (pl.ctas == 2) {
+        attr[nattr].id = cudaLaunchAttributeClusterDimension;
+        attr[nattr].val.clusterDim.x = 2;
+        attr[nattr].val.clusterDim.y = 1;
+        attr[nattr].val.clusterDim.z = 1;
+        ++nattr;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = nattr;
 
     if (pl.path == KX_PATH_TILE) {
         CUtensorMap tmA, tmB, tmB2, tmY, tmR;

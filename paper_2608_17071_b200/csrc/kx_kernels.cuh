@@ -251,6 +251,11 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
     tc_fence_after();
     const uint32_t tmem_base = *s_tmem;
+    // Everything above touched only this CTA's own resources; from here on global memory is
+    // read and written, so the previous kernel in the stream must be complete.  The next
+    // kernel may start its own prologue as soon as it finds a free SM.
+    pdl_wait_prior();
+    pdl_launch_dependents();
 
     Waiter wt;
     wt.abort_flag = s_abort;
@@ -733,6 +738,8 @@ kx_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *s_tmem;
+    pdl_wait_prior();          // prologue above overlapped the previous kernel's tail
+    pdl_launch_dependents();
 
     Waiter wt;
     wt.abort_flag = s_abort;
