@@ -79,6 +79,9 @@ enum { KX_PATH_AUTO = 0, KX_PATH_TILE = 1, KX_PATH_SWAP = 2 };
  *                 split tiles are summed in the FP32 workspace in a fixed order)
  *   narrow_tail   tile path: 0 auto, 1 off, 2 = run the tiles left over after the full
  *                 waves as half-width tiles when they then fit in one extra wave
+ *   cluster_reduce  swap path: 0 auto, 1 = sum the K splits through the FP32 workspace
+ *                 (last CTA to arrive reduces), 2 = the 2..8 splits of a tile form a
+ *                 thread-block cluster and are summed through distributed shared memory
  *   no_pdl        1 = launch without programmatic stream serialization (by default the
  *                 kernel's prologue may overlap the tail of the previous kernel in the
  *                 stream; it waits for that kernel before its first global access)
@@ -101,7 +104,8 @@ typedef struct kx_plan_override {
     int32_t stream_k;
     int32_t narrow_tail;
     int32_t no_pdl;
-    int32_t reserved[4];
+    int32_t cluster_reduce;
+    int32_t reserved[3];
 } kx_plan_override;
 
 /* What the planner chose for a shape (kx_plan_query). */
@@ -119,7 +123,8 @@ typedef struct kx_plan_info {
     int64_t workspace_bytes; /* FP32 split-K / stream-K scratch this plan uses (0 if none) */
     int32_t stream_k;      /* 1 if the tile path runs with stream-K scheduling     */
     int32_t narrow_tiles;  /* number of half-width tail tiles (0 if none)          */
-    int32_t reserved[2];
+    int32_t cluster_reduce;/* 1 if the swap path reduces its splits inside a cluster */
+    int32_t reserved[1];
 } kx_plan_info;
 
 /*

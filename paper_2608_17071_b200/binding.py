@@ -33,7 +33,7 @@ class PlanOverride(ctypes.Structure):
         ("path", ctypes.c_int32), ("block_n", ctypes.c_int32), ("cta_pair", ctypes.c_int32),
         ("split_k", ctypes.c_int32), ("raster_group", ctypes.c_int32), ("max_ctas", ctypes.c_int32),
         ("spin_limit_us", ctypes.c_int32), ("debug_drop_kblocks", ctypes.c_int32),
-        ("stages", ctypes.c_int32), ("stream_k", ctypes.c_int32), ("narrow_tail", ctypes.c_int32), ("no_pdl", ctypes.c_int32), ("reserved", ctypes.c_int32 * 4),
+        ("stages", ctypes.c_int32), ("stream_k", ctypes.c_int32), ("narrow_tail", ctypes.c_int32), ("no_pdl", ctypes.c_int32), ("cluster_reduce", ctypes.c_int32), ("reserved", ctypes.c_int32 * 3),
     ]
 
 
@@ -43,7 +43,7 @@ class PlanInfo(ctypes.Structure):
         ("stages", ctypes.c_int32), ("split_k", ctypes.c_int32), ("raster_group", ctypes.c_int32),
         ("grid", ctypes.c_int32), ("tiles", ctypes.c_int32), ("launches", ctypes.c_int32),
         ("smem_bytes", ctypes.c_int32), ("workspace_bytes", ctypes.c_int64),
-        ("stream_k", ctypes.c_int32), ("narrow_tiles", ctypes.c_int32), ("reserved", ctypes.c_int32 * 2),
+        ("stream_k", ctypes.c_int32), ("narrow_tiles", ctypes.c_int32), ("cluster_reduce", ctypes.c_int32), ("reserved", ctypes.c_int32 * 1),
     ]
 
 

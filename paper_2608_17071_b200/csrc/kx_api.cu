@@ -71,7 +71,8 @@ struct TileVariant {
 };
 struct SwapVariant {
     int bn, stages, smem;
-    const void* fn;
+    const void* fn;           // split-K through the global workspace (any split count)
+    const void* fn_cluster;   // split-K inside a thread-block cluster (2..8 splits)
 };
 
 #define KX_TILE(BN, CTAS, ST, NB)                                                             \
@@ -80,7 +81,11 @@ struct SwapVariant {
             reinterpret_cast<const void*>(&kx_tile_kernel<BN, CTAS, ST, NB>)                  \
     }
 #define KX_SWAP(BN, ST)                                                                       \
-    SwapVariant { BN, ST, SwapCfg<BN, ST>::SMEM_BYTES, reinterpret_cast<const void*>(&kx_swap_kernel<BN, ST>) }
+    SwapVariant {                                                                             \
+        BN, ST, SwapCfg<BN, ST>::SMEM_BYTES,                                                  \
+            reinterpret_cast<const void*>(&kx_swap_kernel<BN, ST, false>),                    \
+            reinterpret_cast<const void*>(&kx_swap_kernel<BN, ST, true>)                      \
+    }
 
 const TileVariant kTileVariants[] = {
     KX_TILE(256, 1, 4, 2), KX_TILE(192, 1, 4, 3), KX_TILE(128, 1, 6, 2), KX_TILE(64, 1, 8, 2),
@@ -147,8 +152,10 @@ int ensure_device(int dev, DeviceCtx** out) {
             ok = ok && cudaFuncSetAttribute(v.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, v.smem) ==
                            cudaSuccess;
         for (const auto& v : kSwapVariants)
-            ok = ok && cudaFuncSetAttribute(v.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, v.smem) ==
-                           cudaSuccess;
+            ok = ok &&
+                 cudaFuncSetAttribute(v.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, v.smem) == cudaSuccess &&
+                 cudaFuncSetAttribute(v.fn_cluster, cudaFuncAttributeMaxDynamicSharedMemorySize, v.smem) ==
+                     cudaSuccess;
         if (!ok) {
             rc = KX_ERR_CUDA;
             break;
@@ -237,6 +244,7 @@ struct Plan {
     int splits = 1;
     int stream_k = 0;
     int sk_tile0 = 0;
+    int cluster_reduce = 0; // swap path: the splits of a tile form a cluster and reduce through DSMEM
     int narrow_tile0 = 0;   // first half-width tail tile id (== units: none)
     int wide_units = 0;     // number of full-width tile positions
     int raster_group = 8;
@@ -285,6 +293,35 @@ int pick_block_n(long long M, long long N, int ctas, int slots) {
         }
     }
     return best;
+}
+
+// How many clusters of `size` CTAs of a swap-kernel variant can be resident at once
+// (a cluster lives inside one GPC, so this is less than SMs / size in general).
+int max_active_clusters(const SwapVariant* v, int size) {
+    static std::mutex mu;
+    static int cache[sizeof(kSwapVariants) / sizeof(kSwapVariants[0])][9];
+    const int vi = static_cast<int>(v - kSwapVariants);
+    std::lock_guard<std::mutex> lk(mu);
+    if (cache[vi][size] != 0) return cache[vi][size];
+    cudaLaunchConfig_t cfg;
+    std::memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3(size * 64, 1, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = v->smem;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = size;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, v->fn_cluster, &cfg) != cudaSuccess) {
+        cudaGetLastError();
+        n = -1;
+    }
+    cache[vi][size] = n > 0 ? n : -1;
+    return cache[vi][size];
 }
 
 int make_plan(long long M, long long N, long long K, const kx_plan_override* ov, int sms, Plan* pl) {
@@ -378,11 +415,26 @@ int make_plan(long long M, long long N, long long K, const kx_plan_override* ov,
         int splits = (ov && ov->split_k > 0) ? ov->split_k : pick_splits(static_cast<int>(tiles), nkb, max_ctas, M, N);
         splits = std::max(1, std::min(splits, std::max(1, nkb)));
         if (splits > 64) return KX_ERR_PLAN;
+        // Cluster reduction (2..8 splits): partials stay in shared memory and are summed
+        // through distributed shared memory.  Needs every CTA of a cluster resident at once,
+        // which the hardware guarantees per cluster; one unit per CTA.
+        int cr = ov ? ov->cluster_reduce : 0;                 // 0 auto, 1 off, 2 on
+        const bool auto_split = !(ov && ov->split_k > 0);
+        if (cr != 1 && auto_split) {
+            // largest cluster size (= split count) whose clusters are all resident at once
+            splits = std::min(splits, 8);
+            while (splits > 1 && max_active_clusters(v, splits) < tiles) --splits;
+        }
+        const bool cr_ok = splits >= 2 && splits <= 8 && !(ov && ov->max_ctas > 0);
+        if (cr == 0) cr = cr_ok ? 2 : 1;
+        if (cr == 2 && !cr_ok) return KX_ERR_PLAN;
+        pl->cluster_reduce = (cr == 2) ? 1 : 0;
+        if (pl->cluster_reduce) pl->fn = v->fn_cluster;
         pl->splits = splits;
-        pl->ws_bytes = splits > 1 ? static_cast<size_t>(splits) * M * N * 4 : 0;
+        pl->ws_bytes = (splits > 1 && !pl->cluster_reduce) ? static_cast<size_t>(splits) * M * N * 4 : 0;
         if (pl->ws_bytes > kWorkspaceBytes) return KX_ERR_WORKSPACE;
         pl->units = static_cast<int>(tiles * splits);
-        pl->grid = std::min(pl->units, max_ctas);
+        pl->grid = pl->cluster_reduce ? pl->units : std::min(pl->units, max_ctas);
     }
     return KX_OK;
 }
@@ -463,9 +515,9 @@ int run(const void* X, const void* W, const void* bias, const void* R, void* Y, 
         attr[nattr].val.programmaticStreamSerializationAllowed = 1;
         ++nattr;
     }
-    if (pl.ctas == 2) {
+    if (pl.ctas == 2 || pl.cluster_reduce) {
         attr[nattr].id = cudaLaunchAttributeClusterDimension;
-        attr[nattr].val.clusterDim.x = 2;
+        attr[nattr].val.clusterDim.x = pl.cluster_reduce ? pl.splits : 2;
         attr[nattr].val.clusterDim.y = 1;
         attr[nattr].val.clusterDim.z = 1;
         ++nattr;
@@ -536,6 +588,9 @@ int run(const void* X, const void* W, const void* bias, const void* R, void* Y, 
         p.bias = static_cast<const uint16_t*>(bias);
         p.R = static_cast<const uint16_t*>(R);
         p.Y = static_cast<uint16_t*>(Y);
+#ifdef KX_TRACE
+        p.trace = g_kx_trace;
+#endif
         void* args[] = {&tmW, &tmX, &p};
         if (cudaLaunchKernelExC(&cfg, pl.fn, args) != cudaSuccess) {
             cudaGetLastError();
@@ -638,6 +693,7 @@ int kx_plan_query(int64_t M, int64_t N, int64_t K, int has_bias, int has_residua
     out->split_k = pl.splits;
     out->stream_k = pl.stream_k;
     out->narrow_tiles = (pl.path == KX_PATH_TILE) ? pl.units - pl.narrow_tile0 : 0;
+    out->cluster_reduce = pl.cluster_reduce;
     out->raster_group = pl.raster_group;
     out->grid = pl.grid;
     out->tiles = pl.units;
@@ -844,6 +900,9 @@ int kx_outproj_residual_noalloc(const void* X, const void* W, const void* bias, 
     p.bias = static_cast<const uint16_t*>(bias);
     p.R = static_cast<const uint16_t*>(R);
     p.Y = static_cast<uint16_t*>(Y);
+#ifdef KX_TRACE
+    p.trace = nullptr;
+#endif
     cudaLaunchConfig_t cfg;
     std::memset(&cfg, 0, sizeof cfg);
     cfg.gridDim = dim3(std::min(p.num_units, ctx->sm_count), 1, 1);

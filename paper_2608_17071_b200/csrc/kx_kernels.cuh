@@ -671,6 +671,7 @@ struct SwapParams {
     const uint16_t* bias;
     const uint16_t* R;
     uint16_t* Y;
+    KX_TRACE_DECL
 };
 
 template <int BN, int STAGES>
@@ -685,11 +686,17 @@ struct SwapCfg {
     static_assert(STAGE_BYTES % 1024 == 0, "stage alignment");
 };
 
-template <int BN, int STAGES>
+// CLUSTER = true: the K splits of one tile form a thread-block cluster (cluster size ==
+// p.splits <= 8, one unit per CTA, grid == num_units).  Each CTA parks its FP32 partial in
+// its own shared memory, the cluster meets on the hardware cluster barrier, and every CTA
+// then finishes a share of the tile's rows by reading all partials through distributed
+// shared memory in split order: no workspace, no atomics, no fences, same deterministic sum.
+template <int BN, int STAGES, bool CLUSTER>
 __global__ void __launch_bounds__(kThreads, 1)
 kx_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
                const SwapParams p) {
     using C = SwapCfg<BN, STAGES>;
+    static_assert(!CLUSTER || BN * 128 * 4 <= STAGES * C::STAGE_BYTES, "partial must fit in the idle ring");
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -710,6 +717,7 @@ kx_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const int nkb = (p.K + kBlockK - 1) / kBlockK;
+    if (threadIdx.x == 0) KX_TRACE_POINT(p, blockIdx.x, 0);
 
     if (threadIdx.x == 0) *s_abort = 0;
     if (warp == 4 && lane == 0) {
@@ -738,8 +746,10 @@ kx_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *s_tmem;
+    if (threadIdx.x == 0) KX_TRACE_POINT(p, blockIdx.x, 1);
     pdl_wait_prior();          // prologue above overlapped the previous kernel's tail
     pdl_launch_dependents();
+    if (threadIdx.x == 0) KX_TRACE_POINT(p, blockIdx.x, 2);
 
     Waiter wt;
     wt.abort_flag = s_abort;
@@ -789,6 +799,8 @@ kx_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
                 for (int kb = kb0; kb < kb1; ++kb) {
                     if (!wt.wait(full(s), ph, kWhereFull)) { ok = false; break; }
                     tc_fence_after();
+                    if (ucount == 0 && kb == kb0) KX_TRACE_POINT(p, blockIdx.x, 3);
+                    if (ucount == 0 && kb == kb1 - 1) KX_TRACE_POINT(p, blockIdx.x, 4);
                     const uint32_t sa = s_stage + s * C::STAGE_BYTES;
                     const uint32_t sb = sa + kABytes;
 #pragma unroll
@@ -834,20 +846,35 @@ kx_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
             if (has_bias && n_ok) bias_v = __uint_as_float(static_cast<uint32_t>(__ldg(p.bias + n)) << 16);
             if (!__all_sync(0xffffffffu, wt.wait(acc_full(b), aph, kWhereAccFull))) { ok = false; break; }
             tc_fence_after();
+            if (etid == 0 && ucount == 0) KX_TRACE_POINT(p, blockIdx.x, 5);
 #pragma unroll 1
             for (int c0 = 0; c0 < m_cnt; c0 += 16) {
                 uint32_t a[16];
                 tmem_ld_32x16(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + b * BN + c0, a);
                 tmem_ld_wait();
-                if (n_ok) {
+                if (CLUSTER && p.splits > 1) {
+                    // partial -> this CTA's shared memory (the operand ring is idle by now):
+                    // red[m_local][128 columns], conflict-free for a fixed row
+                    float* red = reinterpret_cast<float*>(gbase);
+#pragma unroll
+                    for (int i = 0; i < 16; ++i)
+                        if (c0 + i < m_cnt) red[(c0 + i) * 128 + etid] = __uint_as_float(a[i]);
+                } else if (n_ok) {
+                    // R may alias Y (in place), so the compiler cannot move a residual load across
+                    // an output store: fetch the 16 residual values first, then store.
+                    uint16_t rv[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i)
+                        rv[i] = (p.splits == 1 && has_r && c0 + i < m_cnt)
+                                    ? p.R[static_cast<size_t>(m0 + c0 + i) * p.N + n] : static_cast<uint16_t>(0);
 #pragma unroll
                     for (int i = 0; i < 16; ++i) {
                         const int m = m0 + c0 + i;
                         if (c0 + i < m_cnt) {
                             const size_t off = static_cast<size_t>(m) * p.N + n;
                             if (p.splits == 1) {
-                                float v = __uint_as_float(a[i]) + bias_v;
-                                if (has_r) v += __uint_as_float(static_cast<uint32_t>(p.R[off]) << 16);
+                                const float v = __uint_as_float(a[i]) + bias_v +
+                                                __uint_as_float(static_cast<uint32_t>(rv[i]) << 16);
                                 p.Y[off] = static_cast<uint16_t>(pack_bf16x2(v, 0.f) & 0xFFFFu);
                             } else {
                                 p.ws[static_cast<size_t>(sp) * p.M * p.N + off] = __uint_as_float(a[i]);
@@ -859,10 +886,12 @@ kx_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(acc_empty(b));
-            if (p.splits > 1) {
+            if (!CLUSTER && p.splits > 1) {
                 // last CTA to finish this tile sums the splits in fixed order (deterministic)
+                if (etid == 0 && ucount == 0) KX_TRACE_POINT(p, blockIdx.x, 6);
                 __threadfence();
                 if (!epi_sync()) { ok = false; break; }
+                if (etid == 0 && ucount == 0) KX_TRACE_POINT(p, blockIdx.x, 7);
                 if (etid == 0) {
                     const int tile = nt * p.m_tiles + mt;
                     const unsigned int old = atomicAdd(p.counters + tile, 1u);
@@ -871,6 +900,7 @@ kx_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
                     *s_last = last ? 1u : 0u;
                 }
                 if (!epi_sync()) { ok = false; break; }
+                if (etid == 0 && ucount == 0) KX_TRACE_POINT(p, blockIdx.x, 8);
                 if (*s_last) {
                     __threadfence();
                     // Re-mapped for memory-level parallelism: a warp covers one output row of the
@@ -935,9 +965,86 @@ kx_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     }
 
     __syncwarp();
+    if constexpr (CLUSTER) {
+        // Every thread of every CTA of the cluster passes both barriers, whatever happened in
+        // its role above (all waits there are bounded), so the hardware barrier cannot hang.
+        // Rows sp, sp + splits, ... of the tile are finished by this CTA.
+        const bool reducer = warp < 4 && p.splits > 1 && static_cast<int>(blockIdx.x) < p.num_units;
+        int nt = 0, mt = 0, sp = 0, kb0 = 0, kb1 = 0;
+        if (reducer) unit_coords(blockIdx.x, nt, mt, sp, kb0, kb1);
+        const int etid = threadIdx.x;
+        const int n = nt * 128 + etid;
+        const bool n_ok = reducer && n < p.N;
+        const int m0 = mt * BN;
+        const int m_cnt = reducer ? min(BN, p.M - m0) : 0;
+        // residual and bias for this thread's outputs are fetched before the barrier: they do
+        // not depend on the partials, and R may alias Y so the loads must precede the stores
+        constexpr int kPre = 16;
+        uint16_t rv[kPre];
+        float bias_v = 0.f;
+        if (n_ok) {
+            if (p.has_bias) bias_v = __uint_as_float(static_cast<uint32_t>(__ldg(p.bias + n)) << 16);
+#pragma unroll
+            for (int k = 0; k < kPre; ++k) {
+                const int i = sp + k * p.splits;
+                rv[k] = (p.has_r && i < m_cnt) ? p.R[static_cast<size_t>(m0 + i) * p.N + n] : static_cast<uint16_t>(0);
+            }
+        }
+        if (threadIdx.x == 0) KX_TRACE_POINT(p, blockIdx.x, 6);
+        cluster_arrive();
+        cluster_wait();
+        if (threadIdx.x == 0) KX_TRACE_POINT(p, blockIdx.x, 7);
+        if (reducer) {
+            uint32_t rbase[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) rbase[j] = map_to_cta(base, j < p.splits ? j : 0) + etid * 4;
+            // four rows per batch: up to 32 remote loads in flight per thread, summed in split order
+#pragma unroll 1
+            for (int k0 = 0; sp + k0 * p.splits < m_cnt; k0 += 4) {
+                float t[4][8];
+#pragma unroll
+                for (int r4 = 0; r4 < 4; ++r4) {
+                    const int i = sp + (k0 + r4) * p.splits;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        t[r4][j] = (i < m_cnt && j < p.splits) ? ld_cluster_f32(rbase[j] + i * 512) : 0.f;
+                }
+                uint16_t rr[4];
+#pragma unroll
+                for (int r4 = 0; r4 < 4; ++r4) {
+                    const int k = k0 + r4, i = sp + k * p.splits;
+                    rr[r4] = 0;
+                    if (k < kPre) {
+#pragma unroll
+                        for (int kk = 0; kk < kPre; ++kk)
+                            if (kk == k) rr[r4] = rv[kk];
+                    } else if (n_ok && p.has_r && i < m_cnt) {
+                        rr[r4] = p.R[static_cast<size_t>(m0 + i) * p.N + n];
+                    }
+                }
+#pragma unroll
+                for (int r4 = 0; r4 < 4; ++r4) {
+                    const int i = sp + (k0 + r4) * p.splits;
+                    if (i < m_cnt && n_ok) {
+                        float v = 0.f;
+#pragma unroll
+                        for (int j = 0; j < 8; ++j)
+                            if (j < p.splits) v += t[r4][j];
+                        v += bias_v;
+                        v += __uint_as_float(static_cast<uint32_t>(rr[r4]) << 16);
+                        p.Y[static_cast<size_t>(m0 + i) * p.N + n] = static_cast<uint16_t>(pack_bf16x2(v, 0.f) & 0xFFFFu);
+                    }
+                }
+            }
+        }
+        cluster_arrive();
+        cluster_wait();
+    }
+    if (threadIdx.x == 0) KX_TRACE_POINT(p, blockIdx.x, 9);
     tc_fence_before();
     __syncthreads();
     if (warp == 5) tmem_dealloc<1>(tmem_base, C::TMEM_COLS);
+    if (threadIdx.x == 0) KX_TRACE_POINT(p, blockIdx.x, 10);
     if (threadIdx.x == 0 && *s_abort != 0) {
         if (atomicCAS(p.status, 0u, 8u) == 0u) p.status[1] = *s_abort;
     }

@@ -24,6 +24,10 @@ SWAP_VARIANTS = [
     dict(path=S, block_n=32, split_k=3), dict(path=S, block_n=64, split_k=2),
     dict(path=S, block_n=128, split_k=5), dict(path=S, block_n=256, split_k=1),
     dict(path=S, block_n=256, split_k=4),
+    # the same split counts summed through the FP32 workspace instead of the cluster
+    dict(path=S, block_n=16, split_k=4, cluster_reduce=1), dict(path=S, block_n=64, split_k=2, cluster_reduce=1),
+    dict(path=S, block_n=256, split_k=4, cluster_reduce=1), dict(path=S, block_n=32, split_k=12),
+    dict(path=S, block_n=128, split_k=8, cluster_reduce=2),
 ]
 
 
@@ -378,7 +382,8 @@ def test_non_default_stream_and_plan_query():
     assert info.path == T and info.grid >= 1 and info.launches == 1 and info.tiles >= info.grid // 2
     info = kx.kx_plan_query(32, 4096, 4096)
     assert info.path == S and info.block_n == 32 and info.split_k >= 1
-    assert info.workspace_bytes == (info.split_k * 32 * 4096 * 4 if info.split_k > 1 else 0)
+    ws = info.split_k * 32 * 4096 * 4 if (info.split_k > 1 and not info.cluster_reduce) else 0
+    assert info.workspace_bytes == ws and (info.cluster_reduce == 0 or 2 <= info.split_k <= 8)
     with pytest.raises(kx.KxError):
         kx.kx_plan_query(4096, 4096, 4096, ov=kx.make_override(path=T, block_n=96))
     X, W, b, R = ternary_case(256, 512, 256, seed=13)
