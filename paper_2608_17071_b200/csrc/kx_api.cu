@@ -334,10 +334,11 @@ int make_plan(long long M, long long N, long long K, const kx_plan_override* ov,
     if (path == KX_PATH_TILE) {
         // A CTA pair (256 x BN tile, each CTA loading half of the W rows) halves the
         // L2 -> SM operand traffic per flop; used whenever there are enough 256-row
-        // tiles to fill every pair slot.
+        // tiles to fill at least four fifths of the pair slots.
         int ctas = (ov && ov->cta_pair) ? ov->cta_pair : 0;
         if (ctas == 0)
-            ctas = (static_cast<long long>(ceil_div(M, 256)) * ceil_div(N, 256) >= max_ctas / 2 && max_ctas >= 2) ? 2 : 1;
+            ctas = (static_cast<long long>(ceil_div(M, 256)) * ceil_div(N, 256) * 5 >= (max_ctas / 2) * 4 &&
+                    max_ctas >= 2) ? 2 : 1;
         if (ctas != 1 && ctas != 2) return KX_ERR_PLAN;
         const int slots = std::max(1, max_ctas / ctas);
         int bn = ov ? ov->block_n : 0;
