@@ -972,22 +972,30 @@ kx_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         const bool reducer = warp < 4 && p.splits > 1 && static_cast<int>(blockIdx.x) < p.num_units;
         int nt = 0, mt = 0, sp = 0, kb0 = 0, kb1 = 0;
         if (reducer) unit_coords(blockIdx.x, nt, mt, sp, kb0, kb1);
-        const int etid = threadIdx.x;
-        const int n = nt * 128 + etid;
-        const bool n_ok = reducer && n < p.N;
+        // Re-mapped for the reduction: warp q takes this CTA's rows number q, q + 4, ... (the k-th
+        // row of the CTA is tile row sp + k * splits); a lane covers 4 adjacent columns, so every
+        // remote or global access of a warp is one contiguous row segment (512 / 256 bytes).
+        const int n4 = nt * 128 + lane * 4;
+        const bool n_ok = reducer && n4 < p.N;
         const int m0 = mt * BN;
         const int m_cnt = reducer ? min(BN, p.M - m0) : 0;
-        // residual and bias for this thread's outputs are fetched before the barrier: they do
-        // not depend on the partials, and R may alias Y so the loads must precede the stores
-        constexpr int kPre = 16;
-        uint16_t rv[kPre];
-        float bias_v = 0.f;
+        auto tile_row = [&](int k) { return sp + k * p.splits; };
+        // residual and bias for the first rows are fetched before the barrier: they do not
+        // depend on the partials, and R may alias Y so the loads must precede the stores
+        constexpr int kPre = 4;
+        uint2 rv[kPre];
+        float b4[4] = {0.f, 0.f, 0.f, 0.f};
         if (n_ok) {
-            if (p.has_bias) bias_v = __uint_as_float(static_cast<uint32_t>(__ldg(p.bias + n)) << 16);
+            if (p.has_bias) {
+                const uint2 bb = __ldg(reinterpret_cast<const uint2*>(p.bias + n4));
+                b4[0] = bf16_lo(bb.x); b4[1] = bf16_hi(bb.x); b4[2] = bf16_lo(bb.y); b4[3] = bf16_hi(bb.y);
+            }
 #pragma unroll
-            for (int k = 0; k < kPre; ++k) {
-                const int i = sp + k * p.splits;
-                rv[k] = (p.has_r && i < m_cnt) ? p.R[static_cast<size_t>(m0 + i) * p.N + n] : static_cast<uint16_t>(0);
+            for (int u = 0; u < kPre; ++u) {
+                const int i = tile_row(warp + 4 * u);
+                rv[u] = (p.has_r && i < m_cnt)
+                            ? *reinterpret_cast<const uint2*>(p.R + static_cast<size_t>(m0 + i) * p.N + n4)
+                            : make_uint2(0u, 0u);
             }
         }
         if (threadIdx.x == 0) KX_TRACE_POINT(p, blockIdx.x, 6);
@@ -997,42 +1005,41 @@ kx_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         if (reducer) {
             uint32_t rbase[8];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) rbase[j] = map_to_cta(base, j < p.splits ? j : 0) + etid * 4;
-            // four rows per batch: up to 32 remote loads in flight per thread, summed in split order
+            for (int j = 0; j < 8; ++j) rbase[j] = map_to_cta(base, j < p.splits ? j : 0) + lane * 16;
+            // two rows per batch: up to 16 remote 16-byte loads in flight per thread; the sum runs
+            // over the splits in order
 #pragma unroll 1
-            for (int k0 = 0; sp + k0 * p.splits < m_cnt; k0 += 4) {
-                float t[4][8];
+            for (int u0 = 0; tile_row(warp + 4 * u0) < m_cnt; u0 += 2) {
+                float4 t[2][8];
 #pragma unroll
-                for (int r4 = 0; r4 < 4; ++r4) {
-                    const int i = sp + (k0 + r4) * p.splits;
+                for (int r2 = 0; r2 < 2; ++r2) {
+                    const int i = tile_row(warp + 4 * (u0 + r2));
 #pragma unroll
                     for (int j = 0; j < 8; ++j)
-                        t[r4][j] = (i < m_cnt && j < p.splits) ? ld_cluster_f32(rbase[j] + i * 512) : 0.f;
-                }
-                uint16_t rr[4];
-#pragma unroll
-                for (int r4 = 0; r4 < 4; ++r4) {
-                    const int k = k0 + r4, i = sp + k * p.splits;
-                    rr[r4] = 0;
-                    if (k < kPre) {
-#pragma unroll
-                        for (int kk = 0; kk < kPre; ++kk)
-                            if (kk == k) rr[r4] = rv[kk];
-                    } else if (n_ok && p.has_r && i < m_cnt) {
-                        rr[r4] = p.R[static_cast<size_t>(m0 + i) * p.N + n];
-                    }
+                        if (i < m_cnt && j < p.splits) t[r2][j] = ld_cluster_f32x4(rbase[j] + i * 512);
                 }
 #pragma unroll
-                for (int r4 = 0; r4 < 4; ++r4) {
-                    const int i = sp + (k0 + r4) * p.splits;
+                for (int r2 = 0; r2 < 2; ++r2) {
+                    const int u = u0 + r2, i = tile_row(warp + 4 * u);
                     if (i < m_cnt && n_ok) {
-                        float v = 0.f;
+                        const size_t off = static_cast<size_t>(m0 + i) * p.N + n4;
+                        uint2 rr = make_uint2(0u, 0u);
+                        if (u < kPre) {
+#pragma unroll
+                            for (int uu = 0; uu < kPre; ++uu)
+                                if (uu == u) rr = rv[uu];
+                        } else if (p.has_r) {
+                            rr = *reinterpret_cast<const uint2*>(p.R + off);
+                        }
+                        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
                         for (int j = 0; j < 8; ++j)
-                            if (j < p.splits) v += t[r4][j];
-                        v += bias_v;
-                        v += __uint_as_float(static_cast<uint32_t>(rr[r4]) << 16);
-                        p.Y[static_cast<size_t>(m0 + i) * p.N + n] = static_cast<uint16_t>(pack_bf16x2(v, 0.f) & 0xFFFFu);
+                            if (j < p.splits) {
+                                v.x += t[r2][j].x; v.y += t[r2][j].y; v.z += t[r2][j].z; v.w += t[r2][j].w;
+                            }
+                        const float o0 = v.x + b4[0] + bf16_lo(rr.x), o1 = v.y + b4[1] + bf16_hi(rr.x);
+                        const float o2 = v.z + b4[2] + bf16_lo(rr.y), o3 = v.w + b4[3] + bf16_hi(rr.y);
+                        *reinterpret_cast<uint2*>(p.Y + off) = make_uint2(pack_bf16x2(o0, o1), pack_bf16x2(o2, o3));
                     }
                 }
             }
