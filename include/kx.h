@@ -82,6 +82,8 @@ enum { KX_PATH_AUTO = 0, KX_PATH_TILE = 1, KX_PATH_SWAP = 2 };
  *   cluster_reduce  swap path: 0 auto, 1 = sum the K splits through the FP32 workspace
  *                 (last CTA to arrive reduces), 2 = the 2..8 splits of a tile form a
  *                 thread-block cluster and are summed through distributed shared memory
+ *   no_table      1 = ignore the built-in measured plan table and use the heuristic
+ *                 (the table is consulted only when no plan field above is set)
  *   no_pdl        1 = launch without programmatic stream serialization (by default the
  *                 kernel's prologue may overlap the tail of the previous kernel in the
  *                 stream; it waits for that kernel before its first global access)
@@ -105,7 +107,8 @@ typedef struct kx_plan_override {
     int32_t narrow_tail;
     int32_t no_pdl;
     int32_t cluster_reduce;
-    int32_t reserved[3];
+    int32_t no_table;
+    int32_t reserved[2];
 } kx_plan_override;
 
 /* What the planner chose for a shape (kx_plan_query). */
@@ -124,7 +127,7 @@ typedef struct kx_plan_info {
     int32_t stream_k;      /* 1 if the tile path runs with stream-K scheduling     */
     int32_t narrow_tiles;  /* number of half-width tail tiles (0 if none)          */
     int32_t cluster_reduce;/* 1 if the swap path reduces its splits inside a cluster */
-    int32_t reserved[1];
+    int32_t from_table;    /* 1 if the built-in measured plan table supplied this plan */
 } kx_plan_info;
 
 /*

@@ -33,7 +33,7 @@ class PlanOverride(ctypes.Structure):
         ("path", ctypes.c_int32), ("block_n", ctypes.c_int32), ("cta_pair", ctypes.c_int32),
         ("split_k", ctypes.c_int32), ("raster_group", ctypes.c_int32), ("max_ctas", ctypes.c_int32),
         ("spin_limit_us", ctypes.c_int32), ("debug_drop_kblocks", ctypes.c_int32),
-        ("stages", ctypes.c_int32), ("stream_k", ctypes.c_int32), ("narrow_tail", ctypes.c_int32), ("no_pdl", ctypes.c_int32), ("cluster_reduce", ctypes.c_int32), ("reserved", ctypes.c_int32 * 3),
+        ("stages", ctypes.c_int32), ("stream_k", ctypes.c_int32), ("narrow_tail", ctypes.c_int32), ("no_pdl", ctypes.c_int32), ("cluster_reduce", ctypes.c_int32), ("no_table", ctypes.c_int32), ("reserved", ctypes.c_int32 * 2),
     ]
 
 
@@ -43,7 +43,7 @@ class PlanInfo(ctypes.Structure):
         ("stages", ctypes.c_int32), ("split_k", ctypes.c_int32), ("raster_group", ctypes.c_int32),
         ("grid", ctypes.c_int32), ("tiles", ctypes.c_int32), ("launches", ctypes.c_int32),
         ("smem_bytes", ctypes.c_int32), ("workspace_bytes", ctypes.c_int64),
-        ("stream_k", ctypes.c_int32), ("narrow_tiles", ctypes.c_int32), ("cluster_reduce", ctypes.c_int32), ("reserved", ctypes.c_int32 * 1),
+        ("stream_k", ctypes.c_int32), ("narrow_tiles", ctypes.c_int32), ("cluster_reduce", ctypes.c_int32), ("from_table", ctypes.c_int32),
     ]
 
 
@@ -198,7 +198,7 @@ def kx_outproj_residual_noalloc(X, W, bias, R, Y, stream=None, M=None, N=None, K
     return rc
 
 
-def bound_call(X, W, bias, R, Y, stream=None, plain: bool = False):
+def bound_call(X, W, bias, R, Y, stream=None, plain: bool = False, ov: Optional[PlanOverride] = None):
     """Marshal the arguments of kx_outproj_residual (or kx_gemm_bf16 when `plain`)
     once and return a zero-argument callable that enqueues that same C call.
     For callers that repeat one call many times (the Python-side checks and pointer
@@ -210,7 +210,13 @@ def bound_call(X, W, bias, R, Y, stream=None, plain: bool = False):
     lib = load()
     vp = ctypes.c_void_p
     st = vp(_stream(stream))
-    if plain:
+    if ov is not None:
+        # explicit plan: kx_outproj_residual_ex (bias and R optional)
+        _check_bf16("bias", bias, (N,)); _check_bf16("R", R, (M, N))
+        args = (vp(_addr(X)), vp(_addr(W)), vp(_addr(bias)), vp(_addr(R)), vp(_addr(Y)),
+                ctypes.c_int64(M), ctypes.c_int64(N), ctypes.c_int64(K), st, ctypes.byref(ov))
+        fn = lib.kx_outproj_residual_ex
+    elif plain:
         args = (vp(_addr(X)), vp(_addr(W)), vp(_addr(Y)), ctypes.c_int64(M), ctypes.c_int64(N), ctypes.c_int64(K), st)
         fn = lib.kx_gemm_bf16
     else:
@@ -219,7 +225,7 @@ def bound_call(X, W, bias, R, Y, stream=None, plain: bool = False):
                 ctypes.c_int64(M), ctypes.c_int64(N), ctypes.c_int64(K), st)
         fn = lib.kx_outproj_residual
 
-    keep = (X, W, bias, R, Y, stream)
+    keep = (X, W, bias, R, Y, stream, ov)
 
     def run(_keep=keep):
         rc = fn(*args)

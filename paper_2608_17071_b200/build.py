@@ -13,7 +13,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libkx.so")
 SOURCES = ["kx_api.cu"]
-DEPS = ["kx_api.cu", "kx_kernels.cuh", "kx_ptx.cuh", os.path.join("..", "..", "include", "kx.h")]
+DEPS = ["kx_api.cu", "kx_kernels.cuh", "kx_ptx.cuh", "kx_plan_table.inc", os.path.join("..", "..", "include", "kx.h")]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

@@ -244,6 +244,7 @@ struct Plan {
     int splits = 1;
     int stream_k = 0;
     int sk_tile0 = 0;
+    int from_table = 0;     // 1 if the static plan table supplied this plan
     int cluster_reduce = 0; // swap path: the splits of a tile form a cluster and reduce through DSMEM
     int narrow_tile0 = 0;   // first half-width tail tile id (== units: none)
     int wide_units = 0;     // number of full-width tile positions
@@ -295,6 +296,24 @@ int pick_block_n(long long M, long long N, int ctas, int slots) {
     return best;
 }
 
+// Static plan table (measured on B200 by `python -m paper_2608_17071_b200.tune`): per
+// (M bucket, N, K) the plan that beat the heuristic by the tuner's margin and reproduced its
+// output.  Same shape as the paper's artifact for this operator (Appendix A, Algorithm 3):
+// look up the entry for M, use it if it validates, else fall back to the heuristic.
+struct PlanTableEntry {
+    long long m_lo, m_hi, n, k;
+    int path, block_n, cta_pair, split_k, raster_group, stages, stream_k, narrow_tail, cluster_reduce;
+};
+const PlanTableEntry kPlanTable[] = {
+#include "kx_plan_table.inc"
+    {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0}   // sentinel
+};
+const PlanTableEntry* find_table_entry(long long M, long long N, long long K) {
+    for (const PlanTableEntry* e = kPlanTable; e->n != 0; ++e)
+        if (e->n == N && e->k == K && M >= e->m_lo && M <= e->m_hi) return e;
+    return nullptr;
+}
+
 // How many clusters of `size` CTAs of a swap-kernel variant can be resident at once
 // (a cluster lives inside one GPC, so this is less than SMs / size in general).
 int max_active_clusters(const SwapVariant* v, int size) {
@@ -324,7 +343,39 @@ int max_active_clusters(const SwapVariant* v, int size) {
     return cache[vi][size];
 }
 
+int make_plan_from(long long M, long long N, long long K, const kx_plan_override* ov, int sms, Plan* pl);
+
+// Caller's override > static table entry (if it validates) > heuristic.
 int make_plan(long long M, long long N, long long K, const kx_plan_override* ov, int sms, Plan* pl) {
+    const bool pinned = ov && (ov->path || ov->block_n || ov->cta_pair || ov->split_k || ov->raster_group ||
+                               ov->stages || ov->stream_k || ov->narrow_tail || ov->cluster_reduce ||
+                               ov->max_ctas || ov->no_table);
+    if (!pinned) {
+        if (const PlanTableEntry* e = find_table_entry(M, N, K)) {
+            kx_plan_override t;
+            std::memset(&t, 0, sizeof t);
+            if (ov) t = *ov;                      // keeps spin limit / PDL / debug fields
+            t.path = e->path;
+            t.block_n = e->block_n;
+            t.cta_pair = e->cta_pair;
+            t.split_k = e->split_k;
+            t.raster_group = e->raster_group;
+            t.stages = e->stages;
+            t.stream_k = e->stream_k;
+            t.narrow_tail = e->narrow_tail;
+            t.cluster_reduce = e->cluster_reduce;
+            Plan cand;
+            if (make_plan_from(M, N, K, &t, sms, &cand) == KX_OK) {
+                *pl = cand;
+                pl->from_table = 1;
+                return KX_OK;
+            }
+        }
+    }
+    return make_plan_from(M, N, K, ov, sms, pl);
+}
+
+int make_plan_from(long long M, long long N, long long K, const kx_plan_override* ov, int sms, Plan* pl) {
     const int nkb = ceil_div(K, 64);
     int path = ov ? ov->path : KX_PATH_AUTO;
     if (path == KX_PATH_AUTO) path = (M <= 64) ? KX_PATH_SWAP : KX_PATH_TILE;
@@ -695,6 +746,7 @@ int kx_plan_query(int64_t M, int64_t N, int64_t K, int has_bias, int has_residua
     out->stream_k = pl.stream_k;
     out->narrow_tiles = (pl.path == KX_PATH_TILE) ? pl.units - pl.narrow_tile0 : 0;
     out->cluster_reduce = pl.cluster_reduce;
+    out->from_table = pl.from_table;
     out->raster_group = pl.raster_group;
     out->grid = pl.grid;
     out->tiles = pl.units;

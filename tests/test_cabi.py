@@ -120,7 +120,7 @@ def test_bound_call_keeps_its_tensors_alive(lib):
     del X, W, R, Y
     gc.collect()
     assert all(r() is not None for r in refs)
-    assert len(f.tensors) == 6
+    assert len(f.tensors) == 7
     del f
     gc.collect()
     assert all(r() is None for r in refs)
