@@ -189,3 +189,37 @@ double kx_oracle_element(const uint16_t* X, const uint16_t* W, const uint16_t* b
     if (R) s += bf16_widen(R[m * N + n]);
     return s;
 }
+
+/*
+ * RMSNorm of rows of a BF16 matrix (the step that follows the output projection and
+ * first residual in the paper's decoder-layer case study, Appendix A, Algorithm 7: "run
+ * fused add+RMSNorm ..."; the paper prints no formula, so this is the textbook
+ * definition):
+ *
+ *     z[m,n] = h[m,n] / sqrt( (1/N) * sum_j h[m,j]^2 + eps ) * gamma[n]
+ *
+ * h and gamma are BF16 bit patterns widened exactly to double; the sum of squares runs
+ * over j in increasing order in double; the result is kept unrounded.
+ *   H [M,N], gamma [N], rows [nrows] (NULL = rows 0..nrows-1), out [nrows,N].
+ */
+int kx_oracle_rmsnorm_rows(const uint16_t* H, const uint16_t* gamma, double eps, const int64_t* rows,
+                           int64_t nrows, double* out, int64_t M, int64_t N) {
+    if (M < 0 || N <= 0 || nrows < 0 || !H || !gamma || !out) return -1;
+    for (int64_t i = 0; rows && i < nrows; ++i)
+        if (rows[i] < 0 || rows[i] >= M) return -1;
+    if (!rows && nrows > M) return -1;
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < nrows; ++i) {
+        const int64_t m = rows ? rows[i] : i;
+        double ss = 0.0;
+        for (int64_t j = 0; j < N; ++j) {
+            const double h = bf16_widen(H[m * N + j]);
+            ss += h * h;
+        }
+        const double inv = 1.0 / sqrt(ss / (double)N + eps);
+        for (int64_t j = 0; j < N; ++j)
+            out[i * N + j] = bf16_widen(H[m * N + j]) * inv * bf16_widen(gamma[j]);
+    }
+    return 0;
+}
+

@@ -33,6 +33,8 @@ def _load():
         lib.kx_oracle_round_bf16.restype = None
         lib.kx_oracle_widen_bf16.argtypes = [p, p, i64]
         lib.kx_oracle_widen_bf16.restype = None
+        lib.kx_oracle_rmsnorm_rows.argtypes = [p, p, ctypes.c_double, p, i64, p, i64, i64]
+        lib.kx_oracle_rmsnorm_rows.restype = ctypes.c_int
         lib.kx_oracle_max_threads.argtypes = []
         lib.kx_oracle_max_threads.restype = ctypes.c_int
         _lib = lib
@@ -116,3 +118,25 @@ def widen_bf16(bits: np.ndarray) -> np.ndarray:
     out = np.empty(bits.shape, dtype=np.float64)
     _load().kx_oracle_widen_bf16(_ptr(bits), _ptr(out), bits.size)
     return out
+
+
+def rmsnorm(H, gamma, eps: float, rows=None) -> np.ndarray:
+    """RMSNorm of rows of a BF16 matrix: z = h / sqrt(mean_j h_j^2 + eps) * gamma, float64,
+    unrounded (textbook definition; the step after the output projection in the paper's
+    decoder-layer case study, Appendix A, Algorithm 7).  H [M,N] and gamma [N] are uint16
+    BF16 bit patterns; `rows` selects rows (None = all)."""
+    lib = _load()
+    M, N = H.shape
+    H = _bits(H, (M, N), "H")
+    gamma = _bits(gamma, (N,), "gamma")
+    if rows is None:
+        rows_arr, nrows = None, M
+    else:
+        rows_arr = np.ascontiguousarray(rows, dtype=np.int64)
+        nrows = int(rows_arr.size)
+    out = np.empty((nrows, N), dtype=np.float64)
+    rc = lib.kx_oracle_rmsnorm_rows(_ptr(H), _ptr(gamma), float(eps), _ptr(rows_arr), nrows, _ptr(out), M, N)
+    if rc != 0:
+        raise RuntimeError(f"kx_oracle_rmsnorm_rows failed ({rc})")
+    return out
+
