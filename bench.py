@@ -392,6 +392,50 @@ def run_ours(args):
                   f"{w.flops/t/1e12:8.1f} TF {w.algorithmic_bytes/t/1e9:7.0f} GB/s  {r['bound']:6s} "
                   f"{r['frac']*100:5.1f}% of {peaks['source']}", file=sys.stderr, flush=True)
 
+    # ---- the step after the projection: RMSNorm of the new residual stream (rank 0, N = 1 only)
+    norm = []
+    if rank == 0 and world == 1 and not args.no_sweep:
+        lib = kx.load()
+        import ctypes
+        st = ctypes.c_void_p(int(torch.cuda.current_stream().cuda_stream) or None)
+        for (Mn, Nn) in [(4096, 4096), (8192, 8192), (16384, 4096), (512, 8192)]:
+            nbytes = 2.0 * Mn * Nn * 2 + 2.0 * Nn
+            ns = int(max(2, min(24, math.ceil(2.0 * L2_BYTES / nbytes))))
+            g = torch.Generator(device="cuda")
+            g.manual_seed(Mn + Nn)
+            gam = torch.randn(Nn, device="cuda", generator=g).bfloat16()
+            bufs = [(torch.randn(Mn, Nn, device="cuda", generator=g).bfloat16(),
+                     torch.empty(Mn, Nn, dtype=torch.bfloat16, device="cuda")) for _ in range(ns)]
+            calls = []
+            for (Hn, Zn) in bufs:
+                a = (ctypes.c_void_p(Hn.data_ptr()), ctypes.c_void_p(gam.data_ptr()), ctypes.c_float(1e-6),
+                     ctypes.c_void_p(Zn.data_ptr()), ctypes.c_int64(Mn), ctypes.c_int64(Nn), st)
+                calls.append(lambda a=a: lib.kx_rmsnorm(*a))
+            wln = inputs.Workload(f"rmsnorm_{Mn}x{Nn}", Mn, Nn, 8, 0, False, False)
+            t, tbest, iters = time_shape(torch, kx, wln, calls)
+            norm.append({"name": wln.name, "M": Mn, "N": Nn, "us": t * 1e6, "us_best": tbest * 1e6,
+                         "gbs": nbytes / t / 1e9, "bound": "hbm", "frac": nbytes / t / 1e9 / peaks["hbm_gbs"],
+                         "algorithmic_bytes": nbytes, "operand_sets": ns})
+            print(f"[bench] {wln.name:>18s} {t*1e6:9.1f} us (best {tbest*1e6:7.1f}) {nbytes/t/1e9:7.0f} GB/s  hbm    "
+                  f"{nbytes/t/1e9/peaks['hbm_gbs']*100:5.1f}% of {peaks['source']}", file=sys.stderr, flush=True)
+            del bufs, calls
+            torch.cuda.empty_cache()
+        # chained: projection + RMSNorm on the headline workload, against the projection alone
+        gam = torch.randn(wl.N, device="cuda").bfloat16()
+        Xs, Ws, bs, Rs, Ys = sets[0].tensors[:5]
+        Zs = torch.empty_like(Ys)
+        a = (ctypes.c_void_p(Xs.data_ptr()), ctypes.c_void_p(Ws.data_ptr()),
+             ctypes.c_void_p(bs.data_ptr() if bs is not None else None), ctypes.c_void_p(Rs.data_ptr()),
+             ctypes.c_void_p(gam.data_ptr()), ctypes.c_float(1e-6), ctypes.c_void_p(Ys.data_ptr()),
+             ctypes.c_void_p(Zs.data_ptr()), ctypes.c_int64(wl.M), ctypes.c_int64(wl.N), ctypes.c_int64(wl.K), st)
+        if wl.has_residual:
+            tc, tcb, _ = time_shape(torch, kx, wl, [lambda: lib.kx_outproj_residual_rmsnorm(*a)])
+            tp, tpb, _ = time_shape(torch, kx, wl, [sets[0]])
+            norm.append({"name": f"{headline}+rmsnorm", "us": tc * 1e6, "projection_alone_us": tp * 1e6,
+                         "rmsnorm_added_us": (tc - tp) * 1e6, "note": "same operand set for both (warm L2)"})
+            print(f"[bench] {headline}+rmsnorm: {tc*1e6:.1f} us chained vs {tp*1e6:.1f} us projection alone",
+                  file=sys.stderr, flush=True)
+
     # ---- the oracle on the host cores, bounded sample (rank 0, N = 1 only)
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -424,6 +468,7 @@ def run_ours(args):
             "gpu_launches_all_legs": (max(3, args.warmup) + args.steps) * info.launches + launches_e2e,
             "clocks": clk.summary(),
             "shapes": shapes,
+            "rmsnorm": norm,
             "sweep_geomean": {"tflops": geo([s["tflops"] for s in sweep]), "roofline_frac": geo([s["frac"] for s in sweep]),
                               "roofline_frac_nominal": geo([s["frac_nominal"] for s in sweep])},
             "paper_context": "766 TFLOP/s BF16 on one 4096x4096 GEMM, H100 SXM (Section 4.1): other hardware, context only",

@@ -209,6 +209,31 @@ int kx_outproj_residual_noalloc(const void* X, const void* W, const void* bias_o
                                 const void* R_or_null, void* Y, int64_t M, int64_t N, int64_t K,
                                 void* stream);
 
+/*
+ * Z = RMSNorm(H) * gamma, row by row:  z[m,n] = h[m,n] / sqrt(mean_j h[m,j]^2 + eps) * gamma[n].
+ * The step that follows the output projection and first residual in the paper's
+ * decoder-layer case study (Appendix A, Algorithm 7, "run fused add+RMSNorm ..."); the paper
+ * prints no formula, so this is the textbook definition, with the statistics taken from the
+ * BF16 values of H, the arithmetic in FP32 and one rounding to BF16.
+ *   H [M,N], gamma [N], Z [M,N]: device, BF16, 16-byte aligned; eps >= 0.
+ *   N % 8 == 0 and N <= 32768 (a row is held in one CTA's registers); Z may equal H.
+ * One memory-bound kernel (each row read once, written once) on `stream`.
+ */
+int kx_rmsnorm(const void* H, const void* gamma, float eps, void* Z, int64_t M, int64_t N, void* stream);
+
+/*
+ * H = X W^T (+ bias) + R, then Z = RMSNorm(H) * gamma: both outputs of the attention block's
+ * tail (the new residual stream H and the normalised input Z of the MLP).  Algorithm 3 followed
+ * by the RMSNorm step of Algorithm 7.  Two kernels on `stream`, the second launched with
+ * programmatic stream serialization so that its prologue overlaps the first one's tail; for
+ * outputs up to the size of the L2 cache the second kernel reads H from L2.
+ * Arguments as for kx_outproj_residual and kx_rmsnorm.  H may equal R (in place); Z must not
+ * overlap any other tensor.
+ */
+int kx_outproj_residual_rmsnorm(const void* X, const void* W, const void* bias_or_null, const void* R,
+                                const void* gamma, float eps, void* H, void* Z,
+                                int64_t M, int64_t N, int64_t K, void* stream);
+
 /* Fills `out` with the plan the library would use for this shape on the current
  * device (has_residual / has_bias as 0 or 1).  No work is enqueued. */
 int kx_plan_query(int64_t M, int64_t N, int64_t K, int has_bias, int has_residual,

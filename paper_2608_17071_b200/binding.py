@@ -23,7 +23,8 @@ KX_PATH_AUTO, KX_PATH_TILE, KX_PATH_SWAP = 0, 1, 2
 
 EXPORTS = (
     "kx_init", "kx_shutdown", "kx_outproj_residual", "kx_gemm_bf16", "kx_outproj_residual_ex",
-    "kx_outproj_residual_host", "kx_outproj_residual_noalloc", "kx_plan_query", "kx_last_device_status", "kx_status_string",
+    "kx_outproj_residual_host", "kx_outproj_residual_noalloc", "kx_rmsnorm", "kx_outproj_residual_rmsnorm",
+    "kx_plan_query", "kx_last_device_status", "kx_status_string",
     "kx_version",
 )
 
@@ -74,6 +75,8 @@ def load():
     lib.kx_outproj_residual_ex.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, vp, ctypes.POINTER(PlanOverride)]
     lib.kx_outproj_residual_host.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, vp]
     lib.kx_outproj_residual_noalloc.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, vp]
+    lib.kx_rmsnorm.argtypes = [vp, vp, ctypes.c_float, vp, i64, i64, vp]
+    lib.kx_outproj_residual_rmsnorm.argtypes = [vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, i64, i64, i64, vp]
     lib.kx_plan_query.argtypes = [i64, i64, i64, ci, ci, ctypes.POINTER(PlanOverride), ctypes.POINTER(PlanInfo)]
     lib.kx_last_device_status.argtypes = [vp, ctypes.POINTER(ci), ctypes.POINTER(ci)]
     lib.kx_status_string.argtypes = [ci]
@@ -195,6 +198,33 @@ def kx_outproj_residual_noalloc(X, W, bias, R, Y, stream=None, M=None, N=None, K
                                             _stream(stream))
     if check and rc != KX_OK:
         raise KxError(rc, "kx_outproj_residual_noalloc")
+    return rc
+
+
+def kx_rmsnorm(H, gamma, eps: float, Z, stream=None, M=None, N=None, check=True) -> int:
+    """Z = RMSNorm(H) * gamma over the rows of H (BF16, FP32 arithmetic); Z may be H."""
+    if M is None:
+        M, N = H.shape
+        _check_bf16("H", H, (M, N)); _check_bf16("gamma", gamma, (N,)); _check_bf16("Z", Z, (M, N))
+    rc = load().kx_rmsnorm(_addr(H), _addr(gamma), float(eps), _addr(Z), M, N, _stream(stream))
+    if check and rc != KX_OK:
+        raise KxError(rc, "kx_rmsnorm")
+    return rc
+
+
+def kx_outproj_residual_rmsnorm(X, W, bias, R, gamma, eps: float, H, Z, stream=None, M=None, N=None, K=None,
+                                check=True) -> int:
+    """H = X W^T (+ bias) + R and Z = RMSNorm(H) * gamma, two kernels on one stream."""
+    if M is None:
+        M, K = X.shape
+        N = W.shape[0]
+        _check_bf16("X", X, (M, K)); _check_bf16("W", W, (N, K)); _check_bf16("bias", bias, (N,))
+        _check_bf16("R", R, (M, N)); _check_bf16("gamma", gamma, (N,))
+        _check_bf16("H", H, (M, N)); _check_bf16("Z", Z, (M, N))
+    rc = load().kx_outproj_residual_rmsnorm(_addr(X), _addr(W), _addr(bias), _addr(R), _addr(gamma), float(eps),
+                                            _addr(H), _addr(Z), M, N, K, _stream(stream))
+    if check and rc != KX_OK:
+        raise KxError(rc, "kx_outproj_residual_rmsnorm")
     return rc
 
 

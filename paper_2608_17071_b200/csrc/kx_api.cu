@@ -835,6 +835,90 @@ int kx_outproj_residual_host(const void* Xh, const void* Wh, const void* bh, con
     return KX_OK;
 }
 
+// ---------------------------------------------------------------- RMSNorm after the projection
+namespace {
+int launch_rmsnorm(const void* H, const void* gamma, float eps, void* Z, long long M, long long N,
+                   cudaStream_t stream, int sm_count) {
+    cudaLaunchConfig_t cfg;
+    std::memset(&cfg, 0, sizeof cfg);
+    // smallest instantiation whose threads cover a row; shorter rows leave room for more CTAs per SM
+    const long long nvec = N / 8;
+    const void* fn = nullptr;
+    int per_sm = 8;
+    if (nvec <= 1 * kNormThreads) { fn = reinterpret_cast<const void*>(&kx_rmsnorm_kernel<1>); }
+    else if (nvec <= 2 * kNormThreads) { fn = reinterpret_cast<const void*>(&kx_rmsnorm_kernel<2>); }
+    else if (nvec <= 4 * kNormThreads) { fn = reinterpret_cast<const void*>(&kx_rmsnorm_kernel<4>); per_sm = 6; }
+    else if (nvec <= 8 * kNormThreads) { fn = reinterpret_cast<const void*>(&kx_rmsnorm_kernel<8>); per_sm = 4; }
+    else { fn = reinterpret_cast<const void*>(&kx_rmsnorm_kernel<kNormVecs>); per_sm = 2; }
+    cfg.gridDim = dim3(static_cast<unsigned>(std::min<long long>(M, static_cast<long long>(sm_count) * per_sm)), 1, 1);
+    cfg.blockDim = dim3(kNormThreads, 1, 1);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const uint16_t* h = static_cast<const uint16_t*>(H);
+    const uint16_t* g = static_cast<const uint16_t*>(gamma);
+    uint16_t* z = static_cast<uint16_t*>(Z);
+    int n = static_cast<int>(N);
+    void* args[] = {&h, &g, &z, &M, &n, &eps};
+    if (cudaLaunchKernelExC(&cfg, fn, args) != cudaSuccess) {
+        cudaGetLastError();
+        return KX_ERR_CUDA;
+    }
+    return KX_OK;
+}
+
+int validate_rmsnorm(const void* H, const void* gamma, const void* Z, long long M, long long N, float eps) {
+    if (M < 0 || N < 0 || M > 0x7FFFFFFFll / 2) return KX_ERR_SHAPE;
+    if (M == 0 || N == 0) return KX_OK;
+    if ((N % 8) != 0 || N > 8ll * kNormThreads * kNormVecs) return KX_ERR_SHAPE;
+    if (!(eps >= 0.0f)) return KX_ERR_SHAPE;
+    if (!H || !gamma || !Z) return KX_ERR_NULL;
+    if (!aligned16(H) || !aligned16(gamma) || !aligned16(Z)) return KX_ERR_ALIGN;
+    const size_t hb = static_cast<size_t>(M) * N * 2;
+    if (overlaps(Z, hb, gamma, static_cast<size_t>(N) * 2)) return KX_ERR_OVERLAP;
+    if (Z != H && overlaps(Z, hb, H, hb)) return KX_ERR_OVERLAP;
+    return KX_OK;
+}
+}  // namespace
+
+int kx_rmsnorm(const void* H, const void* gamma, float eps, void* Z, int64_t M, int64_t N, void* stream) {
+    int rc = validate_rmsnorm(H, gamma, Z, M, N, eps);
+    if (rc != KX_OK) return rc;
+    if (M == 0 || N == 0) return KX_OK;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return KX_ERR_CUDA;
+    DeviceCtx* ctx = nullptr;
+    rc = ensure_device(dev, &ctx);
+    if (rc != KX_OK) return rc;
+    return launch_rmsnorm(H, gamma, eps, Z, M, N, static_cast<cudaStream_t>(stream), ctx->sm_count);
+}
+
+int kx_outproj_residual_rmsnorm(const void* X, const void* W, const void* bias, const void* R,
+                                const void* gamma, float eps, void* H, void* Z, int64_t M, int64_t N,
+                                int64_t K, void* stream) {
+    int rc = validate(X, W, bias, R, H, M, N, K, true);
+    if (rc != KX_OK) return rc;
+    rc = validate_rmsnorm(H, gamma, Z, M, N, eps);
+    if (rc != KX_OK) return rc;
+    if (M == 0 || N == 0) return KX_OK;
+    const size_t zb = static_cast<size_t>(M) * N * 2;
+    if (Z == H || overlaps(Z, zb, X, static_cast<size_t>(M) * K * 2) ||
+        overlaps(Z, zb, W, static_cast<size_t>(N) * K * 2) || overlaps(Z, zb, bias, static_cast<size_t>(N) * 2) ||
+        overlaps(Z, zb, R, zb) || overlaps(H, zb, gamma, static_cast<size_t>(N) * 2))
+        return KX_ERR_OVERLAP;
+    rc = run(X, W, bias, R, H, M, N, K, stream, nullptr, true);
+    if (rc != KX_OK) return rc;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return KX_ERR_CUDA;
+    DeviceCtx* ctx = nullptr;
+    rc = ensure_device(dev, &ctx);
+    if (rc != KX_OK) return rc;
+    return launch_rmsnorm(H, gamma, eps, Z, M, N, static_cast<cudaStream_t>(stream), ctx->sm_count);
+}
+
 // ---------------------------------------------------------------- no-allocation entry
 namespace {
 struct NoAllocCtx {

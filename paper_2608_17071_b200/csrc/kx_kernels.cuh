@@ -1070,4 +1070,78 @@ __global__ void kx_k0_kernel(const uint16_t* __restrict__ bias, const uint16_t* 
     }
 }
 
+// ===========================================================================
+// kx_rmsnorm_kernel
+// ===========================================================================
+// z[m,n] = h[m,n] * rsqrt(mean_j h[m,j]^2 + eps) * gamma[n] on BF16 rows (the step that follows
+// the output projection and first residual in the decoder layer, Appendix A, Algorithm 7).
+// One CTA per row, persistent over rows.  A row is read from global memory exactly once
+// (16-byte loads, kept in registers), squared and summed in FP32 (fixed order: per thread,
+// then a warp tree, then the warps in order -> deterministic), normalised, scaled and
+// rounded to BF16 once.  Because the whole row is in registers before anything is stored,
+// Z may alias H.  HBM-bound: 2 * N * 2 bytes per row.
+constexpr int kNormThreads = 256;
+constexpr int kNormVecs = 16;                              // at most 16 16-byte vectors per thread: N <= 32768
+
+// NV = 16-byte vectors per thread (N <= NV * 2048): the register footprint, and with it the
+// number of rows in flight per SM, follows the row length.
+template <int NV>
+__global__ void __launch_bounds__(kNormThreads)
+kx_rmsnorm_kernel(const uint16_t* __restrict__ H, const uint16_t* __restrict__ gamma, uint16_t* Z,
+                  long long M, int N, float eps) {
+    __shared__ float s_part[kNormThreads / 32];
+    __shared__ float s_inv;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int nvec = N / 8;
+    pdl_wait_prior();            // H is usually written by the kernel just before this one
+    pdl_launch_dependents();
+    for (long long m = blockIdx.x; m < M; m += gridDim.x) {
+        const uint4* row = reinterpret_cast<const uint4*>(H + m * N);
+        uint4 v[NV];
+        float ss = 0.f;
+#pragma unroll
+        for (int i = 0; i < NV; ++i) {
+            const int idx = tid + i * kNormThreads;
+            if (idx < nvec) {
+                v[i] = row[idx];
+                const uint32_t w4[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const float a = bf16_lo(w4[k]), b = bf16_hi(w4[k]);
+                    ss += a * a;
+                    ss += b * b;
+                }
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+        if (lane == 0) s_part[warp] = ss;
+        __syncthreads();
+        if (tid == 0) {
+            float t = 0.f;
+#pragma unroll
+            for (int w = 0; w < kNormThreads / 32; ++w) t += s_part[w];
+            s_inv = rsqrtf(t / static_cast<float>(N) + eps);
+        }
+        __syncthreads();
+        const float inv = s_inv;
+        uint4* zrow = reinterpret_cast<uint4*>(Z + m * N);
+#pragma unroll
+        for (int i = 0; i < NV; ++i) {
+            const int idx = tid + i * kNormThreads;
+            if (idx < nvec) {
+                const uint4 g = __ldg(reinterpret_cast<const uint4*>(gamma) + idx);
+                const uint32_t h4[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
+                const uint32_t g4[4] = {g.x, g.y, g.z, g.w};
+                uint32_t o4[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    o4[k] = pack_bf16x2(bf16_lo(h4[k]) * inv * bf16_lo(g4[k]), bf16_hi(h4[k]) * inv * bf16_hi(g4[k]));
+                zrow[idx] = make_uint4(o4[0], o4[1], o4[2], o4[3]);
+            }
+        }
+        __syncthreads();         // s_part / s_inv are reused by the next row
+    }
+}
+
 }  // namespace kx

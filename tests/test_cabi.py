@@ -75,6 +75,27 @@ def test_argument_validation_needs_no_device(lib):
     assert lib.kx_outproj_residual_host(X, W, None, None, None, 4, 8, 8, None) == kx.KX_ERR_NULL
 
 
+def test_rmsnorm_argument_validation_needs_no_device(lib):
+    A, MB = 0x10000, 1 << 20
+    H, G, Z = A, A + 64 * MB, A + 128 * MB
+    f = lib.kx_rmsnorm
+    assert f(H, G, 1e-6, Z, 4, 12, None) == kx.KX_ERR_SHAPE          # N % 8
+    assert f(H, G, 1e-6, Z, 4, 32768 + 8, None) == kx.KX_ERR_SHAPE   # row too long for one CTA
+    assert f(H, G, -1.0, Z, 4, 8, None) == kx.KX_ERR_SHAPE           # eps < 0
+    assert f(H, G, float("nan"), Z, 4, 8, None) == kx.KX_ERR_SHAPE
+    assert f(None, G, 1e-6, Z, 4, 8, None) == kx.KX_ERR_NULL
+    assert f(H, G + 2, 1e-6, Z, 4, 8, None) == kx.KX_ERR_ALIGN
+    assert f(H, G, 1e-6, H + 16, 4, 8, None) == kx.KX_ERR_OVERLAP    # partial overlap with H
+    assert f(H, G, 1e-6, G, 4, 8, None) == kx.KX_ERR_OVERLAP
+    assert f(None, None, 1e-6, None, 0, 8, None) == kx.KX_OK
+    g = lib.kx_outproj_residual_rmsnorm
+    X, W, R = A + 192 * MB, A + 256 * MB, A + 320 * MB
+    assert g(X, W, None, R, G, 1e-6, H, H, 4, 8, 8, None) == kx.KX_ERR_OVERLAP   # Z == H
+    assert g(X, W, None, R, G, 1e-6, H, X, 4, 8, 8, None) == kx.KX_ERR_OVERLAP
+    assert g(X, W, None, None, G, 1e-6, H, Z, 4, 8, 8, None) == kx.KX_ERR_NULL   # residual required
+    assert g(X, W, None, R, G, 1e-6, H, Z, 4, 8, 12, None) == kx.KX_ERR_SHAPE
+
+
 def test_binding_rejects_wrong_tensors():
     import torch
     X = torch.zeros(4, 8, dtype=torch.float32)
