@@ -4,5 +4,5 @@ Only tests, the smoke check and the benchmark's CPU-baseline leg import this
 package.  The product (the CUDA library and its Python binding) never does.
 """
 from .oracle import (  # noqa: F401
-    outproj, outproj_rows, element, round_bf16, widen_bf16, max_threads, rmsnorm,
+    outproj, outproj_rows, element, round_bf16, widen_bf16, max_threads, rmsnorm, swiglu,
 )

@@ -223,3 +223,41 @@ int kx_oracle_rmsnorm_rows(const uint16_t* H, const uint16_t* gamma, double eps,
     return 0;
 }
 
+/*
+ * Gate/up projections with the SwiGLU product (the MLP's first half in the paper's
+ * decoder-layer case study, Appendix A, Algorithm 7: "compute BF16 gate/up projections
+ * and a ... SiLU-multiply", fused there as a "SwiGLU epilogue"):
+ *
+ *     g[m,i] = sum_k X[m,k] * Wg[i,k],   u[m,i] = sum_k X[m,k] * Wu[i,k]
+ *     z[m,i] = silu(g[m,i]) * u[m,i],    silu(t) = t / (1 + exp(-t))
+ *
+ * Both sums run over k in increasing order in double (products of BF16 values are exact);
+ * the result is kept unrounded.  X [M,K], Wg and Wu [I,K] BF16 bits; rows [nrows] or NULL;
+ * out [nrows,I]; gate_out / up_out [nrows,I] optional (NULL to skip).
+ */
+int kx_oracle_swiglu_rows(const uint16_t* X, const uint16_t* Wg, const uint16_t* Wu, const int64_t* rows,
+                          int64_t nrows, double* out, double* gate_out, double* up_out,
+                          int64_t M, int64_t I, int64_t K) {
+    if (M < 0 || I < 0 || K < 0 || nrows < 0 || !out) return -1;
+    if (K > 0 && (!X || !Wg || !Wu)) return -1;
+    for (int64_t r = 0; rows && r < nrows; ++r)
+        if (rows[r] < 0 || rows[r] >= M) return -1;
+    if (!rows && nrows > M) return -1;
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int64_t r = 0; r < nrows; ++r) {
+        for (int64_t i = 0; i < I; ++i) {
+            const int64_t m = rows ? rows[r] : r;
+            double g = 0.0, u = 0.0;
+            for (int64_t k = 0; k < K; ++k) {
+                const double x = bf16_widen(X[m * K + k]);
+                g += x * bf16_widen(Wg[i * K + k]);
+                u += x * bf16_widen(Wu[i * K + k]);
+            }
+            out[r * I + i] = g / (1.0 + exp(-g)) * u;
+            if (gate_out) gate_out[r * I + i] = g;
+            if (up_out) up_out[r * I + i] = u;
+        }
+    }
+    return 0;
+}
+

@@ -35,6 +35,8 @@ def _load():
         lib.kx_oracle_widen_bf16.restype = None
         lib.kx_oracle_rmsnorm_rows.argtypes = [p, p, ctypes.c_double, p, i64, p, i64, i64]
         lib.kx_oracle_rmsnorm_rows.restype = ctypes.c_int
+        lib.kx_oracle_swiglu_rows.argtypes = [p, p, p, p, i64, p, p, p, i64, i64, i64]
+        lib.kx_oracle_swiglu_rows.restype = ctypes.c_int
         lib.kx_oracle_max_threads.argtypes = []
         lib.kx_oracle_max_threads.restype = ctypes.c_int
         _lib = lib
@@ -139,4 +141,29 @@ def rmsnorm(H, gamma, eps: float, rows=None) -> np.ndarray:
     if rc != 0:
         raise RuntimeError(f"kx_oracle_rmsnorm_rows failed ({rc})")
     return out
+
+
+def swiglu(X, Wg, Wu, rows=None, want_parts: bool = False):
+    """z = silu(X Wg^T) * (X Wu^T) in float64, unrounded (gate/up projections with the SwiGLU
+    product, Appendix A, Algorithm 7 of the paper).  X [M,K], Wg / Wu [I,K] uint16 BF16 bits.
+    `rows` selects rows of X; with `want_parts` also returns the gate and up pre-activations."""
+    lib = _load()
+    M, K = X.shape
+    I = Wg.shape[0]
+    X = _bits(X, (M, K), "X")
+    Wg = _bits(Wg, (I, K), "Wg")
+    Wu = _bits(Wu, (I, K), "Wu")
+    if rows is None:
+        rows_arr, nrows = None, M
+    else:
+        rows_arr = np.ascontiguousarray(rows, dtype=np.int64)
+        nrows = int(rows_arr.size)
+    out = np.empty((nrows, I), dtype=np.float64)
+    g = np.empty((nrows, I), dtype=np.float64) if want_parts else None
+    u = np.empty((nrows, I), dtype=np.float64) if want_parts else None
+    rc = lib.kx_oracle_swiglu_rows(_ptr(X), _ptr(Wg), _ptr(Wu), _ptr(rows_arr), nrows, _ptr(out), _ptr(g), _ptr(u),
+                                   M, I, K)
+    if rc != 0:
+        raise RuntimeError(f"kx_oracle_swiglu_rows failed ({rc})")
+    return (out, g, u) if want_parts else out
 
