@@ -436,6 +436,39 @@ def run_ours(args):
             print(f"[bench] {headline}+rmsnorm: {tc*1e6:.1f} us chained vs {tp*1e6:.1f} us projection alone",
                   file=sys.stderr, flush=True)
 
+    # ---- gate/up projections with the fused SwiGLU epilogue (rank 0, N = 1 only)
+    swiglu = []
+    if rank == 0 and world == 1 and not args.no_sweep:
+        lib = kx.load()
+        import ctypes
+        st = ctypes.c_void_p(int(torch.cuda.current_stream().cuda_stream) or None)
+        for (Ms, Is, Ks) in [(16384, 14336, 4096), (4096, 14336, 4096), (512, 14336, 4096)]:
+            fl = 4.0 * Ms * Is * Ks
+            nbytes = 2.0 * (Ms * Ks + 2 * Is * Ks + Ms * Is)
+            ns = int(max(2, min(8, math.ceil(2.0 * L2_BYTES / nbytes))))
+            g = torch.Generator(device="cuda")
+            g.manual_seed(Ms + Is)
+            keep, calls = [], []
+            for _ in range(ns):
+                Xs = torch.randn(Ms, Ks, device="cuda", generator=g).bfloat16()
+                Wg = (torch.randn(Is, Ks, device="cuda", generator=g) / math.sqrt(Ks)).bfloat16()
+                Wu = (torch.randn(Is, Ks, device="cuda", generator=g) / math.sqrt(Ks)).bfloat16()
+                Zs = torch.empty(Ms, Is, dtype=torch.bfloat16, device="cuda")
+                keep.append((Xs, Wg, Wu, Zs))
+                a = (ctypes.c_void_p(Xs.data_ptr()), ctypes.c_void_p(Wg.data_ptr()), ctypes.c_void_p(Wu.data_ptr()),
+                     ctypes.c_void_p(Zs.data_ptr()), ctypes.c_int64(Ms), ctypes.c_int64(Is), ctypes.c_int64(Ks), st)
+                calls.append(lambda a=a: lib.kx_gate_up_swiglu(*a))
+            wls = inputs.Workload(f"swiglu_M{Ms}_I{Is}_K{Ks}", Ms, 2 * Is, Ks, 0, False, False)
+            t, tbest, iters = time_shape(torch, kx, wls, calls)
+            t_tensor = fl / (peaks["bf16_tflops"] * 1e12)
+            swiglu.append({"name": wls.name, "M": Ms, "I": Is, "K": Ks, "us": t * 1e6, "us_best": tbest * 1e6,
+                           "tflops": fl / t / 1e12, "gbs": nbytes / t / 1e9, "bound": "tensor",
+                           "frac": t_tensor / t, "frac_nominal": fl / t / 1e12 / 2250.0, "operand_sets": ns})
+            print(f"[bench] {wls.name:>26s} {t*1e6:9.1f} us (best {tbest*1e6:7.1f}) {fl/t/1e12:8.1f} TF  tensor "
+                  f"{t_tensor/t*100:5.1f}% of {peaks['source']}", file=sys.stderr, flush=True)
+            del keep, calls
+            torch.cuda.empty_cache()
+
     # ---- the oracle on the host cores, bounded sample (rank 0, N = 1 only)
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -469,6 +502,7 @@ def run_ours(args):
             "clocks": clk.summary(),
             "shapes": shapes,
             "rmsnorm": norm,
+            "swiglu": swiglu,
             "sweep_geomean": {"tflops": geo([s["tflops"] for s in sweep]), "roofline_frac": geo([s["frac"] for s in sweep]),
                               "roofline_frac_nominal": geo([s["frac_nominal"] for s in sweep])},
             "paper_context": "766 TFLOP/s BF16 on one 4096x4096 GEMM, H100 SXM (Section 4.1): other hardware, context only",

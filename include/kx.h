@@ -234,6 +234,20 @@ int kx_outproj_residual_rmsnorm(const void* X, const void* W, const void* bias_o
                                 const void* gamma, float eps, void* H, void* Z,
                                 int64_t M, int64_t N, int64_t K, void* stream);
 
+/*
+ * Z[M,I] = silu(X Wg^T) * (X Wu^T): the gate and up projections of the MLP with the SwiGLU
+ * product fused into the GEMM epilogue (the paper's decoder-layer case study, Appendix A,
+ * Algorithm 7: "compute ... gate/up projections" with a "SwiGLU epilogue"; silu(t) = t / (1 + e^-t)).
+ *   X [M,K], Wg [I,K], Wu [I,K], Z [M,I]: device, BF16 row-major, 16-byte aligned;
+ *   I % 8 == 0, K % 8 == 0; Z must not overlap an input.  FP32 accumulation, activation and
+ *   product in FP32, one rounding to BF16.
+ * One launch of the large-M tile kernel: each tile accumulates 128 gate and the matching 128 up
+ * columns side by side in tensor memory (in a CTA pair one CTA streams Wg, the other Wu), so
+ * neither pre-activation ever leaves the chip.  FLOPs = 4 M I K.
+ */
+int kx_gate_up_swiglu(const void* X, const void* Wg, const void* Wu, void* Z,
+                      int64_t M, int64_t I, int64_t K, void* stream);
+
 /* Fills `out` with the plan the library would use for this shape on the current
  * device (has_residual / has_bias as 0 or 1).  No work is enqueued. */
 int kx_plan_query(int64_t M, int64_t N, int64_t K, int has_bias, int has_residual,

@@ -24,6 +24,7 @@ KX_PATH_AUTO, KX_PATH_TILE, KX_PATH_SWAP = 0, 1, 2
 EXPORTS = (
     "kx_init", "kx_shutdown", "kx_outproj_residual", "kx_gemm_bf16", "kx_outproj_residual_ex",
     "kx_outproj_residual_host", "kx_outproj_residual_noalloc", "kx_rmsnorm", "kx_outproj_residual_rmsnorm",
+    "kx_gate_up_swiglu",
     "kx_plan_query", "kx_last_device_status", "kx_status_string",
     "kx_version",
 )
@@ -76,6 +77,7 @@ def load():
     lib.kx_outproj_residual_host.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, vp]
     lib.kx_outproj_residual_noalloc.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, vp]
     lib.kx_rmsnorm.argtypes = [vp, vp, ctypes.c_float, vp, i64, i64, vp]
+    lib.kx_gate_up_swiglu.argtypes = [vp, vp, vp, vp, i64, i64, i64, vp]
     lib.kx_outproj_residual_rmsnorm.argtypes = [vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, i64, i64, i64, vp]
     lib.kx_plan_query.argtypes = [i64, i64, i64, ci, ci, ctypes.POINTER(PlanOverride), ctypes.POINTER(PlanInfo)]
     lib.kx_last_device_status.argtypes = [vp, ctypes.POINTER(ci), ctypes.POINTER(ci)]
@@ -198,6 +200,19 @@ def kx_outproj_residual_noalloc(X, W, bias, R, Y, stream=None, M=None, N=None, K
                                             _stream(stream))
     if check and rc != KX_OK:
         raise KxError(rc, "kx_outproj_residual_noalloc")
+    return rc
+
+
+def kx_gate_up_swiglu(X, Wg, Wu, Z, stream=None, M=None, I=None, K=None, check=True) -> int:
+    """Z = silu(X Wg^T) * (X Wu^T) with the SwiGLU product fused into the GEMM epilogue."""
+    if M is None:
+        M, K = X.shape
+        I = Wg.shape[0]
+        _check_bf16("X", X, (M, K)); _check_bf16("Wg", Wg, (I, K)); _check_bf16("Wu", Wu, (I, K))
+        _check_bf16("Z", Z, (M, I))
+    rc = load().kx_gate_up_swiglu(_addr(X), _addr(Wg), _addr(Wu), _addr(Z), M, I, K, _stream(stream))
+    if check and rc != KX_OK:
+        raise KxError(rc, "kx_gate_up_swiglu")
     return rc
 
 

@@ -603,6 +603,7 @@ int run(const void* X, const void* W, const void* bias, const void* R, void* Y, 
         p.has_bias = bias ? 1 : 0;
         p.has_r = R ? 1 : 0;
         p.drop_kblocks = drop;
+        p.swiglu = 0;
         p.sk_tile0 = pl.sk_tile0;
         p.narrow_tile0 = pl.narrow_tile0;
         p.spin_limit_ns = spin_ns;
@@ -829,6 +830,91 @@ int kx_outproj_residual_host(const void* Xh, const void* Wh, const void* bh, con
     if (rc != KX_OK) return rc;
     if (cudaMemcpyAsync(Yh, Yd, static_cast<size_t>(M) * N * 2, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
         cudaStreamSynchronize(stream) != cudaSuccess) {
+        cudaGetLastError();
+        return KX_ERR_CUDA;
+    }
+    return KX_OK;
+}
+
+// ---------------------------------------------------------------- gate/up with SwiGLU epilogue
+int kx_gate_up_swiglu(const void* X, const void* Wg, const void* Wu, void* Z, int64_t M, int64_t I, int64_t K,
+                      void* stream_v) {
+    if (M < 0 || I < 0 || K < 0) return KX_ERR_SHAPE;
+    if (M > 0x7FFFFFFFll / 2 || I > 0x7FFFFFFFll / 4 || K > 0x7FFFFFFFll / 2) return KX_ERR_SHAPE;
+    if (M == 0 || I == 0) return KX_OK;
+    if ((I % 8) != 0 || (K % 8) != 0) return KX_ERR_SHAPE;
+    if (!Z || (K > 0 && (!X || !Wg || !Wu))) return KX_ERR_NULL;
+    if (!aligned16(Z) || (K > 0 && (!aligned16(X) || !aligned16(Wg) || !aligned16(Wu)))) return KX_ERR_ALIGN;
+    const size_t zb = static_cast<size_t>(M) * I * 2, wb = static_cast<size_t>(I) * K * 2;
+    if (overlaps(Z, zb, X, static_cast<size_t>(M) * K * 2) || overlaps(Z, zb, Wg, wb) || overlaps(Z, zb, Wu, wb))
+        return KX_ERR_OVERLAP;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return KX_ERR_CUDA;
+    DeviceCtx* ctx = nullptr;
+    int rc = ensure_device(dev, &ctx);
+    if (rc != KX_OK) return rc;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    if (K == 0) {   // empty sums: silu(0) * 0 = 0
+        const long long total = M * I;
+        const int blocks = static_cast<int>(std::min<long long>((total + 255) / 256, ctx->sm_count * 8));
+        kx_k0_kernel<<<blocks, 256, 0, stream>>>(nullptr, nullptr, static_cast<uint16_t*>(Z), M, I);
+        return cudaGetLastError() == cudaSuccess ? KX_OK : KX_ERR_CUDA;
+    }
+    // one tile = 128 (x2 for a pair) rows by 128 gate + 128 up accumulator columns = 128 output columns
+    kx_plan_override ov;
+    std::memset(&ov, 0, sizeof ov);
+    ov.path = KX_PATH_TILE;
+    ov.block_n = 256;
+    ov.stream_k = 1;
+    ov.narrow_tail = 1;
+    ov.no_table = 1;
+    Plan pl;
+    rc = make_plan_from(M, 2 * I, K, &ov, ctx->sm_count, &pl);
+    if (rc != KX_OK) return rc;
+    CUtensorMap tmA, tmG, tmU, tmZ;
+    if ((rc = get_tmap(X, M, K, 128, &tmA)) != KX_OK) return rc;
+    if ((rc = get_tmap(Wg, I, K, 128, &tmG)) != KX_OK) return rc;
+    if ((rc = get_tmap(Wu, I, K, 128, &tmU)) != KX_OK) return rc;
+    if ((rc = get_tmap(Z, M, I, 32, &tmZ)) != KX_OK) return rc;
+    TileParams p;
+    std::memset(&p, 0, sizeof p);
+    p.M = static_cast<int>(M);
+    p.N = static_cast<int>(I);
+    p.K = static_cast<int>(K);
+    p.tiles_m = pl.tiles_m;
+    p.tiles_n = pl.tiles_n;
+    p.num_tiles = pl.units;
+    p.raster_group = pl.raster_group;
+    p.swiglu = 1;
+    p.sk_tile0 = pl.units;
+    p.narrow_tile0 = pl.units;
+    p.spin_limit_ns = 2000000000ull;
+    p.status = ctx->status;
+    p.ws = ctx->ws;
+    p.counters = ctx->counters;
+    cudaLaunchConfig_t cfg;
+    std::memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3(pl.grid, 1, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = pl.smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    int nattr = 0;
+    attr[nattr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[nattr].val.programmaticStreamSerializationAllowed = 1;
+    ++nattr;
+    if (pl.ctas == 2) {
+        attr[nattr].id = cudaLaunchAttributeClusterDimension;
+        attr[nattr].val.clusterDim.x = 2;
+        attr[nattr].val.clusterDim.y = 1;
+        attr[nattr].val.clusterDim.z = 1;
+        ++nattr;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = nattr;
+    const uint16_t* bias_p = nullptr;
+    void* args[] = {&tmA, &tmG, &tmU, &tmZ, &tmZ, &bias_p, &p};
+    if (cudaLaunchKernelExC(&cfg, pl.fn, args) != cudaSuccess) {
         cudaGetLastError();
         return KX_ERR_CUDA;
     }

@@ -106,6 +106,9 @@ struct TileParams {
     int raster_group;
     int has_bias, has_r;
     int drop_kblocks;
+    int swiglu;                   // 1: gate/up mode.  W rows of a tile = BN/2 rows of Wg (tmB) followed by the same
+                                  // BN/2 rows of Wu (tmB2); the epilogue writes silu(gate) * up, BN/2 columns per
+                                  // tile, N = number of output columns; no bias, no residual
     int sk_tile0;                 // tiles [0, sk_tile0) are taken whole, round-robin over the slots;
                                   // tiles [sk_tile0, num_tiles) are stream-K'd (== num_tiles: none)
     int narrow_tile0;             // tile ids >= narrow_tile0 are half-width tiles: id = narrow_tile0 + 2 * j + half
@@ -289,8 +292,13 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 bool narrow;
                 decode_tile(tile, tm, col, narrow);
                 const int a_row = tm * (128 * CTAS) + static_cast<int>(cta_rank) * 128;
-                const int b_row = col + static_cast<int>(cta_rank) * (narrow ? C::BN_LOAD / 2 : C::BN_LOAD);
-                const CUtensorMap* const mapB = narrow ? &tmB2 : &tmB;
+                const bool sg = p.swiglu != 0;
+                // gate/up mode: both halves of the tile's W rows start at output column col / 2; in a
+                // pair CTA 0 holds the gate rows and CTA 1 the up rows, a single CTA loads both
+                const int b_row = sg ? col / 2
+                                     : col + static_cast<int>(cta_rank) * (narrow ? C::BN_LOAD / 2 : C::BN_LOAD);
+                const CUtensorMap* const mapB =
+                    sg ? ((CTAS == 2 && cta_rank == 1) ? &tmB2 : &tmB) : (narrow ? &tmB2 : &tmB);
                 const uint32_t stage_tx = kABytes + (narrow ? C::B_BYTES / 2 : C::B_BYTES);
                 const int kb_end = kb1 - p.drop_kblocks;
                 for (int kb = kb0; kb < kb_end; ++kb) {
@@ -301,6 +309,7 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         mbar_arrive_expect_tx(full(s), stage_tx);
                         tma_load_2d(sa, &tmA, kb * kBlockK, a_row, full(s));
                         tma_load_2d(sb, mapB, kb * kBlockK, b_row, full(s));
+                        if (sg) tma_load_2d(sb + C::B_BYTES / 2, &tmB2, kb * kBlockK, b_row, full(s));
                     } else {
                         // both CTAs' copies complete on the leader's barrier
                         if (leader) mbar_arrive_expect_tx(full(s), 2 * stage_tx);
@@ -389,8 +398,10 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             int tm, colbase;
             bool narrow;
             decode_tile(tile, tm, colbase, narrow);
+            const bool sg = p.swiglu != 0;
+            if (sg) colbase /= 2;                          // BN/2 output columns per tile
             const int row0 = tm * (128 * CTAS) + static_cast<int>(cta_rank) * 128 + q * 32;
-            const int nchunks = narrow ? C::CHUNKS / 2 : C::CHUNKS;
+            const int nchunks = (narrow || sg) ? C::CHUNKS / 2 : C::CHUNKS;
             const bool whole = (kb0 == 0) && (kb1 == nkb);
             auto chunk_valid = [&](int c) { return (row0 < p.M) && (colbase + c * 64 < p.N); };
             auto issue_r = [&](int c) {                    // lane 0 only
@@ -537,6 +548,21 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     tmem_ld_32x32(tbase + c * 64, acc[0]);
                     tmem_ld_32x32(tbase + c * 64 + 32, acc[1]);
                     tmem_ld_wait();
+                }
+                if (valid && sg) {
+                    // acc holds the gate pre-activations of these 64 output columns; the matching up
+                    // values sit BN/2 accumulator columns further.  z = silu(gate) * up in FP32.
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        uint32_t up[32];
+                        tmem_ld_32x32(tbase + BN / 2 + c * 64 + h * 32, up);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            const float gte = __uint_as_float(acc[h][i]);
+                            acc[h][i] = __float_as_uint(gte / (1.0f + __expf(-gte)) * __uint_as_float(up[i]));
+                        }
+                    }
                 }
                 if (valid && role != kWhole) {
                     // split tile: sum the segments in slot order (own accumulator in its place);
