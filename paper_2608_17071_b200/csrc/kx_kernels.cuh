@@ -1,32 +1,45 @@
-// sm_100a kernels for Y = X W^T (+ bias) + R  (BF16 in/out, FP32 accumulate).
+// sm_100a kernels for Y = X W^T (+ bias) + R  (BF16 in/out, FP32 accumulate) and the two
+// neighbouring steps of the decoder layer.
 //
-// Two kernels share one mainloop design (TMA -> swizzled shared-memory ring ->
+// Two GEMM kernels share one mainloop design (TMA -> swizzled shared-memory ring ->
 // tcgen05.mma into TMEM, warp-specialised, mbarrier hand-offs, double-buffered
 // accumulators so the epilogue of unit i overlaps the mainloop of unit i+1):
 //
-//   kx_tile_kernel  large M.  Output tile = 128 rows of X (x2 for a CTA pair)
-//                   by BN rows of W.  Persistent over a rastered tile list.
-//                   Epilogue per warp: R slab by TMA into swizzled staging,
-//                   tcgen05.ld, + bias + R in FP32, one BF16 rounding, written
-//                   back in place, TMA store to Y.
-//   kx_swap_kernel  small / medium M.  W rows sit on the MMA M axis (128 per
-//                   unit), X rows on the MMA N axis (BN per unit), K may be
-//                   split across CTAs.  W is streamed exactly once through a
-//                   deep ring.  Partials go to an FP32 workspace; the last CTA
-//                   to finish a tile sums the splits in fixed order and applies
-//                   bias + R once.
+//   kx_tile_kernel  large M.  Output tile = 128 rows of X (x2 for a CTA pair,
+//                   cta_group::2) by BN rows of W.  Persistent; every slot walks a
+//                   sequence of segments: whole tiles round-robin over a grouped
+//                   raster, then either half-width tail tiles (the last partial wave
+//                   cut in two) or, on request, a stream-K region whose split tiles
+//                   are finished by the last-arriving holder through an FP32
+//                   workspace.  Epilogue per warp: R slab by TMA into swizzled
+//                   staging, tcgen05.ld, + bias + R in FP32, one BF16 rounding,
+//                   written back in place, TMA store to Y.  In gate/up mode a tile
+//                   holds 128 gate and the matching 128 up columns and the epilogue
+//                   stores silu(gate) * up.
+//   kx_swap_kernel  small M.  W rows sit on the MMA M axis (128 per unit), X rows on
+//                   the MMA N axis (BN per unit), K split across CTAs.  W is streamed
+//                   exactly once through a deep ring.  The splits of a tile are a
+//                   thread-block cluster and are summed through distributed shared
+//                   memory in split order; with more than 8 splits (or on request)
+//                   partials go to an FP32 workspace and the last CTA to finish sums
+//                   them.  Bias and residual are applied once.
+//   kx_rmsnorm_kernel  z = h * rsqrt(mean h^2 + eps) * gamma over BF16 rows, one pass.
 //
-// The operation is the paper's residual GEMM epilogue (Appendix A, Algorithm 3:
-// O <- W^T A + O, alpha = beta = 1, output aliased onto the residual) and the
-// plain GEMM of Section 4.1.  The warp roles follow the curriculum of Table 2
-// (tensor-core pipeline, producer/consumer specialisation, persistent CTAs with
-// raw mbarriers, chunked TMA epilogue, tile scheduling) re-expressed for
-// Blackwell: tcgen05 + TMEM replace WGMMA, and a CTA pair (cta_group::2)
-// replaces the cluster multicast tier.
+// The projection is the paper's residual GEMM epilogue (Appendix A, Algorithm 3:
+// O <- W^T A + O, alpha = beta = 1, output aliased onto the residual) and the plain
+// GEMM of Section 4.1; RMSNorm and the gate/up SwiGLU product are the next steps of the
+// decoder layer in Algorithm 7.  The warp roles follow the curriculum of Table 2
+// (tensor-core pipeline, producer/consumer specialisation, persistent CTAs with raw
+// mbarriers, chunked TMA epilogue, tile scheduling) re-expressed for Blackwell:
+// tcgen05 + TMEM replace WGMMA, and a CTA pair (cta_group::2) replaces the cluster
+// multicast tier.  Both GEMM kernels start with a prologue that touches only the
+// CTA's own resources and then wait for the previous kernel in the stream
+// (programmatic dependent launch).
 //
 // Every wait on an mbarrier is bounded: after `spin_limit_ns` the waiting thread
 // records where it gave up, raises a CTA-wide abort flag and every role falls
-// through to the common teardown (TMEM is always freed).
+// through to the common teardown (TMEM is always freed).  Hardware cluster barriers
+// are executed by every thread after its bounded role, so they cannot hang.
 #pragma once
 #include "kx_ptx.cuh"
 
@@ -61,7 +74,6 @@ struct Waiter {
         atomicCAS(const_cast<uint32_t*>(abort_flag), 0u, where);
         if (peer_abort) st_cluster_u32(peer_abort, where);
     }
-    __device__ __forceinline__ bool aborted() const { return *abort_flag != 0; }
     // true = barrier phase completed; false = gave up (abort raised)
     __device__ __forceinline__ bool wait(uint32_t bar, uint32_t parity, uint32_t where) const {
         if (mbar_try_wait(bar, parity)) return true;
@@ -133,7 +145,6 @@ struct TileCfg {
     static constexpr int TMEM_COLS = tmem_cols_for(2 * BN);
     static constexpr int CHUNKS = BN / 64;                  // 64-column epilogue chunks per tile
     static constexpr int PART_FLOATS = 128 * BN;            // one CTA's FP32 partial of one tile
-    static constexpr bool HAS_NARROW = (BN % 128 == 0) && ((BN / 2 / CTAS) % 8 == 0);   // half-width tail tiles
     static_assert(BN % 64 == 0 && BN <= 256, "BN");
     static_assert(NUM_BARS * 8 + 16 <= 1024, "barrier area");
     static_assert(STAGE_BYTES % 1024 == 0, "stage alignment");
