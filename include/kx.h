@@ -82,6 +82,9 @@ enum { KX_PATH_AUTO = 0, KX_PATH_TILE = 1, KX_PATH_SWAP = 2 };
  *   cluster_reduce  swap path: 0 auto, 1 = sum the K splits through the FP32 workspace
  *                 (last CTA to arrive reduces), 2 = the 2..8 splits of a tile form a
  *                 thread-block cluster and are summed through distributed shared memory
+ *   k_cluster     tile path, one CTA per tile: 2 or 4 = split the K range of every tile over a
+ *                 thread-block cluster of that many CTAs and sum the partial tiles through
+ *                 distributed shared memory (for problems with too few tiles to fill the GPU)
  *   no_table      1 = ignore the built-in measured plan table and use the heuristic
  *                 (the table is consulted only when no plan field above is set)
  *   no_pdl        1 = launch without programmatic stream serialization (by default the
@@ -108,7 +111,8 @@ typedef struct kx_plan_override {
     int32_t no_pdl;
     int32_t cluster_reduce;
     int32_t no_table;
-    int32_t reserved[2];
+    int32_t k_cluster;
+    int32_t reserved[1];
 } kx_plan_override;
 
 /* What the planner chose for a shape (kx_plan_query). */

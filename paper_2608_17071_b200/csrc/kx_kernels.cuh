@@ -121,6 +121,11 @@ struct TileParams {
     int swiglu;                   // 1: gate/up mode.  W rows of a tile = BN/2 rows of Wg (tmB) followed by the same
                                   // BN/2 rows of Wu (tmB2); the epilogue writes silu(gate) * up, BN/2 columns per
                                   // tile, N = number of output columns; no bias, no residual
+    int kcluster;                 // > 1 (single-CTA tiles only): the K range of every tile is split over a
+                                  // thread-block cluster of this many CTAs (grid = tiles x kcluster, one tile per
+                                  // cluster); partials are parked in shared memory and each CTA finishes the
+                                  // 64-column chunks c with c % kcluster == rank by reading all partials
+                                  // through distributed shared memory in rank order
     int sk_tile0;                 // tiles [0, sk_tile0) are taken whole, round-robin over the slots;
                                   // tiles [sk_tile0, num_tiles) are stream-K'd (== num_tiles: none)
     int narrow_tile0;             // tile ids >= narrow_tile0 are half-width tiles: id = narrow_tile0 + 2 * j + half
@@ -163,13 +168,17 @@ __device__ __forceinline__ int sk_slot_of(long long U, int G, long long u) {
 
 // The work of one slot (a CTA or a CTA pair) as a sequence of segments (tile, kb0, kb1).
 struct SegIter {
-    int nkb, sk_tile0, t, tstride;
+    int nkb, sk_tile0, t, tstride, kc_kb0, kc_kb1;
     long long u, u1;
-    __device__ __forceinline__ void init(const TileParams& p, int nkb_, int slot, int slots) {
+    // krank / kcluster: position of this CTA in its K cluster (0 / 1 when there is none)
+    __device__ __forceinline__ void init(const TileParams& p, int nkb_, int slot, int slots, int krank = 0,
+                                         int kcluster = 1) {
         nkb = nkb_;
         sk_tile0 = p.sk_tile0;
         t = slot;
         tstride = slots;
+        kc_kb0 = static_cast<int>((static_cast<long long>(krank) * nkb_) / kcluster);
+        kc_kb1 = static_cast<int>((static_cast<long long>(krank + 1) * nkb_) / kcluster);
         const long long U = static_cast<long long>(p.num_tiles - p.sk_tile0) * nkb_;
         u = sk_begin(U, slots, slot);
         u1 = sk_begin(U, slots, slot + 1);
@@ -177,8 +186,8 @@ struct SegIter {
     __device__ __forceinline__ bool next(int& tile, int& kb0, int& kb1) {
         if (t < sk_tile0) {
             tile = t;
-            kb0 = 0;
-            kb1 = nkb;
+            kb0 = kc_kb0;
+            kb1 = kc_kb1;
             t += tstride;
             return true;
         }
@@ -227,8 +236,10 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const uint32_t cta_rank = (CTAS == 2) ? cluster_ctarank() : 0u;
     const bool leader = (cta_rank == 0);
     const int nkb = (p.K + kBlockK - 1) / kBlockK;
-    const int slot = blockIdx.x / CTAS;
-    const int slots = gridDim.x / CTAS;
+    const int kc = (CTAS == 1 && p.kcluster > 1) ? p.kcluster : 1;   // K-cluster size
+    const int krank = (kc > 1) ? static_cast<int>(cluster_ctarank()) : 0;
+    const int slot = blockIdx.x / (CTAS * kc);
+    const int slots = gridDim.x / (CTAS * kc);
 
     if (threadIdx.x == 0) *s_abort = 0;
     if (warp == 4 && lane == 0) {
@@ -277,7 +288,7 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     wt.limit_ns = p.spin_limit_ns;
 
     SegIter it;
-    it.init(p, nkb, slot, slots);
+    it.init(p, nkb, slot, slots, krank, kc);
     int tile, kb0, kb1;
     // tile id -> tile row, first output column, width class
     auto decode_tile = [&](int t, int& tm, int& col, bool& narrow) {
@@ -332,6 +343,11 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 }
             }
         }
+        if (kc > 1) {            // K-cluster mode: every thread of the cluster passes both barriers
+            __syncwarp();
+            cluster_arrive(); cluster_wait();
+            cluster_arrive(); cluster_wait();
+        }
     } else if (warp == 5) {
         // ------------------------------------------------------------ MMA issuer
         if (leader && lane == 0) {
@@ -379,6 +395,11 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 while (!mbar_try_wait(drain_bar, 0) && ++spins < (1u << 20)) {}
             }
         }
+        if (kc > 1) {
+            __syncwarp();
+            cluster_arrive(); cluster_wait();
+            cluster_arrive(); cluster_wait();
+        }
     } else {
         // ------------------------------------------------------------ epilogue warps
         // Warp q owns TMEM lanes / tile rows 32q..32q+31 and is independent of the other
@@ -392,9 +413,13 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         auto slab4 = [&](float* part, int c) {
             return reinterpret_cast<float4*>(part) + (static_cast<size_t>(c) * 4 + q) * 16 * 32 + lane;
         };
-        enum { kWhole = 0, kFast = 1, kWriter = 2, kSlow = 3, kNone = 4 };
+        enum { kWhole = 0, kFast = 1, kWriter = 2, kSlow = 3, kNone = 4, kCluster = 5 };
         uint32_t scount = 0, rphase = 0;
         bool ok = true;
+        int cluster_bars = 0;                              // K-cluster mode: cluster barriers passed so far
+        // K-cluster mode: a CTA's partial tile parked at the start of its (idle) operand ring, same
+        // float4 order as slab4; `ring` is the shared::cta address of this CTA's copy
+        const uint32_t ring = s_stage;
 
         // partial of (slot sl, tile tl) for this CTA rank: "head" if tl is the first tile the slot touches
         auto part_ptr = [&](int sl, int tl) -> float* {
@@ -414,7 +439,9 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const int row0 = tm * (128 * CTAS) + static_cast<int>(cta_rank) * 128 + q * 32;
             const int nchunks = (narrow || sg) ? C::CHUNKS / 2 : C::CHUNKS;
             const bool whole = (kb0 == 0) && (kb1 == nkb);
-            auto chunk_valid = [&](int c) { return (row0 < p.M) && (colbase + c * 64 < p.N); };
+            auto chunk_inb = [&](int c) { return (row0 < p.M) && (colbase + c * 64 < p.N); };
+            // chunks this warp writes to Y: all of them, or in K-cluster mode those dealt to this CTA
+            auto chunk_valid = [&](int c) { return chunk_inb(c) && (kc == 1 || (c % kc) == krank); };
             auto issue_r = [&](int c) {                    // lane 0 only
                 if (chunk_valid(c)) {
                     const int j = c % NB;
@@ -427,7 +454,7 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             // to (the slot's last segment: its partners ran at the start of their ranges) produce
             // the output.
             const bool last_seg = (it.t >= it.sk_tile0) && (it.u >= it.u1);
-            const bool spec_r = has_r && (whole || last_seg);
+            const bool spec_r = has_r && (whole || last_seg || kc > 1);
             int n_iss = 0;                                 // R chunks requested so far (warp-uniform)
             if (lane == 0) tma_store_wait_read<0>();       // staging buffers of the previous tile are free
             if (spec_r) {
@@ -442,7 +469,7 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             int role = kWhole, s_first = 0, s_last = 0;
             unsigned int* ctr = nullptr;
             bool staged = false;   // the partner's partial already sits in the other accumulator buffer
-            if (!whole) {
+            if (!whole && kc == 1) {
                 const long long ut = static_cast<long long>(tile - p.sk_tile0) * nkb;
                 s_first = sk_slot_of(U, slots, ut);
                 s_last = sk_slot_of(U, slots, ut + nkb - 1);
@@ -492,7 +519,30 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     else mbar_arrive_cluster(map_to_cta(acc_empty(b), 0));
                 }
             };
-            if (!whole) {
+            if (kc > 1) {
+                // K-cluster: park this CTA's partial (every in-bounds chunk) in its own shared memory,
+                // meet the cluster, then finish the chunks dealt to this CTA from all partials
+                role = kCluster;
+#pragma unroll 1
+                for (int c = 0; c < nchunks; ++c) {
+                    if (!chunk_inb(c)) continue;
+                    uint32_t a[2][32];
+                    tmem_ld_32x32(tbase + c * 64, a[0]);
+                    tmem_ld_32x32(tbase + c * 64 + 32, a[1]);
+                    tmem_ld_wait();
+                    const uint32_t dst = ring + (((c * 4 + q) * 16) * 32 + lane) * 16;
+#pragma unroll
+                    for (int i = 0; i < 16; ++i)
+                        asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + i * 512),
+                                     "r"(a[i >> 3][(i & 7) * 4 + 0]), "r"(a[i >> 3][(i & 7) * 4 + 1]),
+                                     "r"(a[i >> 3][(i & 7) * 4 + 2]), "r"(a[i >> 3][(i & 7) * 4 + 3])
+                                     : "memory");
+                }
+                release_acc();
+                cluster_arrive();
+                cluster_wait();
+                ++cluster_bars;
+            } else if (!whole) {
                 if (staged) {
                     role = kFast;
                 } else {
@@ -575,7 +625,29 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         }
                     }
                 }
-                if (valid && role != kWhole) {
+                if (valid && role == kCluster) {
+                    // sum the cluster's partials of this chunk in rank order (16 remote 16-byte loads in
+                    // flight per rank)
+                    float sum[64];
+#pragma unroll
+                    for (int i = 0; i < 64; ++i) sum[i] = 0.f;
+                    const uint32_t off = ring + (((c * 4 + q) * 16) * 32 + lane) * 16;
+#pragma unroll 1
+                    for (int r = 0; r < kc; ++r) {
+                        const uint32_t src = map_to_cta(off, r);
+                        float4 t[16];
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) t[i] = ld_cluster_f32x4(src + i * 512);
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            sum[i * 4 + 0] += t[i].x; sum[i * 4 + 1] += t[i].y;
+                            sum[i * 4 + 2] += t[i].z; sum[i * 4 + 3] += t[i].w;
+                        }
+                    }
+#pragma unroll
+                    for (int i = 0; i < 64; ++i) acc[i >> 5][i & 31] = __float_as_uint(sum[i]);
+                }
+                if (valid && (role == kFast || role == kSlow)) {
                     // split tile: sum the segments in slot order (own accumulator in its place);
                     // all 16 loads of a segment are in flight before the first is consumed
                     float sum[64];
@@ -610,7 +682,7 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
                     for (int i = 0; i < 64; ++i) acc[i >> 5][i & 31] = __float_as_uint(sum[i]);
                 }
-                if (c == nchunks - 1 && role != kSlow) release_acc();
+                if (c == nchunks - 1 && (role == kWhole || role == kFast)) release_acc();
                 if (valid) {
                     if (has_r) {
                         if (!__all_sync(0xffffffffu, wt.wait(r_full(q, j), (rphase >> j) & 1u, kWhereRFull))) {
@@ -673,8 +745,17 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 }
                 __syncwarp();
             }
-            if (role != kWhole && lane == 0) *ctr = 0u;    // every segment has arrived: reset for the next launch
+            if ((role == kFast || role == kSlow) && lane == 0) *ctr = 0u;   // every segment has arrived: reset
             if (q == 0 && lane == 0 && leader) KX_TRACE_POINT(p, slot, (scount - 1) * 4 + 3);
+        }
+        if (kc > 1) {
+            // peers may still be reading this CTA's partial: second barrier; on a give-up path the
+            // barriers skipped above are made up here so that the cluster never hangs
+            __syncwarp();
+            for (; cluster_bars < 2; ++cluster_bars) {
+                cluster_arrive();
+                cluster_wait();
+            }
         }
         if (lane == 0) tma_store_wait_all<0>();
     }

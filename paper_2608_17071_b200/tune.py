@@ -24,7 +24,7 @@ import time
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 FIELDS = ("path", "block_n", "cta_pair", "split_k", "raster_group", "stages", "stream_k", "narrow_tail",
-          "cluster_reduce")
+          "cluster_reduce", "k_cluster")
 ATOL, RTOL = 1e-2, 1.6e-2
 
 
@@ -54,6 +54,9 @@ def candidates(M: int, N: int, K: int, kx):
         out.append(dict(path=T, block_n=256, cta_pair=2, stages=5))
         out.append(dict(path=T, block_n=256, cta_pair=2, narrow_tail=1))
         out.append(dict(path=T, block_n=256, cta_pair=1, narrow_tail=1))
+        for bn in (256, 192, 128):
+            for kc in (2, 4):
+                out.append(dict(path=T, block_n=bn, cta_pair=1, k_cluster=kc))
     return out
 
 

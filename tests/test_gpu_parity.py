@@ -138,6 +138,40 @@ def test_half_width_tail_tiles_exact(ov, max_ctas, M, N):
     assert np.array_equal(run(X, W, b, R, off), y)
 
 
+@pytest.mark.parametrize("bn", [256, 192, 128, 64])
+@pytest.mark.parametrize("kc", [2, 4])
+@pytest.mark.parametrize("M,N,K", [(128, 256, 512), (512, 2048, 2048), (300, 520, 520), (640, 1032, 4096)])
+def test_k_cluster_exact_integer_arithmetic(bn, kc, M, N, K):
+    """Single-CTA tiles whose K range is split over a 2- or 4-CTA cluster; the partial tiles are
+    summed through distributed shared memory in rank order.  Integer-valued data: bit-exact,
+    also in place and without bias / residual."""
+    ov = dict(path=T, block_n=bn, cta_pair=1, k_cluster=kc)
+    X, W, b, R = ternary_case(M, N, K, seed=27)
+    y = run(X, W, b, R, ov)
+    ok, msg = kt.gate_exact(y, oracle.outproj(X, W, b, R))
+    assert ok, msg
+    assert np.array_equal(run(X, W, b, R.copy(), ov, inplace=True), y)
+    ok, msg = kt.gate_exact(run(X, W, None, None, ov), oracle.outproj(X, W))
+    assert ok, msg
+
+
+def test_k_cluster_random_data_and_bad_plans():
+    d = inputs.make_inputs(inputs.all_workloads()["sweep_M512_H2048"], stress=True)
+    ref, absref = oracle.outproj(d["X"], d["W"], d["bias"], d["R"], want_abs=True)
+    for kc in (2, 4):
+        ov = dict(path=T, block_n=256, cta_pair=1, k_cluster=kc)
+        ys = [run(d["X"], d["W"], d["bias"], d["R"], ov) for _ in range(2)]
+        assert np.array_equal(ys[0], ys[1])
+        ok, msg = kt.gate_a(ys[0], ref)
+        assert ok, msg
+        ok, msg = kt.gate_c(ys[0], ref, absref, 2048, rate_limit=3e-2)
+        assert ok, msg
+    for bad in (dict(path=T, block_n=256, cta_pair=2, k_cluster=2), dict(path=T, block_n=256, cta_pair=1, k_cluster=3),
+                dict(path=T, block_n=256, cta_pair=1, k_cluster=2, stream_k=2)):
+        with pytest.raises(kx.KxError):
+            kx.kx_plan_query(512, 2048, 2048, ov=kx.make_override(**bad))
+
+
 @pytest.mark.parametrize("ov", STREAMK_VARIANTS[:2], ids=vid)
 def test_stream_k_random_data_is_deterministic_and_within_gates(ov):
     wl = inputs.all_workloads()["cfg2"]

@@ -17,7 +17,7 @@ pytestmark = pytest.mark.gpu
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 FIELDS = ("path", "block_n", "cta_pair", "split_k", "raster_group", "stages", "stream_k", "narrow_tail",
-          "cluster_reduce")
+          "cluster_reduce", "k_cluster")
 
 
 def table_entries():

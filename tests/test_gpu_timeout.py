@@ -21,8 +21,10 @@ WAIT_FULL = 2   # the MMA issuer's wait for a filled stage
 
 @pytest.mark.parametrize("ov", [dict(path=T, block_n=256, cta_pair=1), dict(path=T, block_n=128, cta_pair=2),
                                 dict(path=S, block_n=128, split_k=2),
-                                dict(path=T, block_n=256, cta_pair=2, stream_k=2)],
-                         ids=["tile", "pair", "swap-splitk", "pair-streamk"])
+                                dict(path=T, block_n=256, cta_pair=2, stream_k=2),
+                                dict(path=T, block_n=128, cta_pair=1, k_cluster=2),
+                                dict(path=S, block_n=128, split_k=2, cluster_reduce=1)],
+                         ids=["tile", "pair", "swap-cluster", "pair-streamk", "tile-kcluster", "swap-workspace"])
 def test_wait_gives_up_and_context_survives(ov):
     import time
     M, N, K = 128, 512, 512
