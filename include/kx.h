@@ -172,7 +172,9 @@ int kx_outproj_residual_ex(const void* X, const void* W, const void* bias_or_nul
  * HOST pointer (pinned memory gives the best copy rate; pageable works).  The
  * call copies X, W, bias, R to library-owned device staging buffers (grown on
  * demand, kept until kx_shutdown), runs the kernel, copies Y back into Y_host
- * and synchronises `stream` before returning.  R_host and bias_host may be NULL.
+ * and synchronises `stream` before returning.  For M >= 2048 the rows are cut
+ * into four slices and copy-in, compute and copy-out of consecutive slices
+ * overlap on three streams (two of them library-owned).  R_host and bias_host may be NULL.
  * Not for use under stream capture (it may allocate and it synchronises).
  */
 int kx_outproj_residual_host(const void* X_host, const void* W_host, const void* bias_host_or_null,

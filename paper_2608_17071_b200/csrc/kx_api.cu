@@ -40,9 +40,11 @@ struct DeviceCtx {
     float* ws = nullptr;
     unsigned int* counters = nullptr;
     unsigned int* status = nullptr;
-    // staging for the *_host entry point
+    // staging, copy streams and events of the *_host entry point
     void* stage = nullptr;
     size_t stage_bytes = 0;
+    cudaStream_t h_in = nullptr, h_out = nullptr;
+    cudaEvent_t h_start = nullptr, h_done = nullptr, h_in_ev[8] = {}, h_k_ev[8] = {};
 };
 DeviceCtx g_ctx[kMaxDevices];
 #ifdef KX_TRACE
@@ -733,6 +735,16 @@ int kx_shutdown(void) {
         if (c.ws) cudaFree(c.ws);
         if (c.counters) cudaFree(c.counters);
         if (c.stage) cudaFree(c.stage);
+        if (c.h_in) {
+            cudaStreamDestroy(c.h_in);
+            cudaStreamDestroy(c.h_out);
+            cudaEventDestroy(c.h_start);
+            cudaEventDestroy(c.h_done);
+            for (int i = 0; i < 8; ++i) {
+                cudaEventDestroy(c.h_in_ev[i]);
+                cudaEventDestroy(c.h_k_ev[i]);
+            }
+        }
         c = DeviceCtx();
     }
     cudaSetDevice(prev);
@@ -840,26 +852,66 @@ int kx_outproj_residual_host(const void* Xh, const void* Wh, const void* bh, con
         }
     }
     char* base = static_cast<char*>(ctx->stage);
-    void* Xd = base;
-    void* Wd = base + xb;
-    void* bd = base + xb + wb;
-    void* Yd = base + xb + wb + bb;
-    bool ok = true;
-    if (K > 0) {
-        ok = ok && cudaMemcpyAsync(Xd, Xh, static_cast<size_t>(M) * K * 2, cudaMemcpyHostToDevice, stream) == cudaSuccess;
-        ok = ok && cudaMemcpyAsync(Wd, Wh, static_cast<size_t>(N) * K * 2, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    char* Xd = base;
+    char* Wd = base + xb;
+    char* bd = base + xb + wb;
+    char* Yd = base + xb + wb + bb;
+    // Rows are independent, so large problems are cut into row slices and pipelined over three
+    // streams: while slice i computes on `stream`, slice i+1 is copied in and slice i-1 copied out
+    // (PCIe is full duplex).  W and bias go first.  Streams and events are created once per device.
+    constexpr int kMaxSlices = 8;
+    {
+        std::lock_guard<std::mutex> lk(g_mu);
+        if (!ctx->h_in) {
+            bool ok = cudaStreamCreateWithFlags(&ctx->h_in, cudaStreamNonBlocking) == cudaSuccess &&
+                      cudaStreamCreateWithFlags(&ctx->h_out, cudaStreamNonBlocking) == cudaSuccess &&
+                      cudaEventCreateWithFlags(&ctx->h_start, cudaEventDisableTiming) == cudaSuccess &&
+                      cudaEventCreateWithFlags(&ctx->h_done, cudaEventDisableTiming) == cudaSuccess;
+            for (int i = 0; i < kMaxSlices && ok; ++i)
+                ok = cudaEventCreateWithFlags(&ctx->h_in_ev[i], cudaEventDisableTiming) == cudaSuccess &&
+                     cudaEventCreateWithFlags(&ctx->h_k_ev[i], cudaEventDisableTiming) == cudaSuccess;
+            if (!ok) {
+                cudaGetLastError();
+                ctx->h_in = nullptr;
+                return KX_ERR_CUDA;
+            }
+        }
     }
-    if (bh) ok = ok && cudaMemcpyAsync(bd, bh, static_cast<size_t>(N) * 2, cudaMemcpyHostToDevice, stream) == cudaSuccess;
-    // the residual is copied straight into the output buffer: the kernel then runs in place (Y == R)
-    if (Rh) ok = ok && cudaMemcpyAsync(Yd, Rh, static_cast<size_t>(M) * N * 2, cudaMemcpyHostToDevice, stream) == cudaSuccess;
-    if (!ok) {
-        cudaGetLastError();
-        return KX_ERR_CUDA;
+    const long long slice_rows = (M >= 2048 && K > 0) ? ((M + 3) / 4 + 255) / 256 * 256 : M;
+    const int slices = static_cast<int>((M + slice_rows - 1) / slice_rows);
+    bool ok = cudaEventRecord(ctx->h_start, stream) == cudaSuccess &&
+              cudaStreamWaitEvent(ctx->h_in, ctx->h_start, 0) == cudaSuccess &&
+              cudaStreamWaitEvent(ctx->h_out, ctx->h_start, 0) == cudaSuccess;
+    if (K > 0)
+        ok = ok && cudaMemcpyAsync(Wd, Wh, static_cast<size_t>(N) * K * 2, cudaMemcpyHostToDevice, ctx->h_in) == cudaSuccess;
+    if (bh) ok = ok && cudaMemcpyAsync(bd, bh, static_cast<size_t>(N) * 2, cudaMemcpyHostToDevice, ctx->h_in) == cudaSuccess;
+    for (int i = 0; i < slices && ok; ++i) {
+        const long long r0 = i * slice_rows, rows = std::min<long long>(slice_rows, M - r0);
+        const size_t xo = static_cast<size_t>(r0) * K * 2, yo = static_cast<size_t>(r0) * N * 2;
+        if (K > 0)
+            ok = ok && cudaMemcpyAsync(Xd + xo, static_cast<const char*>(Xh) + xo, static_cast<size_t>(rows) * K * 2,
+                                       cudaMemcpyHostToDevice, ctx->h_in) == cudaSuccess;
+        // the residual is copied straight into the output buffer: the kernel then runs in place (Y == R)
+        if (Rh)
+            ok = ok && cudaMemcpyAsync(Yd + yo, static_cast<const char*>(Rh) + yo, static_cast<size_t>(rows) * N * 2,
+                                       cudaMemcpyHostToDevice, ctx->h_in) == cudaSuccess;
+        ok = ok && cudaEventRecord(ctx->h_in_ev[i], ctx->h_in) == cudaSuccess &&
+             cudaStreamWaitEvent(stream, ctx->h_in_ev[i], 0) == cudaSuccess;
+        if (!ok) break;
+        rc = run(Xd + xo, Wd, bh ? bd : nullptr, Rh ? Yd + yo : nullptr, Yd + yo, rows, N, K, stream, nullptr, false);
+        if (rc != KX_OK) break;
+        ok = ok && cudaEventRecord(ctx->h_k_ev[i], stream) == cudaSuccess &&
+             cudaStreamWaitEvent(ctx->h_out, ctx->h_k_ev[i], 0) == cudaSuccess &&
+             cudaMemcpyAsync(static_cast<char*>(Yh) + yo, Yd + yo, static_cast<size_t>(rows) * N * 2,
+                             cudaMemcpyDeviceToHost, ctx->h_out) == cudaSuccess;
     }
-    rc = run(Xd, Wd, bh ? bd : nullptr, Rh ? Yd : nullptr, Yd, M, N, K, stream, nullptr, false);
+    // join: `stream` (and the host) continue only after the last slice has been copied out
+    const bool joined = cudaEventRecord(ctx->h_done, ctx->h_out) == cudaSuccess &&
+                        cudaStreamWaitEvent(stream, ctx->h_done, 0) == cudaSuccess &&
+                        cudaStreamSynchronize(ctx->h_in) == cudaSuccess &&
+                        cudaStreamSynchronize(stream) == cudaSuccess;
     if (rc != KX_OK) return rc;
-    if (cudaMemcpyAsync(Yh, Yd, static_cast<size_t>(M) * N * 2, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
-        cudaStreamSynchronize(stream) != cudaSuccess) {
+    if (!ok || !joined) {
         cudaGetLastError();
         return KX_ERR_CUDA;
     }

@@ -402,6 +402,19 @@ def test_host_buffer_entry_point():
     assert np.array_equal(y, run(d["X"], d["W"], d["bias"], d["R"]))
     ok, msg = kt.gate_a(y, oracle.outproj(d["X"], d["W"], d["bias"], d["R"]))
     assert ok, msg
+    # M >= 2048: pipelined row slices; every slice must land in its place (pinned and pageable hosts)
+    M3 = 2304 + 77
+    d3 = inputs.make_inputs(inputs.Workload("t", M3, 264, 520, 73, True, True), stress=True)
+    X3, W3, b3, R3 = ternary_case(M3, 264, 520, seed=74)
+    Y3 = torch.empty(M3, 264, dtype=torch.int16).pin_memory()
+    kx.kx_outproj_residual_host(pin(X3), pin(W3), pin(b3), pin(R3), Y3, M3, 264, 520)
+    ok, msg = kt.gate_exact(Y3.numpy().view(np.uint16), oracle.outproj(X3, W3, b3, R3))
+    assert ok, msg
+    Y3p = np.zeros((M3, 264), dtype=np.uint16)
+    kx.kx_outproj_residual_host(np.ascontiguousarray(d3["X"]), np.ascontiguousarray(d3["W"]), None,
+                                np.ascontiguousarray(d3["R"]), Y3p, M3, 264, 520)
+    ok, msg = kt.gate_a(Y3p, oracle.outproj(d3["X"], d3["W"], None, d3["R"]))
+    assert ok, msg
     # a larger problem afterwards grows the staging buffer
     M2 = 900
     d2 = inputs.make_inputs(inputs.Workload("t", M2, N, K, 72, False, False), stress=True)
