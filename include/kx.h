@@ -85,6 +85,10 @@ enum { KX_PATH_AUTO = 0, KX_PATH_TILE = 1, KX_PATH_SWAP = 2 };
  *   k_cluster     tile path, one CTA per tile: 2 or 4 = split the K range of every tile over a
  *                 thread-block cluster of that many CTAs and sum the partial tiles through
  *                 distributed shared memory (for problems with too few tiles to fill the GPU)
+ *   l2_prefetch   number of leading k-blocks of its first work item whose operand tiles a CTA asks
+ *                 to be brought into L2 before it waits for the previous kernel in the stream
+ *                 (0 = the ring depth, -1 = none).  L2 is the device's coherence point, so a
+ *                 tile requested early still shows every later device write when it is loaded.
  *   no_table      1 = ignore the built-in measured plan table and use the heuristic
  *                 (the table is consulted only when no plan field above is set)
  *   no_pdl        1 = launch without programmatic stream serialization (by default the
@@ -112,7 +116,7 @@ typedef struct kx_plan_override {
     int32_t cluster_reduce;
     int32_t no_table;
     int32_t k_cluster;
-    int32_t reserved[1];
+    int32_t l2_prefetch;
 } kx_plan_override;
 
 /* What the planner chose for a shape (kx_plan_query). */

@@ -35,7 +35,7 @@ class PlanOverride(ctypes.Structure):
         ("path", ctypes.c_int32), ("block_n", ctypes.c_int32), ("cta_pair", ctypes.c_int32),
         ("split_k", ctypes.c_int32), ("raster_group", ctypes.c_int32), ("max_ctas", ctypes.c_int32),
         ("spin_limit_us", ctypes.c_int32), ("debug_drop_kblocks", ctypes.c_int32),
-        ("stages", ctypes.c_int32), ("stream_k", ctypes.c_int32), ("narrow_tail", ctypes.c_int32), ("no_pdl", ctypes.c_int32), ("cluster_reduce", ctypes.c_int32), ("no_table", ctypes.c_int32), ("k_cluster", ctypes.c_int32), ("reserved", ctypes.c_int32 * 1),
+        ("stages", ctypes.c_int32), ("stream_k", ctypes.c_int32), ("narrow_tail", ctypes.c_int32), ("no_pdl", ctypes.c_int32), ("cluster_reduce", ctypes.c_int32), ("no_table", ctypes.c_int32), ("k_cluster", ctypes.c_int32), ("l2_prefetch", ctypes.c_int32),
     ]
 
 

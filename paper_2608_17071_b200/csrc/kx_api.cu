@@ -633,6 +633,7 @@ int run(const void* X, const void* W, const void* bias, const void* R, void* Y, 
         p.has_bias = bias ? 1 : 0;
         p.has_r = R ? 1 : 0;
         p.drop_kblocks = drop;
+        p.pf_kblocks = ov ? ov->l2_prefetch : 0;
         p.swiglu = 0;
         p.kcluster = pl.kcluster;
         p.sk_tile0 = pl.sk_tile0;
@@ -665,6 +666,7 @@ int run(const void* X, const void* W, const void* bias, const void* R, void* Y, 
         p.has_bias = bias ? 1 : 0;
         p.has_r = R ? 1 : 0;
         p.drop_kblocks = drop;
+        p.pf_kblocks = ov ? ov->l2_prefetch : 0;
         p.spin_limit_ns = spin_ns;
         p.status = ctx->status;
         p.ws = ctx->ws;
@@ -1199,6 +1201,7 @@ int kx_outproj_residual_noalloc(const void* X, const void* W, const void* bias, 
     p.has_bias = bias ? 1 : 0;
     p.has_r = R ? 1 : 0;
     p.drop_kblocks = 0;
+    p.pf_kblocks = 0;
     p.spin_limit_ns = 2000000000ull;
     p.status = ctx->status;
     p.ws = partials;

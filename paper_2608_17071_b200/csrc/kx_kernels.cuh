@@ -118,6 +118,7 @@ struct TileParams {
     int raster_group;
     int has_bias, has_r;
     int drop_kblocks;
+    int pf_kblocks;            // L2 prefetch depth before the dependency wait (0 = ring depth, <0 = none)
     int swiglu;                   // 1: gate/up mode.  W rows of a tile = BN/2 rows of Wg (tmB) followed by the same
                                   // BN/2 rows of Wu (tmB2); the epilogue writes silu(gate) * up, BN/2 columns per
                                   // tile, N = number of output columns; no bias, no residual
@@ -241,6 +242,20 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int slot = blockIdx.x / (CTAS * kc);
     const int slots = gridDim.x / (CTAS * kc);
 
+    // tile id -> tile row, first output column, width class
+    auto decode_tile = [&](int t, int& tm, int& col, bool& narrow) {
+        narrow = t >= p.narrow_tile0;
+        int pos = t, half = 0;
+        if (narrow) {
+            const int j = t - p.narrow_tile0;
+            pos = p.narrow_tile0 + (j >> 1);
+            half = j & 1;
+        }
+        int tn;
+        tile_coords(pos, p.tiles_m, p.tiles_n, p.raster_group, tm, tn);
+        col = tn * BN + half * (BN / 2);
+    };
+
     if (threadIdx.x == 0) *s_abort = 0;
     if (warp == 4 && lane == 0) {
         prefetch_tmap(&tmA);
@@ -248,6 +263,30 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (p.narrow_tile0 < p.num_tiles) prefetch_tmap(&tmB2);
         prefetch_tmap(&tmY);
         if (p.has_r) prefetch_tmap(&tmR);
+        // Warm L2 with the first ring-full of this CTA's operand tiles before waiting for the
+        // previous kernel: the cold-miss latency of the first loads then overlaps that kernel's tail.
+        {
+            SegIter pf;
+            pf.init(p, nkb, slot, slots, krank, kc);
+            int t0, k0, k1;
+            if (p.pf_kblocks >= 0 && pf.next(t0, k0, k1)) {
+                int tm, col;
+                bool narrow;
+                decode_tile(t0, tm, col, narrow);
+                const int a_row = tm * (128 * CTAS) + static_cast<int>(cta_rank) * 128;
+                const bool sg = p.swiglu != 0;
+                const int b_row = sg ? col / 2
+                                     : col + static_cast<int>(cta_rank) * (narrow ? C::BN_LOAD / 2 : C::BN_LOAD);
+                const CUtensorMap* const mapB =
+                    sg ? ((CTAS == 2 && cta_rank == 1) ? &tmB2 : &tmB) : (narrow ? &tmB2 : &tmB);
+                const int depth = p.pf_kblocks == 0 ? STAGES : p.pf_kblocks;
+                for (int kb = k0; kb < k1 && kb < k0 + depth; ++kb) {
+                    tma_prefetch_l2_2d(&tmA, kb * kBlockK, a_row);
+                    tma_prefetch_l2_2d(mapB, kb * kBlockK, b_row);
+                    if (CTAS == 1 && sg) tma_prefetch_l2_2d(&tmB2, kb * kBlockK, b_row);
+                }
+            }
+        }
     }
     if (warp == 5) {
         if (lane == 0) {
@@ -290,19 +329,6 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     SegIter it;
     it.init(p, nkb, slot, slots, krank, kc);
     int tile, kb0, kb1;
-    // tile id -> tile row, first output column, width class
-    auto decode_tile = [&](int t, int& tm, int& col, bool& narrow) {
-        narrow = t >= p.narrow_tile0;
-        int pos = t, half = 0;
-        if (narrow) {
-            const int j = t - p.narrow_tile0;
-            pos = p.narrow_tile0 + (j >> 1);
-            half = j & 1;
-        }
-        int tn;
-        tile_coords(pos, p.tiles_m, p.tiles_n, p.raster_group, tm, tn);
-        col = tn * BN + half * (BN / 2);
-    };
 
     if (warp == 4) {
         // ------------------------------------------------------------ TMA producer
@@ -782,6 +808,7 @@ struct SwapParams {
     int n_tiles, m_tiles, splits, num_units;
     int has_bias, has_r;
     int drop_kblocks;
+    int pf_kblocks;            // L2 prefetch depth before the dependency wait (0 = ring depth, <0 = none)
     unsigned long long spin_limit_ns;
     unsigned int* status;
     float* ws;                 // [splits][M][N] FP32 partials (splits > 1)
@@ -841,6 +868,16 @@ kx_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     if (warp == 4 && lane == 0) {
         prefetch_tmap(&tmW);
         prefetch_tmap(&tmX);
+        // Warm L2 with the first ring-full of this CTA's W tiles before waiting for the previous
+        // kernel: the cold-miss latency of the first loads then overlaps that kernel's tail.
+        if (static_cast<int>(blockIdx.x) < p.num_units) {
+            const int sp0 = blockIdx.x % p.splits, tile0 = blockIdx.x / p.splits;
+            const int nt0 = tile0 / p.m_tiles;
+            const int k0 = static_cast<int>((static_cast<long long>(sp0) * nkb) / p.splits);
+            const int k1 = static_cast<int>((static_cast<long long>(sp0 + 1) * nkb) / p.splits);
+            const int depth = p.pf_kblocks == 0 ? STAGES : p.pf_kblocks;
+            for (int kb = k0; kb < k1 && kb < k0 + depth; ++kb) tma_prefetch_l2_2d(&tmW, kb * kBlockK, nt0 * 128);
+        }
     }
     if (warp == 5) {
         if (lane == 0) {

@@ -172,6 +172,33 @@ def test_k_cluster_random_data_and_bad_plans():
             kx.kx_plan_query(512, 2048, 2048, ov=kx.make_override(**bad))
 
 
+@pytest.mark.parametrize("depth", [-1, 0, 1, 3, 1000])
+@pytest.mark.parametrize("base", [dict(path=T, block_n=256, cta_pair=2), dict(path=T, block_n=128, cta_pair=1),
+                                  dict(path=T, block_n=256, cta_pair=1, k_cluster=2), dict(path=T, block_n=256, cta_pair=2, narrow_tail=2),
+                                  dict(path=S, block_n=32, split_k=3), dict(path=S, block_n=16, split_k=4, cluster_reduce=2)], ids=vid)
+def test_l2_prefetch_depth_changes_no_bit(base, depth):
+    """The tiles a CTA requests into L2 ahead of the dependency wait are a hint only: every depth
+    (none, ring depth, shallower, deeper than the K range) gives the same bits, and a weight
+    matrix rewritten by the previous kernel in the stream is still seen (L2 is coherent)."""
+    M, N, K = (600, 776, 1096) if base["path"] == T else (base["block_n"] - 3, 520, 1096)
+    X, W, b, R = ternary_case(M, N, K, seed=31)
+    y = run(X, W, b, R, dict(base, l2_prefetch=depth))
+    ok, msg = kt.gate_exact(y, oracle.outproj(X, W, b, R))
+    assert ok, msg
+    # previous kernel in the stream rewrites W: the prefetch may have run before it finished
+    import torch
+    tX, tR, tb, tW2 = kt.to_dev(X), kt.to_dev(R), kt.to_dev(b), kt.to_dev(W)
+    tW = torch.zeros_like(tW2)
+    eye = torch.eye(K, dtype=torch.bfloat16, device="cuda")
+    tY = kt.nan_filled(M, N)
+    ov = kx.make_override(**dict(base, l2_prefetch=depth))
+    for _ in range(3):
+        tW.zero_()
+        kx.kx_gemm_bf16(tW2, eye, tW)      # W = W . I^T, written by the library's own kernel, whose
+        kx.kx_outproj_residual_ex(tX, tW, tb, tR, tY, ov)   # tail the next prologue overlaps
+    assert np.array_equal(kt.from_dev(tY), y)
+
+
 @pytest.mark.parametrize("ov", STREAMK_VARIANTS[:2], ids=vid)
 def test_stream_k_random_data_is_deterministic_and_within_gates(ov):
     wl = inputs.all_workloads()["cfg2"]
