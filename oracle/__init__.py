@@ -5,4 +5,5 @@ package.  The product (the CUDA library and its Python binding) never does.
 """
 from .oracle import (  # noqa: F401
     outproj, outproj_rows, element, round_bf16, widen_bf16, max_threads, rmsnorm, swiglu,
+    quantize_rows, swiglu_int8, outproj_int8,
 )

@@ -261,3 +261,109 @@ int kx_oracle_swiglu_rows(const uint16_t* X, const uint16_t* Wg, const uint16_t*
     return 0;
 }
 
+
+/*
+ * INT8 branch of the decoder layer (Appendix A, Algorithm 7: "fused add+RMSNorm+activation
+ * quantization", "quantize gate/up weights", "gate/up GEMM with fused dequantization and
+ * SwiGLU epilogue").  The paper names the steps but not the code book; the reading taken here
+ * is the common symmetric one, per row (per token for activations, per output channel for
+ * weights):
+ *
+ *     a      = max_j |z[j]|                        (exact: the inputs are BF16)
+ *     scale  = a / 127,   inv = 127 / a            (each ONE binary32 division; a == 0: 1, 0)
+ *     q[j]   = clamp(rint(z[j] * inv), -127, 127)  (binary32 product, round half to even)
+ *
+ * The code is an integer decided by floating point, so the decision is taken in binary32,
+ * the precision the CUDA path uses, with exactly these operations in this order; nothing
+ * here runs in double.  Z [rows, cols] BF16 bits -> Q [rows, cols] int8, S [rows] float.
+ */
+int kx_oracle_quantize_rows(const uint16_t* Z, int64_t rows, int64_t cols, int8_t* Q, float* S) {
+    if (rows < 0 || cols < 0 || (rows > 0 && (!S || (cols > 0 && (!Z || !Q))))) return -1;
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < rows; ++r) {
+        float a = 0.0f;
+        for (int64_t j = 0; j < cols; ++j) {
+            const float v = fabsf((float)bf16_widen(Z[r * cols + j]));
+            if (v > a) a = v;
+        }
+        const float scale = (a > 0.0f) ? a / 127.0f : 1.0f;
+        const float inv = (a > 0.0f) ? 127.0f / a : 0.0f;
+        S[r] = scale;
+        for (int64_t j = 0; j < cols; ++j) {
+            const float z = (float)bf16_widen(Z[r * cols + j]);
+            float t = rintf(z * inv);
+            if (t > 127.0f) t = 127.0f;
+            if (t < -127.0f) t = -127.0f;
+            Q[r * cols + j] = (int8_t)t;
+        }
+    }
+    return 0;
+}
+
+/*
+ * Integer contraction with dequantisation: acc[m,n] = sum_k Xq[m,k] * Wq[n,k] (exact, int64),
+ * value = acc * sx[m] * sw[n] in double.  Used by the two functions below.
+ */
+static double dq_dot(const int8_t* x, const int8_t* w, int64_t K, float sx, float sw, int64_t* acc_out) {
+    int64_t acc = 0;
+    for (int64_t k = 0; k < K; ++k) acc += (int64_t)x[k] * (int64_t)w[k];
+    if (acc_out) *acc_out = acc;
+    return (double)acc * (double)sx * (double)sw;
+}
+
+/*
+ * Gate/up GEMM on INT8 codes with fused dequantisation and SwiGLU (Appendix A, Algorithm 7):
+ *     g = (Xq Wgq^T)[m,i] * sx[m] * sg[i],  u = (Xq Wuq^T)[m,i] * sx[m] * su[i],
+ *     z = g / (1 + exp(-g)) * u              (double, unrounded)
+ * Xq [M,K], Wgq / Wuq [I,K] int8; sx [M], sg / su [I] float; rows [nrows] or NULL;
+ * out [nrows, I]; gate_acc / up_acc [nrows, I] optional exact integer sums.
+ */
+int kx_oracle_swiglu_int8_rows(const int8_t* Xq, const float* sx, const int8_t* Wgq, const float* sg,
+                               const int8_t* Wuq, const float* su, const int64_t* rows, int64_t nrows,
+                               double* out, int64_t* gate_acc, int64_t* up_acc, int64_t M, int64_t I, int64_t K) {
+    if (M < 0 || I < 0 || K < 0 || nrows < 0 || !out || !sx || !sg || !su) return -1;
+    if (K > 0 && (!Xq || !Wgq || !Wuq)) return -1;
+    for (int64_t r = 0; rows && r < nrows; ++r)
+        if (rows[r] < 0 || rows[r] >= M) return -1;
+    if (!rows && nrows > M) return -1;
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int64_t r = 0; r < nrows; ++r) {
+        for (int64_t i = 0; i < I; ++i) {
+            const int64_t m = rows ? rows[r] : r;
+            int64_t ga = 0, ua = 0;
+            const double g = dq_dot(Xq + m * K, Wgq + i * K, K, sx[m], sg[i], &ga);
+            const double u = dq_dot(Xq + m * K, Wuq + i * K, K, sx[m], su[i], &ua);
+            out[r * I + i] = g / (1.0 + exp(-g)) * u;
+            if (gate_acc) gate_acc[r * I + i] = ga;
+            if (up_acc) up_acc[r * I + i] = ua;
+        }
+    }
+    return 0;
+}
+
+/*
+ * The output projection with residual on INT8 codes (the precision axis of the paper's strategy
+ * space, Section 3.2, applied to the operator of Appendix A, Algorithm 3):
+ *     y[m,n] = (Xq Wq^T)[m,n] * sx[m] * sw[n] + bias[n] + R[m,n]     (double, unrounded)
+ * bias [N] / R [M,N] BF16 bits or NULL.
+ */
+int kx_oracle_outproj_int8_rows(const int8_t* Xq, const float* sx, const int8_t* Wq, const float* sw,
+                                const uint16_t* bias, const uint16_t* R, const int64_t* rows, int64_t nrows,
+                                double* out, int64_t M, int64_t N, int64_t K) {
+    if (M < 0 || N < 0 || K < 0 || nrows < 0 || !out || !sx || !sw) return -1;
+    if (K > 0 && (!Xq || !Wq)) return -1;
+    for (int64_t r = 0; rows && r < nrows; ++r)
+        if (rows[r] < 0 || rows[r] >= M) return -1;
+    if (!rows && nrows > M) return -1;
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int64_t r = 0; r < nrows; ++r) {
+        for (int64_t n = 0; n < N; ++n) {
+            const int64_t m = rows ? rows[r] : r;
+            double y = dq_dot(Xq + m * K, Wq + n * K, K, sx[m], sw[n], 0);
+            if (bias) y += bf16_widen(bias[n]);
+            if (R) y += bf16_widen(R[m * N + n]);
+            out[r * N + n] = y;
+        }
+    }
+    return 0;
+}

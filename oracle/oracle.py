@@ -37,6 +37,9 @@ def _load():
         lib.kx_oracle_rmsnorm_rows.restype = ctypes.c_int
         lib.kx_oracle_swiglu_rows.argtypes = [p, p, p, p, i64, p, p, p, i64, i64, i64]
         lib.kx_oracle_swiglu_rows.restype = ctypes.c_int
+        lib.kx_oracle_quantize_rows.argtypes = [p, i64, i64, p, p]
+        lib.kx_oracle_swiglu_int8_rows.argtypes = [p, p, p, p, p, p, p, i64, p, p, p, i64, i64, i64]
+        lib.kx_oracle_outproj_int8_rows.argtypes = [p, p, p, p, p, p, p, i64, p, i64, i64, i64]
         lib.kx_oracle_max_threads.argtypes = []
         lib.kx_oracle_max_threads.restype = ctypes.c_int
         _lib = lib
@@ -167,3 +170,75 @@ def swiglu(X, Wg, Wu, rows=None, want_parts: bool = False):
         raise RuntimeError(f"kx_oracle_swiglu_rows failed ({rc})")
     return (out, g, u) if want_parts else out
 
+
+
+def _rows_arg(rows, M):
+    if rows is None:
+        return None, M
+    arr = np.ascontiguousarray(rows, dtype=np.int64)
+    return arr, int(arr.size)
+
+
+def _typed(a, dtype, shape, name):
+    a = np.ascontiguousarray(a)
+    if a.dtype != dtype or a.shape != tuple(shape):
+        raise ValueError(f"{name}: expected {np.dtype(dtype).name}{tuple(shape)}, got {a.dtype}{a.shape}")
+    return a
+
+
+def quantize_rows(Z):
+    """Symmetric per-row INT8 code book of BF16 rows (the activation / weight quantisation steps of
+    Appendix A, Algorithm 7): scale = max|z| / 127, q = clamp(rint(z * (127 / max|z|))), every
+    operation in binary32 (a zero row gets scale 1 and codes 0).  Z [rows, cols] uint16 BF16 bits
+    -> (Q int8 [rows, cols], S float32 [rows])."""
+    rows, cols = Z.shape
+    Z = _bits(Z, (rows, cols), "Z")
+    Q = np.empty((rows, cols), dtype=np.int8)
+    S = np.empty((rows,), dtype=np.float32)
+    rc = _load().kx_oracle_quantize_rows(_ptr(Z), rows, cols, _ptr(Q), _ptr(S))
+    if rc != 0:
+        raise RuntimeError(f"kx_oracle_quantize_rows failed ({rc})")
+    return Q, S
+
+
+def swiglu_int8(Xq, sx, Wgq, sg, Wuq, su, rows=None, want_acc: bool = False):
+    """z = silu(g) * u with g = (Xq Wgq^T) sx sg, u = (Xq Wuq^T) sx su: exact integer sums,
+    dequantised and combined in float64, unrounded (INT8 gate/up GEMM with fused dequantisation
+    and SwiGLU epilogue, Appendix A, Algorithm 7).  With `want_acc` also the two int64 sums."""
+    M, K = Xq.shape
+    I = Wgq.shape[0]
+    Xq = _typed(Xq, np.int8, (M, K), "Xq")
+    Wgq = _typed(Wgq, np.int8, (I, K), "Wgq")
+    Wuq = _typed(Wuq, np.int8, (I, K), "Wuq")
+    sx = _typed(sx, np.float32, (M,), "sx")
+    sg = _typed(sg, np.float32, (I,), "sg")
+    su = _typed(su, np.float32, (I,), "su")
+    rows_arr, nrows = _rows_arg(rows, M)
+    out = np.empty((nrows, I), dtype=np.float64)
+    ga = np.empty((nrows, I), dtype=np.int64) if want_acc else None
+    ua = np.empty((nrows, I), dtype=np.int64) if want_acc else None
+    rc = _load().kx_oracle_swiglu_int8_rows(_ptr(Xq), _ptr(sx), _ptr(Wgq), _ptr(sg), _ptr(Wuq), _ptr(su),
+                                            _ptr(rows_arr), nrows, _ptr(out), _ptr(ga), _ptr(ua), M, I, K)
+    if rc != 0:
+        raise RuntimeError(f"kx_oracle_swiglu_int8_rows failed ({rc})")
+    return (out, ga, ua) if want_acc else out
+
+
+def outproj_int8(Xq, sx, Wq, sw, bias=None, R=None, rows=None):
+    """y = (Xq Wq^T) sx sw + bias + R: exact integer sum, the rest in float64, unrounded (the
+    output projection with residual of Appendix A, Algorithm 3, on INT8 codes)."""
+    M, K = Xq.shape
+    N = Wq.shape[0]
+    Xq = _typed(Xq, np.int8, (M, K), "Xq")
+    Wq = _typed(Wq, np.int8, (N, K), "Wq")
+    sx = _typed(sx, np.float32, (M,), "sx")
+    sw = _typed(sw, np.float32, (N,), "sw")
+    bias = _bits(bias, (N,), "bias")
+    R = _bits(R, (M, N), "R")
+    rows_arr, nrows = _rows_arg(rows, M)
+    out = np.empty((nrows, N), dtype=np.float64)
+    rc = _load().kx_oracle_outproj_int8_rows(_ptr(Xq), _ptr(sx), _ptr(Wq), _ptr(sw), _ptr(bias), _ptr(R),
+                                             _ptr(rows_arr), nrows, _ptr(out), M, N, K)
+    if rc != 0:
+        raise RuntimeError(f"kx_oracle_outproj_int8_rows failed ({rc})")
+    return out
