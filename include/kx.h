@@ -258,6 +258,59 @@ int kx_outproj_residual_rmsnorm(const void* X, const void* W, const void* bias_o
 int kx_gate_up_swiglu(const void* X, const void* Wg, const void* Wu, void* Z,
                       int64_t M, int64_t I, int64_t K, void* stream);
 
+/*
+ * ---- INT8 branch of the decoder layer (Appendix A, Algorithm 7: "run fused add+RMSNorm+
+ * activation quantization", "quantize gate/up weights in one launch", "compute gate/up GEMM with
+ * fused dequantization and SwiGLU epilogue"; the residual add is already part of
+ * kx_outproj_residual).  The paper does not print the code book; this library uses the usual
+ * symmetric one, per row (per token for activations, per output channel for weights):
+ *     a = max_j |z_j|,  scale = a / 127,  q_j = clamp(rint(z_j * (127 / a)), -127, 127)
+ * every operation in binary32 (two correctly rounded divisions per row, one product and one
+ * round-half-to-even per element); a row of zeros gets scale 1 and codes 0.  Rows holding a NaN
+ * or an infinity give unspecified codes.
+ *
+ * All pointers are device pointers; codes are int8 row-major, scales FP32; matrices 16-byte
+ * aligned, scale vectors 16-byte aligned (the row scales of X only need 4); cols / K % 16 == 0
+ * (a row of codes is a whole number of 16-byte units), cols <= 32768 for the quantising calls.
+ * Work is enqueued on `stream`; errors are returned as for the other entry points.
+ */
+
+/* Q[rows,cols], S[rows] = code book of the BF16 matrix A[rows,cols].  Q and S must not overlap A
+ * or each other.  One launch, HBM-bound: 3 bytes per element. */
+int kx_quantize_rows_int8(const void* A, void* Q, float* S, int64_t rows, int64_t cols, void* stream);
+
+/* The same for the gate and the up weight matrices [I,K] in ONE launch (rows 0..I-1 of the grid
+ * take Wg, the rest Wu). */
+int kx_quantize_gate_up_int8(const void* Wg, const void* Wu, void* Qg, float* Sg, void* Qu, float* Su,
+                             int64_t I, int64_t K, void* stream);
+
+/* Q, S = code book of z = RMSNorm(H) * gamma, where z is the BF16-rounded result kx_rmsnorm
+ * would write (bit for bit) but never reaches memory: H [M,N] BF16 is read once (2 bytes per
+ * element), Q [M,N] int8 and S [M] written (1 byte per element).  eps >= 0. */
+int kx_rmsnorm_quantize_int8(const void* H, const void* gamma, float eps, void* Q, float* S,
+                             int64_t M, int64_t N, void* stream);
+
+/*
+ * Z[M,I] = silu(g) * u with g = (Xq Wgq^T) sx[m] sg[i], u = (Xq Wuq^T) sx[m] su[i]: INT8 gate/up
+ * GEMM (tcgen05 kind::i8, exact 32-bit integer accumulation in tensor memory) with the
+ * dequantisation and the SwiGLU product in the epilogue (FP32), one rounding to BF16.
+ *   Xq [M,K], Wgq / Wuq [I,K] int8; sx [M], sg / su [I] FP32; Z [M,I] BF16; I % 8 == 0.
+ *   |sum| must stay below 2^31 (K <= 133 000 for full-range codes).  OPs = 4 M I K.
+ */
+int kx_gate_up_swiglu_int8(const void* Xq, const float* sx, const void* Wgq, const float* sg,
+                           const void* Wuq, const float* su, void* Z,
+                           int64_t M, int64_t I, int64_t K, void* stream);
+
+/*
+ * Y[M,N] = (Xq Wq^T) sx[m] sw[n] + bias[n] + R[m,n]: the output projection with residual on INT8
+ * codes (the precision axis of the paper's strategy space, Section 3.2, applied to the operator
+ * of Algorithm 3).  bias / R as for kx_outproj_residual (NULL = absent; R may equal Y).
+ * Large-M tile kernel for every M (no small-M path).
+ */
+int kx_outproj_residual_int8(const void* Xq, const float* sx, const void* Wq, const float* sw,
+                             const void* bias_or_null, const void* R_or_null, void* Y,
+                             int64_t M, int64_t N, int64_t K, void* stream);
+
 /* Fills `out` with the plan the library would use for this shape on the current
  * device (has_residual / has_bias as 0 or 1).  No work is enqueued. */
 int kx_plan_query(int64_t M, int64_t N, int64_t K, int has_bias, int has_residual,

@@ -25,6 +25,8 @@ EXPORTS = (
     "kx_init", "kx_shutdown", "kx_outproj_residual", "kx_gemm_bf16", "kx_outproj_residual_ex",
     "kx_outproj_residual_host", "kx_outproj_residual_noalloc", "kx_rmsnorm", "kx_outproj_residual_rmsnorm",
     "kx_gate_up_swiglu",
+    "kx_quantize_rows_int8", "kx_quantize_gate_up_int8", "kx_rmsnorm_quantize_int8", "kx_gate_up_swiglu_int8",
+    "kx_outproj_residual_int8",
     "kx_plan_query", "kx_last_device_status", "kx_status_string",
     "kx_version",
 )
@@ -79,6 +81,11 @@ def load():
     lib.kx_rmsnorm.argtypes = [vp, vp, ctypes.c_float, vp, i64, i64, vp]
     lib.kx_gate_up_swiglu.argtypes = [vp, vp, vp, vp, i64, i64, i64, vp]
     lib.kx_outproj_residual_rmsnorm.argtypes = [vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, i64, i64, i64, vp]
+    lib.kx_quantize_rows_int8.argtypes = [vp, vp, vp, i64, i64, vp]
+    lib.kx_quantize_gate_up_int8.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, vp]
+    lib.kx_rmsnorm_quantize_int8.argtypes = [vp, vp, ctypes.c_float, vp, vp, i64, i64, vp]
+    lib.kx_gate_up_swiglu_int8.argtypes = [vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, vp]
+    lib.kx_outproj_residual_int8.argtypes = [vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, vp]
     lib.kx_plan_query.argtypes = [i64, i64, i64, ci, ci, ctypes.POINTER(PlanOverride), ctypes.POINTER(PlanInfo)]
     lib.kx_last_device_status.argtypes = [vp, ctypes.POINTER(ci), ctypes.POINTER(ci)]
     lib.kx_status_string.argtypes = [ci]
@@ -114,6 +121,14 @@ def _check_bf16(name, t, shape):
         return
     if t.dtype != torch.bfloat16 or not t.is_contiguous() or tuple(t.shape) != tuple(shape):
         raise ValueError(f"{name}: need a contiguous bfloat16 tensor of shape {tuple(shape)}, "
+                         f"got {t.dtype} {tuple(t.shape)} contiguous={t.is_contiguous()}")
+
+
+def _check(name, t, shape, dtype):
+    if t is None or isinstance(t, int):
+        return
+    if t.dtype != dtype or not t.is_contiguous() or tuple(t.shape) != tuple(shape):
+        raise ValueError(f"{name}: need a contiguous {dtype} tensor of shape {tuple(shape)}, "
                          f"got {t.dtype} {tuple(t.shape)} contiguous={t.is_contiguous()}")
 
 
@@ -213,6 +228,73 @@ def kx_gate_up_swiglu(X, Wg, Wu, Z, stream=None, M=None, I=None, K=None, check=T
     rc = load().kx_gate_up_swiglu(_addr(X), _addr(Wg), _addr(Wu), _addr(Z), M, I, K, _stream(stream))
     if check and rc != KX_OK:
         raise KxError(rc, "kx_gate_up_swiglu")
+    return rc
+
+
+def kx_quantize_rows_int8(A, Q, S, stream=None, check=True) -> int:
+    """Q (int8), S (float32 per row) = symmetric per-row INT8 code book of the BF16 matrix A."""
+    import torch
+    rows, cols = A.shape
+    _check_bf16("A", A, (rows, cols)); _check("Q", Q, (rows, cols), torch.int8); _check("S", S, (rows,), torch.float32)
+    rc = load().kx_quantize_rows_int8(_addr(A), _addr(Q), _addr(S), rows, cols, _stream(stream))
+    if check and rc != KX_OK:
+        raise KxError(rc, "kx_quantize_rows_int8")
+    return rc
+
+
+def kx_quantize_gate_up_int8(Wg, Wu, Qg, Sg, Qu, Su, stream=None, check=True) -> int:
+    """Code books of the gate and the up weight matrices in one launch."""
+    import torch
+    I, K = Wg.shape
+    _check_bf16("Wg", Wg, (I, K)); _check_bf16("Wu", Wu, (I, K))
+    _check("Qg", Qg, (I, K), torch.int8); _check("Qu", Qu, (I, K), torch.int8)
+    _check("Sg", Sg, (I,), torch.float32); _check("Su", Su, (I,), torch.float32)
+    rc = load().kx_quantize_gate_up_int8(_addr(Wg), _addr(Wu), _addr(Qg), _addr(Sg), _addr(Qu), _addr(Su), I, K,
+                                         _stream(stream))
+    if check and rc != KX_OK:
+        raise KxError(rc, "kx_quantize_gate_up_int8")
+    return rc
+
+
+def kx_rmsnorm_quantize_int8(H, gamma, eps: float, Q, S, stream=None, check=True) -> int:
+    """Q, S = code book of RMSNorm(H) * gamma (rounded to BF16 as kx_rmsnorm would), H read once."""
+    import torch
+    M, N = H.shape
+    _check_bf16("H", H, (M, N)); _check_bf16("gamma", gamma, (N,))
+    _check("Q", Q, (M, N), torch.int8); _check("S", S, (M,), torch.float32)
+    rc = load().kx_rmsnorm_quantize_int8(_addr(H), _addr(gamma), float(eps), _addr(Q), _addr(S), M, N, _stream(stream))
+    if check and rc != KX_OK:
+        raise KxError(rc, "kx_rmsnorm_quantize_int8")
+    return rc
+
+
+def kx_gate_up_swiglu_int8(Xq, sx, Wgq, sg, Wuq, su, Z, stream=None, check=True) -> int:
+    """Z = silu((Xq Wgq^T) sx sg) * ((Xq Wuq^T) sx su): INT8 GEMM, dequantisation and SwiGLU fused."""
+    import torch
+    M, K = Xq.shape
+    I = Wgq.shape[0]
+    _check("Xq", Xq, (M, K), torch.int8); _check("Wgq", Wgq, (I, K), torch.int8); _check("Wuq", Wuq, (I, K), torch.int8)
+    _check("sx", sx, (M,), torch.float32); _check("sg", sg, (I,), torch.float32); _check("su", su, (I,), torch.float32)
+    _check_bf16("Z", Z, (M, I))
+    rc = load().kx_gate_up_swiglu_int8(_addr(Xq), _addr(sx), _addr(Wgq), _addr(sg), _addr(Wuq), _addr(su), _addr(Z),
+                                       M, I, K, _stream(stream))
+    if check and rc != KX_OK:
+        raise KxError(rc, "kx_gate_up_swiglu_int8")
+    return rc
+
+
+def kx_outproj_residual_int8(Xq, sx, Wq, sw, bias, R, Y, stream=None, check=True) -> int:
+    """Y = (Xq Wq^T) sx sw + bias + R on INT8 codes; bias / R may be None; R may be Y."""
+    import torch
+    M, K = Xq.shape
+    N = Wq.shape[0]
+    _check("Xq", Xq, (M, K), torch.int8); _check("Wq", Wq, (N, K), torch.int8)
+    _check("sx", sx, (M,), torch.float32); _check("sw", sw, (N,), torch.float32)
+    _check_bf16("bias", bias, (N,)); _check_bf16("R", R, (M, N)); _check_bf16("Y", Y, (M, N))
+    rc = load().kx_outproj_residual_int8(_addr(Xq), _addr(sx), _addr(Wq), _addr(sw), _addr(bias), _addr(R), _addr(Y),
+                                         M, N, K, _stream(stream))
+    if check and rc != KX_OK:
+        raise KxError(rc, "kx_outproj_residual_int8")
     return rc
 
 

@@ -69,7 +69,8 @@ bool log_enabled() {
 // ------------------------------------------------------------------ kernel table
 struct TileVariant {
     int bn, ctas, stages, nb, smem;
-    const void* fn;
+    const void* fn;        // BF16 operands
+    const void* fn_s8;     // signed 8-bit operands, integer accumulators
 };
 struct SwapVariant {
     int bn, stages, smem;
@@ -80,7 +81,8 @@ struct SwapVariant {
 #define KX_TILE(BN, CTAS, ST, NB)                                                             \
     TileVariant {                                                                             \
         BN, CTAS, ST, NB, TileCfg<BN, CTAS, ST, NB>::SMEM_BYTES,                              \
-            reinterpret_cast<const void*>(&kx_tile_kernel<BN, CTAS, ST, NB>)                  \
+            reinterpret_cast<const void*>(&kx_tile_kernel<BN, CTAS, ST, NB, 0>),              \
+            reinterpret_cast<const void*>(&kx_tile_kernel<BN, CTAS, ST, NB, 1>)               \
     }
 #define KX_SWAP(BN, ST)                                                                       \
     SwapVariant {                                                                             \
@@ -151,8 +153,9 @@ int ensure_device(int dev, DeviceCtx** out) {
         }
         bool ok = true;
         for (const auto& v : kTileVariants)
-            ok = ok && cudaFuncSetAttribute(v.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, v.smem) ==
-                           cudaSuccess;
+            ok = ok &&
+                 cudaFuncSetAttribute(v.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, v.smem) == cudaSuccess &&
+                 cudaFuncSetAttribute(v.fn_s8, cudaFuncAttributeMaxDynamicSharedMemorySize, v.smem) == cudaSuccess;
         for (const auto& v : kSwapVariants)
             ok = ok &&
                  cudaFuncSetAttribute(v.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, v.smem) == cudaSuccess &&
@@ -194,9 +197,10 @@ int ensure_device(int dev, DeviceCtx** out) {
 struct TmapKey {
     const void* ptr;
     uint64_t rows, cols;
-    uint32_t box_rows;
+    uint32_t box_rows, elem_bytes;
     bool operator==(const TmapKey& o) const {
-        return ptr == o.ptr && rows == o.rows && cols == o.cols && box_rows == o.box_rows;
+        return ptr == o.ptr && rows == o.rows && cols == o.cols && box_rows == o.box_rows &&
+               elem_bytes == o.elem_bytes;
     }
 };
 struct TmapEntry {
@@ -207,14 +211,16 @@ struct TmapEntry {
 constexpr int kTmapSlots = 64;
 thread_local TmapEntry t_tmaps[kTmapSlots];
 
-// Row-major BF16 matrix [rows, cols]; box = box_rows x 64 columns; 128-byte swizzle;
-// 256-byte L2 promotion; out-of-bounds elements read as zero and are not written.
-int get_tmap(const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows, CUtensorMap* out) {
-    TmapKey key{ptr, rows, cols, box_rows};
+// Row-major matrix [rows, cols] of BF16 (elem_bytes 2) or 8-bit (elem_bytes 1) elements;
+// box = box_rows x 128 bytes of a row; 128-byte swizzle; 256-byte L2 promotion; out-of-bounds
+// elements read as zero and are not written.
+int get_tmap(const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows, CUtensorMap* out,
+             uint32_t elem_bytes = 2) {
+    TmapKey key{ptr, rows, cols, box_rows, elem_bytes};
     uint64_t h = reinterpret_cast<uint64_t>(ptr) >> 4;
     h ^= rows * 0x9E3779B97F4A7C15ull;
     h ^= (cols + 0x7F4A7C15ull) * 0xC2B2AE3D27D4EB4Full;
-    h ^= box_rows * 0x165667B19E3779F9ull;
+    h ^= (box_rows + 1024ull * elem_bytes) * 0x165667B19E3779F9ull;
     h ^= h >> 29;
     TmapEntry& e = t_tmaps[h % kTmapSlots];
     if (e.valid && e.key == key) {
@@ -222,10 +228,11 @@ int get_tmap(const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows, C
         return KX_OK;
     }
     cuuint64_t dims[2] = {cols, rows};
-    cuuint64_t strides[1] = {cols * 2};
-    cuuint32_t box[2] = {64, box_rows};
+    cuuint64_t strides[1] = {cols * elem_bytes};
+    cuuint32_t box[2] = {128u / elem_bytes, box_rows};
     cuuint32_t estr[2] = {1, 1};
-    CUresult r = g_encode(&e.map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides,
+    CUresult r = g_encode(&e.map, elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8,
+                          2, const_cast<void*>(ptr), dims, strides,
                           box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
@@ -257,6 +264,7 @@ struct Plan {
     int smem = 0;
     size_t ws_bytes = 0;
     const void* fn = nullptr;
+    const void* fn_s8 = nullptr;
     int launches = 1;
 };
 
@@ -422,6 +430,7 @@ int make_plan_from(long long M, long long N, long long K, const kx_plan_override
         pl->nb = v->nb;
         pl->smem = v->smem;
         pl->fn = v->fn;
+        pl->fn_s8 = v->fn_s8;
         pl->tiles_m = ceil_div(M, 128 * ctas);
         pl->tiles_n = ceil_div(N, bn);
         pl->units = pl->tiles_m * pl->tiles_n;
@@ -1088,6 +1097,286 @@ int kx_outproj_residual_rmsnorm(const void* X, const void* W, const void* bias, 
     rc = ensure_device(dev, &ctx);
     if (rc != KX_OK) return rc;
     return launch_rmsnorm(H, gamma, eps, Z, M, N, static_cast<cudaStream_t>(stream), ctx->sm_count);
+}
+
+// ---------------------------------------------------------------- INT8 branch
+namespace {
+bool aligned4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3u) == 0; }
+
+int launch_rowquant(const QuantParams& qp, bool norm, cudaStream_t stream, int sm_count) {
+    cudaLaunchConfig_t cfg;
+    std::memset(&cfg, 0, sizeof cfg);
+    const long long nvec = qp.N / 8;
+    const void* fn = nullptr;
+    int per_sm = 8;
+#define KX_QUANT_FN(NV) \
+    (norm ? reinterpret_cast<const void*>(&kx_rowquant_kernel<NV, true>) \
+          : reinterpret_cast<const void*>(&kx_rowquant_kernel<NV, false>))
+    if (nvec <= 1 * kNormThreads) { fn = KX_QUANT_FN(1); }
+    else if (nvec <= 2 * kNormThreads) { fn = KX_QUANT_FN(2); }
+    else if (nvec <= 4 * kNormThreads) { fn = KX_QUANT_FN(4); per_sm = 6; }
+    else if (nvec <= 8 * kNormThreads) { fn = KX_QUANT_FN(8); per_sm = 4; }
+    else { fn = KX_QUANT_FN(kNormVecs); per_sm = 2; }
+#undef KX_QUANT_FN
+    cfg.gridDim = dim3(static_cast<unsigned>(std::min<long long>(qp.M, static_cast<long long>(sm_count) * per_sm)), 1, 1);
+    cfg.blockDim = dim3(kNormThreads, 1, 1);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    QuantParams p = qp;
+    void* args[] = {&p};
+    if (cudaLaunchKernelExC(&cfg, fn, args) != cudaSuccess) {
+        cudaGetLastError();
+        return KX_ERR_CUDA;
+    }
+    return KX_OK;
+}
+
+// rows x cols BF16 source(s) -> int8 codes + one FP32 scale per row
+int validate_quant(const void* A, const void* Q, const float* S, long long rows, long long cols) {
+    if (rows < 0 || cols < 0 || rows > 0x7FFFFFFFll / 2) return KX_ERR_SHAPE;
+    if (rows == 0) return KX_OK;
+    if (!S) return KX_ERR_NULL;
+    if (!aligned4(S)) return KX_ERR_ALIGN;
+    if (cols == 0) return KX_OK;
+    if ((cols % 16) != 0 || cols > 8ll * kNormThreads * kNormVecs) return KX_ERR_SHAPE;
+    if (!A || !Q) return KX_ERR_NULL;
+    if (!aligned16(A) || !aligned16(Q)) return KX_ERR_ALIGN;
+    const size_t ab = static_cast<size_t>(rows) * cols * 2, qb = static_cast<size_t>(rows) * cols,
+                 sb = static_cast<size_t>(rows) * 4;
+    if (overlaps(Q, qb, A, ab) || overlaps(S, sb, A, ab) || overlaps(S, sb, Q, qb)) return KX_ERR_OVERLAP;
+    return KX_OK;
+}
+
+int device_ctx(DeviceCtx** ctx) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return KX_ERR_CUDA;
+    return ensure_device(dev, ctx);
+}
+
+// Shared launcher of the INT8 tile kernel.  swiglu: B = gate rows, B2 = up rows, N = output columns I.
+int run_s8(const void* Xq, const float* sx, const void* Wq, const float* sw, const void* Wq2, const float* sw2,
+           const void* bias, const void* R, void* Y, long long M, long long N, long long K, bool swiglu,
+           cudaStream_t stream) {
+    DeviceCtx* ctx = nullptr;
+    int rc = device_ctx(&ctx);
+    if (rc != KX_OK) return rc;
+    kx_plan_override ov;
+    std::memset(&ov, 0, sizeof ov);
+    ov.path = KX_PATH_TILE;
+    ov.stream_k = 1;          // whole tiles only: partial integer accumulators are never added as FP32
+    ov.no_table = 1;
+    if (swiglu) {
+        ov.block_n = 256;     // 128 gate + 128 up accumulator columns = 128 output columns per tile
+        ov.narrow_tail = 1;
+    }
+    Plan pl;
+    rc = make_plan_from(M, swiglu ? 2 * N : N, K, &ov, ctx->sm_count, &pl);
+    if (rc != KX_OK) return rc;
+    if (pl.kcluster > 1 || pl.stream_k) return KX_ERR_PLAN;
+    CUtensorMap tmA, tmB, tmB2, tmY, tmR;
+    if ((rc = get_tmap(Xq, M, K, 128, &tmA, 1)) != KX_OK) return rc;
+    if (swiglu) {
+        if ((rc = get_tmap(Wq, N, K, 128, &tmB, 1)) != KX_OK) return rc;
+        if ((rc = get_tmap(Wq2, N, K, 128, &tmB2, 1)) != KX_OK) return rc;
+    } else {
+        if ((rc = get_tmap(Wq, N, K, pl.bn / pl.ctas, &tmB, 1)) != KX_OK) return rc;
+        if (pl.narrow_tile0 < pl.units) {
+            if ((rc = get_tmap(Wq, N, K, pl.bn / 2 / pl.ctas, &tmB2, 1)) != KX_OK) return rc;
+        } else {
+            tmB2 = tmB;
+        }
+    }
+    if ((rc = get_tmap(Y, M, N, 32, &tmY)) != KX_OK) return rc;
+    if (R) {
+        if ((rc = get_tmap(R, M, N, 32, &tmR)) != KX_OK) return rc;
+    } else {
+        tmR = tmY;
+    }
+    TileParams p;
+    std::memset(&p, 0, sizeof p);
+    p.M = static_cast<int>(M);
+    p.N = static_cast<int>(N);
+    p.K = static_cast<int>(K);
+    p.tiles_m = pl.tiles_m;
+    p.tiles_n = pl.tiles_n;
+    p.num_tiles = pl.units;
+    p.raster_group = pl.raster_group;
+    p.has_bias = bias ? 1 : 0;
+    p.has_r = R ? 1 : 0;
+    p.swiglu = swiglu ? 1 : 0;
+    p.kcluster = 1;
+    p.sk_tile0 = pl.units;
+    p.narrow_tile0 = pl.narrow_tile0;
+    p.spin_limit_ns = 2000000000ull;
+    p.status = ctx->status;
+    p.ws = ctx->ws;
+    p.counters = ctx->counters;
+    p.sa = sx;
+    p.sb = sw;
+    p.sb2 = sw2;
+    cudaLaunchConfig_t cfg;
+    std::memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3(pl.grid, 1, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = pl.smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    int nattr = 0;
+    attr[nattr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[nattr].val.programmaticStreamSerializationAllowed = 1;
+    ++nattr;
+    if (pl.ctas == 2) {
+        attr[nattr].id = cudaLaunchAttributeClusterDimension;
+        attr[nattr].val.clusterDim.x = 2;
+        attr[nattr].val.clusterDim.y = 1;
+        attr[nattr].val.clusterDim.z = 1;
+        ++nattr;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = nattr;
+    const uint16_t* bias_p = static_cast<const uint16_t*>(bias);
+    void* args[] = {&tmA, &tmB, &tmB2, &tmY, &tmR, &bias_p, &p};
+    if (cudaLaunchKernelExC(&cfg, pl.fn_s8, args) != cudaSuccess) {
+        cudaGetLastError();
+        return KX_ERR_CUDA;
+    }
+    return KX_OK;
+}
+}  // namespace
+
+int kx_quantize_rows_int8(const void* A, void* Q, float* S, int64_t rows, int64_t cols, void* stream) {
+    int rc = validate_quant(A, Q, S, rows, cols);
+    if (rc != KX_OK) return rc;
+    if (rows == 0) return KX_OK;
+    DeviceCtx* ctx = nullptr;
+    if ((rc = device_ctx(&ctx)) != KX_OK) return rc;
+    QuantParams qp;
+    std::memset(&qp, 0, sizeof qp);
+    qp.A0 = qp.A1 = static_cast<const uint16_t*>(A);
+    qp.Q0 = qp.Q1 = static_cast<int8_t*>(Q);
+    qp.S0 = qp.S1 = S;
+    qp.rows0 = rows;
+    qp.M = rows;
+    qp.N = static_cast<int>(cols);
+    return launch_rowquant(qp, false, static_cast<cudaStream_t>(stream), ctx->sm_count);
+}
+
+int kx_quantize_gate_up_int8(const void* Wg, const void* Wu, void* Qg, float* Sg, void* Qu, float* Su, int64_t I,
+                             int64_t K, void* stream) {
+    int rc = validate_quant(Wg, Qg, Sg, I, K);
+    if (rc == KX_OK) rc = validate_quant(Wu, Qu, Su, I, K);
+    if (rc != KX_OK) return rc;
+    if (I == 0) return KX_OK;
+    const size_t qb = static_cast<size_t>(I) * K, sb = static_cast<size_t>(I) * 4, wb = qb * 2;
+    if (overlaps(Qg, qb, Qu, qb) || overlaps(Sg, sb, Su, sb) || overlaps(Qg, qb, Wu, wb) || overlaps(Qu, qb, Wg, wb) ||
+        overlaps(Sg, sb, Qu, qb) || overlaps(Su, sb, Qg, qb) || overlaps(Sg, sb, Wu, wb) || overlaps(Su, sb, Wg, wb))
+        return KX_ERR_OVERLAP;
+    DeviceCtx* ctx = nullptr;
+    if ((rc = device_ctx(&ctx)) != KX_OK) return rc;
+    QuantParams qp;
+    std::memset(&qp, 0, sizeof qp);
+    qp.A0 = static_cast<const uint16_t*>(Wg);
+    qp.A1 = static_cast<const uint16_t*>(Wu);
+    qp.Q0 = static_cast<int8_t*>(Qg);
+    qp.Q1 = static_cast<int8_t*>(Qu);
+    qp.S0 = Sg;
+    qp.S1 = Su;
+    qp.rows0 = I;
+    qp.M = 2 * I;
+    qp.N = static_cast<int>(K);
+    return launch_rowquant(qp, false, static_cast<cudaStream_t>(stream), ctx->sm_count);
+}
+
+int kx_rmsnorm_quantize_int8(const void* H, const void* gamma, float eps, void* Q, float* S, int64_t M, int64_t N,
+                             void* stream) {
+    int rc = validate_quant(H, Q, S, M, N);
+    if (rc != KX_OK) return rc;
+    if (!(eps >= 0.0f)) return KX_ERR_SHAPE;
+    if (M == 0) return KX_OK;
+    if (N > 0) {
+        if (!gamma) return KX_ERR_NULL;
+        if (!aligned16(gamma)) return KX_ERR_ALIGN;
+        if (overlaps(Q, static_cast<size_t>(M) * N, gamma, static_cast<size_t>(N) * 2) ||
+            overlaps(S, static_cast<size_t>(M) * 4, gamma, static_cast<size_t>(N) * 2))
+            return KX_ERR_OVERLAP;
+    }
+    DeviceCtx* ctx = nullptr;
+    if ((rc = device_ctx(&ctx)) != KX_OK) return rc;
+    QuantParams qp;
+    std::memset(&qp, 0, sizeof qp);
+    qp.A0 = qp.A1 = static_cast<const uint16_t*>(H);
+    qp.gamma = static_cast<const uint16_t*>(gamma);
+    qp.Q0 = qp.Q1 = static_cast<int8_t*>(Q);
+    qp.S0 = qp.S1 = S;
+    qp.rows0 = M;
+    qp.M = M;
+    qp.N = static_cast<int>(N);
+    qp.eps = eps;
+    return launch_rowquant(qp, N > 0, static_cast<cudaStream_t>(stream), ctx->sm_count);
+}
+
+namespace {
+int validate_s8(const void* Xq, const float* sx, const void* Wq, const float* sw, const void* Y, long long M,
+                long long N, long long K) {
+    if (M < 0 || N < 0 || K < 0) return KX_ERR_SHAPE;
+    if (M > 0x7FFFFFFFll / 2 || N > 0x7FFFFFFFll / 4 || K > 0x7FFFFFFFll / 2) return KX_ERR_SHAPE;
+    if (M == 0 || N == 0) return KX_OK;
+    if ((N % 8) != 0 || (K % 16) != 0) return KX_ERR_SHAPE;
+    if (!Y) return KX_ERR_NULL;
+    if (!aligned16(Y)) return KX_ERR_ALIGN;
+    if (K == 0) return KX_OK;
+    if (!Xq || !Wq || !sx || !sw) return KX_ERR_NULL;
+    if (!aligned16(Xq) || !aligned16(Wq) || !aligned4(sx) || !aligned16(sw)) return KX_ERR_ALIGN;
+    const size_t yb = static_cast<size_t>(M) * N * 2;
+    if (overlaps(Y, yb, Xq, static_cast<size_t>(M) * K) || overlaps(Y, yb, Wq, static_cast<size_t>(N) * K) ||
+        overlaps(Y, yb, sx, static_cast<size_t>(M) * 4) || overlaps(Y, yb, sw, static_cast<size_t>(N) * 4))
+        return KX_ERR_OVERLAP;
+    return KX_OK;
+}
+}  // namespace
+
+int kx_gate_up_swiglu_int8(const void* Xq, const float* sx, const void* Wgq, const float* sg, const void* Wuq,
+                           const float* su, void* Z, int64_t M, int64_t I, int64_t K, void* stream_v) {
+    int rc = validate_s8(Xq, sx, Wgq, sg, Z, M, I, K);
+    if (rc == KX_OK) rc = validate_s8(Xq, sx, Wuq, su, Z, M, I, K);
+    if (rc != KX_OK) return rc;
+    if (M == 0 || I == 0) return KX_OK;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    if (K == 0) {   // empty sums: silu(0) * 0 = 0
+        DeviceCtx* ctx = nullptr;
+        if ((rc = device_ctx(&ctx)) != KX_OK) return rc;
+        const long long total = M * I;
+        const int blocks = static_cast<int>(std::min<long long>((total + 255) / 256, ctx->sm_count * 8));
+        kx_k0_kernel<<<blocks, 256, 0, stream>>>(nullptr, nullptr, static_cast<uint16_t*>(Z), M, I);
+        return cudaGetLastError() == cudaSuccess ? KX_OK : KX_ERR_CUDA;
+    }
+    return run_s8(Xq, sx, Wgq, sg, Wuq, su, nullptr, nullptr, Z, M, I, K, true, stream);
+}
+
+int kx_outproj_residual_int8(const void* Xq, const float* sx, const void* Wq, const float* sw, const void* bias,
+                             const void* R, void* Y, int64_t M, int64_t N, int64_t K, void* stream_v) {
+    int rc = validate_s8(Xq, sx, Wq, sw, Y, M, N, K);
+    if (rc != KX_OK) return rc;
+    if (M == 0 || N == 0) return KX_OK;
+    if ((bias && !aligned16(bias)) || (R && !aligned16(R))) return KX_ERR_ALIGN;
+    const size_t yb = static_cast<size_t>(M) * N * 2;
+    if (overlaps(Y, yb, bias, static_cast<size_t>(N) * 2)) return KX_ERR_OVERLAP;
+    if (R && R != Y && overlaps(Y, yb, R, yb)) return KX_ERR_OVERLAP;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    if (K == 0) {
+        DeviceCtx* ctx = nullptr;
+        if ((rc = device_ctx(&ctx)) != KX_OK) return rc;
+        const long long total = M * N;
+        const int blocks = static_cast<int>(std::min<long long>((total + 255) / 256, ctx->sm_count * 8));
+        kx_k0_kernel<<<blocks, 256, 0, stream>>>(static_cast<const uint16_t*>(bias), static_cast<const uint16_t*>(R),
+                                                 static_cast<uint16_t*>(Y), M, N);
+        return cudaGetLastError() == cudaSuccess ? KX_OK : KX_ERR_CUDA;
+    }
+    return run_s8(Xq, sx, Wq, sw, nullptr, nullptr, bias, R, Y, M, N, K, false, stream);
 }
 
 // ---------------------------------------------------------------- no-allocation entry

@@ -119,6 +119,9 @@ struct TileParams {
     int has_bias, has_r;
     int drop_kblocks;
     int pf_kblocks;            // L2 prefetch depth before the dependency wait (0 = ring depth, <0 = none)
+    const float* sa;           // KIND 1: scale per row of A [M]
+    const float* sb;           // KIND 1: scale per row of B [N] (gate rows in gate/up mode)
+    const float* sb2;          // KIND 1, gate/up mode: scale per up row [N]
     int swiglu;                   // 1: gate/up mode.  W rows of a tile = BN/2 rows of Wg (tmB) followed by the same
                                   // BN/2 rows of Wu (tmB2); the epilogue writes silu(gate) * up, BN/2 columns per
                                   // tile, N = number of output columns; no bias, no residual
@@ -209,7 +212,11 @@ __device__ __forceinline__ uint32_t ld_acquire_gpu_u32(const unsigned int* p) {
     return v;
 }
 
-template <int BN, int CTAS, int STAGES, int NB>
+// KIND 0: BF16 operands, FP32 accumulators.  KIND 1: signed 8-bit operands (a k-block is 128
+// codes = the same 128 bytes per row), 32-bit integer accumulators, dequantised in the epilogue
+// with a per-row scale of A and a per-row scale of B (stream-K and K-cluster plans, which add
+// partial accumulators as FP32, are not used with KIND 1).
+template <int BN, int CTAS, int STAGES, int NB, int KIND = 0>
 __global__ void __launch_bounds__(kThreads, 1)
 kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmB2, const __grid_constant__ CUtensorMap tmY,
@@ -236,7 +243,8 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int lane = threadIdx.x & 31;
     const uint32_t cta_rank = (CTAS == 2) ? cluster_ctarank() : 0u;
     const bool leader = (cta_rank == 0);
-    const int nkb = (p.K + kBlockK - 1) / kBlockK;
+    constexpr int KBLK = (KIND == 1) ? 2 * kBlockK : kBlockK;   // elements per k-block (128 bytes)
+    const int nkb = (p.K + KBLK - 1) / KBLK;
     const int kc = (CTAS == 1 && p.kcluster > 1) ? p.kcluster : 1;   // K-cluster size
     const int krank = (kc > 1) ? static_cast<int>(cluster_ctarank()) : 0;
     const int slot = blockIdx.x / (CTAS * kc);
@@ -281,9 +289,9 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     sg ? ((CTAS == 2 && cta_rank == 1) ? &tmB2 : &tmB) : (narrow ? &tmB2 : &tmB);
                 const int depth = p.pf_kblocks == 0 ? STAGES : p.pf_kblocks;
                 for (int kb = k0; kb < k1 && kb < k0 + depth; ++kb) {
-                    tma_prefetch_l2_2d(&tmA, kb * kBlockK, a_row);
-                    tma_prefetch_l2_2d(mapB, kb * kBlockK, b_row);
-                    if (CTAS == 1 && sg) tma_prefetch_l2_2d(&tmB2, kb * kBlockK, b_row);
+                    tma_prefetch_l2_2d(&tmA, kb * KBLK, a_row);
+                    tma_prefetch_l2_2d(mapB, kb * KBLK, b_row);
+                    if (CTAS == 1 && sg) tma_prefetch_l2_2d(&tmB2, kb * KBLK, b_row);
                 }
             }
         }
@@ -355,15 +363,15 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     const uint32_t sb = sa + kABytes;
                     if constexpr (CTAS == 1) {
                         mbar_arrive_expect_tx(full(s), stage_tx);
-                        tma_load_2d(sa, &tmA, kb * kBlockK, a_row, full(s));
-                        tma_load_2d(sb, mapB, kb * kBlockK, b_row, full(s));
-                        if (sg) tma_load_2d(sb + C::B_BYTES / 2, &tmB2, kb * kBlockK, b_row, full(s));
+                        tma_load_2d(sa, &tmA, kb * KBLK, a_row, full(s));
+                        tma_load_2d(sb, mapB, kb * KBLK, b_row, full(s));
+                        if (sg) tma_load_2d(sb + C::B_BYTES / 2, &tmB2, kb * KBLK, b_row, full(s));
                     } else {
                         // both CTAs' copies complete on the leader's barrier
                         if (leader) mbar_arrive_expect_tx(full(s), 2 * stage_tx);
                         const uint32_t fb = map_to_cta(full(s), 0);
-                        tma_load_2d_pair(sa, &tmA, kb * kBlockK, a_row, fb);
-                        tma_load_2d_pair(sb, mapB, kb * kBlockK, b_row, fb);
+                        tma_load_2d_pair(sa, &tmA, kb * KBLK, a_row, fb);
+                        tma_load_2d_pair(sb, mapB, kb * KBLK, b_row, fb);
                     }
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
@@ -377,8 +385,9 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     } else if (warp == 5) {
         // ------------------------------------------------------------ MMA issuer
         if (leader && lane == 0) {
-            constexpr uint32_t idesc_wide = idesc_bf16_f32(128 * CTAS, BN);
-            constexpr uint32_t idesc_narrow = idesc_bf16_f32(128 * CTAS, BN / 2);
+            constexpr uint32_t idesc_wide = KIND == 1 ? idesc_s8_s32(128 * CTAS, BN) : idesc_bf16_f32(128 * CTAS, BN);
+            constexpr uint32_t idesc_narrow =
+                KIND == 1 ? idesc_s8_s32(128 * CTAS, BN / 2) : idesc_bf16_f32(128 * CTAS, BN / 2);
             uint32_t s = 0, ph = 0, scount = 0;
             bool ok = true;
             while (ok && it.next(tile, kb0, kb1)) {
@@ -396,9 +405,14 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     const uint32_t sa = s_stage + s * C::STAGE_BYTES;
                     const uint32_t sb = sa + kABytes;
 #pragma unroll
-                    for (int k = 0; k < 4; ++k)
-                        mma_bf16<CTAS>(d, smem_desc_sw128(sa + k * 32), smem_desc_sw128(sb + k * 32), idesc,
-                                       static_cast<uint32_t>((kb - kb0) | k));
+                    for (int k = 0; k < 4; ++k) {
+                        if constexpr (KIND == 1)
+                            mma_s8<CTAS>(d, smem_desc_sw128(sa + k * 32), smem_desc_sw128(sb + k * 32), idesc,
+                                         static_cast<uint32_t>((kb - kb0) | k));
+                        else
+                            mma_bf16<CTAS>(d, smem_desc_sw128(sa + k * 32), smem_desc_sw128(sb + k * 32), idesc,
+                                           static_cast<uint32_t>((kb - kb0) | k));
+                    }
                     if constexpr (CTAS == 1) {
                         mma_commit<1>(empty(s));
                     } else {
@@ -446,6 +460,24 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         // K-cluster mode: a CTA's partial tile parked at the start of its (idle) operand ring, same
         // float4 order as slab4; `ring` is the shared::cta address of this CTA's copy
         const uint32_t ring = s_stage;
+        // KIND 1: integer accumulators -> FP32, times the scale of this lane's A row and of each B row
+        float a_scale = 0.f;
+        auto dequant_half = [&](uint32_t (&a)[32], const float* __restrict__ sb, int n0) {
+#pragma unroll
+            for (int g = 0; g < 8; ++g) {
+                const int n = n0 + g * 4;
+                const float4 s4 = (n + 4 <= p.N) ? __ldg(reinterpret_cast<const float4*>(sb + n))
+                                                 : make_float4(0.f, 0.f, 0.f, 0.f);
+                a[g * 4 + 0] = __float_as_uint(static_cast<float>(static_cast<int>(a[g * 4 + 0])) * (a_scale * s4.x));
+                a[g * 4 + 1] = __float_as_uint(static_cast<float>(static_cast<int>(a[g * 4 + 1])) * (a_scale * s4.y));
+                a[g * 4 + 2] = __float_as_uint(static_cast<float>(static_cast<int>(a[g * 4 + 2])) * (a_scale * s4.z));
+                a[g * 4 + 3] = __float_as_uint(static_cast<float>(static_cast<int>(a[g * 4 + 3])) * (a_scale * s4.w));
+            }
+        };
+        auto dequant = [&](uint32_t (&a0)[32], uint32_t (&a1)[32], const float* __restrict__ sb, int n0) {
+            dequant_half(a0, sb, n0);
+            dequant_half(a1, sb, n0 + 32);
+        };
 
         // partial of (slot sl, tile tl) for this CTA rank: "head" if tl is the first tile the slot touches
         auto part_ptr = [&](int sl, int tl) -> float* {
@@ -463,6 +495,7 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const bool sg = p.swiglu != 0;
             if (sg) colbase /= 2;                          // BN/2 output columns per tile
             const int row0 = tm * (128 * CTAS) + static_cast<int>(cta_rank) * 128 + q * 32;
+            if constexpr (KIND == 1) a_scale = (row0 + lane < p.M) ? __ldg(p.sa + row0 + lane) : 0.f;
             const int nchunks = (narrow || sg) ? C::CHUNKS / 2 : C::CHUNKS;
             const bool whole = (kb0 == 0) && (kb1 == nkb);
             auto chunk_inb = [&](int c) { return (row0 < p.M) && (colbase + c * 64 < p.N); };
@@ -635,6 +668,7 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     tmem_ld_32x32(tbase + c * 64, acc[0]);
                     tmem_ld_32x32(tbase + c * 64 + 32, acc[1]);
                     tmem_ld_wait();
+                    if constexpr (KIND == 1) dequant(acc[0], acc[1], p.sb, col0);
                 }
                 if (valid && sg) {
                     // acc holds the gate pre-activations of these 64 output columns; the matching up
@@ -644,6 +678,7 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         uint32_t up[32];
                         tmem_ld_32x32(tbase + BN / 2 + c * 64 + h * 32, up);
                         tmem_ld_wait();
+                        if constexpr (KIND == 1) dequant_half(up, p.sb2, col0 + h * 32);
 #pragma unroll
                         for (int i = 0; i < 32; ++i) {
                             const float gte = __uint_as_float(acc[h][i]);
@@ -1296,6 +1331,141 @@ kx_rmsnorm_kernel(const uint16_t* __restrict__ H, const uint16_t* __restrict__ g
             }
         }
         __syncthreads();         // s_part / s_inv are reused by the next row
+    }
+}
+
+// ===========================================================================
+// kx_rowquant_kernel
+// ===========================================================================
+// Symmetric per-row INT8 code book (the "activation quantization" fused behind add+RMSNorm and the
+// one-launch gate/up weight quantisation of Appendix A, Algorithm 7):
+//     a = max_j |z_j|,  scale = a / 127,  q_j = clamp(rint(z_j * (127 / a)), -127, 127)
+// with every operation in binary32 (one correctly rounded division each for scale and reciprocal,
+// one product and a round-half-even per element); a zero row gets scale 1 and codes 0.
+// NORM = true: z is the BF16-rounded RMSNorm of the row (same expression, so the same bits, as
+// kx_rmsnorm_kernel) and is never written to memory.  NORM = false: z is the row itself.
+// Rows [0, rows0) come from A0 -> Q0 / S0, rows [rows0, M) from A1 -> Q1 / S1, so that two
+// matrices of the same width (gate and up weights) are quantised by one launch.
+// HBM-bound: 2 N bytes read, N + 4 written per row.
+struct QuantParams {
+    const uint16_t* A0;
+    const uint16_t* A1;
+    const uint16_t* gamma;
+    int8_t* Q0;
+    int8_t* Q1;
+    float* S0;
+    float* S1;
+    long long rows0, M;
+    int N;
+    float eps;
+};
+
+template <int NV, bool NORM>
+__global__ void __launch_bounds__(kNormThreads)
+kx_rowquant_kernel(const QuantParams p) {
+    __shared__ float s_part[kNormThreads / 32];
+    __shared__ float s_bcast;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int N = p.N, nvec = N / 8;
+    pdl_wait_prior();
+    pdl_launch_dependents();
+    for (long long m = blockIdx.x; m < p.M; m += gridDim.x) {
+        const bool second = m >= p.rows0;
+        const long long r = second ? m - p.rows0 : m;
+        const uint4* row = reinterpret_cast<const uint4*>((second ? p.A1 : p.A0) + r * N);
+        uint4 v[NV];
+        float ss = 0.f;
+#pragma unroll
+        for (int i = 0; i < NV; ++i) {
+            const int idx = tid + i * kNormThreads;
+            if (idx < nvec) {
+                v[i] = row[idx];
+                if (NORM) {
+                    const uint32_t w4[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const float a = bf16_lo(w4[k]), b = bf16_hi(w4[k]);
+                        ss += a * a;
+                        ss += b * b;
+                    }
+                }
+            }
+        }
+        if (NORM) {
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+            if (lane == 0) s_part[warp] = ss;
+            __syncthreads();
+            if (tid == 0) {
+                float t = 0.f;
+#pragma unroll
+                for (int w = 0; w < kNormThreads / 32; ++w) t += s_part[w];
+                s_bcast = rsqrtf(t / static_cast<float>(N) + p.eps);
+            }
+            __syncthreads();
+            const float inv = s_bcast;
+            __syncthreads();     // s_part / s_bcast are reused for the maximum below
+#pragma unroll
+            for (int i = 0; i < NV; ++i) {
+                const int idx = tid + i * kNormThreads;
+                if (idx < nvec) {
+                    const uint4 g = __ldg(reinterpret_cast<const uint4*>(p.gamma) + idx);
+                    const uint32_t h4[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
+                    const uint32_t g4[4] = {g.x, g.y, g.z, g.w};
+                    uint32_t o4[4];
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        o4[k] = pack_bf16x2(bf16_lo(h4[k]) * inv * bf16_lo(g4[k]),
+                                            bf16_hi(h4[k]) * inv * bf16_hi(g4[k]));
+                    v[i] = make_uint4(o4[0], o4[1], o4[2], o4[3]);
+                }
+            }
+        }
+        // row maximum of |z| (exact: BF16 values, compared as binary32)
+        float amax = 0.f;
+#pragma unroll
+        for (int i = 0; i < NV; ++i) {
+            const int idx = tid + i * kNormThreads;
+            if (idx < nvec) {
+                const uint32_t w4[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
+#pragma unroll
+                for (int k = 0; k < 4; ++k) amax = fmaxf(amax, fmaxf(fabsf(bf16_lo(w4[k])), fabsf(bf16_hi(w4[k]))));
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+        if (lane == 0) s_part[warp] = amax;
+        __syncthreads();
+        if (tid == 0) {
+            float t = 0.f;
+#pragma unroll
+            for (int w = 0; w < kNormThreads / 32; ++w) t = fmaxf(t, s_part[w]);
+            s_bcast = t;
+            (second ? p.S1 : p.S0)[r] = (t > 0.f) ? __fdiv_rn(t, 127.0f) : 1.0f;
+        }
+        __syncthreads();
+        const float a = s_bcast;
+        const float rcp = (a > 0.f) ? __fdiv_rn(127.0f, a) : 0.f;
+        uint2* qrow = reinterpret_cast<uint2*>((second ? p.Q1 : p.Q0) + r * N);
+#pragma unroll
+        for (int i = 0; i < NV; ++i) {
+            const int idx = tid + i * kNormThreads;
+            if (idx < nvec) {
+                const uint32_t w4[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
+                uint32_t o[2] = {0u, 0u};
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    int q0 = __float2int_rn(__fmul_rn(bf16_lo(w4[k]), rcp));
+                    int q1 = __float2int_rn(__fmul_rn(bf16_hi(w4[k]), rcp));
+                    q0 = max(-127, min(127, q0));
+                    q1 = max(-127, min(127, q1));
+                    o[k >> 1] |= ((static_cast<uint32_t>(q0) & 0xFFu) | ((static_cast<uint32_t>(q1) & 0xFFu) << 8))
+                                 << ((k & 1) * 16);
+                }
+                qrow[idx] = make_uint2(o[0], o[1]);
+            }
+        }
+        __syncthreads();         // s_part / s_bcast are reused by the next row
     }
 }
 
