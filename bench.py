@@ -469,6 +469,99 @@ def run_ours(args):
             del keep, calls
             torch.cuda.empty_cache()
 
+    # ---- INT8 branch: code-book kernels (HBM-bound) and INT8 GEMMs (tensor-bound; the INT8 peak is
+    # taken as twice the measured BF16 GEMM peak, the nominal ratio of the two tensor-core rates)
+    int8 = []
+    if rank == 0 and world == 1 and not args.no_sweep:
+        lib = kx.load()
+        import ctypes
+        vp, i64 = ctypes.c_void_p, ctypes.c_int64
+        st = vp(int(torch.cuda.current_stream().cuda_stream) or None)
+        peak8 = 2.0 * peaks["bf16_tflops"]
+        g = torch.Generator(device="cuda")
+        g.manual_seed(8)
+
+        def report(name, t, tbest, nbytes, ops, ns):
+            bound = "tensor" if ops / (peak8 * 1e12) > nbytes / (peaks["hbm_gbs"] * 1e9) else "hbm"
+            frac = (ops / t / 1e12 / peak8) if bound == "tensor" else (nbytes / t / 1e9 / peaks["hbm_gbs"])
+            int8.append({"name": name, "us": t * 1e6, "us_best": tbest * 1e6, "tops": ops / t / 1e12,
+                         "gbs": nbytes / t / 1e9, "bound": bound, "frac": frac,
+                         "peak": peak8 if bound == "tensor" else peaks["hbm_gbs"], "operand_sets": ns})
+            print(f"[bench] {name:>30s} {t*1e6:9.1f} us (best {tbest*1e6:7.1f}) {ops/t/1e12:8.1f} TOP/s {nbytes/t/1e9:7.0f} GB/s  "
+                  f"{bound:6s} {frac*100:5.1f}% of {peaks['source']}", file=sys.stderr, flush=True)
+
+        for (Mn, Nn) in [(4096, 4096), (16384, 4096)]:
+            nbytes = 3.0 * Mn * Nn + 4.0 * Mn + 2.0 * Nn
+            ns = int(max(2, min(24, math.ceil(2.0 * L2_BYTES / nbytes))))
+            gam = torch.randn(Nn, device="cuda", generator=g).bfloat16()
+            keep, calls = [], []
+            for _ in range(ns):
+                Hn = torch.randn(Mn, Nn, device="cuda", generator=g).bfloat16()
+                Qn = torch.empty(Mn, Nn, dtype=torch.int8, device="cuda")
+                Sn = torch.empty(Mn, dtype=torch.float32, device="cuda")
+                keep.append((Hn, Qn, Sn))
+                a = (vp(Hn.data_ptr()), vp(gam.data_ptr()), ctypes.c_float(1e-6), vp(Qn.data_ptr()), vp(Sn.data_ptr()),
+                     i64(Mn), i64(Nn), st)
+                calls.append(lambda a=a: lib.kx_rmsnorm_quantize_int8(*a))
+            wlq = inputs.Workload(f"rmsnorm_quantize_{Mn}x{Nn}", Mn, Nn, 8, 0, False, False)
+            t, tbest, _ = time_shape(torch, kx, wlq, calls)
+            report(wlq.name, t, tbest, nbytes, 0.0, ns)
+            del keep, calls
+            torch.cuda.empty_cache()
+        for (Ms, Is, Ks) in [(16384, 14336, 4096), (4096, 14336, 4096), (512, 14336, 4096)]:
+            ops = 4.0 * Ms * Is * Ks
+            nbytes = 1.0 * (Ms * Ks + 2 * Is * Ks) + 2.0 * Ms * Is + 4.0 * (Ms + 2 * Is)
+            ns = int(max(2, min(8, math.ceil(2.0 * L2_BYTES / nbytes))))
+            keep, calls = [], []
+            for _ in range(ns):
+                Xq = torch.randint(-127, 128, (Ms, Ks), device="cuda", generator=g, dtype=torch.int8)
+                Wgq = torch.randint(-127, 128, (Is, Ks), device="cuda", generator=g, dtype=torch.int8)
+                Wuq = torch.randint(-127, 128, (Is, Ks), device="cuda", generator=g, dtype=torch.int8)
+                sx = torch.rand(Ms, device="cuda", generator=g) * 2e-2
+                sg = torch.rand(Is, device="cuda", generator=g) * 2e-4
+                su = torch.rand(Is, device="cuda", generator=g) * 2e-4
+                Zs = torch.empty(Ms, Is, dtype=torch.bfloat16, device="cuda")
+                keep.append((Xq, Wgq, Wuq, sx, sg, su, Zs))
+                a = (vp(Xq.data_ptr()), vp(sx.data_ptr()), vp(Wgq.data_ptr()), vp(sg.data_ptr()), vp(Wuq.data_ptr()),
+                     vp(su.data_ptr()), vp(Zs.data_ptr()), i64(Ms), i64(Is), i64(Ks), st)
+                calls.append(lambda a=a: lib.kx_gate_up_swiglu_int8(*a))
+            wls = inputs.Workload(f"swiglu_int8_M{Ms}_I{Is}_K{Ks}", Ms, 2 * Is, Ks, 0, False, False)
+            t, tbest, _ = time_shape(torch, kx, wls, calls)
+            report(wls.name, t, tbest, nbytes, ops, ns)
+            if Ms == 4096:   # the one-launch weight quantisation that feeds it
+                Wg = torch.randn(Is, Ks, device="cuda", generator=g).bfloat16()
+                Wu = torch.randn(Is, Ks, device="cuda", generator=g).bfloat16()
+                Xq, Wgq, Wuq, sx, sg, su, Zs = keep[0]
+                a = (vp(Wg.data_ptr()), vp(Wu.data_ptr()), vp(Wgq.data_ptr()), vp(sg.data_ptr()), vp(Wuq.data_ptr()),
+                     vp(su.data_ptr()), i64(Is), i64(Ks), st)
+                wlw = inputs.Workload(f"quantize_gate_up_I{Is}_K{Ks}", 2 * Is, Ks, 8, 0, False, False)
+                tq, tqb, _ = time_shape(torch, kx, wlw, [lambda: lib.kx_quantize_gate_up_int8(*a)])
+                report(wlw.name, tq, tqb, 3.0 * 2 * Is * Ks + 8.0 * Is, 0.0, 1)
+                del Wg, Wu
+            del keep, calls
+            torch.cuda.empty_cache()
+        for (Mo, No, Ko) in [(4096, 4096, 4096), (16384, 4096, 14336)]:
+            ops = 2.0 * Mo * No * Ko
+            nbytes = 1.0 * (Mo * Ko + No * Ko) + 4.0 * Mo * No + 4.0 * (Mo + No)
+            ns = int(max(2, min(8, math.ceil(2.0 * L2_BYTES / nbytes))))
+            keep, calls = [], []
+            for _ in range(ns):
+                Xq = torch.randint(-127, 128, (Mo, Ko), device="cuda", generator=g, dtype=torch.int8)
+                Wq = torch.randint(-127, 128, (No, Ko), device="cuda", generator=g, dtype=torch.int8)
+                sx = torch.rand(Mo, device="cuda", generator=g) * 2e-2
+                sw = torch.rand(No, device="cuda", generator=g) * 2e-4
+                Rs = torch.randn(Mo, No, device="cuda", generator=g).bfloat16()
+                Ys = torch.empty(Mo, No, dtype=torch.bfloat16, device="cuda")
+                keep.append((Xq, Wq, sx, sw, Rs, Ys))
+                a = (vp(Xq.data_ptr()), vp(sx.data_ptr()), vp(Wq.data_ptr()), vp(sw.data_ptr()), vp(None),
+                     vp(Rs.data_ptr()), vp(Ys.data_ptr()), i64(Mo), i64(No), i64(Ko), st)
+                calls.append(lambda a=a: lib.kx_outproj_residual_int8(*a))
+            wlo = inputs.Workload(f"outproj_int8_M{Mo}_N{No}_K{Ko}", Mo, No, Ko, 0, False, True)
+            t, tbest, _ = time_shape(torch, kx, wlo, calls)
+            report(wlo.name, t, tbest, nbytes, ops, ns)
+            del keep, calls
+            torch.cuda.empty_cache()
+
     # ---- the oracle on the host cores, bounded sample (rank 0, N = 1 only)
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -503,6 +596,7 @@ def run_ours(args):
             "shapes": shapes,
             "rmsnorm": norm,
             "swiglu": swiglu,
+            "int8": int8,
             "sweep_geomean": {"tflops": geo([s["tflops"] for s in sweep]), "roofline_frac": geo([s["frac"] for s in sweep]),
                               "roofline_frac_nominal": geo([s["frac_nominal"] for s in sweep])},
             "paper_context": "766 TFLOP/s BF16 on one 4096x4096 GEMM, H100 SXM (Section 4.1): other hardware, context only",

@@ -1017,6 +1017,14 @@ int kx_gate_up_swiglu(const void* X, const void* Wg, const void* Wu, void* Z, in
 
 // ---------------------------------------------------------------- RMSNorm after the projection
 namespace {
+// Grid of the row kernels (one CTA works on one row at a time).  With fewer than 16 rows per
+// resident CTA a persistent grid ends ragged (4096 rows on 1184 CTAs: 3.46 rows each, so the
+// kernel lasts 4 row-times): launch one CTA per row instead and let the hardware balance them.
+unsigned row_grid(long long M, int sm_count, int per_sm) {
+    const long long resident = static_cast<long long>(sm_count) * per_sm;
+    return static_cast<unsigned>(M <= 16 * resident ? M : resident);
+}
+
 int launch_rmsnorm(const void* H, const void* gamma, float eps, void* Z, long long M, long long N,
                    cudaStream_t stream, int sm_count) {
     cudaLaunchConfig_t cfg;
@@ -1030,7 +1038,7 @@ int launch_rmsnorm(const void* H, const void* gamma, float eps, void* Z, long lo
     else if (nvec <= 4 * kNormThreads) { fn = reinterpret_cast<const void*>(&kx_rmsnorm_kernel<4>); per_sm = 6; }
     else if (nvec <= 8 * kNormThreads) { fn = reinterpret_cast<const void*>(&kx_rmsnorm_kernel<8>); per_sm = 4; }
     else { fn = reinterpret_cast<const void*>(&kx_rmsnorm_kernel<kNormVecs>); per_sm = 2; }
-    cfg.gridDim = dim3(static_cast<unsigned>(std::min<long long>(M, static_cast<long long>(sm_count) * per_sm)), 1, 1);
+    cfg.gridDim = dim3(row_grid(M, sm_count, per_sm), 1, 1);
     cfg.blockDim = dim3(kNormThreads, 1, 1);
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
@@ -1118,7 +1126,7 @@ int launch_rowquant(const QuantParams& qp, bool norm, cudaStream_t stream, int s
     else if (nvec <= 8 * kNormThreads) { fn = KX_QUANT_FN(8); per_sm = 4; }
     else { fn = KX_QUANT_FN(kNormVecs); per_sm = 2; }
 #undef KX_QUANT_FN
-    cfg.gridDim = dim3(static_cast<unsigned>(std::min<long long>(qp.M, static_cast<long long>(sm_count) * per_sm)), 1, 1);
+    cfg.gridDim = dim3(row_grid(qp.M, sm_count, per_sm), 1, 1);
     cfg.blockDim = dim3(kNormThreads, 1, 1);
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];

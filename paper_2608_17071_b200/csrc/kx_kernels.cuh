@@ -1452,17 +1452,15 @@ kx_rowquant_kernel(const QuantParams p) {
             const int idx = tid + i * kNormThreads;
             if (idx < nvec) {
                 const uint32_t w4[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
-                uint32_t o[2] = {0u, 0u};
+                // |z| <= a and rcp = fl(127 / a) keep |z * rcp| below 127.5, so the codes are already
+                // within -127..127; the packing instruction saturates anyway
+                int q[8];
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
-                    int q0 = __float2int_rn(__fmul_rn(bf16_lo(w4[k]), rcp));
-                    int q1 = __float2int_rn(__fmul_rn(bf16_hi(w4[k]), rcp));
-                    q0 = max(-127, min(127, q0));
-                    q1 = max(-127, min(127, q1));
-                    o[k >> 1] |= ((static_cast<uint32_t>(q0) & 0xFFu) | ((static_cast<uint32_t>(q1) & 0xFFu) << 8))
-                                 << ((k & 1) * 16);
+                    q[2 * k] = __float2int_rn(__fmul_rn(bf16_lo(w4[k]), rcp));
+                    q[2 * k + 1] = __float2int_rn(__fmul_rn(bf16_hi(w4[k]), rcp));
                 }
-                qrow[idx] = make_uint2(o[0], o[1]);
+                qrow[idx] = make_uint2(pack_s8x4_sat(q[0], q[1], q[2], q[3]), pack_s8x4_sat(q[4], q[5], q[6], q[7]));
             }
         }
         __syncthreads();         // s_part / s_bcast are reused by the next row

@@ -121,6 +121,13 @@ __device__ __forceinline__ void tma_prefetch_l2_2d(const CUtensorMap* m, int x, 
                  "r"(x), "r"(y)
                  : "memory");
 }
+// Four 32-bit integers -> four signed bytes (b0 lowest), each saturated to [-128, 127].
+__device__ __forceinline__ uint32_t pack_s8x4_sat(int b0, int b1, int b2, int b3) {
+    uint32_t hi, d;
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, 0;" : "=r"(hi) : "r"(b3), "r"(b2));
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(b1), "r"(b0), "r"(hi));
+    return d;
+}
 // 2-D tiled store shared -> global (bulk async group)
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* m, int x, int y, uint32_t src) {
     asm volatile(
