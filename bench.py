@@ -39,7 +39,7 @@ UNIT = "TFLOP/s"
 HEADLINE = "cfg2"
 # DRAM traffic per launch of the dominant kernel from the ncu capture summarised in
 # profiles/ (dram__bytes_read.sum + dram__bytes_write.sum); None until captured.
-NCU_TRAFFIC_BYTES = {"cfg2": 152402944}   # profiles/kx_tile_kernel_pair_cfg2.md
+NCU_TRAFFIC_BYTES = {"cfg2": 154999168}   # profiles/kx_tile_kernel_pair_cfg2.md
 
 
 def load_peaks():
@@ -304,6 +304,7 @@ def run_ours(args):
     peaks = load_peaks()
     wls = inputs.all_workloads()
     headline = args.workload
+    sections = set() if args.no_sweep else set(x for x in args.sections.split(",") if x)
     wl = wls[headline]
 
     # ---- headline workload: seeded bits (rank r draws its own rows: seed offset by rank)
@@ -367,7 +368,7 @@ def run_ours(args):
 
     # ---- every other workload (rank 0, N = 1 only): per-shape roofline lines
     shapes = []
-    if rank == 0 and world == 1 and not args.no_sweep:
+    if rank == 0 and world == 1 and "shapes" in sections:
         order = ["cfg1", "cfg2", "cfg4", "cfg5", "gemm4096"] + [w.name for w in inputs.sweep_workloads()]
         for name in order:
             w = wls[name]
@@ -394,7 +395,7 @@ def run_ours(args):
 
     # ---- the step after the projection: RMSNorm of the new residual stream (rank 0, N = 1 only)
     norm = []
-    if rank == 0 and world == 1 and not args.no_sweep:
+    if rank == 0 and world == 1 and "rmsnorm" in sections:
         lib = kx.load()
         import ctypes
         st = ctypes.c_void_p(int(torch.cuda.current_stream().cuda_stream) or None)
@@ -438,7 +439,7 @@ def run_ours(args):
 
     # ---- gate/up projections with the fused SwiGLU epilogue (rank 0, N = 1 only)
     swiglu = []
-    if rank == 0 and world == 1 and not args.no_sweep:
+    if rank == 0 and world == 1 and "swiglu" in sections:
         lib = kx.load()
         import ctypes
         st = ctypes.c_void_p(int(torch.cuda.current_stream().cuda_stream) or None)
@@ -472,7 +473,7 @@ def run_ours(args):
     # ---- INT8 branch: code-book kernels (HBM-bound) and INT8 GEMMs (tensor-bound; the INT8 peak is
     # taken as twice the measured BF16 GEMM peak, the nominal ratio of the two tensor-core rates)
     int8 = []
-    if rank == 0 and world == 1 and not args.no_sweep:
+    if rank == 0 and world == 1 and "int8" in sections:
         lib = kx.load()
         import ctypes
         vp, i64 = ctypes.c_void_p, ctypes.c_int64
@@ -614,7 +615,9 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--no-sweep", action="store_true")
+    ap.add_argument("--no-sweep", action="store_true", help="headline workload only")
+    ap.add_argument("--sections", default="shapes,rmsnorm,swiglu,int8",
+                    help="comma list of the extra sections to measure after the headline workload")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--workload", default=HEADLINE, help="headline workload name (default: the 4096^3 out-projection)")
