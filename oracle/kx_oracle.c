@@ -367,3 +367,124 @@ int kx_oracle_outproj_int8_rows(const int8_t* Xq, const float* sx, const int8_t*
     }
     return 0;
 }
+
+/*
+ * FP8 (E4M3, the "FN" flavour: bias 7, no infinities, 0x7F / 0xFF = NaN, largest finite 448)
+ * variants of the same three steps, the other low-precision operand type of the paper's
+ * precision axis (Section 3.2).  Decoding is exact; encoding rounds a binary32 value to the
+ * nearest code, ties to the even mantissa, and saturates to +-448 ("satfinite"); NaN -> 0x7F.
+ */
+static double e4m3_decode(uint8_t c) {
+    const int s = c >> 7, e = (c >> 3) & 15, m = c & 7;
+    double v;
+    if (e == 15 && m == 7) return NAN;
+    if (e == 0) v = ldexp((double)m, -9);              /* subnormal: m/8 * 2^-6 */
+    else v = ldexp(1.0 + m / 8.0, e - 7);
+    return s ? -v : v;
+}
+
+static uint8_t e4m3_encode(float x) {
+    const uint8_t s = signbit(x) ? 0x80 : 0;
+    if (isnan(x)) return 0x7F;
+    const float ax = fabsf(x);
+    if (ax > 448.0f) {
+        /* above the largest finite code: everything that would round past 448 saturates */
+        return s | 0x7E;
+    }
+    if (ax < 0.015625f) {                               /* below 2^-6: fixed step 2^-9 */
+        const int q = (int)rintf(ax * 512.0f);          /* exact product; 8 means 2^-6 = code 0x08 */
+        return s | (uint8_t)q;
+    }
+    int e;
+    const float mant = frexpf(ax, &e) * 2.0f;           /* ax = mant * 2^(e-1), mant in [1, 2) */
+    e -= 1;
+    int q = (int)rintf((mant - 1.0f) * 8.0f);           /* exact; ties to even */
+    if (q == 8) { q = 0; e += 1; }
+    int code = ((e + 7) << 3) | q;
+    if (code > 0x7E) code = 0x7E;
+    return s | (uint8_t)code;
+}
+
+int kx_oracle_e4m3_decode(const uint8_t* in, double* out, int64_t n) {
+    if (n < 0 || (n > 0 && (!in || !out))) return -1;
+    for (int64_t i = 0; i < n; ++i) out[i] = e4m3_decode(in[i]);
+    return 0;
+}
+
+int kx_oracle_e4m3_encode(const float* in, uint8_t* out, int64_t n) {
+    if (n < 0 || (n > 0 && (!in || !out))) return -1;
+    for (int64_t i = 0; i < n; ++i) out[i] = e4m3_encode(in[i]);
+    return 0;
+}
+
+/*
+ * Per-row FP8 code book: a = max|z|, scale = a / 448, q = e4m3(z * (448 / a)), every operation
+ * in binary32 as for the INT8 code book above (zero row: scale 1, codes 0).
+ */
+int kx_oracle_quantize_rows_fp8(const uint16_t* Z, int64_t rows, int64_t cols, uint8_t* Q, float* S) {
+    if (rows < 0 || cols < 0 || (rows > 0 && (!S || (cols > 0 && (!Z || !Q))))) return -1;
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < rows; ++r) {
+        float a = 0.0f;
+        for (int64_t j = 0; j < cols; ++j) {
+            const float v = fabsf((float)bf16_widen(Z[r * cols + j]));
+            if (v > a) a = v;
+        }
+        const float inv = (a > 0.0f) ? 448.0f / a : 0.0f;
+        S[r] = (a > 0.0f) ? a / 448.0f : 1.0f;
+        for (int64_t j = 0; j < cols; ++j) {
+            const float z = (float)bf16_widen(Z[r * cols + j]);
+            Q[r * cols + j] = e4m3_encode(z * inv);
+        }
+    }
+    return 0;
+}
+
+static double dq_dot_fp8(const uint8_t* x, const uint8_t* w, int64_t K, float sx, float sw) {
+    double acc = 0.0;                                   /* products of two E4M3 values are exact in double */
+    for (int64_t k = 0; k < K; ++k) acc += e4m3_decode(x[k]) * e4m3_decode(w[k]);
+    return acc * (double)sx * (double)sw;
+}
+
+/* z = silu(g) * u, g = (Xq Wgq^T) sx sg, u = (Xq Wuq^T) sx su on E4M3 codes; double, unrounded. */
+int kx_oracle_swiglu_fp8_rows(const uint8_t* Xq, const float* sx, const uint8_t* Wgq, const float* sg,
+                              const uint8_t* Wuq, const float* su, const int64_t* rows, int64_t nrows,
+                              double* out, int64_t M, int64_t I, int64_t K) {
+    if (M < 0 || I < 0 || K < 0 || nrows < 0 || !out || !sx || !sg || !su) return -1;
+    if (K > 0 && (!Xq || !Wgq || !Wuq)) return -1;
+    for (int64_t r = 0; rows && r < nrows; ++r)
+        if (rows[r] < 0 || rows[r] >= M) return -1;
+    if (!rows && nrows > M) return -1;
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int64_t r = 0; r < nrows; ++r) {
+        for (int64_t i = 0; i < I; ++i) {
+            const int64_t m = rows ? rows[r] : r;
+            const double g = dq_dot_fp8(Xq + m * K, Wgq + i * K, K, sx[m], sg[i]);
+            const double u = dq_dot_fp8(Xq + m * K, Wuq + i * K, K, sx[m], su[i]);
+            out[r * I + i] = g / (1.0 + exp(-g)) * u;
+        }
+    }
+    return 0;
+}
+
+/* y = (Xq Wq^T) sx sw + bias + R on E4M3 codes; double, unrounded. */
+int kx_oracle_outproj_fp8_rows(const uint8_t* Xq, const float* sx, const uint8_t* Wq, const float* sw,
+                               const uint16_t* bias, const uint16_t* R, const int64_t* rows, int64_t nrows,
+                               double* out, int64_t M, int64_t N, int64_t K) {
+    if (M < 0 || N < 0 || K < 0 || nrows < 0 || !out || !sx || !sw) return -1;
+    if (K > 0 && (!Xq || !Wq)) return -1;
+    for (int64_t r = 0; rows && r < nrows; ++r)
+        if (rows[r] < 0 || rows[r] >= M) return -1;
+    if (!rows && nrows > M) return -1;
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int64_t r = 0; r < nrows; ++r) {
+        for (int64_t n = 0; n < N; ++n) {
+            const int64_t m = rows ? rows[r] : r;
+            double y = dq_dot_fp8(Xq + m * K, Wq + n * K, K, sx[m], sw[n]);
+            if (bias) y += bf16_widen(bias[n]);
+            if (R) y += bf16_widen(R[m * N + n]);
+            out[r * N + n] = y;
+        }
+    }
+    return 0;
+}

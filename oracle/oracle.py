@@ -40,6 +40,11 @@ def _load():
         lib.kx_oracle_quantize_rows.argtypes = [p, i64, i64, p, p]
         lib.kx_oracle_swiglu_int8_rows.argtypes = [p, p, p, p, p, p, p, i64, p, p, p, i64, i64, i64]
         lib.kx_oracle_outproj_int8_rows.argtypes = [p, p, p, p, p, p, p, i64, p, i64, i64, i64]
+        lib.kx_oracle_e4m3_decode.argtypes = [p, p, i64]
+        lib.kx_oracle_e4m3_encode.argtypes = [p, p, i64]
+        lib.kx_oracle_quantize_rows_fp8.argtypes = [p, i64, i64, p, p]
+        lib.kx_oracle_swiglu_fp8_rows.argtypes = [p, p, p, p, p, p, p, i64, p, i64, i64, i64]
+        lib.kx_oracle_outproj_fp8_rows.argtypes = [p, p, p, p, p, p, p, i64, p, i64, i64, i64]
         lib.kx_oracle_max_threads.argtypes = []
         lib.kx_oracle_max_threads.restype = ctypes.c_int
         _lib = lib
@@ -241,4 +246,72 @@ def outproj_int8(Xq, sx, Wq, sw, bias=None, R=None, rows=None):
                                              _ptr(rows_arr), nrows, _ptr(out), M, N, K)
     if rc != 0:
         raise RuntimeError(f"kx_oracle_outproj_int8_rows failed ({rc})")
+    return out
+
+
+def e4m3_decode(codes) -> np.ndarray:
+    """FP8 E4M3 (bias 7, no infinities, 0x7F / 0xFF NaN, max 448) bit patterns -> float64, exact."""
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    out = np.empty(codes.shape, dtype=np.float64)
+    _load().kx_oracle_e4m3_decode(_ptr(codes), _ptr(out), codes.size)
+    return out
+
+
+def e4m3_encode(x) -> np.ndarray:
+    """binary32 -> nearest E4M3 code, ties to even, saturating to +-448, NaN -> 0x7F."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    out = np.empty(x.shape, dtype=np.uint8)
+    _load().kx_oracle_e4m3_encode(_ptr(x), _ptr(out), x.size)
+    return out
+
+
+def quantize_rows_fp8(Z):
+    """Per-row FP8 code book of BF16 rows: scale = max|z| / 448, q = e4m3(z * (448 / max|z|)), in
+    binary32 (the other low-precision operand type of the paper's precision axis, Section 3.2).
+    Z uint16 BF16 bits -> (Q uint8 E4M3 bits, S float32)."""
+    rows, cols = Z.shape
+    Z = _bits(Z, (rows, cols), "Z")
+    Q = np.empty((rows, cols), dtype=np.uint8)
+    S = np.empty((rows,), dtype=np.float32)
+    rc = _load().kx_oracle_quantize_rows_fp8(_ptr(Z), rows, cols, _ptr(Q), _ptr(S))
+    if rc != 0:
+        raise RuntimeError(f"kx_oracle_quantize_rows_fp8 failed ({rc})")
+    return Q, S
+
+
+def swiglu_fp8(Xq, sx, Wgq, sg, Wuq, su, rows=None):
+    """z = silu(g) * u on E4M3 codes, g = (Xq Wgq^T) sx sg, u = (Xq Wuq^T) sx su; float64, unrounded."""
+    M, K = Xq.shape
+    I = Wgq.shape[0]
+    Xq = _typed(Xq, np.uint8, (M, K), "Xq")
+    Wgq = _typed(Wgq, np.uint8, (I, K), "Wgq")
+    Wuq = _typed(Wuq, np.uint8, (I, K), "Wuq")
+    sx = _typed(sx, np.float32, (M,), "sx")
+    sg = _typed(sg, np.float32, (I,), "sg")
+    su = _typed(su, np.float32, (I,), "su")
+    rows_arr, nrows = _rows_arg(rows, M)
+    out = np.empty((nrows, I), dtype=np.float64)
+    rc = _load().kx_oracle_swiglu_fp8_rows(_ptr(Xq), _ptr(sx), _ptr(Wgq), _ptr(sg), _ptr(Wuq), _ptr(su),
+                                           _ptr(rows_arr), nrows, _ptr(out), M, I, K)
+    if rc != 0:
+        raise RuntimeError(f"kx_oracle_swiglu_fp8_rows failed ({rc})")
+    return out
+
+
+def outproj_fp8(Xq, sx, Wq, sw, bias=None, R=None, rows=None):
+    """y = (Xq Wq^T) sx sw + bias + R on E4M3 codes; float64, unrounded."""
+    M, K = Xq.shape
+    N = Wq.shape[0]
+    Xq = _typed(Xq, np.uint8, (M, K), "Xq")
+    Wq = _typed(Wq, np.uint8, (N, K), "Wq")
+    sx = _typed(sx, np.float32, (M,), "sx")
+    sw = _typed(sw, np.float32, (N,), "sw")
+    bias = _bits(bias, (N,), "bias")
+    R = _bits(R, (M, N), "R")
+    rows_arr, nrows = _rows_arg(rows, M)
+    out = np.empty((nrows, N), dtype=np.float64)
+    rc = _load().kx_oracle_outproj_fp8_rows(_ptr(Xq), _ptr(sx), _ptr(Wq), _ptr(sw), _ptr(bias), _ptr(R),
+                                            _ptr(rows_arr), nrows, _ptr(out), M, N, K)
+    if rc != 0:
+        raise RuntimeError(f"kx_oracle_outproj_fp8_rows failed ({rc})")
     return out
