@@ -470,8 +470,8 @@ def run_ours(args):
             del keep, calls
             torch.cuda.empty_cache()
 
-    # ---- INT8 branch: code-book kernels (HBM-bound) and INT8 GEMMs (tensor-bound; the INT8 peak is
-    # taken as twice the measured BF16 GEMM peak, the nominal ratio of the two tensor-core rates)
+    # ---- 8-bit branch: code-book kernels (HBM-bound) and INT8 / FP8 GEMMs (tensor-bound; the 8-bit peak
+    # is taken as twice the measured BF16 GEMM peak, the nominal ratio of the tensor-core rates)
     int8 = []
     if rank == 0 and world == 1 and "int8" in sections:
         lib = kx.load()
@@ -539,6 +539,59 @@ def run_ours(args):
                 tq, tqb, _ = time_shape(torch, kx, wlw, [lambda: lib.kx_quantize_gate_up_int8(*a)])
                 report(wlw.name, tq, tqb, 3.0 * 2 * Is * Ks + 8.0 * Is, 0.0, 1)
                 del Wg, Wu
+            del keep, calls
+            torch.cuda.empty_cache()
+        # FP8 E4M3 twins (same kernels, tcgen05 kind::f8f6f4, FP32 accumulation; same nominal peak)
+        F8 = torch.float8_e4m3fn
+        for (Ms, Is, Ks) in [(4096, 14336, 4096)]:
+            ops = 4.0 * Ms * Is * Ks
+            nbytes = 1.0 * (Ms * Ks + 2 * Is * Ks) + 2.0 * Ms * Is + 4.0 * (Ms + 2 * Is)
+            ns = 2
+            keep, calls = [], []
+            for _ in range(ns):
+                Xq = torch.randn(Ms, Ks, device="cuda", generator=g).mul_(100).to(F8)
+                Wgq = torch.randn(Is, Ks, device="cuda", generator=g).mul_(100).to(F8)
+                Wuq = torch.randn(Is, Ks, device="cuda", generator=g).mul_(100).to(F8)
+                sx = torch.rand(Ms, device="cuda", generator=g) * 1e-2
+                sg = torch.rand(Is, device="cuda", generator=g) * 2e-4
+                su = torch.rand(Is, device="cuda", generator=g) * 2e-4
+                Zs = torch.empty(Ms, Is, dtype=torch.bfloat16, device="cuda")
+                keep.append((Xq, Wgq, Wuq, sx, sg, su, Zs))
+                a = (vp(Xq.data_ptr()), vp(sx.data_ptr()), vp(Wgq.data_ptr()), vp(sg.data_ptr()), vp(Wuq.data_ptr()),
+                     vp(su.data_ptr()), vp(Zs.data_ptr()), i64(Ms), i64(Is), i64(Ks), st)
+                calls.append(lambda a=a: lib.kx_gate_up_swiglu_fp8(*a))
+            wls = inputs.Workload(f"swiglu_fp8_M{Ms}_I{Is}_K{Ks}", Ms, 2 * Is, Ks, 0, False, False)
+            t, tbest, _ = time_shape(torch, kx, wls, calls)
+            report(wls.name, t, tbest, nbytes, ops, ns)
+            Hn = torch.randn(Ms, Ks, device="cuda", generator=g).bfloat16()
+            gam = torch.randn(Ks, device="cuda", generator=g).bfloat16()
+            Xq, sx = keep[0][0], keep[0][3]
+            a = (vp(Hn.data_ptr()), vp(gam.data_ptr()), ctypes.c_float(1e-6), vp(Xq.data_ptr()), vp(sx.data_ptr()),
+                 i64(Ms), i64(Ks), st)
+            wlq = inputs.Workload(f"rmsnorm_quantize_fp8_{Ms}x{Ks}", Ms, Ks, 8, 0, False, False)
+            tq, tqb, _ = time_shape(torch, kx, wlq, [lambda: lib.kx_rmsnorm_quantize_fp8(*a)])
+            report(wlq.name + " (warm L2)", tq, tqb, 3.0 * Ms * Ks + 4.0 * Ms + 2.0 * Ks, 0.0, 1)
+            del keep, calls, Hn
+            torch.cuda.empty_cache()
+        for (Mo, No, Ko) in [(4096, 4096, 4096), (16384, 4096, 14336)]:
+            ops = 2.0 * Mo * No * Ko
+            nbytes = 1.0 * (Mo * Ko + No * Ko) + 4.0 * Mo * No + 4.0 * (Mo + No)
+            ns = int(max(2, min(8, math.ceil(2.0 * L2_BYTES / nbytes))))
+            keep, calls = [], []
+            for _ in range(ns):
+                Xq = torch.randn(Mo, Ko, device="cuda", generator=g).mul_(100).to(F8)
+                Wq = torch.randn(No, Ko, device="cuda", generator=g).mul_(100).to(F8)
+                sx = torch.rand(Mo, device="cuda", generator=g) * 1e-2
+                sw = torch.rand(No, device="cuda", generator=g) * 2e-4
+                Rs = torch.randn(Mo, No, device="cuda", generator=g).bfloat16()
+                Ys = torch.empty(Mo, No, dtype=torch.bfloat16, device="cuda")
+                keep.append((Xq, Wq, sx, sw, Rs, Ys))
+                a = (vp(Xq.data_ptr()), vp(sx.data_ptr()), vp(Wq.data_ptr()), vp(sw.data_ptr()), vp(None),
+                     vp(Rs.data_ptr()), vp(Ys.data_ptr()), i64(Mo), i64(No), i64(Ko), st)
+                calls.append(lambda a=a: lib.kx_outproj_residual_fp8(*a))
+            wlo = inputs.Workload(f"outproj_fp8_M{Mo}_N{No}_K{Ko}", Mo, No, Ko, 0, False, True)
+            t, tbest, _ = time_shape(torch, kx, wlo, calls)
+            report(wlo.name, t, tbest, nbytes, ops, ns)
             del keep, calls
             torch.cuda.empty_cache()
         for (Mo, No, Ko) in [(4096, 4096, 4096), (16384, 4096, 14336)]:

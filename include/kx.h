@@ -311,6 +311,28 @@ int kx_outproj_residual_int8(const void* Xq, const float* sx, const void* Wq, co
                              const void* bias_or_null, const void* R_or_null, void* Y,
                              int64_t M, int64_t N, int64_t K, void* stream);
 
+/*
+ * ---- FP8 (E4M3) twins of the five INT8 entry points: the other 8-bit operand type of the
+ * precision axis of the paper's strategy space (Section 3.2).  Codes are FP8 E4M3 bit patterns
+ * (bias 7, no infinities, 0x7F / 0xFF = NaN, largest finite value 448), one byte each; the code
+ * book is
+ *     a = max_j |z_j|,  scale = a / 448,  q_j = e4m3(z_j * (448 / a))
+ * in binary32, the conversion rounding to nearest (ties to even) and saturating at +-448.  The
+ * GEMMs run tcgen05 kind::f8f6f4 with FP32 accumulation; everything else (layouts, alignment,
+ * K % 16 == 0, scale vectors, epilogues, error codes) is as for the INT8 calls above.
+ */
+int kx_quantize_rows_fp8(const void* A, void* Q, float* S, int64_t rows, int64_t cols, void* stream);
+int kx_quantize_gate_up_fp8(const void* Wg, const void* Wu, void* Qg, float* Sg, void* Qu, float* Su,
+                            int64_t I, int64_t K, void* stream);
+int kx_rmsnorm_quantize_fp8(const void* H, const void* gamma, float eps, void* Q, float* S,
+                            int64_t M, int64_t N, void* stream);
+int kx_gate_up_swiglu_fp8(const void* Xq, const float* sx, const void* Wgq, const float* sg,
+                          const void* Wuq, const float* su, void* Z,
+                          int64_t M, int64_t I, int64_t K, void* stream);
+int kx_outproj_residual_fp8(const void* Xq, const float* sx, const void* Wq, const float* sw,
+                            const void* bias_or_null, const void* R_or_null, void* Y,
+                            int64_t M, int64_t N, int64_t K, void* stream);
+
 /* Fills `out` with the plan the library would use for this shape on the current
  * device (has_residual / has_bias as 0 or 1).  No work is enqueued. */
 int kx_plan_query(int64_t M, int64_t N, int64_t K, int has_bias, int has_residual,

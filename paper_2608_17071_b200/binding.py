@@ -27,6 +27,8 @@ EXPORTS = (
     "kx_gate_up_swiglu",
     "kx_quantize_rows_int8", "kx_quantize_gate_up_int8", "kx_rmsnorm_quantize_int8", "kx_gate_up_swiglu_int8",
     "kx_outproj_residual_int8",
+    "kx_quantize_rows_fp8", "kx_quantize_gate_up_fp8", "kx_rmsnorm_quantize_fp8", "kx_gate_up_swiglu_fp8",
+    "kx_outproj_residual_fp8",
     "kx_plan_query", "kx_last_device_status", "kx_status_string",
     "kx_version",
 )
@@ -86,6 +88,12 @@ def load():
     lib.kx_rmsnorm_quantize_int8.argtypes = [vp, vp, ctypes.c_float, vp, vp, i64, i64, vp]
     lib.kx_gate_up_swiglu_int8.argtypes = [vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, vp]
     lib.kx_outproj_residual_int8.argtypes = [vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, vp]
+    for sfx in ("fp8",):
+        getattr(lib, f"kx_quantize_rows_{sfx}").argtypes = lib.kx_quantize_rows_int8.argtypes
+        getattr(lib, f"kx_quantize_gate_up_{sfx}").argtypes = lib.kx_quantize_gate_up_int8.argtypes
+        getattr(lib, f"kx_rmsnorm_quantize_{sfx}").argtypes = lib.kx_rmsnorm_quantize_int8.argtypes
+        getattr(lib, f"kx_gate_up_swiglu_{sfx}").argtypes = lib.kx_gate_up_swiglu_int8.argtypes
+        getattr(lib, f"kx_outproj_residual_{sfx}").argtypes = lib.kx_outproj_residual_int8.argtypes
     lib.kx_plan_query.argtypes = [i64, i64, i64, ci, ci, ctypes.POINTER(PlanOverride), ctypes.POINTER(PlanInfo)]
     lib.kx_last_device_status.argtypes = [vp, ctypes.POINTER(ci), ctypes.POINTER(ci)]
     lib.kx_status_string.argtypes = [ci]
@@ -231,71 +239,103 @@ def kx_gate_up_swiglu(X, Wg, Wu, Z, stream=None, M=None, I=None, K=None, check=T
     return rc
 
 
-def kx_quantize_rows_int8(A, Q, S, stream=None, check=True) -> int:
+def _code_dtype(fmt):
+    import torch
+    if fmt == "int8":
+        return torch.int8
+    if fmt == "fp8":
+        return torch.float8_e4m3fn
+    raise ValueError(f"unknown 8-bit format {fmt!r} (int8 or fp8)")
+
+
+def kx_quantize_rows_int8(A, Q, S, stream=None, check=True, fmt="int8") -> int:
     """Q (int8), S (float32 per row) = symmetric per-row INT8 code book of the BF16 matrix A."""
     import torch
     rows, cols = A.shape
-    _check_bf16("A", A, (rows, cols)); _check("Q", Q, (rows, cols), torch.int8); _check("S", S, (rows,), torch.float32)
-    rc = load().kx_quantize_rows_int8(_addr(A), _addr(Q), _addr(S), rows, cols, _stream(stream))
+    _check_bf16("A", A, (rows, cols)); _check("Q", Q, (rows, cols), _code_dtype(fmt)); _check("S", S, (rows,), torch.float32)
+    rc = getattr(load(), f"kx_quantize_rows_{fmt}")(_addr(A), _addr(Q), _addr(S), rows, cols, _stream(stream))
     if check and rc != KX_OK:
-        raise KxError(rc, "kx_quantize_rows_int8")
+        raise KxError(rc, f"kx_quantize_rows_{fmt}")
     return rc
 
 
-def kx_quantize_gate_up_int8(Wg, Wu, Qg, Sg, Qu, Su, stream=None, check=True) -> int:
+def kx_quantize_gate_up_int8(Wg, Wu, Qg, Sg, Qu, Su, stream=None, check=True, fmt="int8") -> int:
     """Code books of the gate and the up weight matrices in one launch."""
     import torch
     I, K = Wg.shape
     _check_bf16("Wg", Wg, (I, K)); _check_bf16("Wu", Wu, (I, K))
-    _check("Qg", Qg, (I, K), torch.int8); _check("Qu", Qu, (I, K), torch.int8)
+    _check("Qg", Qg, (I, K), _code_dtype(fmt)); _check("Qu", Qu, (I, K), _code_dtype(fmt))
     _check("Sg", Sg, (I,), torch.float32); _check("Su", Su, (I,), torch.float32)
-    rc = load().kx_quantize_gate_up_int8(_addr(Wg), _addr(Wu), _addr(Qg), _addr(Sg), _addr(Qu), _addr(Su), I, K,
-                                         _stream(stream))
+    rc = getattr(load(), f"kx_quantize_gate_up_{fmt}")(_addr(Wg), _addr(Wu), _addr(Qg), _addr(Sg), _addr(Qu), _addr(Su),
+                                                       I, K, _stream(stream))
     if check and rc != KX_OK:
-        raise KxError(rc, "kx_quantize_gate_up_int8")
+        raise KxError(rc, f"kx_quantize_gate_up_{fmt}")
     return rc
 
 
-def kx_rmsnorm_quantize_int8(H, gamma, eps: float, Q, S, stream=None, check=True) -> int:
+def kx_rmsnorm_quantize_int8(H, gamma, eps: float, Q, S, stream=None, check=True, fmt="int8") -> int:
     """Q, S = code book of RMSNorm(H) * gamma (rounded to BF16 as kx_rmsnorm would), H read once."""
     import torch
     M, N = H.shape
     _check_bf16("H", H, (M, N)); _check_bf16("gamma", gamma, (N,))
-    _check("Q", Q, (M, N), torch.int8); _check("S", S, (M,), torch.float32)
-    rc = load().kx_rmsnorm_quantize_int8(_addr(H), _addr(gamma), float(eps), _addr(Q), _addr(S), M, N, _stream(stream))
+    _check("Q", Q, (M, N), _code_dtype(fmt)); _check("S", S, (M,), torch.float32)
+    rc = getattr(load(), f"kx_rmsnorm_quantize_{fmt}")(_addr(H), _addr(gamma), float(eps), _addr(Q), _addr(S), M, N,
+                                                       _stream(stream))
     if check and rc != KX_OK:
-        raise KxError(rc, "kx_rmsnorm_quantize_int8")
+        raise KxError(rc, f"kx_rmsnorm_quantize_{fmt}")
     return rc
 
 
-def kx_gate_up_swiglu_int8(Xq, sx, Wgq, sg, Wuq, su, Z, stream=None, check=True) -> int:
+def kx_gate_up_swiglu_int8(Xq, sx, Wgq, sg, Wuq, su, Z, stream=None, check=True, fmt="int8") -> int:
     """Z = silu((Xq Wgq^T) sx sg) * ((Xq Wuq^T) sx su): INT8 GEMM, dequantisation and SwiGLU fused."""
     import torch
     M, K = Xq.shape
     I = Wgq.shape[0]
-    _check("Xq", Xq, (M, K), torch.int8); _check("Wgq", Wgq, (I, K), torch.int8); _check("Wuq", Wuq, (I, K), torch.int8)
+    cd = _code_dtype(fmt)
+    _check("Xq", Xq, (M, K), cd); _check("Wgq", Wgq, (I, K), cd); _check("Wuq", Wuq, (I, K), cd)
     _check("sx", sx, (M,), torch.float32); _check("sg", sg, (I,), torch.float32); _check("su", su, (I,), torch.float32)
     _check_bf16("Z", Z, (M, I))
-    rc = load().kx_gate_up_swiglu_int8(_addr(Xq), _addr(sx), _addr(Wgq), _addr(sg), _addr(Wuq), _addr(su), _addr(Z),
-                                       M, I, K, _stream(stream))
+    rc = getattr(load(), f"kx_gate_up_swiglu_{fmt}")(_addr(Xq), _addr(sx), _addr(Wgq), _addr(sg), _addr(Wuq), _addr(su),
+                                                     _addr(Z), M, I, K, _stream(stream))
     if check and rc != KX_OK:
-        raise KxError(rc, "kx_gate_up_swiglu_int8")
+        raise KxError(rc, f"kx_gate_up_swiglu_{fmt}")
     return rc
 
 
-def kx_outproj_residual_int8(Xq, sx, Wq, sw, bias, R, Y, stream=None, check=True) -> int:
+def kx_outproj_residual_int8(Xq, sx, Wq, sw, bias, R, Y, stream=None, check=True, fmt="int8") -> int:
     """Y = (Xq Wq^T) sx sw + bias + R on INT8 codes; bias / R may be None; R may be Y."""
     import torch
     M, K = Xq.shape
     N = Wq.shape[0]
-    _check("Xq", Xq, (M, K), torch.int8); _check("Wq", Wq, (N, K), torch.int8)
+    _check("Xq", Xq, (M, K), _code_dtype(fmt)); _check("Wq", Wq, (N, K), _code_dtype(fmt))
     _check("sx", sx, (M,), torch.float32); _check("sw", sw, (N,), torch.float32)
     _check_bf16("bias", bias, (N,)); _check_bf16("R", R, (M, N)); _check_bf16("Y", Y, (M, N))
-    rc = load().kx_outproj_residual_int8(_addr(Xq), _addr(sx), _addr(Wq), _addr(sw), _addr(bias), _addr(R), _addr(Y),
-                                         M, N, K, _stream(stream))
+    rc = getattr(load(), f"kx_outproj_residual_{fmt}")(_addr(Xq), _addr(sx), _addr(Wq), _addr(sw), _addr(bias), _addr(R),
+                                                       _addr(Y), M, N, K, _stream(stream))
     if check and rc != KX_OK:
-        raise KxError(rc, "kx_outproj_residual_int8")
+        raise KxError(rc, f"kx_outproj_residual_{fmt}")
     return rc
+
+
+def kx_quantize_rows_fp8(A, Q, S, **kw) -> int:
+    """FP8 E4M3 twin of kx_quantize_rows_int8 (Q is a float8_e4m3fn tensor)."""
+    return kx_quantize_rows_int8(A, Q, S, fmt="fp8", **kw)
+
+
+def kx_quantize_gate_up_fp8(Wg, Wu, Qg, Sg, Qu, Su, **kw) -> int:
+    return kx_quantize_gate_up_int8(Wg, Wu, Qg, Sg, Qu, Su, fmt="fp8", **kw)
+
+
+def kx_rmsnorm_quantize_fp8(H, gamma, eps: float, Q, S, **kw) -> int:
+    return kx_rmsnorm_quantize_int8(H, gamma, eps, Q, S, fmt="fp8", **kw)
+
+
+def kx_gate_up_swiglu_fp8(Xq, sx, Wgq, sg, Wuq, su, Z, **kw) -> int:
+    return kx_gate_up_swiglu_int8(Xq, sx, Wgq, sg, Wuq, su, Z, fmt="fp8", **kw)
+
+
+def kx_outproj_residual_fp8(Xq, sx, Wq, sw, bias, R, Y, **kw) -> int:
+    return kx_outproj_residual_int8(Xq, sx, Wq, sw, bias, R, Y, fmt="fp8", **kw)
 
 
 def kx_rmsnorm(H, gamma, eps: float, Z, stream=None, M=None, N=None, check=True) -> int:

@@ -71,6 +71,7 @@ struct TileVariant {
     int bn, ctas, stages, nb, smem;
     const void* fn;        // BF16 operands
     const void* fn_s8;     // signed 8-bit operands, integer accumulators
+    const void* fn_f8;     // FP8 E4M3 operands, FP32 accumulators
 };
 struct SwapVariant {
     int bn, stages, smem;
@@ -82,7 +83,8 @@ struct SwapVariant {
     TileVariant {                                                                             \
         BN, CTAS, ST, NB, TileCfg<BN, CTAS, ST, NB>::SMEM_BYTES,                              \
             reinterpret_cast<const void*>(&kx_tile_kernel<BN, CTAS, ST, NB, 0>),              \
-            reinterpret_cast<const void*>(&kx_tile_kernel<BN, CTAS, ST, NB, 1>)               \
+            reinterpret_cast<const void*>(&kx_tile_kernel<BN, CTAS, ST, NB, 1>),              \
+            reinterpret_cast<const void*>(&kx_tile_kernel<BN, CTAS, ST, NB, 2>)               \
     }
 #define KX_SWAP(BN, ST)                                                                       \
     SwapVariant {                                                                             \
@@ -155,7 +157,8 @@ int ensure_device(int dev, DeviceCtx** out) {
         for (const auto& v : kTileVariants)
             ok = ok &&
                  cudaFuncSetAttribute(v.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, v.smem) == cudaSuccess &&
-                 cudaFuncSetAttribute(v.fn_s8, cudaFuncAttributeMaxDynamicSharedMemorySize, v.smem) == cudaSuccess;
+                 cudaFuncSetAttribute(v.fn_s8, cudaFuncAttributeMaxDynamicSharedMemorySize, v.smem) == cudaSuccess &&
+                 cudaFuncSetAttribute(v.fn_f8, cudaFuncAttributeMaxDynamicSharedMemorySize, v.smem) == cudaSuccess;
         for (const auto& v : kSwapVariants)
             ok = ok &&
                  cudaFuncSetAttribute(v.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, v.smem) == cudaSuccess &&
@@ -265,6 +268,7 @@ struct Plan {
     size_t ws_bytes = 0;
     const void* fn = nullptr;
     const void* fn_s8 = nullptr;
+    const void* fn_f8 = nullptr;
     int launches = 1;
 };
 
@@ -431,6 +435,7 @@ int make_plan_from(long long M, long long N, long long K, const kx_plan_override
         pl->smem = v->smem;
         pl->fn = v->fn;
         pl->fn_s8 = v->fn_s8;
+        pl->fn_f8 = v->fn_f8;
         pl->tiles_m = ceil_div(M, 128 * ctas);
         pl->tiles_n = ceil_div(N, bn);
         pl->units = pl->tiles_m * pl->tiles_n;
@@ -1111,15 +1116,18 @@ int kx_outproj_residual_rmsnorm(const void* X, const void* W, const void* bias, 
 namespace {
 bool aligned4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3u) == 0; }
 
-int launch_rowquant(const QuantParams& qp, bool norm, cudaStream_t stream, int sm_count) {
+// fmt: 0 = INT8 codes, 1 = FP8 E4M3 codes
+int launch_rowquant(const QuantParams& qp, bool norm, int fmt, cudaStream_t stream, int sm_count) {
     cudaLaunchConfig_t cfg;
     std::memset(&cfg, 0, sizeof cfg);
     const long long nvec = qp.N / 8;
     const void* fn = nullptr;
     int per_sm = 8;
-#define KX_QUANT_FN(NV) \
-    (norm ? reinterpret_cast<const void*>(&kx_rowquant_kernel<NV, true>) \
-          : reinterpret_cast<const void*>(&kx_rowquant_kernel<NV, false>))
+#define KX_QUANT_FN(NV)                                                                              \
+    (fmt == 1 ? (norm ? reinterpret_cast<const void*>(&kx_rowquant_kernel<NV, true, 1>)              \
+                      : reinterpret_cast<const void*>(&kx_rowquant_kernel<NV, false, 1>))            \
+              : (norm ? reinterpret_cast<const void*>(&kx_rowquant_kernel<NV, true, 0>)              \
+                      : reinterpret_cast<const void*>(&kx_rowquant_kernel<NV, false, 0>)))
     if (nvec <= 1 * kNormThreads) { fn = KX_QUANT_FN(1); }
     else if (nvec <= 2 * kNormThreads) { fn = KX_QUANT_FN(2); }
     else if (nvec <= 4 * kNormThreads) { fn = KX_QUANT_FN(4); per_sm = 6; }
@@ -1165,17 +1173,18 @@ int device_ctx(DeviceCtx** ctx) {
     return ensure_device(dev, ctx);
 }
 
-// Shared launcher of the INT8 tile kernel.  swiglu: B = gate rows, B2 = up rows, N = output columns I.
-int run_s8(const void* Xq, const float* sx, const void* Wq, const float* sw, const void* Wq2, const float* sw2,
-           const void* bias, const void* R, void* Y, long long M, long long N, long long K, bool swiglu,
-           cudaStream_t stream) {
+// Shared launcher of the 8-bit tile kernels.  swiglu: B = gate rows, B2 = up rows, N = output columns I.
+// kind: 1 = INT8 codes, 2 = FP8 E4M3 codes
+int run_q8(int kind, const void* Xq, const float* sx, const void* Wq, const float* sw, const void* Wq2,
+           const float* sw2, const void* bias, const void* R, void* Y, long long M, long long N, long long K,
+           bool swiglu, cudaStream_t stream) {
     DeviceCtx* ctx = nullptr;
     int rc = device_ctx(&ctx);
     if (rc != KX_OK) return rc;
     kx_plan_override ov;
     std::memset(&ov, 0, sizeof ov);
     ov.path = KX_PATH_TILE;
-    ov.stream_k = 1;          // whole tiles only: partial integer accumulators are never added as FP32
+    ov.stream_k = 1;          // whole tiles only: unscaled partial accumulators are never added across CTAs
     ov.no_table = 1;
     if (swiglu) {
         ov.block_n = 256;     // 128 gate + 128 up accumulator columns = 128 output columns per tile
@@ -1248,7 +1257,7 @@ int run_s8(const void* Xq, const float* sx, const void* Wq, const float* sw, con
     cfg.numAttrs = nattr;
     const uint16_t* bias_p = static_cast<const uint16_t*>(bias);
     void* args[] = {&tmA, &tmB, &tmB2, &tmY, &tmR, &bias_p, &p};
-    if (cudaLaunchKernelExC(&cfg, pl.fn_s8, args) != cudaSuccess) {
+    if (cudaLaunchKernelExC(&cfg, kind == 2 ? pl.fn_f8 : pl.fn_s8, args) != cudaSuccess) {
         cudaGetLastError();
         return KX_ERR_CUDA;
     }
@@ -1256,7 +1265,7 @@ int run_s8(const void* Xq, const float* sx, const void* Wq, const float* sw, con
 }
 }  // namespace
 
-int kx_quantize_rows_int8(const void* A, void* Q, float* S, int64_t rows, int64_t cols, void* stream) {
+static int quantize_rows_q8(int fmt, const void* A, void* Q, float* S, int64_t rows, int64_t cols, void* stream) {
     int rc = validate_quant(A, Q, S, rows, cols);
     if (rc != KX_OK) return rc;
     if (rows == 0) return KX_OK;
@@ -1270,10 +1279,10 @@ int kx_quantize_rows_int8(const void* A, void* Q, float* S, int64_t rows, int64_
     qp.rows0 = rows;
     qp.M = rows;
     qp.N = static_cast<int>(cols);
-    return launch_rowquant(qp, false, static_cast<cudaStream_t>(stream), ctx->sm_count);
+    return launch_rowquant(qp, false, fmt, static_cast<cudaStream_t>(stream), ctx->sm_count);
 }
 
-int kx_quantize_gate_up_int8(const void* Wg, const void* Wu, void* Qg, float* Sg, void* Qu, float* Su, int64_t I,
+static int quantize_gate_up_q8(int fmt, const void* Wg, const void* Wu, void* Qg, float* Sg, void* Qu, float* Su, int64_t I,
                              int64_t K, void* stream) {
     int rc = validate_quant(Wg, Qg, Sg, I, K);
     if (rc == KX_OK) rc = validate_quant(Wu, Qu, Su, I, K);
@@ -1296,10 +1305,10 @@ int kx_quantize_gate_up_int8(const void* Wg, const void* Wu, void* Qg, float* Sg
     qp.rows0 = I;
     qp.M = 2 * I;
     qp.N = static_cast<int>(K);
-    return launch_rowquant(qp, false, static_cast<cudaStream_t>(stream), ctx->sm_count);
+    return launch_rowquant(qp, false, fmt, static_cast<cudaStream_t>(stream), ctx->sm_count);
 }
 
-int kx_rmsnorm_quantize_int8(const void* H, const void* gamma, float eps, void* Q, float* S, int64_t M, int64_t N,
+static int rmsnorm_quantize_q8(int fmt, const void* H, const void* gamma, float eps, void* Q, float* S, int64_t M, int64_t N,
                              void* stream) {
     int rc = validate_quant(H, Q, S, M, N);
     if (rc != KX_OK) return rc;
@@ -1324,7 +1333,7 @@ int kx_rmsnorm_quantize_int8(const void* H, const void* gamma, float eps, void* 
     qp.M = M;
     qp.N = static_cast<int>(N);
     qp.eps = eps;
-    return launch_rowquant(qp, N > 0, static_cast<cudaStream_t>(stream), ctx->sm_count);
+    return launch_rowquant(qp, N > 0, fmt, static_cast<cudaStream_t>(stream), ctx->sm_count);
 }
 
 namespace {
@@ -1347,7 +1356,7 @@ int validate_s8(const void* Xq, const float* sx, const void* Wq, const float* sw
 }
 }  // namespace
 
-int kx_gate_up_swiglu_int8(const void* Xq, const float* sx, const void* Wgq, const float* sg, const void* Wuq,
+static int gate_up_swiglu_q8(int kind, const void* Xq, const float* sx, const void* Wgq, const float* sg, const void* Wuq,
                            const float* su, void* Z, int64_t M, int64_t I, int64_t K, void* stream_v) {
     int rc = validate_s8(Xq, sx, Wgq, sg, Z, M, I, K);
     if (rc == KX_OK) rc = validate_s8(Xq, sx, Wuq, su, Z, M, I, K);
@@ -1362,10 +1371,10 @@ int kx_gate_up_swiglu_int8(const void* Xq, const float* sx, const void* Wgq, con
         kx_k0_kernel<<<blocks, 256, 0, stream>>>(nullptr, nullptr, static_cast<uint16_t*>(Z), M, I);
         return cudaGetLastError() == cudaSuccess ? KX_OK : KX_ERR_CUDA;
     }
-    return run_s8(Xq, sx, Wgq, sg, Wuq, su, nullptr, nullptr, Z, M, I, K, true, stream);
+    return run_q8(kind, Xq, sx, Wgq, sg, Wuq, su, nullptr, nullptr, Z, M, I, K, true, stream);
 }
 
-int kx_outproj_residual_int8(const void* Xq, const float* sx, const void* Wq, const float* sw, const void* bias,
+static int outproj_residual_q8(int kind, const void* Xq, const float* sx, const void* Wq, const float* sw, const void* bias,
                              const void* R, void* Y, int64_t M, int64_t N, int64_t K, void* stream_v) {
     int rc = validate_s8(Xq, sx, Wq, sw, Y, M, N, K);
     if (rc != KX_OK) return rc;
@@ -1384,7 +1393,46 @@ int kx_outproj_residual_int8(const void* Xq, const float* sx, const void* Wq, co
                                                  static_cast<uint16_t*>(Y), M, N);
         return cudaGetLastError() == cudaSuccess ? KX_OK : KX_ERR_CUDA;
     }
-    return run_s8(Xq, sx, Wq, sw, nullptr, nullptr, bias, R, Y, M, N, K, false, stream);
+    return run_q8(kind, Xq, sx, Wq, sw, nullptr, nullptr, bias, R, Y, M, N, K, false, stream);
+}
+
+int kx_quantize_rows_int8(const void* A, void* Q, float* S, int64_t rows, int64_t cols, void* stream) {
+    return quantize_rows_q8(0, A, Q, S, rows, cols, stream);
+}
+int kx_quantize_rows_fp8(const void* A, void* Q, float* S, int64_t rows, int64_t cols, void* stream) {
+    return quantize_rows_q8(1, A, Q, S, rows, cols, stream);
+}
+int kx_quantize_gate_up_int8(const void* Wg, const void* Wu, void* Qg, float* Sg, void* Qu, float* Su, int64_t I,
+                             int64_t K, void* stream) {
+    return quantize_gate_up_q8(0, Wg, Wu, Qg, Sg, Qu, Su, I, K, stream);
+}
+int kx_quantize_gate_up_fp8(const void* Wg, const void* Wu, void* Qg, float* Sg, void* Qu, float* Su, int64_t I,
+                            int64_t K, void* stream) {
+    return quantize_gate_up_q8(1, Wg, Wu, Qg, Sg, Qu, Su, I, K, stream);
+}
+int kx_rmsnorm_quantize_int8(const void* H, const void* gamma, float eps, void* Q, float* S, int64_t M, int64_t N,
+                             void* stream) {
+    return rmsnorm_quantize_q8(0, H, gamma, eps, Q, S, M, N, stream);
+}
+int kx_rmsnorm_quantize_fp8(const void* H, const void* gamma, float eps, void* Q, float* S, int64_t M, int64_t N,
+                            void* stream) {
+    return rmsnorm_quantize_q8(1, H, gamma, eps, Q, S, M, N, stream);
+}
+int kx_gate_up_swiglu_int8(const void* Xq, const float* sx, const void* Wgq, const float* sg, const void* Wuq,
+                           const float* su, void* Z, int64_t M, int64_t I, int64_t K, void* stream) {
+    return gate_up_swiglu_q8(1, Xq, sx, Wgq, sg, Wuq, su, Z, M, I, K, stream);
+}
+int kx_gate_up_swiglu_fp8(const void* Xq, const float* sx, const void* Wgq, const float* sg, const void* Wuq,
+                          const float* su, void* Z, int64_t M, int64_t I, int64_t K, void* stream) {
+    return gate_up_swiglu_q8(2, Xq, sx, Wgq, sg, Wuq, su, Z, M, I, K, stream);
+}
+int kx_outproj_residual_int8(const void* Xq, const float* sx, const void* Wq, const float* sw, const void* bias,
+                             const void* R, void* Y, int64_t M, int64_t N, int64_t K, void* stream) {
+    return outproj_residual_q8(1, Xq, sx, Wq, sw, bias, R, Y, M, N, K, stream);
+}
+int kx_outproj_residual_fp8(const void* Xq, const float* sx, const void* Wq, const float* sw, const void* bias,
+                            const void* R, void* Y, int64_t M, int64_t N, int64_t K, void* stream) {
+    return outproj_residual_q8(2, Xq, sx, Wq, sw, bias, R, Y, M, N, K, stream);
 }
 
 // ---------------------------------------------------------------- no-allocation entry

@@ -119,9 +119,9 @@ struct TileParams {
     int has_bias, has_r;
     int drop_kblocks;
     int pf_kblocks;            // L2 prefetch depth before the dependency wait (0 = ring depth, <0 = none)
-    const float* sa;           // KIND 1: scale per row of A [M]
-    const float* sb;           // KIND 1: scale per row of B [N] (gate rows in gate/up mode)
-    const float* sb2;          // KIND 1, gate/up mode: scale per up row [N]
+    const float* sa;           // KIND 1 / 2: scale per row of A [M]
+    const float* sb;           // KIND 1 / 2: scale per row of B [N] (gate rows in gate/up mode)
+    const float* sb2;          // KIND 1 / 2, gate/up mode: scale per up row [N]
     int swiglu;                   // 1: gate/up mode.  W rows of a tile = BN/2 rows of Wg (tmB) followed by the same
                                   // BN/2 rows of Wu (tmB2); the epilogue writes silu(gate) * up, BN/2 columns per
                                   // tile, N = number of output columns; no bias, no residual
@@ -213,9 +213,10 @@ __device__ __forceinline__ uint32_t ld_acquire_gpu_u32(const unsigned int* p) {
 }
 
 // KIND 0: BF16 operands, FP32 accumulators.  KIND 1: signed 8-bit operands (a k-block is 128
-// codes = the same 128 bytes per row), 32-bit integer accumulators, dequantised in the epilogue
-// with a per-row scale of A and a per-row scale of B (stream-K and K-cluster plans, which add
-// partial accumulators as FP32, are not used with KIND 1).
+// codes = the same 128 bytes per row), 32-bit integer accumulators.  KIND 2: FP8 E4M3 operands
+// (same byte geometry), FP32 accumulators.  KIND 1 and 2 are dequantised in the epilogue with a
+// per-row scale of A and a per-row scale of B; they run whole tiles only (the stream-K and
+// K-cluster fix-ups add partial accumulators as unscaled FP32).
 template <int BN, int CTAS, int STAGES, int NB, int KIND = 0>
 __global__ void __launch_bounds__(kThreads, 1)
 kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
@@ -243,7 +244,7 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int lane = threadIdx.x & 31;
     const uint32_t cta_rank = (CTAS == 2) ? cluster_ctarank() : 0u;
     const bool leader = (cta_rank == 0);
-    constexpr int KBLK = (KIND == 1) ? 2 * kBlockK : kBlockK;   // elements per k-block (128 bytes)
+    constexpr int KBLK = (KIND != 0) ? 2 * kBlockK : kBlockK;   // elements per k-block (128 bytes)
     const int nkb = (p.K + KBLK - 1) / KBLK;
     const int kc = (CTAS == 1 && p.kcluster > 1) ? p.kcluster : 1;   // K-cluster size
     const int krank = (kc > 1) ? static_cast<int>(cluster_ctarank()) : 0;
@@ -385,9 +386,12 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     } else if (warp == 5) {
         // ------------------------------------------------------------ MMA issuer
         if (leader && lane == 0) {
-            constexpr uint32_t idesc_wide = KIND == 1 ? idesc_s8_s32(128 * CTAS, BN) : idesc_bf16_f32(128 * CTAS, BN);
-            constexpr uint32_t idesc_narrow =
-                KIND == 1 ? idesc_s8_s32(128 * CTAS, BN / 2) : idesc_bf16_f32(128 * CTAS, BN / 2);
+            constexpr uint32_t idesc_wide = KIND == 1   ? idesc_s8_s32(128 * CTAS, BN)
+                                            : KIND == 2 ? idesc_e4m3_f32(128 * CTAS, BN)
+                                                        : idesc_bf16_f32(128 * CTAS, BN);
+            constexpr uint32_t idesc_narrow = KIND == 1   ? idesc_s8_s32(128 * CTAS, BN / 2)
+                                              : KIND == 2 ? idesc_e4m3_f32(128 * CTAS, BN / 2)
+                                                          : idesc_bf16_f32(128 * CTAS, BN / 2);
             uint32_t s = 0, ph = 0, scount = 0;
             bool ok = true;
             while (ok && it.next(tile, kb0, kb1)) {
@@ -408,6 +412,9 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     for (int k = 0; k < 4; ++k) {
                         if constexpr (KIND == 1)
                             mma_s8<CTAS>(d, smem_desc_sw128(sa + k * 32), smem_desc_sw128(sb + k * 32), idesc,
+                                         static_cast<uint32_t>((kb - kb0) | k));
+                        else if constexpr (KIND == 2)
+                            mma_f8<CTAS>(d, smem_desc_sw128(sa + k * 32), smem_desc_sw128(sb + k * 32), idesc,
                                          static_cast<uint32_t>((kb - kb0) | k));
                         else
                             mma_bf16<CTAS>(d, smem_desc_sw128(sa + k * 32), smem_desc_sw128(sb + k * 32), idesc,
@@ -460,18 +467,20 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         // K-cluster mode: a CTA's partial tile parked at the start of its (idle) operand ring, same
         // float4 order as slab4; `ring` is the shared::cta address of this CTA's copy
         const uint32_t ring = s_stage;
-        // KIND 1: integer accumulators -> FP32, times the scale of this lane's A row and of each B row
+        // KIND 1 / 2: accumulators (integers converted to FP32 / FP32) times the scale of this lane's A row
+        // and of each B row
         float a_scale = 0.f;
+        auto acc_f32 = [](uint32_t v) { return KIND == 1 ? static_cast<float>(static_cast<int>(v)) : __uint_as_float(v); };
         auto dequant_half = [&](uint32_t (&a)[32], const float* __restrict__ sb, int n0) {
 #pragma unroll
             for (int g = 0; g < 8; ++g) {
                 const int n = n0 + g * 4;
                 const float4 s4 = (n + 4 <= p.N) ? __ldg(reinterpret_cast<const float4*>(sb + n))
                                                  : make_float4(0.f, 0.f, 0.f, 0.f);
-                a[g * 4 + 0] = __float_as_uint(static_cast<float>(static_cast<int>(a[g * 4 + 0])) * (a_scale * s4.x));
-                a[g * 4 + 1] = __float_as_uint(static_cast<float>(static_cast<int>(a[g * 4 + 1])) * (a_scale * s4.y));
-                a[g * 4 + 2] = __float_as_uint(static_cast<float>(static_cast<int>(a[g * 4 + 2])) * (a_scale * s4.z));
-                a[g * 4 + 3] = __float_as_uint(static_cast<float>(static_cast<int>(a[g * 4 + 3])) * (a_scale * s4.w));
+                a[g * 4 + 0] = __float_as_uint(acc_f32(a[g * 4 + 0]) * (a_scale * s4.x));
+                a[g * 4 + 1] = __float_as_uint(acc_f32(a[g * 4 + 1]) * (a_scale * s4.y));
+                a[g * 4 + 2] = __float_as_uint(acc_f32(a[g * 4 + 2]) * (a_scale * s4.z));
+                a[g * 4 + 3] = __float_as_uint(acc_f32(a[g * 4 + 3]) * (a_scale * s4.w));
             }
         };
         auto dequant = [&](uint32_t (&a0)[32], uint32_t (&a1)[32], const float* __restrict__ sb, int n0) {
@@ -495,7 +504,7 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const bool sg = p.swiglu != 0;
             if (sg) colbase /= 2;                          // BN/2 output columns per tile
             const int row0 = tm * (128 * CTAS) + static_cast<int>(cta_rank) * 128 + q * 32;
-            if constexpr (KIND == 1) a_scale = (row0 + lane < p.M) ? __ldg(p.sa + row0 + lane) : 0.f;
+            if constexpr (KIND != 0) a_scale = (row0 + lane < p.M) ? __ldg(p.sa + row0 + lane) : 0.f;
             const int nchunks = (narrow || sg) ? C::CHUNKS / 2 : C::CHUNKS;
             const bool whole = (kb0 == 0) && (kb1 == nkb);
             auto chunk_inb = [&](int c) { return (row0 < p.M) && (colbase + c * 64 < p.N); };
@@ -668,7 +677,7 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     tmem_ld_32x32(tbase + c * 64, acc[0]);
                     tmem_ld_32x32(tbase + c * 64 + 32, acc[1]);
                     tmem_ld_wait();
-                    if constexpr (KIND == 1) dequant(acc[0], acc[1], p.sb, col0);
+                    if constexpr (KIND != 0) dequant(acc[0], acc[1], p.sb, col0);
                 }
                 if (valid && sg) {
                     // acc holds the gate pre-activations of these 64 output columns; the matching up
@@ -678,7 +687,7 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         uint32_t up[32];
                         tmem_ld_32x32(tbase + BN / 2 + c * 64 + h * 32, up);
                         tmem_ld_wait();
-                        if constexpr (KIND == 1) dequant_half(up, p.sb2, col0 + h * 32);
+                        if constexpr (KIND != 0) dequant_half(up, p.sb2, col0 + h * 32);
 #pragma unroll
                         for (int i = 0; i < 32; ++i) {
                             const float gte = __uint_as_float(acc[h][i]);
@@ -1337,9 +1346,9 @@ kx_rmsnorm_kernel(const uint16_t* __restrict__ H, const uint16_t* __restrict__ g
 // ===========================================================================
 // kx_rowquant_kernel
 // ===========================================================================
-// Symmetric per-row INT8 code book (the "activation quantization" fused behind add+RMSNorm and the
+// Symmetric per-row code book, INT8 (FMT 0, top code 127) or FP8 E4M3 (FMT 1, top code 448) (the "activation quantization" fused behind add+RMSNorm and the
 // one-launch gate/up weight quantisation of Appendix A, Algorithm 7):
-//     a = max_j |z_j|,  scale = a / 127,  q_j = clamp(rint(z_j * (127 / a)), -127, 127)
+//     a = max_j |z_j|,  scale = a / top,  q_j = code(z_j * (top / a))   (INT8: rint; E4M3: nearest even, saturating)
 // with every operation in binary32 (one correctly rounded division each for scale and reciprocal,
 // one product and a round-half-even per element); a zero row gets scale 1 and codes 0.
 // NORM = true: z is the BF16-rounded RMSNorm of the row (same expression, so the same bits, as
@@ -1360,9 +1369,10 @@ struct QuantParams {
     float eps;
 };
 
-template <int NV, bool NORM>
+template <int NV, bool NORM, int FMT>
 __global__ void __launch_bounds__(kNormThreads)
 kx_rowquant_kernel(const QuantParams p) {
+    constexpr float kTop = (FMT == 1) ? 448.0f : 127.0f;   // largest code magnitude: E4M3 / INT8
     __shared__ float s_part[kNormThreads / 32];
     __shared__ float s_bcast;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -1441,11 +1451,11 @@ kx_rowquant_kernel(const QuantParams p) {
 #pragma unroll
             for (int w = 0; w < kNormThreads / 32; ++w) t = fmaxf(t, s_part[w]);
             s_bcast = t;
-            (second ? p.S1 : p.S0)[r] = (t > 0.f) ? __fdiv_rn(t, 127.0f) : 1.0f;
+            (second ? p.S1 : p.S0)[r] = (t > 0.f) ? __fdiv_rn(t, kTop) : 1.0f;
         }
         __syncthreads();
         const float a = s_bcast;
-        const float rcp = (a > 0.f) ? __fdiv_rn(127.0f, a) : 0.f;
+        const float rcp = (a > 0.f) ? __fdiv_rn(kTop, a) : 0.f;
         uint2* qrow = reinterpret_cast<uint2*>((second ? p.Q1 : p.Q0) + r * N);
 #pragma unroll
         for (int i = 0; i < NV; ++i) {
@@ -1454,13 +1464,20 @@ kx_rowquant_kernel(const QuantParams p) {
                 const uint32_t w4[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
                 // |z| <= a and rcp = fl(127 / a) keep |z * rcp| below 127.5, so the codes are already
                 // within -127..127; the packing instruction saturates anyway
-                int q[8];
+                float t[8];
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
-                    q[2 * k] = __float2int_rn(__fmul_rn(bf16_lo(w4[k]), rcp));
-                    q[2 * k + 1] = __float2int_rn(__fmul_rn(bf16_hi(w4[k]), rcp));
+                    t[2 * k] = __fmul_rn(bf16_lo(w4[k]), rcp);
+                    t[2 * k + 1] = __fmul_rn(bf16_hi(w4[k]), rcp);
                 }
-                qrow[idx] = make_uint2(pack_s8x4_sat(q[0], q[1], q[2], q[3]), pack_s8x4_sat(q[4], q[5], q[6], q[7]));
+                if constexpr (FMT == 1) {
+                    qrow[idx] = make_uint2(pack_e4m3x4(t[0], t[1], t[2], t[3]), pack_e4m3x4(t[4], t[5], t[6], t[7]));
+                } else {
+                    int q[8];
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) q[k] = __float2int_rn(t[k]);
+                    qrow[idx] = make_uint2(pack_s8x4_sat(q[0], q[1], q[2], q[3]), pack_s8x4_sat(q[4], q[5], q[6], q[7]));
+                }
             }
         }
         __syncthreads();         // s_part / s_bcast are reused by the next row

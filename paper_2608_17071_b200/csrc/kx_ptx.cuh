@@ -121,6 +121,13 @@ __device__ __forceinline__ void tma_prefetch_l2_2d(const CUtensorMap* m, int x, 
                  "r"(x), "r"(y)
                  : "memory");
 }
+// Four binary32 values -> four E4M3 codes (b0 lowest): round to nearest even, saturate to +-448.
+__device__ __forceinline__ uint32_t pack_e4m3x4(float b0, float b1, float b2, float b3) {
+    uint16_t lo, hi;
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(lo) : "f"(b1), "f"(b0));
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(hi) : "f"(b3), "f"(b2));
+    return static_cast<uint32_t>(lo) | (static_cast<uint32_t>(hi) << 16);
+}
 // Four 32-bit integers -> four signed bytes (b0 lowest), each saturated to [-128, 127].
 __device__ __forceinline__ uint32_t pack_s8x4_sat(int b0, int b1, int b2, int b3) {
     uint32_t hi, d;
@@ -216,6 +223,29 @@ __device__ __forceinline__ void mma_s8(uint32_t d_tmem, uint64_t adesc, uint64_t
             "{\n\t.reg .pred p;\n\t"
             "setp.ne.b32 p, %4, 0;\n\t"
             "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+            "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+            : "memory");
+}
+// Instruction descriptor: E4M3 x E4M3 -> FP32, both operands K-major, dense.
+__host__ __device__ constexpr uint32_t idesc_e4m3_f32(int mma_m, int mma_n) {
+    return (1u << 4) | (static_cast<uint32_t>(mma_n >> 3) << 17) | (static_cast<uint32_t>(mma_m >> 4) << 24);
+}
+// One K = 32 step of FP8 operands (byte-packed) into FP32 accumulators in tensor memory.
+template <int CTAS>
+__device__ __forceinline__ void mma_f8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                       uint32_t accumulate) {
+    if constexpr (CTAS == 1)
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+            "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+            : "memory");
+    else
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
             "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
             : "memory");
 }
