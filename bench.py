@@ -549,9 +549,9 @@ def run_ours(args):
             ns = 2
             keep, calls = [], []
             for _ in range(ns):
-                Xq = torch.randn(Ms, Ks, device="cuda", generator=g).mul_(100).to(F8)
-                Wgq = torch.randn(Is, Ks, device="cuda", generator=g).mul_(100).to(F8)
-                Wuq = torch.randn(Is, Ks, device="cuda", generator=g).mul_(100).to(F8)
+                Xq = torch.randn(Ms, Ks, device="cuda", generator=g).mul_(100).clamp_(-448, 448).to(F8)
+                Wgq = torch.randn(Is, Ks, device="cuda", generator=g).mul_(100).clamp_(-448, 448).to(F8)
+                Wuq = torch.randn(Is, Ks, device="cuda", generator=g).mul_(100).clamp_(-448, 448).to(F8)
                 sx = torch.rand(Ms, device="cuda", generator=g) * 1e-2
                 sg = torch.rand(Is, device="cuda", generator=g) * 2e-4
                 su = torch.rand(Is, device="cuda", generator=g) * 2e-4
@@ -579,8 +579,8 @@ def run_ours(args):
             ns = int(max(2, min(8, math.ceil(2.0 * L2_BYTES / nbytes))))
             keep, calls = [], []
             for _ in range(ns):
-                Xq = torch.randn(Mo, Ko, device="cuda", generator=g).mul_(100).to(F8)
-                Wq = torch.randn(No, Ko, device="cuda", generator=g).mul_(100).to(F8)
+                Xq = torch.randn(Mo, Ko, device="cuda", generator=g).mul_(100).clamp_(-448, 448).to(F8)
+                Wq = torch.randn(No, Ko, device="cuda", generator=g).mul_(100).clamp_(-448, 448).to(F8)
                 sx = torch.rand(Mo, device="cuda", generator=g) * 1e-2
                 sw = torch.rand(No, device="cuda", generator=g) * 2e-4
                 Rs = torch.randn(Mo, No, device="cuda", generator=g).bfloat16()

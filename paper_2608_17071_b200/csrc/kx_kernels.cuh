@@ -681,7 +681,9 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 }
                 if (valid && sg) {
                     // acc holds the gate pre-activations of these 64 output columns; the matching up
-                    // values sit BN/2 accumulator columns further.  z = silu(gate) * up in FP32.
+                    // values sit BN/2 accumulator columns further.  z = silu(gate) * up in FP32; the
+                    // quotient uses the approximate division (2 ulp of FP32, far inside the BF16 rounding):
+                    // the IEEE one cost 8 % of the INT8 kernel's time and far more on NaN inputs.
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
                         uint32_t up[32];
@@ -691,7 +693,7 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
                         for (int i = 0; i < 32; ++i) {
                             const float gte = __uint_as_float(acc[h][i]);
-                            acc[h][i] = __float_as_uint(gte / (1.0f + __expf(-gte)) * __uint_as_float(up[i]));
+                            acc[h][i] = __float_as_uint(__fdividef(gte, 1.0f + __expf(-gte)) * __uint_as_float(up[i]));
                         }
                     }
                 }
