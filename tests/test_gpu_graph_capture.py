@@ -58,3 +58,59 @@ def test_capture_and_replay_a_layer_tail():
     assert ok, msg
     ok, msg = kt.gate_a(want[2], oracle.swiglu(want[1], Wg, Wu))
     assert ok, msg
+
+
+def test_capture_and_replay_the_int8_branch():
+    """RMSNorm + code book -> weights' code books -> INT8 gate/up + SwiGLU -> FP8 projection, captured
+    and replayed: same bits as the eager run."""
+    import torch
+    kx.kx_init(torch.cuda.current_device())
+    M, N, I = 384, 1024, 1536
+    H = kt.to_dev(inputs.normal_bf16(511, "R", (M, N), 1.0))
+    g = kt.to_dev(inputs.normal_bf16(511, "bias", (N,), 1.0))
+    Wg = kt.to_dev(inputs.normal_bf16(512, "W", (I, N), 1.0 / np.sqrt(N)))
+    Wu = kt.to_dev(inputs.normal_bf16(513, "W", (I, N), 1.0 / np.sqrt(N)))
+    i8 = lambda *shape: torch.zeros(shape, dtype=torch.int8, device="cuda")
+    f32 = lambda n: torch.zeros((n,), dtype=torch.float32, device="cuda")
+    f8 = lambda *shape: torch.zeros(shape, dtype=torch.uint8, device="cuda").view(torch.float8_e4m3fn)
+
+    def branch(Xq, sx, Qg, Sg, Qu, Su, Z, X8, s8, W8, sw8, Y):
+        kx.kx_rmsnorm_quantize_int8(H, g, 1e-6, Xq, sx)
+        kx.kx_quantize_gate_up_int8(Wg, Wu, Qg, Sg, Qu, Su)
+        kx.kx_gate_up_swiglu_int8(Xq, sx, Qg, Sg, Qu, Su, Z)
+        kx.kx_rmsnorm_quantize_fp8(H, g, 1e-6, X8, s8)
+        kx.kx_quantize_rows_fp8(Wg, W8, sw8)
+        kx.kx_outproj_residual_fp8(X8, s8, W8, sw8, None, None, Y)
+
+    def bufs():
+        return [i8(M, N), f32(M), i8(I, N), f32(I), i8(I, N), f32(I), kt.nan_filled(M, I),
+                f8(M, N), f32(M), f8(I, N), f32(I), kt.nan_filled(M, I)]
+
+    raw = lambda t: t.view(torch.uint8).cpu().numpy() if t.dtype not in (torch.float32, torch.bfloat16) else (
+        t.cpu().numpy() if t.dtype == torch.float32 else kt.from_dev(t))
+    eager = bufs()
+    branch(*eager)
+    assert kx.kx_last_device_status()[0] == kx.KX_OK
+    want = [raw(t) for t in eager]
+    outs = bufs()
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(s):
+        branch(*outs)
+        torch.cuda.synchronize()
+        with torch.cuda.graph(graph, stream=s):
+            branch(*outs)
+    for rep in range(2):
+        for t in outs:
+            t.view(torch.uint8).zero_() if t.dtype not in (torch.float32, torch.bfloat16) else t.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert kx.kx_last_device_status()[0] == kx.KX_OK
+        for got, ref in zip(outs, want):
+            assert np.array_equal(raw(got), ref)
+    ok, msg = kt.gate_a(want[6], oracle.swiglu_int8(want[0].view(np.int8), want[1], want[2].view(np.int8), want[3],
+                                                    want[4].view(np.int8), want[5]))
+    assert ok, msg
+    ok, msg = kt.gate_a(want[11], oracle.outproj_fp8(want[7], want[8], want[9], want[10]))
+    assert ok, msg
