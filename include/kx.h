@@ -259,6 +259,23 @@ int kx_gate_up_swiglu(const void* X, const void* Wg, const void* Wu, void* Z,
                       int64_t M, int64_t I, int64_t K, void* stream);
 
 /*
+ * kx_outproj_residual on row-pitched operands: row r of X starts at X + r * ldx elements, and
+ * likewise W (ldw), R (ldr), Y (ldy) -- slices of wider buffers (one head group of a fused
+ * projection, a window of a ring buffer, a padded allocation) without a packing copy.  Algorithm 3
+ * prints the dense case only; the pitches map directly onto the tensor-map row strides, so the
+ * kernels and plans are the dense ones.
+ *   ldx, ldw >= K; ldy >= N; ldr >= N (ignored when R is NULL); every pitch % 8 == 0 (rows stay
+ *   16-byte aligned); base pointers 16-byte aligned; N % 8 == 0.  K may be ANY length here (the
+ *   tail of the last k-block reads as zeros), which also covers reductions that are not a
+ *   multiple of 8 once the rows are padded to one.
+ *   R may equal Y only with ldr == ldy; any other overlap between the spans of Y and an input is
+ *   KX_ERR_OVERLAP.  Elements between N and ldy of a Y row are never written.
+ */
+int kx_outproj_residual_strided(const void* X, int64_t ldx, const void* W, int64_t ldw,
+                                const void* bias_or_null, const void* R_or_null, int64_t ldr,
+                                void* Y, int64_t ldy, int64_t M, int64_t N, int64_t K, void* stream);
+
+/*
  * ---- INT8 branch of the decoder layer (Appendix A, Algorithm 7: "run fused add+RMSNorm+
  * activation quantization", "quantize gate/up weights in one launch", "compute gate/up GEMM with
  * fused dequantization and SwiGLU epilogue"; the residual add is already part of

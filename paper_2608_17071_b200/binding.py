@@ -23,7 +23,7 @@ KX_PATH_AUTO, KX_PATH_TILE, KX_PATH_SWAP = 0, 1, 2
 
 EXPORTS = (
     "kx_init", "kx_shutdown", "kx_outproj_residual", "kx_gemm_bf16", "kx_outproj_residual_ex",
-    "kx_outproj_residual_host", "kx_outproj_residual_noalloc", "kx_rmsnorm", "kx_outproj_residual_rmsnorm",
+    "kx_outproj_residual_host", "kx_outproj_residual_noalloc", "kx_outproj_residual_strided", "kx_rmsnorm", "kx_outproj_residual_rmsnorm",
     "kx_gate_up_swiglu",
     "kx_quantize_rows_int8", "kx_quantize_gate_up_int8", "kx_rmsnorm_quantize_int8", "kx_gate_up_swiglu_int8",
     "kx_outproj_residual_int8",
@@ -80,6 +80,7 @@ def load():
     lib.kx_outproj_residual_ex.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, vp, ctypes.POINTER(PlanOverride)]
     lib.kx_outproj_residual_host.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, vp]
     lib.kx_outproj_residual_noalloc.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, vp]
+    lib.kx_outproj_residual_strided.argtypes = [vp, i64, vp, i64, vp, vp, i64, vp, i64, i64, i64, i64, vp]
     lib.kx_rmsnorm.argtypes = [vp, vp, ctypes.c_float, vp, i64, i64, vp]
     lib.kx_gate_up_swiglu.argtypes = [vp, vp, vp, vp, i64, i64, i64, vp]
     lib.kx_outproj_residual_rmsnorm.argtypes = [vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, i64, i64, i64, vp]
@@ -246,6 +247,30 @@ def _code_dtype(fmt):
     if fmt == "fp8":
         return torch.float8_e4m3fn
     raise ValueError(f"unknown 8-bit format {fmt!r} (int8 or fp8)")
+
+
+def _check_rows(name, t, shape):
+    import torch
+    if t is None:
+        return 0
+    if t.dtype != torch.bfloat16 or tuple(t.shape) != tuple(shape) or (t.shape[1] > 1 and t.stride(1) != 1):
+        raise ValueError(f"{name}: need a bfloat16 tensor of shape {tuple(shape)} with unit column stride, "
+                         f"got {t.dtype} {tuple(t.shape)} strides {tuple(t.stride())}")
+    return int(t.stride(0))
+
+
+def kx_outproj_residual_strided(X, W, bias, R, Y, stream=None, check=True) -> int:
+    """kx_outproj_residual on row-pitched views (column stride 1, any row stride that is a multiple of 8)."""
+    M, K = X.shape
+    N = W.shape[0]
+    ldx, ldw = _check_rows("X", X, (M, K)), _check_rows("W", W, (N, K))
+    ldr, ldy = _check_rows("R", R, (M, N)), _check_rows("Y", Y, (M, N))
+    _check_bf16("bias", bias, (N,))
+    rc = load().kx_outproj_residual_strided(_addr(X), ldx, _addr(W), ldw, _addr(bias), _addr(R), ldr, _addr(Y), ldy,
+                                            M, N, K, _stream(stream))
+    if check and rc != KX_OK:
+        raise KxError(rc, "kx_outproj_residual_strided")
+    return rc
 
 
 def kx_quantize_rows_int8(A, Q, S, stream=None, check=True, fmt="int8") -> int:

@@ -199,10 +199,10 @@ int ensure_device(int dev, DeviceCtx** out) {
 // contents, so rewriting a tensor in place between calls is always seen.
 struct TmapKey {
     const void* ptr;
-    uint64_t rows, cols;
+    uint64_t rows, cols, ld;
     uint32_t box_rows, elem_bytes;
     bool operator==(const TmapKey& o) const {
-        return ptr == o.ptr && rows == o.rows && cols == o.cols && box_rows == o.box_rows &&
+        return ptr == o.ptr && rows == o.rows && cols == o.cols && ld == o.ld && box_rows == o.box_rows &&
                elem_bytes == o.elem_bytes;
     }
 };
@@ -217,12 +217,14 @@ thread_local TmapEntry t_tmaps[kTmapSlots];
 // Row-major matrix [rows, cols] of BF16 (elem_bytes 2) or 8-bit (elem_bytes 1) elements;
 // box = box_rows x 128 bytes of a row; 128-byte swizzle; 256-byte L2 promotion; out-of-bounds
 // elements read as zero and are not written.
+// `ld` = row pitch in elements (0 = cols, a dense matrix).
 int get_tmap(const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows, CUtensorMap* out,
-             uint32_t elem_bytes = 2) {
-    TmapKey key{ptr, rows, cols, box_rows, elem_bytes};
+             uint32_t elem_bytes = 2, uint64_t ld = 0) {
+    if (ld == 0) ld = cols;
+    TmapKey key{ptr, rows, cols, ld, box_rows, elem_bytes};
     uint64_t h = reinterpret_cast<uint64_t>(ptr) >> 4;
     h ^= rows * 0x9E3779B97F4A7C15ull;
-    h ^= (cols + 0x7F4A7C15ull) * 0xC2B2AE3D27D4EB4Full;
+    h ^= (cols + 0x7F4A7C15ull + (ld << 32)) * 0xC2B2AE3D27D4EB4Full;
     h ^= (box_rows + 1024ull * elem_bytes) * 0x165667B19E3779F9ull;
     h ^= h >> 29;
     TmapEntry& e = t_tmaps[h % kTmapSlots];
@@ -231,7 +233,7 @@ int get_tmap(const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows, C
         return KX_OK;
     }
     cuuint64_t dims[2] = {cols, rows};
-    cuuint64_t strides[1] = {cols * elem_bytes};
+    cuuint64_t strides[1] = {ld * elem_bytes};
     cuuint32_t box[2] = {128u / elem_bytes, box_rows};
     cuuint32_t estr[2] = {1, 1};
     CUresult r = g_encode(&e.map, elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8,
@@ -544,10 +546,42 @@ bool overlaps(const void* a, size_t abytes, const void* b, size_t bbytes) {
     return a0 < b0 + bbytes && b0 < a0 + abytes;
 }
 
+// Row pitches in elements; a null `Pitch*` means dense matrices (pitch = row length).
+struct Pitch {
+    long long ldx, ldw, ldr, ldy;
+};
+// bytes from the first to one past the last element of a [rows, cols] BF16 matrix of pitch ld
+size_t span_bytes(long long rows, long long cols, long long ld) {
+    return rows > 0 ? (static_cast<size_t>(rows - 1) * ld + cols) * 2 : 0;
+}
+
 int validate(const void* X, const void* W, const void* bias, const void* R, const void* Y, long long M,
-             long long N, long long K, bool need_r) {
+             long long N, long long K, bool need_r, const Pitch* lds = nullptr) {
     if (M < 0 || N < 0 || K < 0) return KX_ERR_SHAPE;
     if (M > 0x7FFFFFFFll / 2 || N > 0x7FFFFFFFll / 2 || K > 0x7FFFFFFFll / 2) return KX_ERR_SHAPE;
+    if (lds) {
+        // the pitch must cover the row, keep every row 16-byte aligned, and stay addressable by TMA
+        if (lds->ldx < K || lds->ldw < K || lds->ldy < N || (R && lds->ldr < N)) return KX_ERR_SHAPE;
+        if ((lds->ldx % 8) || (lds->ldw % 8) || (lds->ldy % 8) || (R && (lds->ldr % 8))) return KX_ERR_SHAPE;
+        if (lds->ldx > (1ll << 36) || lds->ldw > (1ll << 36) || lds->ldy > (1ll << 36) || lds->ldr > (1ll << 36))
+            return KX_ERR_SHAPE;
+        if (M == 0 || N == 0) return KX_OK;
+        if ((N % 8) != 0) return KX_ERR_SHAPE;          // K may be any length when the pitch is given
+        if (!Y) return KX_ERR_NULL;
+        if (K > 0 && (!X || !W)) return KX_ERR_NULL;
+        if (need_r && !R) return KX_ERR_NULL;
+        if (!aligned16(Y) || (K > 0 && (!aligned16(X) || !aligned16(W))) || (R && !aligned16(R)) ||
+            (bias && !aligned16(bias)))
+            return KX_ERR_ALIGN;
+        const size_t ys = span_bytes(M, N, lds->ldy);
+        if (overlaps(Y, ys, X, span_bytes(M, K, lds->ldx)) || overlaps(Y, ys, W, span_bytes(N, K, lds->ldw)) ||
+            overlaps(Y, ys, bias, static_cast<size_t>(N) * 2))
+            return KX_ERR_OVERLAP;
+        // in place needs the same pitch; any other overlap of the two spans is refused (interleaved
+        // views that happen not to collide element-wise are not worth the risk)
+        if (R && !(R == Y && lds->ldr == lds->ldy) && overlaps(Y, ys, R, span_bytes(M, N, lds->ldr))) return KX_ERR_OVERLAP;
+        return KX_OK;
+    }
     if (M == 0 || N == 0) return KX_OK;
     if ((N % 8) != 0 || (K % 8) != 0) return KX_ERR_SHAPE;
     if (!Y) return KX_ERR_NULL;
@@ -566,10 +600,12 @@ int validate(const void* X, const void* W, const void* bias, const void* R, cons
 
 // ------------------------------------------------------------------ launch
 int run(const void* X, const void* W, const void* bias, const void* R, void* Y, long long M, long long N,
-        long long K, void* stream_v, const kx_plan_override* ov, bool need_r) {
-    int rc = validate(X, W, bias, R, Y, M, N, K, need_r);
+        long long K, void* stream_v, const kx_plan_override* ov, bool need_r, const Pitch* lds = nullptr) {
+    int rc = validate(X, W, bias, R, Y, M, N, K, need_r, lds);
     if (rc != KX_OK) return rc;
     if (M == 0 || N == 0) return KX_OK;
+    const long long ldx = lds ? lds->ldx : K, ldw = lds ? lds->ldw : K, ldr = lds ? lds->ldr : N,
+                    ldy = lds ? lds->ldy : N;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return KX_ERR_CUDA;
     DeviceCtx* ctx = nullptr;
@@ -581,7 +617,8 @@ int run(const void* X, const void* W, const void* bias, const void* R, void* Y, 
         const long long total = M * N;
         const int blocks = static_cast<int>(std::min<long long>((total + 255) / 256, ctx->sm_count * 8));
         kx_k0_kernel<<<blocks, 256, 0, stream>>>(static_cast<const uint16_t*>(bias),
-                                                 static_cast<const uint16_t*>(R), static_cast<uint16_t*>(Y), M, N);
+                                                 static_cast<const uint16_t*>(R), static_cast<uint16_t*>(Y), M, N,
+                                                 ldr, ldy);
         return cudaGetLastError() == cudaSuccess ? KX_OK : KX_ERR_CUDA;
     }
 
@@ -623,16 +660,16 @@ int run(const void* X, const void* W, const void* bias, const void* R, void* Y, 
 
     if (pl.path == KX_PATH_TILE) {
         CUtensorMap tmA, tmB, tmB2, tmY, tmR;
-        if ((rc = get_tmap(X, M, K, 128, &tmA)) != KX_OK) return rc;
-        if ((rc = get_tmap(W, N, K, pl.bn / pl.ctas, &tmB)) != KX_OK) return rc;
+        if ((rc = get_tmap(X, M, K, 128, &tmA, 2, ldx)) != KX_OK) return rc;
+        if ((rc = get_tmap(W, N, K, pl.bn / pl.ctas, &tmB, 2, ldw)) != KX_OK) return rc;
         if (pl.narrow_tile0 < pl.units) {
-            if ((rc = get_tmap(W, N, K, pl.bn / 2 / pl.ctas, &tmB2)) != KX_OK) return rc;
+            if ((rc = get_tmap(W, N, K, pl.bn / 2 / pl.ctas, &tmB2, 2, ldw)) != KX_OK) return rc;
         } else {
             tmB2 = tmB;
         }
-        if ((rc = get_tmap(Y, M, N, 32, &tmY)) != KX_OK) return rc;
+        if ((rc = get_tmap(Y, M, N, 32, &tmY, 2, ldy)) != KX_OK) return rc;
         if (R) {
-            if ((rc = get_tmap(R, M, N, 32, &tmR)) != KX_OK) return rc;
+            if ((rc = get_tmap(R, M, N, 32, &tmR, 2, ldr)) != KX_OK) return rc;
         } else {
             tmR = tmY;
         }
@@ -667,8 +704,8 @@ int run(const void* X, const void* W, const void* bias, const void* R, void* Y, 
         }
     } else {
         CUtensorMap tmW, tmX;
-        if ((rc = get_tmap(W, N, K, 128, &tmW)) != KX_OK) return rc;
-        if ((rc = get_tmap(X, M, K, pl.bn, &tmX)) != KX_OK) return rc;
+        if ((rc = get_tmap(W, N, K, 128, &tmW, 2, ldw)) != KX_OK) return rc;
+        if ((rc = get_tmap(X, M, K, pl.bn, &tmX, 2, ldx)) != KX_OK) return rc;
         SwapParams p;
         p.M = static_cast<int>(M);
         p.N = static_cast<int>(N);
@@ -688,6 +725,8 @@ int run(const void* X, const void* W, const void* bias, const void* R, void* Y, 
         p.bias = static_cast<const uint16_t*>(bias);
         p.R = static_cast<const uint16_t*>(R);
         p.Y = static_cast<uint16_t*>(Y);
+        p.ldr = ldr;
+        p.ldy = ldy;
 #ifdef KX_TRACE
         p.trace = g_kx_trace;
 #endif
@@ -779,6 +818,13 @@ int kx_gemm_bf16(const void* X, const void* W, void* Y, int64_t M, int64_t N, in
 int kx_outproj_residual_ex(const void* X, const void* W, const void* bias, const void* R, void* Y, int64_t M,
                            int64_t N, int64_t K, void* stream, const kx_plan_override* ov) {
     return run(X, W, bias, R, Y, M, N, K, stream, ov, false);
+}
+
+int kx_outproj_residual_strided(const void* X, int64_t ldx, const void* W, int64_t ldw, const void* bias,
+                                const void* R, int64_t ldr, void* Y, int64_t ldy, int64_t M, int64_t N, int64_t K,
+                                void* stream) {
+    Pitch lds{ldx, ldw, R ? ldr : N, ldy};
+    return run(X, W, bias, R, Y, M, N, K, stream, nullptr, false, &lds);
 }
 
 int kx_plan_query(int64_t M, int64_t N, int64_t K, int has_bias, int has_residual,
@@ -955,7 +1001,7 @@ int kx_gate_up_swiglu(const void* X, const void* Wg, const void* Wu, void* Z, in
     if (K == 0) {   // empty sums: silu(0) * 0 = 0
         const long long total = M * I;
         const int blocks = static_cast<int>(std::min<long long>((total + 255) / 256, ctx->sm_count * 8));
-        kx_k0_kernel<<<blocks, 256, 0, stream>>>(nullptr, nullptr, static_cast<uint16_t*>(Z), M, I);
+        kx_k0_kernel<<<blocks, 256, 0, stream>>>(nullptr, nullptr, static_cast<uint16_t*>(Z), M, I, I, I);
         return cudaGetLastError() == cudaSuccess ? KX_OK : KX_ERR_CUDA;
     }
     // one tile = 128 (x2 for a pair) rows by 128 gate + 128 up accumulator columns = 128 output columns
@@ -1368,7 +1414,7 @@ static int gate_up_swiglu_q8(int kind, const void* Xq, const float* sx, const vo
         if ((rc = device_ctx(&ctx)) != KX_OK) return rc;
         const long long total = M * I;
         const int blocks = static_cast<int>(std::min<long long>((total + 255) / 256, ctx->sm_count * 8));
-        kx_k0_kernel<<<blocks, 256, 0, stream>>>(nullptr, nullptr, static_cast<uint16_t*>(Z), M, I);
+        kx_k0_kernel<<<blocks, 256, 0, stream>>>(nullptr, nullptr, static_cast<uint16_t*>(Z), M, I, I, I);
         return cudaGetLastError() == cudaSuccess ? KX_OK : KX_ERR_CUDA;
     }
     return run_q8(kind, Xq, sx, Wgq, sg, Wuq, su, nullptr, nullptr, Z, M, I, K, true, stream);
@@ -1390,7 +1436,7 @@ static int outproj_residual_q8(int kind, const void* Xq, const float* sx, const 
         const long long total = M * N;
         const int blocks = static_cast<int>(std::min<long long>((total + 255) / 256, ctx->sm_count * 8));
         kx_k0_kernel<<<blocks, 256, 0, stream>>>(static_cast<const uint16_t*>(bias), static_cast<const uint16_t*>(R),
-                                                 static_cast<uint16_t*>(Y), M, N);
+                                                 static_cast<uint16_t*>(Y), M, N, N, N);
         return cudaGetLastError() == cudaSuccess ? KX_OK : KX_ERR_CUDA;
     }
     return run_q8(kind, Xq, sx, Wq, sw, nullptr, nullptr, bias, R, Y, M, N, K, false, stream);
@@ -1510,7 +1556,7 @@ int kx_outproj_residual_noalloc(const void* X, const void* W, const void* bias, 
         const long long total = M * N;
         const int blocks = static_cast<int>(std::min<long long>((total + 255) / 256, ctx->sm_count * 8));
         kx_k0_kernel<<<blocks, 256, 0, stream>>>(static_cast<const uint16_t*>(bias),
-                                                 static_cast<const uint16_t*>(R), static_cast<uint16_t*>(Y), M, N);
+                                                 static_cast<const uint16_t*>(R), static_cast<uint16_t*>(Y), M, N, N, N);
         return cudaGetLastError() == cudaSuccess ? KX_OK : KX_ERR_CUDA;
     }
     const int bn = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : M <= 128 ? 128 : 256;
@@ -1554,6 +1600,8 @@ int kx_outproj_residual_noalloc(const void* X, const void* W, const void* bias, 
     p.bias = static_cast<const uint16_t*>(bias);
     p.R = static_cast<const uint16_t*>(R);
     p.Y = static_cast<uint16_t*>(Y);
+    p.ldr = N;
+    p.ldy = N;
 #ifdef KX_TRACE
     p.trace = nullptr;
 #endif

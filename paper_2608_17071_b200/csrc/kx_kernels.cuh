@@ -862,6 +862,7 @@ struct SwapParams {
     const uint16_t* bias;
     const uint16_t* R;
     uint16_t* Y;
+    long long ldr, ldy;        // row pitch of R and Y in elements (N when dense)
     KX_TRACE_DECL
 };
 
@@ -1067,7 +1068,7 @@ kx_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
 #pragma unroll
                     for (int i = 0; i < 16; ++i)
                         rv[i] = (p.splits == 1 && has_r && c0 + i < m_cnt)
-                                    ? p.R[static_cast<size_t>(m0 + c0 + i) * p.N + n] : static_cast<uint16_t>(0);
+                                    ? p.R[static_cast<size_t>(m0 + c0 + i) * p.ldr + n] : static_cast<uint16_t>(0);
 #pragma unroll
                     for (int i = 0; i < 16; ++i) {
                         const int m = m0 + c0 + i;
@@ -1076,7 +1077,7 @@ kx_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
                             if (p.splits == 1) {
                                 const float v = __uint_as_float(a[i]) + bias_v +
                                                 __uint_as_float(static_cast<uint32_t>(rv[i]) << 16);
-                                p.Y[off] = static_cast<uint16_t>(pack_bf16x2(v, 0.f) & 0xFFFFu);
+                                p.Y[static_cast<size_t>(m) * p.ldy + n] = static_cast<uint16_t>(pack_bf16x2(v, 0.f) & 0xFFFFu);
                             } else {
                                 p.ws[static_cast<size_t>(sp) * p.M * p.N + off] = __uint_as_float(a[i]);
                             }
@@ -1125,9 +1126,10 @@ kx_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
                             const size_t off1 = static_cast<size_t>(m0 + (two ? i1 : i0)) * p.N + nq;
                             float4 a0 = make_float4(0.f, 0.f, 0.f, 0.f), a1 = a0;
                             uint2 r0 = make_uint2(0u, 0u), r1 = r0;
+                            const size_t row0 = static_cast<size_t>(m0 + i0), row1 = static_cast<size_t>(m0 + (two ? i1 : i0));
                             if (has_r) {
-                                r0 = *reinterpret_cast<const uint2*>(p.R + off0);
-                                if (two) r1 = *reinterpret_cast<const uint2*>(p.R + off1);
+                                r0 = *reinterpret_cast<const uint2*>(p.R + row0 * p.ldr + nq);
+                                if (two) r1 = *reinterpret_cast<const uint2*>(p.R + row1 * p.ldr + nq);
                             }
 #pragma unroll 1
                             for (int s0 = 0; s0 < p.splits; s0 += 8) {
@@ -1151,12 +1153,12 @@ kx_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
                             {
                                 const float v0 = a0.x + b4[0] + bf16_lo(r0.x), v1 = a0.y + b4[1] + bf16_hi(r0.x);
                                 const float v2 = a0.z + b4[2] + bf16_lo(r0.y), v3 = a0.w + b4[3] + bf16_hi(r0.y);
-                                *reinterpret_cast<uint2*>(p.Y + off0) = make_uint2(pack_bf16x2(v0, v1), pack_bf16x2(v2, v3));
+                                *reinterpret_cast<uint2*>(p.Y + row0 * p.ldy + nq) = make_uint2(pack_bf16x2(v0, v1), pack_bf16x2(v2, v3));
                             }
                             if (two) {
                                 const float v0 = a1.x + b4[0] + bf16_lo(r1.x), v1 = a1.y + b4[1] + bf16_hi(r1.x);
                                 const float v2 = a1.z + b4[2] + bf16_lo(r1.y), v3 = a1.w + b4[3] + bf16_hi(r1.y);
-                                *reinterpret_cast<uint2*>(p.Y + off1) = make_uint2(pack_bf16x2(v0, v1), pack_bf16x2(v2, v3));
+                                *reinterpret_cast<uint2*>(p.Y + row1 * p.ldy + nq) = make_uint2(pack_bf16x2(v0, v1), pack_bf16x2(v2, v3));
                             }
                         }
                     }
@@ -1195,7 +1197,7 @@ kx_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
             for (int u = 0; u < kPre; ++u) {
                 const int i = tile_row(warp + 4 * u);
                 rv[u] = (p.has_r && i < m_cnt)
-                            ? *reinterpret_cast<const uint2*>(p.R + static_cast<size_t>(m0 + i) * p.N + n4)
+                            ? *reinterpret_cast<const uint2*>(p.R + static_cast<size_t>(m0 + i) * p.ldr + n4)
                             : make_uint2(0u, 0u);
             }
         }
@@ -1223,14 +1225,14 @@ kx_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
                 for (int r2 = 0; r2 < 2; ++r2) {
                     const int u = u0 + r2, i = tile_row(warp + 4 * u);
                     if (i < m_cnt && n_ok) {
-                        const size_t off = static_cast<size_t>(m0 + i) * p.N + n4;
+                        const size_t off = static_cast<size_t>(m0 + i) * p.ldy + n4;
                         uint2 rr = make_uint2(0u, 0u);
                         if (u < kPre) {
 #pragma unroll
                             for (int uu = 0; uu < kPre; ++uu)
                                 if (uu == u) rr = rv[uu];
                         } else if (p.has_r) {
-                            rr = *reinterpret_cast<const uint2*>(p.R + off);
+                            rr = *reinterpret_cast<const uint2*>(p.R + static_cast<size_t>(m0 + i) * p.ldr + n4);
                         }
                         float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
@@ -1260,14 +1262,15 @@ kx_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
 
 // K == 0: the sum over k is empty, Y = R (+ bias) or zero.
 __global__ void kx_k0_kernel(const uint16_t* __restrict__ bias, const uint16_t* R, uint16_t* Y, long long M,
-                             long long N) {
+                             long long N, long long ldr, long long ldy) {
     const long long total = M * N;
     for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < total;
          i += static_cast<long long>(gridDim.x) * blockDim.x) {
+        const long long m = i / N, n = i % N;
         float v = 0.f;
-        if (bias) v += __uint_as_float(static_cast<uint32_t>(bias[i % N]) << 16);
-        if (R) v += __uint_as_float(static_cast<uint32_t>(R[i]) << 16);
-        Y[i] = static_cast<uint16_t>(pack_bf16x2(v, 0.f) & 0xFFFFu);
+        if (bias) v += __uint_as_float(static_cast<uint32_t>(bias[n]) << 16);
+        if (R) v += __uint_as_float(static_cast<uint32_t>(R[m * ldr + n]) << 16);
+        Y[m * ldy + n] = static_cast<uint16_t>(pack_bf16x2(v, 0.f) & 0xFFFFu);
     }
 }
 

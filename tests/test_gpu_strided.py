@@ -1,0 +1,92 @@
+"""Row-pitched operands: slices of wider buffers go through the same kernels (tensor-map row
+strides), on every path, and give exactly the bits of the dense call on packed copies."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2608_17071_b200 import binding as kx
+from paper_2608_17071_b200 import inputs
+
+import kxtest as kt
+
+pytestmark = pytest.mark.gpu
+
+
+def wide(bits, ld, pad_value=0x7FC0):
+    """Device buffer [rows, ld] pre-filled with NaN patterns; the matrix sits in the left columns."""
+    rows, cols = bits.shape
+    buf = torch.full((rows, ld), 0, dtype=torch.int16, device="cuda")
+    buf.fill_(np.int16(pad_value).item() if pad_value < 0x8000 else pad_value - 0x10000)
+    buf[:, :cols] = torch.from_numpy(bits.view(np.int16)).cuda()
+    return buf.view(torch.bfloat16)
+
+
+# small-M path (cluster and workspace split-K), single-CTA tiles, K cluster, CTA pairs with a half-width tail
+@pytest.mark.parametrize("M,N,K", [(1, 520, 1096), (37, 2048, 2048), (200, 1024, 4096), (300, 520, 264), (512, 2048, 2048),
+                                   (1000, 776, 1096), (2381, 4096, 512)])
+def test_strided_equals_dense(M, N, K):
+    d = inputs.make_inputs(inputs.Workload("t", M, N, K, 900 + M, True, True), stress=True)
+    Yd = kt.nan_filled(M, N)
+    kx.kx_outproj_residual(kt.to_dev(d["X"]), kt.to_dev(d["W"]), kt.to_dev(d["bias"]), kt.to_dev(d["R"]), Yd)
+    want = kt.from_dev(Yd)
+    ok, msg = kt.gate_a(want, oracle.outproj(d["X"], d["W"], d["bias"], d["R"]))
+    assert ok, msg
+    ldx, ldw, ldr, ldy = K + 64, K + 8, N + 24, N + 40
+    Xw, Ww, Rw = wide(d["X"], ldx), wide(d["W"], ldw), wide(d["R"], ldr)
+    Yw = torch.full((M, ldy), 0, dtype=torch.int16, device="cuda")
+    Yw.fill_(0x1234)
+    Yw = Yw.view(torch.bfloat16)
+    kx.kx_outproj_residual_strided(Xw[:, :K], Ww[:, :K], kt.to_dev(d["bias"]), Rw[:, :N], Yw[:, :N])
+    assert kx.kx_last_device_status()[0] == kx.KX_OK
+    got = Yw.view(torch.int16).cpu().numpy().view(np.uint16)
+    assert np.array_equal(got[:, :N], want)
+    assert (got[:, N:] == 0x1234).all()                      # the padding of Y is never written
+    # in place on a pitched residual stream, and without bias / residual
+    Rw2 = wide(d["R"], ldr, pad_value=0x1234)
+    kx.kx_outproj_residual_strided(Xw[:, :K], Ww[:, :K], kt.to_dev(d["bias"]), Rw2[:, :N], Rw2[:, :N])
+    got2 = Rw2.view(torch.int16).cpu().numpy().view(np.uint16)
+    assert np.array_equal(got2[:, :N], want) and (got2[:, N:] == 0x1234).all()
+    Yp = kt.nan_filled(M, N)
+    kx.kx_gemm_bf16(kt.to_dev(d["X"]), kt.to_dev(d["W"]), Yp)
+    kx.kx_outproj_residual_strided(Xw[:, :K], Ww[:, :K], None, None, Yw[:, :N])
+    assert np.array_equal(Yw.view(torch.int16).cpu().numpy().view(np.uint16)[:, :N], kt.from_dev(Yp))
+
+
+@pytest.mark.parametrize("M,N,K", [(5, 264, 100), (300, 520, 77), (700, 1024, 1001), (64, 128, 1), (130, 256, 63)])
+def test_any_reduction_length_with_padded_rows(M, N, K):
+    """K that is not a multiple of 8 (nor of the 64-wide k-block): rows padded to a multiple of 8; whatever
+    sits in the padding (NaN here) must not reach the result.  Ternary data: bit-exact."""
+    X = inputs.ternary_bf16(910, "X", (M, K))
+    W = inputs.ternary_bf16(910, "W", (N, K))
+    b = inputs.small_int_bf16(910, "bias", (N,), -4, 4)
+    R = inputs.small_int_bf16(910, "R", (M, N), -8, 8)
+    ld = (K + 7) // 8 * 8 + 8
+    Y = kt.nan_filled(M, N)
+    kx.kx_outproj_residual_strided(wide(X, ld)[:, :K], wide(W, ld)[:, :K], kt.to_dev(b), kt.to_dev(R), Y)
+    assert kx.kx_last_device_status()[0] == kx.KX_OK
+    ok, msg = kt.gate_exact(kt.from_dev(Y), oracle.outproj(X, W, b, R))
+    assert ok, msg
+
+
+def test_strided_argument_checks():
+    lib = kx.load()
+    A = 0x100000
+    call = lambda ldx, ldw, ldr, ldy, R=3 * A, Y=4 * A, N=64, K=64: lib.kx_outproj_residual_strided(
+        A, ldx, 2 * A, ldw, None, R, ldr, Y, ldy, 16, N, K, None)
+    assert call(56, 64, 64, 64) == kx.KX_ERR_SHAPE            # pitch shorter than the row
+    assert call(64, 64, 64, 60) == kx.KX_ERR_SHAPE
+    assert call(68, 64, 64, 64) == kx.KX_ERR_SHAPE            # pitch not a multiple of 8
+    assert call(64, 64, 64, 64, N=60) == kx.KX_ERR_SHAPE      # N % 8
+    assert call(64, 64, 64, 72, R=4 * A) == kx.KX_ERR_OVERLAP  # in place needs equal pitches
+    assert call(64, 64, 64, 64, Y=A + 32) == kx.KX_ERR_OVERLAP
+    assert call(64, 64, 64, 64, Y=4 * A + 2) == kx.KX_ERR_ALIGN
+    assert lib.kx_outproj_residual_strided(A, 64, 2 * A, 64, None, None, 0, 4 * A, 64, 0, 64, 64, None) == kx.KX_OK
+    # K == 0 on pitched buffers: Y = R + bias
+    R = inputs.small_int_bf16(920, "R", (6, 16), -8, 8)
+    Rw = wide(R, 40)
+    Yw = torch.zeros((6, 24), dtype=torch.bfloat16, device="cuda")
+    rc = lib.kx_outproj_residual_strided(None, 8, None, 8, None, Rw.data_ptr(), 40, Yw.data_ptr(), 24, 6, 16, 0, None)
+    torch.cuda.synchronize()
+    assert rc == kx.KX_OK
+    assert np.array_equal(Yw.view(torch.int16).cpu().numpy().view(np.uint16)[:, :16], R)
