@@ -265,3 +265,29 @@ def test_fp8_mlp_chain_full_size_sampled_rows():
     ref16 = oracle.swiglu(zn, Wg, Wu)
     z8 = oracle.widen_bf16(z[rows[:8]])
     assert np.sqrt(np.mean((z8 - ref16) ** 2)) / np.sqrt(np.mean(ref16 ** 2)) < 0.08
+
+
+@pytest.mark.parametrize("M,N,K", [(4096, 4096, 4096), (16384, 4096, 14336)])
+def test_fp8_projection_full_sizes_sampled_rows(M, N, K):
+    """The two projection shapes bench.py times for FP8, in that launch configuration: exact on the
+    small-value code set, then realistic codes with a residual within the gates (sampled rows)."""
+    Xq, Wq = small_codes(860, (M, K)), small_codes(861, (N, K))
+    sx, sw = pow2(862, M), pow2(863, N)
+    rows = inputs.sampled_rows(M)[::8]
+    Y = kt.nan_filled(M, N)
+    kx.kx_outproj_residual_fp8(dev8(Xq), dev(sx), dev8(Wq), dev(sw), None, None, Y)
+    status_ok()
+    y = kt.from_dev(Y)
+    assert not np.isnan(oracle.widen_bf16(y)).any()
+    ok, msg = kt.gate_exact(y[rows], oracle.outproj_fp8(Xq, sx, Wq, sw, rows=rows))
+    assert ok, msg
+    Xq2, sx2 = data_codes(864, "X", (M, K), 1.0)
+    Wq2, sw2 = data_codes(865, "W", (N, K), 1.0 / np.sqrt(K))
+    R = inputs.normal_bf16(866, "R", (M, N), 1.0)
+    kx.kx_outproj_residual_fp8(dev8(Xq2), dev(sx2), dev8(Wq2), dev(sw2), None, kt.to_dev(R), Y)
+    status_ok()
+    y = kt.from_dev(Y)
+    ref = oracle.outproj_fp8(Xq2, sx2, Wq2, sw2, None, R, rows=rows)
+    ok, msg = kt.gate_a(y[rows], ref)
+    assert ok, msg
+    assert kt.rel_fro(y[rows], ref) <= 2.0 ** -8

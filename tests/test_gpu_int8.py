@@ -317,3 +317,32 @@ def test_int8_mlp_chain_full_size_sampled_rows():
     ref16 = oracle.swiglu(zn, Wg, Wu)
     z8 = oracle.widen_bf16(z[rows[:8]])
     assert np.sqrt(np.mean((z8 - ref16) ** 2)) / np.sqrt(np.mean(ref16 ** 2)) < 0.05
+
+
+@pytest.mark.parametrize("M,N,K", [(4096, 4096, 4096), (16384, 4096, 14336)])
+def test_int8_projection_full_sizes_sampled_rows(M, N, K):
+    """The two projection shapes bench.py times in its 8-bit section, in that launch configuration:
+    codes in -15..15 keep every sum below 2^24, so with power-of-two scales and no bias / residual the
+    sampled rows must be bit-exact; then general scales with a residual within the gates."""
+    rng = np.random.default_rng(695)
+    Xq = rng.integers(-15, 16, size=(M, K), dtype=np.int8)
+    Wq = rng.integers(-15, 16, size=(N, K), dtype=np.int8)
+    sx, sw = pow2(696, M), pow2(697, N)
+    rows = inputs.sampled_rows(M)[::8]
+    Xd, Wd = dev(Xq), dev(Wq)
+    Y = kt.nan_filled(M, N)
+    kx.kx_outproj_residual_int8(Xd, dev(sx), Wd, dev(sw), None, None, Y)
+    status_ok()
+    y = kt.from_dev(Y)
+    assert not np.isnan(oracle.widen_bf16(y)).any()
+    ok, msg = kt.gate_exact(y[rows], oracle.outproj_int8(Xq, sx, Wq, sw, rows=rows))
+    assert ok, msg
+    sx2, sw2 = scales(698, M, 0.05), scales(699, N, 0.02 / np.sqrt(K))
+    R = inputs.normal_bf16(700, "R", (M, N), 1.0)
+    kx.kx_outproj_residual_int8(Xd, dev(sx2), Wd, dev(sw2), None, kt.to_dev(R), Y)
+    status_ok()
+    y = kt.from_dev(Y)
+    ref = oracle.outproj_int8(Xq, sx2, Wq, sw2, None, R, rows=rows)
+    ok, msg = kt.gate_a(y[rows], ref)
+    assert ok, msg
+    assert float((oracle.round_bf16(ref) != y[rows]).mean()) <= 0.01
