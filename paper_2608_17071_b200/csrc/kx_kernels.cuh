@@ -24,6 +24,12 @@
 //                   partials go to an FP32 workspace and the last CTA to finish sums
 //                   them.  Bias and residual are applied once.
 //   kx_rmsnorm_kernel  z = h * rsqrt(mean h^2 + eps) * gamma over BF16 rows, one pass.
+//   kx_rowquant_kernel per-row 8-bit code book (INT8 or FP8 E4M3 codes + one FP32 scale per row)
+//                   of BF16 rows, optionally of their RMSNorm, one pass.
+//
+// kx_tile_kernel also runs on 8-bit operands (template parameter KIND: tcgen05 kind::i8 with
+// integer accumulators, or kind::f8f6f4 with FP32 accumulators) and then dequantises in its
+// epilogue with one scale per operand row.
 //
 // The projection is the paper's residual GEMM epilogue (Appendix A, Algorithm 3:
 // O <- W^T A + O, alpha = beta = 1, output aliased onto the residual) and the plain
@@ -31,10 +37,10 @@
 // decoder layer in Algorithm 7.  The warp roles follow the curriculum of Table 2
 // (tensor-core pipeline, producer/consumer specialisation, persistent CTAs with raw
 // mbarriers, chunked TMA epilogue, tile scheduling) re-expressed for Blackwell:
-// tcgen05 + TMEM replace WGMMA, and a CTA pair (cta_group::2) replaces the cluster
-// multicast tier.  Both GEMM kernels start with a prologue that touches only the
-// CTA's own resources and then wait for the previous kernel in the stream
-// (programmatic dependent launch).
+// tcgen05 + TMEM replace WGMMA, and a CTA pair (cta_group::2) replaces the tier in which
+// the CTAs of a cluster share operand tiles.  Both GEMM kernels start with a prologue that
+// touches only the CTA's own resources (plus L2 prefetch hints for its first operand tiles)
+// and then wait for the previous kernel in the stream (programmatic dependent launch).
 //
 // Every wait on an mbarrier is bounded: after `spin_limit_ns` the waiting thread
 // records where it gave up, raises a CTA-wide abort flag and every role falls
