@@ -399,7 +399,14 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                                               : KIND == 2 ? idesc_e4m3_f32(128 * CTAS, BN / 2)
                                                           : idesc_bf16_f32(128 * CTAS, BN / 2);
             uint32_t s = 0, ph = 0, scount = 0;
+            // running addresses of the current stage: its `full` barrier, its `empty` barrier as seen from
+            // each CTA of the pair, and the low word of its A-tile descriptor
+            const uint32_t a_lo0 = smem_desc_lo(s_stage);
+            const uint32_t empty_base0 = (CTAS == 1) ? empty(0) : map_to_cta(empty(0), 0);
+            const uint32_t empty_base1 = (CTAS == 1) ? 0u : map_to_cta(empty(0), 1);
+            uint32_t full_bar = full(0), empty_bar0 = empty_base0, empty_bar1 = empty_base1, a_lo = a_lo0;
             bool ok = true;
+            bool have = false;   // the current stage was already seen full by the previous k-block's early test
             while (ok && it.next(tile, kb0, kb1)) {
                 const uint32_t b = scount & 1u, aph = (scount >> 1) & 1u;
                 const uint32_t idesc = (tile >= p.narrow_tile0) ? idesc_narrow : idesc_wide;
@@ -410,29 +417,21 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 KX_TRACE_POINT(p, slot, (scount - 1) * 4 + 1);
                 const uint32_t d = tmem_base + b * BN;
                 for (int kb = kb0; kb < kb1; ++kb) {
-                    if (!wt.wait(full(s), ph, kWhereFull)) { ok = false; break; }
+                    if (!have && !wt.wait(full_bar, ph, kWhereFull)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t sa = s_stage + s * C::STAGE_BYTES;
-                    const uint32_t sb = sa + kABytes;
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        if constexpr (KIND == 1)
-                            mma_s8<CTAS>(d, smem_desc_sw128(sa + k * 32), smem_desc_sw128(sb + k * 32), idesc,
-                                         static_cast<uint32_t>((kb - kb0) | k));
-                        else if constexpr (KIND == 2)
-                            mma_f8<CTAS>(d, smem_desc_sw128(sa + k * 32), smem_desc_sw128(sb + k * 32), idesc,
-                                         static_cast<uint32_t>((kb - kb0) | k));
-                        else
-                            mma_bf16<CTAS>(d, smem_desc_sw128(sa + k * 32), smem_desc_sw128(sb + k * 32), idesc,
-                                           static_cast<uint32_t>((kb - kb0) | k));
-                    }
-                    if constexpr (CTAS == 1) {
-                        mma_commit<1>(empty(s));
+                    // the next stage in ring order (also the first stage of the next tile)
+                    const bool wrap = (s + 1 == STAGES);
+                    const uint32_t next_full = wrap ? full(0) : full_bar + 8u;
+                    have = mma_kblock<CTAS, KIND>(d, a_lo, a_lo + (kABytes >> 4), idesc, static_cast<uint32_t>(kb - kb0),
+                                                  next_full, wrap ? (ph ^ 1u) : ph, empty_bar0, empty_bar1) != 0u;
+                    full_bar = next_full;
+                    if (wrap) {
+                        s = 0; ph ^= 1u;
+                        empty_bar0 = empty_base0; empty_bar1 = empty_base1; a_lo = a_lo0;
                     } else {
-                        mma_commit<2>(map_to_cta(empty(s), 0));
-                        mma_commit<2>(map_to_cta(empty(s), 1));
+                        ++s;
+                        empty_bar0 += 8u; empty_bar1 += 8u; a_lo += C::STAGE_BYTES >> 4;
                     }
-                    if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
                 if (!ok) break;
                 if constexpr (CTAS == 1) {
