@@ -148,11 +148,14 @@ struct TileParams {
     KX_TRACE_DECL
 };
 
-template <int BN, int CTAS, int STAGES, int NB>
+// KBS = k-blocks per ring stage (1 or 2).  With 2, a stage is [A kb][A kb+1][B kb][B kb+1]: one
+// barrier round trip and one commit per eight K steps instead of four.
+template <int BN, int CTAS, int STAGES, int NB, int KBS = 1>
 struct TileCfg {
     static constexpr int BN_LOAD = BN / CTAS;               // W rows this CTA loads per k-block
     static constexpr int B_BYTES = BN_LOAD * 128;
-    static constexpr int STAGE_BYTES = kABytes + B_BYTES;
+    static constexpr int STAGE_BYTES = KBS * (kABytes + B_BYTES);
+    static_assert(KBS == 1 || KBS == 2, "KBS");
     static constexpr int SLAB_BYTES = 32 * 128;             // 32 rows x 64 BF16 per warp per chunk
     static constexpr int EPI_BYTES = 4 * NB * SLAB_BYTES;
     static constexpr int NUM_BARS = 2 * STAGES + 4 + 4 * NB + 1;
@@ -223,12 +226,12 @@ __device__ __forceinline__ uint32_t ld_acquire_gpu_u32(const unsigned int* p) {
 // (same byte geometry), FP32 accumulators.  KIND 1 and 2 are dequantised in the epilogue with a
 // per-row scale of A and a per-row scale of B; they run whole tiles only (the stream-K and
 // K-cluster fix-ups add partial accumulators as unscaled FP32).
-template <int BN, int CTAS, int STAGES, int NB, int KIND = 0>
+template <int BN, int CTAS, int STAGES, int NB, int KIND = 0, int KBS = 1>
 __global__ void __launch_bounds__(kThreads, 1)
 kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmB2, const __grid_constant__ CUtensorMap tmY,
                const __grid_constant__ CUtensorMap tmR, const uint16_t* __restrict__ bias, const TileParams p) {
-    using C = TileCfg<BN, CTAS, STAGES, NB>;
+    using C = TileCfg<BN, CTAS, STAGES, NB, KBS>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -363,22 +366,29 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 const CUtensorMap* const mapB =
                     sg ? ((CTAS == 2 && cta_rank == 1) ? &tmB2 : &tmB) : (narrow ? &tmB2 : &tmB);
                 const uint32_t stage_tx = kABytes + (narrow ? C::B_BYTES / 2 : C::B_BYTES);
-                const int kb_end = kb1 - p.drop_kblocks;
-                for (int kb = kb0; kb < kb_end; ++kb) {
+                // stages of this segment (the test hook withholds whole stages)
+                const int nst = (kb1 - kb0 + KBS - 1) / KBS - p.drop_kblocks;
+                for (int st = 0; st < nst; ++st) {
+                    const int kb = kb0 + st * KBS;
+                    const int nsub = (KBS == 2 && kb + 1 < kb1) ? 2 : 1;     // k-blocks in this stage
                     if (!wt.wait(empty(s), ph ^ 1u, kWhereEmpty)) { ok = false; break; }
                     const uint32_t sa = s_stage + s * C::STAGE_BYTES;
-                    const uint32_t sb = sa + kABytes;
+                    const uint32_t sb = sa + KBS * kABytes;
                     if constexpr (CTAS == 1) {
-                        mbar_arrive_expect_tx(full(s), stage_tx);
-                        tma_load_2d(sa, &tmA, kb * KBLK, a_row, full(s));
-                        tma_load_2d(sb, mapB, kb * KBLK, b_row, full(s));
-                        if (sg) tma_load_2d(sb + C::B_BYTES / 2, &tmB2, kb * KBLK, b_row, full(s));
+                        mbar_arrive_expect_tx(full(s), nsub * stage_tx);
+                        for (int j = 0; j < nsub; ++j) {
+                            tma_load_2d(sa + j * kABytes, &tmA, (kb + j) * KBLK, a_row, full(s));
+                            tma_load_2d(sb + j * C::B_BYTES, mapB, (kb + j) * KBLK, b_row, full(s));
+                            if (sg) tma_load_2d(sb + j * C::B_BYTES + C::B_BYTES / 2, &tmB2, (kb + j) * KBLK, b_row, full(s));
+                        }
                     } else {
                         // both CTAs' copies complete on the leader's barrier
-                        if (leader) mbar_arrive_expect_tx(full(s), 2 * stage_tx);
+                        if (leader) mbar_arrive_expect_tx(full(s), 2 * nsub * stage_tx);
                         const uint32_t fb = map_to_cta(full(s), 0);
-                        tma_load_2d_pair(sa, &tmA, kb * KBLK, a_row, fb);
-                        tma_load_2d_pair(sb, mapB, kb * KBLK, b_row, fb);
+                        for (int j = 0; j < nsub; ++j) {
+                            tma_load_2d_pair(sa + j * kABytes, &tmA, (kb + j) * KBLK, a_row, fb);
+                            tma_load_2d_pair(sb + j * C::B_BYTES, mapB, (kb + j) * KBLK, b_row, fb);
+                        }
                     }
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
@@ -416,14 +426,21 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 tc_fence_after();
                 KX_TRACE_POINT(p, slot, (scount - 1) * 4 + 1);
                 const uint32_t d = tmem_base + b * BN;
-                for (int kb = kb0; kb < kb1; ++kb) {
+                for (int kb = kb0; kb < kb1; kb += KBS) {
                     if (!have && !wt.wait(full_bar, ph, kWhereFull)) { ok = false; break; }
                     tc_fence_after();
                     // the next stage in ring order (also the first stage of the next tile)
                     const bool wrap = (s + 1 == STAGES);
                     const uint32_t next_full = wrap ? full(0) : full_bar + 8u;
-                    have = mma_kblock<CTAS, KIND>(d, a_lo, a_lo + (kABytes >> 4), idesc, static_cast<uint32_t>(kb - kb0),
-                                                  next_full, wrap ? (ph ^ 1u) : ph, empty_bar0, empty_bar1) != 0u;
+                    const uint32_t next_ph = wrap ? (ph ^ 1u) : ph;
+                    const uint32_t b_lo = a_lo + ((KBS * kABytes) >> 4);
+                    if (KBS == 2 && kb + 1 < kb1)
+                        have = mma_kblock<CTAS, KIND, true>(d, a_lo, b_lo, idesc, static_cast<uint32_t>(kb - kb0), next_full,
+                                                            next_ph, empty_bar0, empty_bar1, a_lo + (kABytes >> 4),
+                                                            b_lo + (C::B_BYTES >> 4)) != 0u;
+                    else
+                        have = mma_kblock<CTAS, KIND, false>(d, a_lo, b_lo, idesc, static_cast<uint32_t>(kb - kb0), next_full,
+                                                             next_ph, empty_bar0, empty_bar1) != 0u;
                     full_bar = next_full;
                     if (wrap) {
                         s = 0; ph ^= 1u;

@@ -277,41 +277,40 @@ __device__ __forceinline__ void mma_bf16(uint32_t d_tmem, uint64_t adesc, uint64
 // that releases the stage (to both CTAs of a pair); (4) only now the test's result is read.
 // `acc_first` = 0 makes the first step overwrite the accumulator.  Returns 1 if the next stage was
 // already full.
-#define KX_MMA_STEPS(GROUP, KINDSTR)                                                                       \
-        "setp.ne.b32 p, %5, 0;\n\t"                                                                        \
-        "setp.eq.b32 q, %1, %1;\n\t"                                                                       \
-        "mov.b64 da, {%2, %6};\n\t"                                                                        \
-        "mov.b64 db, {%3, %6};\n\t"                                                                        \
-        "tcgen05.mma.cta_group::" GROUP ".kind::" KINDSTR " [%1], da, db, %4, p;\n\t"                      \
-        "add.u32 al, %2, 2;\n\tadd.u32 bl, %3, 2;\n\tmov.b64 da, {al, %6};\n\tmov.b64 db, {bl, %6};\n\t"     \
+#define KX_MMA_STEPS(GROUP, KINDSTR, A, B, P0)                                                              \
+        "mov.b64 da, {" A ", %6};\n\t"                                                                      \
+        "mov.b64 db, {" B ", %6};\n\t"                                                                      \
+        "tcgen05.mma.cta_group::" GROUP ".kind::" KINDSTR " [%1], da, db, %4, " P0 ";\n\t"                  \
+        "add.u32 al, " A ", 2;\n\tadd.u32 bl, " B ", 2;\n\tmov.b64 da, {al, %6};\n\tmov.b64 db, {bl, %6};\n\t" \
         "tcgen05.mma.cta_group::" GROUP ".kind::" KINDSTR " [%1], da, db, %4, q;\n\t"                      \
-        "add.u32 al, %2, 4;\n\tadd.u32 bl, %3, 4;\n\tmov.b64 da, {al, %6};\n\tmov.b64 db, {bl, %6};\n\t"     \
+        "add.u32 al, " A ", 4;\n\tadd.u32 bl, " B ", 4;\n\tmov.b64 da, {al, %6};\n\tmov.b64 db, {bl, %6};\n\t" \
         "tcgen05.mma.cta_group::" GROUP ".kind::" KINDSTR " [%1], da, db, %4, q;\n\t"                      \
-        "add.u32 al, %2, 6;\n\tadd.u32 bl, %3, 6;\n\tmov.b64 da, {al, %6};\n\tmov.b64 db, {bl, %6};\n\t"     \
+        "add.u32 al, " A ", 6;\n\tadd.u32 bl, " B ", 6;\n\tmov.b64 da, {al, %6};\n\tmov.b64 db, {bl, %6};\n\t" \
         "tcgen05.mma.cta_group::" GROUP ".kind::" KINDSTR " [%1], da, db, %4, q;\n\t"
-#define KX_MMA_KBLOCK1(KINDSTR)                                                                            \
-    asm volatile(                                                                                          \
+#define KX_MMA_HEAD                                                                                        \
         "{\n\t.reg .pred p, q, r;\n\t.reg .b64 da, db;\n\t.reg .b32 al, bl;\n\t"                          \
         "mbarrier.test_wait.parity.shared::cta.b64 r, [%7], %8;\n\t"                                       \
-        KX_MMA_STEPS("1", KINDSTR)                                                                         \
+        "setp.ne.b32 p, %5, 0;\n\t"                                                                        \
+        "setp.eq.b32 q, %1, %1;\n\t"
+#define KX_MMA_TAIL1 \
         "tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%9];\n\t"                  \
-        "selp.u32 %0, 1, 0, r;\n\t}"                                                                       \
-        : "=r"(next_ok)                                                                                    \
-        : "r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(acc_first), "r"(desc_hi), "r"(next_full),     \
-          "r"(next_parity), "r"(empty0), "r"(empty1)                                                       \
-        : "memory")
-#define KX_MMA_KBLOCK2(KINDSTR)                                                                            \
-    asm volatile(                                                                                          \
-        "{\n\t.reg .pred p, q, r;\n\t.reg .b64 da, db;\n\t.reg .b32 al, bl;\n\t"                          \
-        "mbarrier.test_wait.parity.shared::cta.b64 r, [%7], %8;\n\t"                                       \
-        KX_MMA_STEPS("2", KINDSTR)                                                                         \
+        "selp.u32 %0, 1, 0, r;\n\t}"
+#define KX_MMA_TAIL2 \
         "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%9];\n\t"                  \
         "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%10];\n\t"                 \
-        "selp.u32 %0, 1, 0, r;\n\t}"                                                                       \
+        "selp.u32 %0, 1, 0, r;\n\t}"
+#define KX_MMA_OPERANDS                                                                                    \
         : "=r"(next_ok)                                                                                    \
         : "r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(acc_first), "r"(desc_hi), "r"(next_full),     \
-          "r"(next_parity), "r"(empty0), "r"(empty1)                                                       \
-        : "memory")
+          "r"(next_parity), "r"(empty0), "r"(empty1), "r"(a_lo2), "r"(b_lo2)                               \
+        : "memory"
+// one k-block per stage
+#define KX_MMA_KBLOCK(GROUP, KINDSTR, TAIL)                                                                \
+    asm volatile(KX_MMA_HEAD KX_MMA_STEPS(GROUP, KINDSTR, "%2", "%3", "p") TAIL KX_MMA_OPERANDS)
+// two k-blocks per stage: eight K steps between one barrier test and one commit
+#define KX_MMA_KBLOCK_X2(GROUP, KINDSTR, TAIL)                                                             \
+    asm volatile(KX_MMA_HEAD KX_MMA_STEPS(GROUP, KINDSTR, "%2", "%3", "p")                                 \
+                 KX_MMA_STEPS(GROUP, KINDSTR, "%11", "%12", "q") TAIL KX_MMA_OPERANDS)
 constexpr uint32_t kDescHiSw128 = (1024u >> 4) | (1u << 14) | (2u << 29);   // SBO 1024 B, version 1, SWIZZLE_128B
 __device__ __forceinline__ uint32_t smem_desc_lo(uint32_t smem_addr) {
     return ((smem_addr & 0x3FFFFu) >> 4) | (1u << 16);
@@ -319,25 +318,38 @@ __device__ __forceinline__ uint32_t smem_desc_lo(uint32_t smem_addr) {
 // KIND: 0 = BF16 (kind::f16), 1 = signed 8-bit (kind::i8), 2 = FP8 E4M3 (kind::f8f6f4).
 // empty0 / empty1: shared::cluster addresses of the stage's `empty` barrier in CTA 0 / CTA 1 of
 // the pair (empty1 unused for CTAS == 1); next_full / next_parity: the next stage's `full` barrier.
-template <int CTAS, int KIND>
+// TWO: the stage holds a second k-block whose descriptors' low words are a_lo2 / b_lo2.
+template <int CTAS, int KIND, bool TWO>
 __device__ __forceinline__ uint32_t mma_kblock(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc,
                                                uint32_t acc_first, uint32_t next_full, uint32_t next_parity,
-                                               uint32_t empty0, uint32_t empty1) {
+                                               uint32_t empty0, uint32_t empty1, uint32_t a_lo2 = 0,
+                                               uint32_t b_lo2 = 0) {
     const uint32_t desc_hi = kDescHiSw128;
     uint32_t next_ok;
-    if constexpr (CTAS == 1) {
-        if constexpr (KIND == 1) KX_MMA_KBLOCK1("i8");
-        else if constexpr (KIND == 2) KX_MMA_KBLOCK1("f8f6f4");
-        else KX_MMA_KBLOCK1("f16");
-    } else {
-        if constexpr (KIND == 1) KX_MMA_KBLOCK2("i8");
-        else if constexpr (KIND == 2) KX_MMA_KBLOCK2("f8f6f4");
-        else KX_MMA_KBLOCK2("f16");
+#define KX_MMA_DISPATCH(GROUP, TAIL)                                                                       \
+    if constexpr (TWO) {                                                                                   \
+        if constexpr (KIND == 1) KX_MMA_KBLOCK_X2(GROUP, "i8", TAIL);                                      \
+        else if constexpr (KIND == 2) KX_MMA_KBLOCK_X2(GROUP, "f8f6f4", TAIL);                             \
+        else KX_MMA_KBLOCK_X2(GROUP, "f16", TAIL);                                                         \
+    } else {                                                                                               \
+        if constexpr (KIND == 1) KX_MMA_KBLOCK(GROUP, "i8", TAIL);                                         \
+        else if constexpr (KIND == 2) KX_MMA_KBLOCK(GROUP, "f8f6f4", TAIL);                                \
+        else KX_MMA_KBLOCK(GROUP, "f16", TAIL);                                                            \
     }
+    if constexpr (CTAS == 1) {
+        KX_MMA_DISPATCH("1", KX_MMA_TAIL1)
+    } else {
+        KX_MMA_DISPATCH("2", KX_MMA_TAIL2)
+    }
+#undef KX_MMA_DISPATCH
     return next_ok;
 }
-#undef KX_MMA_KBLOCK1
-#undef KX_MMA_KBLOCK2
+#undef KX_MMA_KBLOCK
+#undef KX_MMA_KBLOCK_X2
+#undef KX_MMA_OPERANDS
+#undef KX_MMA_TAIL1
+#undef KX_MMA_TAIL2
+#undef KX_MMA_HEAD
 #undef KX_MMA_STEPS
 // Arrive on an mbarrier once every MMA issued so far by this thread has finished.
 // `bar` is a shared::cluster address (this CTA's own shared::cta address is one).

@@ -18,6 +18,11 @@ TILE_VARIANTS = [
     dict(path=T, block_n=64, cta_pair=1), dict(path=T, block_n=256, cta_pair=2),
     dict(path=T, block_n=128, cta_pair=2), dict(path=T, block_n=192, cta_pair=1),
     dict(path=T, block_n=192, cta_pair=2),
+    # the variants with two k-blocks per ring stage (selected by their stage count)
+    dict(path=T, block_n=256, cta_pair=2, stages=3), dict(path=T, block_n=256, cta_pair=1, stages=2),
+    dict(path=T, block_n=192, cta_pair=1, stages=2), dict(path=T, block_n=128, cta_pair=1, stages=3),
+    dict(path=T, block_n=64, cta_pair=1, stages=4), dict(path=T, block_n=192, cta_pair=2, stages=3),
+    dict(path=T, block_n=128, cta_pair=2, stages=4),
 ]
 SWAP_VARIANTS = [
     dict(path=S, block_n=16, split_k=1), dict(path=S, block_n=16, split_k=4),
@@ -93,6 +98,8 @@ STREAMK_VARIANTS = [
     dict(path=T, block_n=256, cta_pair=1, stream_k=2), dict(path=T, block_n=256, cta_pair=2, stream_k=2),
     dict(path=T, block_n=128, cta_pair=1, stream_k=2), dict(path=T, block_n=192, cta_pair=2, stream_k=2),
     dict(path=T, block_n=64, cta_pair=1, stream_k=2),
+    # two k-blocks per ring stage: segments start at any k-block, stages pair up from there
+    dict(path=T, block_n=256, cta_pair=2, stream_k=2, stages=3), dict(path=T, block_n=128, cta_pair=1, stream_k=2, stages=3),
 ]
 
 
@@ -119,7 +126,9 @@ def test_stream_k_exact_integer_arithmetic(ov, max_ctas, M, N, K):
     (dict(path=T, block_n=256, cta_pair=1), 10, 640, 1280),    # 25 tiles on 10 slots: 20 wide + 10 narrow
     (dict(path=T, block_n=128, cta_pair=2), 12, 700, 520),     # 15 pair tiles on 6 slots, ragged rows and columns
     (dict(path=T, block_n=128, cta_pair=1), 9, 300, 776),
-], ids=["pair256", "single256", "pair128-ragged", "single128-ragged"])
+    (dict(path=T, block_n=256, cta_pair=2, stages=3), 12, 640, 1280),     # two k-blocks per ring stage
+    (dict(path=T, block_n=128, cta_pair=2, stages=4), 12, 700, 520),
+], ids=["pair256", "single256", "pair128-ragged", "single128-ragged", "pair256-2kb", "pair128-2kb-ragged"])
 def test_half_width_tail_tiles_exact(ov, max_ctas, M, N):
     """Tiles left over after the full waves run as half-width tiles (second W tensor map,
     narrower MMA, half the epilogue chunks).  Must be bit-exact, also in place."""
