@@ -441,6 +441,11 @@ int make_plan_from(long long M, long long N, long long K, const kx_plan_override
             static_cast<long long>(ceil_div(M, 256)) * ceil_div(N, 256) >= 2ll * slots) {
             if (const TileVariant* v2 = find_tile(256, 2, 3)) v = v2;
         }
+        // 128-wide single-CTA tiles under an automatic K cluster (M = 256..512, small hidden sizes):
+        // the same variant family, measured 3 % faster there.
+        if (!(ov && ov->stages) && ctas == 1 && bn == 128 && auto_kc == 2) {
+            if (const TileVariant* v2 = find_tile(128, 1, 3)) v = v2;
+        }
         if (ov && ov->split_k > 1) return KX_ERR_PLAN;
         pl->bn = bn;
         pl->ctas = ctas;
