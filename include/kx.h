@@ -73,7 +73,8 @@ enum { KX_PATH_AUTO = 0, KX_PATH_TILE = 1, KX_PATH_SWAP = 2 };
  *   raster_group  tile path: number of 128-row tile rows that share a raster group
  *   max_ctas      cap on the persistent grid (0 = number of SMs)
  *   spin_limit_us bound on every device-side wait (0 = 2 000 000 us)
- *   stages        tile path: pick the variant with this ring depth (0 = default)
+ *   stages        pick the kernel variant with this ring depth (0 = default); variants whose stages
+ *                 hold two k-blocks have their own (smaller) stage counts
  *   stream_k      tile path: 0 auto, 1 = whole tiles per CTA (round-robin), 2 = stream-K
  *                 (every CTA gets an equal contiguous range of (tile, k-block) units;
  *                 split tiles are summed in the FP32 workspace in a fixed order)

@@ -86,11 +86,11 @@ struct SwapVariant {
             reinterpret_cast<const void*>(&kx_tile_kernel<BN, CTAS, ST, NB, 1, KBS>),         \
             reinterpret_cast<const void*>(&kx_tile_kernel<BN, CTAS, ST, NB, 2, KBS>)          \
     }
-#define KX_SWAP(BN, ST)                                                                       \
+#define KX_SWAP(BN, ST, KBS)                                                                  \
     SwapVariant {                                                                             \
-        BN, ST, SwapCfg<BN, ST>::SMEM_BYTES,                                                  \
-            reinterpret_cast<const void*>(&kx_swap_kernel<BN, ST, false>),                    \
-            reinterpret_cast<const void*>(&kx_swap_kernel<BN, ST, true>)                      \
+        BN, ST, SwapCfg<BN, ST, KBS>::SMEM_BYTES,                                             \
+            reinterpret_cast<const void*>(&kx_swap_kernel<BN, ST, false, KBS>),               \
+            reinterpret_cast<const void*>(&kx_swap_kernel<BN, ST, true, KBS>)                 \
     }
 
 // (tile width, CTAs per tile, ring stages, R staging buffers, k-blocks per stage).  The first entry
@@ -102,8 +102,10 @@ const TileVariant kTileVariants[] = {
     KX_TILE(256, 1, 2, 2, 2), KX_TILE(192, 1, 2, 3, 2), KX_TILE(128, 1, 3, 2, 2), KX_TILE(64, 1, 4, 2, 2),
     KX_TILE(256, 2, 3, 2, 2), KX_TILE(192, 2, 3, 3, 2), KX_TILE(128, 2, 4, 2, 2),
 };
+// (X rows per unit, ring stages, k-blocks per stage); first match = default, the rest by `stages`
 const SwapVariant kSwapVariants[] = {
-    KX_SWAP(16, 12), KX_SWAP(32, 11), KX_SWAP(64, 9), KX_SWAP(128, 7), KX_SWAP(256, 4),
+    KX_SWAP(16, 6, 2), KX_SWAP(32, 5, 2), KX_SWAP(64, 4, 2), KX_SWAP(128, 3, 2), KX_SWAP(256, 2, 2),
+    KX_SWAP(16, 12, 1), KX_SWAP(32, 11, 1), KX_SWAP(64, 9, 1), KX_SWAP(128, 7, 1), KX_SWAP(256, 4, 1),
 };
 
 // first variant in table order that matches; stages == 0 matches any depth
@@ -112,9 +114,9 @@ const TileVariant* find_tile(int bn, int ctas, int stages) {
         if (v.bn == bn && v.ctas == ctas && (stages == 0 || v.stages == stages)) return &v;
     return nullptr;
 }
-const SwapVariant* find_swap(int bn) {
+const SwapVariant* find_swap(int bn, int stages = 0) {
     for (const auto& v : kSwapVariants)
-        if (v.bn == bn) return &v;
+        if (v.bn == bn && (stages == 0 || v.stages == stages)) return &v;
     return nullptr;
 }
 
@@ -515,7 +517,7 @@ int make_plan_from(long long M, long long N, long long K, const kx_plan_override
     } else {
         int bn = ov ? ov->block_n : 0;
         if (bn == 0) bn = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : M <= 128 ? 128 : 256;
-        const SwapVariant* v = find_swap(bn);
+        const SwapVariant* v = find_swap(bn, ov ? ov->stages : 0);
         if (!v) return KX_ERR_PLAN;
         if (ov && ov->cta_pair > 1) return KX_ERR_PLAN;
         pl->bn = bn;

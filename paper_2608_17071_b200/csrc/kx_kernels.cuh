@@ -888,10 +888,11 @@ struct SwapParams {
     KX_TRACE_DECL
 };
 
-template <int BN, int STAGES>
+// KBS = k-blocks per ring stage (1 or 2), as in TileCfg: [W kb][W kb+1][X kb][X kb+1].
+template <int BN, int STAGES, int KBS = 1>
 struct SwapCfg {
     static constexpr int B_BYTES = BN * 128;
-    static constexpr int STAGE_BYTES = kABytes + B_BYTES;
+    static constexpr int STAGE_BYTES = KBS * (kABytes + B_BYTES);
     static constexpr int NUM_BARS = 2 * STAGES + 4 + 2;
     static constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + 1024;
     static constexpr int TMEM_COLS = tmem_cols_for(2 * BN);
@@ -905,11 +906,11 @@ struct SwapCfg {
 // its own shared memory, the cluster meets on the hardware cluster barrier, and every CTA
 // then finishes a share of the tile's rows by reading all partials through distributed
 // shared memory in split order: no workspace, no atomics, no fences, same deterministic sum.
-template <int BN, int STAGES, bool CLUSTER>
+template <int BN, int STAGES, bool CLUSTER, int KBS = 1>
 __global__ void __launch_bounds__(kThreads, 1)
 kx_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
                const SwapParams p) {
-    using C = SwapCfg<BN, STAGES>;
+    using C = SwapCfg<BN, STAGES, KBS>;
     static_assert(!CLUSTER || BN * 128 * 4 <= STAGES * C::STAGE_BYTES, "partial must fit in the idle ring");
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -997,13 +998,19 @@ kx_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
             for (int u = blockIdx.x; u < p.num_units && ok; u += gridDim.x) {
                 int nt, mt, sp, kb0, kb1;
                 unit_coords(u, nt, mt, sp, kb0, kb1);
-                kb1 -= p.drop_kblocks;
-                for (int kb = kb0; kb < kb1; ++kb) {
+                // stages of this unit (the test hook withholds whole stages)
+                const int nst = (kb1 - kb0 + KBS - 1) / KBS - p.drop_kblocks;
+                for (int st = 0; st < nst; ++st) {
+                    const int kb = kb0 + st * KBS;
+                    const int nsub = (KBS == 2 && kb + 1 < kb1) ? 2 : 1;
                     if (!wt.wait(empty(s), ph ^ 1u, kWhereEmpty)) { ok = false; break; }
                     const uint32_t sa = s_stage + s * C::STAGE_BYTES;
-                    mbar_arrive_expect_tx(full(s), C::STAGE_BYTES);
-                    tma_load_2d(sa, &tmW, kb * kBlockK, nt * 128, full(s));
-                    tma_load_2d(sa + kABytes, &tmX, kb * kBlockK, mt * BN, full(s));
+                    const uint32_t sb = sa + KBS * kABytes;
+                    mbar_arrive_expect_tx(full(s), nsub * (kABytes + C::B_BYTES));
+                    for (int j = 0; j < nsub; ++j) {
+                        tma_load_2d(sa + j * kABytes, &tmW, (kb + j) * kBlockK, nt * 128, full(s));
+                        tma_load_2d(sb + j * C::B_BYTES, &tmX, (kb + j) * kBlockK, mt * BN, full(s));
+                    }
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
             }
@@ -1012,7 +1019,9 @@ kx_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
         if (lane == 0) {
             constexpr uint32_t idesc = idesc_bf16_f32(128, BN);
             uint32_t s = 0, ph = 0, ucount = 0;
+            const uint32_t a_lo0 = smem_desc_lo(s_stage);
             bool ok = true;
+            bool have = false;   // the current stage was already seen full by the previous stage's early test
             for (int u = blockIdx.x; u < p.num_units && ok; u += gridDim.x, ++ucount) {
                 int nt, mt, sp, kb0, kb1;
                 unit_coords(u, nt, mt, sp, kb0, kb1);
@@ -1020,19 +1029,23 @@ kx_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
                 if (!wt.wait(acc_empty(b), aph ^ 1u, kWhereAccEmpty)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d = tmem_base + b * BN;
-                for (int kb = kb0; kb < kb1; ++kb) {
-                    if (!wt.wait(full(s), ph, kWhereFull)) { ok = false; break; }
+                for (int kb = kb0; kb < kb1; kb += KBS) {
+                    if (!have && !wt.wait(full(s), ph, kWhereFull)) { ok = false; break; }
                     tc_fence_after();
                     if (ucount == 0 && kb == kb0) KX_TRACE_POINT(p, blockIdx.x, 3);
-                    if (ucount == 0 && kb == kb1 - 1) KX_TRACE_POINT(p, blockIdx.x, 4);
-                    const uint32_t sa = s_stage + s * C::STAGE_BYTES;
-                    const uint32_t sb = sa + kABytes;
-#pragma unroll
-                    for (int k = 0; k < 4; ++k)
-                        mma_bf16<1>(d, smem_desc_sw128(sa + k * 32), smem_desc_sw128(sb + k * 32), idesc,
-                                    static_cast<uint32_t>((kb - kb0) | k));
-                    mma_commit<1>(empty(s));
-                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+                    if (ucount == 0 && kb + KBS >= kb1) KX_TRACE_POINT(p, blockIdx.x, 4);
+                    const bool wrap = (s + 1 == STAGES);
+                    const uint32_t next_full = wrap ? full(0) : full(s + 1);
+                    const uint32_t next_ph = wrap ? (ph ^ 1u) : ph;
+                    const uint32_t a_lo = a_lo0 + s * (C::STAGE_BYTES >> 4);
+                    const uint32_t b_lo = a_lo + ((KBS * kABytes) >> 4);
+                    if (KBS == 2 && kb + 1 < kb1)
+                        have = mma_kblock<1, 0, true>(d, a_lo, b_lo, idesc, static_cast<uint32_t>(kb - kb0), next_full, next_ph,
+                                                      empty(s), 0u, a_lo + (kABytes >> 4), b_lo + (C::B_BYTES >> 4)) != 0u;
+                    else
+                        have = mma_kblock<1, 0, false>(d, a_lo, b_lo, idesc, static_cast<uint32_t>(kb - kb0), next_full, next_ph,
+                                                       empty(s), 0u) != 0u;
+                    if (wrap) { s = 0; ph ^= 1u; } else { ++s; }
                 }
                 if (!ok) break;
                 mma_commit<1>(acc_full(b));

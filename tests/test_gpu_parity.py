@@ -33,6 +33,9 @@ SWAP_VARIANTS = [
     dict(path=S, block_n=16, split_k=4, cluster_reduce=1), dict(path=S, block_n=64, split_k=2, cluster_reduce=1),
     dict(path=S, block_n=256, split_k=4, cluster_reduce=1), dict(path=S, block_n=32, split_k=12),
     dict(path=S, block_n=128, split_k=8, cluster_reduce=2),
+    # the variants with one k-block per ring stage (the defaults hold two)
+    dict(path=S, block_n=16, split_k=4, stages=12), dict(path=S, block_n=32, split_k=3, stages=11, cluster_reduce=1),
+    dict(path=S, block_n=64, split_k=2, stages=9), dict(path=S, block_n=128, split_k=5, stages=7), dict(path=S, block_n=256, split_k=1, stages=4),
 ]
 
 
