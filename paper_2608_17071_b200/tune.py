@@ -43,6 +43,8 @@ def candidates(M: int, N: int, K: int, kx):
         bn = 16 if M <= 16 else 32 if M <= 32 else 64 if M <= 64 else 128 if M <= 128 else 256
         for sk in (1, 2, 3, 4, 5, 6, 8):
             out.append(dict(path=S, block_n=bn, split_k=sk))
+        one_kb_swap = {16: 12, 32: 11, 64: 9, 128: 7, 256: 4}
+        out.append(dict(path=S, block_n=bn, stages=one_kb_swap[bn]))
         for sk in (2, 4, 8, 12, 16):
             out.append(dict(path=S, block_n=bn, split_k=sk, cluster_reduce=1))
     if M > 64:
@@ -57,6 +59,15 @@ def candidates(M: int, N: int, K: int, kx):
         for bn in (256, 192, 128):
             for kc in (2, 4):
                 out.append(dict(path=T, block_n=bn, cta_pair=1, k_cluster=kc))
+        # the variants whose ring stages hold two k-blocks (selected by their stage count)
+        two_kb = {(256, 2): 3, (256, 1): 2, (192, 1): 2, (128, 1): 3, (64, 1): 4, (192, 2): 3, (128, 2): 4}
+        one_kb = {(256, 2): 6, (256, 1): 4, (192, 1): 4, (128, 1): 6, (64, 1): 8, (192, 2): 6, (128, 2): 7}
+        for (bn, pair), st in two_kb.items():
+            out.append(dict(path=T, block_n=bn, cta_pair=pair, stages=st))
+            out.append(dict(path=T, block_n=bn, cta_pair=pair, stages=one_kb[(bn, pair)]))
+        for bn in (256, 128):
+            out.append(dict(path=T, block_n=bn, cta_pair=1, k_cluster=2, stages=two_kb[(bn, 1)]))
+            out.append(dict(path=T, block_n=bn, cta_pair=1, k_cluster=2, stages=one_kb[(bn, 1)]))
     return out
 
 
