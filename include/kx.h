@@ -277,6 +277,21 @@ int kx_outproj_residual_strided(const void* X, int64_t ldx, const void* W, int64
                                 void* Y, int64_t ldy, int64_t M, int64_t N, int64_t K, void* stream);
 
 /*
+ * `batch` independent problems of the same shape, dense operands: problem b uses X + b*sx,
+ * W + b*sw, bias + b*sb, R + b*sr, Y + b*sy (strides in elements; sw = 0 shares one weight matrix,
+ * sb = 0 one bias; bias / R may be NULL for all).  Enqueues one kx_outproj_residual per problem on
+ * `stream`, back to back with programmatic dependent launch (each prologue overlaps its
+ * predecessor's tail): a convenience for a handful of large problems (per-expert or per-group
+ * projections), not a grouped kernel for many tiny ones.  Every stride must keep the 16-byte
+ * alignment (multiple of 8); the Y blocks must not overlap each other or an input.  The paper has
+ * no batched case; this is the plain generalisation of Algorithm 3's call.
+ */
+int kx_outproj_residual_batched(const void* X, int64_t sx, const void* W, int64_t sw,
+                                const void* bias_or_null, int64_t sb, const void* R_or_null, int64_t sr,
+                                void* Y, int64_t sy, int64_t M, int64_t N, int64_t K, int64_t batch,
+                                void* stream);
+
+/*
  * ---- INT8 branch of the decoder layer (Appendix A, Algorithm 7: "run fused add+RMSNorm+
  * activation quantization", "quantize gate/up weights in one launch", "compute gate/up GEMM with
  * fused dequantization and SwiGLU epilogue"; the residual add is already part of

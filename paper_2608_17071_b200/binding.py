@@ -23,7 +23,7 @@ KX_PATH_AUTO, KX_PATH_TILE, KX_PATH_SWAP = 0, 1, 2
 
 EXPORTS = (
     "kx_init", "kx_shutdown", "kx_outproj_residual", "kx_gemm_bf16", "kx_outproj_residual_ex",
-    "kx_outproj_residual_host", "kx_outproj_residual_noalloc", "kx_outproj_residual_strided", "kx_rmsnorm", "kx_outproj_residual_rmsnorm",
+    "kx_outproj_residual_host", "kx_outproj_residual_noalloc", "kx_outproj_residual_strided", "kx_outproj_residual_batched", "kx_rmsnorm", "kx_outproj_residual_rmsnorm",
     "kx_gate_up_swiglu",
     "kx_quantize_rows_int8", "kx_quantize_gate_up_int8", "kx_rmsnorm_quantize_int8", "kx_gate_up_swiglu_int8",
     "kx_outproj_residual_int8",
@@ -81,6 +81,7 @@ def load():
     lib.kx_outproj_residual_host.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, vp]
     lib.kx_outproj_residual_noalloc.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, vp]
     lib.kx_outproj_residual_strided.argtypes = [vp, i64, vp, i64, vp, vp, i64, vp, i64, i64, i64, i64, vp]
+    lib.kx_outproj_residual_batched.argtypes = [vp, i64, vp, i64, vp, i64, vp, i64, vp, i64, i64, i64, i64, i64, vp]
     lib.kx_rmsnorm.argtypes = [vp, vp, ctypes.c_float, vp, i64, i64, vp]
     lib.kx_gate_up_swiglu.argtypes = [vp, vp, vp, vp, i64, i64, i64, vp]
     lib.kx_outproj_residual_rmsnorm.argtypes = [vp, vp, vp, vp, vp, ctypes.c_float, vp, vp, i64, i64, i64, vp]
@@ -270,6 +271,26 @@ def kx_outproj_residual_strided(X, W, bias, R, Y, stream=None, check=True) -> in
                                             M, N, K, _stream(stream))
     if check and rc != KX_OK:
         raise KxError(rc, "kx_outproj_residual_strided")
+    return rc
+
+
+def kx_outproj_residual_batched(X, W, bias, R, Y, stream=None, check=True) -> int:
+    """`batch` problems: X [B,M,K], W [B,N,K] or [N,K] (shared), bias [B,N] / [N] / None, R [B,M,N] / None,
+    Y [B,M,N]; contiguous bfloat16 tensors."""
+    B, M, K = X.shape
+    shared_w = W.dim() == 2
+    N = W.shape[-2]
+    _check_bf16("X", X, (B, M, K)); _check_bf16("W", W, (N, K) if shared_w else (B, N, K))
+    _check_bf16("R", R, (B, M, N)); _check_bf16("Y", Y, (B, M, N))
+    sb = 0
+    if bias is not None:
+        shared_b = bias.dim() == 1
+        _check_bf16("bias", bias, (N,) if shared_b else (B, N))
+        sb = 0 if shared_b else N
+    rc = load().kx_outproj_residual_batched(_addr(X), M * K, _addr(W), 0 if shared_w else N * K, _addr(bias), sb,
+                                            _addr(R), M * N, _addr(Y), M * N, M, N, K, B, _stream(stream))
+    if check and rc != KX_OK:
+        raise KxError(rc, "kx_outproj_residual_batched")
     return rc
 
 

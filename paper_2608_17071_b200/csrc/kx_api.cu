@@ -846,6 +846,37 @@ int kx_outproj_residual_strided(const void* X, int64_t ldx, const void* W, int64
     return run(X, W, bias, R, Y, M, N, K, stream, nullptr, false, &lds);
 }
 
+int kx_outproj_residual_batched(const void* X, int64_t sx, const void* W, int64_t sw, const void* bias, int64_t sb,
+                                const void* R, int64_t sr, void* Y, int64_t sy, int64_t M, int64_t N, int64_t K,
+                                int64_t batch, void* stream) {
+    if (batch < 0 || M < 0 || N < 0 || K < 0) return KX_ERR_SHAPE;
+    if (batch == 0 || M == 0 || N == 0) return KX_OK;
+    if (batch > (1 << 20)) return KX_ERR_LIMIT;
+    if ((sx % 8) || (sw % 8) || (sb % 8) || (sr % 8) || (sy % 8)) return KX_ERR_ALIGN;
+    if (sx < 0 || sw < 0 || sb < 0 || sr < 0 || sy < 0) return KX_ERR_SHAPE;
+    // the output blocks must be disjoint, and none may overlap any problem's inputs
+    if (batch > 1 && sy < M * N) return KX_ERR_OVERLAP;
+    const size_t yspan = (static_cast<size_t>(batch - 1) * sy + static_cast<size_t>(M) * N) * 2;
+    const size_t xspan = (static_cast<size_t>(batch - 1) * sx + static_cast<size_t>(M) * K) * 2;
+    const size_t wspan = (static_cast<size_t>(batch - 1) * sw + static_cast<size_t>(N) * K) * 2;
+    const size_t bspan = (static_cast<size_t>(batch - 1) * sb + static_cast<size_t>(N)) * 2;
+    if (overlaps(Y, yspan, X, xspan) || overlaps(Y, yspan, W, wspan) || overlaps(Y, yspan, bias, bspan)) return KX_ERR_OVERLAP;
+    if (R && !(R == Y && sr == sy) &&
+        overlaps(Y, yspan, R, (static_cast<size_t>(batch - 1) * sr + static_cast<size_t>(M) * N) * 2))
+        return KX_ERR_OVERLAP;
+    const uint16_t* x = static_cast<const uint16_t*>(X);
+    const uint16_t* w = static_cast<const uint16_t*>(W);
+    const uint16_t* bb = static_cast<const uint16_t*>(bias);
+    const uint16_t* r = static_cast<const uint16_t*>(R);
+    uint16_t* y = static_cast<uint16_t*>(Y);
+    for (int64_t b = 0; b < batch; ++b) {
+        const int rc = run(x ? x + b * sx : nullptr, w ? w + b * sw : nullptr, bb ? bb + b * sb : nullptr,
+                           r ? r + b * sr : nullptr, y + b * sy, M, N, K, stream, nullptr, false);
+        if (rc != KX_OK) return rc;
+    }
+    return KX_OK;
+}
+
 int kx_plan_query(int64_t M, int64_t N, int64_t K, int has_bias, int has_residual,
                   const kx_plan_override* ov, kx_plan_info* out) {
     (void)has_bias;

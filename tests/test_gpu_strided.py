@@ -90,3 +90,34 @@ def test_strided_argument_checks():
     torch.cuda.synchronize()
     assert rc == kx.KX_OK
     assert np.array_equal(Yw.view(torch.int16).cpu().numpy().view(np.uint16)[:, :16], R)
+
+
+@pytest.mark.parametrize("B,M,N,K,shared", [(3, 200, 520, 264, True), (4, 37, 1024, 1024, False), (2, 1000, 776, 1096, False)])
+def test_batched_equals_a_loop_of_single_calls(B, M, N, K, shared):
+    """The batched entry point is a loop of ordinary calls: the same bits as calling them one by one,
+    with shared or per-problem weights and bias, in place as well."""
+    ds = [inputs.make_inputs(inputs.Workload("t", M, N, K, 930 + b, True, True), stress=True) for b in range(B)]
+    X = torch.stack([kt.to_dev(d["X"]) for d in ds])
+    R = torch.stack([kt.to_dev(d["R"]) for d in ds])
+    W = kt.to_dev(ds[0]["W"]) if shared else torch.stack([kt.to_dev(d["W"]) for d in ds])
+    bias = kt.to_dev(ds[0]["bias"]) if shared else torch.stack([kt.to_dev(d["bias"]) for d in ds])
+    Y = torch.full((B, M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+    kx.kx_outproj_residual_batched(X, W, bias, R, Y)
+    assert kx.kx_last_device_status()[0] == kx.KX_OK
+    for b in range(B):
+        Yb = kt.nan_filled(M, N)
+        kx.kx_outproj_residual(X[b], W if shared else W[b], bias if shared else bias[b], R[b], Yb)
+        assert np.array_equal(kt.from_dev(Y[b].contiguous()), kt.from_dev(Yb))
+    d = ds[B - 1]
+    ok, msg = kt.gate_a(kt.from_dev(Y[B - 1].contiguous()), oracle.outproj(d["X"], ds[0]["W"] if shared else d["W"],
+                                                                            ds[0]["bias"] if shared else d["bias"], d["R"]))
+    assert ok, msg
+    want = kt.from_dev(Y.reshape(B * M, N))
+    Rc = R.clone()
+    kx.kx_outproj_residual_batched(X, W, bias, Rc, Rc)                      # in place
+    assert np.array_equal(kt.from_dev(Rc.reshape(B * M, N)), want)
+    lib = kx.load()
+    A = 0x100000
+    assert lib.kx_outproj_residual_batched(A, 64 * 16, 2 * A, 0, None, 0, None, 0, 4 * A, 16 * 8, 16, 64, 64, 2, None) == kx.KX_ERR_OVERLAP
+    assert lib.kx_outproj_residual_batched(A, 64 * 16 + 4, 2 * A, 0, None, 0, None, 0, 4 * A, 16 * 64, 16, 64, 64, 2, None) == kx.KX_ERR_ALIGN
+    assert lib.kx_outproj_residual_batched(A, 0, 2 * A, 0, None, 0, None, 0, 4 * A, 0, 16, 64, 64, 0, None) == kx.KX_OK
