@@ -266,11 +266,14 @@ int kx_gate_up_swiglu(const void* X, const void* Wg, const void* Wu, void* Z,
  * prints the dense case only; the pitches map directly onto the tensor-map row strides, so the
  * kernels and plans are the dense ones.
  *   ldx, ldw >= K; ldy >= N; ldr >= N (ignored when R is NULL); every pitch % 8 == 0 (rows stay
- *   16-byte aligned); base pointers 16-byte aligned; N % 8 == 0.  K may be ANY length here (the
- *   tail of the last k-block reads as zeros), which also covers reductions that are not a
- *   multiple of 8 once the rows are padded to one.
+ *   16-byte aligned); base pointers 16-byte aligned.  K and N may be ANY length here (the tail of
+ *   the last k-block reads as zeros, the last output columns are clipped), which covers shapes
+ *   that are not multiples of 8 once the rows are padded to one.  A ragged N (N % 8 != 0) always
+ *   runs the large-M tile kernel, also for small M.
  *   R may equal Y only with ldr == ldy; any other overlap between the spans of Y and an input is
- *   KX_ERR_OVERLAP.  Elements between N and ldy of a Y row are never written.
+ *   KX_ERR_OVERLAP.  Elements between N and ldy of a Y row are never written when N % 8 == 0;
+ *   otherwise the padding up to the next multiple of 8 (the rest of the last 16-byte unit) is
+ *   overwritten, nothing beyond it.
  */
 int kx_outproj_residual_strided(const void* X, int64_t ldx, const void* W, int64_t ldw,
                                 const void* bias_or_null, const void* R_or_null, int64_t ldr,

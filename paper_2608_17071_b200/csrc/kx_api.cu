@@ -585,7 +585,7 @@ int validate(const void* X, const void* W, const void* bias, const void* R, cons
         if (lds->ldx > (1ll << 36) || lds->ldw > (1ll << 36) || lds->ldy > (1ll << 36) || lds->ldr > (1ll << 36))
             return KX_ERR_SHAPE;
         if (M == 0 || N == 0) return KX_OK;
-        if ((N % 8) != 0) return KX_ERR_SHAPE;          // K may be any length when the pitch is given
+        // K and N may be any length when the pitches are given (rows stay 16-byte aligned through them)
         if (!Y) return KX_ERR_NULL;
         if (K > 0 && (!X || !W)) return KX_ERR_NULL;
         if (need_r && !R) return KX_ERR_NULL;
@@ -642,6 +642,16 @@ int run(const void* X, const void* W, const void* bias, const void* R, void* Y, 
     }
 
     Plan pl;
+    kx_plan_override ragged;
+    if ((N % 8) != 0) {
+        // only reachable with pitched operands: the small-M kernel's epilogue works in 8-byte column
+        // groups, so a ragged N always takes the tile kernel (TMA clips the last columns)
+        if (ov && ov->path == KX_PATH_SWAP) return KX_ERR_PLAN;
+        std::memset(&ragged, 0, sizeof ragged);
+        if (ov) ragged = *ov;
+        ragged.path = KX_PATH_TILE;
+        ov = &ragged;
+    }
     rc = make_plan(M, N, K, ov, ctx->sm_count, &pl);
     if (rc != KX_OK) return rc;
     const unsigned long long spin_ns =

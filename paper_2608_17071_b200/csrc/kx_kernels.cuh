@@ -802,6 +802,11 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                                     v[2] += bf16_lo(bb.y); v[3] += bf16_hi(bb.y);
                                     v[4] += bf16_lo(bb.z); v[5] += bf16_hi(bb.z);
                                     v[6] += bf16_lo(bb.w); v[7] += bf16_hi(bb.w);
+                                } else if (n < p.N) {
+                                    // ragged last group (N not a multiple of 8, pitched output): one by one
+#pragma unroll
+                                    for (int i = 0; i < 8; ++i)
+                                        if (n + i < p.N) v[i] += __uint_as_float(static_cast<uint32_t>(__ldg(bias + n + i)) << 16);
                                 }
                             }
                             if (has_r) {
