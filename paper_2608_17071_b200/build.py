@@ -17,7 +17,7 @@ DEPS = ["kx_api.cu", "kx_kernels.cuh", "kx_ptx.cuh", "kx_plan_table.inc", os.pat
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-    "-shared", "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "-split-compile", "0",
+    "-shared", "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden",
 ]
 
 
