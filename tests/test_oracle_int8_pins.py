@@ -197,3 +197,36 @@ def test_quantise_then_project_tracks_the_bf16_projection():
     assert np.abs(y8 - y).max() > 0           # it is a different computation
     rms = np.sqrt(np.mean((y8 - y) ** 2)) / np.sqrt(np.mean(y ** 2))
     assert rms < 0.02
+
+
+def test_hand_computed_code_book_fixture():
+    """tests/golden/quantize_rows_8bit.txt: rows whose scale is a power of two, codes worked out by hand
+    (ties to even for INT8; E4M3 bit patterns from the format definition)."""
+    import os
+    path = os.path.join(os.path.dirname(__file__), "golden", "quantize_rows_8bit.txt")
+    fmt, scale, z = None, None, None
+    checked = 0
+    for line in open(path):
+        line = line.split("#")[0].strip()
+        if not line:
+            continue
+        tok = line.split()
+        if tok[0] in ("int8", "fp8"):
+            fmt = tok[0]
+        elif tok[0] == "scale":
+            scale = float(tok[1])
+        elif tok[0] == "z":
+            z = np.array([float(t) for t in tok[1:]])
+        elif tok[0] == "q":
+            want = np.array([int(t, 0) for t in tok[1:]])
+            Z = bits(z.reshape(1, -1))
+            assert np.array_equal(inputs.bf16_bits_to_f32(Z)[0].astype(np.float64), z)      # fixture is BF16-exact
+            if fmt == "int8":
+                Q, S = oracle.quantize_rows(Z)
+                assert np.array_equal(Q[0].astype(np.int64), want), (Q[0], want)
+            else:
+                Q, S = oracle.quantize_rows_fp8(Z)
+                assert np.array_equal(Q[0].astype(np.int64), want), ([hex(v) for v in Q[0]], want)
+            assert S[0] == np.float32(scale)
+            checked += 1
+    assert checked == 3
