@@ -488,3 +488,85 @@ int kx_oracle_outproj_fp8_rows(const uint8_t* Xq, const float* sx, const uint8_t
     }
     return 0;
 }
+
+/*
+ * Block-scaled FP8 ("MXFP8": E4M3 elements, one power-of-two scale per 32 consecutive elements
+ * of a row, stored as an E8M0 byte e meaning 2^(e-127); 0xFF is NaN), the block-scaled member of
+ * the paper's precision axis (Section 3.2; Section 4.3 names the block-scaled tensor-core kinds).
+ * The paper prints no conversion, so this follows the open Microscaling-formats definition:
+ *   shared exponent  se = floor(log2(max|v|)) - 8        (8 = exponent of E4M3's largest binade)
+ *   scale byte       e  = clamp(se + 127, 0, 254)        (an all-zero block takes e = 127)
+ *   element          q  = e4m3(v / 2^(e-127))            (nearest, ties to even, saturating)
+ * The quotient is exact (a power-of-two scaling), so the only rounding is E4M3's.
+ */
+static double e8m0_decode(uint8_t e) {
+    return e == 0xFF ? NAN : ldexp(1.0, (int)e - 127);
+}
+
+int kx_oracle_e8m0_decode(const uint8_t* in, double* out, int64_t n) {
+    if (n < 0 || (n > 0 && (!in || !out))) return -1;
+    for (int64_t i = 0; i < n; ++i) out[i] = e8m0_decode(in[i]);
+    return 0;
+}
+
+/* Z [rows, cols] BF16 -> Q [rows, cols] E4M3 codes, E [rows, ceil(cols/32)] E8M0 bytes (row-major). */
+int kx_oracle_quantize_rows_mx(const uint16_t* Z, int64_t rows, int64_t cols, uint8_t* Q, uint8_t* E) {
+    if (rows < 0 || cols < 0 || (rows > 0 && cols > 0 && (!Z || !Q || !E))) return -1;
+    const int64_t nb = (cols + 31) / 32;
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < rows; ++r) {
+        for (int64_t j = 0; j < nb; ++j) {
+            const int64_t k0 = j * 32, k1 = (k0 + 32 < cols) ? k0 + 32 : cols;
+            double a = 0.0;
+            for (int64_t k = k0; k < k1; ++k) {
+                const double v = fabs(bf16_widen(Z[r * cols + k]));
+                if (v > a) a = v;                       /* NaN never wins the comparison */
+            }
+            int e = 127;
+            if (a > 0.0) {
+                int ex;
+                if (isinf(a)) ex = 129;                 /* treated as the binade above the largest finite one */
+                else (void)frexp(a, &ex);               /* a = f * 2^ex, f in [0.5, 1): floor(log2 a) = ex - 1 */
+                e = (ex - 1) - 8 + 127;
+                if (e < 0) e = 0;
+                if (e > 254) e = 254;
+            }
+            E[r * nb + j] = (uint8_t)e;
+            for (int64_t k = k0; k < k1; ++k) {
+                const double t = ldexp(bf16_widen(Z[r * cols + k]), 127 - e);   /* exact */
+                Q[r * cols + k] = e4m3_encode((float)t);
+            }
+        }
+    }
+    return 0;
+}
+
+/* y = sum over 32-element blocks j of 2^(ex[m,j]-127) 2^(ew[n,j]-127) (xq . wq over the block)
+ *     + bias + R; double, unrounded. */
+int kx_oracle_outproj_mx_rows(const uint8_t* Xq, const uint8_t* ex, const uint8_t* Wq, const uint8_t* ew,
+                              const uint16_t* bias, const uint16_t* R, const int64_t* rows, int64_t nrows,
+                              double* out, int64_t M, int64_t N, int64_t K) {
+    if (M < 0 || N < 0 || K < 0 || nrows < 0 || !out) return -1;
+    if (K > 0 && (!Xq || !Wq || !ex || !ew)) return -1;
+    for (int64_t r = 0; rows && r < nrows; ++r)
+        if (rows[r] < 0 || rows[r] >= M) return -1;
+    if (!rows && nrows > M) return -1;
+    const int64_t nb = (K + 31) / 32;
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int64_t r = 0; r < nrows; ++r) {
+        for (int64_t n = 0; n < N; ++n) {
+            const int64_t m = rows ? rows[r] : r;
+            double y = 0.0;
+            for (int64_t j = 0; j < nb; ++j) {
+                const int64_t k1 = (j * 32 + 32 < K) ? j * 32 + 32 : K;
+                double acc = 0.0;
+                for (int64_t k = j * 32; k < k1; ++k) acc += e4m3_decode(Xq[m * K + k]) * e4m3_decode(Wq[n * K + k]);
+                y += acc * e8m0_decode(ex[m * nb + j]) * e8m0_decode(ew[n * nb + j]);
+            }
+            if (bias) y += bf16_widen(bias[n]);
+            if (R) y += bf16_widen(R[m * N + n]);
+            out[r * N + n] = y;
+        }
+    }
+    return 0;
+}

@@ -45,6 +45,9 @@ def _load():
         lib.kx_oracle_quantize_rows_fp8.argtypes = [p, i64, i64, p, p]
         lib.kx_oracle_swiglu_fp8_rows.argtypes = [p, p, p, p, p, p, p, i64, p, i64, i64, i64]
         lib.kx_oracle_outproj_fp8_rows.argtypes = [p, p, p, p, p, p, p, i64, p, i64, i64, i64]
+        lib.kx_oracle_e8m0_decode.argtypes = [p, p, i64]
+        lib.kx_oracle_quantize_rows_mx.argtypes = [p, i64, i64, p, p]
+        lib.kx_oracle_outproj_mx_rows.argtypes = [p, p, p, p, p, p, p, i64, p, i64, i64, i64]
         lib.kx_oracle_max_threads.argtypes = []
         lib.kx_oracle_max_threads.restype = ctypes.c_int
         _lib = lib
@@ -314,4 +317,48 @@ def outproj_fp8(Xq, sx, Wq, sw, bias=None, R=None, rows=None):
                                             _ptr(rows_arr), nrows, _ptr(out), M, N, K)
     if rc != 0:
         raise RuntimeError(f"kx_oracle_outproj_fp8_rows failed ({rc})")
+    return out
+
+
+def e8m0_decode(e) -> np.ndarray:
+    """E8M0 scale bytes -> float64: 2^(e - 127), 0xFF = NaN."""
+    e = np.ascontiguousarray(e, dtype=np.uint8)
+    out = np.empty(e.shape, dtype=np.float64)
+    _load().kx_oracle_e8m0_decode(_ptr(e), _ptr(out), e.size)
+    return out
+
+
+def quantize_rows_mx(Z):
+    """Block-scaled FP8 code book of BF16 rows (Section 3.2, precision axis): per 32 consecutive elements
+    one E8M0 scale byte e = clamp(floor(log2 max|z|) - 8 + 127, 0, 254) (zero block: 127) and
+    q = e4m3(z / 2^(e-127)).  Z uint16 BF16 bits [rows, cols] -> (Q uint8 [rows, cols],
+    E uint8 [rows, ceil(cols / 32)])."""
+    rows, cols = Z.shape
+    Z = _bits(Z, (rows, cols), "Z")
+    Q = np.empty((rows, cols), dtype=np.uint8)
+    E = np.empty((rows, (cols + 31) // 32), dtype=np.uint8)
+    rc = _load().kx_oracle_quantize_rows_mx(_ptr(Z), rows, cols, _ptr(Q), _ptr(E))
+    if rc != 0:
+        raise RuntimeError(f"kx_oracle_quantize_rows_mx failed ({rc})")
+    return Q, E
+
+
+def outproj_mx(Xq, ex, Wq, ew, bias=None, R=None, rows=None):
+    """y = sum_j 2^(ex[m,j]-127) 2^(ew[n,j]-127) (Xq[m, 32j:32j+32] . Wq[n, 32j:32j+32]) + bias + R on E4M3
+    codes with E8M0 block scales; float64, unrounded."""
+    M, K = Xq.shape
+    N = Wq.shape[0]
+    nb = (K + 31) // 32
+    Xq = _typed(Xq, np.uint8, (M, K), "Xq")
+    Wq = _typed(Wq, np.uint8, (N, K), "Wq")
+    ex = _typed(ex, np.uint8, (M, nb), "ex")
+    ew = _typed(ew, np.uint8, (N, nb), "ew")
+    bias = _bits(bias, (N,), "bias")
+    R = _bits(R, (M, N), "R")
+    rows_arr, nrows = _rows_arg(rows, M)
+    out = np.empty((nrows, N), dtype=np.float64)
+    rc = _load().kx_oracle_outproj_mx_rows(_ptr(Xq), _ptr(ex), _ptr(Wq), _ptr(ew), _ptr(bias), _ptr(R),
+                                           _ptr(rows_arr), nrows, _ptr(out), M, N, K)
+    if rc != 0:
+        raise RuntimeError(f"kx_oracle_outproj_mx_rows failed ({rc})")
     return out
