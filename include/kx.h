@@ -369,6 +369,40 @@ int kx_outproj_residual_fp8(const void* Xq, const float* sx, const void* Wq, con
                             const void* bias_or_null, const void* R_or_null, void* Y,
                             int64_t M, int64_t N, int64_t K, void* stream);
 
+/*
+ * Block-scaled FP8 branch (the block-scaled member of the precision axis of Section 3.2; the
+ * tensor-core kind is the block-scaled tcgen05 family that Section 4.3 names).  Elements are FP8
+ * E4M3 codes; every 32 consecutive elements of a row share one power-of-two scale stored as an
+ * E8M0 byte e (value 2^(e-127); 0xFF is NaN and must not appear).
+ *
+ * Code book (kx_quantize_rows_mxfp8), per block of 32 BF16 values z of a row:
+ *     e = clamp(floor(log2 max|z|) - 8 + 127, 0, 254)   (an all-zero block takes e = 127)
+ *     q = e4m3(z / 2^(e-127))                           (exact quotient; nearest, ties to even, saturating at +-448)
+ * A [rows, cols] BF16 row-major, cols % 32 == 0; Q [rows, cols] bytes; all device pointers, 16-byte
+ * aligned, written by the call (Q, SF) or only read (A); no overlap.
+ *
+ * Scale layout (SF of the code book, SFX / SFW of the projection): chunks of 512 bytes, one per
+ * (128 rows, 128 elements of K), ordered [ceil(rows / 128)][ceil(cols / 128)]; inside a chunk the
+ * scale of row r and 32-element block j sits at byte (r % 32) * 16 + (r % 128) / 32 * 4 + j % 4.
+ * This is the order in which the tensor core's scale copy (32 rows x 16 bytes, repeated for each
+ * 32-lane quarter of tensor memory) wants them, so a chunk goes from global to shared to tensor
+ * memory without being touched.  kx_mx_scale_bytes gives the size of the whole array (< 0 on
+ * negative extents).  Entries of rows >= rows or blocks >= cols / 32 are padding: the code book
+ * writes 127 there; arrays built elsewhere must hold any byte other than 0xFF.
+ *
+ * kx_outproj_residual_mxfp8:
+ *     Y[m,n] = bf16( sum_j 2^(ex[m,j]-127) 2^(ew[n,j]-127) sum_{k in block j} xq[m,k] wq[n,k] + bias[n] + R[m,n] )
+ * Xq [M,K], Wq [N,K] E4M3 bytes, K contiguous; K % 32 == 0, N % 8 == 0; bias / R / Y as in
+ * kx_outproj_residual (R may be Y).  One CTA per 128 x 128 or 128 x 192 tile, FP32 accumulation in
+ * tensor memory, tolerance as for the BF16 path against the exact value of the formula.
+ * Errors: KX_ERR_SHAPE, KX_ERR_NULL, KX_ERR_ALIGN, KX_ERR_OVERLAP as for the calls above.
+ */
+int64_t kx_mx_scale_bytes(int64_t rows, int64_t cols);
+int kx_quantize_rows_mxfp8(const void* A, void* Q, void* SF, int64_t rows, int64_t cols, void* stream);
+int kx_outproj_residual_mxfp8(const void* Xq, const void* SFX, const void* Wq, const void* SFW,
+                              const void* bias_or_null, const void* R_or_null, void* Y,
+                              int64_t M, int64_t N, int64_t K, void* stream);
+
 /* Fills `out` with the plan the library would use for this shape on the current
  * device (has_residual / has_bias as 0 or 1).  No work is enqueued. */
 int kx_plan_query(int64_t M, int64_t N, int64_t K, int has_bias, int has_residual,

@@ -29,6 +29,7 @@ EXPORTS = (
     "kx_outproj_residual_int8",
     "kx_quantize_rows_fp8", "kx_quantize_gate_up_fp8", "kx_rmsnorm_quantize_fp8", "kx_gate_up_swiglu_fp8",
     "kx_outproj_residual_fp8",
+    "kx_mx_scale_bytes", "kx_quantize_rows_mxfp8", "kx_outproj_residual_mxfp8",
     "kx_plan_query", "kx_last_device_status", "kx_status_string",
     "kx_version",
 )
@@ -96,13 +97,18 @@ def load():
         getattr(lib, f"kx_rmsnorm_quantize_{sfx}").argtypes = lib.kx_rmsnorm_quantize_int8.argtypes
         getattr(lib, f"kx_gate_up_swiglu_{sfx}").argtypes = lib.kx_gate_up_swiglu_int8.argtypes
         getattr(lib, f"kx_outproj_residual_{sfx}").argtypes = lib.kx_outproj_residual_int8.argtypes
+    lib.kx_mx_scale_bytes.argtypes = [i64, i64]
+    lib.kx_quantize_rows_mxfp8.argtypes = [vp, vp, vp, i64, i64, vp]
+    lib.kx_outproj_residual_mxfp8.argtypes = [vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, vp]
     lib.kx_plan_query.argtypes = [i64, i64, i64, ci, ci, ctypes.POINTER(PlanOverride), ctypes.POINTER(PlanInfo)]
     lib.kx_last_device_status.argtypes = [vp, ctypes.POINTER(ci), ctypes.POINTER(ci)]
     lib.kx_status_string.argtypes = [ci]
     lib.kx_status_string.restype = ctypes.c_char_p
     lib.kx_version.argtypes = []
     for name in EXPORTS:
-        if name != "kx_status_string":
+        if name == "kx_mx_scale_bytes":
+            getattr(lib, name).restype = i64
+        elif name != "kx_status_string":
             getattr(lib, name).restype = ci
     _lib = lib
     return lib
@@ -481,3 +487,36 @@ def kx_last_device_status(stream=None):
     if rc != KX_OK:
         raise KxError(rc, "kx_last_device_status")
     return code.value, detail.value
+
+
+def kx_mx_scale_bytes(rows: int, cols: int) -> int:
+    """Bytes of the chunked E8M0 scale array of a [rows, cols] block-scaled matrix."""
+    return int(load().kx_mx_scale_bytes(int(rows), int(cols)))
+
+
+def kx_quantize_rows_mxfp8(A, Q, SF, stream=None, check=True) -> int:
+    """Q (float8_e4m3fn [rows, cols]), SF (uint8, kx_mx_scale_bytes(rows, cols) bytes, chunked layout) =
+    block-scaled FP8 code book of the BF16 matrix A (one E8M0 scale per 32 elements of a row)."""
+    import torch
+    rows, cols = A.shape
+    _check_bf16("A", A, (rows, cols)); _check("Q", Q, (rows, cols), torch.float8_e4m3fn)
+    _check("SF", SF, (kx_mx_scale_bytes(rows, cols),), torch.uint8)
+    rc = load().kx_quantize_rows_mxfp8(_addr(A), _addr(Q), _addr(SF), rows, cols, _stream(stream))
+    if check and rc != KX_OK:
+        raise KxError(rc, "kx_quantize_rows_mxfp8")
+    return rc
+
+
+def kx_outproj_residual_mxfp8(Xq, SFX, Wq, SFW, bias, R, Y, stream=None, check=True) -> int:
+    """Y = block-scaled (Xq, SFX) (Wq, SFW)^T + bias + R; bias / R may be None; R may be Y."""
+    import torch
+    M, K = Xq.shape
+    N = Wq.shape[0]
+    _check("Xq", Xq, (M, K), torch.float8_e4m3fn); _check("Wq", Wq, (N, K), torch.float8_e4m3fn)
+    _check("SFX", SFX, (kx_mx_scale_bytes(M, K),), torch.uint8); _check("SFW", SFW, (kx_mx_scale_bytes(N, K),), torch.uint8)
+    _check_bf16("bias", bias, (N,)); _check_bf16("R", R, (M, N)); _check_bf16("Y", Y, (M, N))
+    rc = load().kx_outproj_residual_mxfp8(_addr(Xq), _addr(SFX), _addr(Wq), _addr(SFW), _addr(bias), _addr(R), _addr(Y),
+                                          M, N, K, _stream(stream))
+    if check and rc != KX_OK:
+        raise KxError(rc, "kx_outproj_residual_mxfp8")
+    return rc

@@ -108,6 +108,23 @@ const SwapVariant kSwapVariants[] = {
     KX_SWAP(16, 12, 1), KX_SWAP(32, 11, 1), KX_SWAP(64, 9, 1), KX_SWAP(128, 7, 1), KX_SWAP(256, 4, 1),
 };
 
+// Block-scaled FP8 tile kernels (one CTA per tile; two accumulators and the scale columns share TMEM)
+struct MxVariant {
+    int bn, stages, nb, kbs, smem;
+    const void* fn;
+};
+#define KX_MX(BN, ST, NB, KBS)                                                                \
+    MxVariant {                                                                               \
+        BN, ST, NB, KBS, TileCfg<BN, 1, ST, NB, KBS, 1>::SMEM_BYTES,                          \
+            reinterpret_cast<const void*>(&kx_tile_kernel<BN, 1, ST, NB, 3, KBS>)             \
+    }
+const MxVariant kMxVariants[] = {KX_MX(128, 5, 2, 1), KX_MX(192, 4, 3, 1)};
+const MxVariant* find_mx(int bn) {
+    for (const auto& v : kMxVariants)
+        if (v.bn == bn) return &v;
+    return nullptr;
+}
+
 // first variant in table order that matches; stages == 0 matches any depth
 const TileVariant* find_tile(int bn, int ctas, int stages) {
     for (const auto& v : kTileVariants)
@@ -166,6 +183,8 @@ int ensure_device(int dev, DeviceCtx** out) {
                  cudaFuncSetAttribute(v.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, v.smem) == cudaSuccess &&
                  cudaFuncSetAttribute(v.fn_s8, cudaFuncAttributeMaxDynamicSharedMemorySize, v.smem) == cudaSuccess &&
                  cudaFuncSetAttribute(v.fn_f8, cudaFuncAttributeMaxDynamicSharedMemorySize, v.smem) == cudaSuccess;
+        for (const auto& v : kMxVariants)
+            ok = ok && cudaFuncSetAttribute(v.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, v.smem) == cudaSuccess;
         for (const auto& v : kSwapVariants)
             ok = ok &&
                  cudaFuncSetAttribute(v.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, v.smem) == cudaSuccess &&
@@ -1539,6 +1558,146 @@ int kx_outproj_residual_int8(const void* Xq, const float* sx, const void* Wq, co
 int kx_outproj_residual_fp8(const void* Xq, const float* sx, const void* Wq, const float* sw, const void* bias,
                             const void* R, void* Y, int64_t M, int64_t N, int64_t K, void* stream) {
     return outproj_residual_q8(2, Xq, sx, Wq, sw, bias, R, Y, M, N, K, stream);
+}
+
+// ---------------------------------------------------------------- block-scaled FP8 branch
+namespace {
+long long mx_chunks(long long rows) { return (rows + 127) / 128; }
+}  // namespace
+
+int64_t kx_mx_scale_bytes(int64_t rows, int64_t cols) {
+    if (rows < 0 || cols < 0) return -1;
+    return mx_chunks(rows) * mx_chunks(cols) * 512;
+}
+
+int kx_quantize_rows_mxfp8(const void* A, void* Q, void* SF, int64_t rows, int64_t cols, void* stream) {
+    if (rows < 0 || cols < 0 || rows > 0x7FFFFFFFll / 2 || cols > 0x7FFFFFFFll / 2) return KX_ERR_SHAPE;
+    if ((cols % 32) != 0) return KX_ERR_SHAPE;
+    if (rows == 0 || cols == 0) return KX_OK;
+    if (!A || !Q || !SF) return KX_ERR_NULL;
+    if (!aligned16(A) || !aligned16(Q) || !aligned16(SF)) return KX_ERR_ALIGN;
+    const size_t ab = static_cast<size_t>(rows) * cols * 2, qb = static_cast<size_t>(rows) * cols,
+                 sb = static_cast<size_t>(kx_mx_scale_bytes(rows, cols));
+    if (overlaps(Q, qb, A, ab) || overlaps(SF, sb, A, ab) || overlaps(SF, sb, Q, qb)) return KX_ERR_OVERLAP;
+    DeviceCtx* ctx = nullptr;
+    int rc = device_ctx(&ctx);
+    if (rc != KX_OK) return rc;
+    MxQuantParams p;
+    std::memset(&p, 0, sizeof p);
+    p.A = static_cast<const uint16_t*>(A);
+    p.Q = static_cast<uint8_t*>(Q);
+    p.SF = static_cast<uint8_t*>(SF);
+    p.rows = rows;
+    p.rows_pad = mx_chunks(rows) * 128;
+    p.cols = static_cast<int>(cols);
+    p.kchunks = static_cast<int>(mx_chunks(cols));
+    const long long total = p.rows_pad * p.kchunks * 16;
+    cudaLaunchConfig_t cfg;
+    std::memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3(static_cast<unsigned>(std::min<long long>((total + 255) / 256, ctx->sm_count * 16ll)), 1, 1);
+    cfg.blockDim = dim3(256, 1, 1);
+    cfg.stream = static_cast<cudaStream_t>(stream);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    void* args[] = {&p};
+    if (cudaLaunchKernelExC(&cfg, reinterpret_cast<const void*>(&kx_mxquant_kernel), args) != cudaSuccess) {
+        cudaGetLastError();
+        return KX_ERR_CUDA;
+    }
+    return KX_OK;
+}
+
+int kx_outproj_residual_mxfp8(const void* Xq, const void* SFX, const void* Wq, const void* SFW, const void* bias,
+                              const void* R, void* Y, int64_t M, int64_t N, int64_t K, void* stream_v) {
+    if (M < 0 || N < 0 || K < 0) return KX_ERR_SHAPE;
+    if (M > 0x7FFFFFFFll / 2 || N > 0x7FFFFFFFll / 4 || K > 0x7FFFFFFFll / 2) return KX_ERR_SHAPE;
+    if (M == 0 || N == 0) return KX_OK;
+    if ((N % 8) != 0 || (K % 32) != 0) return KX_ERR_SHAPE;
+    if (!Y) return KX_ERR_NULL;
+    if (!aligned16(Y) || (bias && !aligned16(bias)) || (R && !aligned16(R))) return KX_ERR_ALIGN;
+    const size_t yb = static_cast<size_t>(M) * N * 2;
+    if (overlaps(Y, yb, bias, static_cast<size_t>(N) * 2)) return KX_ERR_OVERLAP;
+    if (R && R != Y && overlaps(Y, yb, R, yb)) return KX_ERR_OVERLAP;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    DeviceCtx* ctx = nullptr;
+    int rc = device_ctx(&ctx);
+    if (rc != KX_OK) return rc;
+    if (K == 0) {
+        const long long total = M * N;
+        const int blocks = static_cast<int>(std::min<long long>((total + 255) / 256, ctx->sm_count * 8));
+        kx_k0_kernel<<<blocks, 256, 0, stream>>>(static_cast<const uint16_t*>(bias), static_cast<const uint16_t*>(R),
+                                                 static_cast<uint16_t*>(Y), M, N, N, N);
+        return cudaGetLastError() == cudaSuccess ? KX_OK : KX_ERR_CUDA;
+    }
+    if (!Xq || !Wq || !SFX || !SFW) return KX_ERR_NULL;
+    if (!aligned16(Xq) || !aligned16(Wq) || !aligned16(SFX) || !aligned16(SFW)) return KX_ERR_ALIGN;
+    if (overlaps(Y, yb, Xq, static_cast<size_t>(M) * K) || overlaps(Y, yb, Wq, static_cast<size_t>(N) * K) ||
+        overlaps(Y, yb, SFX, static_cast<size_t>(kx_mx_scale_bytes(M, K))) ||
+        overlaps(Y, yb, SFW, static_cast<size_t>(kx_mx_scale_bytes(N, K))))
+        return KX_ERR_OVERLAP;
+    // tile width: 192 when it leaves fewer idle tile slots in the last wave than 128
+    const long long tm = (M + 127) / 128;
+    auto waste = [&](int bn) {
+        const long long tiles = tm * ((N + bn - 1) / bn);
+        const long long waves = (tiles + ctx->sm_count - 1) / ctx->sm_count;
+        return static_cast<double>(waves * ctx->sm_count) * bn;          // column-slots paid for
+    };
+    const int bn = (N > 128 && waste(192) < waste(128)) ? 192 : 128;
+    const MxVariant* v = find_mx(bn);
+    if (!v) return KX_ERR_PLAN;
+    const long long tiles_n = (N + bn - 1) / bn, tiles = tm * tiles_n;
+    if (tiles > 0x7FFFFFFFll / 4) return KX_ERR_SHAPE;
+    CUtensorMap tmA, tmB, tmY, tmR;
+    if ((rc = get_tmap(Xq, M, K, 128, &tmA, 1)) != KX_OK) return rc;
+    if ((rc = get_tmap(Wq, N, K, bn, &tmB, 1)) != KX_OK) return rc;
+    if ((rc = get_tmap(Y, M, N, 32, &tmY)) != KX_OK) return rc;
+    if (R) {
+        if ((rc = get_tmap(R, M, N, 32, &tmR)) != KX_OK) return rc;
+    } else {
+        tmR = tmY;
+    }
+    TileParams p;
+    std::memset(&p, 0, sizeof p);
+    p.M = static_cast<int>(M);
+    p.N = static_cast<int>(N);
+    p.K = static_cast<int>(K);
+    p.tiles_m = static_cast<int>(tm);
+    p.tiles_n = static_cast<int>(tiles_n);
+    p.num_tiles = static_cast<int>(tiles);
+    p.raster_group = 8;
+    p.has_bias = bias ? 1 : 0;
+    p.has_r = R ? 1 : 0;
+    p.kcluster = 1;
+    p.sk_tile0 = p.num_tiles;
+    p.narrow_tile0 = p.num_tiles;
+    p.spin_limit_ns = 2000000000ull;
+    p.status = ctx->status;
+    p.ws = ctx->ws;
+    p.counters = ctx->counters;
+    p.sfa = static_cast<const uint8_t*>(SFX);
+    p.sfb = static_cast<const uint8_t*>(SFW);
+    p.sfb_chunks = static_cast<int>(mx_chunks(N));
+    cudaLaunchConfig_t cfg;
+    std::memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3(static_cast<unsigned>(std::min<long long>(tiles, ctx->sm_count)), 1, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = v->smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const uint16_t* bias_p = static_cast<const uint16_t*>(bias);
+    void* args[] = {&tmA, &tmB, &tmB, &tmY, &tmR, &bias_p, &p};
+    if (cudaLaunchKernelExC(&cfg, v->fn, args) != cudaSuccess) {
+        cudaGetLastError();
+        return KX_ERR_CUDA;
+    }
+    return KX_OK;
 }
 
 // ---------------------------------------------------------------- no-allocation entry

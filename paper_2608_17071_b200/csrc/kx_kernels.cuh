@@ -128,6 +128,9 @@ struct TileParams {
     const float* sa;           // KIND 1 / 2: scale per row of A [M]
     const float* sb;           // KIND 1 / 2: scale per row of B [N] (gate rows in gate/up mode)
     const float* sb2;          // KIND 1 / 2, gate/up mode: scale per up row [N]
+    const uint8_t* sfa;        // KIND 3: E8M0 block scales of A, 512-byte chunks [ceil(M/128)][k-blocks]
+    const uint8_t* sfb;        // KIND 3: E8M0 block scales of B, same layout over N
+    int sfb_chunks;            // KIND 3: ceil(N / 128)
     int swiglu;                   // 1: gate/up mode.  W rows of a tile = BN/2 rows of Wg (tmB) followed by the same
                                   // BN/2 rows of Wu (tmB2); the epilogue writes silu(gate) * up, BN/2 columns per
                                   // tile, N = number of output columns; no bias, no residual
@@ -150,7 +153,10 @@ struct TileParams {
 
 // KBS = k-blocks per ring stage (1 or 2).  With 2, a stage is [A kb][A kb+1][B kb][B kb+1]: one
 // barrier round trip and one commit per eight K steps instead of four.
-template <int BN, int CTAS, int STAGES, int NB, int KBS = 1>
+// MX = 1 (block-scaled operands): every stage also holds, per k-block, one 512-byte scale chunk of
+// the A tile and SFB_CHUNKS of the B tile; 48 TMEM columns after the two accumulators take four
+// rotating sets of scale columns (4 for A, 8 for B).
+template <int BN, int CTAS, int STAGES, int NB, int KBS = 1, int MX = 0>
 struct TileCfg {
     static constexpr int BN_LOAD = BN / CTAS;               // W rows this CTA loads per k-block
     static constexpr int B_BYTES = BN_LOAD * 128;
@@ -159,8 +165,13 @@ struct TileCfg {
     static constexpr int SLAB_BYTES = 32 * 128;             // 32 rows x 64 BF16 per warp per chunk
     static constexpr int EPI_BYTES = 4 * NB * SLAB_BYTES;
     static constexpr int NUM_BARS = 2 * STAGES + 4 + 4 * NB + 1;
-    static constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + EPI_BYTES + 1024;
-    static constexpr int TMEM_COLS = tmem_cols_for(2 * BN);
+    static constexpr int SFB_CHUNKS = (BN > 128) ? 2 : 1;
+    static constexpr int SF_KB_BYTES = MX ? 512 * (1 + SFB_CHUNKS) : 0;     // scale bytes per k-block
+    static constexpr int SF_STAGE = KBS * SF_KB_BYTES;
+    static constexpr int SMEM_BYTES = 1024 + STAGES * (STAGE_BYTES + SF_STAGE) + EPI_BYTES + 1024;
+    static constexpr int TMEM_COLS = tmem_cols_for(2 * BN + (MX ? 48 : 0));
+    static_assert(!MX || (CTAS == 1 && BN <= 192), "block-scaled variants: one CTA per tile, two accumulators + scales in TMEM");
+    static_assert(SMEM_BYTES <= 232448, "shared memory");
     static constexpr int CHUNKS = BN / 64;                  // 64-column epilogue chunks per tile
     static constexpr int PART_FLOATS = 128 * BN;            // one CTA's FP32 partial of one tile
     static_assert(BN % 64 == 0 && BN <= 256, "BN");
@@ -225,20 +236,25 @@ __device__ __forceinline__ uint32_t ld_acquire_gpu_u32(const unsigned int* p) {
 // codes = the same 128 bytes per row), 32-bit integer accumulators.  KIND 2: FP8 E4M3 operands
 // (same byte geometry), FP32 accumulators.  KIND 1 and 2 are dequantised in the epilogue with a
 // per-row scale of A and a per-row scale of B; they run whole tiles only (the stream-K and
-// K-cluster fix-ups add partial accumulators as unscaled FP32).
+// K-cluster fix-ups add partial accumulators as unscaled FP32).  KIND 3: FP8 E4M3 operands with one
+// E8M0 scale per 32 elements of a row (tcgen05 kind::mxf8f6f4.block_scale): the scales travel through
+// the ring beside the operand tiles, are copied to TMEM before the four K steps of their k-block, and
+// the FP32 accumulators need no dequantisation; one CTA per tile, whole full-width tiles only.
 template <int BN, int CTAS, int STAGES, int NB, int KIND = 0, int KBS = 1>
 __global__ void __launch_bounds__(kThreads, 1)
 kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmB2, const __grid_constant__ CUtensorMap tmY,
                const __grid_constant__ CUtensorMap tmR, const uint16_t* __restrict__ bias, const TileParams p) {
-    using C = TileCfg<BN, CTAS, STAGES, NB, KBS>;
+    using C = TileCfg<BN, CTAS, STAGES, NB, KBS, KIND == 3 ? 1 : 0>;
+    constexpr bool kRowScaled = (KIND == 1 || KIND == 2);       // dequantised in the epilogue
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t* const gbase = smem_raw + (base - raw);
     const uint32_t s_stage = base;
     const uint32_t s_epi = base + STAGES * C::STAGE_BYTES;
-    const uint32_t s_bar = s_epi + C::EPI_BYTES;
+    const uint32_t s_sf = s_epi + C::EPI_BYTES;                 // KIND 3: scale chunks, one slot per stage
+    const uint32_t s_bar = s_sf + STAGES * C::SF_STAGE;
     auto full = [&](int s) { return s_bar + 8u * s; };
     auto empty = [&](int s) { return s_bar + 8u * (STAGES + s); };
     auto acc_full = [&](int b) { return s_bar + 8u * (2 * STAGES + b); };
@@ -375,7 +391,22 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     const uint32_t sa = s_stage + s * C::STAGE_BYTES;
                     const uint32_t sb = sa + KBS * kABytes;
                     if constexpr (CTAS == 1) {
-                        mbar_arrive_expect_tx(full(s), nsub * stage_tx);
+                        mbar_arrive_expect_tx(full(s), nsub * (stage_tx + C::SF_KB_BYTES));
+                        if constexpr (KIND == 3) {
+                            // scale chunks of this tile's rows for k-block kb: chunk (row / 128, kb); a B
+                            // chunk past the end of the array (ragged last tile) is replaced by the last one,
+                            // its rows are zero-filled operand rows
+                            const int c0 = col >> 7;
+                            for (int j = 0; j < nsub; ++j) {
+                                const uint32_t dst = s_sf + s * C::SF_STAGE + j * C::SF_KB_BYTES;
+                                bulk_load(dst, p.sfa + (static_cast<size_t>(tm) * nkb + (kb + j)) * 512, 512, full(s));
+                                for (int i = 0; i < C::SFB_CHUNKS; ++i) {
+                                    const int ch = min(c0 + i, p.sfb_chunks - 1);
+                                    bulk_load(dst + 512 * (1 + i), p.sfb + (static_cast<size_t>(ch) * nkb + (kb + j)) * 512,
+                                              512, full(s));
+                                }
+                            }
+                        }
                         for (int j = 0; j < nsub; ++j) {
                             tma_load_2d(sa + j * kABytes, &tmA, (kb + j) * KBLK, a_row, full(s));
                             tma_load_2d(sb + j * C::B_BYTES, mapB, (kb + j) * KBLK, b_row, full(s));
@@ -404,11 +435,13 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (leader && lane == 0) {
             constexpr uint32_t idesc_wide = KIND == 1   ? idesc_s8_s32(128 * CTAS, BN)
                                             : KIND == 2 ? idesc_e4m3_f32(128 * CTAS, BN)
+                                            : KIND == 3 ? idesc_mxf8(128, BN)
                                                         : idesc_bf16_f32(128 * CTAS, BN);
             constexpr uint32_t idesc_narrow = KIND == 1   ? idesc_s8_s32(128 * CTAS, BN / 2)
                                               : KIND == 2 ? idesc_e4m3_f32(128 * CTAS, BN / 2)
                                                           : idesc_bf16_f32(128 * CTAS, BN / 2);
             uint32_t s = 0, ph = 0, scount = 0;
+            [[maybe_unused]] uint32_t mx_set = 0;              // KIND 3: k-blocks issued so far (scale column set)
             // running addresses of the current stage: its `full` barrier, its `empty` barrier as seen from
             // each CTA of the pair, and the low word of its A-tile descriptor
             const uint32_t a_lo0 = smem_desc_lo(s_stage);
@@ -426,6 +459,46 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 tc_fence_after();
                 KX_TRACE_POINT(p, slot, (scount - 1) * 4 + 1);
                 const uint32_t d = tmem_base + b * BN;
+                if constexpr (KIND == 3) {
+                    // block-scaled: per k-block, scale chunks -> TMEM (a rotating set of 12 columns), then
+                    // four K = 32 steps that each name their byte of the scale columns
+                    int tm, col;
+                    bool narrow;
+                    decode_tile(tile, tm, col, narrow);
+                    const uint32_t b_off = static_cast<uint32_t>(col & 127) >> 5;   // first B row's 32-row group in its chunk
+                    for (int kb = kb0; kb < kb1; kb += KBS) {
+                        if (!wt.wait(full_bar, ph, kWhereFull)) { ok = false; break; }
+                        tc_fence_after();
+                        const int nsub = (KBS == 2 && kb + 1 < kb1) ? 2 : 1;
+                        const uint32_t sf0 = s_sf + s * C::SF_STAGE;
+                        for (int j = 0; j < nsub; ++j) {
+                            const uint32_t cols = tmem_base + 2 * BN + (mx_set & 3u) * 12u;
+                            ++mx_set;
+                            const uint32_t sf = sf0 + j * C::SF_KB_BYTES;
+                            tmem_cp_scales(cols, smem_desc_scales(sf));
+                            tmem_cp_scales(cols + 4, smem_desc_scales(sf + 512));
+                            if (C::SFB_CHUNKS == 2) tmem_cp_scales(cols + 8, smem_desc_scales(sf + 1024));
+                            const uint32_t al = a_lo + j * (kABytes >> 4);
+                            const uint32_t bl = a_lo + ((KBS * kABytes) >> 4) + j * (C::B_BYTES >> 4);
+#pragma unroll
+                            for (uint32_t i = 0; i < 4; ++i) {
+                                const uint64_t ad = (static_cast<uint64_t>(kDescHiSw128) << 32) | (al + 2 * i);
+                                const uint64_t bd = (static_cast<uint64_t>(kDescHiSw128) << 32) | (bl + 2 * i);
+                                mma_mxf8(d, ad, bd, idesc_wide | (i << 29) | (i << 4), cols | (i << 30),
+                                         (cols + 4 + b_off) | (i << 30), (kb > kb0 || j > 0 || i > 0) ? 1u : 0u);
+                            }
+                        }
+                        mma_commit<1>(empty_bar0);
+                        full_bar = (s + 1 == STAGES) ? full(0) : full_bar + 8u;
+                        if (s + 1 == STAGES) {
+                            s = 0; ph ^= 1u;
+                            empty_bar0 = empty_base0; a_lo = a_lo0;
+                        } else {
+                            ++s;
+                            empty_bar0 += 8u; a_lo += C::STAGE_BYTES >> 4;
+                        }
+                    }
+                } else
                 for (int kb = kb0; kb < kb1; kb += KBS) {
                     if (!have && !wt.wait(full_bar, ph, kWhereFull)) { ok = false; break; }
                     tc_fence_after();
@@ -526,7 +599,7 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const bool sg = p.swiglu != 0;
             if (sg) colbase /= 2;                          // BN/2 output columns per tile
             const int row0 = tm * (128 * CTAS) + static_cast<int>(cta_rank) * 128 + q * 32;
-            if constexpr (KIND != 0) a_scale = (row0 + lane < p.M) ? __ldg(p.sa + row0 + lane) : 0.f;
+            if constexpr (kRowScaled) a_scale = (row0 + lane < p.M) ? __ldg(p.sa + row0 + lane) : 0.f;
             const int nchunks = (narrow || sg) ? C::CHUNKS / 2 : C::CHUNKS;
             const bool whole = (kb0 == 0) && (kb1 == nkb);
             auto chunk_inb = [&](int c) { return (row0 < p.M) && (colbase + c * 64 < p.N); };
@@ -699,7 +772,7 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     tmem_ld_32x32(tbase + c * 64, acc[0]);
                     tmem_ld_32x32(tbase + c * 64 + 32, acc[1]);
                     tmem_ld_wait();
-                    if constexpr (KIND != 0) dequant(acc[0], acc[1], p.sb, col0);
+                    if constexpr (kRowScaled) dequant(acc[0], acc[1], p.sb, col0);
                 }
                 if (valid && sg) {
                     // acc holds the gate pre-activations of these 64 output columns; the matching up
@@ -711,7 +784,7 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         uint32_t up[32];
                         tmem_ld_32x32(tbase + BN / 2 + c * 64 + h * 32, up);
                         tmem_ld_wait();
-                        if constexpr (KIND != 0) dequant_half(up, p.sb2, col0 + h * 32);
+                        if constexpr (kRowScaled) dequant_half(up, p.sb2, col0 + h * 32);
 #pragma unroll
                         for (int i = 0; i < 32; ++i) {
                             const float gte = __uint_as_float(acc[h][i]);
@@ -1526,6 +1599,62 @@ kx_rowquant_kernel(const QuantParams p) {
             }
         }
         __syncthreads();         // s_part / s_bcast are reused by the next row
+    }
+}
+
+// ===========================================================================
+// kx_mxquant_kernel: BF16 rows -> block-scaled FP8 (E4M3 codes, one E8M0 scale per 32 elements)
+// ===========================================================================
+// Four threads share a 32-element block (8 elements each).  Scale byte e = max(exponent field of
+// max|z| - 8, 0) (127 for an all-zero block), code = e4m3(z * 2^(127 - e)): the product is exact, so
+// the conversion instruction's rounding is the only one.  Scales are written in the chunked layout
+// the tile kernel loads: chunk (row / 128, k / 128) = 512 bytes, byte (row % 32) * 16 +
+// (row % 128) / 32 * 4 + (k / 32) % 4; entries of rows and blocks outside the matrix are set to 127.
+struct MxQuantParams {
+    const uint16_t* A;
+    uint8_t* Q;
+    uint8_t* SF;
+    long long rows, rows_pad;
+    int cols, kchunks;
+};
+
+__global__ void __launch_bounds__(256) kx_mxquant_kernel(const MxQuantParams p) {
+    pdl_wait_prior();
+    pdl_launch_dependents();
+    const int qpr = p.kchunks * 16;                       // 8-element groups per padded row
+    const long long total = p.rows_pad * qpr;             // a multiple of 32: warps stay whole
+    const long long step = static_cast<long long>(gridDim.x) * blockDim.x;
+    for (long long it = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; it < total; it += step) {
+        const long long r = it / qpr;
+        const int rem = static_cast<int>(it - r * qpr);
+        const int j = rem >> 2, k = rem * 8;
+        const bool in = (r < p.rows) && (k < p.cols);
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (in) v = *reinterpret_cast<const uint4*>(p.A + r * p.cols + k);
+        const uint32_t w4[4] = {v.x, v.y, v.z, v.w};
+        float z[8], amax = 0.f;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            z[2 * i] = bf16_lo(w4[i]);
+            z[2 * i + 1] = bf16_hi(w4[i]);
+            amax = fmaxf(amax, fmaxf(fabsf(z[2 * i]), fabsf(z[2 * i + 1])));
+        }
+        amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
+        amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
+        const int field = static_cast<int>(__float_as_uint(amax) >> 23);
+        const int e = (amax > 0.f) ? max(field - 8, 0) : 127;
+        const float mult = __uint_as_float(static_cast<uint32_t>(254 - e) << 23);      // 2^(127 - e), e <= 247
+        if (in) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) z[i] = __fmul_rn(z[i], mult);
+            *reinterpret_cast<uint2*>(p.Q + r * p.cols + k) =
+                make_uint2(pack_e4m3x4(z[0], z[1], z[2], z[3]), pack_e4m3x4(z[4], z[5], z[6], z[7]));
+        }
+        if ((rem & 3) == 0) {
+            const long long chunk = (r >> 7) * p.kchunks + (j >> 2);
+            const int off = static_cast<int>(r & 31) * 16 + static_cast<int>((r & 127) >> 5) * 4 + (j & 3);
+            p.SF[chunk * 512 + off] = static_cast<uint8_t>(in ? e : 127);
+        }
     }
 }
 

@@ -351,6 +351,43 @@ __device__ __forceinline__ uint32_t mma_kblock(uint32_t d_tmem, uint32_t a_lo, u
 #undef KX_MMA_TAIL2
 #undef KX_MMA_HEAD
 #undef KX_MMA_STEPS
+// ------------------------------------------------------------------ block-scaled FP8 (kind::mxf8f6f4)
+// Instruction descriptor of the block-scaled kind: E4M3 A and B (format 0), both K-major, E8M0
+// scales (bit 23), N >> 3 at bit 17, M >> 4 at bit 24.  The byte of the scale column that a K = 32
+// step uses (0..3 = which 32-element block of the 128-element k-block) goes into bits 4..5 (B) and
+// 29..30 (A).
+__host__ __device__ constexpr uint32_t idesc_mxf8(int m, int n) {
+    return (1u << 23) | (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(m >> 4) << 24);
+}
+// Shared-memory descriptor of one 128-row scale chunk (32 rows of 16 bytes, 512 contiguous bytes):
+// K-major, no swizzle, 8-row core matrices 128 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_scales(uint32_t smem_addr) {
+    const uint32_t lo = (smem_addr & 0x3FFFFu) >> 4;
+    const uint32_t hi = (128u >> 4) | (1u << 14);
+    return (static_cast<uint64_t>(hi) << 32) | lo;
+}
+// 32 rows x 16 bytes of shared memory -> 4 TMEM columns, the same data in each of the four 32-lane
+// quarters.  Ordered with the MMAs issued before and after it by the same thread.
+__device__ __forceinline__ void tmem_cp_scales(uint32_t taddr, uint64_t sdesc) {
+    asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+}
+// D[tmem] (+)= (A * scale_a) * (B * scale_b)^T, one K = 32 step; sfa / sfb = TMEM column of the scales
+__device__ __forceinline__ void mma_mxf8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                         uint32_t sfa, uint32_t sfb, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::mxf8f6f4.block_scale [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa), "r"(sfb)
+        : "memory");
+}
+// Plain (untiled) bulk copy global -> this CTA's shared memory, completing on an mbarrier.  Both
+// addresses 16-byte aligned, size a multiple of 16.
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                 "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+
 // Arrive on an mbarrier once every MMA issued so far by this thread has finished.
 // `bar` is a shared::cluster address (this CTA's own shared::cta address is one).
 template <int CTAS>
