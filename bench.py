@@ -616,6 +616,44 @@ def run_ours(args):
             del keep, calls
             torch.cuda.empty_cache()
 
+        # block-scaled FP8: the code book (BF16 -> codes + one scale byte per 32 elements), then the projection on
+        # those codes (scales stay on the device in the layout the kernel loads)
+        for (Mo, No, Ko) in [(4096, 4096, 4096), (16384, 4096, 14336)]:
+            ops = 2.0 * Mo * No * Ko
+            nbytes = 1.0 * (Mo * Ko + No * Ko) * (1.0 + 1.0 / 32) + 4.0 * Mo * No
+            ns = int(max(2, min(8, math.ceil(2.0 * L2_BYTES / nbytes))))
+            keep, calls, qcalls = [], [], []
+            for _ in range(ns):
+                Xs = torch.randn(Mo, Ko, device="cuda", generator=g).bfloat16()
+                Ws = (torch.randn(No, Ko, device="cuda", generator=g) / math.sqrt(Ko)).bfloat16()
+                Xq = torch.empty(Mo, Ko, device="cuda", dtype=torch.uint8)
+                Wq = torch.empty(No, Ko, device="cuda", dtype=torch.uint8)
+                sfx = torch.empty(int(lib.kx_mx_scale_bytes(i64(Mo), i64(Ko))), device="cuda", dtype=torch.uint8)
+                sfw = torch.empty(int(lib.kx_mx_scale_bytes(i64(No), i64(Ko))), device="cuda", dtype=torch.uint8)
+                Rs = torch.randn(Mo, No, device="cuda", generator=g).bfloat16()
+                Ys = torch.empty(Mo, No, dtype=torch.bfloat16, device="cuda")
+                qa = (vp(Xs.data_ptr()), vp(Xq.data_ptr()), vp(sfx.data_ptr()), i64(Mo), i64(Ko), st)
+                rcq = lib.kx_quantize_rows_mxfp8(*qa)
+                rcq = rcq or lib.kx_quantize_rows_mxfp8(vp(Ws.data_ptr()), vp(Wq.data_ptr()), vp(sfw.data_ptr()), i64(No),
+                                                        i64(Ko), st)
+                if rcq != 0:
+                    raise SystemExit(f"kx_quantize_rows_mxfp8 failed ({rcq})")
+                torch.cuda.synchronize()
+                keep.append((Xs, Xq, Wq, sfx, sfw, Rs, Ys))
+                del Ws
+                a = (vp(Xq.data_ptr()), vp(sfx.data_ptr()), vp(Wq.data_ptr()), vp(sfw.data_ptr()), vp(None),
+                     vp(Rs.data_ptr()), vp(Ys.data_ptr()), i64(Mo), i64(No), i64(Ko), st)
+                calls.append(lambda a=a: lib.kx_outproj_residual_mxfp8(*a))
+                qcalls.append(lambda qa=qa: lib.kx_quantize_rows_mxfp8(*qa))
+            wlo = inputs.Workload(f"outproj_mxfp8_M{Mo}_N{No}_K{Ko}", Mo, No, Ko, 0, False, True)
+            t, tbest, _ = time_shape(torch, kx, wlo, calls)
+            report(wlo.name, t, tbest, nbytes, ops, ns)
+            wlq = inputs.Workload(f"quantize_rows_mxfp8_M{Mo}_K{Ko}", Mo, Ko, 0, 0, False, False)
+            t, tbest, _ = time_shape(torch, kx, wlq, qcalls)
+            report(wlq.name, t, tbest, Mo * Ko * (3.0 + 1.0 / 32), 0.0, ns)
+            del keep, calls, qcalls
+            torch.cuda.empty_cache()
+
     # ---- the oracle on the host cores, bounded sample (rank 0, N = 1 only)
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

@@ -29,7 +29,7 @@ EXPORTS = (
     "kx_outproj_residual_int8",
     "kx_quantize_rows_fp8", "kx_quantize_gate_up_fp8", "kx_rmsnorm_quantize_fp8", "kx_gate_up_swiglu_fp8",
     "kx_outproj_residual_fp8",
-    "kx_mx_scale_bytes", "kx_quantize_rows_mxfp8", "kx_outproj_residual_mxfp8",
+    "kx_mx_scale_bytes", "kx_quantize_rows_mxfp8", "kx_outproj_residual_mxfp8", "kx_outproj_residual_mxfp8_ex",
     "kx_plan_query", "kx_last_device_status", "kx_status_string",
     "kx_version",
 )
@@ -100,6 +100,7 @@ def load():
     lib.kx_mx_scale_bytes.argtypes = [i64, i64]
     lib.kx_quantize_rows_mxfp8.argtypes = [vp, vp, vp, i64, i64, vp]
     lib.kx_outproj_residual_mxfp8.argtypes = [vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, vp]
+    lib.kx_outproj_residual_mxfp8_ex.argtypes = [vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, vp, ctypes.POINTER(PlanOverride)]
     lib.kx_plan_query.argtypes = [i64, i64, i64, ci, ci, ctypes.POINTER(PlanOverride), ctypes.POINTER(PlanInfo)]
     lib.kx_last_device_status.argtypes = [vp, ctypes.POINTER(ci), ctypes.POINTER(ci)]
     lib.kx_status_string.argtypes = [ci]
@@ -507,16 +508,21 @@ def kx_quantize_rows_mxfp8(A, Q, SF, stream=None, check=True) -> int:
     return rc
 
 
-def kx_outproj_residual_mxfp8(Xq, SFX, Wq, SFW, bias, R, Y, stream=None, check=True) -> int:
-    """Y = block-scaled (Xq, SFX) (Wq, SFW)^T + bias + R; bias / R may be None; R may be Y."""
+def kx_outproj_residual_mxfp8(Xq, SFX, Wq, SFW, bias, R, Y, stream=None, check=True, override=None) -> int:
+    """Y = block-scaled (Xq, SFX) (Wq, SFW)^T + bias + R; bias / R may be None; R may be Y.
+    override: a PlanOverride (block_n, cta_pair, raster_group) or None."""
     import torch
     M, K = Xq.shape
     N = Wq.shape[0]
     _check("Xq", Xq, (M, K), torch.float8_e4m3fn); _check("Wq", Wq, (N, K), torch.float8_e4m3fn)
     _check("SFX", SFX, (kx_mx_scale_bytes(M, K),), torch.uint8); _check("SFW", SFW, (kx_mx_scale_bytes(N, K),), torch.uint8)
     _check_bf16("bias", bias, (N,)); _check_bf16("R", R, (M, N)); _check_bf16("Y", Y, (M, N))
-    rc = load().kx_outproj_residual_mxfp8(_addr(Xq), _addr(SFX), _addr(Wq), _addr(SFW), _addr(bias), _addr(R), _addr(Y),
-                                          M, N, K, _stream(stream))
+    if override is None:
+        rc = load().kx_outproj_residual_mxfp8(_addr(Xq), _addr(SFX), _addr(Wq), _addr(SFW), _addr(bias), _addr(R), _addr(Y),
+                                              M, N, K, _stream(stream))
+    else:
+        rc = load().kx_outproj_residual_mxfp8_ex(_addr(Xq), _addr(SFX), _addr(Wq), _addr(SFW), _addr(bias), _addr(R),
+                                                 _addr(Y), M, N, K, _stream(stream), ctypes.byref(override))
     if check and rc != KX_OK:
         raise KxError(rc, "kx_outproj_residual_mxfp8")
     return rc

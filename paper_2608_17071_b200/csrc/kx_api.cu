@@ -110,18 +110,21 @@ const SwapVariant kSwapVariants[] = {
 
 // Block-scaled FP8 tile kernels (one CTA per tile; two accumulators and the scale columns share TMEM)
 struct MxVariant {
-    int bn, stages, nb, kbs, smem;
+    int bn, ctas, stages, nb, kbs, smem;
     const void* fn;
 };
-#define KX_MX(BN, ST, NB, KBS)                                                                \
+#define KX_MX(BN, CTAS, ST, NB, KBS)                                                          \
     MxVariant {                                                                               \
-        BN, ST, NB, KBS, TileCfg<BN, 1, ST, NB, KBS, 1>::SMEM_BYTES,                          \
-            reinterpret_cast<const void*>(&kx_tile_kernel<BN, 1, ST, NB, 3, KBS>)             \
+        BN, CTAS, ST, NB, KBS, TileCfg<BN, CTAS, ST, NB, KBS, 1>::SMEM_BYTES,                 \
+            reinterpret_cast<const void*>(&kx_tile_kernel<BN, CTAS, ST, NB, 3, KBS>)          \
     }
-const MxVariant kMxVariants[] = {KX_MX(128, 5, 2, 1), KX_MX(192, 4, 3, 1)};
-const MxVariant* find_mx(int bn) {
+// (tile width, CTAs per tile, ring stages, R staging buffers, k-blocks per stage); first match = default,
+// the rest by the `stages` field of the plan override
+const MxVariant kMxVariants[] = {KX_MX(128, 1, 5, 2, 1), KX_MX(192, 1, 4, 3, 1), KX_MX(192, 2, 5, 3, 1),
+                                 KX_MX(128, 2, 6, 2, 1), KX_MX(128, 1, 2, 2, 2), KX_MX(192, 1, 2, 3, 2)};
+const MxVariant* find_mx(int bn, int ctas, int stages = 0) {
     for (const auto& v : kMxVariants)
-        if (v.bn == bn) return &v;
+        if (v.bn == bn && v.ctas == ctas && (stages == 0 || v.stages == stages)) return &v;
     return nullptr;
 }
 
@@ -269,6 +272,37 @@ int get_tmap(const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows, C
     if (r != CUDA_SUCCESS) {
         e.valid = false;
         if (log_enabled()) std::fprintf(stderr, "[kx] cuTensorMapEncodeTiled failed: %d\n", static_cast<int>(r));
+        return KX_ERR_CUDA;
+    }
+    e.key = key;
+    e.valid = true;
+    *out = e.map;
+    return KX_OK;
+}
+
+// Scale chunks of a block-scaled operand as a 2-D tensor [chunks][128 32-bit words], one chunk
+// (512 contiguous bytes, no swizzle) per box.  Shares the descriptor cache (box_rows 1, 4-byte elements).
+int get_tmap_scales(const void* ptr, uint64_t chunks, CUtensorMap* out) {
+    TmapKey key{ptr, chunks, 128, 128, 1, 4};
+    uint64_t h = reinterpret_cast<uint64_t>(ptr) >> 4;
+    h ^= chunks * 0x9E3779B97F4A7C15ull;
+    h ^= 0x51ED270B27D4EB4Full;
+    h ^= h >> 29;
+    TmapEntry& e = t_tmaps[h % kTmapSlots];
+    if (e.valid && e.key == key) {
+        *out = e.map;
+        return KX_OK;
+    }
+    cuuint64_t dims[2] = {128, chunks};
+    cuuint64_t strides[1] = {512};
+    cuuint32_t box[2] = {128, 1};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = g_encode(&e.map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        e.valid = false;
+        if (log_enabled()) std::fprintf(stderr, "[kx] cuTensorMapEncodeTiled (scales) failed: %d\n", static_cast<int>(r));
         return KX_ERR_CUDA;
     }
     e.key = key;
@@ -745,7 +779,7 @@ int run(const void* X, const void* W, const void* bias, const void* R, void* Y, 
         p.trace = g_kx_trace;
 #endif
         const uint16_t* bias_p = static_cast<const uint16_t*>(bias);
-        void* args[] = {&tmA, &tmB, &tmB2, &tmY, &tmR, &bias_p, &p};
+        void* args[] = {&tmA, &tmB, &tmB2, &tmY, &tmR, &tmR, &bias_p, &p};
         if (cudaLaunchKernelExC(&cfg, pl.fn, args) != cudaSuccess) {
             cudaGetLastError();
             return KX_ERR_CUDA;
@@ -1137,7 +1171,7 @@ int kx_gate_up_swiglu(const void* X, const void* Wg, const void* Wu, void* Z, in
     cfg.attrs = attr;
     cfg.numAttrs = nattr;
     const uint16_t* bias_p = nullptr;
-    void* args[] = {&tmA, &tmG, &tmU, &tmZ, &tmZ, &bias_p, &p};
+    void* args[] = {&tmA, &tmG, &tmU, &tmZ, &tmZ, &tmZ, &bias_p, &p};
     if (cudaLaunchKernelExC(&cfg, pl.fn, args) != cudaSuccess) {
         cudaGetLastError();
         return KX_ERR_CUDA;
@@ -1381,7 +1415,7 @@ int run_q8(int kind, const void* Xq, const float* sx, const void* Wq, const floa
     cfg.attrs = attr;
     cfg.numAttrs = nattr;
     const uint16_t* bias_p = static_cast<const uint16_t*>(bias);
-    void* args[] = {&tmA, &tmB, &tmB2, &tmY, &tmR, &bias_p, &p};
+    void* args[] = {&tmA, &tmB, &tmB2, &tmY, &tmR, &tmR, &bias_p, &p};
     if (cudaLaunchKernelExC(&cfg, kind == 2 ? pl.fn_f8 : pl.fn_s8, args) != cudaSuccess) {
         cudaGetLastError();
         return KX_ERR_CUDA;
@@ -1610,8 +1644,10 @@ int kx_quantize_rows_mxfp8(const void* A, void* Q, void* SF, int64_t rows, int64
     return KX_OK;
 }
 
-int kx_outproj_residual_mxfp8(const void* Xq, const void* SFX, const void* Wq, const void* SFW, const void* bias,
-                              const void* R, void* Y, int64_t M, int64_t N, int64_t K, void* stream_v) {
+namespace {
+int outproj_residual_mx(const void* Xq, const void* SFX, const void* Wq, const void* SFW, const void* bias,
+                        const void* R, void* Y, int64_t M, int64_t N, int64_t K, void* stream_v,
+                        const kx_plan_override* ov) {
     if (M < 0 || N < 0 || K < 0) return KX_ERR_SHAPE;
     if (M > 0x7FFFFFFFll / 2 || N > 0x7FFFFFFFll / 4 || K > 0x7FFFFFFFll / 2) return KX_ERR_SHAPE;
     if (M == 0 || N == 0) return KX_OK;
@@ -1638,21 +1674,33 @@ int kx_outproj_residual_mxfp8(const void* Xq, const void* SFX, const void* Wq, c
         overlaps(Y, yb, SFX, static_cast<size_t>(kx_mx_scale_bytes(M, K))) ||
         overlaps(Y, yb, SFW, static_cast<size_t>(kx_mx_scale_bytes(N, K))))
         return KX_ERR_OVERLAP;
-    // tile width: 192 when it leaves fewer idle tile slots in the last wave than 128
-    const long long tm = (M + 127) / 128;
-    auto waste = [&](int bn) {
-        const long long tiles = tm * ((N + bn - 1) / bn);
-        const long long waves = (tiles + ctx->sm_count - 1) / ctx->sm_count;
-        return static_cast<double>(waves * ctx->sm_count) * bn;          // column-slots paid for
-    };
-    const int bn = (N > 128 && waste(192) < waste(128)) ? 192 : 128;
-    const MxVariant* v = find_mx(bn);
-    if (!v) return KX_ERR_PLAN;
+    // Tile shape: the candidate with the smallest estimated time = waves x columns per tile / relative
+    // tile rate (a CTA pair shares the W tile and halves the issue work per flop; measured ratios).
+    const MxVariant* v = nullptr;
+    if (ov && (ov->block_n || ov->cta_pair || ov->stages)) {
+        v = find_mx(ov->block_n ? ov->block_n : 128, ov->cta_pair ? ov->cta_pair : 1, ov->stages);
+        if (!v) return KX_ERR_PLAN;
+    } else {
+        double best = 0.0;
+        for (const auto& c : kMxVariants) {
+            const long long slots = ctx->sm_count / c.ctas;
+            const long long tiles = ((M + 128 * c.ctas - 1) / (128 * c.ctas)) * ((N + c.bn - 1) / c.bn);
+            const long long waves = (tiles + slots - 1) / slots;
+            const double rate = (c.ctas == 2 ? 1.3 : 1.0) * (c.bn == 192 ? 1.08 : 1.0);
+            const double t = static_cast<double>(waves) * c.bn / rate;
+            if (!v || t < best) { v = &c; best = t; }
+        }
+    }
+    const int bn = v->bn, ctas = v->ctas;
+    const long long tm = (M + 128 * ctas - 1) / (128 * ctas);
     const long long tiles_n = (N + bn - 1) / bn, tiles = tm * tiles_n;
     if (tiles > 0x7FFFFFFFll / 4) return KX_ERR_SHAPE;
-    CUtensorMap tmA, tmB, tmY, tmR;
+    const long long kchunks = mx_chunks(K);
+    CUtensorMap tmA, tmB, tmY, tmR, tmSA, tmSB;
     if ((rc = get_tmap(Xq, M, K, 128, &tmA, 1)) != KX_OK) return rc;
-    if ((rc = get_tmap(Wq, N, K, bn, &tmB, 1)) != KX_OK) return rc;
+    if ((rc = get_tmap(Wq, N, K, bn / ctas, &tmB, 1)) != KX_OK) return rc;
+    if ((rc = get_tmap_scales(SFX, mx_chunks(M) * kchunks, &tmSA)) != KX_OK) return rc;
+    if ((rc = get_tmap_scales(SFW, mx_chunks(N) * kchunks, &tmSB)) != KX_OK) return rc;
     if ((rc = get_tmap(Y, M, N, 32, &tmY)) != KX_OK) return rc;
     if (R) {
         if ((rc = get_tmap(R, M, N, 32, &tmR)) != KX_OK) return rc;
@@ -1667,7 +1715,7 @@ int kx_outproj_residual_mxfp8(const void* Xq, const void* SFX, const void* Wq, c
     p.tiles_m = static_cast<int>(tm);
     p.tiles_n = static_cast<int>(tiles_n);
     p.num_tiles = static_cast<int>(tiles);
-    p.raster_group = 8;
+    p.raster_group = (ov && ov->raster_group > 0) ? ov->raster_group : 8;
     p.has_bias = bias ? 1 : 0;
     p.has_r = R ? 1 : 0;
     p.kcluster = 1;
@@ -1677,27 +1725,46 @@ int kx_outproj_residual_mxfp8(const void* Xq, const void* SFX, const void* Wq, c
     p.status = ctx->status;
     p.ws = ctx->ws;
     p.counters = ctx->counters;
-    p.sfa = static_cast<const uint8_t*>(SFX);
-    p.sfb = static_cast<const uint8_t*>(SFW);
     p.sfb_chunks = static_cast<int>(mx_chunks(N));
     cudaLaunchConfig_t cfg;
     std::memset(&cfg, 0, sizeof cfg);
-    cfg.gridDim = dim3(static_cast<unsigned>(std::min<long long>(tiles, ctx->sm_count)), 1, 1);
+    const long long slots = std::min<long long>(tiles, ctx->sm_count / ctas);
+    cfg.gridDim = dim3(static_cast<unsigned>(slots * ctas), 1, 1);
     cfg.blockDim = dim3(kThreads, 1, 1);
     cfg.dynamicSmemBytes = v->smem;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchAttribute attr[2];
+    int nattr = 0;
+    attr[nattr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[nattr].val.programmaticStreamSerializationAllowed = 1;
+    ++nattr;
+    if (ctas == 2) {
+        attr[nattr].id = cudaLaunchAttributeClusterDimension;
+        attr[nattr].val.clusterDim.x = 2;
+        attr[nattr].val.clusterDim.y = 1;
+        attr[nattr].val.clusterDim.z = 1;
+        ++nattr;
+    }
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = nattr;
     const uint16_t* bias_p = static_cast<const uint16_t*>(bias);
-    void* args[] = {&tmA, &tmB, &tmB, &tmY, &tmR, &bias_p, &p};
+    void* args[] = {&tmA, &tmB, &tmSA, &tmY, &tmR, &tmSB, &bias_p, &p};
     if (cudaLaunchKernelExC(&cfg, v->fn, args) != cudaSuccess) {
         cudaGetLastError();
         return KX_ERR_CUDA;
     }
     return KX_OK;
+}
+}  // namespace
+
+int kx_outproj_residual_mxfp8(const void* Xq, const void* SFX, const void* Wq, const void* SFW, const void* bias,
+                              const void* R, void* Y, int64_t M, int64_t N, int64_t K, void* stream) {
+    return outproj_residual_mx(Xq, SFX, Wq, SFW, bias, R, Y, M, N, K, stream, nullptr);
+}
+int kx_outproj_residual_mxfp8_ex(const void* Xq, const void* SFX, const void* Wq, const void* SFW, const void* bias,
+                                 const void* R, void* Y, int64_t M, int64_t N, int64_t K, void* stream,
+                                 const kx_plan_override* ov) {
+    return outproj_residual_mx(Xq, SFX, Wq, SFW, bias, R, Y, M, N, K, stream, ov);
 }
 
 // ---------------------------------------------------------------- no-allocation entry

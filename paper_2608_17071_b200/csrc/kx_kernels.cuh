@@ -128,9 +128,7 @@ struct TileParams {
     const float* sa;           // KIND 1 / 2: scale per row of A [M]
     const float* sb;           // KIND 1 / 2: scale per row of B [N] (gate rows in gate/up mode)
     const float* sb2;          // KIND 1 / 2, gate/up mode: scale per up row [N]
-    const uint8_t* sfa;        // KIND 3: E8M0 block scales of A, 512-byte chunks [ceil(M/128)][k-blocks]
-    const uint8_t* sfb;        // KIND 3: E8M0 block scales of B, same layout over N
-    int sfb_chunks;            // KIND 3: ceil(N / 128)
+    int sfb_chunks;            // KIND 3: ceil(N / 128) = rows of 128-row scale chunks of B
     int swiglu;                   // 1: gate/up mode.  W rows of a tile = BN/2 rows of Wg (tmB) followed by the same
                                   // BN/2 rows of Wu (tmB2); the epilogue writes silu(gate) * up, BN/2 columns per
                                   // tile, N = number of output columns; no bias, no residual
@@ -170,7 +168,7 @@ struct TileCfg {
     static constexpr int SF_STAGE = KBS * SF_KB_BYTES;
     static constexpr int SMEM_BYTES = 1024 + STAGES * (STAGE_BYTES + SF_STAGE) + EPI_BYTES + 1024;
     static constexpr int TMEM_COLS = tmem_cols_for(2 * BN + (MX ? 48 : 0));
-    static_assert(!MX || (CTAS == 1 && BN <= 192), "block-scaled variants: one CTA per tile, two accumulators + scales in TMEM");
+    static_assert(!MX || BN <= 192, "block-scaled variants: two accumulators and the scale columns share TMEM");
     static_assert(SMEM_BYTES <= 232448, "shared memory");
     static constexpr int CHUNKS = BN / 64;                  // 64-column epilogue chunks per tile
     static constexpr int PART_FLOATS = 128 * BN;            // one CTA's FP32 partial of one tile
@@ -239,12 +237,14 @@ __device__ __forceinline__ uint32_t ld_acquire_gpu_u32(const unsigned int* p) {
 // K-cluster fix-ups add partial accumulators as unscaled FP32).  KIND 3: FP8 E4M3 operands with one
 // E8M0 scale per 32 elements of a row (tcgen05 kind::mxf8f6f4.block_scale): the scales travel through
 // the ring beside the operand tiles, are copied to TMEM before the four K steps of their k-block, and
-// the FP32 accumulators need no dequantisation; one CTA per tile, whole full-width tiles only.
+// the FP32 accumulators need no dequantisation; whole full-width tiles only.  Its scale chunks come
+// through two more tensor maps: tmB2 = scales of A, tmS = scales of B, both [chunks][128 words].
 template <int BN, int CTAS, int STAGES, int NB, int KIND = 0, int KBS = 1>
 __global__ void __launch_bounds__(kThreads, 1)
 kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmB2, const __grid_constant__ CUtensorMap tmY,
-               const __grid_constant__ CUtensorMap tmR, const uint16_t* __restrict__ bias, const TileParams p) {
+               const __grid_constant__ CUtensorMap tmR, const __grid_constant__ CUtensorMap tmS,
+               const uint16_t* __restrict__ bias, const TileParams p) {
     using C = TileCfg<BN, CTAS, STAGES, NB, KBS, KIND == 3 ? 1 : 0>;
     constexpr bool kRowScaled = (KIND == 1 || KIND == 2);       // dequantised in the epilogue
     extern __shared__ uint8_t smem_raw[];
@@ -294,7 +294,8 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (warp == 4 && lane == 0) {
         prefetch_tmap(&tmA);
         prefetch_tmap(&tmB);
-        if (p.narrow_tile0 < p.num_tiles) prefetch_tmap(&tmB2);
+        if (p.narrow_tile0 < p.num_tiles || KIND == 3) prefetch_tmap(&tmB2);
+        if (KIND == 3) prefetch_tmap(&tmS);
         prefetch_tmap(&tmY);
         if (p.has_r) prefetch_tmap(&tmR);
         // Warm L2 with the first ring-full of this CTA's operand tiles before waiting for the
@@ -390,23 +391,26 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     if (!wt.wait(empty(s), ph ^ 1u, kWhereEmpty)) { ok = false; break; }
                     const uint32_t sa = s_stage + s * C::STAGE_BYTES;
                     const uint32_t sb = sa + KBS * kABytes;
-                    if constexpr (CTAS == 1) {
-                        mbar_arrive_expect_tx(full(s), nsub * (stage_tx + C::SF_KB_BYTES));
-                        if constexpr (KIND == 3) {
-                            // scale chunks of this tile's rows for k-block kb: chunk (row / 128, kb); a B
-                            // chunk past the end of the array (ragged last tile) is replaced by the last one,
-                            // its rows are zero-filled operand rows
-                            const int c0 = col >> 7;
-                            for (int j = 0; j < nsub; ++j) {
-                                const uint32_t dst = s_sf + s * C::SF_STAGE + j * C::SF_KB_BYTES;
-                                bulk_load(dst, p.sfa + (static_cast<size_t>(tm) * nkb + (kb + j)) * 512, 512, full(s));
-                                for (int i = 0; i < C::SFB_CHUNKS; ++i) {
-                                    const int ch = min(c0 + i, p.sfb_chunks - 1);
-                                    bulk_load(dst + 512 * (1 + i), p.sfb + (static_cast<size_t>(ch) * nkb + (kb + j)) * 512,
-                                              512, full(s));
-                                }
+                    if constexpr (KIND == 3) {
+                        // scale chunks of this CTA's A rows and of all the tile's B rows for k-block kb:
+                        // chunk (row / 128, kb).  A B chunk past the end of the array (ragged last tile) is
+                        // replaced by the last one: its rows belong to zero-filled operand rows.
+                        const int c0 = col >> 7;
+                        const uint32_t fb = (CTAS == 1) ? full(s) : map_to_cta(full(s), 0);
+                        for (int j = 0; j < nsub; ++j) {
+                            const uint32_t dst = s_sf + s * C::SF_STAGE + j * C::SF_KB_BYTES;
+                            const int ya = (tm * CTAS + static_cast<int>(cta_rank)) * nkb + kb + j;
+                            if constexpr (CTAS == 1) tma_load_2d(dst, &tmB2, 0, ya, fb);
+                            else tma_load_2d_pair(dst, &tmB2, 0, ya, fb);
+                            for (int i = 0; i < C::SFB_CHUNKS; ++i) {
+                                const int yb = min(c0 + i, p.sfb_chunks - 1) * nkb + kb + j;
+                                if constexpr (CTAS == 1) tma_load_2d(dst + 512 * (1 + i), &tmS, 0, yb, fb);
+                                else tma_load_2d_pair(dst + 512 * (1 + i), &tmS, 0, yb, fb);
                             }
                         }
+                    }
+                    if constexpr (CTAS == 1) {
+                        mbar_arrive_expect_tx(full(s), nsub * (stage_tx + C::SF_KB_BYTES));
                         for (int j = 0; j < nsub; ++j) {
                             tma_load_2d(sa + j * kABytes, &tmA, (kb + j) * KBLK, a_row, full(s));
                             tma_load_2d(sb + j * C::B_BYTES, mapB, (kb + j) * KBLK, b_row, full(s));
@@ -414,7 +418,7 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         }
                     } else {
                         // both CTAs' copies complete on the leader's barrier
-                        if (leader) mbar_arrive_expect_tx(full(s), 2 * nsub * stage_tx);
+                        if (leader) mbar_arrive_expect_tx(full(s), 2 * nsub * (stage_tx + C::SF_KB_BYTES));
                         const uint32_t fb = map_to_cta(full(s), 0);
                         for (int j = 0; j < nsub; ++j) {
                             tma_load_2d_pair(sa + j * kABytes, &tmA, (kb + j) * KBLK, a_row, fb);
@@ -435,7 +439,7 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (leader && lane == 0) {
             constexpr uint32_t idesc_wide = KIND == 1   ? idesc_s8_s32(128 * CTAS, BN)
                                             : KIND == 2 ? idesc_e4m3_f32(128 * CTAS, BN)
-                                            : KIND == 3 ? idesc_mxf8(128, BN)
+                                            : KIND == 3 ? idesc_mxf8(128 * CTAS, BN)
                                                         : idesc_bf16_f32(128 * CTAS, BN);
             constexpr uint32_t idesc_narrow = KIND == 1   ? idesc_s8_s32(128 * CTAS, BN / 2)
                                               : KIND == 2 ? idesc_e4m3_f32(128 * CTAS, BN / 2)
@@ -475,27 +479,20 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                             const uint32_t cols = tmem_base + 2 * BN + (mx_set & 3u) * 12u;
                             ++mx_set;
                             const uint32_t sf = sf0 + j * C::SF_KB_BYTES;
-                            tmem_cp_scales(cols, smem_desc_scales(sf));
-                            tmem_cp_scales(cols + 4, smem_desc_scales(sf + 512));
-                            if (C::SFB_CHUNKS == 2) tmem_cp_scales(cols + 8, smem_desc_scales(sf + 1024));
                             const uint32_t al = a_lo + j * (kABytes >> 4);
                             const uint32_t bl = a_lo + ((KBS * kABytes) >> 4) + j * (C::B_BYTES >> 4);
-#pragma unroll
-                            for (uint32_t i = 0; i < 4; ++i) {
-                                const uint64_t ad = (static_cast<uint64_t>(kDescHiSw128) << 32) | (al + 2 * i);
-                                const uint64_t bd = (static_cast<uint64_t>(kDescHiSw128) << 32) | (bl + 2 * i);
-                                mma_mxf8(d, ad, bd, idesc_wide | (i << 29) | (i << 4), cols | (i << 30),
-                                         (cols + 4 + b_off) | (i << 30), (kb > kb0 || j > 0 || i > 0) ? 1u : 0u);
-                            }
+                            mma_kblock_mx<CTAS, C::SFB_CHUNKS>(d, al, bl, idesc_wide, (kb > kb0 || j > 0) ? 1u : 0u,
+                                                               (sf & 0x3FFFFu) >> 4, cols, cols + 4 + b_off);
                         }
-                        mma_commit<1>(empty_bar0);
+                        mma_commit<CTAS>(empty_bar0);
+                        if constexpr (CTAS == 2) mma_commit<2>(empty_bar1);
                         full_bar = (s + 1 == STAGES) ? full(0) : full_bar + 8u;
                         if (s + 1 == STAGES) {
                             s = 0; ph ^= 1u;
-                            empty_bar0 = empty_base0; a_lo = a_lo0;
+                            empty_bar0 = empty_base0; empty_bar1 = empty_base1; a_lo = a_lo0;
                         } else {
                             ++s;
-                            empty_bar0 += 8u; a_lo += C::STAGE_BYTES >> 4;
+                            empty_bar0 += 8u; empty_bar1 += 8u; a_lo += C::STAGE_BYTES >> 4;
                         }
                     }
                 } else

@@ -368,25 +368,72 @@ __device__ __forceinline__ uint64_t smem_desc_scales(uint32_t smem_addr) {
 }
 // 32 rows x 16 bytes of shared memory -> 4 TMEM columns, the same data in each of the four 32-lane
 // quarters.  Ordered with the MMAs issued before and after it by the same thread.
+// With CTAS == 2 each CTA of the pair copies from its own shared memory (same offset) into its own
+// tensor memory.
+template <int CTAS>
 __device__ __forceinline__ void tmem_cp_scales(uint32_t taddr, uint64_t sdesc) {
-    asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+    if constexpr (CTAS == 1)
+        asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+    else
+        asm volatile("tcgen05.cp.cta_group::2.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
 }
 // D[tmem] (+)= (A * scale_a) * (B * scale_b)^T, one K = 32 step; sfa / sfb = TMEM column of the scales
+template <int CTAS>
 __device__ __forceinline__ void mma_mxf8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
                                          uint32_t sfa, uint32_t sfb, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::mxf8f6f4.block_scale [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
-        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa), "r"(sfb)
-        : "memory");
+    if constexpr (CTAS == 1)
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::mxf8f6f4.block_scale [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
+            ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa), "r"(sfb)
+            : "memory");
+    else
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::2.kind::mxf8f6f4.block_scale [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
+            ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa), "r"(sfb)
+            : "memory");
 }
-// Plain (untiled) bulk copy global -> this CTA's shared memory, completing on an mbarrier.  Both
-// addresses 16-byte aligned, size a multiple of 16.
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-                 "l"(src), "r"(bytes), "r"(bar)
-                 : "memory");
+// One k-block (128 FP8 elements) of the block-scaled kind in a single instruction block: the scale
+// chunks (A, then CHUNKS of B, 512 bytes apart in shared memory) go to TMEM columns cols, cols + 4
+// (, cols + 8), then four K = 32 steps, step i reading byte i of the scale columns (sfb = first
+// scale column of the tile's B rows).  a_lo / b_lo / sf_lo are the low words of the shared-memory
+// descriptors; acc_first = 0 makes step 0 overwrite the accumulator.
+#define KX_MX_CP(G, OFFS, OFFT)                                                                            \
+        "add.u32 t, %6, " OFFS ";\n\tmov.b64 ds, {t, %7};\n\tadd.u32 sa, %8, " OFFT ";\n\t"               \
+        "tcgen05.cp.cta_group::" G ".32x128b.warpx4 [sa], ds;\n\t"
+#define KX_MX_STEP(G, KOFF, IDOFF, SFOFF, P)                                                               \
+        "add.u32 al, %1, " KOFF ";\n\tadd.u32 bl, %2, " KOFF ";\n\tmov.b64 da, {al, %4};\n\tmov.b64 db, {bl, %4};\n\t" \
+        "add.u32 id, %3, " IDOFF ";\n\tadd.u32 sa, %8, " SFOFF ";\n\tadd.u32 sb, %9, " SFOFF ";\n\t"         \
+        "tcgen05.mma.cta_group::" G ".kind::mxf8f6f4.block_scale [%0], da, db, id, [sa], [sb], " P ";\n\t"
+#define KX_MX_BODY(G, CP2)                                                                                 \
+    asm volatile(                                                                                          \
+        "{\n\t.reg .pred p, q;\n\t.reg .b64 da, db, ds;\n\t.reg .b32 al, bl, t, sa, sb, id;\n\t"          \
+        "setp.ne.b32 p, %5, 0;\n\tsetp.eq.b32 q, %0, %0;\n\t"                                             \
+        KX_MX_CP(G, "0", "0") KX_MX_CP(G, "32", "4") CP2                                                   \
+        KX_MX_STEP(G, "0", "0", "0", "p")                                                                  \
+        KX_MX_STEP(G, "2", "0x20000010", "0x40000000", "q")                                                \
+        KX_MX_STEP(G, "4", "0x40000020", "0x80000000", "q")                                                \
+        KX_MX_STEP(G, "6", "0x60000030", "0xC0000000", "q")                                                \
+        "}" ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(desc_hi), "r"(acc_first), "r"(sf_lo),     \
+        "r"(sf_hi), "r"(cols), "r"(sfb)                                                                    \
+        : "memory")
+template <int CTAS, int CHUNKS>
+__device__ __forceinline__ void mma_kblock_mx(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc,
+                                              uint32_t acc_first, uint32_t sf_lo, uint32_t cols, uint32_t sfb) {
+    const uint32_t desc_hi = kDescHiSw128;
+    const uint32_t sf_hi = (128u >> 4) | (1u << 14);
+    if constexpr (CTAS == 1) {
+        if constexpr (CHUNKS == 2) KX_MX_BODY("1", KX_MX_CP("1", "64", "8"));
+        else KX_MX_BODY("1", "");
+    } else {
+        if constexpr (CHUNKS == 2) KX_MX_BODY("2", KX_MX_CP("2", "64", "8"));
+        else KX_MX_BODY("2", "");
+    }
 }
+#undef KX_MX_BODY
+#undef KX_MX_STEP
+#undef KX_MX_CP
 
 // Arrive on an mbarrier once every MMA issued so far by this thread has finished.
 // `bar` is a shared::cluster address (this CTA's own shared::cta address is one).

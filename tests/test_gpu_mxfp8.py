@@ -100,15 +100,21 @@ def small_codes(seed, shape):
     return SMALL[np.random.default_rng(seed).integers(0, len(SMALL), size=shape)]
 
 
-def run_proj(Xq, ex, Wq, ew, b=None, R=None, inplace=False):
+# (tile columns, CTAs per tile, ring stages: 0 = default variant, 2 = the variants whose stages hold two k-blocks)
+VARIANTS = [(128, 1, 0), (192, 1, 0), (128, 2, 0), (192, 2, 0), (128, 1, 2), (192, 1, 2)]
+
+
+def run_proj(Xq, ex, Wq, ew, b=None, R=None, inplace=False, variant=None):
     (M, K), N = Xq.shape, Wq.shape[0]
+    ov = None if variant is None else kx.make_override(block_n=variant[0], cta_pair=variant[1], stages=variant[2])
     if inplace:
         Y = kt.to_dev(R)
         Rd = Y
     else:
         Y = kt.nan_filled(M, N)
         Rd = kt.to_dev(R)
-    kx.kx_outproj_residual_mxfp8(dev8(Xq), dev(chunked(ex, K)), dev8(Wq), dev(chunked(ew, K)), kt.to_dev(b), Rd, Y)
+    kx.kx_outproj_residual_mxfp8(dev8(Xq), dev(chunked(ex, K)), dev8(Wq), dev(chunked(ew, K)), kt.to_dev(b), Rd, Y,
+                                 override=ov)
     status_ok()
     return kt.from_dev(Y)
 
@@ -127,6 +133,23 @@ def test_mx_projection_exact_on_small_values(M, N, K):
     ex = rng.integers(126, 129, size=(M, nb), dtype=np.uint8)
     ew = rng.integers(125, 128, size=(N, nb), dtype=np.uint8)
     ok, msg = kt.gate_exact(run_proj(Xq, ex, Wq, ew), oracle.outproj_mx(Xq, ex, Wq, ew))
+    assert ok, msg
+
+
+@pytest.mark.parametrize("variant", VARIANTS)
+@pytest.mark.parametrize("M,N,K", [(128, 128, 128), (300, 520, 288), (1000, 776, 1056), (7, 64, 32), (260, 960, 384),
+                                   (2500, 3080, 416), (4096, 4096 + 192, 128)])
+def test_mx_projection_every_tile_shape(variant, M, N, K):
+    """The same exact-sum construction forced through each tile shape (single CTA / CTA pair, 128 / 192
+    columns; with 192 columns every second tile starts in the middle of a scale chunk), with bias and R."""
+    rng = np.random.default_rng(940 + M + N + K)
+    nb = K // 32
+    Xq, Wq = small_codes(941 + M, (M, K)), small_codes(942 + N, (N, K))
+    ex = rng.integers(126, 129, size=(M, nb), dtype=np.uint8)
+    ew = rng.integers(125, 128, size=(N, nb), dtype=np.uint8)
+    b = inputs.small_int_bf16(943, "bias", (N,), -4, 4)
+    R = inputs.small_int_bf16(943, "R", (M, N), -8, 8)
+    ok, msg = kt.gate_exact(run_proj(Xq, ex, Wq, ew, b, R, variant=variant), oracle.outproj_mx(Xq, ex, Wq, ew, b, R))
     assert ok, msg
 
 
@@ -217,6 +240,8 @@ def test_mx_edges_and_argument_checks():
     assert lib.kx_outproj_residual_mxfp8(*args(sx=None)) == kx.KX_ERR_NULL
     assert lib.kx_outproj_residual_mxfp8(*args(w=w.data_ptr() + 8)) == kx.KX_ERR_ALIGN
     assert lib.kx_outproj_residual_mxfp8(*args(y=x.data_ptr())) == kx.KX_ERR_OVERLAP
+    ov = kx.make_override(block_n=256)
+    assert lib.kx_outproj_residual_mxfp8_ex(*args(), ov) == kx.KX_ERR_PLAN
     A = kt.to_dev(inputs.normal_bf16(3, "X", (8, 64), 1.0))
     Q = torch.empty((8, 64), dtype=torch.uint8, device="cuda")
     SF = torch.empty((512,), dtype=torch.uint8, device="cuda")
