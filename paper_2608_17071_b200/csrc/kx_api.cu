@@ -118,10 +118,13 @@ struct MxVariant {
         BN, CTAS, ST, NB, KBS, TileCfg<BN, CTAS, ST, NB, KBS, 1>::SMEM_BYTES,                 \
             reinterpret_cast<const void*>(&kx_tile_kernel<BN, CTAS, ST, NB, 3, KBS>)          \
     }
-// (tile width, CTAs per tile, ring stages, R staging buffers, k-blocks per stage); first match = default,
-// the rest by the `stages` field of the plan override
+// (tile width, CTAs per tile, ring stages, R staging buffers, k-blocks per stage).  The planner picks among
+// the single-CTA shapes; the pair shapes are reached through the plan override only (the kernel is bound
+// by the issue rate of its one MMA lane - four K = 32 steps, two or three scale copies and a commit per
+// 128-byte k-block - and a pair does not lower that count per CTA: measured 4-9 % slower).  Stages of two
+// k-blocks were 6-12 % slower here (two-stage ring) and are not instantiated.
 const MxVariant kMxVariants[] = {KX_MX(128, 1, 5, 2, 1), KX_MX(192, 1, 4, 3, 1), KX_MX(192, 2, 5, 3, 1),
-                                 KX_MX(128, 2, 6, 2, 1), KX_MX(128, 1, 2, 2, 2), KX_MX(192, 1, 2, 3, 2)};
+                                 KX_MX(128, 2, 6, 2, 1)};
 const MxVariant* find_mx(int bn, int ctas, int stages = 0) {
     for (const auto& v : kMxVariants)
         if (v.bn == bn && v.ctas == ctas && (stages == 0 || v.stages == stages)) return &v;
@@ -1674,8 +1677,8 @@ int outproj_residual_mx(const void* Xq, const void* SFX, const void* Wq, const v
         overlaps(Y, yb, SFX, static_cast<size_t>(kx_mx_scale_bytes(M, K))) ||
         overlaps(Y, yb, SFW, static_cast<size_t>(kx_mx_scale_bytes(N, K))))
         return KX_ERR_OVERLAP;
-    // Tile shape: the candidate with the smallest estimated time = waves x columns per tile / relative
-    // tile rate (a CTA pair shares the W tile and halves the issue work per flop; measured ratios).
+    // Tile shape: the single-CTA candidate with the smallest estimated time = waves x time per k-block of a
+    // tile (measured: about 550 clocks at 128 columns, 650 at 192).
     const MxVariant* v = nullptr;
     if (ov && (ov->block_n || ov->cta_pair || ov->stages)) {
         v = find_mx(ov->block_n ? ov->block_n : 128, ov->cta_pair ? ov->cta_pair : 1, ov->stages);
@@ -1683,11 +1686,10 @@ int outproj_residual_mx(const void* Xq, const void* SFX, const void* Wq, const v
     } else {
         double best = 0.0;
         for (const auto& c : kMxVariants) {
-            const long long slots = ctx->sm_count / c.ctas;
-            const long long tiles = ((M + 128 * c.ctas - 1) / (128 * c.ctas)) * ((N + c.bn - 1) / c.bn);
-            const long long waves = (tiles + slots - 1) / slots;
-            const double rate = (c.ctas == 2 ? 1.3 : 1.0) * (c.bn == 192 ? 1.08 : 1.0);
-            const double t = static_cast<double>(waves) * c.bn / rate;
+            if (c.ctas != 1) continue;
+            const long long tiles = ((M + 127) / 128) * ((N + c.bn - 1) / c.bn);
+            const long long waves = (tiles + ctx->sm_count - 1) / ctx->sm_count;
+            const double t = static_cast<double>(waves) * (c.bn == 192 ? 650.0 : 550.0);
             if (!v || t < best) { v = &c; best = t; }
         }
     }

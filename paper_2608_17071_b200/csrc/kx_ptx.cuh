@@ -359,44 +359,11 @@ __device__ __forceinline__ uint32_t mma_kblock(uint32_t d_tmem, uint32_t a_lo, u
 __host__ __device__ constexpr uint32_t idesc_mxf8(int m, int n) {
     return (1u << 23) | (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(m >> 4) << 24);
 }
-// Shared-memory descriptor of one 128-row scale chunk (32 rows of 16 bytes, 512 contiguous bytes):
-// K-major, no swizzle, 8-row core matrices 128 bytes apart.
-__device__ __forceinline__ uint64_t smem_desc_scales(uint32_t smem_addr) {
-    const uint32_t lo = (smem_addr & 0x3FFFFu) >> 4;
-    const uint32_t hi = (128u >> 4) | (1u << 14);
-    return (static_cast<uint64_t>(hi) << 32) | lo;
-}
-// 32 rows x 16 bytes of shared memory -> 4 TMEM columns, the same data in each of the four 32-lane
-// quarters.  Ordered with the MMAs issued before and after it by the same thread.
-// With CTAS == 2 each CTA of the pair copies from its own shared memory (same offset) into its own
-// tensor memory.
-template <int CTAS>
-__device__ __forceinline__ void tmem_cp_scales(uint32_t taddr, uint64_t sdesc) {
-    if constexpr (CTAS == 1)
-        asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
-    else
-        asm volatile("tcgen05.cp.cta_group::2.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
-}
-// D[tmem] (+)= (A * scale_a) * (B * scale_b)^T, one K = 32 step; sfa / sfb = TMEM column of the scales
-template <int CTAS>
-__device__ __forceinline__ void mma_mxf8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                         uint32_t sfa, uint32_t sfb, uint32_t accumulate) {
-    if constexpr (CTAS == 1)
-        asm volatile(
-            "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-            "tcgen05.mma.cta_group::1.kind::mxf8f6f4.block_scale [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
-            ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa), "r"(sfb)
-            : "memory");
-    else
-        asm volatile(
-            "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-            "tcgen05.mma.cta_group::2.kind::mxf8f6f4.block_scale [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
-            ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa), "r"(sfb)
-            : "memory");
-}
 // One k-block (128 FP8 elements) of the block-scaled kind in a single instruction block: the scale
-// chunks (A, then CHUNKS of B, 512 bytes apart in shared memory) go to TMEM columns cols, cols + 4
-// (, cols + 8), then four K = 32 steps, step i reading byte i of the scale columns (sfb = first
+// chunks (A, then CHUNKS of B, 512 bytes apart in shared memory; each 32 rows x 16 bytes, described
+// K-major without swizzle, 8-row core matrices 128 bytes apart) are copied to TMEM columns cols,
+// cols + 4 (, cols + 8) - 4 columns each, the same data in every 32-lane quarter; with a CTA pair
+// each CTA copies from its own shared memory into its own tensor memory - then four K = 32 steps, step i reading byte i of the scale columns (sfb = first
 // scale column of the tile's B rows).  a_lo / b_lo / sf_lo are the low words of the shared-memory
 // descriptors; acc_first = 0 makes step 0 overwrite the accumulator.
 #define KX_MX_CP(G, OFFS, OFFT)                                                                            \
