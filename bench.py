@@ -616,6 +616,24 @@ def run_ours(args):
             del keep, calls
             torch.cuda.empty_cache()
 
+        for (Mn, Nn) in [(4096, 4096), (16384, 4096)]:
+            nbytes = (3.0 + 1.0 / 32) * Mn * Nn + 2.0 * Nn
+            ns = int(max(2, min(24, math.ceil(2.0 * L2_BYTES / nbytes))))
+            gam = torch.randn(Nn, device="cuda", generator=g).bfloat16()
+            sfn = torch.empty(int(lib.kx_mx_scale_bytes(i64(Mn), i64(Nn))), device="cuda", dtype=torch.uint8)
+            keep, calls = [], []
+            for _ in range(ns):
+                Hn = torch.randn(Mn, Nn, device="cuda", generator=g).bfloat16()
+                Qn = torch.empty(Mn, Nn, dtype=torch.uint8, device="cuda")
+                keep.append((Hn, Qn))
+                a = (vp(Hn.data_ptr()), vp(gam.data_ptr()), ctypes.c_float(1e-6), vp(Qn.data_ptr()), vp(sfn.data_ptr()),
+                     i64(Mn), i64(Nn), st)
+                calls.append(lambda a=a: lib.kx_rmsnorm_quantize_mxfp8(*a))
+            wlq = inputs.Workload(f"rmsnorm_quantize_mxfp8_{Mn}x{Nn}", Mn, Nn, 8, 0, False, False)
+            t, tbest, _ = time_shape(torch, kx, wlq, calls)
+            report(wlq.name, t, tbest, nbytes, 0.0, ns)
+            del keep, calls
+            torch.cuda.empty_cache()
         # block-scaled FP8: the code book (BF16 -> codes + one scale byte per 32 elements), then the projection on
         # those codes (scales stay on the device in the layout the kernel loads)
         for (Mo, No, Ko) in [(4096, 4096, 4096), (16384, 4096, 14336)]:

@@ -378,8 +378,11 @@ int kx_outproj_residual_fp8(const void* Xq, const float* sx, const void* Wq, con
  * Code book (kx_quantize_rows_mxfp8), per block of 32 BF16 values z of a row:
  *     e = clamp(floor(log2 max|z|) - 8 + 127, 0, 254)   (an all-zero block takes e = 127)
  *     q = e4m3(z / 2^(e-127))                           (exact quotient; nearest, ties to even, saturating at +-448)
- * A [rows, cols] BF16 row-major, cols % 32 == 0; Q [rows, cols] bytes; all device pointers, 16-byte
- * aligned, written by the call (Q, SF) or only read (A); no overlap.
+ * A [rows, cols] BF16 row-major, cols % 32 == 0, cols <= 32768; Q [rows, cols] bytes; all device
+ * pointers, 16-byte aligned, written by the call (Q, SF) or only read (A); no overlap.
+ * kx_rmsnorm_quantize_mxfp8 is the same code book of RMSNorm(H) * gamma (the step after the projection in
+ * the decoder layer of Appendix A, Algorithm 7, with the block-scaled format): z is rounded to BF16
+ * exactly as kx_rmsnorm would write it and never reaches memory; H [M, N], gamma [N] BF16, eps >= 0.
  *
  * Scale layout (SF of the code book, SFX / SFW of the projection): chunks of 512 bytes, one per
  * (128 rows, 128 elements of K), ordered [ceil(rows / 128)][ceil(cols / 128)]; inside a chunk the
@@ -401,6 +404,8 @@ int kx_outproj_residual_fp8(const void* Xq, const float* sx, const void* Wq, con
  */
 int64_t kx_mx_scale_bytes(int64_t rows, int64_t cols);
 int kx_quantize_rows_mxfp8(const void* A, void* Q, void* SF, int64_t rows, int64_t cols, void* stream);
+int kx_rmsnorm_quantize_mxfp8(const void* H, const void* gamma, float eps, void* Q, void* SF,
+                              int64_t M, int64_t N, void* stream);
 int kx_outproj_residual_mxfp8(const void* Xq, const void* SFX, const void* Wq, const void* SFW,
                               const void* bias_or_null, const void* R_or_null, void* Y,
                               int64_t M, int64_t N, int64_t K, void* stream);

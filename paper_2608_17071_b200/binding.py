@@ -29,7 +29,7 @@ EXPORTS = (
     "kx_outproj_residual_int8",
     "kx_quantize_rows_fp8", "kx_quantize_gate_up_fp8", "kx_rmsnorm_quantize_fp8", "kx_gate_up_swiglu_fp8",
     "kx_outproj_residual_fp8",
-    "kx_mx_scale_bytes", "kx_quantize_rows_mxfp8", "kx_outproj_residual_mxfp8", "kx_outproj_residual_mxfp8_ex",
+    "kx_mx_scale_bytes", "kx_quantize_rows_mxfp8", "kx_rmsnorm_quantize_mxfp8", "kx_outproj_residual_mxfp8", "kx_outproj_residual_mxfp8_ex",
     "kx_plan_query", "kx_last_device_status", "kx_status_string",
     "kx_version",
 )
@@ -99,6 +99,7 @@ def load():
         getattr(lib, f"kx_outproj_residual_{sfx}").argtypes = lib.kx_outproj_residual_int8.argtypes
     lib.kx_mx_scale_bytes.argtypes = [i64, i64]
     lib.kx_quantize_rows_mxfp8.argtypes = [vp, vp, vp, i64, i64, vp]
+    lib.kx_rmsnorm_quantize_mxfp8.argtypes = [vp, vp, ctypes.c_float, vp, vp, i64, i64, vp]
     lib.kx_outproj_residual_mxfp8.argtypes = [vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, vp]
     lib.kx_outproj_residual_mxfp8_ex.argtypes = [vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, vp, ctypes.POINTER(PlanOverride)]
     lib.kx_plan_query.argtypes = [i64, i64, i64, ci, ci, ctypes.POINTER(PlanOverride), ctypes.POINTER(PlanInfo)]
@@ -505,6 +506,18 @@ def kx_quantize_rows_mxfp8(A, Q, SF, stream=None, check=True) -> int:
     rc = load().kx_quantize_rows_mxfp8(_addr(A), _addr(Q), _addr(SF), rows, cols, _stream(stream))
     if check and rc != KX_OK:
         raise KxError(rc, "kx_quantize_rows_mxfp8")
+    return rc
+
+
+def kx_rmsnorm_quantize_mxfp8(H, gamma, eps: float, Q, SF, stream=None, check=True) -> int:
+    """Q, SF = block-scaled FP8 code book of RMSNorm(H) * gamma (rounded to BF16 as kx_rmsnorm would), H read once."""
+    import torch
+    M, N = H.shape
+    _check_bf16("H", H, (M, N)); _check_bf16("gamma", gamma, (N,)); _check("Q", Q, (M, N), torch.float8_e4m3fn)
+    _check("SF", SF, (kx_mx_scale_bytes(M, N),), torch.uint8)
+    rc = load().kx_rmsnorm_quantize_mxfp8(_addr(H), _addr(gamma), float(eps), _addr(Q), _addr(SF), M, N, _stream(stream))
+    if check and rc != KX_OK:
+        raise KxError(rc, "kx_rmsnorm_quantize_mxfp8")
     return rc
 
 

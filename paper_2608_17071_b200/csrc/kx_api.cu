@@ -1278,7 +1278,7 @@ int kx_outproj_residual_rmsnorm(const void* X, const void* W, const void* bias, 
 namespace {
 bool aligned4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3u) == 0; }
 
-// fmt: 0 = INT8 codes, 1 = FP8 E4M3 codes
+// fmt: 0 = INT8 codes, 1 = FP8 E4M3 codes (one scale per row); 2 = FP8 E4M3 codes with one E8M0 scale per 32 elements
 int launch_rowquant(const QuantParams& qp, bool norm, int fmt, cudaStream_t stream, int sm_count) {
     cudaLaunchConfig_t cfg;
     std::memset(&cfg, 0, sizeof cfg);
@@ -1286,10 +1286,12 @@ int launch_rowquant(const QuantParams& qp, bool norm, int fmt, cudaStream_t stre
     const void* fn = nullptr;
     int per_sm = 8;
 #define KX_QUANT_FN(NV)                                                                              \
-    (fmt == 1 ? (norm ? reinterpret_cast<const void*>(&kx_rowquant_kernel<NV, true, 1>)              \
-                      : reinterpret_cast<const void*>(&kx_rowquant_kernel<NV, false, 1>))            \
-              : (norm ? reinterpret_cast<const void*>(&kx_rowquant_kernel<NV, true, 0>)              \
-                      : reinterpret_cast<const void*>(&kx_rowquant_kernel<NV, false, 0>)))
+    (fmt == 2 ? (norm ? reinterpret_cast<const void*>(&kx_rowquant_kernel<NV, true, 2>)              \
+                      : reinterpret_cast<const void*>(&kx_rowquant_kernel<NV, false, 2>))            \
+     : fmt == 1 ? (norm ? reinterpret_cast<const void*>(&kx_rowquant_kernel<NV, true, 1>)            \
+                        : reinterpret_cast<const void*>(&kx_rowquant_kernel<NV, false, 1>))          \
+                : (norm ? reinterpret_cast<const void*>(&kx_rowquant_kernel<NV, true, 0>)            \
+                        : reinterpret_cast<const void*>(&kx_rowquant_kernel<NV, false, 0>)))
     if (nvec <= 1 * kNormThreads) { fn = KX_QUANT_FN(1); }
     else if (nvec <= 2 * kNormThreads) { fn = KX_QUANT_FN(2); }
     else if (nvec <= 4 * kNormThreads) { fn = KX_QUANT_FN(4); per_sm = 6; }
@@ -1607,44 +1609,45 @@ int64_t kx_mx_scale_bytes(int64_t rows, int64_t cols) {
     return mx_chunks(rows) * mx_chunks(cols) * 512;
 }
 
-int kx_quantize_rows_mxfp8(const void* A, void* Q, void* SF, int64_t rows, int64_t cols, void* stream) {
-    if (rows < 0 || cols < 0 || rows > 0x7FFFFFFFll / 2 || cols > 0x7FFFFFFFll / 2) return KX_ERR_SHAPE;
-    if ((cols % 32) != 0) return KX_ERR_SHAPE;
+namespace {
+// H [rows, cols] BF16 (optionally RMS-normalised with gamma first) -> E4M3 codes + chunked E8M0 scale bytes
+int quantize_rows_mx(const void* H, const void* gamma, float eps, void* Q, void* SF, int64_t rows, int64_t cols,
+                     void* stream) {
+    if (rows < 0 || cols < 0 || rows > 0x7FFFFFFFll / 2) return KX_ERR_SHAPE;
+    if ((cols % 32) != 0 || cols > 8ll * kNormThreads * kNormVecs) return KX_ERR_SHAPE;
+    if (gamma && !(eps >= 0.0f)) return KX_ERR_SHAPE;
     if (rows == 0 || cols == 0) return KX_OK;
-    if (!A || !Q || !SF) return KX_ERR_NULL;
-    if (!aligned16(A) || !aligned16(Q) || !aligned16(SF)) return KX_ERR_ALIGN;
-    const size_t ab = static_cast<size_t>(rows) * cols * 2, qb = static_cast<size_t>(rows) * cols,
-                 sb = static_cast<size_t>(kx_mx_scale_bytes(rows, cols));
-    if (overlaps(Q, qb, A, ab) || overlaps(SF, sb, A, ab) || overlaps(SF, sb, Q, qb)) return KX_ERR_OVERLAP;
+    if (!H || !Q || !SF) return KX_ERR_NULL;
+    if (!aligned16(H) || !aligned16(Q) || !aligned16(SF) || (gamma && !aligned16(gamma))) return KX_ERR_ALIGN;
+    const size_t hb = static_cast<size_t>(rows) * cols * 2, qb = static_cast<size_t>(rows) * cols,
+                 sb = static_cast<size_t>(kx_mx_scale_bytes(rows, cols)), gb = static_cast<size_t>(cols) * 2;
+    if (overlaps(Q, qb, H, hb) || overlaps(SF, sb, H, hb) || overlaps(SF, sb, Q, qb)) return KX_ERR_OVERLAP;
+    if (gamma && (overlaps(Q, qb, gamma, gb) || overlaps(SF, sb, gamma, gb))) return KX_ERR_OVERLAP;
     DeviceCtx* ctx = nullptr;
     int rc = device_ctx(&ctx);
     if (rc != KX_OK) return rc;
-    MxQuantParams p;
-    std::memset(&p, 0, sizeof p);
-    p.A = static_cast<const uint16_t*>(A);
-    p.Q = static_cast<uint8_t*>(Q);
-    p.SF = static_cast<uint8_t*>(SF);
-    p.rows = rows;
-    p.rows_pad = mx_chunks(rows) * 128;
-    p.cols = static_cast<int>(cols);
-    p.kchunks = static_cast<int>(mx_chunks(cols));
-    const long long total = p.rows_pad * p.kchunks * 16;
-    cudaLaunchConfig_t cfg;
-    std::memset(&cfg, 0, sizeof cfg);
-    cfg.gridDim = dim3(static_cast<unsigned>(std::min<long long>((total + 255) / 256, ctx->sm_count * 16ll)), 1, 1);
-    cfg.blockDim = dim3(256, 1, 1);
-    cfg.stream = static_cast<cudaStream_t>(stream);
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    void* args[] = {&p};
-    if (cudaLaunchKernelExC(&cfg, reinterpret_cast<const void*>(&kx_mxquant_kernel), args) != cudaSuccess) {
-        cudaGetLastError();
-        return KX_ERR_CUDA;
-    }
-    return KX_OK;
+    QuantParams qp;
+    std::memset(&qp, 0, sizeof qp);
+    qp.A0 = qp.A1 = static_cast<const uint16_t*>(H);
+    qp.gamma = static_cast<const uint16_t*>(gamma);
+    qp.Q0 = qp.Q1 = static_cast<int8_t*>(Q);
+    qp.SF0 = static_cast<uint8_t*>(SF);
+    qp.rows0 = rows;
+    qp.M = rows;
+    qp.N = static_cast<int>(cols);
+    qp.kchunks = static_cast<int>(mx_chunks(cols));
+    qp.eps = eps;
+    return launch_rowquant(qp, gamma != nullptr, 2, static_cast<cudaStream_t>(stream), ctx->sm_count);
+}
+}  // namespace
+
+int kx_quantize_rows_mxfp8(const void* A, void* Q, void* SF, int64_t rows, int64_t cols, void* stream) {
+    return quantize_rows_mx(A, nullptr, 0.0f, Q, SF, rows, cols, stream);
+}
+int kx_rmsnorm_quantize_mxfp8(const void* H, const void* gamma, float eps, void* Q, void* SF, int64_t M, int64_t N,
+                              void* stream) {
+    if (M > 0 && N > 0 && !gamma) return KX_ERR_NULL;
+    return quantize_rows_mx(H, gamma, eps, Q, SF, M, N, stream);
 }
 
 namespace {

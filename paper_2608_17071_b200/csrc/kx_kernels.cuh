@@ -1471,6 +1471,12 @@ kx_rmsnorm_kernel(const uint16_t* __restrict__ H, const uint16_t* __restrict__ g
 // Rows [0, rows0) come from A0 -> Q0 / S0, rows [rows0, M) from A1 -> Q1 / S1, so that two
 // matrices of the same width (gate and up weights) are quantised by one launch.
 // HBM-bound: 2 N bytes read, N + 4 written per row.
+// FMT 2: block-scaled FP8 instead - one E8M0 scale byte per 32 consecutive elements (four neighbouring
+// threads), e = max(exponent field of the block maximum - 8, 0) (127 for an all-zero block), code =
+// e4m3(z * 2^(127 - e)) (exact product, so the conversion's rounding is the only one); no row-wide
+// maximum.  Scale bytes go to SF0 in 512-byte chunks, chunk (row / 128, k / 128), byte
+// (row % 32) * 16 + (row % 128) / 32 * 4 + (k / 32) % 4; entries of blocks past the row end and of the
+// rows up to the next multiple of 128 are padding and are set to 127.  One matrix per launch.
 struct QuantParams {
     const uint16_t* A0;
     const uint16_t* A1;
@@ -1479,8 +1485,10 @@ struct QuantParams {
     int8_t* Q1;
     float* S0;
     float* S1;
+    uint8_t* SF0;          // FMT 2: chunked scale bytes
     long long rows0, M;
     int N;
+    int kchunks;           // FMT 2: ceil(N / 128)
     float eps;
 };
 
@@ -1546,6 +1554,51 @@ kx_rowquant_kernel(const QuantParams p) {
                 }
             }
         }
+        if constexpr (FMT == 2) {
+            uint2* qrow = reinterpret_cast<uint2*>(p.Q0 + r * N);
+            uint8_t* const sfrow = p.SF0 + (r >> 7) * p.kchunks * 512 + (r & 31) * 16 + ((r & 127) >> 5) * 4;
+            const int nb = N >> 5;
+#pragma unroll
+            for (int i = 0; i < NV; ++i) {
+                const int idx = tid + i * kNormThreads;
+                const bool valid = idx < nvec;
+                const uint32_t w4[4] = {valid ? v[i].x : 0u, valid ? v[i].y : 0u, valid ? v[i].z : 0u, valid ? v[i].w : 0u};
+                float z[8], bmax = 0.f;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    z[2 * k] = bf16_lo(w4[k]);
+                    z[2 * k + 1] = bf16_hi(w4[k]);
+                    bmax = fmaxf(bmax, fmaxf(fabsf(z[2 * k]), fabsf(z[2 * k + 1])));
+                }
+                // N % 32 == 0: the four threads of a block are all valid or all invalid, and sit in one warp
+                bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, 1));
+                bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, 2));
+                if (valid) {
+                    const int field = static_cast<int>(__float_as_uint(bmax) >> 23);
+                    const int e = (bmax > 0.f) ? max(field - 8, 0) : 127;
+                    const float mult = __uint_as_float(static_cast<uint32_t>(254 - e) << 23);   // 2^(127 - e), e <= 247
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) z[k] = __fmul_rn(z[k], mult);
+                    qrow[idx] = make_uint2(pack_e4m3x4(z[0], z[1], z[2], z[3]), pack_e4m3x4(z[4], z[5], z[6], z[7]));
+                    if ((tid & 3) == 0) {
+                        const int j = idx >> 2;
+                        sfrow[(j >> 2) * 512 + (j & 3)] = static_cast<uint8_t>(e);
+                        if (j == nb - 1)                     // blocks past the row end inside the last chunk
+                            for (int jj = nb; jj < p.kchunks * 4; ++jj) sfrow[(jj >> 2) * 512 + (jj & 3)] = 127;
+                    }
+                }
+            }
+            if (r == p.M - 1) {                              // rows up to the next multiple of 128
+                const long long pad_rows = ((p.M + 127) & ~127ll) - p.M;
+                const int per_row = p.kchunks * 4;
+                for (long long t = tid; t < pad_rows * per_row; t += kNormThreads) {
+                    const long long rr = p.M + t / per_row;
+                    const int jj = static_cast<int>(t % per_row);
+                    p.SF0[((rr >> 7) * p.kchunks + (jj >> 2)) * 512 + (rr & 31) * 16 + ((rr & 127) >> 5) * 4 + (jj & 3)] = 127;
+                }
+            }
+            continue;
+        }
         // row maximum of |z| (exact: BF16 values, compared as binary32)
         float amax = 0.f;
 #pragma unroll
@@ -1596,62 +1649,6 @@ kx_rowquant_kernel(const QuantParams p) {
             }
         }
         __syncthreads();         // s_part / s_bcast are reused by the next row
-    }
-}
-
-// ===========================================================================
-// kx_mxquant_kernel: BF16 rows -> block-scaled FP8 (E4M3 codes, one E8M0 scale per 32 elements)
-// ===========================================================================
-// Four threads share a 32-element block (8 elements each).  Scale byte e = max(exponent field of
-// max|z| - 8, 0) (127 for an all-zero block), code = e4m3(z * 2^(127 - e)): the product is exact, so
-// the conversion instruction's rounding is the only one.  Scales are written in the chunked layout
-// the tile kernel loads: chunk (row / 128, k / 128) = 512 bytes, byte (row % 32) * 16 +
-// (row % 128) / 32 * 4 + (k / 32) % 4; entries of rows and blocks outside the matrix are set to 127.
-struct MxQuantParams {
-    const uint16_t* A;
-    uint8_t* Q;
-    uint8_t* SF;
-    long long rows, rows_pad;
-    int cols, kchunks;
-};
-
-__global__ void __launch_bounds__(256) kx_mxquant_kernel(const MxQuantParams p) {
-    pdl_wait_prior();
-    pdl_launch_dependents();
-    const int qpr = p.kchunks * 16;                       // 8-element groups per padded row
-    const long long total = p.rows_pad * qpr;             // a multiple of 32: warps stay whole
-    const long long step = static_cast<long long>(gridDim.x) * blockDim.x;
-    for (long long it = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; it < total; it += step) {
-        const long long r = it / qpr;
-        const int rem = static_cast<int>(it - r * qpr);
-        const int j = rem >> 2, k = rem * 8;
-        const bool in = (r < p.rows) && (k < p.cols);
-        uint4 v = make_uint4(0u, 0u, 0u, 0u);
-        if (in) v = *reinterpret_cast<const uint4*>(p.A + r * p.cols + k);
-        const uint32_t w4[4] = {v.x, v.y, v.z, v.w};
-        float z[8], amax = 0.f;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            z[2 * i] = bf16_lo(w4[i]);
-            z[2 * i + 1] = bf16_hi(w4[i]);
-            amax = fmaxf(amax, fmaxf(fabsf(z[2 * i]), fabsf(z[2 * i + 1])));
-        }
-        amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
-        amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
-        const int field = static_cast<int>(__float_as_uint(amax) >> 23);
-        const int e = (amax > 0.f) ? max(field - 8, 0) : 127;
-        const float mult = __uint_as_float(static_cast<uint32_t>(254 - e) << 23);      // 2^(127 - e), e <= 247
-        if (in) {
-#pragma unroll
-            for (int i = 0; i < 8; ++i) z[i] = __fmul_rn(z[i], mult);
-            *reinterpret_cast<uint2*>(p.Q + r * p.cols + k) =
-                make_uint2(pack_e4m3x4(z[0], z[1], z[2], z[3]), pack_e4m3x4(z[4], z[5], z[6], z[7]));
-        }
-        if ((rem & 3) == 0) {
-            const long long chunk = (r >> 7) * p.kchunks + (j >> 2);
-            const int off = static_cast<int>(r & 31) * 16 + static_cast<int>((r & 127) >> 5) * 4 + (j & 3);
-            p.SF[chunk * 512 + off] = static_cast<uint8_t>(in ? e : 127);
-        }
     }
 }
 

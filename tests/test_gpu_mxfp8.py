@@ -78,6 +78,23 @@ def test_mx_code_book_bit_exact(rows, cols):
     assert np.array_equal(SF, chunked(Er, cols))
 
 
+@pytest.mark.parametrize("M,N", [(130, 4096), (1000, 5120), (9, 32768), (300, 1056), (5, 32)])
+def test_mx_rmsnorm_code_book(M, N):
+    """Fused RMSNorm + code book = code book of the device's own BF16 RMSNorm output, bit for bit."""
+    H = inputs.normal_bf16(950 + N, "R", (M, N), 1.3)
+    g = inputs.normal_bf16(950 + N, "bias", (N,), 1.0)
+    Z = kt.nan_filled(M, N)
+    kx.kx_rmsnorm(kt.to_dev(H), kt.to_dev(g), 1e-6, Z)
+    Q = torch.full((M, N), 0x55, dtype=torch.uint8, device="cuda").view(F8)
+    SF = torch.full((kx.kx_mx_scale_bytes(M, N),), 0xEE, dtype=torch.uint8, device="cuda")
+    kx.kx_rmsnorm_quantize_mxfp8(kt.to_dev(H), kt.to_dev(g), 1e-6, Q, SF)
+    Qr, Er = oracle.quantize_rows_mx(kt.from_dev(Z))
+    assert np.array_equal(host8(Q), Qr) and np.array_equal(SF.cpu().numpy(), chunked(Er, N))
+    # and the RMSNorm itself is the oracle's within BF16 rounding (its own parity is tested elsewhere)
+    ref = oracle.rmsnorm(H, g, 1e-6)
+    assert kt.rel_fro(kt.from_dev(Z), ref) <= 2.0 ** -8
+
+
 def test_mx_code_book_grid_and_saturation():
     vals = oracle.e4m3_decode(np.arange(0x5F, 0x7F, dtype=np.uint8))
     d = oracle.e4m3_decode(np.arange(0x40, 0x7F, dtype=np.uint8))
@@ -249,4 +266,6 @@ def test_mx_edges_and_argument_checks():
     assert lib.kx_quantize_rows_mxfp8(A.data_ptr(), None, SF.data_ptr(), 8, 64, None) == kx.KX_ERR_NULL
     assert lib.kx_quantize_rows_mxfp8(A.data_ptr(), A.data_ptr(), SF.data_ptr(), 8, 64, None) == kx.KX_ERR_OVERLAP
     assert lib.kx_quantize_rows_mxfp8(A.data_ptr(), Q.data_ptr(), SF.data_ptr(), 0, 64, None) == kx.KX_OK
+    assert lib.kx_quantize_rows_mxfp8(A.data_ptr(), Q.data_ptr(), SF.data_ptr(), 1, 32768 + 32, None) == kx.KX_ERR_SHAPE
+    assert lib.kx_rmsnorm_quantize_mxfp8(A.data_ptr(), None, 1e-6, Q.data_ptr(), SF.data_ptr(), 8, 64, None) == kx.KX_ERR_NULL
     status_ok()
