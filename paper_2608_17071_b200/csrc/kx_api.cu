@@ -122,9 +122,11 @@ struct MxVariant {
 // the single-CTA shapes; the pair shapes are reached through the plan override only (the kernel is bound
 // by the issue rate of its one MMA lane - four K = 32 steps, two or three scale copies and a commit per
 // 128-byte k-block - and a pair does not lower that count per CTA: measured 4-9 % slower).  Stages of two
-// k-blocks were 6-12 % slower here (two-stage ring) and are not instantiated.
-const MxVariant kMxVariants[] = {KX_MX(128, 1, 5, 2, 1), KX_MX(192, 1, 4, 3, 1), KX_MX(192, 2, 5, 3, 1),
-                                 KX_MX(128, 2, 6, 2, 1)};
+// k-blocks were 6-12 % slower here (two-stage ring) and are not instantiated.  The 256-column shape has a
+// single accumulator buffer (two would fill tensor memory), so its epilogue is not hidden behind the next
+// tile's MMAs; it still wins when K is long because every MMA does a third more work.
+const MxVariant kMxVariants[] = {KX_MX(128, 1, 5, 2, 1), KX_MX(192, 1, 4, 3, 1), KX_MX(256, 1, 4, 1, 1),
+                                 KX_MX(192, 2, 5, 3, 1), KX_MX(128, 2, 6, 2, 1)};
 const MxVariant* find_mx(int bn, int ctas, int stages = 0) {
     for (const auto& v : kMxVariants)
         if (v.bn == bn && v.ctas == ctas && (stages == 0 || v.stages == stages)) return &v;
@@ -1680,8 +1682,9 @@ int outproj_residual_mx(const void* Xq, const void* SFX, const void* Wq, const v
         overlaps(Y, yb, SFX, static_cast<size_t>(kx_mx_scale_bytes(M, K))) ||
         overlaps(Y, yb, SFW, static_cast<size_t>(kx_mx_scale_bytes(N, K))))
         return KX_ERR_OVERLAP;
-    // Tile shape: the single-CTA candidate with the smallest estimated time = waves x time per k-block of a
-    // tile (measured: about 550 clocks at 128 columns, 650 at 192).
+    // Tile shape: the single-CTA candidate with the smallest estimated time = waves x (k-blocks x time per
+    // k-block + exposed epilogue), with the measured 0.375 / 0.443 / 0.519 us per k-block at 128 / 192 / 256
+    // columns and 2.7 us of epilogue per tile that the single-accumulator 256-column shape cannot hide.
     const MxVariant* v = nullptr;
     if (ov && (ov->block_n || ov->cta_pair || ov->stages)) {
         v = find_mx(ov->block_n ? ov->block_n : 128, ov->cta_pair ? ov->cta_pair : 1, ov->stages);
@@ -1692,7 +1695,8 @@ int outproj_residual_mx(const void* Xq, const void* SFX, const void* Wq, const v
             if (c.ctas != 1) continue;
             const long long tiles = ((M + 127) / 128) * ((N + c.bn - 1) / c.bn);
             const long long waves = (tiles + ctx->sm_count - 1) / ctx->sm_count;
-            const double t = static_cast<double>(waves) * (c.bn == 192 ? 650.0 : 550.0);
+            const double per_kb = c.bn == 256 ? 0.519 : c.bn == 192 ? 0.443 : 0.375;
+            const double t = static_cast<double>(waves) * (static_cast<double>((K + 127) / 128) * per_kb + (c.bn == 256 ? 2.7 : 0.0));
             if (!v || t < best) { v = &c; best = t; }
         }
     }

@@ -167,8 +167,10 @@ struct TileCfg {
     static constexpr int SF_KB_BYTES = MX ? 512 * (1 + SFB_CHUNKS) : 0;     // scale bytes per k-block
     static constexpr int SF_STAGE = KBS * SF_KB_BYTES;
     static constexpr int SMEM_BYTES = 1024 + STAGES * (STAGE_BYTES + SF_STAGE) + EPI_BYTES + 1024;
-    static constexpr int TMEM_COLS = tmem_cols_for(2 * BN + (MX ? 48 : 0));
-    static_assert(!MX || BN <= 192, "block-scaled variants: two accumulators and the scale columns share TMEM");
+    // accumulator buffers in tensor memory: two, so that the epilogue of one tile overlaps the MMAs of the
+    // next - except the 256-column block-scaled tile, where two would leave no room for the scale columns
+    static constexpr int ACC_BUFS = (MX && BN > 192) ? 1 : 2;
+    static constexpr int TMEM_COLS = tmem_cols_for(ACC_BUFS * BN + (MX ? 48 : 0));
     static_assert(SMEM_BYTES <= 232448, "shared memory");
     static constexpr int CHUNKS = BN / 64;                  // 64-column epilogue chunks per tile
     static constexpr int PART_FLOATS = 128 * BN;            // one CTA's FP32 partial of one tile
@@ -455,7 +457,8 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             bool ok = true;
             bool have = false;   // the current stage was already seen full by the previous k-block's early test
             while (ok && it.next(tile, kb0, kb1)) {
-                const uint32_t b = scount & 1u, aph = (scount >> 1) & 1u;
+                const uint32_t b = (C::ACC_BUFS == 2) ? (scount & 1u) : 0u;
+                const uint32_t aph = (C::ACC_BUFS == 2) ? ((scount >> 1) & 1u) : (scount & 1u);
                 const uint32_t idesc = (tile >= p.narrow_tile0) ? idesc_narrow : idesc_wide;
                 ++scount;
                 KX_TRACE_POINT(p, slot, (scount - 1) * 4 + 0);
@@ -476,7 +479,7 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         const int nsub = (KBS == 2 && kb + 1 < kb1) ? 2 : 1;
                         const uint32_t sf0 = s_sf + s * C::SF_STAGE;
                         for (int j = 0; j < nsub; ++j) {
-                            const uint32_t cols = tmem_base + 2 * BN + (mx_set & 3u) * 12u;
+                            const uint32_t cols = tmem_base + C::ACC_BUFS * BN + (mx_set & 3u) * 12u;
                             ++mx_set;
                             const uint32_t sf = sf0 + j * C::SF_KB_BYTES;
                             const uint32_t al = a_lo + j * (kABytes >> 4);
@@ -588,7 +591,8 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         };
 
         while (ok && it.next(tile, kb0, kb1)) {
-            const uint32_t b = scount & 1u, aph = (scount >> 1) & 1u;
+            const uint32_t b = (C::ACC_BUFS == 2) ? (scount & 1u) : 0u;
+            const uint32_t aph = (C::ACC_BUFS == 2) ? ((scount >> 1) & 1u) : (scount & 1u);
             ++scount;
             int tm, colbase;
             bool narrow;

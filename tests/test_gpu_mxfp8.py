@@ -118,7 +118,7 @@ def small_codes(seed, shape):
 
 
 # (tile columns, CTAs per tile, ring stages: 0 = default variant)
-VARIANTS = [(128, 1, 0), (192, 1, 0), (128, 2, 0), (192, 2, 0)]
+VARIANTS = [(128, 1, 0), (192, 1, 0), (128, 2, 0), (192, 2, 0), (256, 1, 0)]
 
 
 def run_proj(Xq, ex, Wq, ew, b=None, R=None, inplace=False, variant=None):
@@ -257,7 +257,7 @@ def test_mx_edges_and_argument_checks():
     assert lib.kx_outproj_residual_mxfp8(*args(sx=None)) == kx.KX_ERR_NULL
     assert lib.kx_outproj_residual_mxfp8(*args(w=w.data_ptr() + 8)) == kx.KX_ERR_ALIGN
     assert lib.kx_outproj_residual_mxfp8(*args(y=x.data_ptr())) == kx.KX_ERR_OVERLAP
-    ov = kx.make_override(block_n=256)
+    ov = kx.make_override(block_n=64)
     assert lib.kx_outproj_residual_mxfp8_ex(*args(), ov) == kx.KX_ERR_PLAN
     A = kt.to_dev(inputs.normal_bf16(3, "X", (8, 64), 1.0))
     Q = torch.empty((8, 64), dtype=torch.uint8, device="cuda")
