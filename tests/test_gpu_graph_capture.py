@@ -114,3 +114,48 @@ def test_capture_and_replay_the_int8_branch():
     assert ok, msg
     ok, msg = kt.gate_a(want[11], oracle.outproj_fp8(want[7], want[8], want[9], want[10]))
     assert ok, msg
+
+
+def test_capture_and_replay_the_block_scaled_branch():
+    """RMSNorm + block-scaled code book -> weights' code book -> block-scaled projection with residual,
+    captured and replayed: same bits as the eager run (no allocation or host work in the calls)."""
+    import torch
+    kx.kx_init(torch.cuda.current_device())
+    M, N, K = 384, 1160, 1024
+    H = kt.to_dev(inputs.normal_bf16(521, "R", (M, K), 1.0))
+    g = kt.to_dev(inputs.normal_bf16(521, "bias", (K,), 1.0))
+    W = kt.to_dev(inputs.normal_bf16(522, "W", (N, K), 1.0 / np.sqrt(K)))
+    R = kt.to_dev(inputs.normal_bf16(523, "R", (M, N), 1.0))
+    f8 = lambda *shape: torch.zeros(shape, dtype=torch.uint8, device="cuda").view(torch.float8_e4m3fn)
+    u8 = lambda n: torch.zeros((n,), dtype=torch.uint8, device="cuda")
+
+    def branch(Xq, SFX, Wq, SFW, Y):
+        kx.kx_rmsnorm_quantize_mxfp8(H, g, 1e-6, Xq, SFX)
+        kx.kx_quantize_rows_mxfp8(W, Wq, SFW)
+        kx.kx_outproj_residual_mxfp8(Xq, SFX, Wq, SFW, None, R, Y)
+
+    def bufs():
+        return [f8(M, K), u8(kx.kx_mx_scale_bytes(M, K)), f8(N, K), u8(kx.kx_mx_scale_bytes(N, K)), kt.nan_filled(M, N)]
+
+    raw = lambda t: kt.from_dev(t) if t.dtype == torch.bfloat16 else t.view(torch.uint8).cpu().numpy()
+    eager = bufs()
+    branch(*eager)
+    assert kx.kx_last_device_status()[0] == kx.KX_OK
+    want = [raw(t) for t in eager]
+    outs = bufs()
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(s):
+        branch(*outs)
+        torch.cuda.synchronize()
+        with torch.cuda.graph(graph, stream=s):
+            branch(*outs)
+    for rep in range(2):
+        for t in outs:
+            t.zero_() if t.dtype == torch.bfloat16 else t.view(torch.uint8).zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert kx.kx_last_device_status()[0] == kx.KX_OK
+        for got, ref in zip(outs, want):
+            assert np.array_equal(raw(got), ref)

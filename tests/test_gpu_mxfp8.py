@@ -170,6 +170,28 @@ def test_mx_projection_every_tile_shape(variant, M, N, K):
     assert ok, msg
 
 
+@pytest.mark.parametrize("chunk", range(4))
+def test_mx_random_shapes_and_tile_shapes_are_exact(chunk):
+    """Seeded random (M, N, K, tile shape, bias / residual / in place) cases of the exact-sum construction."""
+    rng = np.random.default_rng(9600 + chunk)
+    for case in range(12):
+        M = int(rng.choice([1, 5, 64, 127, 128, 129, 200, 256, 300, 513, 700, 1024]))
+        N = 8 * int(rng.integers(1, 160))
+        K = 32 * int(rng.integers(1, 40))
+        variant = VARIANTS[int(rng.integers(0, len(VARIANTS)))] if rng.integers(0, 4) else None
+        nb = K // 32
+        Xq, Wq = small_codes(rng.integers(1 << 30), (M, K)), small_codes(rng.integers(1 << 30), (N, K))
+        ex = rng.integers(126, 129, size=(M, nb), dtype=np.uint8)
+        ew = rng.integers(125, 128, size=(N, nb), dtype=np.uint8)
+        b = inputs.small_int_bf16(961 + case, "bias", (N,), -4, 4) if rng.integers(0, 2) else None
+        R = inputs.small_int_bf16(962 + case, "R", (M, N), -8, 8) if rng.integers(0, 2) else None
+        inplace = R is not None and bool(rng.integers(0, 2))
+        ref = oracle.outproj_mx(Xq, ex, Wq, ew, b, R)
+        y = run_proj(Xq, ex, Wq, ew, b, R.copy() if inplace else R, inplace=inplace, variant=variant)
+        ok, msg = kt.gate_exact(y, ref)
+        assert ok, (M, N, K, variant, b is not None, R is not None, inplace, msg)
+
+
 def test_mx_projection_exact_with_small_integer_epilogue():
     M, N, K = 600, 776, 96
     vals = np.array([0x00, 0x38, 0xB8], dtype=np.uint8)                     # 0, +-1
