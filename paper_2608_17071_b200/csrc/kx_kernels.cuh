@@ -622,7 +622,9 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             int n_iss = 0;                                 // R chunks requested so far (warp-uniform)
             if (lane == 0) tma_store_wait_read<0>();       // staging buffers of the previous tile are free
             if (spec_r) {
-                const int pre = (NB - 1 < nchunks) ? NB - 1 : nchunks;
+                // (a single buffer is free at this point too: the previous tile's stores were waited for above)
+                const int pre0 = (NB > 1) ? NB - 1 : 1;
+                const int pre = (pre0 < nchunks) ? pre0 : nchunks;
                 for (; n_iss < pre; ++n_iss)
                     if (lane == 0) issue_r(n_iss);
             }
@@ -905,7 +907,9 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     if (lane == 0) {
                         tma_store_2d(&tmY, col0, row0, buf);
                         tma_store_commit();
-                        tma_store_wait_read<1>();          // the store before this one has left its buffer
+                        // the store before this one has left its buffer (with a single buffer: this store itself,
+                        // because the next R slab is requested into the buffer it reads)
+                        tma_store_wait_read<(NB > 1) ? 1 : 0>();
                     }
                 } else if (lane == 0) {
                     tma_store_wait_read<0>();              // nothing stored for this chunk: drain the last store
