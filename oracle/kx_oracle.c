@@ -570,3 +570,111 @@ int kx_oracle_outproj_mx_rows(const uint8_t* Xq, const uint8_t* ex, const uint8_
     }
     return 0;
 }
+
+/*
+ * 4-bit block-scaled format ("NVFP4", the format of the paper's Section 4.3 task): E2M1 elements
+ * (sign, 2 exponent bits with bias 1, 1 mantissa bit: magnitudes 0, 0.5, 1, 1.5, 2, 3, 4, 6), two per
+ * byte (the element with the even k index in the low nibble), one E4M3 scale byte per 16 consecutive
+ * elements of a row, and one binary32 scale gs for the whole tensor:
+ *     value = e2m1(q) * e4m3(s) * gs.
+ * The paper prints no conversion; the code book below is this build's reading, every step in binary32:
+ *     a  = max |z| over the block
+ *     s  = e4m3( a / (6 gs) )                  (nearest, ties to even, saturating at 448)
+ *     r  = 1 / (e4m3_value(s) * gs)            (codes are all zero when s decodes to zero)
+ *     q  = e2m1( z * r )                       (nearest, ties to the even code, saturating at 6)
+ */
+static double e2m1_decode(uint8_t nib) {
+    const int s = (nib >> 3) & 1, e = (nib >> 1) & 3, m = nib & 1;
+    const double v = (e == 0) ? 0.5 * m : ldexp(1.0 + 0.5 * m, e - 1);
+    return s ? -v : v;
+}
+
+static uint8_t e2m1_encode(float x) {
+    static const float grid[8] = {0.0f, 0.5f, 1.0f, 1.5f, 2.0f, 3.0f, 4.0f, 6.0f};
+    const uint8_t s = signbit(x) ? 8 : 0;
+    if (isnan(x)) return 7;                               /* no NaN code: the largest magnitude */
+    const float ax = fabsf(x);
+    if (ax >= 6.0f) return s | 7;
+    int best = 0;
+    for (int c = 1; c < 8; ++c) {
+        const float dc = fabsf(grid[c] - ax), db = fabsf(grid[best] - ax);      /* exact differences */
+        if (dc < db || (dc == db && (c & 1) == 0)) best = c;
+    }
+    return s | (uint8_t)best;
+}
+
+int kx_oracle_e2m1_decode(const uint8_t* in, double* out, int64_t n) {
+    if (n < 0 || (n > 0 && (!in || !out))) return -1;
+    for (int64_t i = 0; i < n; ++i) out[i] = e2m1_decode(in[i] & 15);
+    return 0;
+}
+
+int kx_oracle_e2m1_encode(const float* in, uint8_t* out, int64_t n) {
+    if (n < 0 || (n > 0 && (!in || !out))) return -1;
+    for (int64_t i = 0; i < n; ++i) out[i] = e2m1_encode(in[i]);
+    return 0;
+}
+
+/* Z [rows, cols] BF16 (cols even) -> Q [rows, cols / 2] packed nibbles, S [rows, ceil(cols / 16)] E4M3 bytes. */
+int kx_oracle_quantize_rows_nvfp4(const uint16_t* Z, int64_t rows, int64_t cols, float gs, uint8_t* Q, uint8_t* S) {
+    if (rows < 0 || cols < 0 || (cols & 1) || !(gs > 0.0f) || (rows > 0 && cols > 0 && (!Z || !Q || !S))) return -1;
+    const int64_t nb = (cols + 15) / 16;
+#pragma omp parallel for schedule(static)
+    for (int64_t r = 0; r < rows; ++r) {
+        for (int64_t j = 0; j < nb; ++j) {
+            const int64_t k0 = j * 16, k1 = (k0 + 16 < cols) ? k0 + 16 : cols;
+            float a = 0.0f;
+            for (int64_t k = k0; k < k1; ++k) {
+                const float v = fabsf((float)bf16_widen(Z[r * cols + k]));
+                if (v > a) a = v;
+            }
+            const float d6 = 6.0f * gs;                    /* one binary32 product */
+            const uint8_t sb = e4m3_encode(a / d6);        /* one binary32 division, then the E4M3 rounding */
+            S[r * nb + j] = sb;
+            const float sd = (float)e4m3_decode(sb);
+            const float dq = sd * gs;                      /* binary32 product */
+            const float rcp = (dq > 0.0f) ? 1.0f / dq : 0.0f;
+            for (int64_t k = k0; k < k1; k += 2) {
+                const float z0 = (float)bf16_widen(Z[r * cols + k]), z1 = (float)bf16_widen(Z[r * cols + k + 1]);
+                const uint8_t q0 = (dq > 0.0f) ? e2m1_encode(z0 * rcp) : 0;
+                const uint8_t q1 = (dq > 0.0f) ? e2m1_encode(z1 * rcp) : 0;
+                Q[(r * cols + k) / 2] = (uint8_t)(q0 | (q1 << 4));
+            }
+        }
+    }
+    return 0;
+}
+
+/* y = alpha * sum over 16-element blocks j of e4m3(sx[m,j]) e4m3(sw[n,j]) (xq . wq over the block)
+ *     + bias + R; double, unrounded.  Xq [M, K/2], Wq [N, K/2] packed nibbles. */
+int kx_oracle_outproj_nvfp4_rows(const uint8_t* Xq, const uint8_t* sx, const uint8_t* Wq, const uint8_t* sw,
+                                 double alpha, const uint16_t* bias, const uint16_t* R, const int64_t* rows,
+                                 int64_t nrows, double* out, int64_t M, int64_t N, int64_t K) {
+    if (M < 0 || N < 0 || K < 0 || (K & 1) || nrows < 0 || !out) return -1;
+    if (K > 0 && (!Xq || !Wq || !sx || !sw)) return -1;
+    for (int64_t r = 0; rows && r < nrows; ++r)
+        if (rows[r] < 0 || rows[r] >= M) return -1;
+    if (!rows && nrows > M) return -1;
+    const int64_t nb = (K + 15) / 16, kb = K / 2;
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int64_t r = 0; r < nrows; ++r) {
+        for (int64_t n = 0; n < N; ++n) {
+            const int64_t m = rows ? rows[r] : r;
+            double y = 0.0;
+            for (int64_t j = 0; j < nb; ++j) {
+                const int64_t k1 = (j * 16 + 16 < K) ? j * 16 + 16 : K;
+                double acc = 0.0;
+                for (int64_t k = j * 16; k < k1; ++k) {
+                    const uint8_t xb = Xq[m * kb + k / 2], wb = Wq[n * kb + k / 2];
+                    acc += e2m1_decode((k & 1) ? xb >> 4 : xb & 15) * e2m1_decode((k & 1) ? wb >> 4 : wb & 15);
+                }
+                y += acc * e4m3_decode(sx[m * nb + j]) * e4m3_decode(sw[n * nb + j]);
+            }
+            y *= alpha;
+            if (bias) y += bf16_widen(bias[n]);
+            if (R) y += bf16_widen(R[m * N + n]);
+            out[r * N + n] = y;
+        }
+    }
+    return 0;
+}

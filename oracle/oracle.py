@@ -48,6 +48,10 @@ def _load():
         lib.kx_oracle_e8m0_decode.argtypes = [p, p, i64]
         lib.kx_oracle_quantize_rows_mx.argtypes = [p, i64, i64, p, p]
         lib.kx_oracle_outproj_mx_rows.argtypes = [p, p, p, p, p, p, p, i64, p, i64, i64, i64]
+        lib.kx_oracle_e2m1_decode.argtypes = [p, p, i64]
+        lib.kx_oracle_e2m1_encode.argtypes = [p, p, i64]
+        lib.kx_oracle_quantize_rows_nvfp4.argtypes = [p, i64, i64, ctypes.c_float, p, p]
+        lib.kx_oracle_outproj_nvfp4_rows.argtypes = [p, p, p, p, ctypes.c_double, p, p, p, i64, p, i64, i64, i64]
         lib.kx_oracle_max_threads.argtypes = []
         lib.kx_oracle_max_threads.restype = ctypes.c_int
         _lib = lib
@@ -361,4 +365,57 @@ def outproj_mx(Xq, ex, Wq, ew, bias=None, R=None, rows=None):
                                            _ptr(rows_arr), nrows, _ptr(out), M, N, K)
     if rc != 0:
         raise RuntimeError(f"kx_oracle_outproj_mx_rows failed ({rc})")
+    return out
+
+
+def e2m1_decode(nibbles) -> np.ndarray:
+    """E2M1 codes (low 4 bits of each byte) -> float64: +-{0, 0.5, 1, 1.5, 2, 3, 4, 6}."""
+    nib = np.ascontiguousarray(nibbles, dtype=np.uint8)
+    out = np.empty(nib.shape, dtype=np.float64)
+    _load().kx_oracle_e2m1_decode(_ptr(nib), _ptr(out), nib.size)
+    return out
+
+
+def e2m1_encode(x) -> np.ndarray:
+    """binary32 -> nearest E2M1 code, ties to the even code, saturating at +-6."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    out = np.empty(x.shape, dtype=np.uint8)
+    _load().kx_oracle_e2m1_encode(_ptr(x), _ptr(out), x.size)
+    return out
+
+
+def quantize_rows_nvfp4(Z, gs: float):
+    """4-bit block-scaled code book of BF16 rows (the format of the Section 4.3 task): per 16 consecutive
+    elements s = e4m3(max|z| / (6 gs)), q = e2m1(z / (e4m3_value(s) gs)), every step in binary32.
+    Z uint16 BF16 bits [rows, cols] -> (Q uint8 [rows, cols / 2] two codes per byte, low nibble first,
+    S uint8 [rows, ceil(cols / 16)] E4M3 bytes)."""
+    rows, cols = Z.shape
+    Z = _bits(Z, (rows, cols), "Z")
+    Q = np.empty((rows, cols // 2), dtype=np.uint8)
+    S = np.empty((rows, (cols + 15) // 16), dtype=np.uint8)
+    rc = _load().kx_oracle_quantize_rows_nvfp4(_ptr(Z), rows, cols, ctypes.c_float(gs), _ptr(Q), _ptr(S))
+    if rc != 0:
+        raise RuntimeError(f"kx_oracle_quantize_rows_nvfp4 failed ({rc})")
+    return Q, S
+
+
+def outproj_nvfp4(Xq, sx, Wq, sw, alpha: float, bias=None, R=None, rows=None):
+    """y = alpha * sum_j e4m3(sx[m,j]) e4m3(sw[n,j]) (Xq[m, block j] . Wq[n, block j]) + bias + R on packed E2M1
+    codes with one E4M3 scale per 16 elements; float64, unrounded."""
+    M, kb = Xq.shape
+    N = Wq.shape[0]
+    K = 2 * kb
+    nb = (K + 15) // 16
+    Xq = _typed(Xq, np.uint8, (M, kb), "Xq")
+    Wq = _typed(Wq, np.uint8, (N, kb), "Wq")
+    sx = _typed(sx, np.uint8, (M, nb), "sx")
+    sw = _typed(sw, np.uint8, (N, nb), "sw")
+    bias = _bits(bias, (N,), "bias")
+    R = _bits(R, (M, N), "R")
+    rows_arr, nrows = _rows_arg(rows, M)
+    out = np.empty((nrows, N), dtype=np.float64)
+    rc = _load().kx_oracle_outproj_nvfp4_rows(_ptr(Xq), _ptr(sx), _ptr(Wq), _ptr(sw), ctypes.c_double(alpha), _ptr(bias),
+                                              _ptr(R), _ptr(rows_arr), nrows, _ptr(out), M, N, K)
+    if rc != 0:
+        raise RuntimeError(f"kx_oracle_outproj_nvfp4_rows failed ({rc})")
     return out
