@@ -414,6 +414,40 @@ int kx_outproj_residual_mxfp8_ex(const void* Xq, const void* SFX, const void* Wq
                                  int64_t M, int64_t N, int64_t K, void* stream,
                                  const kx_plan_override* override_or_null);
 
+/*
+ * 4-bit block-scaled branch (the number format of the Section 4.3 task, "E2M1 with 1x16 block scaling", and
+ * the tensor-core kind it runs on).  Elements are E2M1 codes (sign, two exponent bits, one mantissa bit:
+ * magnitudes 0, 0.5, 1, 1.5, 2, 3, 4, 6), two per byte with the even k index in the low nibble; every 16
+ * consecutive elements of a row share one E4M3 scale byte (non-negative, never NaN); one binary32 scale gs
+ * belongs to the whole tensor:  value = e2m1(q) * e4m3(s) * gs.
+ *
+ * Code book (kx_quantize_rows_nvfp4), per block of 16 BF16 values z, every step in binary32:
+ *     s = e4m3( max|z| / (6 gs) )        nearest, ties to even, saturating at 448
+ *     q = e2m1( z * (1 / (value(s) gs)) )   nearest, ties to the even code, saturating at +-6; all codes 0
+ *                                           when s decodes to zero
+ * gs > 0 is the caller's (typically max|A| / (448 * 6)).  A [rows, cols] BF16, cols % 16 == 0, cols <= 32768;
+ * Q [rows, cols / 2] bytes; SF as below; device pointers, 16-byte aligned, no overlap.
+ *
+ * Scale layout: chunks of 512 bytes, one per (128 rows, 64 elements of K), ordered
+ * [ceil(rows / 128)][ceil(cols / 64)]; inside a chunk the scale of row r and 16-element block j sits at
+ * byte (r % 32) * 16 + (r % 128) / 32 * 4 + j % 4 (the 512-byte atom of Section 4.3).
+ * kx_nvfp4_scale_bytes gives the size of the array.  Padding entries (rows >= rows, blocks >= cols / 16) are
+ * written as 0 by the code book; arrays built elsewhere must hold finite E4M3 bytes there.
+ *
+ * kx_outproj_residual_nvfp4:
+ *     Y[m,n] = bf16( alpha * sum_j e4m3(sx[m,j]) e4m3(sw[n,j]) sum_{k in block j} xq[m,k] wq[n,k] + bias[n] + R[m,n] )
+ * with alpha = the product of the two tensor scales.  Xq [M, K/2], Wq [N, K/2] bytes; K % 32 == 0,
+ * N % 8 == 0; bias / R / Y as in kx_outproj_residual (R may be Y).  One CTA per 128 x 128 / 192 / 256 tile
+ * (tcgen05 kind::mxf4nvf4.block_scale, FP32 accumulation); the override may name block_n and raster_group
+ * (NULL = automatic).  Errors as for the calls above.
+ */
+int64_t kx_nvfp4_scale_bytes(int64_t rows, int64_t cols);
+int kx_quantize_rows_nvfp4(const void* A, float gs, void* Q, void* SF, int64_t rows, int64_t cols, void* stream);
+int kx_outproj_residual_nvfp4(const void* Xq, const void* SFX, const void* Wq, const void* SFW, float alpha,
+                              const void* bias_or_null, const void* R_or_null, void* Y,
+                              int64_t M, int64_t N, int64_t K, void* stream,
+                              const kx_plan_override* override_or_null);
+
 /* Fills `out` with the plan the library would use for this shape on the current
  * device (has_residual / has_bias as 0 or 1).  No work is enqueued. */
 int kx_plan_query(int64_t M, int64_t N, int64_t K, int has_bias, int has_residual,

@@ -30,6 +30,7 @@ EXPORTS = (
     "kx_quantize_rows_fp8", "kx_quantize_gate_up_fp8", "kx_rmsnorm_quantize_fp8", "kx_gate_up_swiglu_fp8",
     "kx_outproj_residual_fp8",
     "kx_mx_scale_bytes", "kx_quantize_rows_mxfp8", "kx_rmsnorm_quantize_mxfp8", "kx_outproj_residual_mxfp8", "kx_outproj_residual_mxfp8_ex",
+    "kx_nvfp4_scale_bytes", "kx_quantize_rows_nvfp4", "kx_outproj_residual_nvfp4",
     "kx_plan_query", "kx_last_device_status", "kx_status_string",
     "kx_version",
 )
@@ -102,13 +103,17 @@ def load():
     lib.kx_rmsnorm_quantize_mxfp8.argtypes = [vp, vp, ctypes.c_float, vp, vp, i64, i64, vp]
     lib.kx_outproj_residual_mxfp8.argtypes = [vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, vp]
     lib.kx_outproj_residual_mxfp8_ex.argtypes = [vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, vp, ctypes.POINTER(PlanOverride)]
+    lib.kx_nvfp4_scale_bytes.argtypes = [i64, i64]
+    lib.kx_quantize_rows_nvfp4.argtypes = [vp, ctypes.c_float, vp, vp, i64, i64, vp]
+    lib.kx_outproj_residual_nvfp4.argtypes = [vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, i64, i64, i64, vp,
+                                              ctypes.POINTER(PlanOverride)]
     lib.kx_plan_query.argtypes = [i64, i64, i64, ci, ci, ctypes.POINTER(PlanOverride), ctypes.POINTER(PlanInfo)]
     lib.kx_last_device_status.argtypes = [vp, ctypes.POINTER(ci), ctypes.POINTER(ci)]
     lib.kx_status_string.argtypes = [ci]
     lib.kx_status_string.restype = ctypes.c_char_p
     lib.kx_version.argtypes = []
     for name in EXPORTS:
-        if name == "kx_mx_scale_bytes":
+        if name in ("kx_mx_scale_bytes", "kx_nvfp4_scale_bytes"):
             getattr(lib, name).restype = i64
         elif name != "kx_status_string":
             getattr(lib, name).restype = ci
@@ -538,4 +543,39 @@ def kx_outproj_residual_mxfp8(Xq, SFX, Wq, SFW, bias, R, Y, stream=None, check=T
                                                  _addr(Y), M, N, K, _stream(stream), ctypes.byref(override))
     if check and rc != KX_OK:
         raise KxError(rc, "kx_outproj_residual_mxfp8")
+    return rc
+
+
+def kx_nvfp4_scale_bytes(rows: int, cols: int) -> int:
+    """Bytes of the chunked E4M3 scale array of a [rows, cols] 4-bit block-scaled matrix."""
+    return int(load().kx_nvfp4_scale_bytes(int(rows), int(cols)))
+
+
+def kx_quantize_rows_nvfp4(A, gs: float, Q, SF, stream=None, check=True) -> int:
+    """Q (uint8 [rows, cols / 2], two E2M1 codes per byte), SF (uint8, kx_nvfp4_scale_bytes(rows, cols) bytes) =
+    4-bit block-scaled code book of the BF16 matrix A with tensor scale gs."""
+    import torch
+    rows, cols = A.shape
+    _check_bf16("A", A, (rows, cols)); _check("Q", Q, (rows, cols // 2), torch.uint8)
+    _check("SF", SF, (kx_nvfp4_scale_bytes(rows, cols),), torch.uint8)
+    rc = load().kx_quantize_rows_nvfp4(_addr(A), float(gs), _addr(Q), _addr(SF), rows, cols, _stream(stream))
+    if check and rc != KX_OK:
+        raise KxError(rc, "kx_quantize_rows_nvfp4")
+    return rc
+
+
+def kx_outproj_residual_nvfp4(Xq, SFX, Wq, SFW, alpha: float, bias, R, Y, stream=None, check=True, override=None) -> int:
+    """Y = alpha * block-scaled (Xq, SFX) (Wq, SFW)^T + bias + R on packed E2M1 codes; bias / R may be None."""
+    import torch
+    M, kb = Xq.shape
+    N = Wq.shape[0]
+    K = 2 * kb
+    _check("Xq", Xq, (M, kb), torch.uint8); _check("Wq", Wq, (N, kb), torch.uint8)
+    _check("SFX", SFX, (kx_nvfp4_scale_bytes(M, K),), torch.uint8); _check("SFW", SFW, (kx_nvfp4_scale_bytes(N, K),), torch.uint8)
+    _check_bf16("bias", bias, (N,)); _check_bf16("R", R, (M, N)); _check_bf16("Y", Y, (M, N))
+    rc = load().kx_outproj_residual_nvfp4(_addr(Xq), _addr(SFX), _addr(Wq), _addr(SFW), float(alpha), _addr(bias), _addr(R),
+                                          _addr(Y), M, N, K, _stream(stream),
+                                          ctypes.byref(override) if override is not None else None)
+    if check and rc != KX_OK:
+        raise KxError(rc, "kx_outproj_residual_nvfp4")
     return rc

@@ -133,6 +133,15 @@ const MxVariant* find_mx(int bn, int ctas, int stages = 0) {
     return nullptr;
 }
 
+// 4-bit block-scaled tile kernels: (tile width, ring stages, R staging buffers); the 256-column shape has a
+// single accumulator buffer like its 8-bit sibling
+#define KX_NV(BN, ST, NB)                                                                     \
+    MxVariant {                                                                               \
+        BN, 1, ST, NB, 1, TileCfg<BN, 1, ST, NB, 1, 2>::SMEM_BYTES,                           \
+            reinterpret_cast<const void*>(&kx_tile_kernel<BN, 1, ST, NB, 4, 1>)               \
+    }
+const MxVariant kNvVariants[] = {KX_NV(128, 5, 2), KX_NV(192, 4, 2), KX_NV(256, 3, 2)};
+
 // first variant in table order that matches; stages == 0 matches any depth
 const TileVariant* find_tile(int bn, int ctas, int stages) {
     for (const auto& v : kTileVariants)
@@ -192,6 +201,8 @@ int ensure_device(int dev, DeviceCtx** out) {
                  cudaFuncSetAttribute(v.fn_s8, cudaFuncAttributeMaxDynamicSharedMemorySize, v.smem) == cudaSuccess &&
                  cudaFuncSetAttribute(v.fn_f8, cudaFuncAttributeMaxDynamicSharedMemorySize, v.smem) == cudaSuccess;
         for (const auto& v : kMxVariants)
+            ok = ok && cudaFuncSetAttribute(v.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, v.smem) == cudaSuccess;
+        for (const auto& v : kNvVariants)
             ok = ok && cudaFuncSetAttribute(v.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, v.smem) == cudaSuccess;
         for (const auto& v : kSwapVariants)
             ok = ok &&
@@ -287,11 +298,11 @@ int get_tmap(const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows, C
 
 // Scale chunks of a block-scaled operand as a 2-D tensor [chunks][128 32-bit words], one chunk
 // (512 contiguous bytes, no swizzle) per box.  Shares the descriptor cache (box_rows 1, 4-byte elements).
-int get_tmap_scales(const void* ptr, uint64_t chunks, CUtensorMap* out) {
-    TmapKey key{ptr, chunks, 128, 128, 1, 4};
+int get_tmap_scales(const void* ptr, uint64_t chunks, CUtensorMap* out, uint32_t box_chunks = 1) {
+    TmapKey key{ptr, chunks, 128, 128, box_chunks, 4};
     uint64_t h = reinterpret_cast<uint64_t>(ptr) >> 4;
     h ^= chunks * 0x9E3779B97F4A7C15ull;
-    h ^= 0x51ED270B27D4EB4Full;
+    h ^= 0x51ED270B27D4EB4Full * box_chunks;
     h ^= h >> 29;
     TmapEntry& e = t_tmaps[h % kTmapSlots];
     if (e.valid && e.key == key) {
@@ -300,7 +311,7 @@ int get_tmap_scales(const void* ptr, uint64_t chunks, CUtensorMap* out) {
     }
     cuuint64_t dims[2] = {128, chunks};
     cuuint64_t strides[1] = {512};
-    cuuint32_t box[2] = {128, 1};
+    cuuint32_t box[2] = {128, box_chunks};
     cuuint32_t estr[2] = {1, 1};
     CUresult r = g_encode(&e.map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void*>(ptr), dims, strides, box, estr,
                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -1280,7 +1291,8 @@ int kx_outproj_residual_rmsnorm(const void* X, const void* W, const void* bias, 
 namespace {
 bool aligned4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3u) == 0; }
 
-// fmt: 0 = INT8 codes, 1 = FP8 E4M3 codes (one scale per row); 2 = FP8 E4M3 codes with one E8M0 scale per 32 elements
+// fmt: 0 = INT8 codes, 1 = FP8 E4M3 codes (one scale per row); 2 = FP8 E4M3 codes with one E8M0 scale per 32
+// elements; 3 = E2M1 codes with one E4M3 scale per 16 elements (never behind RMSNorm)
 int launch_rowquant(const QuantParams& qp, bool norm, int fmt, cudaStream_t stream, int sm_count) {
     cudaLaunchConfig_t cfg;
     std::memset(&cfg, 0, sizeof cfg);
@@ -1288,7 +1300,8 @@ int launch_rowquant(const QuantParams& qp, bool norm, int fmt, cudaStream_t stre
     const void* fn = nullptr;
     int per_sm = 8;
 #define KX_QUANT_FN(NV)                                                                              \
-    (fmt == 2 ? (norm ? reinterpret_cast<const void*>(&kx_rowquant_kernel<NV, true, 2>)              \
+    (fmt == 3 ? reinterpret_cast<const void*>(&kx_rowquant_kernel<NV, false, 3>)                     \
+     : fmt == 2 ? (norm ? reinterpret_cast<const void*>(&kx_rowquant_kernel<NV, true, 2>)            \
                       : reinterpret_cast<const void*>(&kx_rowquant_kernel<NV, false, 2>))            \
      : fmt == 1 ? (norm ? reinterpret_cast<const void*>(&kx_rowquant_kernel<NV, true, 1>)            \
                         : reinterpret_cast<const void*>(&kx_rowquant_kernel<NV, false, 1>))          \
@@ -1774,6 +1787,136 @@ int kx_outproj_residual_mxfp8_ex(const void* Xq, const void* SFX, const void* Wq
                                  const void* R, void* Y, int64_t M, int64_t N, int64_t K, void* stream,
                                  const kx_plan_override* ov) {
     return outproj_residual_mx(Xq, SFX, Wq, SFW, bias, R, Y, M, N, K, stream, ov);
+}
+
+// ---------------------------------------------------------------- 4-bit block-scaled branch
+int64_t kx_nvfp4_scale_bytes(int64_t rows, int64_t cols) {
+    if (rows < 0 || cols < 0) return -1;
+    return mx_chunks(rows) * ((cols + 63) / 64) * 512;
+}
+
+int kx_quantize_rows_nvfp4(const void* A, float gs, void* Q, void* SF, int64_t rows, int64_t cols, void* stream) {
+    if (rows < 0 || cols < 0 || rows > 0x7FFFFFFFll / 2) return KX_ERR_SHAPE;
+    if ((cols % 16) != 0 || cols > 8ll * kNormThreads * kNormVecs || !(gs > 0.0f) || !(gs < INFINITY)) return KX_ERR_SHAPE;
+    if (rows == 0 || cols == 0) return KX_OK;
+    if (!A || !Q || !SF) return KX_ERR_NULL;
+    if (!aligned16(A) || !aligned16(Q) || !aligned16(SF)) return KX_ERR_ALIGN;
+    const size_t ab = static_cast<size_t>(rows) * cols * 2, qb = static_cast<size_t>(rows) * cols / 2,
+                 sb = static_cast<size_t>(kx_nvfp4_scale_bytes(rows, cols));
+    if (overlaps(Q, qb, A, ab) || overlaps(SF, sb, A, ab) || overlaps(SF, sb, Q, qb)) return KX_ERR_OVERLAP;
+    DeviceCtx* ctx = nullptr;
+    int rc = device_ctx(&ctx);
+    if (rc != KX_OK) return rc;
+    QuantParams qp;
+    std::memset(&qp, 0, sizeof qp);
+    qp.A0 = qp.A1 = static_cast<const uint16_t*>(A);
+    qp.Q0 = qp.Q1 = static_cast<int8_t*>(Q);
+    qp.SF0 = static_cast<uint8_t*>(SF);
+    qp.rows0 = rows;
+    qp.M = rows;
+    qp.N = static_cast<int>(cols);
+    qp.kchunks = static_cast<int>((cols + 63) / 64);
+    qp.gs = gs;
+    return launch_rowquant(qp, false, 3, static_cast<cudaStream_t>(stream), ctx->sm_count);
+}
+
+int kx_outproj_residual_nvfp4(const void* Xq, const void* SFX, const void* Wq, const void* SFW, float alpha,
+                              const void* bias, const void* R, void* Y, int64_t M, int64_t N, int64_t K, void* stream_v,
+                              const kx_plan_override* ov) {
+    if (M < 0 || N < 0 || K < 0) return KX_ERR_SHAPE;
+    if (M > 0x7FFFFFFFll / 2 || N > 0x7FFFFFFFll / 4 || K > 0x7FFFFFFFll / 2) return KX_ERR_SHAPE;
+    if (M == 0 || N == 0) return KX_OK;
+    if ((N % 8) != 0 || (K % 32) != 0) return KX_ERR_SHAPE;
+    if (!Y) return KX_ERR_NULL;
+    if (!aligned16(Y) || (bias && !aligned16(bias)) || (R && !aligned16(R))) return KX_ERR_ALIGN;
+    const size_t yb = static_cast<size_t>(M) * N * 2;
+    if (overlaps(Y, yb, bias, static_cast<size_t>(N) * 2)) return KX_ERR_OVERLAP;
+    if (R && R != Y && overlaps(Y, yb, R, yb)) return KX_ERR_OVERLAP;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    DeviceCtx* ctx = nullptr;
+    int rc = device_ctx(&ctx);
+    if (rc != KX_OK) return rc;
+    if (K == 0) {
+        const long long total = M * N;
+        const int blocks = static_cast<int>(std::min<long long>((total + 255) / 256, ctx->sm_count * 8));
+        kx_k0_kernel<<<blocks, 256, 0, stream>>>(static_cast<const uint16_t*>(bias), static_cast<const uint16_t*>(R),
+                                                 static_cast<uint16_t*>(Y), M, N, N, N);
+        return cudaGetLastError() == cudaSuccess ? KX_OK : KX_ERR_CUDA;
+    }
+    if (!Xq || !Wq || !SFX || !SFW) return KX_ERR_NULL;
+    if (!aligned16(Xq) || !aligned16(Wq) || !aligned16(SFX) || !aligned16(SFW)) return KX_ERR_ALIGN;
+    if (overlaps(Y, yb, Xq, static_cast<size_t>(M) * K / 2) || overlaps(Y, yb, Wq, static_cast<size_t>(N) * K / 2) ||
+        overlaps(Y, yb, SFX, static_cast<size_t>(kx_nvfp4_scale_bytes(M, K))) ||
+        overlaps(Y, yb, SFW, static_cast<size_t>(kx_nvfp4_scale_bytes(N, K))))
+        return KX_ERR_OVERLAP;
+    // tile width: fewest (waves x columns per tile), wider tiles first on ties (more work per issued MMA)
+    const MxVariant* v = nullptr;
+    if (ov && ov->block_n) {
+        for (const auto& c : kNvVariants)
+            if (c.bn == ov->block_n) v = &c;
+        if (!v) return KX_ERR_PLAN;
+    } else {
+        long long best = 0;
+        for (const auto& c : kNvVariants) {
+            const long long tiles = ((M + 127) / 128) * ((N + c.bn - 1) / c.bn);
+            const long long cost = ((tiles + ctx->sm_count - 1) / ctx->sm_count) * (c.bn + 64);
+            if (!v || cost <= best) { v = &c; best = cost; }
+        }
+    }
+    const int bn = v->bn;
+    const long long tm = (M + 127) / 128, tiles_n = (N + bn - 1) / bn, tiles = tm * tiles_n;
+    if (tiles > 0x7FFFFFFFll / 4) return KX_ERR_SHAPE;
+    const long long kch = (K + 63) / 64;
+    CUtensorMap tmA, tmB, tmY, tmR, tmSA, tmSB;
+    if ((rc = get_tmap(Xq, M, K / 2, 128, &tmA, 1)) != KX_OK) return rc;
+    if ((rc = get_tmap(Wq, N, K / 2, bn, &tmB, 1)) != KX_OK) return rc;
+    if ((rc = get_tmap_scales(SFX, mx_chunks(M) * kch, &tmSA, 4)) != KX_OK) return rc;
+    if ((rc = get_tmap_scales(SFW, mx_chunks(N) * kch, &tmSB, 4)) != KX_OK) return rc;
+    if ((rc = get_tmap(Y, M, N, 32, &tmY)) != KX_OK) return rc;
+    if (R) {
+        if ((rc = get_tmap(R, M, N, 32, &tmR)) != KX_OK) return rc;
+    } else {
+        tmR = tmY;
+    }
+    TileParams p;
+    std::memset(&p, 0, sizeof p);
+    p.M = static_cast<int>(M);
+    p.N = static_cast<int>(N);
+    p.K = static_cast<int>(K / 2);            // bytes per operand row
+    p.tiles_m = static_cast<int>(tm);
+    p.tiles_n = static_cast<int>(tiles_n);
+    p.num_tiles = static_cast<int>(tiles);
+    p.raster_group = (ov && ov->raster_group > 0) ? ov->raster_group : 8;
+    p.has_bias = bias ? 1 : 0;
+    p.has_r = R ? 1 : 0;
+    p.kcluster = 1;
+    p.sk_tile0 = p.num_tiles;
+    p.narrow_tile0 = p.num_tiles;
+    p.spin_limit_ns = 2000000000ull;
+    p.status = ctx->status;
+    p.ws = ctx->ws;
+    p.counters = ctx->counters;
+    p.sfb_chunks = static_cast<int>(mx_chunks(N));
+    p.sf_kchunks = static_cast<int>(kch);
+    p.alpha = alpha;
+    cudaLaunchConfig_t cfg;
+    std::memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3(static_cast<unsigned>(std::min<long long>(tiles, ctx->sm_count)), 1, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = v->smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const uint16_t* bias_p = static_cast<const uint16_t*>(bias);
+    void* args[] = {&tmA, &tmB, &tmSA, &tmY, &tmR, &tmSB, &bias_p, &p};
+    if (cudaLaunchKernelExC(&cfg, v->fn, args) != cudaSuccess) {
+        cudaGetLastError();
+        return KX_ERR_CUDA;
+    }
+    return KX_OK;
 }
 
 // ---------------------------------------------------------------- no-allocation entry

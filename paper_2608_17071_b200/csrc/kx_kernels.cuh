@@ -128,7 +128,9 @@ struct TileParams {
     const float* sa;           // KIND 1 / 2: scale per row of A [M]
     const float* sb;           // KIND 1 / 2: scale per row of B [N] (gate rows in gate/up mode)
     const float* sb2;          // KIND 1 / 2, gate/up mode: scale per up row [N]
-    int sfb_chunks;            // KIND 3: ceil(N / 128) = rows of 128-row scale chunks of B
+    int sfb_chunks;            // KIND 3 / 4: ceil(N / 128) = rows of 128-row scale chunks of B
+    int sf_kchunks;            // KIND 4: scale chunks per 128 rows along K = ceil(K / 64)
+    float alpha;               // KIND 4: product of the two tensor scales, applied to the accumulators
     int swiglu;                   // 1: gate/up mode.  W rows of a tile = BN/2 rows of Wg (tmB) followed by the same
                                   // BN/2 rows of Wu (tmB2); the epilogue writes silu(gate) * up, BN/2 columns per
                                   // tile, N = number of output columns; no bias, no residual
@@ -164,7 +166,8 @@ struct TileCfg {
     static constexpr int EPI_BYTES = 4 * NB * SLAB_BYTES;
     static constexpr int NUM_BARS = 2 * STAGES + 4 + 4 * NB + 1;
     static constexpr int SFB_CHUNKS = (BN > 128) ? 2 : 1;
-    static constexpr int SF_KB_BYTES = MX ? 512 * (1 + SFB_CHUNKS) : 0;     // scale bytes per k-block
+    // scale bytes per k-block: MX 1 = one chunk per operand row block, MX 2 (16-element blocks) = four
+    static constexpr int SF_KB_BYTES = MX == 1 ? 512 * (1 + SFB_CHUNKS) : MX == 2 ? 2048 * (1 + SFB_CHUNKS) : 0;
     static constexpr int SF_STAGE = KBS * SF_KB_BYTES;
     static constexpr int SMEM_BYTES = 1024 + STAGES * (STAGE_BYTES + SF_STAGE) + EPI_BYTES + 1024;
     // accumulator buffers in tensor memory: two, so that the epilogue of one tile overlaps the MMAs of the
@@ -241,13 +244,18 @@ __device__ __forceinline__ uint32_t ld_acquire_gpu_u32(const unsigned int* p) {
 // the ring beside the operand tiles, are copied to TMEM before the four K steps of their k-block, and
 // the FP32 accumulators need no dequantisation; whole full-width tiles only.  Its scale chunks come
 // through two more tensor maps: tmB2 = scales of A, tmS = scales of B, both [chunks][128 words].
+// KIND 4: 4-bit E2M1 operands, two per byte, with one E4M3 scale per 16 elements (tcgen05
+// kind::mxf4nvf4.block_scale): a k-block is 256 elements = four K = 64 steps, each with scale chunks of
+// its own (four per 128 rows and k-block, fetched as one box); the accumulators are multiplied by
+// alpha (the product of the two tensor scales) in the epilogue.  p.K counts bytes for this kind.
 template <int BN, int CTAS, int STAGES, int NB, int KIND = 0, int KBS = 1>
 __global__ void __launch_bounds__(kThreads, 1)
 kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmB2, const __grid_constant__ CUtensorMap tmY,
                const __grid_constant__ CUtensorMap tmR, const __grid_constant__ CUtensorMap tmS,
                const uint16_t* __restrict__ bias, const TileParams p) {
-    using C = TileCfg<BN, CTAS, STAGES, NB, KBS, KIND == 3 ? 1 : 0>;
+    using C = TileCfg<BN, CTAS, STAGES, NB, KBS, KIND == 3 ? 1 : KIND == 4 ? 2 : 0>;
+    static_assert(KIND != 4 || (CTAS == 1 && KBS == 1), "4-bit kind: one CTA per tile, one k-block per stage");
     constexpr bool kRowScaled = (KIND == 1 || KIND == 2);       // dequantised in the epilogue
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -271,7 +279,9 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int lane = threadIdx.x & 31;
     const uint32_t cta_rank = (CTAS == 2) ? cluster_ctarank() : 0u;
     const bool leader = (cta_rank == 0);
-    constexpr int KBLK = (KIND != 0) ? 2 * kBlockK : kBlockK;   // elements per k-block (128 bytes)
+    // k-block = 128 bytes of a row: 64 BF16 or 128 8-bit elements; for the 4-bit kind p.K counts bytes
+    // (two elements each), so a k-block is 128 of those as well
+    constexpr int KBLK = (KIND != 0) ? 2 * kBlockK : kBlockK;
     const int nkb = (p.K + KBLK - 1) / KBLK;
     const int kc = (CTAS == 1 && p.kcluster > 1) ? p.kcluster : 1;   // K-cluster size
     const int krank = (kc > 1) ? static_cast<int>(cluster_ctarank()) : 0;
@@ -296,8 +306,8 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (warp == 4 && lane == 0) {
         prefetch_tmap(&tmA);
         prefetch_tmap(&tmB);
-        if (p.narrow_tile0 < p.num_tiles || KIND == 3) prefetch_tmap(&tmB2);
-        if (KIND == 3) prefetch_tmap(&tmS);
+        if (p.narrow_tile0 < p.num_tiles || KIND >= 3) prefetch_tmap(&tmB2);
+        if (KIND >= 3) prefetch_tmap(&tmS);
         prefetch_tmap(&tmY);
         if (p.has_r) prefetch_tmap(&tmR);
         // Warm L2 with the first ring-full of this CTA's operand tiles before waiting for the
@@ -411,6 +421,16 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                             }
                         }
                     }
+                    if constexpr (KIND == 4) {
+                        // 16-element blocks: four scale chunks per 128 rows and k-block (one per K = 64 step),
+                        // contiguous, fetched as one 2048-byte box per operand row block
+                        const int c0 = col >> 7;
+                        const uint32_t dst = s_sf + s * C::SF_STAGE;
+                        tma_load_2d(dst, &tmB2, 0, tm * p.sf_kchunks + kb * 4, full(s));
+                        for (int i = 0; i < C::SFB_CHUNKS; ++i)
+                            tma_load_2d(dst + 2048 * (1 + i), &tmS, 0, min(c0 + i, p.sfb_chunks - 1) * p.sf_kchunks + kb * 4,
+                                        full(s));
+                    }
                     if constexpr (CTAS == 1) {
                         mbar_arrive_expect_tx(full(s), nsub * (stage_tx + C::SF_KB_BYTES));
                         for (int j = 0; j < nsub; ++j) {
@@ -442,6 +462,7 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             constexpr uint32_t idesc_wide = KIND == 1   ? idesc_s8_s32(128 * CTAS, BN)
                                             : KIND == 2 ? idesc_e4m3_f32(128 * CTAS, BN)
                                             : KIND == 3 ? idesc_mxf8(128 * CTAS, BN)
+                                            : KIND == 4 ? idesc_nvf4(128, BN)
                                                         : idesc_bf16_f32(128 * CTAS, BN);
             constexpr uint32_t idesc_narrow = KIND == 1   ? idesc_s8_s32(128 * CTAS, BN / 2)
                                               : KIND == 2 ? idesc_e4m3_f32(128 * CTAS, BN / 2)
@@ -466,7 +487,28 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 tc_fence_after();
                 KX_TRACE_POINT(p, slot, (scount - 1) * 4 + 1);
                 const uint32_t d = tmem_base + b * BN;
-                if constexpr (KIND == 3) {
+                if constexpr (KIND == 4) {
+                    int tm, col;
+                    bool narrow;
+                    decode_tile(tile, tm, col, narrow);
+                    const uint32_t b_off = static_cast<uint32_t>(col & 127) >> 5;
+                    for (int kb = kb0; kb < kb1; ++kb) {
+                        if (!wt.wait(full_bar, ph, kWhereFull)) { ok = false; break; }
+                        tc_fence_after();
+                        const uint32_t sf = s_sf + s * C::SF_STAGE;
+                        mma_kblock_nv<C::SFB_CHUNKS>(d, a_lo, a_lo + (kABytes >> 4), idesc_wide, (kb > kb0) ? 1u : 0u,
+                                                     (sf & 0x3FFFFu) >> 4, tmem_base + C::ACC_BUFS * BN, b_off);
+                        mma_commit<1>(empty_bar0);
+                        full_bar = (s + 1 == STAGES) ? full(0) : full_bar + 8u;
+                        if (s + 1 == STAGES) {
+                            s = 0; ph ^= 1u;
+                            empty_bar0 = empty_base0; a_lo = a_lo0;
+                        } else {
+                            ++s;
+                            empty_bar0 += 8u; a_lo += C::STAGE_BYTES >> 4;
+                        }
+                    }
+                } else if constexpr (KIND == 3) {
                     // block-scaled: per k-block, scale chunks -> TMEM (a rotating set of 12 columns), then
                     // four K = 32 steps that each name their byte of the scale columns
                     int tm, col;
@@ -776,6 +818,11 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     tmem_ld_32x32(tbase + c * 64 + 32, acc[1]);
                     tmem_ld_wait();
                     if constexpr (kRowScaled) dequant(acc[0], acc[1], p.sb, col0);
+                    if constexpr (KIND == 4) {
+#pragma unroll
+                        for (int i = 0; i < 64; ++i)
+                            acc[i >> 5][i & 31] = __float_as_uint(__uint_as_float(acc[i >> 5][i & 31]) * p.alpha);
+                    }
                 }
                 if (valid && sg) {
                     // acc holds the gate pre-activations of these 64 output columns; the matching up
@@ -1485,6 +1532,10 @@ kx_rmsnorm_kernel(const uint16_t* __restrict__ H, const uint16_t* __restrict__ g
 // maximum.  Scale bytes go to SF0 in 512-byte chunks, chunk (row / 128, k / 128), byte
 // (row % 32) * 16 + (row % 128) / 32 * 4 + (k / 32) % 4; entries of blocks past the row end and of the
 // rows up to the next multiple of 128 are padding and are set to 127.  One matrix per launch.
+// FMT 3: 4-bit block-scaled - per 16 consecutive elements (two neighbouring threads) s = e4m3(max|z| / (6 gs)),
+// codes e2m1(z * (1 / (value(s) gs))), every step in binary32; two codes per byte, even k in the low
+// nibble; scale bytes chunked as for FMT 2 but one chunk per (128 rows, 64 elements): byte
+// (row % 32) * 16 + (row % 128) / 32 * 4 + (k / 16) % 4; padding entries are set to 0.
 struct QuantParams {
     const uint16_t* A0;
     const uint16_t* A1;
@@ -1496,8 +1547,9 @@ struct QuantParams {
     uint8_t* SF0;          // FMT 2: chunked scale bytes
     long long rows0, M;
     int N;
-    int kchunks;           // FMT 2: ceil(N / 128)
+    int kchunks;           // FMT 2: ceil(N / 128); FMT 3: ceil(N / 64)
     float eps;
+    float gs;              // FMT 3: tensor scale (> 0)
 };
 
 template <int NV, bool NORM, int FMT>
@@ -1603,6 +1655,51 @@ kx_rowquant_kernel(const QuantParams p) {
                     const long long rr = p.M + t / per_row;
                     const int jj = static_cast<int>(t % per_row);
                     p.SF0[((rr >> 7) * p.kchunks + (jj >> 2)) * 512 + (rr & 31) * 16 + ((rr & 127) >> 5) * 4 + (jj & 3)] = 127;
+                }
+            }
+            continue;
+        }
+        if constexpr (FMT == 3) {
+            uint32_t* qrow = reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(p.Q0) + r * (N / 2));
+            uint8_t* const sfrow = p.SF0 + (r >> 7) * p.kchunks * 512 + (r & 31) * 16 + ((r & 127) >> 5) * 4;
+            const int nb = N >> 4;
+            const float d6 = __fmul_rn(6.0f, p.gs);
+#pragma unroll
+            for (int i = 0; i < NV; ++i) {
+                const int idx = tid + i * kNormThreads;
+                const bool valid = idx < nvec;
+                const uint32_t w4[4] = {valid ? v[i].x : 0u, valid ? v[i].y : 0u, valid ? v[i].z : 0u, valid ? v[i].w : 0u};
+                float z[8], bmax = 0.f;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    z[2 * k] = bf16_lo(w4[k]);
+                    z[2 * k + 1] = bf16_hi(w4[k]);
+                    bmax = fmaxf(bmax, fmaxf(fabsf(z[2 * k]), fabsf(z[2 * k + 1])));
+                }
+                // N % 16 == 0: the two threads of a block are both valid or both invalid
+                bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, 1));
+                if (valid) {
+                    const uint32_t sb = pack_e4m3x4(__fdiv_rn(bmax, d6), 0.f, 0.f, 0.f) & 0xFFu;
+                    const float dq = __fmul_rn(e4m3_to_f32(sb), p.gs);
+                    const float rcp = (dq > 0.f) ? __fdiv_rn(1.0f, dq) : 0.f;
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) z[k] = __fmul_rn(z[k], rcp);
+                    qrow[idx] = (dq > 0.f) ? pack_e2m1x8(z) : 0u;
+                    if ((tid & 1) == 0) {
+                        const int j = idx >> 1;
+                        sfrow[(j >> 2) * 512 + (j & 3)] = static_cast<uint8_t>(sb);
+                        if (j == nb - 1)
+                            for (int jj = nb; jj < p.kchunks * 4; ++jj) sfrow[(jj >> 2) * 512 + (jj & 3)] = 0;
+                    }
+                }
+            }
+            if (r == p.M - 1) {
+                const long long pad_rows = ((p.M + 127) & ~127ll) - p.M;
+                const int per_row = p.kchunks * 4;
+                for (long long t = tid; t < pad_rows * per_row; t += kNormThreads) {
+                    const long long rr = p.M + t / per_row;
+                    const int jj = static_cast<int>(t % per_row);
+                    p.SF0[((rr >> 7) * p.kchunks + (jj >> 2)) * 512 + (rr & 31) * 16 + ((rr & 127) >> 5) * 4 + (jj & 3)] = 0;
                 }
             }
             continue;

@@ -1,6 +1,7 @@
 // Inline-PTX wrappers for sm_100a: mbarrier, TMA (cp.async.bulk.tensor), tcgen05
 // (TMEM allocation, MMA, commit, load) and cluster helpers.
 #pragma once
+#include <cuda_fp16.h>
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -401,6 +402,60 @@ __device__ __forceinline__ void mma_kblock_mx(uint32_t d_tmem, uint32_t a_lo, ui
 #undef KX_MX_BODY
 #undef KX_MX_STEP
 #undef KX_MX_CP
+
+// ------------------------------------------------------------------ 4-bit block-scaled kind (kind::mxf4nvf4)
+// E2M1 elements packed two per byte (a 128-byte swizzle row holds 256 of them = four K = 64 steps), one
+// E4M3 scale per 16 elements: a K = 64 step reads all four bytes of a 32-bit scale column per row.
+// Instruction descriptor: A = B = E2M1 (format 1), K-major, E4M3 scales (bit 23 clear).
+__host__ __device__ constexpr uint32_t idesc_nvf4(int m, int n) {
+    return (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(m >> 4) << 24);
+}
+// One k-block: for each of its four K = 64 steps, the step's scale chunks (A, then CHUNKS of B; the four
+// steps' chunks of one operand are contiguous, 512 bytes each, operands 2048 bytes apart) are copied to 12
+// TMEM columns of their own, then the step is issued.  sfb_off = first scale column of the tile's B rows
+// inside the B chunks.
+template <int CHUNKS>
+__device__ __forceinline__ void mma_kblock_nv(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc,
+                                              uint32_t acc_first, uint32_t sf_lo, uint32_t cols, uint32_t sfb_off) {
+    const uint64_t hi = static_cast<uint64_t>(kDescHiSw128) << 32;
+    const uint64_t sf_hi = static_cast<uint64_t>((128u >> 4) | (1u << 14)) << 32;
+#pragma unroll
+    for (uint32_t i = 0; i < 4; ++i) {
+        const uint32_t c = cols + 12u * i;
+        asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(c), "l"(sf_hi | (sf_lo + 32u * i)) : "memory");
+        asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(c + 4u), "l"(sf_hi | (sf_lo + 128u + 32u * i))
+                     : "memory");
+        if constexpr (CHUNKS == 2)
+            asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(c + 8u),
+                         "l"(sf_hi | (sf_lo + 256u + 32u * i))
+                         : "memory");
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::mxf4nvf4.block_scale.scale_vec::4X [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
+            ::"r"(d_tmem), "l"(hi | (a_lo + 2u * i)), "l"(hi | (b_lo + 2u * i)), "r"(idesc),
+              "r"((acc_first != 0u || i > 0u) ? 1u : 0u), "r"(c), "r"(c + 4u + sfb_off)
+            : "memory");
+    }
+}
+// two binary32 values -> one byte of two E2M1 codes (nearest, ties to even, saturating): `lo` in the low nibble
+__device__ __forceinline__ uint32_t pack_e2m1x8(const float (&z)[8]) {
+    uint32_t r;
+    asm("{\n\t.reg .b8 b0, b1, b2, b3;\n\t"
+        "cvt.rn.satfinite.e2m1x2.f32 b0, %2, %1;\n\t"
+        "cvt.rn.satfinite.e2m1x2.f32 b1, %4, %3;\n\t"
+        "cvt.rn.satfinite.e2m1x2.f32 b2, %6, %5;\n\t"
+        "cvt.rn.satfinite.e2m1x2.f32 b3, %8, %7;\n\t"
+        "mov.b32 %0, {b0, b1, b2, b3};\n\t}"
+        : "=r"(r)
+        : "f"(z[0]), "f"(z[1]), "f"(z[2]), "f"(z[3]), "f"(z[4]), "f"(z[5]), "f"(z[6]), "f"(z[7]));
+    return r;
+}
+// one E4M3 byte -> binary32 (exact)
+__device__ __forceinline__ float e4m3_to_f32(uint32_t byte) {
+    uint32_t h2;
+    asm("{\n\t.reg .b16 t;\n\tcvt.u16.u32 t, %1;\n\tcvt.rn.f16x2.e4m3x2 %0, t;\n\t}" : "=r"(h2) : "r"(byte & 0xFFu));
+    return __half2float(__ushort_as_half(static_cast<unsigned short>(h2 & 0xFFFFu)));
+}
 
 // Arrive on an mbarrier once every MMA issued so far by this thread has finished.
 // `bar` is a shared::cluster address (this CTA's own shared::cta address is one).
