@@ -672,6 +672,50 @@ def run_ours(args):
             del keep, calls, qcalls
             torch.cuda.empty_cache()
 
+        # 4-bit block-scaled: the code book, then the projection on those codes; peak = 4 x the BF16 GEMM peak
+        peak4 = 4.0 * peaks["bf16_tflops"]
+        for (Mo, No, Ko) in [(4096, 4096, 4096), (16384, 4096, 14336)]:
+            ops = 2.0 * Mo * No * Ko
+            nbytes = 0.5 * (Mo * Ko + No * Ko) * (1.0 + 1.0 / 8) + 4.0 * Mo * No
+            ns = int(max(2, min(8, math.ceil(2.0 * L2_BYTES / nbytes))))
+            keep, calls, qcalls = [], [], []
+            for _ in range(ns):
+                Xs = torch.randn(Mo, Ko, device="cuda", generator=g).bfloat16()
+                Ws = (torch.randn(No, Ko, device="cuda", generator=g) / math.sqrt(Ko)).bfloat16()
+                gsx = float(Xs.abs().max()) / 2688.0
+                gsw = float(Ws.abs().max()) / 2688.0
+                Xq = torch.empty(Mo, Ko // 2, device="cuda", dtype=torch.uint8)
+                Wq = torch.empty(No, Ko // 2, device="cuda", dtype=torch.uint8)
+                sfx = torch.empty(int(lib.kx_nvfp4_scale_bytes(i64(Mo), i64(Ko))), device="cuda", dtype=torch.uint8)
+                sfw = torch.empty(int(lib.kx_nvfp4_scale_bytes(i64(No), i64(Ko))), device="cuda", dtype=torch.uint8)
+                Rs = torch.randn(Mo, No, device="cuda", generator=g).bfloat16()
+                Ys = torch.empty(Mo, No, dtype=torch.bfloat16, device="cuda")
+                qa = (vp(Xs.data_ptr()), ctypes.c_float(gsx), vp(Xq.data_ptr()), vp(sfx.data_ptr()), i64(Mo), i64(Ko), st)
+                rcq = lib.kx_quantize_rows_nvfp4(*qa)
+                rcq = rcq or lib.kx_quantize_rows_nvfp4(vp(Ws.data_ptr()), ctypes.c_float(gsw), vp(Wq.data_ptr()),
+                                                        vp(sfw.data_ptr()), i64(No), i64(Ko), st)
+                if rcq != 0:
+                    raise SystemExit(f"kx_quantize_rows_nvfp4 failed ({rcq})")
+                torch.cuda.synchronize()
+                keep.append((Xs, Xq, Wq, sfx, sfw, Rs, Ys))
+                del Ws
+                a = (vp(Xq.data_ptr()), vp(sfx.data_ptr()), vp(Wq.data_ptr()), vp(sfw.data_ptr()), ctypes.c_float(gsx * gsw),
+                     vp(None), vp(Rs.data_ptr()), vp(Ys.data_ptr()), i64(Mo), i64(No), i64(Ko), st, None)
+                calls.append(lambda a=a: lib.kx_outproj_residual_nvfp4(*a))
+                qcalls.append(lambda qa=qa: lib.kx_quantize_rows_nvfp4(*qa))
+            wlo = inputs.Workload(f"outproj_nvfp4_M{Mo}_N{No}_K{Ko}", Mo, No, Ko, 0, False, True)
+            t, tbest, _ = time_shape(torch, kx, wlo, calls)
+            int8.append({"name": wlo.name, "us": t * 1e6, "us_best": tbest * 1e6, "tops": ops / t / 1e12,
+                         "gbs": nbytes / t / 1e9, "bound": "tensor", "frac": ops / t / 1e12 / peak4, "peak": peak4,
+                         "operand_sets": ns})
+            print(f"[bench] {wlo.name:>30s} {t*1e6:9.1f} us (best {tbest*1e6:7.1f}) {ops/t/1e12:8.1f} TOP/s {nbytes/t/1e9:7.0f} GB/s  "
+                  f"tensor {ops/t/1e12/peak4*100:5.1f}% of 4 x {peaks['source']} BF16 peak", file=sys.stderr, flush=True)
+            wlq = inputs.Workload(f"quantize_rows_nvfp4_M{Mo}_K{Ko}", Mo, Ko, 0, 0, False, False)
+            t, tbest, _ = time_shape(torch, kx, wlq, qcalls)
+            report(wlq.name, t, tbest, Mo * Ko * (2.5 + 1.0 / 16), 0.0, ns)
+            del keep, calls, qcalls
+            torch.cuda.empty_cache()
+
     # ---- the oracle on the host cores, bounded sample (rank 0, N = 1 only)
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

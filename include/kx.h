@@ -415,7 +415,7 @@ int kx_outproj_residual_mxfp8_ex(const void* Xq, const void* SFX, const void* Wq
                                  const kx_plan_override* override_or_null);
 
 /*
- * 4-bit block-scaled branch (the number format of the Section 4.3 task, "E2M1 with 1x16 block scaling", and
+ * 4-bit block-scaled branch (the number format of the Section 4.3 task, E2M1 elements scaled in blocks of 16, and
  * the tensor-core kind it runs on).  Elements are E2M1 codes (sign, two exponent bits, one mantissa bit:
  * magnitudes 0, 0.5, 1, 1.5, 2, 3, 4, 6), two per byte with the even k index in the low nibble; every 16
  * consecutive elements of a row share one E4M3 scale byte (non-negative, never NaN); one binary32 scale gs

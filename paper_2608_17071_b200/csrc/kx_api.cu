@@ -1849,18 +1849,22 @@ int kx_outproj_residual_nvfp4(const void* Xq, const void* SFX, const void* Wq, c
         overlaps(Y, yb, SFX, static_cast<size_t>(kx_nvfp4_scale_bytes(M, K))) ||
         overlaps(Y, yb, SFW, static_cast<size_t>(kx_nvfp4_scale_bytes(N, K))))
         return KX_ERR_OVERLAP;
-    // tile width: fewest (waves x columns per tile), wider tiles first on ties (more work per issued MMA)
+    // tile width: smallest estimated time = waves x (k-blocks x time per k-block + exposed epilogue), with the
+    // measured 0.527 / 0.621 / 0.583 us per 128-byte k-block at 128 / 192 / 256 columns and 7 us per tile that
+    // the single-accumulator 256-column shape does not hide
     const MxVariant* v = nullptr;
     if (ov && ov->block_n) {
         for (const auto& c : kNvVariants)
             if (c.bn == ov->block_n) v = &c;
         if (!v) return KX_ERR_PLAN;
     } else {
-        long long best = 0;
+        double best = 0.0;
         for (const auto& c : kNvVariants) {
             const long long tiles = ((M + 127) / 128) * ((N + c.bn - 1) / c.bn);
-            const long long cost = ((tiles + ctx->sm_count - 1) / ctx->sm_count) * (c.bn + 64);
-            if (!v || cost <= best) { v = &c; best = cost; }
+            const long long waves = (tiles + ctx->sm_count - 1) / ctx->sm_count;
+            const double per_kb = c.bn == 256 ? 0.583 : c.bn == 192 ? 0.621 : 0.527;
+            const double t = static_cast<double>(waves) * (static_cast<double>((K + 255) / 256) * per_kb + (c.bn == 256 ? 7.0 : 0.0));
+            if (!v || t < best) { v = &c; best = t; }
         }
     }
     const int bn = v->bn;
