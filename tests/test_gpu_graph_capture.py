@@ -159,3 +159,48 @@ def test_capture_and_replay_the_block_scaled_branch():
         assert kx.kx_last_device_status()[0] == kx.KX_OK
         for got, ref in zip(outs, want):
             assert np.array_equal(raw(got), ref)
+
+
+def test_capture_and_replay_the_4bit_branch():
+    """4-bit code books -> 4-bit block-scaled projection with residual, captured and replayed: same bits."""
+    import torch
+    kx.kx_init(torch.cuda.current_device())
+    M, N, K = 384, 1160, 1024
+    X = kt.to_dev(inputs.normal_bf16(531, "X", (M, K), 1.0))
+    W = kt.to_dev(inputs.normal_bf16(532, "W", (N, K), 1.0 / np.sqrt(K)))
+    R = kt.to_dev(inputs.normal_bf16(533, "R", (M, N), 1.0))
+    gsx, gsw = 6.0 / 2688.0, 0.2 / 2688.0
+    u8 = lambda *shape: torch.zeros(shape, dtype=torch.uint8, device="cuda")
+
+    def branch(Xq, SFX, Wq, SFW, Y):
+        kx.kx_quantize_rows_nvfp4(X, gsx, Xq, SFX)
+        kx.kx_quantize_rows_nvfp4(W, gsw, Wq, SFW)
+        kx.kx_outproj_residual_nvfp4(Xq, SFX, Wq, SFW, gsx * gsw, None, R, Y)
+
+    def bufs():
+        return [u8(M, K // 2), u8(kx.kx_nvfp4_scale_bytes(M, K)), u8(N, K // 2), u8(kx.kx_nvfp4_scale_bytes(N, K)),
+                kt.nan_filled(M, N)]
+
+    raw = lambda t: kt.from_dev(t) if t.dtype == torch.bfloat16 else t.cpu().numpy()
+    eager = bufs()
+    branch(*eager)
+    assert kx.kx_last_device_status()[0] == kx.KX_OK
+    want = [raw(t) for t in eager]
+    assert want[0].any() and not np.isnan(oracle.widen_bf16(want[4])).any()
+    outs = bufs()
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(s):
+        branch(*outs)
+        torch.cuda.synchronize()
+        with torch.cuda.graph(graph, stream=s):
+            branch(*outs)
+    for rep in range(2):
+        for t in outs:
+            t.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert kx.kx_last_device_status()[0] == kx.KX_OK
+        for got, ref in zip(outs, want):
+            assert np.array_equal(raw(got), ref)

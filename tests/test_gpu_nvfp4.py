@@ -127,6 +127,29 @@ def test_nvfp4_projection_exact_on_small_values(variant, M, N, K):
     assert ok, msg
 
 
+@pytest.mark.parametrize("chunk", range(3))
+def test_nvfp4_random_shapes_and_tile_shapes_are_exact(chunk):
+    """Seeded random (M, N, K, tile shape, bias / residual / in place) cases of the exact-sum construction."""
+    rng = np.random.default_rng(9700 + chunk)
+    for case in range(12):
+        M = int(rng.choice([1, 5, 64, 127, 128, 129, 200, 256, 300, 513, 700, 1024]))
+        N = 8 * int(rng.integers(1, 160))
+        K = 32 * int(rng.integers(1, 40))
+        variant = VARIANTS[int(rng.integers(0, len(VARIANTS)))] if rng.integers(0, 4) else None
+        nb = K // 16
+        Xq, Wq = pack(small_codes(rng.integers(1 << 30), (M, K))), pack(small_codes(rng.integers(1 << 30), (N, K)))
+        sx = np.array([0x30, 0x38, 0x40], np.uint8)[rng.integers(0, 3, size=(M, nb))]
+        sw = np.array([0x28, 0x30, 0x38], np.uint8)[rng.integers(0, 3, size=(N, nb))]
+        b = inputs.small_int_bf16(971 + case, "bias", (N,), -4, 4) if rng.integers(0, 2) else None
+        R = inputs.small_int_bf16(972 + case, "R", (M, N), -8, 8) if rng.integers(0, 2) else None
+        inplace = R is not None and bool(rng.integers(0, 2))
+        alpha = float(rng.choice([0.25, 0.5, 1.0, 2.0]))
+        ref = oracle.outproj_nvfp4(Xq, sx, Wq, sw, alpha, b, R)
+        y = run_proj(Xq, sx, Wq, sw, alpha, b, R.copy() if inplace else R, inplace=inplace, variant=variant)
+        ok, msg = kt.gate_exact(y, ref)
+        assert ok, (M, N, K, variant, alpha, b is not None, R is not None, inplace, msg)
+
+
 @pytest.mark.parametrize("M,N,K", [(300, 520, 288), (1000, 776, 1056), (2500, 3080, 4096)])
 def test_nvfp4_projection_realistic_codes(M, N, K):
     X = inputs.normal_bf16(1120 + M, "X", (M, K), 1.0)
