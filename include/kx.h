@@ -396,10 +396,11 @@ int kx_outproj_residual_fp8(const void* Xq, const float* sx, const void* Wq, con
  * kx_outproj_residual_mxfp8:
  *     Y[m,n] = bf16( sum_j 2^(ex[m,j]-127) 2^(ew[n,j]-127) sum_{k in block j} xq[m,k] wq[n,k] + bias[n] + R[m,n] )
  * Xq [M,K], Wq [N,K] E4M3 bytes, K contiguous; K % 32 == 0, N % 8 == 0; bias / R / Y as in
- * kx_outproj_residual (R may be Y).  Tiles of 128 or 192 columns by 128 rows (one CTA) or 256 rows
- * (a CTA pair), FP32 accumulation in tensor memory, tolerance as for the BF16 path against the
- * exact value of the formula.  The _ex form takes a plan override of which block_n (128 / 192),
- * cta_pair (1 / 2) and raster_group are honoured (tests, tuning); NULL = automatic.
+ * kx_outproj_residual (R may be Y).  Tiles of 128, 192 or 256 columns by 128 rows (one CTA), or of 128 / 192
+ * columns by 256 rows (a CTA pair), FP32 accumulation in tensor memory, tolerance as for the BF16 path
+ * against the exact value of the formula.  The _ex form takes a plan override of which block_n
+ * (128 / 192 / 256), cta_pair (1 / 2) and raster_group are honoured (tests, tuning); NULL = automatic
+ * (single-CTA tiles, width by an estimate of waves x time per tile).
  * Errors: KX_ERR_SHAPE, KX_ERR_NULL, KX_ERR_ALIGN, KX_ERR_OVERLAP as for the calls above.
  */
 int64_t kx_mx_scale_bytes(int64_t rows, int64_t cols);
