@@ -291,3 +291,43 @@ def test_mx_edges_and_argument_checks():
     assert lib.kx_quantize_rows_mxfp8(A.data_ptr(), Q.data_ptr(), SF.data_ptr(), 1, 32768 + 32, None) == kx.KX_ERR_SHAPE
     assert lib.kx_rmsnorm_quantize_mxfp8(A.data_ptr(), None, 1e-6, Q.data_ptr(), SF.data_ptr(), 8, 64, None) == kx.KX_ERR_NULL
     status_ok()
+
+
+@pytest.mark.parametrize("M,N,K", [(4096, 4096, 4096), (16384, 4096, 14336)])
+def test_mx_projection_full_sizes_sampled_rows(M, N, K):
+    """The two projection shapes bench.py times for the block-scaled kind, in that launch configuration:
+    exact on the small-value construction (block scales {1/2, 1} x {1/4, 1/2}: every partial sum stays an
+    exactly representable multiple of 2^-5), then device-made code books of normal data with a residual
+    within the gates; sampled rows."""
+    rng = np.random.default_rng(980)
+    nb = K // 32
+    Xq, Wq = small_codes(981, (M, K)), small_codes(982, (N, K))
+    ex = rng.integers(126, 128, size=(M, nb), dtype=np.uint8)
+    ew = rng.integers(125, 127, size=(N, nb), dtype=np.uint8)
+    rows = inputs.sampled_rows(M)[::8]
+    Y = kt.nan_filled(M, N)
+    kx.kx_outproj_residual_mxfp8(dev8(Xq), dev(chunked(ex, K)), dev8(Wq), dev(chunked(ew, K)), None, None, Y)
+    status_ok()
+    y = kt.from_dev(Y)
+    assert not np.isnan(oracle.widen_bf16(y)).any()
+    ok, msg = kt.gate_exact(y[rows], oracle.outproj_mx(Xq, ex, Wq, ew, rows=rows))
+    assert ok, msg
+    X = inputs.normal_bf16(983, "X", (M, K), 1.0)
+    W = inputs.normal_bf16(984, "W", (N, K), 1.0 / np.sqrt(K))
+    R = inputs.normal_bf16(985, "R", (M, N), 1.0)
+    Xd = torch.empty((M, K), dtype=torch.uint8, device="cuda").view(F8)
+    Wd = torch.empty((N, K), dtype=torch.uint8, device="cuda").view(F8)
+    SFX = torch.empty((kx.kx_mx_scale_bytes(M, K),), dtype=torch.uint8, device="cuda")
+    SFW = torch.empty((kx.kx_mx_scale_bytes(N, K),), dtype=torch.uint8, device="cuda")
+    kx.kx_quantize_rows_mxfp8(kt.to_dev(X), Xd, SFX)
+    kx.kx_quantize_rows_mxfp8(kt.to_dev(W), Wd, SFW)
+    kx.kx_outproj_residual_mxfp8(Xd, SFX, Wd, SFW, None, kt.to_dev(R), Y)
+    status_ok()
+    y = kt.from_dev(Y)
+    xq, ex2 = oracle.quantize_rows_mx(X)
+    wq, ew2 = oracle.quantize_rows_mx(W)
+    assert np.array_equal(host8(Xd)[rows], xq[rows]) and np.array_equal(SFW.cpu().numpy(), chunked(ew2, K))
+    ref = oracle.outproj_mx(xq, ex2, wq, ew2, None, R, rows=rows)
+    ok, msg = kt.gate_a(y[rows], ref)
+    assert ok, msg
+    assert kt.rel_fro(y[rows], ref) <= 2.0 ** -8

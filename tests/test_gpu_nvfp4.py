@@ -229,3 +229,45 @@ def test_nvfp4_edges_and_argument_checks():
     assert lib.kx_quantize_rows_nvfp4(A.data_ptr(), 1.0, None, SF.data_ptr(), 8, 64, None) == kx.KX_ERR_NULL
     assert lib.kx_quantize_rows_nvfp4(A.data_ptr(), 1.0, Q.data_ptr(), SF.data_ptr(), 0, 64, None) == kx.KX_OK
     status_ok()
+
+
+@pytest.mark.parametrize("M,N,K", [(4096, 4096, 4096), (16384, 4096, 14336)])
+def test_nvfp4_projection_full_sizes_sampled_rows(M, N, K):
+    """The two projection shapes bench.py times for the 4-bit kind, in that launch configuration: exact on
+    the small-value construction (block scales {1/2, 1} x {1/4, 1/2}), then device-made code books of normal
+    data with a residual within the gates; sampled rows."""
+    rng = np.random.default_rng(1180)
+    nb = K // 16
+    Xq, Wq = pack(small_codes(1181, (M, K))), pack(small_codes(1182, (N, K)))
+    sx = np.array([0x30, 0x38], np.uint8)[rng.integers(0, 2, size=(M, nb))]
+    sw = np.array([0x28, 0x30], np.uint8)[rng.integers(0, 2, size=(N, nb))]
+    rows = inputs.sampled_rows(M)[::8]
+    Y = kt.nan_filled(M, N)
+    kx.kx_outproj_residual_nvfp4(dev(Xq), dev(chunked(sx, K)), dev(Wq), dev(chunked(sw, K)), 1.0, None, None, Y)
+    status_ok()
+    y = kt.from_dev(Y)
+    assert not np.isnan(oracle.widen_bf16(y)).any()
+    ok, msg = kt.gate_exact(y[rows], oracle.outproj_nvfp4(Xq, sx, Wq, sw, 1.0, rows=rows))
+    assert ok, msg
+    X = inputs.normal_bf16(1183, "X", (M, K), 1.0)
+    W = inputs.normal_bf16(1184, "W", (N, K), 1.0 / np.sqrt(K))
+    R = inputs.normal_bf16(1185, "R", (M, N), 1.0)
+    gsx = float(np.float32(np.abs(inputs.bf16_bits_to_f32(X)).max() / 2688.0))
+    gsw = float(np.float32(np.abs(inputs.bf16_bits_to_f32(W)).max() / 2688.0))
+    alpha = float(np.float32(gsx) * np.float32(gsw))
+    Xd = torch.empty((M, K // 2), dtype=torch.uint8, device="cuda")
+    Wd = torch.empty((N, K // 2), dtype=torch.uint8, device="cuda")
+    SFX = torch.empty((kx.kx_nvfp4_scale_bytes(M, K),), dtype=torch.uint8, device="cuda")
+    SFW = torch.empty((kx.kx_nvfp4_scale_bytes(N, K),), dtype=torch.uint8, device="cuda")
+    kx.kx_quantize_rows_nvfp4(kt.to_dev(X), gsx, Xd, SFX)
+    kx.kx_quantize_rows_nvfp4(kt.to_dev(W), gsw, Wd, SFW)
+    kx.kx_outproj_residual_nvfp4(Xd, SFX, Wd, SFW, alpha, None, kt.to_dev(R), Y)
+    status_ok()
+    y = kt.from_dev(Y)
+    xq, sx2 = oracle.quantize_rows_nvfp4(X, gsx)
+    wq, sw2 = oracle.quantize_rows_nvfp4(W, gsw)
+    assert np.array_equal(Xd.cpu().numpy()[rows], xq[rows]) and np.array_equal(SFW.cpu().numpy(), chunked(sw2, K))
+    ref = oracle.outproj_nvfp4(xq, sx2, wq, sw2, alpha, None, R, rows=rows)
+    ok, msg = kt.gate_a(y[rows], ref)
+    assert ok, msg
+    assert kt.rel_fro(y[rows], ref) <= 2.0 ** -8
