@@ -419,3 +419,12 @@ def outproj_nvfp4(Xq, sx, Wq, sw, alpha: float, bias=None, R=None, rows=None):
     if rc != 0:
         raise RuntimeError(f"kx_oracle_outproj_nvfp4_rows failed ({rc})")
     return out
+
+
+def swiglu_mx(Xq, ex, Wgq, eg, Wuq, eu, rows=None):
+    """z = silu(g) * u with g, u the block-scaled FP8 products of Xq with the gate and the up weights (the
+    gate/up step of Appendix A, Algorithm 7, on block-scaled operands); float64, unrounded.  Two calls of
+    the block-scaled projection and the activation written out."""
+    g = outproj_mx(Xq, ex, Wgq, eg, rows=rows)
+    u = outproj_mx(Xq, ex, Wuq, eu, rows=rows)
+    return g / (1.0 + np.exp(-g)) * u

@@ -168,3 +168,23 @@ def test_mx_projection_equals_bf16_projection():
     ex3[3, 0] = 0xFF
     y = oracle.outproj_mx(Xq, ex3, Wq, ew)
     assert np.isnan(y[3]).all() and not np.isnan(y[[0, 1, 2, 4]]).any()
+
+
+def test_mx_swiglu_equals_bf16_swiglu():
+    """On operands the BF16 format represents exactly, the (separately pinned) BF16 SwiGLU oracle must agree;
+    gate and up are not interchangeable."""
+    M, I, K = 5, 9, 96
+    Xq, ex, Wgq, eg = mx_case(M, I, K, 8)
+    _, _, Wuq, eu = mx_case(M, I, K, 9)
+    Xq &= 0xB7                      # |x| < 1
+    ex[:] = 127
+    X = bits(oracle.e4m3_decode(Xq) * np.repeat(oracle.e8m0_decode(ex), 32, axis=1))
+    Wg = bits(oracle.e4m3_decode(Wgq) * np.repeat(oracle.e8m0_decode(eg), 32, axis=1))
+    Wu = bits(oracle.e4m3_decode(Wuq) * np.repeat(oracle.e8m0_decode(eu), 32, axis=1))
+    z = oracle.swiglu_mx(Xq, ex, Wgq, eg, Wuq, eu)
+    zw, g, u = oracle.swiglu(X, Wg, Wu, want_parts=True)
+    assert np.max(np.abs(z - zw)) <= 1e-13 * max(1.0, np.abs(zw).max())
+    assert np.abs(g).max() > 0.3
+    assert not np.allclose(oracle.swiglu_mx(Xq, ex, Wuq, eu, Wgq, eg), z)
+    rows = np.array([4, 1])
+    assert np.array_equal(oracle.swiglu_mx(Xq, ex, Wgq, eg, Wuq, eu, rows=rows), z[rows])
