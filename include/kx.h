@@ -410,6 +410,16 @@ int kx_rmsnorm_quantize_mxfp8(const void* H, const void* gamma, float eps, void*
 int kx_outproj_residual_mxfp8(const void* Xq, const void* SFX, const void* Wq, const void* SFW,
                               const void* bias_or_null, const void* R_or_null, void* Y,
                               int64_t M, int64_t N, int64_t K, void* stream);
+/* Block-scaled gate/up step: kx_quantize_gate_up_mxfp8 writes the code books of the gate and the up weights
+ * (Wg, Wu [I, K] BF16 -> Qg, Qu [I, K] codes) and their scale arrays back to back into SFGU (gate first;
+ * 2 * kx_mx_scale_bytes(I, K) bytes).  kx_gate_up_swiglu_mxfp8 computes
+ *     Z[m,i] = bf16( silu(g) * u ),  g / u = the block-scaled products of row m of Xq with row i of Wgq / Wuq
+ * (Appendix A, Algorithm 7's gate/up GEMM with SwiGLU epilogue on block-scaled operands).  K % 32 == 0,
+ * I % 8 == 0; Z [M, I] BF16; no bias, no residual; pointers and errors as above. */
+int kx_quantize_gate_up_mxfp8(const void* Wg, const void* Wu, void* Qg, void* Qu, void* SFGU,
+                              int64_t I, int64_t K, void* stream);
+int kx_gate_up_swiglu_mxfp8(const void* Xq, const void* SFX, const void* Wgq, const void* Wuq, const void* SFGU,
+                            void* Z, int64_t M, int64_t I, int64_t K, void* stream);
 int kx_outproj_residual_mxfp8_ex(const void* Xq, const void* SFX, const void* Wq, const void* SFW,
                                  const void* bias_or_null, const void* R_or_null, void* Y,
                                  int64_t M, int64_t N, int64_t K, void* stream,

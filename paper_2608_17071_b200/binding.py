@@ -30,6 +30,7 @@ EXPORTS = (
     "kx_quantize_rows_fp8", "kx_quantize_gate_up_fp8", "kx_rmsnorm_quantize_fp8", "kx_gate_up_swiglu_fp8",
     "kx_outproj_residual_fp8",
     "kx_mx_scale_bytes", "kx_quantize_rows_mxfp8", "kx_rmsnorm_quantize_mxfp8", "kx_outproj_residual_mxfp8", "kx_outproj_residual_mxfp8_ex",
+    "kx_quantize_gate_up_mxfp8", "kx_gate_up_swiglu_mxfp8",
     "kx_nvfp4_scale_bytes", "kx_quantize_rows_nvfp4", "kx_outproj_residual_nvfp4",
     "kx_plan_query", "kx_last_device_status", "kx_status_string",
     "kx_version",
@@ -103,6 +104,8 @@ def load():
     lib.kx_rmsnorm_quantize_mxfp8.argtypes = [vp, vp, ctypes.c_float, vp, vp, i64, i64, vp]
     lib.kx_outproj_residual_mxfp8.argtypes = [vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, vp]
     lib.kx_outproj_residual_mxfp8_ex.argtypes = [vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, vp, ctypes.POINTER(PlanOverride)]
+    lib.kx_quantize_gate_up_mxfp8.argtypes = [vp, vp, vp, vp, vp, i64, i64, vp]
+    lib.kx_gate_up_swiglu_mxfp8.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, vp]
     lib.kx_nvfp4_scale_bytes.argtypes = [i64, i64]
     lib.kx_quantize_rows_nvfp4.argtypes = [vp, ctypes.c_float, vp, vp, i64, i64, vp]
     lib.kx_outproj_residual_nvfp4.argtypes = [vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, i64, i64, i64, vp,
@@ -543,6 +546,34 @@ def kx_outproj_residual_mxfp8(Xq, SFX, Wq, SFW, bias, R, Y, stream=None, check=T
                                                  _addr(Y), M, N, K, _stream(stream), ctypes.byref(override))
     if check and rc != KX_OK:
         raise KxError(rc, "kx_outproj_residual_mxfp8")
+    return rc
+
+
+def kx_quantize_gate_up_mxfp8(Wg, Wu, Qg, Qu, SFGU, stream=None, check=True) -> int:
+    """Block-scaled code books of the gate and the up weights; SFGU = gate scales followed by up scales."""
+    import torch
+    I, K = Wg.shape
+    _check_bf16("Wg", Wg, (I, K)); _check_bf16("Wu", Wu, (I, K))
+    _check("Qg", Qg, (I, K), torch.float8_e4m3fn); _check("Qu", Qu, (I, K), torch.float8_e4m3fn)
+    _check("SFGU", SFGU, (2 * kx_mx_scale_bytes(I, K),), torch.uint8)
+    rc = load().kx_quantize_gate_up_mxfp8(_addr(Wg), _addr(Wu), _addr(Qg), _addr(Qu), _addr(SFGU), I, K, _stream(stream))
+    if check and rc != KX_OK:
+        raise KxError(rc, "kx_quantize_gate_up_mxfp8")
+    return rc
+
+
+def kx_gate_up_swiglu_mxfp8(Xq, SFX, Wgq, Wuq, SFGU, Z, stream=None, check=True) -> int:
+    """Z = silu(g) * u on block-scaled FP8 operands (g / u = products of Xq with the gate / up weights)."""
+    import torch
+    M, K = Xq.shape
+    I = Wgq.shape[0]
+    _check("Xq", Xq, (M, K), torch.float8_e4m3fn); _check("Wgq", Wgq, (I, K), torch.float8_e4m3fn)
+    _check("Wuq", Wuq, (I, K), torch.float8_e4m3fn); _check("SFX", SFX, (kx_mx_scale_bytes(M, K),), torch.uint8)
+    _check("SFGU", SFGU, (2 * kx_mx_scale_bytes(I, K),), torch.uint8); _check_bf16("Z", Z, (M, I))
+    rc = load().kx_gate_up_swiglu_mxfp8(_addr(Xq), _addr(SFX), _addr(Wgq), _addr(Wuq), _addr(SFGU), _addr(Z), M, I, K,
+                                        _stream(stream))
+    if check and rc != KX_OK:
+        raise KxError(rc, "kx_gate_up_swiglu_mxfp8")
     return rc
 
 

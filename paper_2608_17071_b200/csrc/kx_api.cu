@@ -1789,6 +1789,104 @@ int kx_outproj_residual_mxfp8_ex(const void* Xq, const void* SFX, const void* Wq
     return outproj_residual_mx(Xq, SFX, Wq, SFW, bias, R, Y, M, N, K, stream, ov);
 }
 
+// Code books of the gate and the up weights; their scale arrays are written back to back (gate first), the
+// layout kx_gate_up_swiglu_mxfp8 reads.
+int kx_quantize_gate_up_mxfp8(const void* Wg, const void* Wu, void* Qg, void* Qu, void* SFGU, int64_t I, int64_t K,
+                              void* stream) {
+    if (I < 0 || K < 0) return KX_ERR_SHAPE;
+    const int64_t half = kx_mx_scale_bytes(I, K);
+    if (I > 0 && K > 0 && !SFGU) return KX_ERR_NULL;
+    const size_t qb = static_cast<size_t>(I) * K;
+    if (I > 0 && K > 0 && (overlaps(Qg, qb, Qu, qb) || overlaps(Qg, qb, Wu, qb * 2) || overlaps(Qu, qb, Wg, qb * 2) ||
+                           overlaps(SFGU, static_cast<size_t>(2 * half), Wg, qb * 2) ||
+                           overlaps(SFGU, static_cast<size_t>(2 * half), Wu, qb * 2) ||
+                           overlaps(SFGU, static_cast<size_t>(2 * half), Qg, qb) ||
+                           overlaps(SFGU, static_cast<size_t>(2 * half), Qu, qb)))
+        return KX_ERR_OVERLAP;
+    int rc = quantize_rows_mx(Wg, nullptr, 0.0f, Qg, SFGU, I, K, stream);
+    if (rc != KX_OK) return rc;
+    return quantize_rows_mx(Wu, nullptr, 0.0f, Qu, static_cast<uint8_t*>(SFGU) + half, I, K, stream);
+}
+
+// Z = silu(g) * u, g / u = block-scaled products of Xq with the gate / up weights: the 256-column single-CTA tile
+// kernel in gate/up mode (128 gate + 128 up accumulator columns = 128 output columns per tile).
+int kx_gate_up_swiglu_mxfp8(const void* Xq, const void* SFX, const void* Wgq, const void* Wuq, const void* SFGU, void* Z,
+                            int64_t M, int64_t I, int64_t K, void* stream_v) {
+    if (M < 0 || I < 0 || K < 0) return KX_ERR_SHAPE;
+    if (M > 0x7FFFFFFFll / 2 || I > 0x7FFFFFFFll / 4 || K > 0x7FFFFFFFll / 2) return KX_ERR_SHAPE;
+    if (M == 0 || I == 0) return KX_OK;
+    if ((I % 8) != 0 || (K % 32) != 0) return KX_ERR_SHAPE;
+    if (!Z) return KX_ERR_NULL;
+    if (!aligned16(Z)) return KX_ERR_ALIGN;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    DeviceCtx* ctx = nullptr;
+    int rc = device_ctx(&ctx);
+    if (rc != KX_OK) return rc;
+    if (K == 0) {   // empty sums: silu(0) * 0 = 0
+        const long long total = M * I;
+        const int blocks = static_cast<int>(std::min<long long>((total + 255) / 256, ctx->sm_count * 8));
+        kx_k0_kernel<<<blocks, 256, 0, stream>>>(nullptr, nullptr, static_cast<uint16_t*>(Z), M, I, I, I);
+        return cudaGetLastError() == cudaSuccess ? KX_OK : KX_ERR_CUDA;
+    }
+    if (!Xq || !Wgq || !Wuq || !SFX || !SFGU) return KX_ERR_NULL;
+    if (!aligned16(Xq) || !aligned16(Wgq) || !aligned16(Wuq) || !aligned16(SFX) || !aligned16(SFGU)) return KX_ERR_ALIGN;
+    const size_t zb = static_cast<size_t>(M) * I * 2, wb = static_cast<size_t>(I) * K;
+    if (overlaps(Z, zb, Xq, static_cast<size_t>(M) * K) || overlaps(Z, zb, Wgq, wb) || overlaps(Z, zb, Wuq, wb) ||
+        overlaps(Z, zb, SFX, static_cast<size_t>(kx_mx_scale_bytes(M, K))) ||
+        overlaps(Z, zb, SFGU, static_cast<size_t>(2 * kx_mx_scale_bytes(I, K))))
+        return KX_ERR_OVERLAP;
+    const MxVariant* v = find_mx(256, 1);
+    if (!v) return KX_ERR_PLAN;
+    const long long tm = (M + 127) / 128, tiles_n = (I + 127) / 128, tiles = tm * tiles_n;
+    if (tiles > 0x7FFFFFFFll / 4) return KX_ERR_SHAPE;
+    const long long kchunks = mx_chunks(K);
+    CUtensorMap tmA, tmG, tmU, tmZ, tmSA, tmSB;
+    if ((rc = get_tmap(Xq, M, K, 128, &tmA, 1)) != KX_OK) return rc;
+    if ((rc = get_tmap(Wgq, I, K, 128, &tmG, 1)) != KX_OK) return rc;
+    if ((rc = get_tmap(Wuq, I, K, 128, &tmU, 1)) != KX_OK) return rc;
+    if ((rc = get_tmap_scales(SFX, mx_chunks(M) * kchunks, &tmSA)) != KX_OK) return rc;
+    if ((rc = get_tmap_scales(SFGU, 2 * mx_chunks(I) * kchunks, &tmSB)) != KX_OK) return rc;
+    if ((rc = get_tmap(Z, M, I, 32, &tmZ)) != KX_OK) return rc;
+    TileParams p;
+    std::memset(&p, 0, sizeof p);
+    p.M = static_cast<int>(M);
+    p.N = static_cast<int>(I);
+    p.K = static_cast<int>(K);
+    p.tiles_m = static_cast<int>(tm);
+    p.tiles_n = static_cast<int>(tiles_n);
+    p.num_tiles = static_cast<int>(tiles);
+    p.raster_group = 8;
+    p.swiglu = 1;
+    p.kcluster = 1;
+    p.sk_tile0 = p.num_tiles;
+    p.narrow_tile0 = p.num_tiles;
+    p.spin_limit_ns = 2000000000ull;
+    p.status = ctx->status;
+    p.ws = ctx->ws;
+    p.counters = ctx->counters;
+    p.sfb_chunks = static_cast<int>(mx_chunks(I));
+    cudaLaunchConfig_t cfg;
+    std::memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3(static_cast<unsigned>(std::min<long long>(tiles, ctx->sm_count)), 1, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = v->smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const uint16_t* bias_p = nullptr;
+    // gate/up mode of the block-scaled kind: tmB = gate weights, tmB2 = up weights, tmR = scales of X, tmS = scales of
+    // the gate rows followed by those of the up rows
+    void* args[] = {&tmA, &tmG, &tmU, &tmZ, &tmSA, &tmSB, &bias_p, &p};
+    if (cudaLaunchKernelExC(&cfg, v->fn, args) != cudaSuccess) {
+        cudaGetLastError();
+        return KX_ERR_CUDA;
+    }
+    return KX_OK;
+}
+
 // ---------------------------------------------------------------- 4-bit block-scaled branch
 int64_t kx_nvfp4_scale_bytes(int64_t rows, int64_t cols) {
     if (rows < 0 || cols < 0) return -1;

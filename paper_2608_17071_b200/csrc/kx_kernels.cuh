@@ -407,15 +407,21 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         // scale chunks of this CTA's A rows and of all the tile's B rows for k-block kb:
                         // chunk (row / 128, kb).  A B chunk past the end of the array (ragged last tile) is
                         // replaced by the last one: its rows belong to zero-filled operand rows.
-                        const int c0 = col >> 7;
+                        // Gate/up mode (one CTA per tile, 256 accumulator columns): the tile's 128 gate rows and
+                        // 128 up rows are one aligned chunk each; the up scales follow the gate scales in the
+                        // same array (sfb_chunks chunk rows further), and the A scales come through tmR (unused
+                        // otherwise: no residual in this mode) because tmB2 carries the up weights.
+                        const int c0 = sg ? (col >> 8) : (col >> 7);
+                        const CUtensorMap* const mapSA = sg ? &tmR : &tmB2;
                         const uint32_t fb = (CTAS == 1) ? full(s) : map_to_cta(full(s), 0);
                         for (int j = 0; j < nsub; ++j) {
                             const uint32_t dst = s_sf + s * C::SF_STAGE + j * C::SF_KB_BYTES;
                             const int ya = (tm * CTAS + static_cast<int>(cta_rank)) * nkb + kb + j;
-                            if constexpr (CTAS == 1) tma_load_2d(dst, &tmB2, 0, ya, fb);
-                            else tma_load_2d_pair(dst, &tmB2, 0, ya, fb);
+                            if constexpr (CTAS == 1) tma_load_2d(dst, mapSA, 0, ya, fb);
+                            else tma_load_2d_pair(dst, mapSA, 0, ya, fb);
                             for (int i = 0; i < C::SFB_CHUNKS; ++i) {
-                                const int yb = min(c0 + i, p.sfb_chunks - 1) * nkb + kb + j;
+                                const int ch = sg ? (i == 0 ? c0 : p.sfb_chunks + c0) : min(c0 + i, p.sfb_chunks - 1);
+                                const int yb = ch * nkb + kb + j;
                                 if constexpr (CTAS == 1) tma_load_2d(dst + 512 * (1 + i), &tmS, 0, yb, fb);
                                 else tma_load_2d_pair(dst + 512 * (1 + i), &tmS, 0, yb, fb);
                             }

@@ -331,3 +331,95 @@ def test_mx_projection_full_sizes_sampled_rows(M, N, K):
     ok, msg = kt.gate_a(y[rows], ref)
     assert ok, msg
     assert kt.rel_fro(y[rows], ref) <= 2.0 ** -8
+
+
+# ------------------------------------------------------------------ gate/up + SwiGLU
+def run_swiglu(Xq, ex, Wgq, eg, Wuq, eu):
+    (M, K), I = Xq.shape, Wgq.shape[0]
+    Z = kt.nan_filled(M, I)
+    sfgu = np.concatenate([chunked(eg, K), chunked(eu, K)])
+    kx.kx_gate_up_swiglu_mxfp8(dev8(Xq), dev(chunked(ex, K)), dev8(Wgq), dev8(Wuq), dev(sfgu), Z)
+    status_ok()
+    return kt.from_dev(Z)
+
+
+def check_swiglu(z_bits, ref):
+    ok, msg = kt.gate_a(z_bits, ref)
+    assert ok, msg
+    assert kt.rel_fro(z_bits, ref) <= 2.0 ** -8
+    z = oracle.widen_bf16(z_bits)
+    assert (np.abs(z - ref) <= 2.0 ** -7 * np.abs(ref) + 2e-3).all()
+
+
+@pytest.mark.parametrize("M,I,K", [(128, 128, 128), (300, 520, 288), (640, 1024, 512), (7, 776, 1120),
+                                   (2048, 4096, 512), (2500, 3080, 288)])
+def test_mx_swiglu_matches_oracle(M, I, K):
+    Xq, ex = oracle.quantize_rows_mx(inputs.normal_bf16(990 + M, "X", (M, K), 1.0))
+    Wgq, eg = oracle.quantize_rows_mx(inputs.normal_bf16(991, "W", (I, K), 1.0 / np.sqrt(K)))
+    Wuq, eu = oracle.quantize_rows_mx(inputs.normal_bf16(992, "W", (I, K), 1.0 / np.sqrt(K)))
+    check_swiglu(run_swiglu(Xq, ex, Wgq, eg, Wuq, eu), oracle.swiglu_mx(Xq, ex, Wgq, eg, Wuq, eu))
+
+
+def test_mx_swiglu_exact_pins_and_pairing():
+    """u = 1 exactly (one-hot up rows) leaves silu(g) for an exactly representable g; one-hot gate rows select
+    which up row pairs with which gate row; the scale arrays of gate and up are not interchangeable."""
+    M, I, K = 130, 264, 64
+    rng = np.random.default_rng(993)
+    Xq = small_codes(994, (M, K))
+    Xq[:, 0] = 0x38                                            # x[:, 0] = 1
+    ex = np.full((M, 2), 127, np.uint8)
+    Wgq = small_codes(995, (I, K))
+    eg = rng.integers(124, 127, size=(I, 2), dtype=np.uint8)
+    Wuq = np.zeros((I, K), np.uint8)
+    Wuq[:, 0] = 0x38                                           # u = 1 * 2^(eu - 127)
+    eu = rng.integers(127, 130, size=(I, 2), dtype=np.uint8)
+    z = run_swiglu(Xq, ex, Wgq, eg, Wuq, eu)
+    ref = oracle.swiglu_mx(Xq, ex, Wgq, eg, Wuq, eu)
+    check_swiglu(z, ref)
+    g = oracle.outproj_mx(Xq, ex, Wgq, eg)
+    assert np.allclose(ref, g / (1 + np.exp(-g)) * (2.0 ** (eu[:, 0].astype(np.float64) - 127))[None, :])
+    assert np.abs(ref).max() > 1.0
+    # swapping the two halves of the scale array changes the result
+    Z = kt.nan_filled(M, I)
+    sfug = np.concatenate([chunked(eu, K), chunked(eg, K)])
+    kx.kx_gate_up_swiglu_mxfp8(dev8(Xq), dev(chunked(ex, K)), dev8(Wgq), dev8(Wuq), dev(sfug), Z)
+    assert not np.array_equal(kt.from_dev(Z), z)
+
+
+def test_mx_gate_up_code_books_and_chain_on_device():
+    """Code books of both weight matrices in the layout the GEMM reads, then RMSNorm + code book -> gate/up + SwiGLU
+    on the device, against the oracle on the oracle's code books (bit-identical to the device's)."""
+    M, I, K = 520, 1160, 1024
+    H = inputs.normal_bf16(996, "R", (M, K), 1.3)
+    gam = inputs.normal_bf16(996, "bias", (K,), 1.0)
+    Wg = inputs.normal_bf16(997, "W", (I, K), 1.0 / np.sqrt(K))
+    Wu = inputs.normal_bf16(998, "W", (I, K), 1.0 / np.sqrt(K))
+    f8 = lambda *shape: torch.empty(shape, dtype=torch.uint8, device="cuda").view(F8)
+    Qg, Qu, Xq = f8(I, K), f8(I, K), f8(M, K)
+    SFGU = torch.full((2 * kx.kx_mx_scale_bytes(I, K),), 0xEE, dtype=torch.uint8, device="cuda")
+    SFX = torch.empty((kx.kx_mx_scale_bytes(M, K),), dtype=torch.uint8, device="cuda")
+    kx.kx_quantize_gate_up_mxfp8(kt.to_dev(Wg), kt.to_dev(Wu), Qg, Qu, SFGU)
+    Zn = kt.nan_filled(M, K)
+    kx.kx_rmsnorm(kt.to_dev(H), kt.to_dev(gam), 1e-6, Zn)
+    kx.kx_rmsnorm_quantize_mxfp8(kt.to_dev(H), kt.to_dev(gam), 1e-6, Xq, SFX)
+    Z = kt.nan_filled(M, I)
+    kx.kx_gate_up_swiglu_mxfp8(Xq, SFX, Qg, Qu, SFGU, Z)
+    status_ok()
+    qg, eg = oracle.quantize_rows_mx(Wg)
+    qu, eu = oracle.quantize_rows_mx(Wu)
+    xq, ex = oracle.quantize_rows_mx(kt.from_dev(Zn))
+    assert np.array_equal(host8(Qg), qg) and np.array_equal(host8(Qu), qu) and np.array_equal(host8(Xq), xq)
+    assert np.array_equal(SFGU.cpu().numpy(), np.concatenate([chunked(eg, K), chunked(eu, K)]))
+    check_swiglu(kt.from_dev(Z), oracle.swiglu_mx(xq, ex, qg, eg, qu, eu))
+
+
+def test_mx_swiglu_full_size_sampled_rows():
+    """The gate/up shape of the benchmark (M = 4096 tokens, I = 14336, K = 4096) on sampled rows."""
+    M, I, K = 4096, 14336, 4096
+    Xq, ex = oracle.quantize_rows_mx(inputs.normal_bf16(999, "X", (M, K), 1.0))
+    Wgq, eg = oracle.quantize_rows_mx(inputs.normal_bf16(1000, "W", (I, K), 1.0 / np.sqrt(K)))
+    Wuq, eu = oracle.quantize_rows_mx(inputs.normal_bf16(1001, "W", (I, K), 1.0 / np.sqrt(K)))
+    rows = inputs.sampled_rows(M)[::8]
+    z = run_swiglu(Xq, ex, Wgq, eg, Wuq, eu)
+    assert not np.isnan(oracle.widen_bf16(z)).any()
+    check_swiglu(z[rows], oracle.swiglu_mx(Xq, ex, Wgq, eg, Wuq, eu, rows=rows))
