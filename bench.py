@@ -672,6 +672,38 @@ def run_ours(args):
             del keep, calls, qcalls
             torch.cuda.empty_cache()
 
+        # block-scaled gate/up + SwiGLU on device-made code books (weights' scale arrays back to back)
+        for (Ms, Is, Ks) in [(4096, 14336, 4096)]:
+            ops = 4.0 * Ms * Is * Ks
+            nbytes = 1.0 * (Ms * Ks + 2 * Is * Ks) * (1.0 + 1.0 / 32) + 2.0 * Ms * Is
+            ns = 2
+            keep, calls = [], []
+            for _ in range(ns):
+                Xs = torch.randn(Ms, Ks, device="cuda", generator=g).bfloat16()
+                Wgs = (torch.randn(Is, Ks, device="cuda", generator=g) / math.sqrt(Ks)).bfloat16()
+                Wus = (torch.randn(Is, Ks, device="cuda", generator=g) / math.sqrt(Ks)).bfloat16()
+                Xq = torch.empty(Ms, Ks, device="cuda", dtype=torch.uint8)
+                Qg = torch.empty(Is, Ks, device="cuda", dtype=torch.uint8)
+                Qu = torch.empty(Is, Ks, device="cuda", dtype=torch.uint8)
+                sfx = torch.empty(int(lib.kx_mx_scale_bytes(i64(Ms), i64(Ks))), device="cuda", dtype=torch.uint8)
+                sfgu = torch.empty(2 * int(lib.kx_mx_scale_bytes(i64(Is), i64(Ks))), device="cuda", dtype=torch.uint8)
+                Zs = torch.empty(Ms, Is, dtype=torch.bfloat16, device="cuda")
+                rcq = lib.kx_quantize_rows_mxfp8(vp(Xs.data_ptr()), vp(Xq.data_ptr()), vp(sfx.data_ptr()), i64(Ms), i64(Ks), st)
+                rcq = rcq or lib.kx_quantize_gate_up_mxfp8(vp(Wgs.data_ptr()), vp(Wus.data_ptr()), vp(Qg.data_ptr()),
+                                                           vp(Qu.data_ptr()), vp(sfgu.data_ptr()), i64(Is), i64(Ks), st)
+                if rcq != 0:
+                    raise SystemExit(f"block-scaled code books failed ({rcq})")
+                torch.cuda.synchronize()
+                del Xs, Wgs, Wus
+                keep.append((Xq, Qg, Qu, sfx, sfgu, Zs))
+                a = (vp(Xq.data_ptr()), vp(sfx.data_ptr()), vp(Qg.data_ptr()), vp(Qu.data_ptr()), vp(sfgu.data_ptr()),
+                     vp(Zs.data_ptr()), i64(Ms), i64(Is), i64(Ks), st)
+                calls.append(lambda a=a: lib.kx_gate_up_swiglu_mxfp8(*a))
+            wls = inputs.Workload(f"swiglu_mxfp8_M{Ms}_I{Is}_K{Ks}", Ms, 2 * Is, Ks, 0, False, False)
+            t, tbest, _ = time_shape(torch, kx, wls, calls)
+            report(wls.name, t, tbest, nbytes, ops, ns)
+            del keep, calls
+            torch.cuda.empty_cache()
         # 4-bit block-scaled: the code book, then the projection on those codes; peak = 4 x the BF16 GEMM peak
         peak4 = 4.0 * peaks["bf16_tflops"]
         for (Mo, No, Ko) in [(4096, 4096, 4096), (16384, 4096, 14336)]:
