@@ -8,5 +8,5 @@ from .oracle import (  # noqa: F401
     quantize_rows, swiglu_int8, outproj_int8,
     e4m3_decode, e4m3_encode, quantize_rows_fp8, swiglu_fp8, outproj_fp8,
     e8m0_decode, quantize_rows_mx, outproj_mx, swiglu_mx,
-    e2m1_decode, e2m1_encode, quantize_rows_nvfp4, outproj_nvfp4,
+    e2m1_decode, e2m1_encode, quantize_rows_nvfp4, outproj_nvfp4, swiglu_nvfp4,
 )

@@ -428,3 +428,12 @@ def swiglu_mx(Xq, ex, Wgq, eg, Wuq, eu, rows=None):
     g = outproj_mx(Xq, ex, Wgq, eg, rows=rows)
     u = outproj_mx(Xq, ex, Wuq, eu, rows=rows)
     return g / (1.0 + np.exp(-g)) * u
+
+
+
+def swiglu_nvfp4(Xq, sx, Wgq, sg, Wuq, su, alpha_g: float, alpha_u: float, rows=None):
+    """z = silu(g) * u with g = alpha_g * (block-scaled 4-bit product of Xq with the gate weights), u likewise with the
+    up weights; float64, unrounded.  Two calls of the 4-bit projection and the activation written out."""
+    g = outproj_nvfp4(Xq, sx, Wgq, sg, alpha_g, rows=rows)
+    u = outproj_nvfp4(Xq, sx, Wuq, su, alpha_u, rows=rows)
+    return g / (1.0 + np.exp(-g)) * u

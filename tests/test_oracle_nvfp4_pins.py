@@ -158,3 +158,20 @@ def test_nvfp4_projection_equals_bf16_projection():
     Xb[:, :16] = 0
     Xb[:, 24:] = 0
     assert np.allclose(d[1], oracle.outproj_nvfp4(Xb, sx, Wq, sw, 1.0)[1], rtol=1e-12, atol=0)
+
+
+def test_nvfp4_swiglu_equals_bf16_swiglu():
+    M, I, K = 5, 9, 48
+    Xq, sx, Wgq, sg = nv_case(M, I, K, 8)
+    _, _, Wuq, su = nv_case(M, I, K, 9)
+    sx[:] = 0x28                                                                   # 0.25
+    X = bits(oracle.e2m1_decode(unpack(Xq)) * np.repeat(oracle.e4m3_decode(sx), 16, axis=1)[:, :K] * 0.5)
+    Wg = bits(oracle.e2m1_decode(unpack(Wgq)) * np.repeat(oracle.e4m3_decode(sg), 16, axis=1)[:, :K] * 0.25)
+    Wu = bits(oracle.e2m1_decode(unpack(Wuq)) * np.repeat(oracle.e4m3_decode(su), 16, axis=1)[:, :K])
+    z = oracle.swiglu_nvfp4(Xq, sx, Wgq, sg, Wuq, su, 0.125, 0.5)
+    zw, g, u = oracle.swiglu(X, Wg, Wu, want_parts=True)
+    assert np.max(np.abs(z - zw)) <= 1e-13 * max(1.0, np.abs(zw).max())
+    assert np.abs(g).max() > 0.3
+    assert not np.allclose(oracle.swiglu_nvfp4(Xq, sx, Wgq, sg, Wuq, su, 0.5, 0.125), z)   # the two alphas are not interchangeable
+    rows = np.array([4, 1])
+    assert np.array_equal(oracle.swiglu_nvfp4(Xq, sx, Wgq, sg, Wuq, su, 0.125, 0.5, rows=rows), z[rows])
