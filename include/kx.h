@@ -454,6 +454,19 @@ int kx_outproj_residual_mxfp8_ex(const void* Xq, const void* SFX, const void* Wq
  */
 int64_t kx_nvfp4_scale_bytes(int64_t rows, int64_t cols);
 int kx_quantize_rows_nvfp4(const void* A, float gs, void* Q, void* SF, int64_t rows, int64_t cols, void* stream);
+/* The other steps of the layer on the 4-bit format, mirroring the block-scaled FP8 calls:
+ * kx_rmsnorm_quantize_nvfp4 = code book of RMSNorm(H) * gamma (rounded to BF16 as kx_rmsnorm writes it) with
+ * tensor scale gs; kx_quantize_gate_up_nvfp4 = code books of the gate and up weights (tensor scales gsg, gsu),
+ * scale arrays back to back in SFGU (gate first; 2 * kx_nvfp4_scale_bytes(I, K) bytes);
+ * kx_gate_up_swiglu_nvfp4: Z[m,i] = bf16( silu(alpha_g g) * (alpha_u u) ) with g / u the block-scaled sums of row
+ * m of Xq with row i of Wgq / Wuq and alpha_g / alpha_u = tensor scale of X times that of the gate / up
+ * weights.  K % 32 == 0, I % 8 == 0. */
+int kx_rmsnorm_quantize_nvfp4(const void* H, const void* gamma, float eps, float gs, void* Q, void* SF,
+                              int64_t M, int64_t N, void* stream);
+int kx_quantize_gate_up_nvfp4(const void* Wg, const void* Wu, float gsg, float gsu, void* Qg, void* Qu, void* SFGU,
+                              int64_t I, int64_t K, void* stream);
+int kx_gate_up_swiglu_nvfp4(const void* Xq, const void* SFX, const void* Wgq, const void* Wuq, const void* SFGU,
+                            float alpha_g, float alpha_u, void* Z, int64_t M, int64_t I, int64_t K, void* stream);
 int kx_outproj_residual_nvfp4(const void* Xq, const void* SFX, const void* Wq, const void* SFW, float alpha,
                               const void* bias_or_null, const void* R_or_null, void* Y,
                               int64_t M, int64_t N, int64_t K, void* stream,

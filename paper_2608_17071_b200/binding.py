@@ -32,6 +32,7 @@ EXPORTS = (
     "kx_mx_scale_bytes", "kx_quantize_rows_mxfp8", "kx_rmsnorm_quantize_mxfp8", "kx_outproj_residual_mxfp8", "kx_outproj_residual_mxfp8_ex",
     "kx_quantize_gate_up_mxfp8", "kx_gate_up_swiglu_mxfp8",
     "kx_nvfp4_scale_bytes", "kx_quantize_rows_nvfp4", "kx_outproj_residual_nvfp4",
+    "kx_rmsnorm_quantize_nvfp4", "kx_quantize_gate_up_nvfp4", "kx_gate_up_swiglu_nvfp4",
     "kx_plan_query", "kx_last_device_status", "kx_status_string",
     "kx_version",
 )
@@ -110,6 +111,10 @@ def load():
     lib.kx_quantize_rows_nvfp4.argtypes = [vp, ctypes.c_float, vp, vp, i64, i64, vp]
     lib.kx_outproj_residual_nvfp4.argtypes = [vp, vp, vp, vp, ctypes.c_float, vp, vp, vp, i64, i64, i64, vp,
                                               ctypes.POINTER(PlanOverride)]
+    cf = ctypes.c_float
+    lib.kx_rmsnorm_quantize_nvfp4.argtypes = [vp, vp, cf, cf, vp, vp, i64, i64, vp]
+    lib.kx_quantize_gate_up_nvfp4.argtypes = [vp, vp, cf, cf, vp, vp, vp, i64, i64, vp]
+    lib.kx_gate_up_swiglu_nvfp4.argtypes = [vp, vp, vp, vp, vp, cf, cf, vp, i64, i64, i64, vp]
     lib.kx_plan_query.argtypes = [i64, i64, i64, ci, ci, ctypes.POINTER(PlanOverride), ctypes.POINTER(PlanInfo)]
     lib.kx_last_device_status.argtypes = [vp, ctypes.POINTER(ci), ctypes.POINTER(ci)]
     lib.kx_status_string.argtypes = [ci]
@@ -609,4 +614,46 @@ def kx_outproj_residual_nvfp4(Xq, SFX, Wq, SFW, alpha: float, bias, R, Y, stream
                                           ctypes.byref(override) if override is not None else None)
     if check and rc != KX_OK:
         raise KxError(rc, "kx_outproj_residual_nvfp4")
+    return rc
+
+
+def kx_rmsnorm_quantize_nvfp4(H, gamma, eps: float, gs: float, Q, SF, stream=None, check=True) -> int:
+    """Q, SF = 4-bit block-scaled code book of RMSNorm(H) * gamma (rounded to BF16 as kx_rmsnorm would) with tensor scale gs."""
+    import torch
+    M, N = H.shape
+    _check_bf16("H", H, (M, N)); _check_bf16("gamma", gamma, (N,)); _check("Q", Q, (M, N // 2), torch.uint8)
+    _check("SF", SF, (kx_nvfp4_scale_bytes(M, N),), torch.uint8)
+    rc = load().kx_rmsnorm_quantize_nvfp4(_addr(H), _addr(gamma), float(eps), float(gs), _addr(Q), _addr(SF), M, N,
+                                          _stream(stream))
+    if check and rc != KX_OK:
+        raise KxError(rc, "kx_rmsnorm_quantize_nvfp4")
+    return rc
+
+
+def kx_quantize_gate_up_nvfp4(Wg, Wu, gsg: float, gsu: float, Qg, Qu, SFGU, stream=None, check=True) -> int:
+    """4-bit code books of the gate and the up weights; SFGU = gate scales followed by up scales."""
+    import torch
+    I, K = Wg.shape
+    _check_bf16("Wg", Wg, (I, K)); _check_bf16("Wu", Wu, (I, K))
+    _check("Qg", Qg, (I, K // 2), torch.uint8); _check("Qu", Qu, (I, K // 2), torch.uint8)
+    _check("SFGU", SFGU, (2 * kx_nvfp4_scale_bytes(I, K),), torch.uint8)
+    rc = load().kx_quantize_gate_up_nvfp4(_addr(Wg), _addr(Wu), float(gsg), float(gsu), _addr(Qg), _addr(Qu), _addr(SFGU),
+                                          I, K, _stream(stream))
+    if check and rc != KX_OK:
+        raise KxError(rc, "kx_quantize_gate_up_nvfp4")
+    return rc
+
+
+def kx_gate_up_swiglu_nvfp4(Xq, SFX, Wgq, Wuq, SFGU, alpha_g: float, alpha_u: float, Z, stream=None, check=True) -> int:
+    """Z = silu(alpha_g g) * (alpha_u u) on packed 4-bit block-scaled operands."""
+    import torch
+    M, kb = Xq.shape
+    I, K = Wgq.shape[0], 2 * kb
+    _check("Xq", Xq, (M, kb), torch.uint8); _check("Wgq", Wgq, (I, kb), torch.uint8); _check("Wuq", Wuq, (I, kb), torch.uint8)
+    _check("SFX", SFX, (kx_nvfp4_scale_bytes(M, K),), torch.uint8)
+    _check("SFGU", SFGU, (2 * kx_nvfp4_scale_bytes(I, K),), torch.uint8); _check_bf16("Z", Z, (M, I))
+    rc = load().kx_gate_up_swiglu_nvfp4(_addr(Xq), _addr(SFX), _addr(Wgq), _addr(Wuq), _addr(SFGU), float(alpha_g),
+                                        float(alpha_u), _addr(Z), M, I, K, _stream(stream))
+    if check and rc != KX_OK:
+        raise KxError(rc, "kx_gate_up_swiglu_nvfp4")
     return rc

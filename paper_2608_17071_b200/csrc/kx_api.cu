@@ -1292,7 +1292,7 @@ namespace {
 bool aligned4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3u) == 0; }
 
 // fmt: 0 = INT8 codes, 1 = FP8 E4M3 codes (one scale per row); 2 = FP8 E4M3 codes with one E8M0 scale per 32
-// elements; 3 = E2M1 codes with one E4M3 scale per 16 elements (never behind RMSNorm)
+// elements; 3 = E2M1 codes with one E4M3 scale per 16 elements and a tensor scale
 int launch_rowquant(const QuantParams& qp, bool norm, int fmt, cudaStream_t stream, int sm_count) {
     cudaLaunchConfig_t cfg;
     std::memset(&cfg, 0, sizeof cfg);
@@ -1300,7 +1300,8 @@ int launch_rowquant(const QuantParams& qp, bool norm, int fmt, cudaStream_t stre
     const void* fn = nullptr;
     int per_sm = 8;
 #define KX_QUANT_FN(NV)                                                                              \
-    (fmt == 3 ? reinterpret_cast<const void*>(&kx_rowquant_kernel<NV, false, 3>)                     \
+    (fmt == 3 ? (norm ? reinterpret_cast<const void*>(&kx_rowquant_kernel<NV, true, 3>)              \
+                      : reinterpret_cast<const void*>(&kx_rowquant_kernel<NV, false, 3>))            \
      : fmt == 2 ? (norm ? reinterpret_cast<const void*>(&kx_rowquant_kernel<NV, true, 2>)            \
                       : reinterpret_cast<const void*>(&kx_rowquant_kernel<NV, false, 2>))            \
      : fmt == 1 ? (norm ? reinterpret_cast<const void*>(&kx_rowquant_kernel<NV, true, 1>)            \
@@ -1893,29 +1894,61 @@ int64_t kx_nvfp4_scale_bytes(int64_t rows, int64_t cols) {
     return mx_chunks(rows) * ((cols + 63) / 64) * 512;
 }
 
-int kx_quantize_rows_nvfp4(const void* A, float gs, void* Q, void* SF, int64_t rows, int64_t cols, void* stream) {
+namespace {
+int quantize_rows_nv(const void* A, const void* gamma, float eps, float gs, void* Q, void* SF, int64_t rows, int64_t cols,
+                     void* stream) {
     if (rows < 0 || cols < 0 || rows > 0x7FFFFFFFll / 2) return KX_ERR_SHAPE;
     if ((cols % 16) != 0 || cols > 8ll * kNormThreads * kNormVecs || !(gs > 0.0f) || !(gs < INFINITY)) return KX_ERR_SHAPE;
+    if (gamma && !(eps >= 0.0f)) return KX_ERR_SHAPE;
     if (rows == 0 || cols == 0) return KX_OK;
     if (!A || !Q || !SF) return KX_ERR_NULL;
-    if (!aligned16(A) || !aligned16(Q) || !aligned16(SF)) return KX_ERR_ALIGN;
+    if (!aligned16(A) || !aligned16(Q) || !aligned16(SF) || (gamma && !aligned16(gamma))) return KX_ERR_ALIGN;
     const size_t ab = static_cast<size_t>(rows) * cols * 2, qb = static_cast<size_t>(rows) * cols / 2,
-                 sb = static_cast<size_t>(kx_nvfp4_scale_bytes(rows, cols));
+                 sb = static_cast<size_t>(kx_nvfp4_scale_bytes(rows, cols)), gb = static_cast<size_t>(cols) * 2;
     if (overlaps(Q, qb, A, ab) || overlaps(SF, sb, A, ab) || overlaps(SF, sb, Q, qb)) return KX_ERR_OVERLAP;
+    if (gamma && (overlaps(Q, qb, gamma, gb) || overlaps(SF, sb, gamma, gb))) return KX_ERR_OVERLAP;
     DeviceCtx* ctx = nullptr;
     int rc = device_ctx(&ctx);
     if (rc != KX_OK) return rc;
     QuantParams qp;
     std::memset(&qp, 0, sizeof qp);
     qp.A0 = qp.A1 = static_cast<const uint16_t*>(A);
+    qp.gamma = static_cast<const uint16_t*>(gamma);
     qp.Q0 = qp.Q1 = static_cast<int8_t*>(Q);
     qp.SF0 = static_cast<uint8_t*>(SF);
     qp.rows0 = rows;
     qp.M = rows;
     qp.N = static_cast<int>(cols);
     qp.kchunks = static_cast<int>((cols + 63) / 64);
+    qp.eps = eps;
     qp.gs = gs;
-    return launch_rowquant(qp, false, 3, static_cast<cudaStream_t>(stream), ctx->sm_count);
+    return launch_rowquant(qp, gamma != nullptr, 3, static_cast<cudaStream_t>(stream), ctx->sm_count);
+}
+}  // namespace
+
+int kx_quantize_rows_nvfp4(const void* A, float gs, void* Q, void* SF, int64_t rows, int64_t cols, void* stream) {
+    return quantize_rows_nv(A, nullptr, 0.0f, gs, Q, SF, rows, cols, stream);
+}
+int kx_rmsnorm_quantize_nvfp4(const void* H, const void* gamma, float eps, float gs, void* Q, void* SF, int64_t M,
+                              int64_t N, void* stream) {
+    if (M > 0 && N > 0 && !gamma) return KX_ERR_NULL;
+    return quantize_rows_nv(H, gamma, eps, gs, Q, SF, M, N, stream);
+}
+int kx_quantize_gate_up_nvfp4(const void* Wg, const void* Wu, float gsg, float gsu, void* Qg, void* Qu, void* SFGU,
+                              int64_t I, int64_t K, void* stream) {
+    if (I < 0 || K < 0) return KX_ERR_SHAPE;
+    const int64_t half = kx_nvfp4_scale_bytes(I, K);
+    if (I > 0 && K > 0 && !SFGU) return KX_ERR_NULL;
+    const size_t qb = static_cast<size_t>(I) * K / 2, wb = static_cast<size_t>(I) * K * 2;
+    if (I > 0 && K > 0 && (overlaps(Qg, qb, Qu, qb) || overlaps(Qg, qb, Wu, wb) || overlaps(Qu, qb, Wg, wb) ||
+                           overlaps(SFGU, static_cast<size_t>(2 * half), Wg, wb) ||
+                           overlaps(SFGU, static_cast<size_t>(2 * half), Wu, wb) ||
+                           overlaps(SFGU, static_cast<size_t>(2 * half), Qg, qb) ||
+                           overlaps(SFGU, static_cast<size_t>(2 * half), Qu, qb)))
+        return KX_ERR_OVERLAP;
+    int rc = quantize_rows_nv(Wg, nullptr, 0.0f, gsg, Qg, SFGU, I, K, stream);
+    if (rc != KX_OK) return rc;
+    return quantize_rows_nv(Wu, nullptr, 0.0f, gsu, Qu, static_cast<uint8_t*>(SFGU) + half, I, K, stream);
 }
 
 int kx_outproj_residual_nvfp4(const void* Xq, const void* SFX, const void* Wq, const void* SFW, float alpha,
@@ -2014,6 +2047,88 @@ int kx_outproj_residual_nvfp4(const void* Xq, const void* SFX, const void* Wq, c
     cfg.numAttrs = 1;
     const uint16_t* bias_p = static_cast<const uint16_t*>(bias);
     void* args[] = {&tmA, &tmB, &tmSA, &tmY, &tmR, &tmSB, &bias_p, &p};
+    if (cudaLaunchKernelExC(&cfg, v->fn, args) != cudaSuccess) {
+        cudaGetLastError();
+        return KX_ERR_CUDA;
+    }
+    return KX_OK;
+}
+
+// Z = silu(g) * u on 4-bit block-scaled operands: the 256-column single-accumulator shape in gate/up mode;
+// alpha_g / alpha_u = tensor scale of X times that of the gate / up weights.
+int kx_gate_up_swiglu_nvfp4(const void* Xq, const void* SFX, const void* Wgq, const void* Wuq, const void* SFGU,
+                            float alpha_g, float alpha_u, void* Z, int64_t M, int64_t I, int64_t K, void* stream_v) {
+    if (M < 0 || I < 0 || K < 0) return KX_ERR_SHAPE;
+    if (M > 0x7FFFFFFFll / 2 || I > 0x7FFFFFFFll / 4 || K > 0x7FFFFFFFll / 2) return KX_ERR_SHAPE;
+    if (M == 0 || I == 0) return KX_OK;
+    if ((I % 8) != 0 || (K % 32) != 0) return KX_ERR_SHAPE;
+    if (!Z) return KX_ERR_NULL;
+    if (!aligned16(Z)) return KX_ERR_ALIGN;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    DeviceCtx* ctx = nullptr;
+    int rc = device_ctx(&ctx);
+    if (rc != KX_OK) return rc;
+    if (K == 0) {   // empty sums: silu(0) * 0 = 0
+        const long long total = M * I;
+        const int blocks = static_cast<int>(std::min<long long>((total + 255) / 256, ctx->sm_count * 8));
+        kx_k0_kernel<<<blocks, 256, 0, stream>>>(nullptr, nullptr, static_cast<uint16_t*>(Z), M, I, I, I);
+        return cudaGetLastError() == cudaSuccess ? KX_OK : KX_ERR_CUDA;
+    }
+    if (!Xq || !Wgq || !Wuq || !SFX || !SFGU) return KX_ERR_NULL;
+    if (!aligned16(Xq) || !aligned16(Wgq) || !aligned16(Wuq) || !aligned16(SFX) || !aligned16(SFGU)) return KX_ERR_ALIGN;
+    const size_t zb = static_cast<size_t>(M) * I * 2, wb = static_cast<size_t>(I) * K / 2;
+    if (overlaps(Z, zb, Xq, static_cast<size_t>(M) * K / 2) || overlaps(Z, zb, Wgq, wb) || overlaps(Z, zb, Wuq, wb) ||
+        overlaps(Z, zb, SFX, static_cast<size_t>(kx_nvfp4_scale_bytes(M, K))) ||
+        overlaps(Z, zb, SFGU, static_cast<size_t>(2 * kx_nvfp4_scale_bytes(I, K))))
+        return KX_ERR_OVERLAP;
+    const MxVariant* v = nullptr;
+    for (const auto& c : kNvVariants)
+        if (c.bn == 256) v = &c;
+    if (!v) return KX_ERR_PLAN;
+    const long long tm = (M + 127) / 128, tiles_n = (I + 127) / 128, tiles = tm * tiles_n;
+    if (tiles > 0x7FFFFFFFll / 4) return KX_ERR_SHAPE;
+    const long long kch = (K + 63) / 64;
+    CUtensorMap tmA, tmG, tmU, tmZ, tmSA, tmSB;
+    if ((rc = get_tmap(Xq, M, K / 2, 128, &tmA, 1)) != KX_OK) return rc;
+    if ((rc = get_tmap(Wgq, I, K / 2, 128, &tmG, 1)) != KX_OK) return rc;
+    if ((rc = get_tmap(Wuq, I, K / 2, 128, &tmU, 1)) != KX_OK) return rc;
+    if ((rc = get_tmap_scales(SFX, mx_chunks(M) * kch, &tmSA, 4)) != KX_OK) return rc;
+    if ((rc = get_tmap_scales(SFGU, 2 * mx_chunks(I) * kch, &tmSB, 4)) != KX_OK) return rc;
+    if ((rc = get_tmap(Z, M, I, 32, &tmZ)) != KX_OK) return rc;
+    TileParams p;
+    std::memset(&p, 0, sizeof p);
+    p.M = static_cast<int>(M);
+    p.N = static_cast<int>(I);
+    p.K = static_cast<int>(K / 2);
+    p.tiles_m = static_cast<int>(tm);
+    p.tiles_n = static_cast<int>(tiles_n);
+    p.num_tiles = static_cast<int>(tiles);
+    p.raster_group = 8;
+    p.swiglu = 1;
+    p.kcluster = 1;
+    p.sk_tile0 = p.num_tiles;
+    p.narrow_tile0 = p.num_tiles;
+    p.spin_limit_ns = 2000000000ull;
+    p.status = ctx->status;
+    p.ws = ctx->ws;
+    p.counters = ctx->counters;
+    p.sfb_chunks = static_cast<int>(mx_chunks(I));
+    p.sf_kchunks = static_cast<int>(kch);
+    p.alpha = alpha_g;
+    p.alpha2 = alpha_u;
+    cudaLaunchConfig_t cfg;
+    std::memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3(static_cast<unsigned>(std::min<long long>(tiles, ctx->sm_count)), 1, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = v->smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const uint16_t* bias_p = nullptr;
+    void* args[] = {&tmA, &tmG, &tmU, &tmZ, &tmSA, &tmSB, &bias_p, &p};
     if (cudaLaunchKernelExC(&cfg, v->fn, args) != cudaSuccess) {
         cudaGetLastError();
         return KX_ERR_CUDA;

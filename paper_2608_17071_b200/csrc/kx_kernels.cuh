@@ -131,6 +131,7 @@ struct TileParams {
     int sfb_chunks;            // KIND 3 / 4: ceil(N / 128) = rows of 128-row scale chunks of B
     int sf_kchunks;            // KIND 4: scale chunks per 128 rows along K = ceil(K / 64)
     float alpha;               // KIND 4: product of the two tensor scales, applied to the accumulators
+    float alpha2;              // KIND 4, gate/up mode: the same for the up accumulators (alpha: the gate ones)
     int swiglu;                   // 1: gate/up mode.  W rows of a tile = BN/2 rows of Wg (tmB) followed by the same
                                   // BN/2 rows of Wu (tmB2); the epilogue writes silu(gate) * up, BN/2 columns per
                                   // tile, N = number of output columns; no bias, no residual
@@ -430,12 +431,15 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     if constexpr (KIND == 4) {
                         // 16-element blocks: four scale chunks per 128 rows and k-block (one per K = 64 step),
                         // contiguous, fetched as one 2048-byte box per operand row block
-                        const int c0 = col >> 7;
+                        // (gate/up mode: as for KIND 3 - gate chunk, then the up chunk sfb_chunks rows further; the
+                        // scales of A through tmR)
+                        const int c0 = sg ? (col >> 8) : (col >> 7);
                         const uint32_t dst = s_sf + s * C::SF_STAGE;
-                        tma_load_2d(dst, &tmB2, 0, tm * p.sf_kchunks + kb * 4, full(s));
-                        for (int i = 0; i < C::SFB_CHUNKS; ++i)
-                            tma_load_2d(dst + 2048 * (1 + i), &tmS, 0, min(c0 + i, p.sfb_chunks - 1) * p.sf_kchunks + kb * 4,
-                                        full(s));
+                        tma_load_2d(dst, sg ? &tmR : &tmB2, 0, tm * p.sf_kchunks + kb * 4, full(s));
+                        for (int i = 0; i < C::SFB_CHUNKS; ++i) {
+                            const int ch = sg ? (i == 0 ? c0 : p.sfb_chunks + c0) : min(c0 + i, p.sfb_chunks - 1);
+                            tma_load_2d(dst + 2048 * (1 + i), &tmS, 0, ch * p.sf_kchunks + kb * 4, full(s));
+                        }
                     }
                     if constexpr (CTAS == 1) {
                         mbar_arrive_expect_tx(full(s), nsub * (stage_tx + C::SF_KB_BYTES));
@@ -841,6 +845,10 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         tmem_ld_32x32(tbase + BN / 2 + c * 64 + h * 32, up);
                         tmem_ld_wait();
                         if constexpr (kRowScaled) dequant_half(up, p.sb2, col0 + h * 32);
+                        if constexpr (KIND == 4) {
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) up[i] = __float_as_uint(__uint_as_float(up[i]) * p.alpha2);
+                        }
 #pragma unroll
                         for (int i = 0; i < 32; ++i) {
                             const float gte = __uint_as_float(acc[h][i]);

@@ -271,3 +271,93 @@ def test_nvfp4_projection_full_sizes_sampled_rows(M, N, K):
     ok, msg = kt.gate_a(y[rows], ref)
     assert ok, msg
     assert kt.rel_fro(y[rows], ref) <= 2.0 ** -8
+
+
+# ------------------------------------------------------------------ RMSNorm-fused code book, gate/up + SwiGLU
+@pytest.mark.parametrize("M,N", [(130, 4096), (1000, 5120), (9, 32768), (300, 1040)])
+def test_nvfp4_rmsnorm_code_book(M, N):
+    """Fused RMSNorm + code book = code book of the device's own BF16 RMSNorm output, bit for bit."""
+    H = inputs.normal_bf16(1150 + N, "R", (M, N), 1.3)
+    g = inputs.normal_bf16(1150 + N, "bias", (N,), 1.0)
+    Z = kt.nan_filled(M, N)
+    kx.kx_rmsnorm(kt.to_dev(H), kt.to_dev(g), 1e-6, Z)
+    gs = 8.0 / 2688.0
+    Q = torch.full((M, N // 2), 0x55, dtype=torch.uint8, device="cuda")
+    SF = torch.full((kx.kx_nvfp4_scale_bytes(M, N),), 0xEE, dtype=torch.uint8, device="cuda")
+    kx.kx_rmsnorm_quantize_nvfp4(kt.to_dev(H), kt.to_dev(g), 1e-6, gs, Q, SF)
+    Qr, Sr = oracle.quantize_rows_nvfp4(kt.from_dev(Z), gs)
+    assert np.array_equal(Q.cpu().numpy(), Qr) and np.array_equal(SF.cpu().numpy(), chunked(Sr, N))
+
+
+def check_swiglu(z_bits, ref):
+    ok, msg = kt.gate_a(z_bits, ref)
+    assert ok, msg
+    assert kt.rel_fro(z_bits, ref) <= 2.0 ** -8
+    z = oracle.widen_bf16(z_bits)
+    assert (np.abs(z - ref) <= 2.0 ** -7 * np.abs(ref) + 2e-3).all()
+
+
+def run_swiglu(Xq, sx, Wgq, sg, Wuq, su, ag, au):
+    M, I, K = Xq.shape[0], Wgq.shape[0], Xq.shape[1] * 2
+    Z = kt.nan_filled(M, I)
+    sfgu = np.concatenate([chunked(sg, K), chunked(su, K)])
+    kx.kx_gate_up_swiglu_nvfp4(dev(Xq), dev(chunked(sx, K)), dev(Wgq), dev(Wuq), dev(sfgu), ag, au, Z)
+    status_ok()
+    return kt.from_dev(Z)
+
+
+def codes_of(seed, name, shape, std):
+    A = inputs.normal_bf16(seed, name, shape, std)
+    gs = float(np.float32(np.abs(inputs.bf16_bits_to_f32(A)).max() / 2688.0))
+    Q, S = oracle.quantize_rows_nvfp4(A, gs)
+    return Q, S, gs
+
+
+@pytest.mark.parametrize("M,I,K", [(128, 128, 256), (300, 520, 288), (640, 1024, 512), (7, 776, 1120),
+                                   (2048, 4096, 512), (2500, 3080, 288)])
+def test_nvfp4_swiglu_matches_oracle(M, I, K):
+    Xq, sx, gx = codes_of(1160 + M, "X", (M, K), 1.0)
+    Wgq, sg, gg = codes_of(1161, "W", (I, K), 1.0 / np.sqrt(K))
+    Wuq, su, gu = codes_of(1162, "W", (I, K), 2.0 / np.sqrt(K))
+    ag, au = float(np.float32(gx) * np.float32(gg)), float(np.float32(gx) * np.float32(gu))
+    check_swiglu(run_swiglu(Xq, sx, Wgq, sg, Wuq, su, ag, au), oracle.swiglu_nvfp4(Xq, sx, Wgq, sg, Wuq, su, ag, au))
+
+
+def test_nvfp4_gate_up_code_books_and_chain_on_device():
+    M, I, K = 520, 1160, 1024
+    H = inputs.normal_bf16(1170, "R", (M, K), 1.3)
+    gam = inputs.normal_bf16(1170, "bias", (K,), 1.0)
+    Wg = inputs.normal_bf16(1171, "W", (I, K), 1.0 / np.sqrt(K))
+    Wu = inputs.normal_bf16(1172, "W", (I, K), 1.0 / np.sqrt(K))
+    gsx, gsg, gsu = 8.0 / 2688.0, 0.2 / 2688.0, 0.25 / 2688.0
+    u8 = lambda *shape: torch.empty(shape, dtype=torch.uint8, device="cuda")
+    Qg, Qu, Xq = u8(I, K // 2), u8(I, K // 2), u8(M, K // 2)
+    SFGU = torch.full((2 * kx.kx_nvfp4_scale_bytes(I, K),), 0xEE, dtype=torch.uint8, device="cuda")
+    SFX = u8(kx.kx_nvfp4_scale_bytes(M, K))
+    kx.kx_quantize_gate_up_nvfp4(kt.to_dev(Wg), kt.to_dev(Wu), gsg, gsu, Qg, Qu, SFGU)
+    Zn = kt.nan_filled(M, K)
+    kx.kx_rmsnorm(kt.to_dev(H), kt.to_dev(gam), 1e-6, Zn)
+    kx.kx_rmsnorm_quantize_nvfp4(kt.to_dev(H), kt.to_dev(gam), 1e-6, gsx, Xq, SFX)
+    Z = kt.nan_filled(M, I)
+    ag, au = float(np.float32(gsx) * np.float32(gsg)), float(np.float32(gsx) * np.float32(gsu))
+    kx.kx_gate_up_swiglu_nvfp4(Xq, SFX, Qg, Qu, SFGU, ag, au, Z)
+    status_ok()
+    qg, sg = oracle.quantize_rows_nvfp4(Wg, gsg)
+    qu, su = oracle.quantize_rows_nvfp4(Wu, gsu)
+    xq, sx = oracle.quantize_rows_nvfp4(kt.from_dev(Zn), gsx)
+    assert np.array_equal(Qg.cpu().numpy(), qg) and np.array_equal(Qu.cpu().numpy(), qu) and np.array_equal(Xq.cpu().numpy(), xq)
+    assert np.array_equal(SFGU.cpu().numpy(), np.concatenate([chunked(sg, K), chunked(su, K)]))
+    check_swiglu(kt.from_dev(Z), oracle.swiglu_nvfp4(xq, sx, qg, sg, qu, su, ag, au))
+
+
+def test_nvfp4_swiglu_full_size_sampled_rows():
+    """The gate/up shape of the benchmark (M = 4096 tokens, I = 14336, K = 4096) on sampled rows."""
+    M, I, K = 4096, 14336, 4096
+    Xq, sx, gx = codes_of(1175, "X", (M, K), 1.0)
+    Wgq, sg, gg = codes_of(1176, "W", (I, K), 1.0 / np.sqrt(K))
+    Wuq, su, gu = codes_of(1177, "W", (I, K), 1.0 / np.sqrt(K))
+    ag, au = float(np.float32(gx) * np.float32(gg)), float(np.float32(gx) * np.float32(gu))
+    rows = inputs.sampled_rows(M)[::8]
+    z = run_swiglu(Xq, sx, Wgq, sg, Wuq, su, ag, au)
+    assert not np.isnan(oracle.widen_bf16(z)).any()
+    check_swiglu(z[rows], oracle.swiglu_nvfp4(Xq, sx, Wgq, sg, Wuq, su, ag, au, rows=rows))
