@@ -748,6 +748,46 @@ def run_ours(args):
             del keep, calls, qcalls
             torch.cuda.empty_cache()
 
+        # 4-bit gate/up + SwiGLU on device-made code books
+        for (Ms, Is, Ks) in [(4096, 14336, 4096)]:
+            ops = 4.0 * Ms * Is * Ks
+            nbytes = 0.5 * (Ms * Ks + 2 * Is * Ks) * (1.0 + 1.0 / 8) + 2.0 * Ms * Is
+            ns = 2
+            keep, calls = [], []
+            for _ in range(ns):
+                Xs = torch.randn(Ms, Ks, device="cuda", generator=g).bfloat16()
+                Wgs = (torch.randn(Is, Ks, device="cuda", generator=g) / math.sqrt(Ks)).bfloat16()
+                Wus = (torch.randn(Is, Ks, device="cuda", generator=g) / math.sqrt(Ks)).bfloat16()
+                gsx, gsg, gsu = (float(t.abs().max()) / 2688.0 for t in (Xs, Wgs, Wus))
+                Xq = torch.empty(Ms, Ks // 2, device="cuda", dtype=torch.uint8)
+                Qg = torch.empty(Is, Ks // 2, device="cuda", dtype=torch.uint8)
+                Qu = torch.empty(Is, Ks // 2, device="cuda", dtype=torch.uint8)
+                sfx = torch.empty(int(lib.kx_nvfp4_scale_bytes(i64(Ms), i64(Ks))), device="cuda", dtype=torch.uint8)
+                sfgu = torch.empty(2 * int(lib.kx_nvfp4_scale_bytes(i64(Is), i64(Ks))), device="cuda", dtype=torch.uint8)
+                Zs = torch.empty(Ms, Is, dtype=torch.bfloat16, device="cuda")
+                rcq = lib.kx_quantize_rows_nvfp4(vp(Xs.data_ptr()), ctypes.c_float(gsx), vp(Xq.data_ptr()), vp(sfx.data_ptr()),
+                                                 i64(Ms), i64(Ks), st)
+                rcq = rcq or lib.kx_quantize_gate_up_nvfp4(vp(Wgs.data_ptr()), vp(Wus.data_ptr()), ctypes.c_float(gsg),
+                                                           ctypes.c_float(gsu), vp(Qg.data_ptr()), vp(Qu.data_ptr()),
+                                                           vp(sfgu.data_ptr()), i64(Is), i64(Ks), st)
+                if rcq != 0:
+                    raise SystemExit(f"4-bit code books failed ({rcq})")
+                torch.cuda.synchronize()
+                del Xs, Wgs, Wus
+                keep.append((Xq, Qg, Qu, sfx, sfgu, Zs))
+                a = (vp(Xq.data_ptr()), vp(sfx.data_ptr()), vp(Qg.data_ptr()), vp(Qu.data_ptr()), vp(sfgu.data_ptr()),
+                     ctypes.c_float(gsx * gsg), ctypes.c_float(gsx * gsu), vp(Zs.data_ptr()), i64(Ms), i64(Is), i64(Ks), st)
+                calls.append(lambda a=a: lib.kx_gate_up_swiglu_nvfp4(*a))
+            wls = inputs.Workload(f"swiglu_nvfp4_M{Ms}_I{Is}_K{Ks}", Ms, 2 * Is, Ks, 0, False, False)
+            t, tbest, _ = time_shape(torch, kx, wls, calls)
+            int8.append({"name": wls.name, "us": t * 1e6, "us_best": tbest * 1e6, "tops": ops / t / 1e12,
+                         "gbs": nbytes / t / 1e9, "bound": "tensor", "frac": ops / t / 1e12 / peak4, "peak": peak4,
+                         "operand_sets": ns})
+            print(f"[bench] {wls.name:>30s} {t*1e6:9.1f} us (best {tbest*1e6:7.1f}) {ops/t/1e12:8.1f} TOP/s {nbytes/t/1e9:7.0f} GB/s  "
+                  f"tensor {ops/t/1e12/peak4*100:5.1f}% of 4 x {peaks['source']} BF16 peak", file=sys.stderr, flush=True)
+            del keep, calls
+            torch.cuda.empty_cache()
+
     # ---- the oracle on the host cores, bounded sample (rank 0, N = 1 only)
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
