@@ -1631,7 +1631,6 @@ kx_rowquant_kernel(const QuantParams p) {
         if constexpr (FMT == 2) {
             uint2* qrow = reinterpret_cast<uint2*>(p.Q0 + r * N);
             uint8_t* const sfrow = p.SF0 + (r >> 7) * p.kchunks * 512 + (r & 31) * 16 + ((r & 127) >> 5) * 4;
-            const int nb = N >> 5;
 #pragma unroll
             for (int i = 0; i < NV; ++i) {
                 const int idx = tid + i * kNormThreads;
@@ -1647,20 +1646,22 @@ kx_rowquant_kernel(const QuantParams p) {
                 // N % 32 == 0: the four threads of a block are all valid or all invalid, and sit in one warp
                 bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, 1));
                 bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, 2));
+                uint32_t e = 127u;                           // lanes past the row end carry the padding value
                 if (valid) {
                     const int field = static_cast<int>(__float_as_uint(bmax) >> 23);
-                    const int e = (bmax > 0.f) ? max(field - 8, 0) : 127;
-                    const float mult = __uint_as_float(static_cast<uint32_t>(254 - e) << 23);   // 2^(127 - e), e <= 247
+                    e = (bmax > 0.f) ? static_cast<uint32_t>(max(field - 8, 0)) : 127u;
+                    const float mult = __uint_as_float((254u - e) << 23);   // 2^(127 - e), e <= 247
 #pragma unroll
                     for (int k = 0; k < 8; ++k) z[k] = __fmul_rn(z[k], mult);
                     qrow[idx] = make_uint2(pack_e4m3x4(z[0], z[1], z[2], z[3]), pack_e4m3x4(z[4], z[5], z[6], z[7]));
-                    if ((tid & 3) == 0) {
-                        const int j = idx >> 2;
-                        sfrow[(j >> 2) * 512 + (j & 3)] = static_cast<uint8_t>(e);
-                        if (j == nb - 1)                     // blocks past the row end inside the last chunk
-                            for (int jj = nb; jj < p.kchunks * 4; ++jj) sfrow[(jj >> 2) * 512 + (jj & 3)] = 127;
-                    }
                 }
+                // the scale bytes of four neighbouring blocks (16 lanes) are adjacent in a chunk: one 32-bit store,
+                // which also writes the padding entries of a last chunk that the row fills only in part
+                uint32_t word = e;
+                word |= __shfl_down_sync(0xffffffffu, e, 4) << 8;
+                word |= __shfl_down_sync(0xffffffffu, e, 8) << 16;
+                word |= __shfl_down_sync(0xffffffffu, e, 12) << 24;
+                if (valid && (tid & 15) == 0) *reinterpret_cast<uint32_t*>(sfrow + (idx >> 4) * 512) = word;
             }
             if (r == p.M - 1) {                              // rows up to the next multiple of 128
                 const long long pad_rows = ((p.M + 127) & ~127ll) - p.M;
@@ -1676,7 +1677,6 @@ kx_rowquant_kernel(const QuantParams p) {
         if constexpr (FMT == 3) {
             uint32_t* qrow = reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(p.Q0) + r * (N / 2));
             uint8_t* const sfrow = p.SF0 + (r >> 7) * p.kchunks * 512 + (r & 31) * 16 + ((r & 127) >> 5) * 4;
-            const int nb = N >> 4;
             const float d6 = __fmul_rn(6.0f, p.gs);
 #pragma unroll
             for (int i = 0; i < NV; ++i) {
@@ -1692,20 +1692,21 @@ kx_rowquant_kernel(const QuantParams p) {
                 }
                 // N % 16 == 0: the two threads of a block are both valid or both invalid
                 bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, 1));
+                uint32_t sb = 0u;                            // lanes past the row end carry the padding value
                 if (valid) {
-                    const uint32_t sb = pack_e4m3x4(__fdiv_rn(bmax, d6), 0.f, 0.f, 0.f) & 0xFFu;
+                    sb = pack_e4m3x4(__fdiv_rn(bmax, d6), 0.f, 0.f, 0.f) & 0xFFu;
                     const float dq = __fmul_rn(e4m3_to_f32(sb), p.gs);
                     const float rcp = (dq > 0.f) ? __fdiv_rn(1.0f, dq) : 0.f;
 #pragma unroll
                     for (int k = 0; k < 8; ++k) z[k] = __fmul_rn(z[k], rcp);
                     qrow[idx] = (dq > 0.f) ? pack_e2m1x8(z) : 0u;
-                    if ((tid & 1) == 0) {
-                        const int j = idx >> 1;
-                        sfrow[(j >> 2) * 512 + (j & 3)] = static_cast<uint8_t>(sb);
-                        if (j == nb - 1)
-                            for (int jj = nb; jj < p.kchunks * 4; ++jj) sfrow[(jj >> 2) * 512 + (jj & 3)] = 0;
-                    }
                 }
+                // four neighbouring blocks (8 lanes) -> one 32-bit store of their scale bytes, padding included
+                uint32_t word = sb;
+                word |= __shfl_down_sync(0xffffffffu, sb, 2) << 8;
+                word |= __shfl_down_sync(0xffffffffu, sb, 4) << 16;
+                word |= __shfl_down_sync(0xffffffffu, sb, 6) << 24;
+                if (valid && (tid & 7) == 0) *reinterpret_cast<uint32_t*>(sfrow + (idx >> 3) * 512) = word;
             }
             if (r == p.M - 1) {
                 const long long pad_rows = ((p.M + 127) & ~127ll) - p.M;
