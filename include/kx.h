@@ -59,17 +59,21 @@ typedef enum kx_status {
 
 /* Execution paths (the scheduling strategy of Table 1 names split-K and
  * persistent kernels; the per-M specialisation follows Algorithm 3's per-M plan). */
-enum { KX_PATH_AUTO = 0, KX_PATH_TILE = 1, KX_PATH_SWAP = 2 };
+enum { KX_PATH_AUTO = 0, KX_PATH_TILE = 1, KX_PATH_SWAP = 2, KX_PATH_GEMV = 3 };
 
 /*
  * Plan override for tests, profiling and tuning.  Zero-initialise for "auto".
  *   path          KX_PATH_AUTO / KX_PATH_TILE (128-row output tiles, persistent,
  *                 TMA-store epilogue) / KX_PATH_SWAP (small M: W rows on the MMA
- *                 M axis, split-K, W streamed once)
+ *                 M axis, split-K, W streamed once) / KX_PATH_GEMV (M <= 4 and K % 8 == 0:
+ *                 no tensor core, every CTA streams a few rows of W and reduces over K with
+ *                 FP32 warp reductions)
  *   block_n       tile path: 64, 128, 192 or 256 output columns per tile;
- *                 swap path: 16, 32, 64, 128 or 256 X rows per unit
+ *                 swap path: 16, 32, 64, 128 or 256 X rows per unit;
+ *                 GEMV path: 1, 2 or 4 rows of W (output columns) per CTA
  *   cta_pair      0 auto, 1 = one CTA per tile, 2 = CTA pair per 256-row tile
- *   split_k       swap path only: number of K splits (1..64)
+ *   split_k       swap path: number of K splits (1..64);
+ *                 GEMV path: 1..16 warps per CTA that share the K range of its rows
  *   raster_group  tile path: number of 128-row tile rows that share a raster group
  *   max_ctas      cap on the persistent grid (0 = number of SMs)
  *   spin_limit_us bound on every device-side wait (0 = 2 000 000 us)
@@ -82,7 +86,10 @@ enum { KX_PATH_AUTO = 0, KX_PATH_TILE = 1, KX_PATH_SWAP = 2 };
  *                 waves as half-width tiles when they then fit in one extra wave
  *   cluster_reduce  swap path: 0 auto, 1 = sum the K splits through the FP32 workspace
  *                 (last CTA to arrive reduces), 2 = the 2..8 splits of a tile form a
- *                 thread-block cluster and are summed through distributed shared memory
+ *                 thread-block cluster and the CTA that finishes a row reads the partials of
+ *                 its peers through distributed shared memory, 3 = the same cluster, but every
+ *                 CTA stores its partial rows into the shared memory of their finishers and
+ *                 signals an mbarrier there (X rows per unit <= 128)
  *   k_cluster     tile path, one CTA per tile: 2 or 4 = split the K range of every tile over a
  *                 thread-block cluster of that many CTAs and sum the partial tiles through
  *                 distributed shared memory (for problems with too few tiles to fill the GPU)
@@ -122,7 +129,7 @@ typedef struct kx_plan_override {
 
 /* What the planner chose for a shape (kx_plan_query). */
 typedef struct kx_plan_info {
-    int32_t path;          /* KX_PATH_TILE or KX_PATH_SWAP                         */
+    int32_t path;          /* KX_PATH_TILE, KX_PATH_SWAP or KX_PATH_GEMV           */
     int32_t block_n;
     int32_t cta_pair;      /* 1 or 2                                               */
     int32_t stages;        /* depth of the TMA -> MMA shared-memory ring           */
@@ -135,7 +142,7 @@ typedef struct kx_plan_info {
     int64_t workspace_bytes; /* FP32 split-K / stream-K scratch this plan uses (0 if none) */
     int32_t stream_k;      /* 1 if the tile path runs with stream-K scheduling     */
     int32_t narrow_tiles;  /* number of half-width tail tiles (0 if none)          */
-    int32_t cluster_reduce;/* 1 if the swap path reduces its splits inside a cluster */
+    int32_t cluster_reduce;/* swap path: 0 = workspace, 1 = cluster (partials pulled), 2 = cluster (partials pushed) */
     int32_t from_table;    /* 1 if the built-in measured plan table supplied this plan */
 } kx_plan_info;
 

@@ -11,6 +11,7 @@
 #include <cstring>
 #include <mutex>
 
+#include "kx_internal.h"
 #include "kx_kernels.cuh"
 
 // Fixed scratch of kx_outproj_residual_noalloc: FP32 split-K partial sums followed by
@@ -76,7 +77,9 @@ struct TileVariant {
 struct SwapVariant {
     int bn, stages, smem;
     const void* fn;           // split-K through the global workspace (any split count)
-    const void* fn_cluster;   // split-K inside a thread-block cluster (2..8 splits)
+    const void* fn_cluster;   // split-K inside a thread-block cluster (2..8 splits), partials pulled by the finishers
+    const void* fn_push;      // the same with partials pushed to the finishers (null: not instantiated)
+    int smem_push;            // its shared memory (ring of its own depth + receive area)
 };
 
 #define KX_TILE(BN, CTAS, ST, NB, KBS)                                                        \
@@ -89,8 +92,17 @@ struct SwapVariant {
 #define KX_SWAP(BN, ST, KBS)                                                                  \
     SwapVariant {                                                                             \
         BN, ST, SwapCfg<BN, ST, KBS>::SMEM_BYTES,                                             \
-            reinterpret_cast<const void*>(&kx_swap_kernel<BN, ST, false, KBS>),               \
-            reinterpret_cast<const void*>(&kx_swap_kernel<BN, ST, true, KBS>)                 \
+            reinterpret_cast<const void*>(&kx_swap_kernel<BN, ST, 0, KBS>),                   \
+            reinterpret_cast<const void*>(&kx_swap_kernel<BN, ST, 1, KBS>), nullptr, 0        \
+    }
+// with a push-mode kernel whose ring has PST stages (the receive area takes the rest of shared memory)
+#define KX_SWAP_P(BN, ST, KBS, PST)                                                           \
+    SwapVariant {                                                                             \
+        BN, ST, SwapCfg<BN, ST, KBS>::SMEM_BYTES,                                             \
+            reinterpret_cast<const void*>(&kx_swap_kernel<BN, ST, 0, KBS>),                   \
+            reinterpret_cast<const void*>(&kx_swap_kernel<BN, ST, 1, KBS>),                   \
+            reinterpret_cast<const void*>(&kx_swap_kernel<BN, PST, 2, KBS>),                  \
+            SwapCfg<BN, PST, KBS, true>::SMEM_BYTES                                           \
     }
 
 // (tile width, CTAs per tile, ring stages, R staging buffers, k-blocks per stage).  The first entry
@@ -104,7 +116,7 @@ const TileVariant kTileVariants[] = {
 };
 // (X rows per unit, ring stages, k-blocks per stage); first match = default, the rest by `stages`
 const SwapVariant kSwapVariants[] = {
-    KX_SWAP(16, 6, 2), KX_SWAP(32, 5, 2), KX_SWAP(64, 4, 2), KX_SWAP(128, 3, 2), KX_SWAP(256, 2, 2),
+    KX_SWAP_P(16, 6, 2, 5), KX_SWAP_P(32, 5, 2, 5), KX_SWAP_P(64, 4, 2, 3), KX_SWAP_P(128, 3, 2, 2), KX_SWAP(256, 2, 2),
     KX_SWAP(16, 12, 1), KX_SWAP(32, 11, 1), KX_SWAP(64, 9, 1), KX_SWAP(128, 7, 1), KX_SWAP(256, 4, 1),
 };
 
@@ -208,7 +220,9 @@ int ensure_device(int dev, DeviceCtx** out) {
             ok = ok &&
                  cudaFuncSetAttribute(v.fn, cudaFuncAttributeMaxDynamicSharedMemorySize, v.smem) == cudaSuccess &&
                  cudaFuncSetAttribute(v.fn_cluster, cudaFuncAttributeMaxDynamicSharedMemorySize, v.smem) ==
-                     cudaSuccess;
+                     cudaSuccess &&
+                 (!v.fn_push ||
+                  cudaFuncSetAttribute(v.fn_push, cudaFuncAttributeMaxDynamicSharedMemorySize, v.smem_push) == cudaSuccess);
         if (!ok) {
             rc = KX_ERR_CUDA;
             break;
@@ -409,9 +423,10 @@ const PlanTableEntry* find_table_entry(long long M, long long N, long long K) {
 
 // How many clusters of `size` CTAs of a swap-kernel variant can be resident at once
 // (a cluster lives inside one GPC, so this is less than SMs / size in general).
-int max_active_clusters(const SwapVariant* v, int size) {
+int max_active_clusters(const SwapVariant* v, int size, bool push = false) {
     static std::mutex mu;
-    static int cache[sizeof(kSwapVariants) / sizeof(kSwapVariants[0])][9];
+    static int cache2[2][sizeof(kSwapVariants) / sizeof(kSwapVariants[0])][9];
+    auto& cache = cache2[push ? 1 : 0];
     const int vi = static_cast<int>(v - kSwapVariants);
     std::lock_guard<std::mutex> lk(mu);
     if (cache[vi][size] != 0) return cache[vi][size];
@@ -419,7 +434,7 @@ int max_active_clusters(const SwapVariant* v, int size) {
     std::memset(&cfg, 0, sizeof cfg);
     cfg.gridDim = dim3(size * 64, 1, 1);
     cfg.blockDim = dim3(kThreads, 1, 1);
-    cfg.dynamicSmemBytes = v->smem;
+    cfg.dynamicSmemBytes = push ? v->smem_push : v->smem;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = size;
@@ -428,7 +443,7 @@ int max_active_clusters(const SwapVariant* v, int size) {
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, v->fn_cluster, &cfg) != cudaSuccess) {
+    if (cudaOccupancyMaxActiveClusters(&n, push ? v->fn_push : v->fn_cluster, &cfg) != cudaSuccess) {
         cudaGetLastError();
         n = -1;
     }
@@ -472,7 +487,36 @@ int make_plan(long long M, long long N, long long K, const kx_plan_override* ov,
 int make_plan_from(long long M, long long N, long long K, const kx_plan_override* ov, int sms, Plan* pl) {
     const int nkb = ceil_div(K, 64);
     int path = ov ? ov->path : KX_PATH_AUTO;
-    if (path == KX_PATH_AUTO) path = (M <= 64) ? KX_PATH_SWAP : KX_PATH_TILE;
+    // A handful of rows: the CUDA-core kernel that only streams W (needs whole 16-byte chunks of K and
+    // output columns in groups of its rows-per-CTA count).
+    const bool gemv_ok = M <= kGemvMaxM && K >= 8 && (K % 8) == 0 && (N % 8) == 0;
+    if (path == KX_PATH_AUTO) path = gemv_ok ? KX_PATH_GEMV : (M <= 64) ? KX_PATH_SWAP : KX_PATH_TILE;
+    if (path == KX_PATH_GEMV) {
+        if (!gemv_ok) return KX_ERR_PLAN;
+        if (ov && (ov->cta_pair > 1 || ov->stream_k > 1 || ov->narrow_tail > 1 || ov->cluster_reduce > 1 ||
+                   ov->k_cluster > 1 || ov->max_ctas > 0 || ov->stages > 0 || ov->raster_group > 0))
+            return KX_ERR_PLAN;
+        // rows of W per CTA (block_n) and warps per CTA sharing the K range (split_k).  Defaults measured on
+        // B200 for M = 1, K = N = 2048..8192: four rows per CTA and one warp per 128 chunks of a row (at
+        // least four): 4 / 4 / 5 / 8 warps were the best or within noise of it at K = 2048 / 4096 / 5120 / 8192.
+        const int rw = (ov && ov->block_n) ? ov->block_n : 4;
+        const int warps = (ov && ov->split_k) ? ov->split_k
+                                              : std::max(4, std::min(16, static_cast<int>((K / 8 + 64) / 128)));
+        if (!gemv_variant_exists(rw, warps)) return KX_ERR_PLAN;
+        pl->path = path;
+        pl->bn = rw;
+        pl->ctas = 1;
+        pl->splits = warps;
+        pl->stages = 0;
+        pl->smem = 0;
+        pl->tiles_n = static_cast<int>(N / rw);
+        pl->tiles_m = 1;
+        pl->units = pl->tiles_n;
+        pl->grid = pl->tiles_n;
+        pl->ws_bytes = 0;
+        pl->sk_tile0 = pl->narrow_tile0 = pl->units;
+        return KX_OK;
+    }
     if (path != KX_PATH_TILE && path != KX_PATH_SWAP) return KX_ERR_PLAN;
     const int max_ctas = (ov && ov->max_ctas > 0) ? std::min(ov->max_ctas, sms) : sms;
     pl->path = path;
@@ -604,18 +648,28 @@ int make_plan_from(long long M, long long N, long long K, const kx_plan_override
         // Cluster reduction (2..8 splits): partials stay in shared memory and are summed
         // through distributed shared memory.  Needs every CTA of a cluster resident at once,
         // which the hardware guarantees per cluster; one unit per CTA.
-        int cr = ov ? ov->cluster_reduce : 0;                 // 0 auto, 1 off, 2 on
+        int cr = ov ? ov->cluster_reduce : 0;                 // 0 auto, 1 off, 2 pull, 3 push
         const bool auto_split = !(ov && ov->split_k > 0);
+        // The push form runs by request only: measured on B200 it is no faster than the pull form (its
+        // 16 to 32 remote 4-byte stores per thread take as long as the pull form's barrier and remote loads:
+        // 12.2 vs 11.6 us at M = 32, N = K = 4096; 27.5 vs 27.6 at 8192).
+        const bool push = (cr == 3);
+        if (cr == 3 && !v->fn_push) return KX_ERR_PLAN;
         if (cr != 1 && auto_split) {
             // largest cluster size (= split count) whose clusters are all resident at once
             splits = std::min(splits, 8);
-            while (splits > 1 && max_active_clusters(v, splits) < tiles) --splits;
+            while (splits > 1 && max_active_clusters(v, splits, push) < tiles) --splits;
         }
         const bool cr_ok = splits >= 2 && splits <= 8 && !(ov && ov->max_ctas > 0);
-        if (cr == 0) cr = cr_ok ? 2 : 1;
-        if (cr == 2 && !cr_ok) return KX_ERR_PLAN;
-        pl->cluster_reduce = (cr == 2) ? 1 : 0;
-        if (pl->cluster_reduce) pl->fn = v->fn_cluster;
+        if (cr == 0) cr = cr_ok ? (push ? 3 : 2) : 1;
+        if (cr >= 2 && !cr_ok) return KX_ERR_PLAN;
+        if (cr < 1 || cr > 3) return KX_ERR_PLAN;
+        pl->cluster_reduce = (cr >= 2) ? cr - 1 : 0;          // 0 workspace, 1 pull, 2 push
+        if (cr == 2) pl->fn = v->fn_cluster;
+        if (cr == 3) {
+            pl->fn = v->fn_push;
+            pl->smem = v->smem_push;
+        }
         pl->splits = splits;
         pl->ws_bytes = (splits > 1 && !pl->cluster_reduce) ? static_cast<size_t>(splits) * M * N * 4 : 0;
         if (pl->ws_bytes > kWorkspaceBytes) return KX_ERR_WORKSPACE;
@@ -715,7 +769,7 @@ int run(const void* X, const void* W, const void* bias, const void* R, void* Y, 
     if ((N % 8) != 0) {
         // only reachable with pitched operands: the small-M kernel's epilogue works in 8-byte column
         // groups, so a ragged N always takes the tile kernel (TMA clips the last columns)
-        if (ov && ov->path == KX_PATH_SWAP) return KX_ERR_PLAN;
+        if (ov && (ov->path == KX_PATH_SWAP || ov->path == KX_PATH_GEMV)) return KX_ERR_PLAN;
         std::memset(&ragged, 0, sizeof ragged);
         if (ov) ragged = *ov;
         ragged.path = KX_PATH_TILE;
@@ -730,6 +784,25 @@ int run(const void* X, const void* W, const void* bias, const void* R, void* Y, 
     if (log_enabled())
         std::fprintf(stderr, "[kx] M=%lld N=%lld K=%lld path=%d bn=%d ctas=%d stages=%d splits=%d streamk=%d grid=%d units=%d\n",
                      M, N, K, pl.path, pl.bn, pl.ctas, pl.stages, pl.splits, pl.stream_k, pl.grid, pl.units);
+
+    if (pl.path == KX_PATH_GEMV) {
+        GemvLaunch g;
+        g.X = X; g.W = W; g.bias = bias; g.R = R; g.Y = Y;
+        g.M = M; g.N = N; g.K = K;
+        g.ldx = ldx; g.ldw = ldw; g.ldr = ldr; g.ldy = ldy;
+        g.rows_per_cta = pl.bn;
+        g.warps = pl.splits;
+        // L2 request ahead of the dependency wait: `l2_prefetch` k-blocks of 128 bytes of every row when
+        // given, none when negative; by default the whole row while W is small against the L2 (measured:
+        // 3.3 vs 3.6 us at 2048^2, 7.7 vs 8.1 at 4096^2) and its first 2 KB beyond (whole rows of a 52 MB or
+        // 134 MB matrix push the running kernel's lines out: 11.6 vs 11.0 us at 5120^2)
+        const long long row_bytes = K * 2;
+        const int pf = ov ? ov->l2_prefetch : 0;
+        const long long pf_default = (N * row_bytes <= (48ll << 20)) ? row_bytes : std::min<long long>(row_bytes, 2048);
+        g.pf_bytes = pf < 0 ? 0 : static_cast<int>(pf == 0 ? pf_default : std::min<long long>(row_bytes, 128ll * pf));
+        g.pdl = !(ov && ov->no_pdl);
+        return launch_gemv(g, stream);
+    }
 
     cudaLaunchConfig_t cfg;
     std::memset(&cfg, 0, sizeof cfg);

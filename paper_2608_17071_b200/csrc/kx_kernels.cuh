@@ -69,7 +69,7 @@ constexpr int kBlockK = 64;           // BF16 elements per k-block = one 128-byt
 constexpr int kABytes = 128 * 128;    // 128 operand rows x 128 bytes
 
 constexpr uint32_t kWhereEmpty = 1, kWhereFull = 2, kWhereAccEmpty = 3, kWhereAccFull = 4,
-                   kWhereRFull = 5, kWhereDrain = 6;
+                   kWhereRFull = 5, kWhereDrain = 6, kWherePartials = 7;
 
 struct Waiter {
     volatile uint32_t* abort_flag;   // this CTA's shared abort word
@@ -79,6 +79,22 @@ struct Waiter {
     __device__ __forceinline__ void raise(uint32_t where) const {
         atomicCAS(const_cast<uint32_t*>(abort_flag), 0u, where);
         if (peer_abort) st_cluster_u32(peer_abort, where);
+    }
+    // the same for a barrier on which other CTAs of the cluster arrive (acquire at cluster scope)
+    __device__ __forceinline__ bool wait_cluster(uint32_t bar, uint32_t parity, uint32_t where) const {
+        if (mbar_try_wait_cluster(bar, parity)) return true;
+        const unsigned long long t0 = globaltimer_ns();
+        uint32_t it = 0;
+        for (;;) {
+            if (mbar_try_wait_cluster(bar, parity)) return true;
+            if ((++it & 15u) == 0u) {
+                if (*abort_flag != 0) return false;
+                if (globaltimer_ns() - t0 > limit_ns) {
+                    raise(where);
+                    return false;
+                }
+            }
+        }
     }
     // true = barrier phase completed; false = gave up (abort raised)
     __device__ __forceinline__ bool wait(uint32_t bar, uint32_t parity, uint32_t where) const {
@@ -1033,41 +1049,57 @@ struct SwapParams {
 };
 
 // KBS = k-blocks per ring stage (1 or 2), as in TileCfg: [W kb][W kb+1][X kb][X kb+1].
-template <int BN, int STAGES, int KBS = 1>
+// PUSH: room for the partial rows that the other CTAs of a cluster send to this one (see MODE 2 below):
+// up to BN + 7 rows of 128 FP32 values.
+template <int BN, int STAGES, int KBS = 1, bool PUSH = false>
 struct SwapCfg {
     static constexpr int B_BYTES = BN * 128;
     static constexpr int STAGE_BYTES = KBS * (kABytes + B_BYTES);
-    static constexpr int NUM_BARS = 2 * STAGES + 4 + 2;
-    static constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + 1024;
+    static constexpr int NUM_BARS = 2 * STAGES + 4 + 3;
+    static constexpr int RECV_BYTES = PUSH ? (BN + 8) * 512 : 0;
+    static constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + RECV_BYTES + 1024;
+    static_assert(SMEM_BYTES <= 232448, "shared memory");
     static constexpr int TMEM_COLS = tmem_cols_for(2 * BN);
     static_assert(BN % 16 == 0 && BN >= 16 && BN <= 256, "BN");
     static_assert(NUM_BARS * 8 + 16 <= 1024, "barrier area");
     static_assert(STAGE_BYTES % 1024 == 0, "stage alignment");
 };
 
-// CLUSTER = true: the K splits of one tile form a thread-block cluster (cluster size ==
-// p.splits <= 8, one unit per CTA, grid == num_units).  Each CTA parks its FP32 partial in
-// its own shared memory, the cluster meets on the hardware cluster barrier, and every CTA
-// then finishes a share of the tile's rows by reading all partials through distributed
-// shared memory in split order: no workspace, no atomics, no fences, same deterministic sum.
-template <int BN, int STAGES, bool CLUSTER, int KBS = 1>
+// MODE 0: K splits are summed through the FP32 workspace by the last CTA of a tile to arrive.
+// MODE 1 and 2: the K splits of one tile form a thread-block cluster (cluster size == p.splits <= 8, one
+// unit per CTA, grid == num_units) and row i of the tile is finished by CTA i % splits, which sums the
+// partials in split order: no workspace, no atomics, same deterministic sum.
+//   MODE 1 (pull): each CTA parks its FP32 partial in its own shared memory (the idle operand ring), the
+//   cluster meets on the hardware cluster barrier, and the finishers read the partials through distributed
+//   shared memory.
+//   MODE 2 (push): each CTA stores the rows of its partial straight from registers into the receive area of
+//   their finishers (st.shared::cluster) and arrives on the finisher's mbarrier; a finisher waits on that one
+//   (bounded) barrier and then sums from its own shared memory.  No round trip of remote loads and no
+//   cluster-wide meeting on the critical path: the hardware cluster barrier is only used to make sure that
+//   every CTA has started before the first remote store and that none leaves while a peer might still
+//   write to it, and both of its waits are reached long after everybody arrived.
+template <int BN, int STAGES, int MODE, int KBS = 1>
 __global__ void __launch_bounds__(kThreads, 1)
 kx_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
                const SwapParams p) {
-    using C = SwapCfg<BN, STAGES, KBS>;
+    constexpr bool CLUSTER = (MODE == 1);
+    constexpr bool PUSH = (MODE == 2);
+    using C = SwapCfg<BN, STAGES, KBS, PUSH>;
     static_assert(!CLUSTER || BN * 128 * 4 <= STAGES * C::STAGE_BYTES, "partial must fit in the idle ring");
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t* const gbase = smem_raw + (base - raw);
     const uint32_t s_stage = base;
-    const uint32_t s_bar = base + STAGES * C::STAGE_BYTES;
+    const uint32_t s_recv = base + STAGES * C::STAGE_BYTES;  // MODE 2: partial rows pushed by the cluster
+    const uint32_t s_bar = s_recv + C::RECV_BYTES;
     auto full = [&](int s) { return s_bar + 8u * s; };
     auto empty = [&](int s) { return s_bar + 8u * (STAGES + s); };
     auto acc_full = [&](int b) { return s_bar + 8u * (2 * STAGES + b); };
     auto acc_empty = [&](int b) { return s_bar + 8u * (2 * STAGES + 2 + b); };
     const uint32_t drain_bar = s_bar + 8u * (2 * STAGES + 4);
     const uint32_t epi_bar = s_bar + 8u * (2 * STAGES + 5);   // the four epilogue warps meet here
+    const uint32_t red_bar = s_bar + 8u * (2 * STAGES + 6);   // MODE 2: every pushing warp of the cluster arrives here
     volatile uint32_t* const s_tmem =
         reinterpret_cast<volatile uint32_t*>(gbase + (s_bar - base) + 8 * C::NUM_BARS);
     volatile uint32_t* const s_abort = s_tmem + 1;
@@ -1105,6 +1137,7 @@ kx_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
             }
             mbar_init(drain_bar, 1);
             mbar_init(epi_bar, 4);
+            mbar_init(red_bar, 4 * static_cast<uint32_t>(p.splits));
             fence_mbar_init();
         }
         __syncwarp();
@@ -1114,6 +1147,10 @@ kx_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    // MODE 2: first cluster barrier (every CTA has started and initialised its barriers); each thread
+    // waits for it only where it first needs it, after the main loop
+    if constexpr (PUSH) cluster_arrive();
+    [[maybe_unused]] bool pushed_wait = false;       // MODE 2: this thread has passed the first cluster wait
     const uint32_t tmem_base = *s_tmem;
     if (threadIdx.x == 0) KX_TRACE_POINT(p, blockIdx.x, 1);
     pdl_wait_prior();          // prologue above overlapped the previous kernel's tail
@@ -1159,6 +1196,11 @@ kx_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
                 }
             }
         }
+        if constexpr (PUSH) {
+            __syncwarp();
+            cluster_wait();
+            cluster_arrive_relaxed();
+        }
     } else if (warp == 5) {
         if (lane == 0) {
             constexpr uint32_t idesc = idesc_bf16_f32(128, BN);
@@ -1200,6 +1242,11 @@ kx_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
                 while (!mbar_try_wait(drain_bar, 0) && ++spins < (1u << 20)) {}
             }
         }
+        if constexpr (PUSH) {
+            __syncwarp();
+            cluster_wait();
+            cluster_arrive_relaxed();
+        }
     } else {
         // epilogue: lane <-> one W row (output column n); TMEM columns <-> output rows m
         const int q = warp;
@@ -1228,12 +1275,31 @@ kx_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
             if (!__all_sync(0xffffffffu, wt.wait(acc_full(b), aph, kWhereAccFull))) { ok = false; break; }
             tc_fence_after();
             if (etid == 0 && ucount == 0) KX_TRACE_POINT(p, blockIdx.x, 5);
+            if constexpr (PUSH) {
+                if (!pushed_wait) {                       // every CTA of the cluster is up: remote stores may begin
+                    __syncwarp();
+                    cluster_wait();
+                    pushed_wait = true;
+                }
+            }
 #pragma unroll 1
             for (int c0 = 0; c0 < m_cnt; c0 += 16) {
                 uint32_t a[16];
                 tmem_ld_32x16(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + b * BN + c0, a);
                 tmem_ld_wait();
-                if (CLUSTER && p.splits > 1) {
+                if (PUSH && p.splits > 1) {
+                    // row i of the tile is finished by CTA i % splits; this split's partial of that row goes
+                    // into slot [sp][i / splits] of that CTA's receive area (128 columns per row: a warp
+                    // writes 128 contiguous bytes)
+                    const int rows_per = (BN + p.splits - 1) / p.splits;
+                    int d = c0 % p.splits, k = c0 / p.splits;
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        if (c0 + i < m_cnt)
+                            st_cluster_u32(map_to_cta(s_recv + static_cast<uint32_t>(((sp * rows_per + k) * 128 + etid) * 4), d), a[i]);
+                        if (++d == p.splits) { d = 0; ++k; }
+                    }
+                } else if (CLUSTER && p.splits > 1) {
                     // partial -> this CTA's shared memory (the operand ring is idle by now):
                     // red[m_local][128 columns], conflict-free for a fixed row
                     float* red = reinterpret_cast<float*>(gbase);
@@ -1267,7 +1333,18 @@ kx_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(acc_empty(b));
-            if (!CLUSTER && p.splits > 1) {
+            if (PUSH && p.splits > 1) {
+                // this warp's rows are on their way: tell every finisher (the fence of an arriving lane orders
+                // the whole warp's stores, which the warp barrier above made known to it, before its arrival)
+                if (etid == 0) KX_TRACE_POINT(p, blockIdx.x, 8);
+                if (lane < p.splits) {                    // lane d tells finisher d
+                    fence_acq_rel_cluster();
+                    mbar_arrive_cluster_relaxed(map_to_cta(red_bar, lane));
+                }
+                __syncwarp();
+                if (etid == 0) KX_TRACE_POINT(p, blockIdx.x, 12);
+            }
+            if (MODE == 0 && p.splits > 1) {
                 // last CTA to finish this tile sums the splits in fixed order (deterministic)
                 if (etid == 0 && ucount == 0) KX_TRACE_POINT(p, blockIdx.x, 6);
                 __threadfence();
@@ -1347,6 +1424,79 @@ kx_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     }
 
     __syncwarp();
+    if constexpr (PUSH) {
+        // Finish the rows dealt to this CTA from the partials its peers (and itself) pushed.  Warps 0-3
+        // still owe the second arrival of the cluster barrier (and the first wait if their loop ended
+        // early); warps 4 and 5 have done both above.
+        const bool reducer = warp < 4 && p.splits > 1 && static_cast<int>(blockIdx.x) < p.num_units;
+        if (warp < 4) {
+            int nt = 0, mt = 0, sp = 0, kb0 = 0, kb1 = 0;
+            if (reducer) unit_coords(blockIdx.x, nt, mt, sp, kb0, kb1);
+            const int n4 = nt * 128 + lane * 4;
+            const bool n_ok = reducer && n4 < p.N;
+            const int m0 = mt * BN;
+            const int m_cnt = reducer ? min(BN, p.M - m0) : 0;
+            const int rows_per = (BN + p.splits - 1) / p.splits;
+            auto tile_row = [&](int k) { return sp + k * p.splits; };
+            // residual and bias of the first rows are fetched before the wait: they do not depend on the
+            // partials, and R may alias Y so the loads must precede the stores
+            constexpr int kPre = 4;
+            uint2 rv[kPre];
+            float b4[4] = {0.f, 0.f, 0.f, 0.f};
+            if (n_ok) {
+                if (p.has_bias) {
+                    const uint2 bb = __ldg(reinterpret_cast<const uint2*>(p.bias + n4));
+                    b4[0] = bf16_lo(bb.x); b4[1] = bf16_hi(bb.x); b4[2] = bf16_lo(bb.y); b4[3] = bf16_hi(bb.y);
+                }
+#pragma unroll
+                for (int u = 0; u < kPre; ++u) {
+                    const int i = tile_row(warp + 4 * u);
+                    rv[u] = (p.has_r && i < m_cnt)
+                                ? *reinterpret_cast<const uint2*>(p.R + static_cast<size_t>(m0 + i) * p.ldr + n4)
+                                : make_uint2(0u, 0u);
+                }
+            }
+            // first cluster wait if the epilogue loop never reached it (a wait that gave up; warp-uniform),
+            // then the second arrival: this thread's remote stores and arrivals are all issued
+            if (!pushed_wait) cluster_wait();
+            cluster_arrive_relaxed();
+            if (threadIdx.x == 0) KX_TRACE_POINT(p, blockIdx.x, 6);
+            bool have = true;
+            if (reducer) have = __all_sync(0xffffffffu, wt.wait_cluster(red_bar, 0u, kWherePartials));
+            if (threadIdx.x == 0) KX_TRACE_POINT(p, blockIdx.x, 7);
+            if (reducer && have) {
+#pragma unroll 1
+                for (int u = 0; tile_row(warp + 4 * u) < m_cnt; ++u) {
+                    const int k = warp + 4 * u, i = tile_row(k);
+                    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+                    const uint32_t src = s_recv + static_cast<uint32_t>((k * 128 + lane * 4) * 4);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        if (j < p.splits) {
+                            float4 t;
+                            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                                         : "=f"(t.x), "=f"(t.y), "=f"(t.z), "=f"(t.w)
+                                         : "r"(src + static_cast<uint32_t>(j * rows_per * 512)));
+                            v.x += t.x; v.y += t.y; v.z += t.z; v.w += t.w;
+                        }
+                    if (n_ok) {
+                        uint2 rr = make_uint2(0u, 0u);
+                        if (u < kPre) {
+#pragma unroll
+                            for (int uu = 0; uu < kPre; ++uu)
+                                if (uu == u) rr = rv[uu];
+                        } else if (p.has_r) {
+                            rr = *reinterpret_cast<const uint2*>(p.R + static_cast<size_t>(m0 + i) * p.ldr + n4);
+                        }
+                        const float o0 = v.x + b4[0] + bf16_lo(rr.x), o1 = v.y + b4[1] + bf16_hi(rr.x);
+                        const float o2 = v.z + b4[2] + bf16_lo(rr.y), o3 = v.w + b4[3] + bf16_hi(rr.y);
+                        *reinterpret_cast<uint2*>(p.Y + static_cast<size_t>(m0 + i) * p.ldy + n4) =
+                            make_uint2(pack_bf16x2(o0, o1), pack_bf16x2(o2, o3));
+                    }
+                }
+            }
+        }
+    }
     if constexpr (CLUSTER) {
         // Every thread of every CTA of the cluster passes both barriers, whatever happened in
         // its role above (all waits there are bounded), so the hardware barrier cannot hang.
@@ -1427,6 +1577,12 @@ kx_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
             }
         }
         cluster_arrive();
+        cluster_wait();
+    }
+    if constexpr (PUSH) {
+        // second cluster wait: no CTA leaves while a peer (one that is late, or whose finisher gave up)
+        // might still store into its receive area
+        __syncwarp();
         cluster_wait();
     }
     if (threadIdx.x == 0) KX_TRACE_POINT(p, blockIdx.x, 9);

@@ -36,6 +36,11 @@ SWAP_VARIANTS = [
     # the variants with one k-block per ring stage (the defaults hold two)
     dict(path=S, block_n=16, split_k=4, stages=12), dict(path=S, block_n=32, split_k=3, stages=11, cluster_reduce=1),
     dict(path=S, block_n=64, split_k=2, stages=9), dict(path=S, block_n=128, split_k=5, stages=7), dict(path=S, block_n=256, split_k=1, stages=4),
+    # cluster reduction with the partial rows pushed to their finishers (3) or pulled by them (2)
+    dict(path=S, block_n=16, split_k=4, cluster_reduce=3), dict(path=S, block_n=32, split_k=3, cluster_reduce=3),
+    dict(path=S, block_n=32, split_k=8, cluster_reduce=3), dict(path=S, block_n=64, split_k=2, cluster_reduce=3),
+    dict(path=S, block_n=128, split_k=7, cluster_reduce=3), dict(path=S, block_n=32, split_k=3, cluster_reduce=2),
+    dict(path=S, block_n=64, split_k=6, cluster_reduce=2),
 ]
 
 
@@ -187,7 +192,8 @@ def test_k_cluster_random_data_and_bad_plans():
 @pytest.mark.parametrize("depth", [-1, 0, 1, 3, 1000])
 @pytest.mark.parametrize("base", [dict(path=T, block_n=256, cta_pair=2), dict(path=T, block_n=128, cta_pair=1),
                                   dict(path=T, block_n=256, cta_pair=1, k_cluster=2), dict(path=T, block_n=256, cta_pair=2, narrow_tail=2),
-                                  dict(path=S, block_n=32, split_k=3), dict(path=S, block_n=16, split_k=4, cluster_reduce=2)], ids=vid)
+                                  dict(path=S, block_n=32, split_k=3), dict(path=S, block_n=16, split_k=4, cluster_reduce=2),
+                                  dict(path=S, block_n=32, split_k=4, cluster_reduce=3)], ids=vid)
 def test_l2_prefetch_depth_changes_no_bit(base, depth):
     """The tiles a CTA requests into L2 ahead of the dependency wait are a hint only: every depth
     (none, ring depth, shallower, deeper than the K range) gives the same bits, and a weight
@@ -251,7 +257,8 @@ def test_zero_weight_returns_residual_plus_bias(ov):
     assert np.array_equal(y, oracle.round_bf16(f(d["R"]) + f(d["bias"])[None, :]))
 
 
-@pytest.mark.parametrize("ov", [TILE_VARIANTS[0], TILE_VARIANTS[2], TILE_VARIANTS[3], SWAP_VARIANTS[2], SWAP_VARIANTS[6]], ids=vid)
+@pytest.mark.parametrize("ov", [TILE_VARIANTS[0], TILE_VARIANTS[2], TILE_VARIANTS[3], SWAP_VARIANTS[2], SWAP_VARIANTS[6],
+                                SWAP_VARIANTS[18]], ids=vid)
 def test_selectors(ov):
     """W a permutation matrix picks columns of X; one-hot X picks columns of W."""
     M = 24 if ov["path"] == S and ov["block_n"] < 128 else 260
@@ -278,7 +285,7 @@ def test_power_of_two_scaling_is_bitwise(ov):
 
 
 @pytest.mark.parametrize("ov", [None, TILE_VARIANTS[0], TILE_VARIANTS[2], TILE_VARIANTS[3], TILE_VARIANTS[4],
-                                SWAP_VARIANTS[1], SWAP_VARIANTS[5], SWAP_VARIANTS[6]],
+                                SWAP_VARIANTS[1], SWAP_VARIANTS[5], SWAP_VARIANTS[6], SWAP_VARIANTS[18], SWAP_VARIANTS[20]],
                          ids=lambda v: "auto" if v is None else vid(v))
 def test_in_place_matches_out_of_place(ov):
     """Y aliased onto R (the paper's destination/residual aliasing) gives the same bits."""
@@ -470,6 +477,10 @@ def test_non_default_stream_and_plan_query():
     assert info.path == S and info.block_n == 32 and info.split_k >= 1
     ws = info.split_k * 32 * 4096 * 4 if (info.split_k > 1 and not info.cluster_reduce) else 0
     assert info.workspace_bytes == ws and (info.cluster_reduce == 0 or 2 <= info.split_k <= 8)
+    assert info.cluster_reduce == 1          # the splits form a cluster; finishers pull the partial rows
+    assert kx.kx_plan_query(32, 4096, 4096, ov=kx.make_override(path=S, cluster_reduce=3)).cluster_reduce == 2
+    with pytest.raises(kx.KxError):          # no push form with 256 rows of X per unit
+        kx.kx_plan_query(200, 4096, 4096, ov=kx.make_override(path=S, block_n=256, split_k=2, cluster_reduce=3))
     with pytest.raises(kx.KxError):
         kx.kx_plan_query(4096, 4096, 4096, ov=kx.make_override(path=T, block_n=96))
     X, W, b, R = ternary_case(256, 512, 256, seed=13)
