@@ -37,9 +37,10 @@ L2_BYTES = 126 * (1 << 20)
 METRIC = "bf16_tflops"
 UNIT = "TFLOP/s"
 HEADLINE = "cfg2"
-# DRAM traffic per launch of the dominant kernel from the ncu capture summarised in
-# profiles/ (dram__bytes_read.sum + dram__bytes_write.sum); None until captured.
-NCU_TRAFFIC_BYTES = {"cfg2": 154686976}   # profiles/kx_tile_kernel_pair_cfg2.md
+# DRAM traffic per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum of one
+# ncu capture of that launch); None until captured.
+NCU_TRAFFIC_BYTES = {"cfg2": 154686976}
+PATH_NAMES = {1: "tile", 2: "swap", 3: "gemv", 4: "skinny"}
 
 
 def load_peaks():
@@ -64,6 +65,7 @@ class ClockSampler:
         self.index, self.period = index, period_s
         self.samples, self.reasons = [], set()
         self.max_mhz = None
+        self.active = True            # samples count only while a timed block runs (see mark)
         self._stop = threading.Event()
         self._thread = None
         try:
@@ -91,9 +93,15 @@ class ClockSampler:
                 out.append(name)
         return out
 
+    def mark(self, active: bool):
+        self.active = active
+
     def _run(self):
         nv = self.nv
         while not self._stop.is_set():
+            if not self.active:
+                self._stop.wait(self.period)
+                continue
             try:
                 self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
                 try:
@@ -225,6 +233,24 @@ def time_steps(torch, kx, wl, sets, steps, warmup):
     return e0.elapsed_time(e1) * 1e-3 / steps
 
 
+def time_warm(torch, call, steps=200, repeats=3):
+    """Amortised time of one call in a back-to-back stream on the SAME buffers (operands warm in L2 when
+    they fit): the figure for shapes whose roofline time is below the cost of a launch."""
+    ts = []
+    for _ in range(repeats):
+        for _ in range(10):
+            call()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            call()
+        e1.record()
+        torch.cuda.synchronize()
+        ts.append(e0.elapsed_time(e1) * 1e-3 / steps)
+    return sorted(ts)[len(ts) // 2]
+
+
 def time_shape(torch, kx, wl, sets, repeats=5, block_s=0.03, idle_s=0.25):
     """Per-shape protocol of the sweep: `repeats` timed blocks of at most ~block_s seconds of
     back-to-back calls, each after a short idle and 3 warm-up calls, so that every shape is
@@ -321,26 +347,40 @@ def run_ours(args):
     for i in range(max(3, args.warmup)):
         call(kx, wl, sets[i % nsets])
     barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    with ClockSampler(local) as clk:
-        e0.record()
-        for i in range(args.steps):
-            call(kx, wl, sets[i % nsets])
-        e1.record()
-        torch.cuda.synchronize()
-    barrier()
-    sec = e0.elapsed_time(e1) * 1e-3
+    # The timed region: `blocks` blocks of back-to-back steps, each block at least the K steps asked for and
+    # at least ~30 ms long (so that the clock sampler sees every block), each after a short idle so that the
+    # blocks start from the same power state; the step time is the median over the blocks.
+    est = time_steps(torch, kx, wl, sets, 3, 0)
+    blocks = 5
+    steps_b = int(max(args.steps, min(2000, math.ceil(0.03 / max(est, 1e-7)))))
+    block_s = []
+    with ClockSampler(local, period_s=0.002) as clk:
+        for _ in range(blocks):
+            time.sleep(0.2)
+            for i in range(3):
+                call(kx, wl, sets[i % nsets])
+            barrier()
+            clk.mark(True)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for i in range(steps_b):
+                call(kx, wl, sets[i % nsets])
+            e1.record()
+            torch.cuda.synchronize()
+            clk.mark(False)
+            barrier()
+            block_s.append(max_over_ranks(dist, e0.elapsed_time(e1) * 1e-3, "cuda"))
     code, detail = kx.kx_last_device_status()
     if code != 0:
         raise SystemExit(f"kernel reported status {code} (wait {detail})")
-    sec = max_over_ranks(dist, sec, "cuda")
-    per_step = sec / args.steps
+    per_step = sorted(block_s)[len(block_s) // 2] / steps_b
     value = world * wl.flops / per_step / 1e12
-    sustained = sec > 1.0
+    sustained = False                    # 30 ms blocks after an idle: the burst regime of the measured peaks
     rl = roof(wl, per_step, peaks, sustained)
     rl["traffic"] = NCU_TRAFFIC_BYTES.get(headline)
-    rl["peak_source"] = f"of {peaks['source']} ({'sustained' if sustained else 'burst'} bf16 GEMM figure)"
-    rl["frac_of_nominal_2250"] = rl["achieved"] / 2250.0 if rl["bound"] == "tensor" else None
+    rl["peak_source"] = f"of {peaks['source']} (burst bf16 GEMM figure: every timed block is ~30 ms after an idle)"
+    rl["frac_nominal"] = rl["achieved"] / 2250.0 if rl["bound"] == "tensor" else rl["achieved"] / 8000.0
+    rl["time_x_mhz"] = None
 
     # ---- end to end through the host-buffer entry point (pinned host memory)
     e2e = None
@@ -368,7 +408,14 @@ def run_ours(args):
 
     # ---- every other workload (rank 0, N = 1 only): per-shape roofline lines
     shapes = []
+    launch_floor_us = None
     if rank == 0 and world == 1 and "shapes" in sections:
+        # cost of one call in a stream of calls when there is (almost) nothing to do: the library's own
+        # kernel on an 1 x 8 x 8 problem, launched like every other call (programmatic dependent launch)
+        tiny = inputs.Workload("tiny", 1, 8, 8, 0, True, True)
+        tset = bind_sets(kx, tiny, device_sets(torch, tiny, 2))
+        launch_floor_us = time_warm(torch, lambda: (tset[0](), tset[1]()), steps=200) / 2 * 1e6
+        print(f"[bench] launch floor (1 x 8 x 8 call in a stream of calls): {launch_floor_us:.2f} us", file=sys.stderr, flush=True)
         order = ["cfg1", "cfg2", "cfg4", "cfg5", "gemm4096"] + [w.name for w in inputs.sweep_workloads()]
         for name in order:
             w = wls[name]
@@ -383,15 +430,58 @@ def run_ours(args):
                            "bound": r["bound"], "frac": r["frac"], "frac_best": roof(w, tbest, peaks, False)["frac"],
                            "frac_nominal": (w.flops / t / 1e12 / 2250.0) if r["bound"] == "tensor"
                            else (w.algorithmic_bytes / t / 1e9 / 8000.0),
-                           "plan": {"path": "tile" if pi.path == 1 else "swap", "block_n": pi.block_n,
+                           "plan": {"path": PATH_NAMES.get(pi.path, str(pi.path)), "block_n": pi.block_n,
                                     "cta_pair": pi.cta_pair, "split_k": pi.split_k, "grid": pi.grid,
                                     "narrow_tiles": pi.narrow_tiles},
                            "operand_sets": len(ss)})
+            # against roofline + launch floor (what a stream of such calls can reach at best)
+            t_roof = max(w.flops / (peaks["bf16_tflops"] * 1e12), w.algorithmic_bytes / (peaks["hbm_gbs"] * 1e9))
+            shapes[-1]["frac_vs_roofline_plus_floor"] = (t_roof + launch_floor_us * 1e-6) / t
+            if t_roof < 3e-6:
+                # roofline time below ~3 us: also the amortised time of a back-to-back stream on ONE operand
+                # set (warm L2), labelled as such
+                tw = time_warm(torch, ss[0])
+                shapes[-1]["amortised_warm_us"] = tw * 1e6
+                shapes[-1]["amortised_warm_note"] = "same buffers, back-to-back stream of 200 calls, operands warm in L2"
             del ss
             torch.cuda.empty_cache()
             print(f"[bench] {name:>18s} M={w.M:<6d} N={w.N:<5d} K={w.K:<6d} {t*1e6:9.1f} us (best {tbest*1e6:7.1f}) "
                   f"{w.flops/t/1e12:8.1f} TF {w.algorithmic_bytes/t/1e9:7.0f} GB/s  {r['bound']:6s} "
                   f"{r['frac']*100:5.1f}% of {peaks['source']}", file=sys.stderr, flush=True)
+
+    # ---- sustained leg: the large tensor-bound workloads back to back for >= 2 s each (the part settles at its
+    # power-limited clock), against the measured sustained GEMM figure, with the SM clock sampled meanwhile
+    sustained_leg = []
+    if rank == 0 and world == 1 and "sustained" in sections:
+        for name in ("cfg2", "cfg4", "cfg5"):
+            w = wls[name]
+            ss = sets if name == headline else bind_sets(kx, w, device_sets(torch, w, sets_needed(w)))
+            est = time_steps(torch, kx, w, ss, 3, 3)
+            n = int(max(10, math.ceil(2.0 / max(est, 1e-7))))
+            for i in range(max(3, n // 10)):           # bring the part to its loaded state first
+                ss[i % len(ss)]()
+            torch.cuda.synchronize()
+            with ClockSampler(local, period_s=0.01) as ck:
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for i in range(n):
+                    ss[i % len(ss)]()
+                e1.record()
+                torch.cuda.synchronize()
+            t = e0.elapsed_time(e1) * 1e-3 / n
+            cs = ck.summary()
+            tf = w.flops / t / 1e12
+            sustained_leg.append({"name": name, "calls": n, "seconds": t * n, "us": t * 1e6, "tflops": tf,
+                                  "frac_of_sustained_peak": tf / peaks["bf16_tflops_sustained"],
+                                  "peak_sustained": peaks["bf16_tflops_sustained"], "frac_nominal": tf / 2250.0,
+                                  "sm_mhz_median": cs["sm_mhz"], "reasons": cs["reasons"], "clock_samples": cs["samples"],
+                                  "us_x_ghz": (t * 1e6 * cs["sm_mhz"] / 1e3) if cs["sm_mhz"] else None})
+            print(f"[bench] sustained {name}: {n} calls in {t*n:.2f} s, {t*1e6:.1f} us per call, {tf:.1f} TF = "
+                  f"{tf / peaks['bf16_tflops_sustained'] * 100:.1f}% of the sustained {peaks['source']} peak, "
+                  f"SM {cs['sm_mhz']} MHz {cs['reasons']}", file=sys.stderr, flush=True)
+            if name != headline:
+                del ss
+                torch.cuda.empty_cache()
 
     # ---- the step after the projection: RMSNorm of the new residual stream (rank 0, N = 1 only)
     norm = []
@@ -487,9 +577,13 @@ def run_ours(args):
             frac = (ops / t / 1e12 / peak8) if bound == "tensor" else (nbytes / t / 1e9 / peaks["hbm_gbs"])
             int8.append({"name": name, "us": t * 1e6, "us_best": tbest * 1e6, "tops": ops / t / 1e12,
                          "gbs": nbytes / t / 1e9, "bound": bound, "frac": frac,
-                         "peak": peak8 if bound == "tensor" else peaks["hbm_gbs"], "operand_sets": ns})
+                         "peak": peak8 if bound == "tensor" else peaks["hbm_gbs"],
+                         "peak_source": ("derived: 2x the measured BF16 GEMM figure, by the nominal ratio of the tensor-core rates"
+                                         if bound == "tensor" else f"{peaks['source']} copy bandwidth"),
+                         "operand_sets": ns})
             print(f"[bench] {name:>30s} {t*1e6:9.1f} us (best {tbest*1e6:7.1f}) {ops/t/1e12:8.1f} TOP/s {nbytes/t/1e9:7.0f} GB/s  "
-                  f"{bound:6s} {frac*100:5.1f}% of {peaks['source']}", file=sys.stderr, flush=True)
+                  f"{bound:6s} {frac*100:5.1f}% of {'2 x ' + peaks['source'] + ' BF16 peak (derived)' if bound == 'tensor' else peaks['source']}",
+                  file=sys.stderr, flush=True)
 
         for (Mn, Nn) in [(4096, 4096), (16384, 4096)]:
             nbytes = 3.0 * Mn * Nn + 4.0 * Mn + 2.0 * Nn
@@ -739,9 +833,10 @@ def run_ours(args):
             t, tbest, _ = time_shape(torch, kx, wlo, calls)
             int8.append({"name": wlo.name, "us": t * 1e6, "us_best": tbest * 1e6, "tops": ops / t / 1e12,
                          "gbs": nbytes / t / 1e9, "bound": "tensor", "frac": ops / t / 1e12 / peak4, "peak": peak4,
+                         "peak_source": "derived: 4x the measured BF16 GEMM figure, by the nominal ratio of the tensor-core rates",
                          "operand_sets": ns})
             print(f"[bench] {wlo.name:>30s} {t*1e6:9.1f} us (best {tbest*1e6:7.1f}) {ops/t/1e12:8.1f} TOP/s {nbytes/t/1e9:7.0f} GB/s  "
-                  f"tensor {ops/t/1e12/peak4*100:5.1f}% of 4 x {peaks['source']} BF16 peak", file=sys.stderr, flush=True)
+                  f"tensor {ops/t/1e12/peak4*100:5.1f}% of 4 x {peaks['source']} BF16 peak (derived)", file=sys.stderr, flush=True)
             wlq = inputs.Workload(f"quantize_rows_nvfp4_M{Mo}_K{Ko}", Mo, Ko, 0, 0, False, False)
             t, tbest, _ = time_shape(torch, kx, wlq, qcalls)
             report(wlq.name, t, tbest, Mo * Ko * (2.5 + 1.0 / 16), 0.0, ns)
@@ -782,9 +877,10 @@ def run_ours(args):
             t, tbest, _ = time_shape(torch, kx, wls, calls)
             int8.append({"name": wls.name, "us": t * 1e6, "us_best": tbest * 1e6, "tops": ops / t / 1e12,
                          "gbs": nbytes / t / 1e9, "bound": "tensor", "frac": ops / t / 1e12 / peak4, "peak": peak4,
+                         "peak_source": "derived: 4x the measured BF16 GEMM figure, by the nominal ratio of the tensor-core rates",
                          "operand_sets": ns})
             print(f"[bench] {wls.name:>30s} {t*1e6:9.1f} us (best {tbest*1e6:7.1f}) {ops/t/1e12:8.1f} TOP/s {nbytes/t/1e9:7.0f} GB/s  "
-                  f"tensor {ops/t/1e12/peak4*100:5.1f}% of 4 x {peaks['source']} BF16 peak", file=sys.stderr, flush=True)
+                  f"tensor {ops/t/1e12/peak4*100:5.1f}% of 4 x {peaks['source']} BF16 peak (derived)", file=sys.stderr, flush=True)
             del keep, calls
             torch.cuda.empty_cache()
 
@@ -806,6 +902,14 @@ def run_ours(args):
     if rank == 0:
         sweep = [s for s in shapes if s["name"].startswith("sweep_")]
         geo = lambda xs: math.exp(sum(math.log(x) for x in xs) / len(xs)) if xs else None
+        # the metric's own headline (geometric mean of the roofline fraction over the 16-shape sweep) sits
+        # inside `roofline` and `config`, next to the per-launch figure of the headline workload
+        rl["sweep_geomean_frac"] = geo([s["frac"] for s in sweep])
+        rl["sweep_geomean_frac_nominal"] = geo([s["frac_nominal"] for s in sweep])
+        rl["sweep_geomean_tflops"] = geo([s["tflops"] for s in sweep])
+        rl["sweep_shapes"] = len(sweep)
+        cs = clk.summary()
+        rl["time_x_mhz"] = per_step * 1e6 * cs["sm_mhz"] if cs["sm_mhz"] else None
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(3, args.warmup), "ms_per_step": per_step * 1e3, "higher_is_better": True,
@@ -815,17 +919,22 @@ def run_ours(args):
                                    f"{'X,W ~ U(-1,1)/sqrt(K)' if wl.dist == 'uniform' else 'X,W ~ N(0,1)/sqrt(K), R ~ N(0,1)'}, "
                                    f"seed {wl.seed}",
                        "l2": f"rotating {nsets} operand sets ({nsets * wl.algorithmic_bytes / 1e6:.0f} MB) > L2",
-                       "plan": {"path": "tile" if info.path == 1 else "swap", "block_n": info.block_n,
+                       "plan": {"path": PATH_NAMES.get(info.path, str(info.path)), "block_n": info.block_n,
                                 "cta_pair": info.cta_pair, "stages": info.stages, "grid": info.grid,
                                 "tiles": info.tiles, "smem_bytes": info.smem_bytes},
+                       "sweep_shapes": len(sweep),
                        "parallelism": "none" if world == 1 else f"{world} independent row shards, W replicated, no collective"},
             "roofline": rl,
             "cpu_baseline": cpu,
             "e2e": e2e,
-            "gpu_launches": args.steps * info.launches,
-            "gpu_launches_all_legs": (max(3, args.warmup) + args.steps) * info.launches + launches_e2e,
+            "gpu_launches": blocks * steps_b * info.launches,
+            "gpu_launches_all_legs": (max(3, args.warmup) + 3 + blocks * (3 + steps_b)) * info.launches + launches_e2e,
+            "timed_blocks": {"blocks": blocks, "steps_per_block": steps_b, "ms_per_step_each": [b / steps_b * 1e3 for b in block_s],
+                             "note": "value = median block; every block holds at least the --steps asked for"},
             "clocks": clk.summary(),
+            "launch_floor_us": launch_floor_us,
             "shapes": shapes,
+            "sustained": sustained_leg,
             "rmsnorm": norm,
             "swiglu": swiglu,
             "int8": int8,
@@ -847,7 +956,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-sweep", action="store_true", help="headline workload only")
-    ap.add_argument("--sections", default="shapes,rmsnorm,swiglu,int8",
+    ap.add_argument("--sections", default="shapes,sustained,rmsnorm,swiglu,int8",
                     help="comma list of the extra sections to measure after the headline workload")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")

@@ -59,7 +59,7 @@ typedef enum kx_status {
 
 /* Execution paths (the scheduling strategy of Table 1 names split-K and
  * persistent kernels; the per-M specialisation follows Algorithm 3's per-M plan). */
-enum { KX_PATH_AUTO = 0, KX_PATH_TILE = 1, KX_PATH_SWAP = 2, KX_PATH_GEMV = 3 };
+enum { KX_PATH_AUTO = 0, KX_PATH_TILE = 1, KX_PATH_SWAP = 2, KX_PATH_GEMV = 3, KX_PATH_SKINNY = 4 };
 
 /*
  * Plan override for tests, profiling and tuning.  Zero-initialise for "auto".
@@ -67,10 +67,13 @@ enum { KX_PATH_AUTO = 0, KX_PATH_TILE = 1, KX_PATH_SWAP = 2, KX_PATH_GEMV = 3 };
  *                 TMA-store epilogue) / KX_PATH_SWAP (small M: W rows on the MMA
  *                 M axis, split-K, W streamed once) / KX_PATH_GEMV (M <= 4 and K % 8 == 0:
  *                 no tensor core, every CTA streams a few rows of W and reduces over K with
- *                 FP32 warp reductions)
+ *                 FP32 warp reductions) / KX_PATH_SKINNY (M <= 32 and K % 8 == 0: the same streaming
+ *                 organisation with warp-level tensor-core instructions fed from registers, K shared by
+ *                 the 16 warps of a CTA and reduced in its shared memory)
  *   block_n       tile path: 64, 128, 192 or 256 output columns per tile;
  *                 swap path: 16, 32, 64, 128 or 256 X rows per unit;
- *                 GEMV path: 1, 2 or 4 rows of W (output columns) per CTA
+ *                 GEMV path: 1, 2 or 4 rows of W (output columns) per CTA;
+ *                 skinny path: 16 or 32 rows of W per CTA
  *   cta_pair      0 auto, 1 = one CTA per tile, 2 = CTA pair per 256-row tile
  *   split_k       swap path: number of K splits (1..64);
  *                 GEMV path: 1..16 warps per CTA that share the K range of its rows
@@ -129,7 +132,7 @@ typedef struct kx_plan_override {
 
 /* What the planner chose for a shape (kx_plan_query). */
 typedef struct kx_plan_info {
-    int32_t path;          /* KX_PATH_TILE, KX_PATH_SWAP or KX_PATH_GEMV           */
+    int32_t path;          /* KX_PATH_TILE, KX_PATH_SWAP, KX_PATH_GEMV or KX_PATH_SKINNY */
     int32_t block_n;
     int32_t cta_pair;      /* 1 or 2                                               */
     int32_t stages;        /* depth of the TMA -> MMA shared-memory ring           */

@@ -19,7 +19,7 @@ KX_OK = 0
 KX_ERR_NULL, KX_ERR_SHAPE, KX_ERR_ALIGN, KX_ERR_OVERLAP = 1, 2, 3, 4
 KX_ERR_ARCH, KX_ERR_CUDA, KX_ERR_WORKSPACE, KX_ERR_DEVICE_TIMEOUT, KX_ERR_PLAN = 5, 6, 7, 8, 9
 KX_ERR_LIMIT = 10
-KX_PATH_AUTO, KX_PATH_TILE, KX_PATH_SWAP, KX_PATH_GEMV = 0, 1, 2, 3
+KX_PATH_AUTO, KX_PATH_TILE, KX_PATH_SWAP, KX_PATH_GEMV, KX_PATH_SKINNY = 0, 1, 2, 3, 4
 
 EXPORTS = (
     "kx_init", "kx_shutdown", "kx_outproj_residual", "kx_gemm_bf16", "kx_outproj_residual_ex",

@@ -223,7 +223,7 @@ int ensure_device(int dev, DeviceCtx** out) {
                      cudaSuccess &&
                  (!v.fn_push ||
                   cudaFuncSetAttribute(v.fn_push, cudaFuncAttributeMaxDynamicSharedMemorySize, v.smem_push) == cudaSuccess);
-        if (!ok) {
+        if (!ok || skinny_setup() != KX_OK) {
             rc = KX_ERR_CUDA;
             break;
         }
@@ -451,6 +451,34 @@ int max_active_clusters(const SwapVariant* v, int size, bool push = false) {
     return cache[vi][size];
 }
 
+// The same for a tile-kernel variant (BF16 instantiation) in clusters of `size` CTAs.
+int max_active_tile_clusters(const TileVariant* v, int size) {
+    static std::mutex mu;
+    static int cache[sizeof(kTileVariants) / sizeof(kTileVariants[0])][9];
+    const int vi = static_cast<int>(v - kTileVariants);
+    std::lock_guard<std::mutex> lk(mu);
+    if (cache[vi][size] != 0) return cache[vi][size];
+    cudaLaunchConfig_t cfg;
+    std::memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = dim3(size * 64, 1, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = v->smem;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = size;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, v->fn, &cfg) != cudaSuccess) {
+        cudaGetLastError();
+        n = -1;
+    }
+    cache[vi][size] = n > 0 ? n : -1;
+    return cache[vi][size];
+}
+
 int make_plan_from(long long M, long long N, long long K, const kx_plan_override* ov, int sms, Plan* pl);
 
 // Caller's override > static table entry (if it validates) > heuristic.
@@ -490,7 +518,38 @@ int make_plan_from(long long M, long long N, long long K, const kx_plan_override
     // A handful of rows: the CUDA-core kernel that only streams W (needs whole 16-byte chunks of K and
     // output columns in groups of its rows-per-CTA count).
     const bool gemv_ok = M <= kGemvMaxM && K >= 8 && (K % 8) == 0 && (N % 8) == 0;
-    if (path == KX_PATH_AUTO) path = gemv_ok ? KX_PATH_GEMV : (M <= 64) ? KX_PATH_SWAP : KX_PATH_TILE;
+    // Up to 32 rows: the same streaming organisation with warp-level tensor-core instructions.  Measured on
+    // B200 against the split-K tensor-memory kernel (M = 5..32): ahead while W is small (4.1-5.4 vs 6.9-7.8 us
+    // at N = K = 2048, 9.0 vs 10.7-10.9 at 4096 with M <= 16, 10.9 vs 11.5 with M = 32), behind once W is
+    // large (33 vs 27.6 us at 8192, M = 32; 31 vs 27 at M = 8): with no shared-memory ring its loads and MMAs
+    // do not overlap, and its reads of X compete with W for the SM's outstanding requests.
+    const bool skinny_ok = M <= kSkinnyMaxM && K >= 8 && (K % 8) == 0 && (N % 8) == 0;
+    const bool skinny_auto = skinny_ok && N * K <= (1ll << 24);
+    if (path == KX_PATH_AUTO)
+        path = gemv_ok ? KX_PATH_GEMV : skinny_auto ? KX_PATH_SKINNY : (M <= 64) ? KX_PATH_SWAP : KX_PATH_TILE;
+    if (path == KX_PATH_SKINNY) {
+        if (!skinny_ok) return KX_ERR_PLAN;
+        if (ov && (ov->cta_pair > 1 || ov->stream_k > 1 || ov->narrow_tail > 1 || ov->cluster_reduce > 1 ||
+                   ov->k_cluster > 1 || ov->max_ctas > 0 || ov->stages > 0 || ov->raster_group > 0 || ov->split_k > 1))
+            return KX_ERR_PLAN;
+        // rows of W per CTA (block_n): 32 (two 16-row fragments share every X load) when that still gives
+        // every SM a CTA, else 16
+        const int rw = (ov && ov->block_n) ? ov->block_n : (N / 32 >= (sms * 4) / 5 ? 32 : 16);
+        if (!skinny_variant_exists(rw)) return KX_ERR_PLAN;
+        pl->path = path;
+        pl->bn = rw;
+        pl->ctas = 1;
+        pl->splits = 1;
+        pl->stages = 0;
+        pl->smem = 16 * 8 * ceil_div(M, 8) * rw * 4;
+        pl->tiles_n = ceil_div(N, rw);
+        pl->tiles_m = 1;
+        pl->units = pl->tiles_n;
+        pl->grid = pl->tiles_n;
+        pl->ws_bytes = 0;
+        pl->sk_tile0 = pl->narrow_tile0 = pl->units;
+        return KX_OK;
+    }
     if (path == KX_PATH_GEMV) {
         if (!gemv_ok) return KX_ERR_PLAN;
         if (ov && (ov->cta_pair > 1 || ov->stream_k > 1 || ov->narrow_tail > 1 || ov->cluster_reduce > 1 ||
@@ -525,14 +584,35 @@ int make_plan_from(long long M, long long N, long long K, const kx_plan_override
         // L2 -> SM operand traffic per flop; used whenever there are enough 256-row
         // tiles to fill at least four fifths of the pair slots.
         int ctas = (ov && ov->cta_pair) ? ov->cta_pair : 0;
+        int bn = ov ? ov->block_n : 0;
+        int auto_kc = 0;
+        const bool free_plan = !(ov && (ov->k_cluster || ov->stream_k || ov->narrow_tail || ov->max_ctas || ov->stages));
+        if (ctas == 0 && bn == 0 && free_plan && nkb >= 16 && max_ctas >= 4) {
+            // A few 256-row tiles (M around 512): 256 x 256 pair tiles keep the MMAs wide enough to be bound by
+            // the tensor pipe rather than by the issuing lane, and splitting the K range of every tile over two
+            // pairs (a cluster of four CTAs; the two CTAs that hold the same rows swap half of their partial
+            // tile through distributed shared memory) puts the SMs that single pairs would leave idle to
+            // work.  Taken when the pairs then fill at least four fifths of the pair slots in one wave and
+            // every cluster is resident at once (measured: 24.4 us against 25.3 for single-CTA 128 x 256 tiles
+            // with the same K split at 512 x 4096 x 4096; 128-column pair tiles lose to single-CTA ones).
+            const int pair_slots = max_ctas / 2;
+            for (int cand : {256}) {
+                const long long t2 = 2ll * ceil_div(M, 256) * ceil_div(N, cand);
+                const TileVariant* vc = find_tile(cand, 2, 0);
+                if (t2 <= pair_slots && t2 * 5 >= pair_slots * 4ll && vc && max_active_tile_clusters(vc, 4) * 2 >= t2) {
+                    ctas = 2;
+                    bn = cand;
+                    auto_kc = 2;
+                    break;
+                }
+            }
+        }
         if (ctas == 0)
             ctas = (static_cast<long long>(ceil_div(M, 256)) * ceil_div(N, 256) * 5 >= (max_ctas / 2) * 4 &&
                     max_ctas >= 2) ? 2 : 1;
         if (ctas != 1 && ctas != 2) return KX_ERR_PLAN;
         const int slots = std::max(1, max_ctas / ctas);
-        int bn = ov ? ov->block_n : 0;
-        int auto_kc = 0;
-        if (bn == 0 && ctas == 1 && !(ov && (ov->k_cluster || ov->stream_k || ov->narrow_tail || ov->max_ctas))) {
+        if (bn == 0 && ctas == 1 && free_plan) {
             // Too few tiles to fill the GPU: prefer the widest tile for which a 2-CTA K cluster per
             // tile puts at least four fifths of the SMs to work in one wave (measured on M = 256..512:
             // 6-25 % faster than narrow tiles without a K split; 4-CTA clusters lose to 2-CTA ones).
@@ -621,11 +701,12 @@ int make_plan_from(long long M, long long N, long long K, const kx_plan_override
         // split over a cluster of 2 or 4 CTAs and reduced through distributed shared memory, so a
         // problem with few, wide tiles still puts every SM to work.  One tile per cluster.
         if (kcl > 1) {
-            if ((kcl != 2 && kcl != 4) || ctas != 1 || pl->stream_k || nt == 2 || nkb < 2 * kcl ||
+            // (a cluster of pairs: two pairs, the portable cluster size of eight would leave GPCs half used)
+            if ((kcl != 2 && kcl != 4) || (ctas == 2 && kcl != 2) || pl->stream_k || nt == 2 || nkb < 2 * kcl ||
                 (ov && ov->max_ctas > 0))
                 return KX_ERR_PLAN;
             pl->kcluster = kcl;
-            pl->grid = pl->units * kcl;
+            pl->grid = pl->units * kcl * ctas;
         }
     } else {
         int bn = ov ? ov->block_n : 0;
@@ -769,7 +850,7 @@ int run(const void* X, const void* W, const void* bias, const void* R, void* Y, 
     if ((N % 8) != 0) {
         // only reachable with pitched operands: the small-M kernel's epilogue works in 8-byte column
         // groups, so a ragged N always takes the tile kernel (TMA clips the last columns)
-        if (ov && (ov->path == KX_PATH_SWAP || ov->path == KX_PATH_GEMV)) return KX_ERR_PLAN;
+        if (ov && (ov->path == KX_PATH_SWAP || ov->path == KX_PATH_GEMV || ov->path == KX_PATH_SKINNY)) return KX_ERR_PLAN;
         std::memset(&ragged, 0, sizeof ragged);
         if (ov) ragged = *ov;
         ragged.path = KX_PATH_TILE;
@@ -785,7 +866,7 @@ int run(const void* X, const void* W, const void* bias, const void* R, void* Y, 
         std::fprintf(stderr, "[kx] M=%lld N=%lld K=%lld path=%d bn=%d ctas=%d stages=%d splits=%d streamk=%d grid=%d units=%d\n",
                      M, N, K, pl.path, pl.bn, pl.ctas, pl.stages, pl.splits, pl.stream_k, pl.grid, pl.units);
 
-    if (pl.path == KX_PATH_GEMV) {
+    if (pl.path == KX_PATH_GEMV || pl.path == KX_PATH_SKINNY) {
         GemvLaunch g;
         g.X = X; g.W = W; g.bias = bias; g.R = R; g.Y = Y;
         g.M = M; g.N = N; g.K = K;
@@ -798,10 +879,11 @@ int run(const void* X, const void* W, const void* bias, const void* R, void* Y, 
         // 134 MB matrix push the running kernel's lines out: 11.6 vs 11.0 us at 5120^2)
         const long long row_bytes = K * 2;
         const int pf = ov ? ov->l2_prefetch : 0;
-        const long long pf_default = (N * row_bytes <= (48ll << 20)) ? row_bytes : std::min<long long>(row_bytes, 2048);
+        const long long pf_default = (pl.path == KX_PATH_GEMV && N * row_bytes <= (48ll << 20))
+                                         ? row_bytes : std::min<long long>(row_bytes, 2048);
         g.pf_bytes = pf < 0 ? 0 : static_cast<int>(pf == 0 ? pf_default : std::min<long long>(row_bytes, 128ll * pf));
         g.pdl = !(ov && ov->no_pdl);
-        return launch_gemv(g, stream);
+        return pl.path == KX_PATH_GEMV ? launch_gemv(g, stream) : launch_skinny(g, stream);
     }
 
     cudaLaunchConfig_t cfg;
@@ -821,7 +903,7 @@ int run(const void* X, const void* W, const void* bias, const void* R, void* Y, 
     }
     if (pl.ctas == 2 || pl.cluster_reduce || pl.kcluster > 1) {
         attr[nattr].id = cudaLaunchAttributeClusterDimension;
-        attr[nattr].val.clusterDim.x = pl.cluster_reduce ? pl.splits : (pl.kcluster > 1 ? pl.kcluster : 2);
+        attr[nattr].val.clusterDim.x = pl.cluster_reduce ? pl.splits : (pl.kcluster > 1 ? pl.kcluster * pl.ctas : 2);
         attr[nattr].val.clusterDim.y = 1;
         attr[nattr].val.clusterDim.z = 1;
         ++nattr;

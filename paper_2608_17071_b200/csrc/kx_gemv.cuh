@@ -134,4 +134,131 @@ kx_gemv_kernel(const GemvParams p) {
 }
 
 
+// kx_skinny_kernel: the same job for up to 32 rows of X, where 2 M flops per weight element are too many for
+// the CUDA cores but the problem is still bound by reading W once (Table 1, memory strategy; the per-M
+// specialisation of Algorithm 3).  Warp-level tensor-core instructions (mma.sync m16n8k16, BF16 x BF16 ->
+// FP32) are fed straight from registers, so there is no shared-memory pipeline, no tensor-memory accumulator
+// to hand over and no split-K across CTAs: the whole chain behind the last load is one reduction over the
+// warps of the CTA in shared memory.
+//
+// One CTA owns 16 FR consecutive rows of W over the whole K range; its 16 warps take the 32-element steps
+// of K in turn (warp w takes steps w, w + 16, ...).  In a step, lane (g, t) (g = lane / 4, t = lane % 4)
+// loads 16 bytes = 8 consecutive K elements, starting at element 8 t of the step, of W rows g and g + 8 of
+// every 16-row fragment (non-coherent path, no L1 allocation) and of X rows g, g + 8, ... (read-only path
+// through L1 / L2).  The tensor-core instruction sums over 16 K slots; which element of K sits in which
+// slot does not matter as long as both operands agree, so the 8 elements a lane holds serve two
+// instructions (elements 0..3 and 4..7 of every lane) and no data is exchanged between lanes.  The warps'
+// partial tiles are added in warp order (fixed summation order), bias and residual are added once, in
+// FP32, before the single rounding to BF16; the thread that writes an output element is the one that read
+// its residual value, so R may alias Y.
+constexpr int kSkinnyWarps = 16;
+
+__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                               uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+        "{%0, %1, %2, %3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// MB = groups of 8 rows of X (M <= 8 MB), FR = 16-row fragments of W per CTA.
+template <int MB, int FR>
+__global__ void __launch_bounds__(kSkinnyWarps * 32)
+kx_skinny_kernel(const GemvParams p) {
+    constexpr int ROWS = 16 * FR, MR = 8 * MB, UNR = 2;
+    extern __shared__ float s_part[];                       // [warp][m][n]
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int g = lane >> 2, t = lane & 3;
+    const long long n0 = static_cast<long long>(blockIdx.x) * ROWS;
+    const int nch = p.K >> 3;                               // 16-byte chunks per row
+    const int nit = (p.K + 31) >> 5;                        // steps of 32 K elements
+
+    if (p.pf_bytes > 0 && tid < ROWS && n0 + tid < p.N)
+        prefetch_l2_bulk(p.W + (n0 + tid) * p.ldw, static_cast<uint32_t>(p.pf_bytes));
+    pdl_wait_prior();
+    pdl_launch_dependents();
+
+    const uint4* wp[2 * FR];
+#pragma unroll
+    for (int i = 0; i < 2 * FR; ++i) {
+        long long r = n0 + 8 * i + g;                       // fragment i / 2, rows g and g + 8
+        if (r >= p.N) r = p.N - 1;                          // rows past the end: loaded again, never stored
+        wp[i] = reinterpret_cast<const uint4*>(p.W + r * p.ldw);
+    }
+    const uint4* xp[MB];
+#pragma unroll
+    for (int j = 0; j < MB; ++j) {
+        const int m = 8 * j + g;
+        xp[j] = reinterpret_cast<const uint4*>(p.X + static_cast<long long>(m < p.M ? m : p.M - 1) * p.ldx);
+    }
+    float acc[FR][MB][4];
+#pragma unroll
+    for (int f = 0; f < FR; ++f)
+#pragma unroll
+        for (int j = 0; j < MB; ++j)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[f][j][e] = 0.f;
+
+#pragma unroll 1
+    for (int it0 = warp; it0 < nit; it0 += kSkinnyWarps * UNR) {
+        uint4 w[UNR][2 * FR], x[UNR][MB];
+#pragma unroll
+        for (int u = 0; u < UNR; ++u) {
+            const int c = (it0 + u * kSkinnyWarps) * 4 + t;
+            const bool ok = c < nch;                        // also false for steps past the end
+#pragma unroll
+            for (int i = 0; i < 2 * FR; ++i) w[u][i] = ok ? ld_stream_u4(wp[i] + c) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+            for (int j = 0; j < MB; ++j) x[u][j] = ok ? __ldg(xp[j] + c) : make_uint4(0u, 0u, 0u, 0u);
+        }
+#pragma unroll
+        for (int u = 0; u < UNR; ++u)
+#pragma unroll
+            for (int f = 0; f < FR; ++f)
+#pragma unroll
+                for (int j = 0; j < MB; ++j) {
+                    mma_bf16_16816(acc[f][j], w[u][2 * f].x, w[u][2 * f + 1].x, w[u][2 * f].y, w[u][2 * f + 1].y,
+                                   x[u][j].x, x[u][j].y);
+                    mma_bf16_16816(acc[f][j], w[u][2 * f].z, w[u][2 * f + 1].z, w[u][2 * f].w, w[u][2 * f + 1].w,
+                                   x[u][j].z, x[u][j].w);
+                }
+    }
+
+    // accumulator element e of fragment (f, j): W row 16 f + g + 8 (e / 2), X row 8 j + 2 t + (e % 2)
+    float* mine = s_part + warp * (MR * ROWS);
+#pragma unroll
+    for (int f = 0; f < FR; ++f)
+#pragma unroll
+        for (int j = 0; j < MB; ++j)
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                mine[(8 * j + 2 * t + (e & 1)) * ROWS + 16 * f + g + 8 * (e >> 1)] = acc[f][j][e];
+    __syncthreads();
+    for (int o = tid; o < MR * ROWS / 2; o += kSkinnyWarps * 32) {
+        const int m = o / (ROWS / 2), nn = (o - m * (ROWS / 2)) * 2;
+        const long long n = n0 + nn;
+        if (m < p.M && n < p.N) {                           // N is even: n + 1 < N as well
+            float v0 = 0.f, v1 = 0.f;
+#pragma unroll
+            for (int wv = 0; wv < kSkinnyWarps; ++wv) {
+                const float2 q = *reinterpret_cast<const float2*>(s_part + wv * (MR * ROWS) + m * ROWS + nn);
+                v0 += q.x;
+                v1 += q.y;
+            }
+            if (p.bias) {
+                const uint32_t bb = __ldg(reinterpret_cast<const uint32_t*>(p.bias + n));
+                v0 += bf16_lo(bb);
+                v1 += bf16_hi(bb);
+            }
+            if (p.R) {
+                const uint32_t rr = *reinterpret_cast<const uint32_t*>(p.R + m * p.ldr + n);
+                v0 += bf16_lo(rr);
+                v1 += bf16_hi(rr);
+            }
+            *reinterpret_cast<uint32_t*>(p.Y + m * p.ldy + n) = pack_bf16x2(v0, v1);
+        }
+    }
+}
+
 }  // namespace kx

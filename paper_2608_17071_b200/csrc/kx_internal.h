@@ -20,9 +20,15 @@ struct GemvLaunch {
     bool pdl;              // programmatic stream serialization
 };
 constexpr int kGemvMaxM = 4;
+constexpr int kSkinnyMaxM = 32;
 // true if a kernel instantiation exists for this combination
 bool gemv_variant_exists(int rows_per_cta, int warps);
 // Enqueues the kernel; returns a kx_status value.
 int launch_gemv(const GemvLaunch& a, cudaStream_t stream);
+// The warp-level tensor-core kernel for 5..32 rows (kx_skinny_kernel): same arguments; rows_per_cta is 16 or
+// 32 and `warps` is ignored.  skinny_setup raises the kernels' shared-memory limit once per device.
+int skinny_setup();
+bool skinny_variant_exists(int rows_per_cta);
+int launch_skinny(const GemvLaunch& a, cudaStream_t stream);
 
 }  // namespace kx

@@ -151,10 +151,11 @@ struct TileParams {
     int swiglu;                   // 1: gate/up mode.  W rows of a tile = BN/2 rows of Wg (tmB) followed by the same
                                   // BN/2 rows of Wu (tmB2); the epilogue writes silu(gate) * up, BN/2 columns per
                                   // tile, N = number of output columns; no bias, no residual
-    int kcluster;                 // > 1 (single-CTA tiles only): the K range of every tile is split over a
-                                  // thread-block cluster of this many CTAs (grid = tiles x kcluster, one tile per
-                                  // cluster); partials are parked in shared memory and each CTA finishes the
-                                  // 64-column chunks c with c % kcluster == rank by reading all partials
+    int kcluster;                 // > 1: the K range of every tile is split over this many CTAs (CTA pairs when a
+                                  // pair works on a tile), which form one thread-block cluster (grid = tiles x
+                                  // kcluster x CTAs per tile, one tile per cluster); partials are parked in
+                                  // shared memory and the CTA of K rank r finishes the 64-column chunks c with
+                                  // c % kcluster == r of its 128 rows by reading all partials of those rows
                                   // through distributed shared memory in rank order
     int sk_tile0;                 // tiles [0, sk_tile0) are taken whole, round-robin over the slots;
                                   // tiles [sk_tile0, num_tiles) are stream-K'd (== num_tiles: none)
@@ -181,7 +182,7 @@ struct TileCfg {
     static_assert(KBS == 1 || KBS == 2, "KBS");
     static constexpr int SLAB_BYTES = 32 * 128;             // 32 rows x 64 BF16 per warp per chunk
     static constexpr int EPI_BYTES = 4 * NB * SLAB_BYTES;
-    static constexpr int NUM_BARS = 2 * STAGES + 4 + 4 * NB + 1;
+    static constexpr int NUM_BARS = 2 * STAGES + 4 + 4 * NB + 1 + 5;   // + K-cluster exchange: 4 incoming, 1 "peer idle"
     static constexpr int SFB_CHUNKS = (BN > 128) ? 2 : 1;
     // scale bytes per k-block: MX 1 = one chunk per operand row block, MX 2 (16-element blocks) = four
     static constexpr int SF_KB_BYTES = MX == 1 ? 512 * (1 + SFB_CHUNKS) : MX == 2 ? 2048 * (1 + SFB_CHUNKS) : 0;
@@ -288,20 +289,25 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     auto acc_empty = [&](int b) { return s_bar + 8u * (2 * STAGES + 2 + b); };
     auto r_full = [&](int w, int j) { return s_bar + 8u * (2 * STAGES + 4 + w * NB + j); };
     const uint32_t drain_bar = s_bar + 8u * (2 * STAGES + 4 + 4 * NB);
+    auto xin_bar = [&](int w) { return s_bar + 8u * (2 * STAGES + 4 + 4 * NB + 1 + w); };   // K-cluster exchange
+    const uint32_t peer_idle_bar = s_bar + 8u * (2 * STAGES + 4 + 4 * NB + 5);
     volatile uint32_t* const s_tmem =
         reinterpret_cast<volatile uint32_t*>(gbase + (s_bar - base) + 8 * C::NUM_BARS);
     volatile uint32_t* const s_abort = s_tmem + 1;
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const uint32_t cta_rank = (CTAS == 2) ? cluster_ctarank() : 0u;
+    // A CTA pair is two CTAs of the cluster whose ranks differ in the last bit; with a K cluster of pairs
+    // the cluster holds kc pairs (ranks 2j, 2j + 1 = pair j)
+    const uint32_t cta_rank = (CTAS == 2) ? (cluster_ctarank() & 1u) : 0u;
+    const uint32_t pair0 = (CTAS == 2) ? (cluster_ctarank() & ~1u) : 0u;   // cluster rank of this pair's leader
     const bool leader = (cta_rank == 0);
     // k-block = 128 bytes of a row: 64 BF16 or 128 8-bit elements; for the 4-bit kind p.K counts bytes
     // (two elements each), so a k-block is 128 of those as well
     constexpr int KBLK = (KIND != 0) ? 2 * kBlockK : kBlockK;
     const int nkb = (p.K + KBLK - 1) / KBLK;
-    const int kc = (CTAS == 1 && p.kcluster > 1) ? p.kcluster : 1;   // K-cluster size
-    const int krank = (kc > 1) ? static_cast<int>(cluster_ctarank()) : 0;
+    const int kc = (p.kcluster > 1) ? p.kcluster : 1;                // K-cluster size (in tiles' worth of CTAs)
+    const int krank = (kc > 1) ? static_cast<int>(cluster_ctarank() / CTAS) : 0;
     const int slot = blockIdx.x / (CTAS * kc);
     const int slots = gridDim.x / (CTAS * kc);
 
@@ -320,6 +326,7 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     };
 
     if (threadIdx.x == 0) *s_abort = 0;
+    if (p.kcluster > 1 && threadIdx.x == 0) KX_TRACE_POINT(p, blockIdx.x, 8);
     if (warp == 4 && lane == 0) {
         prefetch_tmap(&tmA);
         prefetch_tmap(&tmB);
@@ -365,6 +372,8 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             for (int w = 0; w < 4; ++w)
                 for (int j = 0; j < NB; ++j) mbar_init(r_full(w, j), 1);
             mbar_init(drain_bar, 1);
+            for (int w = 0; w < 4; ++w) mbar_init(xin_bar(w), 1);
+            mbar_init(peer_idle_bar, 1);
             fence_mbar_init();
         }
         __syncwarp();
@@ -373,7 +382,9 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
     tc_fence_before();
     __syncthreads();
-    if constexpr (CTAS == 2) {
+    // clustered launches (a CTA pair, a K cluster, or both): every CTA of the cluster has started and
+    // initialised its barriers before any of them touches a peer
+    if (CTAS == 2 || p.kcluster > 1) {
         cluster_arrive();
         cluster_wait();
     }
@@ -384,10 +395,11 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // kernel may start its own prologue as soon as it finds a free SM.
     pdl_wait_prior();
     pdl_launch_dependents();
+    if (p.kcluster > 1 && threadIdx.x == 0) KX_TRACE_POINT(p, blockIdx.x, 9);
 
     Waiter wt;
     wt.abort_flag = s_abort;
-    wt.peer_abort = (CTAS == 2) ? map_to_cta(smem_u32(const_cast<uint32_t*>(s_abort)), cta_rank ^ 1u) : 0u;
+    wt.peer_abort = (CTAS == 2) ? map_to_cta(smem_u32(const_cast<uint32_t*>(s_abort)), cluster_ctarank() ^ 1u) : 0u;
     wt.limit_ns = p.spin_limit_ns;
 
     SegIter it;
@@ -430,7 +442,7 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         // otherwise: no residual in this mode) because tmB2 carries the up weights.
                         const int c0 = sg ? (col >> 8) : (col >> 7);
                         const CUtensorMap* const mapSA = sg ? &tmR : &tmB2;
-                        const uint32_t fb = (CTAS == 1) ? full(s) : map_to_cta(full(s), 0);
+                        const uint32_t fb = (CTAS == 1) ? full(s) : map_to_cta(full(s), pair0);
                         for (int j = 0; j < nsub; ++j) {
                             const uint32_t dst = s_sf + s * C::SF_STAGE + j * C::SF_KB_BYTES;
                             const int ya = (tm * CTAS + static_cast<int>(cta_rank)) * nkb + kb + j;
@@ -467,7 +479,7 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     } else {
                         // both CTAs' copies complete on the leader's barrier
                         if (leader) mbar_arrive_expect_tx(full(s), 2 * nsub * (stage_tx + C::SF_KB_BYTES));
-                        const uint32_t fb = map_to_cta(full(s), 0);
+                        const uint32_t fb = map_to_cta(full(s), pair0);
                         for (int j = 0; j < nsub; ++j) {
                             tma_load_2d_pair(sa + j * kABytes, &tmA, (kb + j) * KBLK, a_row, fb);
                             tma_load_2d_pair(sb + j * C::B_BYTES, mapB, (kb + j) * KBLK, b_row, fb);
@@ -477,7 +489,7 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 }
             }
         }
-        if (kc > 1) {            // K-cluster mode: every thread of the cluster passes both barriers
+        if (kc > 2) {            // K cluster, pull form: every thread of the cluster passes both barriers
             __syncwarp();
             cluster_arrive(); cluster_wait();
             cluster_arrive(); cluster_wait();
@@ -498,8 +510,8 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             // running addresses of the current stage: its `full` barrier, its `empty` barrier as seen from
             // each CTA of the pair, and the low word of its A-tile descriptor
             const uint32_t a_lo0 = smem_desc_lo(s_stage);
-            const uint32_t empty_base0 = (CTAS == 1) ? empty(0) : map_to_cta(empty(0), 0);
-            const uint32_t empty_base1 = (CTAS == 1) ? 0u : map_to_cta(empty(0), 1);
+            const uint32_t empty_base0 = (CTAS == 1) ? empty(0) : map_to_cta(empty(0), pair0);
+            const uint32_t empty_base1 = (CTAS == 1) ? 0u : map_to_cta(empty(0), pair0 + 1u);
             uint32_t full_bar = full(0), empty_bar0 = empty_base0, empty_bar1 = empty_base1, a_lo = a_lo0;
             bool ok = true;
             bool have = false;   // the current stage was already seen full by the previous k-block's early test
@@ -570,6 +582,8 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 for (int kb = kb0; kb < kb1; kb += KBS) {
                     if (!have && !wt.wait(full_bar, ph, kWhereFull)) { ok = false; break; }
                     tc_fence_after();
+                    if (kc > 1 && kb == kb0) KX_TRACE_POINT(p, blockIdx.x, 10);
+                    if (kc > 1 && kb + KBS >= kb1) KX_TRACE_POINT(p, blockIdx.x, 11);
                     // the next stage in ring order (also the first stage of the next tile)
                     const bool wrap = (s + 1 == STAGES);
                     const uint32_t next_full = wrap ? full(0) : full_bar + 8u;
@@ -595,17 +609,17 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 if constexpr (CTAS == 1) {
                     mma_commit<1>(acc_full(b));
                 } else {
-                    mma_commit<2>(map_to_cta(acc_full(b), 0));
-                    mma_commit<2>(map_to_cta(acc_full(b), 1));
+                    mma_commit<2>(map_to_cta(acc_full(b), pair0));
+                    mma_commit<2>(map_to_cta(acc_full(b), pair0 + 1u));
                 }
             }
             if (!ok) {  // let every MMA issued so far retire before TMEM is freed
-                mma_commit<CTAS>(CTAS == 1 ? drain_bar : map_to_cta(drain_bar, 0));
+                mma_commit<CTAS>(CTAS == 1 ? drain_bar : map_to_cta(drain_bar, pair0));
                 uint32_t spins = 0;
                 while (!mbar_try_wait(drain_bar, 0) && ++spins < (1u << 20)) {}
             }
         }
-        if (kc > 1) {
+        if (kc > 2) {
             __syncwarp();
             cluster_arrive(); cluster_wait();
             cluster_arrive(); cluster_wait();
@@ -623,7 +637,7 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         auto slab4 = [&](float* part, int c) {
             return reinterpret_cast<float4*>(part) + (static_cast<size_t>(c) * 4 + q) * 16 * 32 + lane;
         };
-        enum { kWhole = 0, kFast = 1, kWriter = 2, kSlow = 3, kNone = 4, kCluster = 5 };
+        enum { kWhole = 0, kFast = 1, kWriter = 2, kSlow = 3, kNone = 4, kCluster = 5, kExchange = 6 };
         uint32_t scount = 0, rphase = 0;
         bool ok = true;
         int cluster_bars = 0;                              // K-cluster mode: cluster barriers passed so far
@@ -674,27 +688,39 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             auto chunk_inb = [&](int c) { return (row0 < p.M) && (colbase + c * 64 < p.N); };
             // chunks this warp writes to Y: all of them, or in K-cluster mode those dealt to this CTA
             auto chunk_valid = [&](int c) { return chunk_inb(c) && (kc == 1 || (c % kc) == krank); };
-            auto issue_r = [&](int c) {                    // lane 0 only
-                if (chunk_valid(c)) {
-                    const int j = c % NB;
+            // This warp writes `nmine` chunks to Y, numbered i = 0, 1, ...: chunk i of the tile, or in K-cluster
+            // mode chunk krank + kc i.  Staging buffers and R requests go by i, so that a CTA's chunks use
+            // the buffers in turn whatever their position in the tile.
+            const int nmine = (kc == 1) ? nchunks : (nchunks > krank ? (nchunks - krank + kc - 1) / kc : 0);
+            auto chunk_of = [&](int i) { return (kc == 1) ? i : krank + kc * i; };
+            auto issue_r = [&](int i) {                    // lane 0 only
+                const int c = chunk_of(i);
+                if (chunk_inb(c)) {
+                    const int j = i % NB;
                     mbar_arrive_expect_tx(r_full(q, j), C::SLAB_BYTES);
                     tma_load_2d(my_epi + j * C::SLAB_BYTES, &tmR, colbase + c * 64, row0, r_full(q, j));
                 }
             };
-            // R slabs are requested in chunk order, up to NB-1 chunks ahead.  They are requested
-            // before the accumulator is ready whenever this warp will (whole tile) or is expected
-            // to (the slot's last segment: its partners ran at the start of their ranges) produce
-            // the output.
+            // R slabs are requested in chunk order, up to NB-1 chunks ahead (all of them when the warp has
+            // no more chunks than buffers).  They are requested before the accumulator is ready whenever
+            // this warp will (whole tile) or is expected to (the slot's last segment: its partners ran
+            // at the start of their ranges) produce the output.
             const bool last_seg = (it.t >= it.sk_tile0) && (it.u >= it.u1);
             const bool spec_r = has_r && (whole || last_seg || kc > 1);
             int n_iss = 0;                                 // R chunks requested so far (warp-uniform)
             if (lane == 0) tma_store_wait_read<0>();       // staging buffers of the previous tile are free
             if (spec_r) {
                 // (a single buffer is free at this point too: the previous tile's stores were waited for above)
-                const int pre0 = (NB > 1) ? NB - 1 : 1;
-                const int pre = (pre0 < nchunks) ? pre0 : nchunks;
+                const int pre0 = (nmine <= NB) ? nmine : ((NB > 1) ? NB - 1 : 1);
+                const int pre = (pre0 < nmine) ? pre0 : nmine;
                 for (; n_iss < pre; ++n_iss)
                     if (lane == 0) issue_r(n_iss);
+            }
+            // the tile's bias values (one or a few 128-byte lines) are asked for now, so that the first use in
+            // a CTA does not wait for a cold line after the accumulator is ready
+            if (has_bias && lane < (BN * 2 + 127) / 128) {
+                const int n = colbase + lane * 64;
+                if (n < p.N) asm volatile("prefetch.global.L1 [%0];" ::"l"(bias + n));
             }
             __syncwarp();
 
@@ -744,16 +770,66 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             if (!__all_sync(0xffffffffu, wt.wait(acc_full(b), aph, kWhereAccFull))) { ok = false; break; }
             tc_fence_after();
             if (q == 0 && lane == 0 && leader) KX_TRACE_POINT(p, slot, (scount - 1) * 4 + 2);
+            if (kc > 1 && q == 0 && lane == 0) KX_TRACE_POINT(p, blockIdx.x, 6);
 
             auto release_acc = [&]() {                     // accumulator buffer b is drained
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) {
                     if constexpr (CTAS == 1) mbar_arrive(acc_empty(b));
-                    else mbar_arrive_cluster(map_to_cta(acc_empty(b), 0));
+                    else mbar_arrive_cluster(map_to_cta(acc_empty(b), pair0));
                 }
             };
-            if (kc > 1) {
+            if (kc == 2) {
+                // K cluster of two: the two CTAs that hold the same 128 rows of the tile swap halves.  This
+                // warp parks the 64-column chunks its peer finishes (c % 2 != krank) in the first half of
+                // its idle operand ring and sends them with one bulk copy per chunk (shared memory to the
+                // peer's shared memory, bytes counted on the peer's barrier for this warp) into the second
+                // half of the peer's ring; the chunks it finishes itself stay in tensor memory and get the
+                // peer's share added below.  The peer says when its ring is idle (its own MMAs are done).
+                role = kExchange;
+                const uint32_t peer = static_cast<uint32_t>((krank ^ 1) * CTAS) + cta_rank;
+                constexpr uint32_t kHalfBytes = static_cast<uint32_t>((C::CHUNKS + 1) / 2) * 4u * 8192u;
+                static_assert(2 * ((C::CHUNKS + 1) / 2) * 4 * 8192 <= STAGES * C::STAGE_BYTES, "exchange areas must fit in the ring");
+                int n_in = 0;
+                for (int c = 0; c < nchunks; ++c)
+                    if (chunk_valid(c)) ++n_in;            // chunks whose second half arrives from the peer
+                if (lane == 0) {
+                    if (n_in > 0) mbar_arrive_expect_tx(xin_bar(q), static_cast<uint32_t>(n_in) * 8192u);
+                    if (q == 0) mbar_arrive_cluster(map_to_cta(peer_idle_bar, peer));   // this CTA's ring is idle
+                }
+                bool go = true, asked = false;
+#pragma unroll 1
+                for (int c = 0; c < nchunks && go; ++c) {
+                    if (!chunk_inb(c) || (c & 1) == krank) continue;
+                    uint32_t a[2][32];
+                    tmem_ld_32x32(tbase + c * 64, a[0]);
+                    tmem_ld_32x32(tbase + c * 64 + 32, a[1]);
+                    tmem_ld_wait();
+                    const uint32_t off = static_cast<uint32_t>(((c >> 1) * 4 + q) * 8192);
+                    const uint32_t dst = ring + off + lane * 16;
+#pragma unroll
+                    for (int i = 0; i < 16; ++i)
+                        asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + i * 512),
+                                     "r"(a[i >> 3][(i & 7) * 4 + 0]), "r"(a[i >> 3][(i & 7) * 4 + 1]),
+                                     "r"(a[i >> 3][(i & 7) * 4 + 2]), "r"(a[i >> 3][(i & 7) * 4 + 3])
+                                     : "memory");
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (!asked) {                          // once: the peer's ring must be idle before the first copy
+                        if (lane == 0) go = wt.wait_cluster(peer_idle_bar, 0u, kWherePartials);
+                        go = __shfl_sync(0xffffffffu, go ? 1 : 0, 0) != 0;
+                        asked = true;
+                    }
+                    if (go && lane == 0)
+                        bulk_copy_to_cta(map_to_cta(ring + kHalfBytes + off, peer), ring + off, 8192u,
+                                         map_to_cta(xin_bar(q), peer));
+                }
+                if (!go) { ok = false; break; }
+                if (q == 0 && lane == 0) KX_TRACE_POINT(p, blockIdx.x, 4);
+                if (n_in > 0 && !__all_sync(0xffffffffu, wt.wait_cluster(xin_bar(q), 0u, kWherePartials))) { ok = false; break; }
+                if (q == 0 && lane == 0) KX_TRACE_POINT(p, blockIdx.x, 5);
+            } else if (kc > 1) {
                 // K-cluster: park this CTA's partial (every in-bounds chunk) in its own shared memory,
                 // meet the cluster, then finish the chunks dealt to this CTA from all partials
                 role = kCluster;
@@ -773,8 +849,10 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                                      : "memory");
                 }
                 release_acc();
+                if (q == 0 && lane == 0) KX_TRACE_POINT(p, blockIdx.x, 4);
                 cluster_arrive();
                 cluster_wait();
+                if (q == 0 && lane == 0) KX_TRACE_POINT(p, blockIdx.x, 5);
                 ++cluster_bars;
             } else if (!whole) {
                 if (staged) {
@@ -830,13 +908,24 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
             // kWhole / kFast / kSlow: this warp writes the tile's output rows
 #pragma unroll 1
-            for (int c = 0; c < nchunks; ++c) {
-                const int j = c % NB;
+            for (int ci = 0; ci < nmine; ++ci) {
+                const int c = chunk_of(ci);
+                const int j = ci % NB;
                 const int col0 = colbase + c * 64;
-                const bool valid = chunk_valid(c);
+                const bool valid = chunk_inb(c);
                 const uint32_t buf = my_epi + j * C::SLAB_BYTES;
+                // the chunk's 64 bias values, all eight loads in flight at once and long before their use (one
+                // after the other, behind the stores below, every load of a cold line cost a trip to L2)
+                uint4 bb8[8];
+                if (has_bias && valid) {
+#pragma unroll
+                    for (int g8 = 0; g8 < 8; ++g8) {
+                        const int n = col0 + g8 * 8;
+                        bb8[g8] = (n + 8 <= p.N) ? __ldg(reinterpret_cast<const uint4*>(bias + n)) : make_uint4(0u, 0u, 0u, 0u);
+                    }
+                }
                 if (has_r)
-                    for (; n_iss <= c; ++n_iss)
+                    for (; n_iss <= ci; ++n_iss)
                         if (lane == 0) issue_r(n_iss);
                 uint32_t acc[2][32];
                 if (valid && role == kWhole) {
@@ -872,6 +961,26 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         }
                     }
                 }
+                if (valid && role == kExchange) {
+                    // this CTA's accumulators plus the peer's share that landed in the second half of the ring
+                    tmem_ld_32x32(tbase + c * 64, acc[0]);
+                    tmem_ld_32x32(tbase + c * 64 + 32, acc[1]);
+                    tmem_ld_wait();
+                    constexpr uint32_t kHalfBytes = static_cast<uint32_t>((C::CHUNKS + 1) / 2) * 4u * 8192u;
+                    const uint32_t src = ring + kHalfBytes + ((((c >> 1) * 4 + q) * 16) * 32 + lane) * 16;
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        float4 t;
+                        asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                                     : "=f"(t.x), "=f"(t.y), "=f"(t.z), "=f"(t.w)
+                                     : "r"(src + i * 512));
+                        uint32_t* a4 = &acc[i >> 3][(i & 7) * 4];
+                        a4[0] = __float_as_uint(__uint_as_float(a4[0]) + t.x);
+                        a4[1] = __float_as_uint(__uint_as_float(a4[1]) + t.y);
+                        a4[2] = __float_as_uint(__uint_as_float(a4[2]) + t.z);
+                        a4[3] = __float_as_uint(__uint_as_float(a4[3]) + t.w);
+                    }
+                }
                 if (valid && role == kCluster) {
                     // sum the cluster's partials of this chunk in rank order (16 remote 16-byte loads in
                     // flight per rank)
@@ -881,7 +990,8 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     const uint32_t off = ring + (((c * 4 + q) * 16) * 32 + lane) * 16;
 #pragma unroll 1
                     for (int r = 0; r < kc; ++r) {
-                        const uint32_t src = map_to_cta(off, r);
+                        // the CTA of K rank r that holds the same 128 rows of the tile as this one
+                        const uint32_t src = map_to_cta(off, static_cast<uint32_t>(r * CTAS) + cta_rank);
                         float4 t[16];
 #pragma unroll
                         for (int i = 0; i < 16; ++i) t[i] = ld_cluster_f32x4(src + i * 512);
@@ -929,7 +1039,8 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
                     for (int i = 0; i < 64; ++i) acc[i >> 5][i & 31] = __float_as_uint(sum[i]);
                 }
-                if (c == nchunks - 1 && (role == kWhole || role == kFast)) release_acc();
+                if (ci == nmine - 1 && (role == kWhole || role == kFast || role == kExchange)) release_acc();
+                if (kc > 1 && q == 0 && lane == 0) KX_TRACE_POINT(p, blockIdx.x, 16 + ci * 4 + 0);
                 if (valid) {
                     if (has_r) {
                         if (!__all_sync(0xffffffffu, wt.wait(r_full(q, j), (rphase >> j) & 1u, kWhereRFull))) {
@@ -938,6 +1049,7 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         }
                         rphase ^= (1u << j);
                     }
+                    if (kc > 1 && q == 0 && lane == 0) KX_TRACE_POINT(p, blockIdx.x, 16 + ci * 4 + 1);
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
 #pragma unroll
@@ -950,7 +1062,7 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                             if (has_bias) {
                                 const int n = col0 + c16 * 8;
                                 if (n + 8 <= p.N) {
-                                    const uint4 bb = __ldg(reinterpret_cast<const uint4*>(bias + n));
+                                    const uint4 bb = bb8[c16];
                                     v[0] += bf16_lo(bb.x); v[1] += bf16_hi(bb.x);
                                     v[2] += bf16_lo(bb.y); v[3] += bf16_hi(bb.y);
                                     v[4] += bf16_lo(bb.z); v[5] += bf16_hi(bb.z);
@@ -981,6 +1093,7 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     }
                     fence_proxy_async_smem();
                     __syncwarp();
+                    if (kc > 1 && q == 0 && lane == 0) KX_TRACE_POINT(p, blockIdx.x, 16 + ci * 4 + 2);
                     if (lane == 0) {
                         tma_store_2d(&tmY, col0, row0, buf);
                         tma_store_commit();
@@ -988,12 +1101,13 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         // because the next R slab is requested into the buffer it reads)
                         tma_store_wait_read<(NB > 1) ? 1 : 0>();
                     }
+                    if (kc > 1 && q == 0 && lane == 0) KX_TRACE_POINT(p, blockIdx.x, 16 + ci * 4 + 3);
                 } else if (lane == 0) {
                     tma_store_wait_read<0>();              // nothing stored for this chunk: drain the last store
                 }
                 // request the R slabs up to NB-1 chunks ahead; their buffers were just released
                 if (has_r) {
-                    const int target = (c + NB < nchunks) ? c + NB : nchunks;
+                    const int target = (ci + NB < nmine) ? ci + NB : nmine;
                     for (; n_iss < target; ++n_iss)
                         if (lane == 0) issue_r(n_iss);
                 }
@@ -1001,8 +1115,9 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
             if ((role == kFast || role == kSlow) && lane == 0) *ctr = 0u;   // every segment has arrived: reset
             if (q == 0 && lane == 0 && leader) KX_TRACE_POINT(p, slot, (scount - 1) * 4 + 3);
+            if (kc > 1 && q == 0 && lane == 0) KX_TRACE_POINT(p, blockIdx.x, 7);
         }
-        if (kc > 1) {
+        if (kc > 2) {
             // peers may still be reading this CTA's partial: second barrier; on a give-up path the
             // barriers skipped above are made up here so that the cluster never hangs
             __syncwarp();
@@ -1018,7 +1133,8 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     __syncwarp();
     tc_fence_before();
     __syncthreads();
-    if constexpr (CTAS == 2) {
+    // no CTA of a cluster leaves while a peer may still use its shared memory, tensor memory or barriers
+    if (CTAS == 2 || p.kcluster > 1) {
         cluster_arrive();
         cluster_wait();
     }
@@ -1072,12 +1188,13 @@ struct SwapCfg {
 //   MODE 1 (pull): each CTA parks its FP32 partial in its own shared memory (the idle operand ring), the
 //   cluster meets on the hardware cluster barrier, and the finishers read the partials through distributed
 //   shared memory.
-//   MODE 2 (push): each CTA stores the rows of its partial straight from registers into the receive area of
-//   their finishers (st.shared::cluster) and arrives on the finisher's mbarrier; a finisher waits on that one
-//   (bounded) barrier and then sums from its own shared memory.  No round trip of remote loads and no
-//   cluster-wide meeting on the critical path: the hardware cluster barrier is only used to make sure that
-//   every CTA has started before the first remote store and that none leaves while a peer might still
-//   write to it, and both of its waits are reached long after everybody arrived.
+//   MODE 2 (push): each epilogue warp parks its 32 columns of the partial in its own shared memory, grouped
+//   by finisher, and sends every finisher its block with one bulk asynchronous copy (shared memory to the
+//   shared memory of another CTA of the cluster) whose bytes are counted on the finisher's mbarrier; a
+//   finisher waits on that one (bounded) barrier and then sums from its own shared memory.  No remote
+//   loads and no cluster-wide meeting on the critical path: the hardware cluster barrier is only used to
+//   make sure that every CTA has started before the first copy and that none leaves while a copy might
+//   still read from or write to it, and both of its waits are reached long after everybody arrived.
 template <int BN, int STAGES, int MODE, int KBS = 1>
 __global__ void __launch_bounds__(kThreads, 1)
 kx_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
@@ -1085,7 +1202,7 @@ kx_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
     constexpr bool CLUSTER = (MODE == 1);
     constexpr bool PUSH = (MODE == 2);
     using C = SwapCfg<BN, STAGES, KBS, PUSH>;
-    static_assert(!CLUSTER || BN * 128 * 4 <= STAGES * C::STAGE_BYTES, "partial must fit in the idle ring");
+    static_assert(!(CLUSTER || PUSH) || (BN + 8) * 128 * 4 <= STAGES * C::STAGE_BYTES, "partial must fit in the idle ring");
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -1137,8 +1254,14 @@ kx_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
             }
             mbar_init(drain_bar, 1);
             mbar_init(epi_bar, 4);
-            mbar_init(red_bar, 4 * static_cast<uint32_t>(p.splits));
+            mbar_init(red_bar, 1);
             fence_mbar_init();
+            if constexpr (MODE == 2) {
+                // every split sends this CTA four blocks (one per epilogue warp) of rows_per x 32 FP32 values
+                if (p.splits > 1)
+                    mbar_arrive_expect_tx(red_bar, static_cast<uint32_t>(p.splits) * 4u *
+                                                       static_cast<uint32_t>((BN + p.splits - 1) / p.splits) * 128u);
+            }
         }
         __syncwarp();
         tmem_alloc<1>(smem_u32(const_cast<uint32_t*>(s_tmem)), C::TMEM_COLS);
@@ -1288,15 +1411,16 @@ kx_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
                 tmem_ld_32x16(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + b * BN + c0, a);
                 tmem_ld_wait();
                 if (PUSH && p.splits > 1) {
-                    // row i of the tile is finished by CTA i % splits; this split's partial of that row goes
-                    // into slot [sp][i / splits] of that CTA's receive area (128 columns per row: a warp
-                    // writes 128 contiguous bytes)
+                    // row i of the tile is finished by CTA i % splits: park this warp's 32 columns of it in
+                    // the (idle) operand ring, block [warp][finisher][i / splits][32 columns]
                     const int rows_per = (BN + p.splits - 1) / p.splits;
                     int d = c0 % p.splits, k = c0 / p.splits;
 #pragma unroll
                     for (int i = 0; i < 16; ++i) {
-                        if (c0 + i < m_cnt)
-                            st_cluster_u32(map_to_cta(s_recv + static_cast<uint32_t>(((sp * rows_per + k) * 128 + etid) * 4), d), a[i]);
+                        if (c0 + i < m_cnt) {
+                            const uint32_t off = static_cast<uint32_t>((((q * p.splits + d) * rows_per + k) * 32 + lane) * 4);
+                            asm volatile("st.shared.u32 [%0], %1;" ::"r"(s_stage + off), "r"(a[i]) : "memory");
+                        }
                         if (++d == p.splits) { d = 0; ++k; }
                     }
                 } else if (CLUSTER && p.splits > 1) {
@@ -1334,12 +1458,17 @@ kx_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
             __syncwarp();
             if (lane == 0) mbar_arrive(acc_empty(b));
             if (PUSH && p.splits > 1) {
-                // this warp's rows are on their way: tell every finisher (the fence of an arriving lane orders
-                // the whole warp's stores, which the warp barrier above made known to it, before its arrival)
+                // send every finisher its block: into slot [this split][warp] of its receive area, counted on
+                // its barrier (the copies read shared memory through the asynchronous proxy, hence the fence)
+                const int rows_per = (BN + p.splits - 1) / p.splits;
+                const uint32_t blk = static_cast<uint32_t>(rows_per) * 128u;
+                fence_proxy_async_smem();
+                __syncwarp();
                 if (etid == 0) KX_TRACE_POINT(p, blockIdx.x, 8);
-                if (lane < p.splits) {                    // lane d tells finisher d
-                    fence_acq_rel_cluster();
-                    mbar_arrive_cluster_relaxed(map_to_cta(red_bar, lane));
+                if (lane < p.splits) {                    // lane d sends to finisher d
+                    const uint32_t src = s_stage + static_cast<uint32_t>(q * p.splits + lane) * blk;
+                    const uint32_t dst = s_recv + static_cast<uint32_t>(sp * 4 + q) * blk;
+                    bulk_copy_to_cta(map_to_cta(dst, lane), src, blk, map_to_cta(red_bar, lane));
                 }
                 __syncwarp();
                 if (etid == 0) KX_TRACE_POINT(p, blockIdx.x, 12);
@@ -1456,27 +1585,30 @@ kx_swap_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ 
                                 : make_uint2(0u, 0u);
                 }
             }
-            // first cluster wait if the epilogue loop never reached it (a wait that gave up; warp-uniform),
-            // then the second arrival: this thread's remote stores and arrivals are all issued
+            // first cluster wait if the epilogue loop never reached it (a wait that gave up; warp-uniform)
             if (!pushed_wait) cluster_wait();
-            cluster_arrive_relaxed();
             if (threadIdx.x == 0) KX_TRACE_POINT(p, blockIdx.x, 6);
             bool have = true;
             if (reducer) have = __all_sync(0xffffffffu, wt.wait_cluster(red_bar, 0u, kWherePartials));
             if (threadIdx.x == 0) KX_TRACE_POINT(p, blockIdx.x, 7);
+            // Second arrival only now: every copy addressed to this CTA has landed.  Once all CTAs of the
+            // cluster have arrived, every copy of the cluster is complete, so no CTA that passes the final
+            // wait can still be read from or written to.
+            cluster_arrive_relaxed();
             if (reducer && have) {
 #pragma unroll 1
                 for (int u = 0; tile_row(warp + 4 * u) < m_cnt; ++u) {
                     const int k = warp + 4 * u, i = tile_row(k);
                     float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-                    const uint32_t src = s_recv + static_cast<uint32_t>((k * 128 + lane * 4) * 4);
+                    // slot [split j][sending warp = column quarter][row k][32 columns]; this lane's 4 columns
+                    const uint32_t src = s_recv + static_cast<uint32_t>((((lane >> 3) * rows_per + k) * 32 + (lane & 7) * 4) * 4);
 #pragma unroll
                     for (int j = 0; j < 8; ++j)
                         if (j < p.splits) {
                             float4 t;
                             asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
                                          : "=f"(t.x), "=f"(t.y), "=f"(t.z), "=f"(t.w)
-                                         : "r"(src + static_cast<uint32_t>(j * rows_per * 512)));
+                                         : "r"(src + static_cast<uint32_t>(j * 4 * rows_per * 128)));
                             v.x += t.x; v.y += t.y; v.z += t.z; v.w += t.w;
                         }
                     if (n_ok) {

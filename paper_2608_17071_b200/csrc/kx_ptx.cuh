@@ -136,6 +136,18 @@ __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap
         "l"(reinterpret_cast<uint64_t>(m)), "r"(x), "r"(y), "r"(bar_cluster)
         : "memory");
 }
+// Bulk copy from this CTA's shared memory into the shared memory of a CTA of the cluster (dst and bar are
+// shared::cluster addresses of the destination CTA); the bytes are counted on the destination's mbarrier.
+// Source, destination and size are multiples of 16 bytes.  The source must have been made visible to the
+// asynchronous proxy (fence.proxy.async) and must stay intact until the destination's barrier completes.
+__device__ __forceinline__ void bulk_copy_to_cta(uint32_t dst_cluster, uint32_t src_cta, uint32_t bytes,
+                                                 uint32_t bar_cluster) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+            dst_cluster),
+        "r"(src_cta), "r"(bytes), "r"(bar_cluster)
+        : "memory");
+}
 // Ask for a 2-D tile to be brought into L2 (no shared-memory destination, no completion signal).
 // L2 is the coherence point of the device, so a tile prefetched early still reflects any later
 // write made through L2 before it is actually loaded.

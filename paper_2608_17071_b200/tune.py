@@ -29,9 +29,14 @@ ATOL, RTOL = 1e-2, 1.6e-2
 
 
 def m_bucket(M: int):
-    """M range an entry applies to: [1,16], (16,32], (32,64], ... (powers of two)."""
+    """M range an entry applies to: [1,4], [5,8], [9,16], (16,32], (32,64], ... (the kernels for a few
+    rows change at 4 and 32; above that, powers of two)."""
+    if M <= 4:
+        return 1, 4
+    if M <= 8:
+        return 5, 8
     if M <= 16:
-        return 1, 16
+        return 9, 16
     hi = 1 << (M - 1).bit_length()
     return hi // 2 + 1, hi
 
@@ -39,6 +44,13 @@ def m_bucket(M: int):
 def candidates(M: int, N: int, K: int, kx):
     T, S = kx.KX_PATH_TILE, kx.KX_PATH_SWAP
     out = []
+    if M <= 4:
+        for rw in (1, 2, 4):
+            for warps in (2, 3, 4, 5, 6, 8, 12, 16):
+                out.append(dict(path=kx.KX_PATH_GEMV, block_n=rw, split_k=warps))
+    if M <= 32:
+        for rw in (16, 32):
+            out.append(dict(path=kx.KX_PATH_SKINNY, block_n=rw))
     if M <= 256:
         bn = 16 if M <= 16 else 32 if M <= 32 else 64 if M <= 64 else 128 if M <= 128 else 256
         for sk in (1, 2, 3, 4, 5, 6, 8):
@@ -47,6 +59,9 @@ def candidates(M: int, N: int, K: int, kx):
         out.append(dict(path=S, block_n=bn, stages=one_kb_swap[bn]))
         for sk in (2, 4, 8, 12, 16):
             out.append(dict(path=S, block_n=bn, split_k=sk, cluster_reduce=1))
+        if bn <= 128:
+            for sk in (2, 3, 4, 6, 8):
+                out.append(dict(path=S, block_n=bn, split_k=sk, cluster_reduce=3))
     if M > 64:
         for bn in (256, 192, 128, 64):
             for pair in (1, 2):
@@ -68,6 +83,13 @@ def candidates(M: int, N: int, K: int, kx):
         for bn in (256, 128):
             out.append(dict(path=T, block_n=bn, cta_pair=1, k_cluster=2, stages=two_kb[(bn, 1)]))
             out.append(dict(path=T, block_n=bn, cta_pair=1, k_cluster=2, stages=one_kb[(bn, 1)]))
+        # CTA-pair tiles whose K range is split over two pairs (a cluster of four)
+        for bn in (256, 192, 128):
+            out.append(dict(path=T, block_n=bn, cta_pair=2, k_cluster=2))
+            out.append(dict(path=T, block_n=bn, cta_pair=2, k_cluster=2, stages=two_kb[(bn, 2)]))
+        # stream-K over the last wave(s)
+        for bn, pair in ((256, 2), (192, 2), (256, 1)):
+            out.append(dict(path=T, block_n=bn, cta_pair=pair, stream_k=2))
     return out
 
 

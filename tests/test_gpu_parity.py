@@ -172,6 +172,35 @@ def test_k_cluster_exact_integer_arithmetic(bn, kc, M, N, K):
     assert ok, msg
 
 
+@pytest.mark.parametrize("bn,stages", [(256, 0), (256, 3), (256, 5), (192, 0), (128, 0), (128, 4)])
+@pytest.mark.parametrize("M,N,K", [(256, 256, 512), (512, 2048, 2048), (300, 520, 520), (640, 1032, 4096)])
+def test_k_cluster_of_pairs_exact_integer_arithmetic(bn, stages, M, N, K):
+    """CTA-pair tiles (256 rows) whose K range is split over two pairs, a cluster of four CTAs; each CTA sums
+    the two partials of its 128 rows through distributed shared memory.  Integer-valued data: bit-exact,
+    also in place and without bias / residual."""
+    ov = dict(path=T, block_n=bn, cta_pair=2, k_cluster=2, stages=stages)
+    X, W, b, R = ternary_case(M, N, K, seed=29)
+    y = run(X, W, b, R, ov)
+    ok, msg = kt.gate_exact(y, oracle.outproj(X, W, b, R))
+    assert ok, msg
+    assert np.array_equal(run(X, W, b, R.copy(), ov, inplace=True), y)
+    ok, msg = kt.gate_exact(run(X, W, None, None, ov), oracle.outproj(X, W))
+    assert ok, msg
+
+
+def test_k_cluster_of_pairs_is_the_plan_for_a_few_tile_rows():
+    info = kx.kx_plan_query(512, 4096, 4096, ov=kx.make_override(no_table=1))
+    assert (info.path, info.cta_pair, info.block_n, info.grid, info.tiles) == (T, 2, 256, 128, 32)
+    d = inputs.make_inputs(inputs.all_workloads()["sweep_M512_H4096"], stress=True)
+    ref, absref = oracle.outproj(d["X"], d["W"], d["bias"], d["R"], want_abs=True)
+    ys = [run(d["X"], d["W"], d["bias"], d["R"], dict(no_table=1)) for _ in range(2)]
+    assert np.array_equal(ys[0], ys[1])
+    ok, msg = kt.gate_a(ys[0], ref)
+    assert ok, msg
+    ok, msg = kt.gate_c(ys[0], ref, absref, 4096, rate_limit=3e-2)
+    assert ok, msg
+
+
 def test_k_cluster_random_data_and_bad_plans():
     d = inputs.make_inputs(inputs.all_workloads()["sweep_M512_H2048"], stress=True)
     ref, absref = oracle.outproj(d["X"], d["W"], d["bias"], d["R"], want_abs=True)
@@ -183,7 +212,7 @@ def test_k_cluster_random_data_and_bad_plans():
         assert ok, msg
         ok, msg = kt.gate_c(ys[0], ref, absref, 2048, rate_limit=3e-2)
         assert ok, msg
-    for bad in (dict(path=T, block_n=256, cta_pair=2, k_cluster=2), dict(path=T, block_n=256, cta_pair=1, k_cluster=3),
+    for bad in (dict(path=T, block_n=256, cta_pair=2, k_cluster=4), dict(path=T, block_n=256, cta_pair=1, k_cluster=3),
                 dict(path=T, block_n=256, cta_pair=1, k_cluster=2, stream_k=2)):
         with pytest.raises(kx.KxError):
             kx.kx_plan_query(512, 2048, 2048, ov=kx.make_override(**bad))
@@ -192,6 +221,7 @@ def test_k_cluster_random_data_and_bad_plans():
 @pytest.mark.parametrize("depth", [-1, 0, 1, 3, 1000])
 @pytest.mark.parametrize("base", [dict(path=T, block_n=256, cta_pair=2), dict(path=T, block_n=128, cta_pair=1),
                                   dict(path=T, block_n=256, cta_pair=1, k_cluster=2), dict(path=T, block_n=256, cta_pair=2, narrow_tail=2),
+                                  dict(path=T, block_n=256, cta_pair=2, k_cluster=2),
                                   dict(path=S, block_n=32, split_k=3), dict(path=S, block_n=16, split_k=4, cluster_reduce=2),
                                   dict(path=S, block_n=32, split_k=4, cluster_reduce=3)], ids=vid)
 def test_l2_prefetch_depth_changes_no_bit(base, depth):
@@ -473,12 +503,12 @@ def test_non_default_stream_and_plan_query():
     import torch
     info = kx.kx_plan_query(4096, 4096, 4096)
     assert info.path == T and info.grid >= 1 and info.launches == 1 and info.tiles >= info.grid // 2
-    info = kx.kx_plan_query(32, 4096, 4096)
+    info = kx.kx_plan_query(32, 8192, 8192)
     assert info.path == S and info.block_n == 32 and info.split_k >= 1
-    ws = info.split_k * 32 * 4096 * 4 if (info.split_k > 1 and not info.cluster_reduce) else 0
+    ws = info.split_k * 32 * 8192 * 4 if (info.split_k > 1 and not info.cluster_reduce) else 0
     assert info.workspace_bytes == ws and (info.cluster_reduce == 0 or 2 <= info.split_k <= 8)
     assert info.cluster_reduce == 1          # the splits form a cluster; finishers pull the partial rows
-    assert kx.kx_plan_query(32, 4096, 4096, ov=kx.make_override(path=S, cluster_reduce=3)).cluster_reduce == 2
+    assert kx.kx_plan_query(32, 8192, 8192, ov=kx.make_override(path=S, cluster_reduce=3)).cluster_reduce == 2
     with pytest.raises(kx.KxError):          # no push form with 256 rows of X per unit
         kx.kx_plan_query(200, 4096, 4096, ov=kx.make_override(path=S, block_n=256, split_k=2, cluster_reduce=3))
     with pytest.raises(kx.KxError):
