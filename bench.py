@@ -251,6 +251,34 @@ def time_warm(torch, call, steps=200, repeats=3):
     return sorted(ts)[len(ts) // 2]
 
 
+def time_graph(torch, calls, n=100, repeats=5):
+    """Device-side time of one call inside a CUDA graph of `n` back-to-back calls (round-robin over `calls`):
+    no host launch cost between the kernels, the programmatic dependencies between them kept by the capture."""
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        bound = [c.rebind(side) if hasattr(c, "rebind") else c for c in calls]
+        for i in range(3):
+            bound[i % len(bound)]()
+        side.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            for i in range(n):
+                bound[i % len(bound)]()
+        ts = []
+        for _ in range(repeats):
+            g.replay()
+            side.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(side)
+            g.replay()
+            e1.record(side)
+            side.synchronize()
+            ts.append(e0.elapsed_time(e1) * 1e-3 / n)
+    torch.cuda.current_stream().wait_stream(side)
+    return sorted(ts)[len(ts) // 2]
+
+
 def time_shape(torch, kx, wl, sets, repeats=5, block_s=0.03, idle_s=0.25):
     """Per-shape protocol of the sweep: `repeats` timed blocks of at most ~block_s seconds of
     back-to-back calls, each after a short idle and 3 warm-up calls, so that every shape is
@@ -408,14 +436,16 @@ def run_ours(args):
 
     # ---- every other workload (rank 0, N = 1 only): per-shape roofline lines
     shapes = []
-    launch_floor_us = None
+    launch_floor_us = launch_floor_host_us = None
     if rank == 0 and world == 1 and "shapes" in sections:
         # cost of one call in a stream of calls when there is (almost) nothing to do: the library's own
         # kernel on an 1 x 8 x 8 problem, launched like every other call (programmatic dependent launch)
         tiny = inputs.Workload("tiny", 1, 8, 8, 0, True, True)
         tset = bind_sets(kx, tiny, device_sets(torch, tiny, 2))
-        launch_floor_us = time_warm(torch, lambda: (tset[0](), tset[1]()), steps=200) / 2 * 1e6
-        print(f"[bench] launch floor (1 x 8 x 8 call in a stream of calls): {launch_floor_us:.2f} us", file=sys.stderr, flush=True)
+        launch_floor_us = time_graph(torch, tset, n=200) * 1e6          # device side: inside a CUDA graph
+        launch_floor_host_us = time_warm(torch, lambda: (tset[0](), tset[1]()), steps=200) / 2 * 1e6   # eager stream of calls
+        print(f"[bench] launch floor (1 x 8 x 8 call): {launch_floor_us:.2f} us per call inside a CUDA graph, "
+              f"{launch_floor_host_us:.2f} us in an eager stream of calls (host launch rate)", file=sys.stderr, flush=True)
         order = ["cfg1", "cfg2", "cfg4", "cfg5", "gemm4096"] + [w.name for w in inputs.sweep_workloads()]
         for name in order:
             w = wls[name]
@@ -440,9 +470,10 @@ def run_ours(args):
             if t_roof < 3e-6:
                 # roofline time below ~3 us: also the amortised time of a back-to-back stream on ONE operand
                 # set (warm L2), labelled as such
-                tw = time_warm(torch, ss[0])
+                tw = time_graph(torch, [ss[0]], n=200)
                 shapes[-1]["amortised_warm_us"] = tw * 1e6
-                shapes[-1]["amortised_warm_note"] = "same buffers, back-to-back stream of 200 calls, operands warm in L2"
+                shapes[-1]["amortised_warm_note"] = ("one operand set (warm in L2), 200 back-to-back calls replayed from a "
+                                                     "CUDA graph: device time per call without host launch cost")
             del ss
             torch.cuda.empty_cache()
             print(f"[bench] {name:>18s} M={w.M:<6d} N={w.N:<5d} K={w.K:<6d} {t*1e6:9.1f} us (best {tbest*1e6:7.1f}) "
@@ -933,6 +964,7 @@ def run_ours(args):
                              "note": "value = median block; every block holds at least the --steps asked for"},
             "clocks": clk.summary(),
             "launch_floor_us": launch_floor_us,
+            "launch_floor_host_us": launch_floor_host_us,
             "shapes": shapes,
             "sustained": sustained_leg,
             "rmsnorm": norm,

@@ -84,7 +84,9 @@ enum { KX_PATH_AUTO = 0, KX_PATH_TILE = 1, KX_PATH_SWAP = 2, KX_PATH_GEMV = 3, K
  *                 hold two k-blocks have their own (smaller) stage counts
  *   stream_k      tile path: 0 auto, 1 = whole tiles per CTA (round-robin), 2 = stream-K
  *                 (every CTA gets an equal contiguous range of (tile, k-block) units;
- *                 split tiles are summed in the FP32 workspace in a fixed order)
+ *                 split tiles are summed in the FP32 workspace in a fixed order), 3 = the tiles
+ *                 left over after the full waves are split that way and run FIRST, the rest whole
+ *                 (the summing of a split tile then overlaps the next tile's main loop)
  *   narrow_tail   tile path: 0 auto, 1 off, 2 = run the tiles left over after the full
  *                 waves as half-width tiles when they then fit in one extra wave
  *   cluster_reduce  swap path: 0 auto, 1 = sum the K splits through the FP32 workspace
@@ -143,7 +145,7 @@ typedef struct kx_plan_info {
     int32_t launches;      /* kernels enqueued per call                            */
     int32_t smem_bytes;    /* dynamic shared memory per CTA                        */
     int64_t workspace_bytes; /* FP32 split-K / stream-K scratch this plan uses (0 if none) */
-    int32_t stream_k;      /* 1 if the tile path runs with stream-K scheduling     */
+    int32_t stream_k;      /* tile path: 1 = stream-K over the last waves, 2 = over the leftover tiles, first */
     int32_t narrow_tiles;  /* number of half-width tail tiles (0 if none)          */
     int32_t cluster_reduce;/* swap path: 0 = workspace, 1 = cluster (partials pulled), 2 = cluster (partials pushed) */
     int32_t from_table;    /* 1 if the built-in measured plan table supplied this plan */
@@ -154,6 +156,18 @@ typedef struct kx_plan_info {
  * attributes, the split-K workspace and its counters) so that later calls do
  * no allocation.  Idempotent, thread-safe.  Without it, the first kx_* call on
  * a device does the same lazily (so make that first call outside stream capture).
+ *
+ * Shared state and concurrency.  Each device has ONE FP32 workspace, one array of tile counters and
+ * one status word, shared by every stream and host thread.  Calls whose plan uses the workspace
+ * (kx_plan_info.workspace_bytes > 0: split-K through the workspace, i.e. more than 8 splits, a capped
+ * grid or cluster_reduce = 1, and stream-K) must not overlap on the GPU with one another: order them
+ * on one stream or with events, as for kx_outproj_residual_noalloc's built-in scratch.  The heuristic
+ * plans of kx_outproj_residual / kx_gemm_bf16 / _strided / _batched use no workspace (cluster
+ * reductions and whole tiles), so those calls may overlap freely; an entry of the built-in measured
+ * plan table may name a workspace plan for its shape, and kx_plan_query tells (workspace_bytes).  kx_outproj_residual_host also owns
+ * one staging buffer and one set of copy streams per device: its calls must not overlap each other.
+ * Host-side entry is thread-safe (the per-device state is built once under a lock; descriptor caches
+ * are per thread).
  */
 int kx_init(int device);
 
@@ -225,6 +239,12 @@ int kx_outproj_residual_host(const void* X_host, const void* W_host, const void*
  * and partial sums are rewritten before they are read.  Two calls that run on the GPU at
  * the same time (different streams, or different host threads on one device) would race
  * on the array: order them on one stream or with events.
+ *
+ * Errors raised by the kernel itself (a bounded wait that gave up) are read with
+ * kx_last_device_status, which allocates nothing either.  Two environment variables, read once at
+ * the first call on a device, exist for tests only: KX_NOALLOC_SPIN_US (bound on device-side waits,
+ * default 2 000 000) and KX_NOALLOC_DEBUG_DROP (the loader withholds that many stages, so a wait
+ * runs out and the call reports KX_ERR_DEVICE_TIMEOUT; the kernel still exits cleanly).
  */
 int kx_outproj_residual_noalloc(const void* X, const void* W, const void* bias_or_null,
                                 const void* R_or_null, void* Y, int64_t M, int64_t N, int64_t K,
@@ -491,6 +511,8 @@ int kx_plan_query(int64_t M, int64_t N, int64_t K, int has_bias, int has_residua
  * Synchronises `stream`, then reads and clears the current device's kernel
  * status word.  *code_out is KX_OK or KX_ERR_DEVICE_TIMEOUT; *detail_out (may be
  * NULL) identifies which wait gave up.  Debug/test use: it blocks the host.
+ * Allocates nothing and needs no kx_init: the status word is part of the library's device
+ * image (callers of kx_outproj_residual_noalloc may use it).
  */
 int kx_last_device_status(void* stream, int* code_out, int* detail_out);
 

@@ -466,6 +466,8 @@ def bound_call(X, W, bias, R, Y, stream=None, plain: bool = False, ov: Optional[
         if rc != KX_OK:
             raise KxError(rc, fn.__name__)
     run.tensors = keep
+    # the same call bound to another stream (a capture stream, for instance)
+    run.rebind = lambda new_stream: bound_call(X, W, bias, R, Y, stream=new_stream, plain=plain, ov=ov)
     return run
 
 

@@ -6,6 +6,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <atomic>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -36,7 +37,7 @@ constexpr int kMaxCounters = 1 << 16;
 __device__ unsigned int g_kx_status[4];
 
 struct DeviceCtx {
-    bool ready = false;
+    std::atomic<bool> ready{false};   // set last (release) by the thread that built the state; read with acquire
     int sm_count = 0;
     float* ws = nullptr;
     unsigned int* counters = nullptr;
@@ -170,12 +171,12 @@ const SwapVariant* find_swap(int bn, int stages = 0) {
 int ensure_device(int dev, DeviceCtx** out) {
     if (dev < 0 || dev >= kMaxDevices) return KX_ERR_CUDA;
     DeviceCtx& c = g_ctx[dev];
-    if (c.ready) {
+    if (c.ready.load(std::memory_order_acquire)) {
         *out = &c;
         return KX_OK;
     }
     std::lock_guard<std::mutex> lk(g_mu);
-    if (c.ready) {
+    if (c.ready.load(std::memory_order_relaxed)) {
         *out = &c;
         return KX_OK;
     }
@@ -239,7 +240,7 @@ int ensure_device(int dev, DeviceCtx** out) {
             rc = KX_ERR_CUDA;
             break;
         }
-        c.ready = true;
+        c.ready.store(true, std::memory_order_release);
     } while (false);
     if (rc != KX_OK) {
         cudaGetLastError();
@@ -348,6 +349,7 @@ struct Plan {
     int splits = 1;
     int stream_k = 0;
     int sk_tile0 = 0;
+    int sk_first_tiles = 0; // > 0: the stream-K region is the first so many tiles (sk_tile0 == units)
     int from_table = 0;     // 1 if the static plan table supplied this plan
     int kcluster = 1;       // tile path: CTAs per K cluster (1 = none)
     int cluster_reduce = 0; // swap path: the splits of a tile form a cluster and reduce through DSMEM
@@ -675,11 +677,25 @@ int make_plan_from(long long M, long long N, long long K, const kx_plan_override
         (void)dp_eff;
         if (sk == 0) sk = 1;
         if (sk == 2 && !sk_fits) return KX_ERR_WORKSPACE;
-        if (sk != 1 && sk != 2) return KX_ERR_PLAN;
+        if (sk != 1 && sk != 2 && sk != 3) return KX_ERR_PLAN;
         pl->stream_k = (sk == 2) ? 1 : 0;
         pl->sk_tile0 = pl->stream_k ? sk_tile0 : pl->units;
         pl->grid = (pl->stream_k ? (sk_tile0 > 0 ? slots : sk_slots) : std::min(pl->units, slots)) * ctas;
         pl->ws_bytes = pl->stream_k ? sk_ws : 0;
+        if (sk == 3) {
+            // Stream-K FIRST: the tiles left over after the full waves are cut into equal ranges of (tile,
+            // k-block) units, one per slot, and run before the whole tiles; a slot that ends a split tile
+            // parks its partial in the workspace (or, arriving last, adds its partners' partials) in its
+            // epilogue warps while its next whole tile is already in the main loop.
+            if (rem == 0 || full_waves < 1) return KX_ERR_PLAN;
+            const size_t ws1 = static_cast<size_t>(slots) * 2 * ctas * 128 * bn * sizeof(float);
+            if (ws1 > kWorkspaceBytes || static_cast<long long>(rem) * ctas * 4 > kMaxCounters) return KX_ERR_WORKSPACE;
+            pl->stream_k = 2;
+            pl->sk_first_tiles = rem;
+            pl->sk_tile0 = pl->units;
+            pl->grid = slots * ctas;
+            pl->ws_bytes = ws1;
+        }
         // Half-width tail: when the tiles left over after the full waves fit, cut in two, into
         // one more (half as long) wave, run them as 128*ctas x BN/2 tiles.  No reduction, no
         // workspace; 4096 x 4096 on 74 pair slots becomes 3 + 1/2 wave-times instead of 4.
@@ -941,6 +957,7 @@ int run(const void* X, const void* W, const void* bias, const void* R, void* Y, 
         p.swiglu = 0;
         p.kcluster = pl.kcluster;
         p.sk_tile0 = pl.sk_tile0;
+        p.sk_first_tiles = pl.sk_first_tiles;
         p.narrow_tile0 = pl.narrow_tile0;
         p.spin_limit_ns = spin_ns;
         p.status = ctx->status;
@@ -1037,7 +1054,7 @@ int kx_shutdown(void) {
     cudaGetDevice(&prev);
     for (int d = 0; d < kMaxDevices; ++d) {
         DeviceCtx& c = g_ctx[d];
-        if (!c.ready && !c.stage) continue;
+        if (!c.ready.load(std::memory_order_acquire) && !c.stage) continue;
         cudaSetDevice(d);
         cudaDeviceSynchronize();
         if (c.ws) cudaFree(c.ws);
@@ -1053,7 +1070,16 @@ int kx_shutdown(void) {
                 cudaEventDestroy(c.h_k_ev[i]);
             }
         }
-        c = DeviceCtx();
+        c.ready.store(false, std::memory_order_release);
+        c.sm_count = 0;
+        c.ws = nullptr;
+        c.counters = nullptr;
+        c.status = nullptr;
+        c.stage = nullptr;
+        c.stage_bytes = 0;
+        c.h_in = c.h_out = nullptr;
+        c.h_start = c.h_done = nullptr;
+        for (int i = 0; i < 8; ++i) c.h_in_ev[i] = c.h_k_ev[i] = nullptr;
     }
     cudaSetDevice(prev);
     return KX_OK;
@@ -1149,18 +1175,27 @@ int kx_last_device_status(void* stream, int* code_out, int* detail_out) {
     if (!code_out) return KX_ERR_NULL;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return KX_ERR_CUDA;
-    DeviceCtx* ctx = nullptr;
-    int rc = ensure_device(dev, &ctx);
-    if (rc != KX_OK) return rc;
+    if (dev < 0 || dev >= kMaxDevices) return KX_ERR_CUDA;
+    // The status words are a device symbol of the library image: their address is looked up, nothing is
+    // allocated, and the per-device state of the allocating entry points is neither needed nor created
+    // (so a caller of kx_outproj_residual_noalloc can read its kernel's status too).
+    unsigned int* status = nullptr;
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&status), g_kx_status) != cudaSuccess || !status) {
+        cudaGetLastError();
+        return KX_ERR_CUDA;
+    }
     if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return KX_ERR_CUDA;
     unsigned int h[4] = {0, 0, 0, 0};
-    if (cudaMemcpy(h, ctx->status, sizeof h, cudaMemcpyDeviceToHost) != cudaSuccess) return KX_ERR_CUDA;
+    if (cudaMemcpy(h, status, sizeof h, cudaMemcpyDeviceToHost) != cudaSuccess) return KX_ERR_CUDA;
     *code_out = static_cast<int>(h[0]);
     if (detail_out) *detail_out = static_cast<int>(h[1]);
     if (h[0] != 0) {
-        // a kernel that gave up may have left split-K tile counters part-way
-        if (cudaMemset(ctx->status, 0, sizeof h) != cudaSuccess ||
-            cudaMemset(ctx->counters, 0, kMaxCounters * sizeof(unsigned int)) != cudaSuccess)
+        // a kernel that gave up may have left split-K tile counters part-way (the counters of the no-allocation
+        // entry point are cleared before each of its launches anyway)
+        if (cudaMemset(status, 0, sizeof h) != cudaSuccess) return KX_ERR_CUDA;
+        DeviceCtx& c = g_ctx[dev];
+        if (c.ready.load(std::memory_order_acquire) &&
+            cudaMemset(c.counters, 0, kMaxCounters * sizeof(unsigned int)) != cudaSuccess)
             return KX_ERR_CUDA;
     }
     return KX_OK;
@@ -1463,13 +1498,38 @@ int launch_rowquant(const QuantParams& qp, bool norm, int fmt, cudaStream_t stre
                         : reinterpret_cast<const void*>(&kx_rowquant_kernel<NV, false, 1>))          \
                 : (norm ? reinterpret_cast<const void*>(&kx_rowquant_kernel<NV, true, 0>)            \
                         : reinterpret_cast<const void*>(&kx_rowquant_kernel<NV, false, 0>)))
-    if (nvec <= 1 * kNormThreads) { fn = KX_QUANT_FN(1); }
+#define KX_QUANTW_FN(NV)                                                                             \
+    (fmt == 3 ? (norm ? reinterpret_cast<const void*>(&kx_rowquant_warp_kernel<NV, true, 3>)         \
+                      : reinterpret_cast<const void*>(&kx_rowquant_warp_kernel<NV, false, 3>))       \
+     : fmt == 2 ? (norm ? reinterpret_cast<const void*>(&kx_rowquant_warp_kernel<NV, true, 2>)       \
+                      : reinterpret_cast<const void*>(&kx_rowquant_warp_kernel<NV, false, 2>))       \
+     : fmt == 1 ? (norm ? reinterpret_cast<const void*>(&kx_rowquant_warp_kernel<NV, true, 1>)       \
+                        : reinterpret_cast<const void*>(&kx_rowquant_warp_kernel<NV, false, 1>))     \
+                : (norm ? reinterpret_cast<const void*>(&kx_rowquant_warp_kernel<NV, true, 0>)       \
+                        : reinterpret_cast<const void*>(&kx_rowquant_warp_kernel<NV, false, 0>)))
+    // Rows of up to 4096 elements: one warp per row (no block barriers; same bits).  KX_ROWQUANT_CTA=1 in the
+    // environment keeps the CTA-per-row kernel (for A/B timing).
+    static const bool force_cta = [] {
+        const char* e = std::getenv("KX_ROWQUANT_CTA");
+        return e && e[0] == '1';
+    }();
+    bool warp_form = false;
+    if (!force_cta && nvec <= 2 * kNormThreads && qp.M >= 64) {
+        fn = (nvec <= kNormThreads) ? KX_QUANTW_FN(1) : KX_QUANTW_FN(2);
+        warp_form = true;
+    } else if (nvec <= 1 * kNormThreads) { fn = KX_QUANT_FN(1); }
     else if (nvec <= 2 * kNormThreads) { fn = KX_QUANT_FN(2); }
     else if (nvec <= 4 * kNormThreads) { fn = KX_QUANT_FN(4); per_sm = 6; }
     else if (nvec <= 8 * kNormThreads) { fn = KX_QUANT_FN(8); per_sm = 4; }
     else { fn = KX_QUANT_FN(kNormVecs); per_sm = 2; }
 #undef KX_QUANT_FN
-    cfg.gridDim = dim3(row_grid(qp.M, sm_count, per_sm), 1, 1);
+#undef KX_QUANTW_FN
+    if (warp_form) {
+        const long long ctas = (qp.M + 7) / 8;
+        cfg.gridDim = dim3(static_cast<unsigned>(std::min<long long>(ctas, static_cast<long long>(sm_count) * 8)), 1, 1);
+    } else {
+        cfg.gridDim = dim3(row_grid(qp.M, sm_count, per_sm), 1, 1);
+    }
     cfg.blockDim = dim3(kNormThreads, 1, 1);
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
@@ -2296,6 +2356,8 @@ namespace {
 struct NoAllocCtx {
     bool ready = false;
     int sm_count = 0;
+    int debug_drop_kblocks = 0;         // test hook (KX_NOALLOC_DEBUG_DROP): the producer withholds stages
+    unsigned long long spin_limit_ns = 2000000000ull;   // bound on device-side waits (KX_NOALLOC_SPIN_US)
     unsigned char* scratch = nullptr;   // device address of g_kx_noalloc_scratch on this device
     unsigned int* status = nullptr;
 };
@@ -2344,6 +2406,14 @@ int noalloc_setup(int dev, NoAllocCtx** out) {
     c.sm_count = sms;
     c.scratch = ptr;
     c.status = st;
+    // Test hooks, read once here: they make a device-side wait run out from the host side (the producer
+    // issues fewer stages than the consumer expects) so that the give-up path and the status read can be
+    // exercised through this entry point, which takes no plan override.  Never set in production.
+    if (const char* e = std::getenv("KX_NOALLOC_DEBUG_DROP")) c.debug_drop_kblocks = std::max(0, std::atoi(e));
+    if (const char* e = std::getenv("KX_NOALLOC_SPIN_US")) {
+        const long long us = std::atoll(e);
+        if (us > 0) c.spin_limit_ns = static_cast<unsigned long long>(us) * 1000ull;
+    }
     c.ready = true;
     *out = &c;
     return KX_OK;
@@ -2401,9 +2471,9 @@ int kx_outproj_residual_noalloc(const void* X, const void* W, const void* bias, 
     p.num_units = n_tiles * splits;
     p.has_bias = bias ? 1 : 0;
     p.has_r = R ? 1 : 0;
-    p.drop_kblocks = 0;
+    p.drop_kblocks = ctx->debug_drop_kblocks;
     p.pf_kblocks = 0;
-    p.spin_limit_ns = 2000000000ull;
+    p.spin_limit_ns = ctx->spin_limit_ns;
     p.status = ctx->status;
     p.ws = partials;
     p.counters = counters;

@@ -159,6 +159,10 @@ struct TileParams {
                                   // through distributed shared memory in rank order
     int sk_tile0;                 // tiles [0, sk_tile0) are taken whole, round-robin over the slots;
                                   // tiles [sk_tile0, num_tiles) are stream-K'd (== num_tiles: none)
+    int sk_first_tiles;           // > 0: the stream-K region is the FIRST sk_first_tiles tiles instead (sk_tile0 ==
+                                  // num_tiles): every slot starts with its share of their (tile, k-block) units and
+                                  // then takes the remaining tiles whole, round-robin, so that the fix-up of a
+                                  // split tile runs in the epilogue warps under the main loop of the next tile
     int narrow_tile0;             // tile ids >= narrow_tile0 are half-width tiles: id = narrow_tile0 + 2 * j + half
                                   // covers columns [half * BN/2, +BN/2) of full-width position narrow_tile0 + j
                                   // (== num_tiles: none; never combined with stream-K)
@@ -213,38 +217,49 @@ __device__ __forceinline__ int sk_slot_of(long long U, int G, long long u) {
 
 // The work of one slot (a CTA or a CTA pair) as a sequence of segments (tile, kb0, kb1).
 struct SegIter {
-    int nkb, sk_tile0, t, tstride, kc_kb0, kc_kb1;
+    int nkb, t, t_end, tstride, kc_kb0, kc_kb1, sk_base;
+    bool sk_first;
     long long u, u1;
     // krank / kcluster: position of this CTA in its K cluster (0 / 1 when there is none)
     __device__ __forceinline__ void init(const TileParams& p, int nkb_, int slot, int slots, int krank = 0,
                                          int kcluster = 1) {
         nkb = nkb_;
-        sk_tile0 = p.sk_tile0;
-        t = slot;
+        sk_first = p.sk_first_tiles > 0;
+        sk_base = sk_first ? 0 : p.sk_tile0;                       // first tile of the stream-K region
+        const int sk_tiles = sk_first ? p.sk_first_tiles : p.num_tiles - p.sk_tile0;
+        t = (sk_first ? p.sk_first_tiles : 0) + slot;              // whole tiles: [.., t_end), round-robin
+        t_end = sk_first ? p.num_tiles : p.sk_tile0;
         tstride = slots;
         kc_kb0 = static_cast<int>((static_cast<long long>(krank) * nkb_) / kcluster);
         kc_kb1 = static_cast<int>((static_cast<long long>(krank + 1) * nkb_) / kcluster);
-        const long long U = static_cast<long long>(p.num_tiles - p.sk_tile0) * nkb_;
+        const long long U = static_cast<long long>(sk_tiles) * nkb_;
         u = sk_begin(U, slots, slot);
         u1 = sk_begin(U, slots, slot + 1);
     }
-    __device__ __forceinline__ bool next(int& tile, int& kb0, int& kb1) {
-        if (t < sk_tile0) {
-            tile = t;
-            kb0 = kc_kb0;
-            kb1 = kc_kb1;
-            t += tstride;
-            return true;
-        }
+    __device__ __forceinline__ bool next_whole(int& tile, int& kb0, int& kb1) {
+        if (t >= t_end) return false;
+        tile = t;
+        kb0 = kc_kb0;
+        kb1 = kc_kb1;
+        t += tstride;
+        return true;
+    }
+    __device__ __forceinline__ bool next_sk(int& tile, int& kb0, int& kb1) {
         if (u >= u1) return false;
         const int st = static_cast<int>(u / nkb);
-        tile = sk_tile0 + st;
+        tile = sk_base + st;
         kb0 = static_cast<int>(u - static_cast<long long>(st) * nkb);
         const long long len = min(static_cast<long long>(nkb - kb0), u1 - u);
         kb1 = kb0 + static_cast<int>(len);
         u += len;
         return true;
     }
+    __device__ __forceinline__ bool next(int& tile, int& kb0, int& kb1) {
+        if (sk_first) return next_sk(tile, kb0, kb1) || next_whole(tile, kb0, kb1);
+        return next_whole(tile, kb0, kb1) || next_sk(tile, kb0, kb1);
+    }
+    // nothing left after the segment that next() returned last
+    __device__ __forceinline__ bool exhausted() const { return t >= t_end && u >= u1; }
 };
 
 __device__ __forceinline__ uint32_t ld_acquire_gpu_u32(const unsigned int* p) {
@@ -631,7 +646,8 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const int q = warp;
         const uint32_t my_epi = s_epi + q * NB * C::SLAB_BYTES;
         const bool has_r = p.has_r != 0, has_bias = p.has_bias != 0;
-        const long long U = static_cast<long long>(p.num_tiles - p.sk_tile0) * nkb;   // stream-K units
+        const int sk_base = (p.sk_first_tiles > 0) ? 0 : p.sk_tile0;                  // first stream-K tile
+        const long long U = static_cast<long long>(p.sk_first_tiles > 0 ? p.sk_first_tiles : p.num_tiles - p.sk_tile0) * nkb;   // stream-K units
         // Inside a partial, the 64 FP32 values a thread holds for chunk c live at float4 index
         // ((c*4 + q)*16 + g)*32 + lane, g = 0..15: every warp-wide access is 512 contiguous bytes.
         auto slab4 = [&](float* part, int c) {
@@ -667,7 +683,7 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
         // partial of (slot sl, tile tl) for this CTA rank: "head" if tl is the first tile the slot touches
         auto part_ptr = [&](int sl, int tl) -> float* {
-            const int first_tile = p.sk_tile0 + static_cast<int>(sk_begin(U, slots, sl) / nkb);
+            const int first_tile = sk_base + static_cast<int>(sk_begin(U, slots, sl) / nkb);
             const size_t idx = (static_cast<size_t>(sl) * 2 + (tl == first_tile ? 0 : 1)) * CTAS + cta_rank;
             return p.ws + idx * C::PART_FLOATS;
         };
@@ -705,7 +721,7 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             // no more chunks than buffers).  They are requested before the accumulator is ready whenever
             // this warp will (whole tile) or is expected to (the slot's last segment: its partners ran
             // at the start of their ranges) produce the output.
-            const bool last_seg = (it.t >= it.sk_tile0) && (it.u >= it.u1);
+            const bool last_seg = it.exhausted();
             const bool spec_r = has_r && (whole || last_seg || kc > 1);
             int n_iss = 0;                                 // R chunks requested so far (warp-uniform)
             if (lane == 0) tma_store_wait_read<0>();       // staging buffers of the previous tile are free
@@ -730,7 +746,7 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             unsigned int* ctr = nullptr;
             bool staged = false;   // the partner's partial already sits in the other accumulator buffer
             if (!whole && kc == 1) {
-                const long long ut = static_cast<long long>(tile - p.sk_tile0) * nkb;
+                const long long ut = static_cast<long long>(tile - sk_base) * nkb;
                 s_first = sk_slot_of(U, slots, ut);
                 s_last = sk_slot_of(U, slots, ut + nkb - 1);
                 ctr = p.counters + (static_cast<size_t>(tile) * CTAS + cta_rank) * 4 + q;
@@ -916,10 +932,13 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 const uint32_t buf = my_epi + j * C::SLAB_BYTES;
                 // the chunk's 64 bias values, all eight loads in flight at once and long before their use (one
                 // after the other, behind the stores below, every load of a cold line cost a trip to L2)
-                uint4 bb8[8];
-                if (has_bias && valid) {
+                // (not in the row-scaled 8-bit kinds, whose dequantisation already fills the register file: they
+                // load each vector where it is used)
+                constexpr int kPreBias = kRowScaled ? 1 : 8;
+                uint4 bb8[kPreBias];
+                if (!kRowScaled && has_bias && valid) {
 #pragma unroll
-                    for (int g8 = 0; g8 < 8; ++g8) {
+                    for (int g8 = 0; g8 < kPreBias; ++g8) {
                         const int n = col0 + g8 * 8;
                         bb8[g8] = (n + 8 <= p.N) ? __ldg(reinterpret_cast<const uint4*>(bias + n)) : make_uint4(0u, 0u, 0u, 0u);
                     }
@@ -1050,19 +1069,31 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         rphase ^= (1u << j);
                     }
                     if (kc > 1 && q == 0 && lane == 0) KX_TRACE_POINT(p, blockIdx.x, 16 + ci * 4 + 1);
+                    // three phases, so that the shared-memory latencies overlap: the residual vectors of this
+                    // lane's row are read first (all eight; four at a time in the row-scaled kinds, which have
+                    // fewer registers to spare), then the outputs are formed, then written back in place
+                    constexpr int PH = kRowScaled ? 4 : 8;
 #pragma unroll
-                    for (int h = 0; h < 2; ++h) {
+                    for (int c0 = 0; c0 < 8; c0 += PH) {
+                        uint4 rr8[PH];
+                        if (has_r) {
 #pragma unroll
-                        for (int g = 0; g < 4; ++g) {
-                            const int c16 = h * 4 + g;     // 16-byte group inside the 128-byte row
-                            const uint32_t addr = buf + lane * 128 + ((c16 ^ (lane & 7)) << 4);
+                            for (int u = 0; u < PH; ++u)
+                                asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+                                             : "=r"(rr8[u].x), "=r"(rr8[u].y), "=r"(rr8[u].z), "=r"(rr8[u].w)
+                                             : "r"(buf + lane * 128 + (((c0 + u) ^ (lane & 7)) << 4)));
+                        }
+#pragma unroll
+                        for (int u = 0; u < PH; ++u) {
+                            const int c16 = c0 + u;        // 16-byte group inside the 128-byte row
+                            const int h = c16 >> 2, g = c16 & 3;
                             float v[8];
 #pragma unroll
                             for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(acc[h][g * 8 + i]);
                             if (has_bias) {
                                 const int n = col0 + c16 * 8;
                                 if (n + 8 <= p.N) {
-                                    const uint4 bb = bb8[c16];
+                                    const uint4 bb = kRowScaled ? __ldg(reinterpret_cast<const uint4*>(bias + n)) : bb8[kRowScaled ? 0 : c16];
                                     v[0] += bf16_lo(bb.x); v[1] += bf16_hi(bb.x);
                                     v[2] += bf16_lo(bb.y); v[3] += bf16_hi(bb.y);
                                     v[4] += bf16_lo(bb.z); v[5] += bf16_hi(bb.z);
@@ -1075,21 +1106,20 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                                 }
                             }
                             if (has_r) {
-                                uint4 rr;
-                                asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
-                                             : "=r"(rr.x), "=r"(rr.y), "=r"(rr.z), "=r"(rr.w)
-                                             : "r"(addr));
+                                const uint4 rr = rr8[u];
                                 v[0] += bf16_lo(rr.x); v[1] += bf16_hi(rr.x);
                                 v[2] += bf16_lo(rr.y); v[3] += bf16_hi(rr.y);
                                 v[4] += bf16_lo(rr.z); v[5] += bf16_hi(rr.z);
                                 v[6] += bf16_lo(rr.w); v[7] += bf16_hi(rr.w);
                             }
-                            const uint32_t o0 = pack_bf16x2(v[0], v[1]), o1 = pack_bf16x2(v[2], v[3]);
-                            const uint32_t o2 = pack_bf16x2(v[4], v[5]), o3 = pack_bf16x2(v[6], v[7]);
-                            asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(o0),
-                                         "r"(o1), "r"(o2), "r"(o3)
-                                         : "memory");
+                            rr8[u] = make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]),       // reused for the output
+                                                pack_bf16x2(v[4], v[5]), pack_bf16x2(v[6], v[7]));
                         }
+#pragma unroll
+                        for (int u = 0; u < PH; ++u)
+                            asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(buf + lane * 128 + (((c0 + u) ^ (lane & 7)) << 4)),
+                                         "r"(rr8[u].x), "r"(rr8[u].y), "r"(rr8[u].z), "r"(rr8[u].w)
+                                         : "memory");
                     }
                     fence_proxy_async_smem();
                     __syncwarp();
@@ -2057,6 +2087,184 @@ kx_rowquant_kernel(const QuantParams p) {
             }
         }
         __syncthreads();         // s_part / s_bcast are reused by the next row
+    }
+}
+
+// The same code books with one WARP per row (rows of up to 4096 elements): lane l plays the threads l, l + 32,
+// ..., l + 224 of the CTA-per-row kernel above, one after the other, and keeps their vectors in registers,
+// so there is no block barrier and no shared memory; a CTA of eight warps works on eight rows at once.
+// Every partial sum is formed in the order of the CTA-per-row kernel (per played thread over its vectors,
+// a shuffle tree per played warp, the played warps in order), so RMSNorm statistics, and with them every
+// code and scale, come out bit for bit the same.
+template <int NV, bool NORM, int FMT>
+__global__ void __launch_bounds__(kNormThreads)
+kx_rowquant_warp_kernel(const QuantParams p) {
+    constexpr float kTop = (FMT == 1) ? 448.0f : 127.0f;
+    constexpr int VT = kNormThreads / 32;                  // played warps per lane
+    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+    const int N = p.N, nvec = N / 8;
+    pdl_wait_prior();
+    pdl_launch_dependents();
+    for (long long m = static_cast<long long>(blockIdx.x) * VT + wib; m < p.M; m += static_cast<long long>(gridDim.x) * VT) {
+        const bool second = m >= p.rows0;
+        const long long r = second ? m - p.rows0 : m;
+        const uint4* row = reinterpret_cast<const uint4*>((second ? p.A1 : p.A0) + r * N);
+        uint4 v[VT][NV];
+        float ssw[VT];
+#pragma unroll
+        for (int w = 0; w < VT; ++w) {
+            ssw[w] = 0.f;
+#pragma unroll
+            for (int i = 0; i < NV; ++i) {
+                const int idx = w * 32 + lane + i * kNormThreads;
+                if (idx < nvec) {
+                    v[w][i] = row[idx];
+                    if (NORM) {
+                        const uint32_t w4[4] = {v[w][i].x, v[w][i].y, v[w][i].z, v[w][i].w};
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            const float a = bf16_lo(w4[k]), b = bf16_hi(w4[k]);
+                            ssw[w] += a * a;
+                            ssw[w] += b * b;
+                        }
+                    }
+                }
+            }
+        }
+        if (NORM) {
+            float t = 0.f;
+#pragma unroll
+            for (int w = 0; w < VT; ++w) {
+                float s = ssw[w];
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+                t += s;
+            }
+            const float inv = rsqrtf(t / static_cast<float>(N) + p.eps);
+#pragma unroll
+            for (int w = 0; w < VT; ++w)
+#pragma unroll
+                for (int i = 0; i < NV; ++i) {
+                    const int idx = w * 32 + lane + i * kNormThreads;
+                    if (idx < nvec) {
+                        const uint4 g = __ldg(reinterpret_cast<const uint4*>(p.gamma) + idx);
+                        const uint32_t h4[4] = {v[w][i].x, v[w][i].y, v[w][i].z, v[w][i].w};
+                        const uint32_t g4[4] = {g.x, g.y, g.z, g.w};
+                        uint32_t o4[4];
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)
+                            o4[k] = pack_bf16x2(bf16_lo(h4[k]) * inv * bf16_lo(g4[k]),
+                                                bf16_hi(h4[k]) * inv * bf16_hi(g4[k]));
+                        v[w][i] = make_uint4(o4[0], o4[1], o4[2], o4[3]);
+                    }
+                }
+        }
+        if constexpr (FMT == 2 || FMT == 3) {
+            uint8_t* const sfrow = p.SF0 + (r >> 7) * p.kchunks * 512 + (r & 31) * 16 + ((r & 127) >> 5) * 4;
+            const float d6 = __fmul_rn(6.0f, p.gs);
+#pragma unroll
+            for (int w = 0; w < VT; ++w)
+#pragma unroll
+                for (int i = 0; i < NV; ++i) {
+                    const int idx = w * 32 + lane + i * kNormThreads;
+                    const bool valid = idx < nvec;
+                    const uint32_t w4[4] = {valid ? v[w][i].x : 0u, valid ? v[w][i].y : 0u, valid ? v[w][i].z : 0u,
+                                            valid ? v[w][i].w : 0u};
+                    float z[8], bmax = 0.f;
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        z[2 * k] = bf16_lo(w4[k]);
+                        z[2 * k + 1] = bf16_hi(w4[k]);
+                        bmax = fmaxf(bmax, fmaxf(fabsf(z[2 * k]), fabsf(z[2 * k + 1])));
+                    }
+                    bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, 1));
+                    if constexpr (FMT == 2) {
+                        bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, 2));
+                        uint32_t e = 127u;
+                        if (valid) {
+                            const int field = static_cast<int>(__float_as_uint(bmax) >> 23);
+                            e = (bmax > 0.f) ? static_cast<uint32_t>(max(field - 8, 0)) : 127u;
+                            const float mult = __uint_as_float((254u - e) << 23);
+#pragma unroll
+                            for (int k = 0; k < 8; ++k) z[k] = __fmul_rn(z[k], mult);
+                            reinterpret_cast<uint2*>(p.Q0 + r * N)[idx] =
+                                make_uint2(pack_e4m3x4(z[0], z[1], z[2], z[3]), pack_e4m3x4(z[4], z[5], z[6], z[7]));
+                        }
+                        uint32_t word = e;
+                        word |= __shfl_down_sync(0xffffffffu, e, 4) << 8;
+                        word |= __shfl_down_sync(0xffffffffu, e, 8) << 16;
+                        word |= __shfl_down_sync(0xffffffffu, e, 12) << 24;
+                        if (valid && (lane & 15) == 0) *reinterpret_cast<uint32_t*>(sfrow + (idx >> 4) * 512) = word;
+                    } else {
+                        uint32_t sb = 0u;
+                        if (valid) {
+                            sb = pack_e4m3x4(__fdiv_rn(bmax, d6), 0.f, 0.f, 0.f) & 0xFFu;
+                            const float dq = __fmul_rn(e4m3_to_f32(sb), p.gs);
+                            const float rcp = (dq > 0.f) ? __fdiv_rn(1.0f, dq) : 0.f;
+#pragma unroll
+                            for (int k = 0; k < 8; ++k) z[k] = __fmul_rn(z[k], rcp);
+                            reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(p.Q0) + r * (N / 2))[idx] =
+                                (dq > 0.f) ? pack_e2m1x8(z) : 0u;
+                        }
+                        uint32_t word = sb;
+                        word |= __shfl_down_sync(0xffffffffu, sb, 2) << 8;
+                        word |= __shfl_down_sync(0xffffffffu, sb, 4) << 16;
+                        word |= __shfl_down_sync(0xffffffffu, sb, 6) << 24;
+                        if (valid && (lane & 7) == 0) *reinterpret_cast<uint32_t*>(sfrow + (idx >> 3) * 512) = word;
+                    }
+                }
+            if (r == p.M - 1) {                              // rows up to the next multiple of 128: padding entries
+                const long long pad_rows = ((p.M + 127) & ~127ll) - p.M;
+                const int per_row = p.kchunks * 4;
+                for (long long t = lane; t < pad_rows * per_row; t += 32) {
+                    const long long rr = p.M + t / per_row;
+                    const int jj = static_cast<int>(t % per_row);
+                    p.SF0[((rr >> 7) * p.kchunks + (jj >> 2)) * 512 + (rr & 31) * 16 + ((rr & 127) >> 5) * 4 + (jj & 3)] =
+                        (FMT == 2) ? 127 : 0;
+                }
+            }
+        } else {
+            float amax = 0.f;
+#pragma unroll
+            for (int w = 0; w < VT; ++w)
+#pragma unroll
+                for (int i = 0; i < NV; ++i) {
+                    const int idx = w * 32 + lane + i * kNormThreads;
+                    if (idx < nvec) {
+                        const uint32_t w4[4] = {v[w][i].x, v[w][i].y, v[w][i].z, v[w][i].w};
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) amax = fmaxf(amax, fmaxf(fabsf(bf16_lo(w4[k])), fabsf(bf16_hi(w4[k]))));
+                    }
+                }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+            if (lane == 0) (second ? p.S1 : p.S0)[r] = (amax > 0.f) ? __fdiv_rn(amax, kTop) : 1.0f;
+            const float rcp = (amax > 0.f) ? __fdiv_rn(kTop, amax) : 0.f;
+            uint2* qrow = reinterpret_cast<uint2*>((second ? p.Q1 : p.Q0) + r * N);
+#pragma unroll
+            for (int w = 0; w < VT; ++w)
+#pragma unroll
+                for (int i = 0; i < NV; ++i) {
+                    const int idx = w * 32 + lane + i * kNormThreads;
+                    if (idx < nvec) {
+                        const uint32_t w4[4] = {v[w][i].x, v[w][i].y, v[w][i].z, v[w][i].w};
+                        float t[8];
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            t[2 * k] = __fmul_rn(bf16_lo(w4[k]), rcp);
+                            t[2 * k + 1] = __fmul_rn(bf16_hi(w4[k]), rcp);
+                        }
+                        if constexpr (FMT == 1) {
+                            qrow[idx] = make_uint2(pack_e4m3x4(t[0], t[1], t[2], t[3]), pack_e4m3x4(t[4], t[5], t[6], t[7]));
+                        } else {
+                            int q[8];
+#pragma unroll
+                            for (int k = 0; k < 8; ++k) q[k] = __float2int_rn(t[k]);
+                            qrow[idx] = make_uint2(pack_s8x4_sat(q[0], q[1], q[2], q[3]), pack_s8x4_sat(q[4], q[5], q[6], q[7]));
+                        }
+                    }
+                }
+        }
     }
 }
 

@@ -21,7 +21,8 @@ def draw_cases(n, seed):
     extra = [dict(path=T, block_n=256, cta_pair=1, k_cluster=2), dict(path=T, block_n=128, cta_pair=1, k_cluster=2, stages=3),
              dict(path=T, block_n=192, cta_pair=1, k_cluster=4), dict(path=T, block_n=256, cta_pair=2, narrow_tail=2, stages=3),
              dict(path=T, block_n=128, cta_pair=1, narrow_tail=2), dict(path=T, block_n=256, cta_pair=2, k_cluster=2),
-             dict(path=T, block_n=128, cta_pair=2, k_cluster=2, stages=4), None]
+             dict(path=T, block_n=128, cta_pair=2, k_cluster=2, stages=4), dict(path=T, block_n=256, cta_pair=2, stream_k=3),
+             dict(path=T, block_n=128, cta_pair=1, stream_k=3, stages=3), None]
     pool = TILE_VARIANTS + SWAP_VARIANTS + STREAMK_VARIANTS + extra
     while len(cases) < n:
         ov = pool[int(rng.integers(0, len(pool)))]

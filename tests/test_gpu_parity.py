@@ -129,6 +129,35 @@ def test_stream_k_exact_integer_arithmetic(ov, max_ctas, M, N, K):
     assert np.array_equal(y, y2)
 
 
+@pytest.mark.parametrize("ov,max_ctas,M,N,K", [
+    (dict(path=T, block_n=256, cta_pair=2), 12, 640, 1280, 520),     # 15 pair tiles on 6 slots: 3 split first, 12 whole
+    (dict(path=T, block_n=256, cta_pair=2, stages=3), 12, 640, 1280, 4096),
+    (dict(path=T, block_n=256, cta_pair=1), 10, 640, 1280, 1096),    # 25 tiles on 10 slots: 5 split first
+    (dict(path=T, block_n=128, cta_pair=2), 12, 700, 520, 264),      # ragged rows and columns
+    (dict(path=T, block_n=192, cta_pair=1, stages=2), 9, 300, 776, 2048),
+    (dict(path=T, block_n=64, cta_pair=1), 37, 1000, 776, 520),
+    (dict(path=T, block_n=256, cta_pair=2), 0, 4096, 2304, 264),     # full grid: 144 pair tiles on 74 slots
+], ids=["pair256", "pair256-2kb-longk", "single256", "pair128-ragged", "single192-2kb", "single64", "pair256-fullgrid"])
+def test_stream_k_first_exact_integer_arithmetic(ov, max_ctas, M, N, K):
+    """The tiles left over after the full waves are cut into equal (tile, k-block) ranges and run first; the slot
+    that ends a split tile last adds the parked partials in fixed order while the next whole tile is in its main
+    loop.  Integer-valued data: bit-exact, the same bits in place and on a second run, also without residual."""
+    o = dict(ov, max_ctas=max_ctas, stream_k=3)
+    info = kx.kx_plan_query(M, N, K, ov=kx.make_override(**o))
+    assert info.stream_k == 2 and info.workspace_bytes > 0 and info.narrow_tiles == 0
+    X, W, b, R = ternary_case(M, N, K, seed=25)
+    ref = oracle.outproj(X, W, b, R)
+    y = run(X, W, b, R, o)
+    ok, msg = kt.gate_exact(y, ref)
+    assert ok, msg
+    assert np.array_equal(run(X, W, b, R.copy(), o, inplace=True), y)
+    assert np.array_equal(run(X, W, b, R, o), y)
+    ok, msg = kt.gate_exact(run(X, W, None, None, o), oracle.outproj(X, W))
+    assert ok, msg
+    with pytest.raises(kx.KxError):            # nothing is left over: no region to split
+        kx.kx_plan_query(512, 512, 512, ov=kx.make_override(path=T, block_n=256, cta_pair=1, max_ctas=4, stream_k=3))
+
+
 @pytest.mark.parametrize("ov,max_ctas,M,N", [
     (dict(path=T, block_n=256, cta_pair=2), 12, 640, 1280),    # 15 pair tiles on 6 slots: 12 wide + 6 narrow
     (dict(path=T, block_n=256, cta_pair=1), 10, 640, 1280),    # 25 tiles on 10 slots: 20 wide + 10 narrow
@@ -247,7 +276,7 @@ def test_l2_prefetch_depth_changes_no_bit(base, depth):
     assert np.array_equal(kt.from_dev(tY), y)
 
 
-@pytest.mark.parametrize("ov", STREAMK_VARIANTS[:2], ids=vid)
+@pytest.mark.parametrize("ov", STREAMK_VARIANTS[:2] + [dict(path=T, block_n=256, cta_pair=2, stream_k=3, max_ctas=8)], ids=vid)
 def test_stream_k_random_data_is_deterministic_and_within_gates(ov):
     wl = inputs.all_workloads()["cfg2"]
     d = inputs.make_inputs(wl, stress=True, M=1100, N=1304, K=4096)
