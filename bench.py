@@ -39,7 +39,9 @@ UNIT = "TFLOP/s"
 HEADLINE = "cfg2"
 # DRAM traffic per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum of one
 # ncu capture of that launch); None until captured.
-NCU_TRAFFIC_BYTES = {"cfg2": 154686976}
+NCU_TRAFFIC_BYTES = {"cfg2": 154900000, "cfg5": 3213600000, "sweep_M1_H4096": 33600000, "sweep_M1_H8192": 137700000,
+                     "sweep_M32_H2048": 8700000, "sweep_M32_H4096": 34100000, "sweep_M32_H8192": 139100000,
+                     "sweep_M512_H4096": 42100000}
 PATH_NAMES = {1: "tile", 2: "swap", 3: "gemv", 4: "skinny"}
 
 
@@ -380,7 +382,7 @@ def run_ours(args):
     # blocks start from the same power state; the step time is the median over the blocks.
     est = time_steps(torch, kx, wl, sets, 3, 0)
     blocks = 5
-    steps_b = int(max(args.steps, min(2000, math.ceil(0.03 / max(est, 1e-7)))))
+    steps_b = int(max(args.steps, min(2000, math.ceil(args.block_ms * 1e-3 / max(est, 1e-7)))))
     block_s = []
     with ClockSampler(local, period_s=0.002) as clk:
         for _ in range(blocks):
@@ -463,6 +465,7 @@ def run_ours(args):
                            "plan": {"path": PATH_NAMES.get(pi.path, str(pi.path)), "block_n": pi.block_n,
                                     "cta_pair": pi.cta_pair, "split_k": pi.split_k, "grid": pi.grid,
                                     "narrow_tiles": pi.narrow_tiles},
+                           "traffic": NCU_TRAFFIC_BYTES.get(name),
                            "operand_sets": len(ss)})
             # against roofline + launch floor (what a stream of such calls can reach at best)
             t_roof = max(w.flops / (peaks["bf16_tflops"] * 1e12), w.algorithmic_bytes / (peaks["hbm_gbs"] * 1e9))
@@ -991,6 +994,9 @@ def main():
     ap.add_argument("--sections", default="shapes,sustained,rmsnorm,swiglu,int8",
                     help="comma list of the extra sections to measure after the headline workload")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--block-ms", type=float, default=30.0,
+                    help="minimum length of each of the five timed blocks of the headline (0: exactly --steps calls per "
+                         "block, for profiler captures)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--workload", default=HEADLINE, help="headline workload name (default: the 4096^3 out-projection)")
     args = ap.parse_args()

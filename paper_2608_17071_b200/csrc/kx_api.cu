@@ -1498,38 +1498,13 @@ int launch_rowquant(const QuantParams& qp, bool norm, int fmt, cudaStream_t stre
                         : reinterpret_cast<const void*>(&kx_rowquant_kernel<NV, false, 1>))          \
                 : (norm ? reinterpret_cast<const void*>(&kx_rowquant_kernel<NV, true, 0>)            \
                         : reinterpret_cast<const void*>(&kx_rowquant_kernel<NV, false, 0>)))
-#define KX_QUANTW_FN(NV)                                                                             \
-    (fmt == 3 ? (norm ? reinterpret_cast<const void*>(&kx_rowquant_warp_kernel<NV, true, 3>)         \
-                      : reinterpret_cast<const void*>(&kx_rowquant_warp_kernel<NV, false, 3>))       \
-     : fmt == 2 ? (norm ? reinterpret_cast<const void*>(&kx_rowquant_warp_kernel<NV, true, 2>)       \
-                      : reinterpret_cast<const void*>(&kx_rowquant_warp_kernel<NV, false, 2>))       \
-     : fmt == 1 ? (norm ? reinterpret_cast<const void*>(&kx_rowquant_warp_kernel<NV, true, 1>)       \
-                        : reinterpret_cast<const void*>(&kx_rowquant_warp_kernel<NV, false, 1>))     \
-                : (norm ? reinterpret_cast<const void*>(&kx_rowquant_warp_kernel<NV, true, 0>)       \
-                        : reinterpret_cast<const void*>(&kx_rowquant_warp_kernel<NV, false, 0>)))
-    // Rows of up to 4096 elements: one warp per row (no block barriers; same bits).  KX_ROWQUANT_CTA=1 in the
-    // environment keeps the CTA-per-row kernel (for A/B timing).
-    static const bool force_cta = [] {
-        const char* e = std::getenv("KX_ROWQUANT_CTA");
-        return e && e[0] == '1';
-    }();
-    bool warp_form = false;
-    if (!force_cta && nvec <= 2 * kNormThreads && qp.M >= 64) {
-        fn = (nvec <= kNormThreads) ? KX_QUANTW_FN(1) : KX_QUANTW_FN(2);
-        warp_form = true;
-    } else if (nvec <= 1 * kNormThreads) { fn = KX_QUANT_FN(1); }
+    if (nvec <= 1 * kNormThreads) { fn = KX_QUANT_FN(1); }
     else if (nvec <= 2 * kNormThreads) { fn = KX_QUANT_FN(2); }
     else if (nvec <= 4 * kNormThreads) { fn = KX_QUANT_FN(4); per_sm = 6; }
     else if (nvec <= 8 * kNormThreads) { fn = KX_QUANT_FN(8); per_sm = 4; }
     else { fn = KX_QUANT_FN(kNormVecs); per_sm = 2; }
 #undef KX_QUANT_FN
-#undef KX_QUANTW_FN
-    if (warp_form) {
-        const long long ctas = (qp.M + 7) / 8;
-        cfg.gridDim = dim3(static_cast<unsigned>(std::min<long long>(ctas, static_cast<long long>(sm_count) * 8)), 1, 1);
-    } else {
-        cfg.gridDim = dim3(row_grid(qp.M, sm_count, per_sm), 1, 1);
-    }
+    cfg.gridDim = dim3(row_grid(qp.M, sm_count, per_sm), 1, 1);
     cfg.blockDim = dim3(kNormThreads, 1, 1);
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];

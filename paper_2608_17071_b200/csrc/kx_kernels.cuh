@@ -2090,182 +2090,4 @@ kx_rowquant_kernel(const QuantParams p) {
     }
 }
 
-// The same code books with one WARP per row (rows of up to 4096 elements): lane l plays the threads l, l + 32,
-// ..., l + 224 of the CTA-per-row kernel above, one after the other, and keeps their vectors in registers,
-// so there is no block barrier and no shared memory; a CTA of eight warps works on eight rows at once.
-// Every partial sum is formed in the order of the CTA-per-row kernel (per played thread over its vectors,
-// a shuffle tree per played warp, the played warps in order), so RMSNorm statistics, and with them every
-// code and scale, come out bit for bit the same.
-template <int NV, bool NORM, int FMT>
-__global__ void __launch_bounds__(kNormThreads)
-kx_rowquant_warp_kernel(const QuantParams p) {
-    constexpr float kTop = (FMT == 1) ? 448.0f : 127.0f;
-    constexpr int VT = kNormThreads / 32;                  // played warps per lane
-    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
-    const int N = p.N, nvec = N / 8;
-    pdl_wait_prior();
-    pdl_launch_dependents();
-    for (long long m = static_cast<long long>(blockIdx.x) * VT + wib; m < p.M; m += static_cast<long long>(gridDim.x) * VT) {
-        const bool second = m >= p.rows0;
-        const long long r = second ? m - p.rows0 : m;
-        const uint4* row = reinterpret_cast<const uint4*>((second ? p.A1 : p.A0) + r * N);
-        uint4 v[VT][NV];
-        float ssw[VT];
-#pragma unroll
-        for (int w = 0; w < VT; ++w) {
-            ssw[w] = 0.f;
-#pragma unroll
-            for (int i = 0; i < NV; ++i) {
-                const int idx = w * 32 + lane + i * kNormThreads;
-                if (idx < nvec) {
-                    v[w][i] = row[idx];
-                    if (NORM) {
-                        const uint32_t w4[4] = {v[w][i].x, v[w][i].y, v[w][i].z, v[w][i].w};
-#pragma unroll
-                        for (int k = 0; k < 4; ++k) {
-                            const float a = bf16_lo(w4[k]), b = bf16_hi(w4[k]);
-                            ssw[w] += a * a;
-                            ssw[w] += b * b;
-                        }
-                    }
-                }
-            }
-        }
-        if (NORM) {
-            float t = 0.f;
-#pragma unroll
-            for (int w = 0; w < VT; ++w) {
-                float s = ssw[w];
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-                t += s;
-            }
-            const float inv = rsqrtf(t / static_cast<float>(N) + p.eps);
-#pragma unroll
-            for (int w = 0; w < VT; ++w)
-#pragma unroll
-                for (int i = 0; i < NV; ++i) {
-                    const int idx = w * 32 + lane + i * kNormThreads;
-                    if (idx < nvec) {
-                        const uint4 g = __ldg(reinterpret_cast<const uint4*>(p.gamma) + idx);
-                        const uint32_t h4[4] = {v[w][i].x, v[w][i].y, v[w][i].z, v[w][i].w};
-                        const uint32_t g4[4] = {g.x, g.y, g.z, g.w};
-                        uint32_t o4[4];
-#pragma unroll
-                        for (int k = 0; k < 4; ++k)
-                            o4[k] = pack_bf16x2(bf16_lo(h4[k]) * inv * bf16_lo(g4[k]),
-                                                bf16_hi(h4[k]) * inv * bf16_hi(g4[k]));
-                        v[w][i] = make_uint4(o4[0], o4[1], o4[2], o4[3]);
-                    }
-                }
-        }
-        if constexpr (FMT == 2 || FMT == 3) {
-            uint8_t* const sfrow = p.SF0 + (r >> 7) * p.kchunks * 512 + (r & 31) * 16 + ((r & 127) >> 5) * 4;
-            const float d6 = __fmul_rn(6.0f, p.gs);
-#pragma unroll
-            for (int w = 0; w < VT; ++w)
-#pragma unroll
-                for (int i = 0; i < NV; ++i) {
-                    const int idx = w * 32 + lane + i * kNormThreads;
-                    const bool valid = idx < nvec;
-                    const uint32_t w4[4] = {valid ? v[w][i].x : 0u, valid ? v[w][i].y : 0u, valid ? v[w][i].z : 0u,
-                                            valid ? v[w][i].w : 0u};
-                    float z[8], bmax = 0.f;
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        z[2 * k] = bf16_lo(w4[k]);
-                        z[2 * k + 1] = bf16_hi(w4[k]);
-                        bmax = fmaxf(bmax, fmaxf(fabsf(z[2 * k]), fabsf(z[2 * k + 1])));
-                    }
-                    bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, 1));
-                    if constexpr (FMT == 2) {
-                        bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, 2));
-                        uint32_t e = 127u;
-                        if (valid) {
-                            const int field = static_cast<int>(__float_as_uint(bmax) >> 23);
-                            e = (bmax > 0.f) ? static_cast<uint32_t>(max(field - 8, 0)) : 127u;
-                            const float mult = __uint_as_float((254u - e) << 23);
-#pragma unroll
-                            for (int k = 0; k < 8; ++k) z[k] = __fmul_rn(z[k], mult);
-                            reinterpret_cast<uint2*>(p.Q0 + r * N)[idx] =
-                                make_uint2(pack_e4m3x4(z[0], z[1], z[2], z[3]), pack_e4m3x4(z[4], z[5], z[6], z[7]));
-                        }
-                        uint32_t word = e;
-                        word |= __shfl_down_sync(0xffffffffu, e, 4) << 8;
-                        word |= __shfl_down_sync(0xffffffffu, e, 8) << 16;
-                        word |= __shfl_down_sync(0xffffffffu, e, 12) << 24;
-                        if (valid && (lane & 15) == 0) *reinterpret_cast<uint32_t*>(sfrow + (idx >> 4) * 512) = word;
-                    } else {
-                        uint32_t sb = 0u;
-                        if (valid) {
-                            sb = pack_e4m3x4(__fdiv_rn(bmax, d6), 0.f, 0.f, 0.f) & 0xFFu;
-                            const float dq = __fmul_rn(e4m3_to_f32(sb), p.gs);
-                            const float rcp = (dq > 0.f) ? __fdiv_rn(1.0f, dq) : 0.f;
-#pragma unroll
-                            for (int k = 0; k < 8; ++k) z[k] = __fmul_rn(z[k], rcp);
-                            reinterpret_cast<uint32_t*>(reinterpret_cast<uint8_t*>(p.Q0) + r * (N / 2))[idx] =
-                                (dq > 0.f) ? pack_e2m1x8(z) : 0u;
-                        }
-                        uint32_t word = sb;
-                        word |= __shfl_down_sync(0xffffffffu, sb, 2) << 8;
-                        word |= __shfl_down_sync(0xffffffffu, sb, 4) << 16;
-                        word |= __shfl_down_sync(0xffffffffu, sb, 6) << 24;
-                        if (valid && (lane & 7) == 0) *reinterpret_cast<uint32_t*>(sfrow + (idx >> 3) * 512) = word;
-                    }
-                }
-            if (r == p.M - 1) {                              // rows up to the next multiple of 128: padding entries
-                const long long pad_rows = ((p.M + 127) & ~127ll) - p.M;
-                const int per_row = p.kchunks * 4;
-                for (long long t = lane; t < pad_rows * per_row; t += 32) {
-                    const long long rr = p.M + t / per_row;
-                    const int jj = static_cast<int>(t % per_row);
-                    p.SF0[((rr >> 7) * p.kchunks + (jj >> 2)) * 512 + (rr & 31) * 16 + ((rr & 127) >> 5) * 4 + (jj & 3)] =
-                        (FMT == 2) ? 127 : 0;
-                }
-            }
-        } else {
-            float amax = 0.f;
-#pragma unroll
-            for (int w = 0; w < VT; ++w)
-#pragma unroll
-                for (int i = 0; i < NV; ++i) {
-                    const int idx = w * 32 + lane + i * kNormThreads;
-                    if (idx < nvec) {
-                        const uint32_t w4[4] = {v[w][i].x, v[w][i].y, v[w][i].z, v[w][i].w};
-#pragma unroll
-                        for (int k = 0; k < 4; ++k) amax = fmaxf(amax, fmaxf(fabsf(bf16_lo(w4[k])), fabsf(bf16_hi(w4[k]))));
-                    }
-                }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
-            if (lane == 0) (second ? p.S1 : p.S0)[r] = (amax > 0.f) ? __fdiv_rn(amax, kTop) : 1.0f;
-            const float rcp = (amax > 0.f) ? __fdiv_rn(kTop, amax) : 0.f;
-            uint2* qrow = reinterpret_cast<uint2*>((second ? p.Q1 : p.Q0) + r * N);
-#pragma unroll
-            for (int w = 0; w < VT; ++w)
-#pragma unroll
-                for (int i = 0; i < NV; ++i) {
-                    const int idx = w * 32 + lane + i * kNormThreads;
-                    if (idx < nvec) {
-                        const uint32_t w4[4] = {v[w][i].x, v[w][i].y, v[w][i].z, v[w][i].w};
-                        float t[8];
-#pragma unroll
-                        for (int k = 0; k < 4; ++k) {
-                            t[2 * k] = __fmul_rn(bf16_lo(w4[k]), rcp);
-                            t[2 * k + 1] = __fmul_rn(bf16_hi(w4[k]), rcp);
-                        }
-                        if constexpr (FMT == 1) {
-                            qrow[idx] = make_uint2(pack_e4m3x4(t[0], t[1], t[2], t[3]), pack_e4m3x4(t[4], t[5], t[6], t[7]));
-                        } else {
-                            int q[8];
-#pragma unroll
-                            for (int k = 0; k < 8; ++k) q[k] = __float2int_rn(t[k]);
-                            qrow[idx] = make_uint2(pack_s8x4_sat(q[0], q[1], q[2], q[3]), pack_s8x4_sat(q[4], q[5], q[6], q[7]));
-                        }
-                    }
-                }
-        }
-    }
-}
-
 }  // namespace kx
