@@ -1962,6 +1962,9 @@ int outproj_residual_mx(const void* Xq, const void* SFX, const void* Wq, const v
     cfg.numAttrs = nattr;
     const uint16_t* bias_p = static_cast<const uint16_t*>(bias);
     void* args[] = {&tmA, &tmB, &tmSA, &tmY, &tmR, &tmSB, &bias_p, &p};
+#ifdef KX_TRACE
+    p.trace = g_kx_trace;
+#endif
     if (cudaLaunchKernelExC(&cfg, v->fn, args) != cudaSuccess) {
         cudaGetLastError();
         return KX_ERR_CUDA;
@@ -2071,6 +2074,9 @@ int kx_gate_up_swiglu_mxfp8(const void* Xq, const void* SFX, const void* Wgq, co
     // gate/up mode of the block-scaled kind: tmB = gate weights, tmB2 = up weights, tmR = scales of X, tmS = scales of
     // the gate rows followed by those of the up rows
     void* args[] = {&tmA, &tmG, &tmU, &tmZ, &tmSA, &tmSB, &bias_p, &p};
+#ifdef KX_TRACE
+    p.trace = g_kx_trace;
+#endif
     if (cudaLaunchKernelExC(&cfg, v->fn, args) != cudaSuccess) {
         cudaGetLastError();
         return KX_ERR_CUDA;
@@ -2171,8 +2177,8 @@ int kx_outproj_residual_nvfp4(const void* Xq, const void* SFX, const void* Wq, c
         overlaps(Y, yb, SFW, static_cast<size_t>(kx_nvfp4_scale_bytes(N, K))))
         return KX_ERR_OVERLAP;
     // tile width: smallest estimated time = waves x (k-blocks x time per k-block + exposed epilogue), with the
-    // measured 0.527 / 0.621 / 0.583 us per 128-byte k-block at 128 / 192 / 256 columns and 7 us per tile that
-    // the single-accumulator 256-column shape does not hide
+    // measured 0.43 / 0.52 / 0.70 us per 128-byte k-block at 128 / 192 / 256 columns (with the scale copies on the two
+    // scale warps) and 7 us per tile that the single-accumulator 256-column shape does not hide
     const MxVariant* v = nullptr;
     if (ov && ov->block_n) {
         for (const auto& c : kNvVariants)
@@ -2183,7 +2189,7 @@ int kx_outproj_residual_nvfp4(const void* Xq, const void* SFX, const void* Wq, c
         for (const auto& c : kNvVariants) {
             const long long tiles = ((M + 127) / 128) * ((N + c.bn - 1) / c.bn);
             const long long waves = (tiles + ctx->sm_count - 1) / ctx->sm_count;
-            const double per_kb = c.bn == 256 ? 0.583 : c.bn == 192 ? 0.621 : 0.527;
+            const double per_kb = c.bn == 256 ? 0.70 : c.bn == 192 ? 0.52 : 0.43;
             const double t = static_cast<double>(waves) * (static_cast<double>((K + 255) / 256) * per_kb + (c.bn == 256 ? 7.0 : 0.0));
             if (!v || t < best) { v = &c; best = t; }
         }
@@ -2227,7 +2233,7 @@ int kx_outproj_residual_nvfp4(const void* Xq, const void* SFX, const void* Wq, c
     cudaLaunchConfig_t cfg;
     std::memset(&cfg, 0, sizeof cfg);
     cfg.gridDim = dim3(static_cast<unsigned>(std::min<long long>(tiles, ctx->sm_count)), 1, 1);
-    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.blockDim = dim3(kThreadsScaled, 1, 1);
     cfg.dynamicSmemBytes = v->smem;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
@@ -2237,6 +2243,9 @@ int kx_outproj_residual_nvfp4(const void* Xq, const void* SFX, const void* Wq, c
     cfg.numAttrs = 1;
     const uint16_t* bias_p = static_cast<const uint16_t*>(bias);
     void* args[] = {&tmA, &tmB, &tmSA, &tmY, &tmR, &tmSB, &bias_p, &p};
+#ifdef KX_TRACE
+    p.trace = g_kx_trace;
+#endif
     if (cudaLaunchKernelExC(&cfg, v->fn, args) != cudaSuccess) {
         cudaGetLastError();
         return KX_ERR_CUDA;
@@ -2309,7 +2318,7 @@ int kx_gate_up_swiglu_nvfp4(const void* Xq, const void* SFX, const void* Wgq, co
     cudaLaunchConfig_t cfg;
     std::memset(&cfg, 0, sizeof cfg);
     cfg.gridDim = dim3(static_cast<unsigned>(std::min<long long>(tiles, ctx->sm_count)), 1, 1);
-    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.blockDim = dim3(kThreadsScaled, 1, 1);
     cfg.dynamicSmemBytes = v->smem;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
@@ -2319,6 +2328,9 @@ int kx_gate_up_swiglu_nvfp4(const void* Xq, const void* SFX, const void* Wgq, co
     cfg.numAttrs = 1;
     const uint16_t* bias_p = nullptr;
     void* args[] = {&tmA, &tmG, &tmU, &tmZ, &tmSA, &tmSB, &bias_p, &p};
+#ifdef KX_TRACE
+    p.trace = g_kx_trace;
+#endif
     if (cudaLaunchKernelExC(&cfg, v->fn, args) != cudaSuccess) {
         cudaGetLastError();
         return KX_ERR_CUDA;
@@ -2467,6 +2479,9 @@ int kx_outproj_residual_noalloc(const void* X, const void* W, const void* bias, 
     cfg.dynamicSmemBytes = v->smem;
     cfg.stream = stream;
     void* args[] = {&tmW, &tmX, &p};
+#ifdef KX_TRACE
+    p.trace = g_kx_trace;
+#endif
     if (cudaLaunchKernelExC(&cfg, v->fn, args) != cudaSuccess) {
         cudaGetLastError();
         return KX_ERR_CUDA;

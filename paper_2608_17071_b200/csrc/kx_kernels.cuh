@@ -53,6 +53,10 @@
 // records %globaltimer at up to 64 points; compiled out otherwise.
 #ifdef KX_TRACE
 #define KX_TRACE_DECL unsigned long long* trace;
+#define KX_TRACE_CLK(p, slot, idx)                                                          \
+    do {                                                                                     \
+        if ((p).trace && (idx) < 64) (p).trace[static_cast<size_t>(slot) * 64 + (idx)] = static_cast<unsigned long long>(clock64()); \
+    } while (0)
 #define KX_TRACE_POINT(p, slot, idx)                                                        \
     do {                                                                                     \
         if ((p).trace && (idx) < 64) (p).trace[static_cast<size_t>(slot) * 64 + (idx)] = globaltimer_ns(); \
@@ -60,11 +64,13 @@
 #else
 #define KX_TRACE_DECL
 #define KX_TRACE_POINT(p, slot, idx) do { } while (0)
+#define KX_TRACE_CLK(p, slot, idx) do { } while (0)
 #endif
 
 namespace kx {
 
 constexpr int kThreads = 192;         // warps 0-3 epilogue, 4 TMA producer, 5 MMA issuer
+constexpr int kThreadsScaled = 256;   // block-scaled kinds: two more warps whose lane 0 copies scale chunks to tensor memory
 constexpr int kBlockK = 64;           // BF16 elements per k-block = one 128-byte swizzle row
 constexpr int kABytes = 128 * 128;    // 128 operand rows x 128 bytes
 
@@ -186,7 +192,8 @@ struct TileCfg {
     static_assert(KBS == 1 || KBS == 2, "KBS");
     static constexpr int SLAB_BYTES = 32 * 128;             // 32 rows x 64 BF16 per warp per chunk
     static constexpr int EPI_BYTES = 4 * NB * SLAB_BYTES;
-    static constexpr int NUM_BARS = 2 * STAGES + 4 + 4 * NB + 1 + 5;   // + K-cluster exchange: 4 incoming, 1 "peer idle"
+    static constexpr int NUM_BARS = 2 * STAGES + 4 + 4 * NB + 1 + 5 + 2;   // + K-cluster exchange: 4 incoming, 1 "peer idle";
+                                                                           // + block-scaled kinds: 2 "scale columns ready"
     static constexpr int SFB_CHUNKS = (BN > 128) ? 2 : 1;
     // scale bytes per k-block: MX 1 = one chunk per operand row block, MX 2 (16-element blocks) = four
     static constexpr int SF_KB_BYTES = MX == 1 ? 512 * (1 + SFB_CHUNKS) : MX == 2 ? 2048 * (1 + SFB_CHUNKS) : 0;
@@ -195,7 +202,11 @@ struct TileCfg {
     // accumulator buffers in tensor memory: two, so that the epilogue of one tile overlaps the MMAs of the
     // next - except the 256-column block-scaled tile, where two would leave no room for the scale columns
     static constexpr int ACC_BUFS = (MX && BN > 192) ? 1 : 2;
-    static constexpr int TMEM_COLS = tmem_cols_for(ACC_BUFS * BN + (MX ? 48 : 0));
+    // scale columns behind the accumulators: four rotating sets of 12 (8-bit kind: one k-block's A + B chunks,
+    // copied by the MMA lane itself) or two alternating sets of 48 (4-bit kind: four K steps of 12, copied by the
+    // scale warps)
+    static constexpr int SF_SET_COLS = MX == 2 ? 48 : 12;
+    static constexpr int TMEM_COLS = tmem_cols_for(ACC_BUFS * BN + (MX == 2 ? 96 : MX == 1 ? 48 : 0));
     static_assert(SMEM_BYTES <= 232448, "shared memory");
     static constexpr int CHUNKS = BN / 64;                  // 64-column epilogue chunks per tile
     static constexpr int PART_FLOATS = 128 * BN;            // one CTA's FP32 partial of one tile
@@ -282,7 +293,7 @@ __device__ __forceinline__ uint32_t ld_acquire_gpu_u32(const unsigned int* p) {
 // its own (four per 128 rows and k-block, fetched as one box); the accumulators are multiplied by
 // alpha (the product of the two tensor scales) in the epilogue.  p.K counts bytes for this kind.
 template <int BN, int CTAS, int STAGES, int NB, int KIND = 0, int KBS = 1>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(KIND == 4 ? kThreadsScaled : kThreads, 1)
 kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmB2, const __grid_constant__ CUtensorMap tmY,
                const __grid_constant__ CUtensorMap tmR, const __grid_constant__ CUtensorMap tmS,
@@ -306,6 +317,7 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const uint32_t drain_bar = s_bar + 8u * (2 * STAGES + 4 + 4 * NB);
     auto xin_bar = [&](int w) { return s_bar + 8u * (2 * STAGES + 4 + 4 * NB + 1 + w); };   // K-cluster exchange
     const uint32_t peer_idle_bar = s_bar + 8u * (2 * STAGES + 4 + 4 * NB + 5);
+    auto sf_ready = [&](uint32_t set) { return s_bar + 8u * (2 * STAGES + 4 + 4 * NB + 6 + set); };   // block-scaled kinds
     volatile uint32_t* const s_tmem =
         reinterpret_cast<volatile uint32_t*>(gbase + (s_bar - base) + 8 * C::NUM_BARS);
     volatile uint32_t* const s_abort = s_tmem + 1;
@@ -389,6 +401,8 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             mbar_init(drain_bar, 1);
             for (int w = 0; w < 4; ++w) mbar_init(xin_bar(w), 1);
             mbar_init(peer_idle_bar, 1);
+            mbar_init(sf_ready(0), KIND == 4 ? 2 : 1);    // 4-bit kind: two scale warps share the copies of a k-block
+            mbar_init(sf_ready(1), KIND == 4 ? 2 : 1);
             fence_mbar_init();
         }
         __syncwarp();
@@ -530,6 +544,7 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             uint32_t full_bar = full(0), empty_bar0 = empty_base0, empty_bar1 = empty_base1, a_lo = a_lo0;
             bool ok = true;
             bool have = false;   // the current stage was already seen full by the previous k-block's early test
+            [[maybe_unused]] bool have_sf = false;   // block-scaled kinds: likewise for the scale columns of the current k-block
             while (ok && it.next(tile, kb0, kb1)) {
                 const uint32_t b = (C::ACC_BUFS == 2) ? (scount & 1u) : 0u;
                 const uint32_t aph = (C::ACC_BUFS == 2) ? ((scount >> 1) & 1u) : (scount & 1u);
@@ -541,24 +556,39 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 KX_TRACE_POINT(p, slot, (scount - 1) * 4 + 1);
                 const uint32_t d = tmem_base + b * BN;
                 if constexpr (KIND == 4) {
+                    // 4-bit block-scaled: the scale chunks of a k-block are copied to tensor memory by the scale warps
+                    // (two alternating column sets); this lane waits for the operands and for the columns, then
+                    // issues only the four K steps and the commit that releases the stage (and, two k-blocks
+                    // later, lets the scale warp overwrite the set)
                     int tm, col;
                     bool narrow;
                     decode_tile(tile, tm, col, narrow);
-                    const uint32_t b_off = static_cast<uint32_t>(col & 127) >> 5;
+                    const uint32_t b_off = static_cast<uint32_t>(col & 127) >> 5;   // first B row's 32-row group in its chunk
                     for (int kb = kb0; kb < kb1; ++kb) {
-                        if (!wt.wait(full_bar, ph, kWhereFull)) { ok = false; break; }
+                        const uint32_t set = mx_set & 1u, sfpar = (mx_set >> 1) & 1u;
+                        ++mx_set;
+                        if (!have && !wt.wait(full_bar, ph, kWhereFull)) { ok = false; break; }
+                        if (!have_sf && !wt.wait(sf_ready(set), sfpar, kWhereFull)) { ok = false; break; }
                         tc_fence_after();
-                        const uint32_t sf = s_sf + s * C::SF_STAGE;
-                        mma_kblock_nv<C::SFB_CHUNKS>(d, a_lo, a_lo + (kABytes >> 4), idesc_wide, (kb > kb0) ? 1u : 0u,
-                                                     (sf & 0x3FFFFu) >> 4, tmem_base + C::ACC_BUFS * BN, b_off);
+                        // the NEXT k-block's two barriers are tested now (non-blocking) and the answers read after
+                        // the commit below: in steady state both are long complete and cost no wait at all
+                        const bool wrap = (s + 1 == STAGES);
+                        const uint32_t next_full = wrap ? full(0) : full_bar + 8u;
+                        const uint32_t t_full = mbar_test_wait(next_full, wrap ? (ph ^ 1u) : ph);
+                        const uint32_t t_sf = mbar_test_wait(sf_ready(set ^ 1u), (mx_set >> 1) & 1u);
+                        const uint32_t cols = tmem_base + C::ACC_BUFS * BN + set * C::SF_SET_COLS;
+                        const uint32_t b_lo = a_lo + (kABytes >> 4);
+                        mma_kblock_nv_steps(d, a_lo, b_lo, idesc_wide, (kb > kb0) ? 1u : 0u, cols, b_off);
                         mma_commit<1>(empty_bar0);
-                        full_bar = (s + 1 == STAGES) ? full(0) : full_bar + 8u;
-                        if (s + 1 == STAGES) {
+                        have = t_full != 0u;
+                        have_sf = t_sf != 0u;
+                        full_bar = next_full;
+                        if (wrap) {
                             s = 0; ph ^= 1u;
-                            empty_bar0 = empty_base0; a_lo = a_lo0;
+                            empty_bar0 = empty_base0; empty_bar1 = empty_base1; a_lo = a_lo0;
                         } else {
                             ++s;
-                            empty_bar0 += 8u; a_lo += C::STAGE_BYTES >> 4;
+                            empty_bar0 += 8u; empty_bar1 += 8u; a_lo += C::STAGE_BYTES >> 4;
                         }
                     }
                 } else if constexpr (KIND == 3) {
@@ -638,6 +668,43 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             __syncwarp();
             cluster_arrive(); cluster_wait();
             cluster_arrive(); cluster_wait();
+        }
+    } else if (warp >= 6) {
+        // ------------------------------------------------------------ scale warps (block-scaled kinds only)
+        // 4-bit kind (a k-block needs 8 to 12 scale copies): warp 6 copies the chunks of K steps 0 and 1, warp 7 those
+        // of steps 2 and 3.  (The 8-bit kind needs 2 or 3 copies per k-block and keeps them in the MMA lane: moved
+        // here they cost one more barrier wait per k-block than they saved: 83 vs 76 us at 4096^3.)
+        if constexpr (KIND == 4) {
+            if (lane == 0) {
+                uint32_t s = 0, ph = 0, cnt = 0;          // cnt = k-blocks handled so far (all tiles of this CTA)
+                bool ok = true;
+                while (ok && it.next(tile, kb0, kb1)) {
+                    for (int kb = kb0; kb < kb1 && ok; ++kb) {
+                        // the scale chunks of this k-block have landed (same barrier as the operand tiles) ...
+                        [[maybe_unused]] const int tk = (warp == 6 && cnt >= 8u && cnt < 12u) ? static_cast<int>(cnt) - 8 : -1;
+                        if (tk >= 0) KX_TRACE_CLK(p, blockIdx.x, 32 + tk * 5 + 0);
+                        if (!wt.wait(full(s), ph, kWhereFull)) { ok = false; break; }
+                        if (tk >= 0) KX_TRACE_CLK(p, blockIdx.x, 32 + tk * 5 + 1);
+                        // ... and the MMAs that read this column set two k-blocks ago are done: the commit that
+                        // released their stage has completed that stage's `empty` phase
+                        if (cnt >= 2u) {
+                            const uint32_t c2 = cnt - 2u;
+                            if (!wt.wait(empty(c2 % STAGES), (c2 / STAGES) & 1u, kWhereEmpty)) { ok = false; break; }
+                        }
+                        tc_fence_after();
+                        if (tk >= 0) KX_TRACE_CLK(p, blockIdx.x, 32 + tk * 5 + 2);
+                        const uint32_t set = cnt & 1u;
+                        const uint32_t cols = tmem_base + C::ACC_BUFS * BN + set * C::SF_SET_COLS;
+                        const uint32_t sf = s_sf + s * C::SF_STAGE;
+                        sf_copy_nv<C::SFB_CHUNKS>((sf & 0x3FFFFu) >> 4, cols, warp == 6 ? 0u : 2u, warp == 6 ? 2u : 4u);
+                        if (tk >= 0) KX_TRACE_CLK(p, blockIdx.x, 32 + tk * 5 + 3);
+                        mma_commit<1>(sf_ready(set));
+                        if (tk >= 0) KX_TRACE_CLK(p, blockIdx.x, 32 + tk * 5 + 4);
+                        ++cnt;
+                        if (++s == STAGES) { s = 0; ph ^= 1u; }
+                    }
+                }
+            }
         }
     } else {
         // ------------------------------------------------------------ epilogue warps

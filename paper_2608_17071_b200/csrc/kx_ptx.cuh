@@ -89,6 +89,18 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 
+// non-blocking test of a phase (no suspension): the result can be read long after the instruction was issued
+__device__ __forceinline__ uint32_t mbar_test_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok;
+}
 // the same test with acquire semantics at cluster scope: pairs with arrivals made by other CTAs of the cluster
 __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
     uint32_t ok;
@@ -434,6 +446,7 @@ __device__ __forceinline__ void mma_kblock_mx(uint32_t d_tmem, uint32_t a_lo, ui
         else KX_MX_BODY("2", "");
     }
 }
+
 #undef KX_MX_BODY
 #undef KX_MX_STEP
 #undef KX_MX_CP
@@ -464,6 +477,37 @@ __device__ __forceinline__ void mma_kblock_nv(uint32_t d_tmem, uint32_t a_lo, ui
             asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(c + 8u),
                          "l"(sf_hi | (sf_lo + 256u + 32u * i))
                          : "memory");
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::mxf4nvf4.block_scale.scale_vec::4X [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
+            ::"r"(d_tmem), "l"(hi | (a_lo + 2u * i)), "l"(hi | (b_lo + 2u * i)), "r"(idesc),
+              "r"((acc_first != 0u || i > 0u) ? 1u : 0u), "r"(c), "r"(c + 4u + sfb_off)
+            : "memory");
+    }
+}
+// The two halves of the above for kernels in which another thread copies the scales: all copies of a k-block
+// (step i: A chunk and CHUNKS of B into columns cols + 12 i ...) and the four K = 64 steps alone.
+template <int CHUNKS>
+__device__ __forceinline__ void sf_copy_nv(uint32_t sf_lo, uint32_t cols, uint32_t step0, uint32_t step1) {
+    const uint64_t sf_hi = static_cast<uint64_t>((128u >> 4) | (1u << 14)) << 32;
+#pragma unroll
+    for (uint32_t i = step0; i < step1; ++i) {
+        const uint32_t c = cols + 12u * i;
+        asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(c), "l"(sf_hi | (sf_lo + 32u * i)) : "memory");
+        asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(c + 4u), "l"(sf_hi | (sf_lo + 128u + 32u * i))
+                     : "memory");
+        if constexpr (CHUNKS == 2)
+            asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(c + 8u),
+                         "l"(sf_hi | (sf_lo + 256u + 32u * i))
+                         : "memory");
+    }
+}
+__device__ __forceinline__ void mma_kblock_nv_steps(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc,
+                                                    uint32_t acc_first, uint32_t cols, uint32_t sfb_off) {
+    const uint64_t hi = static_cast<uint64_t>(kDescHiSw128) << 32;
+#pragma unroll
+    for (uint32_t i = 0; i < 4; ++i) {
+        const uint32_t c = cols + 12u * i;
         asm volatile(
             "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
             "tcgen05.mma.cta_group::1.kind::mxf4nvf4.block_scale.scale_vec::4X [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
