@@ -212,9 +212,9 @@ def sets_needed(wl, factor=2.0, cap=24):
     return int(max(2, min(cap, math.ceil(factor * L2_BYTES / per))))
 
 
-def bind_sets(kx, wl, sets):
-    """One pre-marshalled C-ABI call per operand set (on the current stream)."""
-    return [kx.bound_call(X, W, b, R, Y, plain=not wl.has_residual) for (X, W, b, R, Y) in sets]
+def bind_sets(kx, wl, sets, ov=None):
+    """One pre-marshalled C-ABI call per operand set (on the current stream); `ov`: an explicit plan."""
+    return [kx.bound_call(X, W, b, R, Y, plain=not wl.has_residual, ov=ov) for (X, W, b, R, Y) in sets]
 
 
 def call(kx, wl, s):
@@ -366,8 +366,9 @@ def run_ours(args):
     # ---- headline workload: seeded bits (rank r draws its own rows: seed offset by rank)
     bits = shard_inputs(inputs, wl, rank)
     nsets = sets_needed(wl)
-    sets = bind_sets(kx, wl, device_sets(torch, wl, nsets, bits))
-    info = kx.kx_plan_query(wl.M, wl.N, wl.K, wl.has_bias, wl.has_residual)
+    plan_ov = kx.make_override(**json.loads(args.plan)) if args.plan else None
+    sets = bind_sets(kx, wl, device_sets(torch, wl, nsets, bits), ov=plan_ov)
+    info = kx.kx_plan_query(wl.M, wl.N, wl.K, wl.has_bias, wl.has_residual, ov=plan_ov)
 
     def barrier():
         if dist is not None:
@@ -955,7 +956,8 @@ def run_ours(args):
                        "l2": f"rotating {nsets} operand sets ({nsets * wl.algorithmic_bytes / 1e6:.0f} MB) > L2",
                        "plan": {"path": PATH_NAMES.get(info.path, str(info.path)), "block_n": info.block_n,
                                 "cta_pair": info.cta_pair, "stages": info.stages, "grid": info.grid,
-                                "tiles": info.tiles, "smem_bytes": info.smem_bytes},
+                                "tiles": info.tiles, "smem_bytes": info.smem_bytes, "raster_group": info.raster_group,
+                                "override": json.loads(args.plan) if args.plan else None},
                        "sweep_shapes": len(sweep),
                        "parallelism": "none" if world == 1 else f"{world} independent row shards, W replicated, no collective"},
             "roofline": rl,
@@ -994,6 +996,9 @@ def main():
     ap.add_argument("--sections", default="shapes,sustained,rmsnorm,swiglu,int8",
                     help="comma list of the extra sections to measure after the headline workload")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--plan", default=None,
+                    help="JSON object of plan-override fields for the headline workload (tuning and profiling), "
+                         "e.g. '{\"raster_group\": 4}'")
     ap.add_argument("--block-ms", type=float, default=30.0,
                     help="minimum length of each of the five timed blocks of the headline (0: exactly --steps calls per "
                          "block, for profiler captures)")

@@ -16,8 +16,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "build")
 LIB = os.path.join(HERE, "libkx.so")
-SOURCES = ["kx_api.cu", "kx_gemv.cu"]
-HEADERS = ["kx_kernels.cuh", "kx_ptx.cuh", "kx_gemv.cuh", "kx_internal.h", "kx_plan_table.inc",
+SOURCES = ["kx_api.cu", "kx_gemv.cu", "kx_rowcode.cu"]
+HEADERS = ["kx_kernels.cuh", "kx_ptx.cuh", "kx_gemv.cuh", "kx_rowcode.cuh", "kx_internal.h", "kx_plan_table.inc",
            os.path.join("..", "..", "include", "kx.h")]
 
 NVCC_FLAGS = [

@@ -368,6 +368,19 @@ struct Plan {
 
 int ceil_div(long long a, long long b) { return static_cast<int>((a + b - 1) / b); }
 
+// Tile rows per raster group.  Tiles are visited group by group (all tile columns of one group of
+// tile rows, then the next group), so W comes from HBM once per group unless all of it stays in L2,
+// and the group's X panel (group x tile rows x one operand row) has to stay in L2 while the tile
+// columns go by.  Measured on long gate/up and QKV shapes: traffic and time are lowest with the
+// largest power-of-two group whose X panel is at most 36 MB; beyond that the panel itself is
+// evicted and both get worse.  W of at most 48 MB stays resident anyway: the group stays 8.
+int auto_raster_group(long long tile_rows, long long row_bytes, long long w_bytes) {
+    int g = 8;
+    if (w_bytes > (48ll << 20))
+        while (g < 64 && 2ll * g * tile_rows * row_bytes <= (36ll << 20)) g *= 2;
+    return g;
+}
+
 // Split-K factor of the small-M path: enough units to give every SM one (a single
 // wave: the reduction tail of a second wave costs more than it buys), each split at
 // least four k-blocks long, partials inside the workspace.
@@ -655,7 +668,11 @@ int make_plan_from(long long M, long long N, long long K, const kx_plan_override
         pl->tiles_m = ceil_div(M, 128 * ctas);
         pl->tiles_n = ceil_div(N, bn);
         pl->units = pl->tiles_m * pl->tiles_n;
-        pl->raster_group = (ov && ov->raster_group > 0) ? ov->raster_group : 8;
+        pl->raster_group = (ov && ov->raster_group > 0) ? ov->raster_group
+                                                        : auto_raster_group(128ll * ctas, 2ll * K, 2ll * N * K);
+#ifdef KX_TRACE
+        if (const char* e = std::getenv("KX_DEV_RASTER")) pl->raster_group = std::max(1, std::atoi(e));
+#endif
         pl->splits = 1;
         // Stream-K on the tail: when whole tiles would leave part of the last wave idle, the
         // full waves but one stay whole-tile work and the remaining (slots + r) tiles are cut
@@ -1390,6 +1407,16 @@ namespace {
 // Grid of the row kernels (one CTA works on one row at a time).  With fewer than 16 rows per
 // resident CTA a persistent grid ends ragged (4096 rows on 1184 CTAs: 3.46 rows each, so the
 // kernel lasts 4 row-times): launch one CTA per row instead and let the hardware balance them.
+// development build only: KX_DEV_OLD_ROWS=1 keeps the long-row kernels for every row length (A/B timing)
+bool dev_old_rows() {
+#ifdef KX_TRACE
+    const char* e = std::getenv("KX_DEV_OLD_ROWS");
+    return e && e[0] == '1';
+#else
+    return false;
+#endif
+}
+
 unsigned row_grid(long long M, int sm_count, int per_sm) {
     const long long resident = static_cast<long long>(sm_count) * per_sm;
     return static_cast<unsigned>(M <= 16 * resident ? M : resident);
@@ -1397,6 +1424,18 @@ unsigned row_grid(long long M, int sm_count, int per_sm) {
 
 int launch_rmsnorm(const void* H, const void* gamma, float eps, void* Z, long long M, long long N,
                    cudaStream_t stream, int sm_count) {
+    if (N <= kRowCodeMaxN && !dev_old_rows()) {      // the kernel for short rows (same bits as its fused forms)
+        QuantParams qp;
+        std::memset(&qp, 0, sizeof qp);
+        qp.A0 = static_cast<const uint16_t*>(H);
+        qp.gamma = static_cast<const uint16_t*>(gamma);
+        qp.Q0 = static_cast<int8_t*>(Z);
+        qp.rows0 = M;
+        qp.M = M;
+        qp.N = static_cast<int>(N);
+        qp.eps = eps;
+        return launch_rowcode(qp, true, 4, stream, sm_count);
+    }
     cudaLaunchConfig_t cfg;
     std::memset(&cfg, 0, sizeof cfg);
     // smallest instantiation whose threads cover a row; shorter rows leave room for more CTAs per SM
@@ -1484,6 +1523,7 @@ bool aligned4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3u) == 0
 // fmt: 0 = INT8 codes, 1 = FP8 E4M3 codes (one scale per row); 2 = FP8 E4M3 codes with one E8M0 scale per 32
 // elements; 3 = E2M1 codes with one E4M3 scale per 16 elements and a tensor scale
 int launch_rowquant(const QuantParams& qp, bool norm, int fmt, cudaStream_t stream, int sm_count) {
+    if (qp.N <= kRowCodeMaxN && !dev_old_rows()) return launch_rowcode(qp, norm, fmt, stream, sm_count);
     cudaLaunchConfig_t cfg;
     std::memset(&cfg, 0, sizeof cfg);
     const long long nvec = qp.N / 8;
@@ -1564,6 +1604,7 @@ int run_q8(int kind, const void* Xq, const float* sx, const void* Wq, const floa
     rc = make_plan_from(M, swiglu ? 2 * N : N, K, &ov, ctx->sm_count, &pl);
     if (rc != KX_OK) return rc;
     if (pl.kcluster > 1 || pl.stream_k) return KX_ERR_PLAN;
+    pl.raster_group = auto_raster_group(128ll * pl.ctas, K, (swiglu ? 2ll : 1ll) * N * K);   // one-byte operands
     CUtensorMap tmA, tmB, tmB2, tmY, tmR;
     if ((rc = get_tmap(Xq, M, K, 128, &tmA, 1)) != KX_OK) return rc;
     if (swiglu) {
@@ -1928,7 +1969,7 @@ int outproj_residual_mx(const void* Xq, const void* SFX, const void* Wq, const v
     p.tiles_m = static_cast<int>(tm);
     p.tiles_n = static_cast<int>(tiles_n);
     p.num_tiles = static_cast<int>(tiles);
-    p.raster_group = (ov && ov->raster_group > 0) ? ov->raster_group : 8;
+    p.raster_group = (ov && ov->raster_group > 0) ? ov->raster_group : auto_raster_group(128ll * ctas, K, N * K);
     p.has_bias = bias ? 1 : 0;
     p.has_r = R ? 1 : 0;
     p.kcluster = 1;
@@ -2049,7 +2090,7 @@ int kx_gate_up_swiglu_mxfp8(const void* Xq, const void* SFX, const void* Wgq, co
     p.tiles_m = static_cast<int>(tm);
     p.tiles_n = static_cast<int>(tiles_n);
     p.num_tiles = static_cast<int>(tiles);
-    p.raster_group = 8;
+    p.raster_group = auto_raster_group(128, K, 2 * I * K);
     p.swiglu = 1;
     p.kcluster = 1;
     p.sk_tile0 = p.num_tiles;
@@ -2217,7 +2258,7 @@ int kx_outproj_residual_nvfp4(const void* Xq, const void* SFX, const void* Wq, c
     p.tiles_m = static_cast<int>(tm);
     p.tiles_n = static_cast<int>(tiles_n);
     p.num_tiles = static_cast<int>(tiles);
-    p.raster_group = (ov && ov->raster_group > 0) ? ov->raster_group : 8;
+    p.raster_group = (ov && ov->raster_group > 0) ? ov->raster_group : auto_raster_group(128, K / 2, N * K / 2);
     p.has_bias = bias ? 1 : 0;
     p.has_r = R ? 1 : 0;
     p.kcluster = 1;
@@ -2302,7 +2343,7 @@ int kx_gate_up_swiglu_nvfp4(const void* Xq, const void* SFX, const void* Wgq, co
     p.tiles_m = static_cast<int>(tm);
     p.tiles_n = static_cast<int>(tiles_n);
     p.num_tiles = static_cast<int>(tiles);
-    p.raster_group = 8;
+    p.raster_group = auto_raster_group(128, K / 2, I * K);
     p.swiglu = 1;
     p.kcluster = 1;
     p.sk_tile0 = p.num_tiles;

@@ -31,4 +31,25 @@ int skinny_setup();
 bool skinny_variant_exists(int rows_per_cta);
 int launch_skinny(const GemvLaunch& a, cudaStream_t stream);
 
+// Arguments of the row kernels (RMSNorm, code books; see kx_kernels.cuh and kx_rowcode.cuh).
+struct QuantParams {
+    const uint16_t* A0;
+    const uint16_t* A1;
+    const uint16_t* gamma;
+    int8_t* Q0;
+    int8_t* Q1;
+    float* S0;
+    float* S1;
+    uint8_t* SF0;          // FMT 2: chunked scale bytes
+    long long rows0, M;
+    int N;
+    int kchunks;           // FMT 2: ceil(N / 128); FMT 3: ceil(N / 64)
+    float eps;
+    float gs;              // FMT 3: tensor scale (> 0)
+};
+// The kernels for rows of at most kRowCodeMaxN elements (kx_rowcode.cuh).  fmt: 0 INT8 / 1 E4M3 codes with one
+// scale per row, 2 / 3 the block-scaled 8-bit / 4-bit formats, 4 the BF16 RMSNorm itself (qp.Q0 = output).
+constexpr int kRowCodeMaxN = 8192;
+int launch_rowcode(const QuantParams& qp, bool norm, int fmt, cudaStream_t stream, int sm_count);
+
 }  // namespace kx

@@ -47,6 +47,7 @@
 // through to the common teardown (TMEM is always freed).  Hardware cluster barriers
 // are executed by every thread after its bounded role, so they cannot hang.
 #pragma once
+#include "kx_internal.h"
 #include "kx_ptx.cuh"
 
 // Optional timeline instrumentation (development builds only: -DKX_TRACE).  Each slot
@@ -1935,21 +1936,6 @@ kx_rmsnorm_kernel(const uint16_t* __restrict__ H, const uint16_t* __restrict__ g
 // codes e2m1(z * (1 / (value(s) gs))), every step in binary32; two codes per byte, even k in the low
 // nibble; scale bytes chunked as for FMT 2 but one chunk per (128 rows, 64 elements): byte
 // (row % 32) * 16 + (row % 128) / 32 * 4 + (k / 16) % 4; padding entries are set to 0.
-struct QuantParams {
-    const uint16_t* A0;
-    const uint16_t* A1;
-    const uint16_t* gamma;
-    int8_t* Q0;
-    int8_t* Q1;
-    float* S0;
-    float* S1;
-    uint8_t* SF0;          // FMT 2: chunked scale bytes
-    long long rows0, M;
-    int N;
-    int kchunks;           // FMT 2: ceil(N / 128); FMT 3: ceil(N / 64)
-    float eps;
-    float gs;              // FMT 3: tensor scale (> 0)
-};
 
 template <int NV, bool NORM, int FMT>
 __global__ void __launch_bounds__(kNormThreads)

@@ -158,6 +158,20 @@ def test_stream_k_first_exact_integer_arithmetic(ov, max_ctas, M, N, K):
         kx.kx_plan_query(512, 512, 512, ov=kx.make_override(path=T, block_n=256, cta_pair=1, max_ctas=4, stream_k=3))
 
 
+@pytest.mark.parametrize("group", [1, 3, 16, 64])
+@pytest.mark.parametrize("pair", [1, 2])
+def test_raster_group_exact_integer_arithmetic(group, pair):
+    """The raster group only reorders tiles: any group size, one larger than the number of tile rows and one that
+    does not divide it included, gives the exact result."""
+    M, N, K = 1100, 1304, 328
+    o = dict(path=T, block_n=128, cta_pair=pair, raster_group=group, max_ctas=8)
+    info = kx.kx_plan_query(M, N, K, ov=kx.make_override(**o))
+    assert info.raster_group == group
+    X, W, b, R = ternary_case(M, N, K, seed=27)
+    ok, msg = kt.gate_exact(run(X, W, b, R, o), oracle.outproj(X, W, b, R))
+    assert ok, msg
+
+
 @pytest.mark.parametrize("ov,max_ctas,M,N", [
     (dict(path=T, block_n=256, cta_pair=2), 12, 640, 1280),    # 15 pair tiles on 6 slots: 12 wide + 6 narrow
     (dict(path=T, block_n=256, cta_pair=1), 10, 640, 1280),    # 25 tiles on 10 slots: 20 wide + 10 narrow
