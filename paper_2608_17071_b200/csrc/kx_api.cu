@@ -224,7 +224,7 @@ int ensure_device(int dev, DeviceCtx** out) {
                      cudaSuccess &&
                  (!v.fn_push ||
                   cudaFuncSetAttribute(v.fn_push, cudaFuncAttributeMaxDynamicSharedMemorySize, v.smem_push) == cudaSuccess);
-        if (!ok || skinny_setup() != KX_OK) {
+        if (!ok || skinny_setup() != KX_OK || rowcode_setup() != KX_OK) {
             rc = KX_ERR_CUDA;
             break;
         }

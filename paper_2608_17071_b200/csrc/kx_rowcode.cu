@@ -5,14 +5,17 @@
 
 #include <algorithm>
 #include <mutex>
+#include <cstdlib>
 #include <cstring>
 
 namespace kx {
 namespace {
 
 template <int G, int NV>
-const void* rowcode_fn(bool norm, int fmt) {
-#define KX_RC(NORM, FMT) reinterpret_cast<const void*>(&kx_rowcode_kernel<G, NV, NORM, FMT>)
+const void* rowcode_fn(bool norm, int fmt, bool full) {
+#define KX_RC(NORM, FMT) \
+    (full ? reinterpret_cast<const void*>(&kx_rowcode_kernel<G, NV, NORM, FMT, true>) \
+          : reinterpret_cast<const void*>(&kx_rowcode_kernel<G, NV, NORM, FMT, false>))
     switch (fmt) {
         case 0: return norm ? KX_RC(true, 0) : KX_RC(false, 0);
         case 1: return norm ? KX_RC(true, 1) : KX_RC(false, 1);
@@ -24,22 +27,27 @@ const void* rowcode_fn(bool norm, int fmt) {
 #undef KX_RC
 }
 
+}  // namespace
+
+namespace {
+constexpr int ring_bytes(int nv) { return kRowDepth * nv * kRowThreads * 16; }
+
 // CTAs of one instantiation that fit on an SM (asked once per kernel; 1..8)
-int ctas_per_sm(const void* fn) {
+int ctas_per_sm(const void* fn, int smem) {
     static std::mutex mu;
-    static const void* fns[64];
-    static int counts[64];
+    static const void* fns[128];
+    static int counts[128];
     static int used = 0;
     std::lock_guard<std::mutex> lock(mu);
     for (int i = 0; i < used; ++i)
         if (fns[i] == fn) return counts[i];
     int n = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, fn, kRowThreads, 0) != cudaSuccess) {
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, fn, kRowThreads, smem) != cudaSuccess) {
         cudaGetLastError();
         n = 2;
     }
     n = std::max(1, std::min(n, 8));
-    if (used < 64) {
+    if (used < 128) {
         fns[used] = fn;
         counts[used] = n;
         ++used;
@@ -49,24 +57,58 @@ int ctas_per_sm(const void* fn) {
 
 }  // namespace
 
+int rowcode_setup() {
+    const bool tf[2] = {false, true};
+    for (bool norm : tf)
+        for (int fmt = 0; fmt <= 4; ++fmt) {
+            const void* fns[12] = {rowcode_fn<128, 1>(norm, fmt, false), rowcode_fn<128, 2>(norm, fmt, false),
+                                   rowcode_fn<128, 3>(norm, fmt, false), rowcode_fn<128, 4>(norm, fmt, false),
+                                   rowcode_fn<256, 3>(norm, fmt, false), rowcode_fn<256, 4>(norm, fmt, false),
+                                   rowcode_fn<128, 1>(norm, fmt, true),  rowcode_fn<128, 2>(norm, fmt, true),
+                                   rowcode_fn<128, 3>(norm, fmt, true),  rowcode_fn<128, 4>(norm, fmt, true),
+                                   rowcode_fn<256, 3>(norm, fmt, true),  rowcode_fn<256, 4>(norm, fmt, true)};
+            const int nvs[12] = {1, 2, 3, 4, 3, 4, 1, 2, 3, 4, 3, 4};
+            for (int i = 0; i < 12; ++i)
+                if (fns[i] &&
+                    cudaFuncSetAttribute(fns[i], cudaFuncAttributeMaxDynamicSharedMemorySize, ring_bytes(nvs[i])) != cudaSuccess) {
+                    cudaGetLastError();
+                    return KX_ERR_CUDA;
+                }
+        }
+    return KX_OK;
+}
+
 int launch_rowcode(const QuantParams& qp, bool norm, int fmt, cudaStream_t stream, int sm_count) {
     if (qp.N < 8 || qp.N > kRowCodeMaxN || (qp.N % 8) != 0 || qp.M < 1) return KX_ERR_PLAN;
     const int nvec = qp.N / 8;
     // the fewest vectors per thread that cover the row with 128 threads; 256 threads for the longest rows
     const void* fn = nullptr;
-    int rows_per_cta = 2;
-    if (nvec <= 128) fn = rowcode_fn<128, 1>(norm, fmt);
-    else if (nvec <= 256) fn = rowcode_fn<128, 2>(norm, fmt);
-    else if (nvec <= 512) fn = rowcode_fn<128, 4>(norm, fmt);
-    else { fn = rowcode_fn<256, 4>(norm, fmt); rows_per_cta = 1; }
+    int rows_per_cta = 2, nv = 4;
+    if (nvec <= 128) { fn = rowcode_fn<128, 1>(norm, fmt, nvec == 128); nv = 1; }
+    else if (nvec <= 256) { fn = rowcode_fn<128, 2>(norm, fmt, nvec == 256); nv = 2; }
+    else if (nvec <= 384) { fn = rowcode_fn<128, 3>(norm, fmt, nvec == 384); nv = 3; }
+    else if (nvec <= 512) fn = rowcode_fn<128, 4>(norm, fmt, nvec == 512);
+    else if (nvec <= 768) { fn = rowcode_fn<256, 3>(norm, fmt, nvec == 768); nv = 3; rows_per_cta = 1; }
+    else { fn = rowcode_fn<256, 4>(norm, fmt, nvec == 1024); rows_per_cta = 1; }
     if (!fn) return KX_ERR_PLAN;
+    const int smem = ring_bytes(nv);
     const long long steps = (qp.M + rows_per_cta - 1) / rows_per_cta;
-    // persistent over row steps: as many CTAs as fit on the device at once, fewer when there is less work
-    const long long resident = static_cast<long long>(ctas_per_sm(fn)) * sm_count;
+    // The fused kernels (normalisation + code book) are bound by instruction issue: one persistent CTA per slot,
+    // which pays for gamma and the first loads once.  The plain ones (normalisation only, code book only) are
+    // HBM-bound, and under a saturated memory system SMs progress at different rates: they get about 3.5 steps per
+    // CTA (at most 8 CTAs per slot), so that the hardware's block scheduler evens the SMs out.
+    const long long resident = static_cast<long long>(ctas_per_sm(fn, smem)) * sm_count;
+    long long mult = 1;
+    if (!norm || fmt == 4) mult = std::max(1ll, std::min(8ll, (2 * steps) / (7 * resident)));
+#ifdef KX_TRACE
+    if (const char* e = std::getenv("KX_DEV_ROW_GRID_MULT")) mult = std::max(1, std::atoi(e));
+#endif
+    const long long grid = std::min(steps, resident * mult);
     cudaLaunchConfig_t cfg;
     std::memset(&cfg, 0, sizeof cfg);
-    cfg.gridDim = dim3(static_cast<unsigned>(std::min(steps, resident)), 1, 1);
+    cfg.gridDim = dim3(static_cast<unsigned>(grid), 1, 1);
     cfg.blockDim = dim3(kRowThreads, 1, 1);
+    cfg.dynamicSmemBytes = static_cast<size_t>(smem);
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;

@@ -12,7 +12,7 @@
 //   * the FP32 arithmetic runs two elements per instruction (mul / fma .f32x2: the same IEEE results as
 //     the scalar forms), the maxima are taken on packed BF16 pairs (exact: a maximum rounds nothing),
 //     and gamma is widened to FP32 once per thread and kept in registers across rows;
-//   * a thread copies its own vectors of the next two row steps into a private slot of shared memory
+//   * a thread copies its own vectors of the next three row steps into private slots of shared memory
 //     with cp.async while it works on the current one, so the HBM latency of a row is not paid between
 //     its barriers; nothing but the issuing thread ever reads a slot, hence no barrier guards it.
 //
@@ -27,7 +27,8 @@
 namespace kx {
 
 constexpr int kRowThreads = 256;
-constexpr int kRowDepth = 2;          // row steps in flight per thread besides the current one
+constexpr int kRowDepth = 3;          // row steps a thread has in flight or in use: enough bytes on their way per SM
+                                      // to keep HBM busy when reads compete with the previous kernel's write-back
 
 // ---- two binary32 values in one 64-bit register (sm_100: one instruction for both lanes)
 __device__ __forceinline__ uint64_t f2_pack(float lo, float hi) {
@@ -81,16 +82,19 @@ __device__ __forceinline__ void group_barrier(int id, int threads) {
 // FMT 0 INT8 / 1 E4M3 codes with one FP32 scale per row; 2 E4M3 codes with one E8M0 scale per 32 elements;
 // 3 E2M1 codes with one E4M3 scale per 16 elements and a tensor scale; 4 BF16 (the RMSNorm itself, NORM only:
 // Q0 is then the BF16 output, which may be the input).  The formats' definitions are those of
-// kx_rowquant_kernel.  G * NV * 8 >= N.
-template <int G, int NV, bool NORM, int FMT>
-__global__ void __launch_bounds__(kRowThreads, 2)
+// kx_rowquant_kernel.  G * NV * 8 >= N; FULL: equal (every vector of every thread lies inside the row).
+template <int G, int NV, bool NORM, int FMT, bool FULL>
+#ifndef KX_ROW_MINB
+#define KX_ROW_MINB 2
+#endif
+__global__ void __launch_bounds__(kRowThreads, KX_ROW_MINB)
 kx_rowcode_kernel(const QuantParams p) {
     static_assert(G == 128 || G == 256, "threads per row");
     static_assert(FMT != 4 || NORM, "format 4 is the normalised row");
     constexpr int RPC = kRowThreads / G;                 // rows per CTA and step
     constexpr int WG = G / 32;                           // warps per row
     constexpr float kTop = (FMT == 1) ? 448.0f : 127.0f;
-    __shared__ uint4 s_ring[kRowDepth][NV][kRowThreads];
+    extern __shared__ uint4 s_ring[];                    // [kRowDepth][NV][kRowThreads]
     __shared__ __align__(16) float s_sum[2][RPC][WG];
     __shared__ __align__(16) float s_max[2][RPC][WG];
     const int tid = threadIdx.x, lane = tid & 31;
@@ -100,7 +104,8 @@ kx_rowcode_kernel(const QuantParams p) {
 
     bool valid[NV];
 #pragma unroll
-    for (int i = 0; i < NV; ++i) valid[i] = g + i * G < nvec;
+    for (int i = 0; i < NV; ++i) valid[i] = FULL || g + i * G < nvec;
+    const float inv_n = 1.0f / static_cast<float>(N);
     uint64_t gam[NORM ? NV : 1][4];                      // gamma, widened once (weights: not produced by the previous kernel)
     if constexpr (NORM) {
 #pragma unroll
@@ -128,7 +133,7 @@ kx_rowcode_kernel(const QuantParams p) {
             const uint4* src = src_of(m);
 #pragma unroll
             for (int i = 0; i < NV; ++i)
-                if (valid[i]) cp_async16(smem_u32(&s_ring[slot][i][tid]), src + g + i * G);
+                if (valid[i]) cp_async16(smem_u32(&s_ring[(slot * NV + i) * kRowThreads + tid]), src + g + i * G);
         }
         cp_async_commit();
     };
@@ -144,7 +149,11 @@ kx_rowcode_kernel(const QuantParams p) {
         cp_async_wait<kRowDepth - 1>();
         uint4 v[NV];
 #pragma unroll
-        for (int i = 0; i < NV; ++i) v[i] = (valid[i] && live) ? s_ring[slot][i][tid] : make_uint4(0u, 0u, 0u, 0u);
+        for (int i = 0; i < NV; ++i) {
+            // a group without a row (last step of an odd row count) computes on whatever the slot holds and stores nothing
+            if (FULL) v[i] = s_ring[(slot * NV + i) * kRowThreads + tid];
+            else v[i] = (valid[i] && live) ? s_ring[(slot * NV + i) * kRowThreads + tid] : make_uint4(0u, 0u, 0u, 0u);
+        }
 
         if constexpr (NORM) {
             uint64_t h2[NV][4];
@@ -168,9 +177,15 @@ kx_rowcode_kernel(const QuantParams p) {
             if (lane == 0) s_sum[par][gi][wg] = ss;
             group_barrier(1 + gi, G);
             float t = 0.f;
+            {
+                float part[WG];
 #pragma unroll
-            for (int w = 0; w < WG; ++w) t += s_sum[par][gi][w];
-            const float inv = rsqrtf(t / static_cast<float>(N) + p.eps);
+                for (int w = 0; w < WG; w += 4)
+                    *reinterpret_cast<float4*>(&part[w]) = *reinterpret_cast<const float4*>(&s_sum[par][gi][w]);
+#pragma unroll
+                for (int w = 0; w < WG; ++w) t += part[w];
+            }
+            const float inv = rsqrtf(t * inv_n + p.eps);
             const uint64_t inv2 = f2_pack(inv, inv);
 #pragma unroll
             for (int i = 0; i < NV; ++i) {
@@ -214,13 +229,9 @@ kx_rowcode_kernel(const QuantParams p) {
                     for (int k = 0; k < 4; ++k) f2_unpack(f2_mul(f2_from_bf16x2(w4[k]), mult2), z[2 * k], z[2 * k + 1]);
                     qrow[idx] = make_uint2(pack_e4m3x4(z[0], z[1], z[2], z[3]), pack_e4m3x4(z[4], z[5], z[6], z[7]));
                 }
-                // the scale bytes of four neighbouring blocks (16 lanes) are adjacent in a chunk: one 32-bit store,
-                // which also writes the padding entries of a last chunk that the row fills only in part
-                uint32_t word = e;
-                word |= __shfl_down_sync(0xffffffffu, e, 4) << 8;
-                word |= __shfl_down_sync(0xffffffffu, e, 8) << 16;
-                word |= __shfl_down_sync(0xffffffffu, e, 12) << 24;
-                if (ok && (g & 15) == 0) *reinterpret_cast<uint32_t*>(sfrow + (idx >> 4) * 512) = word;
+                // one byte per block, stored by the block's first lane; lanes past the row end but inside the row's
+                // last chunk write that chunk's padding entries
+                if (live && (g & 3) == 0 && (idx >> 4) < p.kchunks) sfrow[(idx >> 4) * 512 + ((idx >> 2) & 3)] = static_cast<uint8_t>(e);
             }
             if (live && r == p.M - 1) {                      // rows up to the next multiple of 128
                 const long long pad_rows = ((p.M + 127) & ~127ll) - p.M;
@@ -257,12 +268,8 @@ kx_rowcode_kernel(const QuantParams p) {
                     for (int k = 0; k < 4; ++k) f2_unpack(f2_mul(f2_from_bf16x2(w4[k]), rcp2), z[2 * k], z[2 * k + 1]);
                     qrow[idx] = (dq > 0.f) ? pack_e2m1x8(z) : 0u;
                 }
-                // four neighbouring blocks (8 lanes) -> one 32-bit store of their scale bytes, padding included
-                uint32_t word = sb;
-                word |= __shfl_down_sync(0xffffffffu, sb, 2) << 8;
-                word |= __shfl_down_sync(0xffffffffu, sb, 4) << 16;
-                word |= __shfl_down_sync(0xffffffffu, sb, 6) << 24;
-                if (ok && (g & 7) == 0) *reinterpret_cast<uint32_t*>(sfrow + (idx >> 3) * 512) = word;
+                // one byte per block, stored by the block's first lane, the padding entries of the row's last chunk included
+                if (live && (g & 1) == 0 && (idx >> 3) < p.kchunks) sfrow[(idx >> 3) * 512 + ((idx >> 1) & 3)] = static_cast<uint8_t>(sb);
             }
             if (live && r == p.M - 1) {
                 const long long pad_rows = ((p.M + 127) & ~127ll) - p.M;
@@ -288,9 +295,17 @@ kx_rowcode_kernel(const QuantParams p) {
             if (lane == 0) s_max[par][gi][wg] = fmaxf(bf16_lo(mx), bf16_hi(mx));
             group_barrier(1 + gi, G);
             float a = 0.f;
+            {
+                float part[WG];
 #pragma unroll
-            for (int w = 0; w < WG; ++w) a = fmaxf(a, s_max[par][gi][w]);
-            if (g == 0 && live) (second ? p.S1 : p.S0)[r] = (a > 0.f) ? __fdiv_rn(a, kTop) : 1.0f;
+                for (int w = 0; w < WG; w += 4)
+                    *reinterpret_cast<float4*>(&part[w]) = *reinterpret_cast<const float4*>(&s_max[par][gi][w]);
+#pragma unroll
+                for (int w = 0; w < WG; ++w) a = fmaxf(a, part[w]);
+            }
+            if (wg == 0) {                                   // one warp of the group pays for the scale's division
+                if (g == 0 && live) (second ? p.S1 : p.S0)[r] = (a > 0.f) ? __fdiv_rn(a, kTop) : 1.0f;
+            }
             const float rcp = (a > 0.f) ? __fdiv_rn(kTop, a) : 0.f;
             const uint64_t rcp2 = f2_pack(rcp, rcp);
             if (live) {

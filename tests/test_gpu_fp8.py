@@ -41,7 +41,7 @@ def gpu_quantize(A):
     return host8(Q), S.cpu().numpy()
 
 
-@pytest.mark.parametrize("rows,cols", [(1, 16), (5, 48), (300, 2064), (129, 4096), (3, 32768), (700, 1024)])
+@pytest.mark.parametrize("rows,cols", [(1, 16), (5, 48), (300, 2064), (129, 4096), (3, 32768), (700, 1024), (7, 3072), (5, 2560), (9, 7168), (5, 6144), (9000, 256)])
 def test_fp8_code_book_bit_exact(rows, cols):
     A = inputs.normal_bf16(700 + cols, "X", (rows, cols), 2.5)
     if rows > 2:
@@ -85,7 +85,7 @@ def test_fp8_gate_up_and_rmsnorm_code_books():
     for Q, S, W in ((Qg, Sg, Wg), (Qu, Su, Wu)):
         Qr, Sr = oracle.quantize_rows_fp8(W)
         assert np.array_equal(host8(Q), Qr) and np.array_equal(S.cpu().numpy(), Sr)
-    for (M, N) in [(130, 4096), (1000, 5120), (9, 32768)]:
+    for (M, N) in [(130, 4096), (1000, 5120), (9, 32768), (7, 3072), (3, 8192), (9, 7168), (9000, 256)]:
         H = inputs.normal_bf16(720 + N, "R", (M, N), 1.3)
         g = inputs.normal_bf16(720 + N, "bias", (N,), 1.0)
         Z = kt.nan_filled(M, N)

@@ -33,7 +33,7 @@ def gpu_quantize(A):
     return Q.cpu().numpy(), S.cpu().numpy()
 
 
-@pytest.mark.parametrize("rows,cols", [(1, 16), (5, 48), (300, 2064), (129, 4096), (40, 8192), (3, 32768), (700, 1024)])
+@pytest.mark.parametrize("rows,cols", [(1, 16), (5, 48), (300, 2064), (129, 4096), (40, 8192), (3, 32768), (700, 1024), (7, 3072), (5, 2560), (9, 7168), (5, 6144), (9000, 256)])
 def test_quantize_rows_bit_exact(rows, cols):
     A = inputs.normal_bf16(500 + cols, "X", (rows, cols), 2.5)
     if rows > 2:
@@ -72,7 +72,7 @@ def test_quantize_gate_and_up_in_one_launch():
         assert np.array_equal(Q.cpu().numpy(), Qr) and np.array_equal(S.cpu().numpy(), Sr)
 
 
-@pytest.mark.parametrize("M,N", [(3, 272), (130, 4096), (9, 32768), (1000, 5120), (2500, 2048)])
+@pytest.mark.parametrize("M,N", [(3, 272), (130, 4096), (9, 32768), (1000, 5120), (2500, 2048), (7, 3072), (3, 8192), (5, 6144), (9, 7168), (5, 2560), (9000, 256)])
 def test_rmsnorm_quantize(M, N):
     """The fused kernel quantises exactly the BF16 values kx_rmsnorm writes: the code book of
     that (device-computed) z, taken by the oracle, must be reproduced bit for bit; z itself is

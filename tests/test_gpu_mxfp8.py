@@ -60,7 +60,7 @@ def test_scale_bytes():
     assert kx.kx_mx_scale_bytes(-1, 64) < 0
 
 
-@pytest.mark.parametrize("rows,cols", [(1, 32), (5, 96), (300, 2080), (129, 4096), (3, 32768), (700, 1024), (128, 128)])
+@pytest.mark.parametrize("rows,cols", [(1, 32), (5, 96), (300, 2080), (129, 4096), (3, 32768), (700, 1024), (128, 128), (7, 3072), (5, 2560), (9, 7168), (5, 6144), (9000, 256)])
 def test_mx_code_book_bit_exact(rows, cols):
     A = inputs.normal_bf16(900 + cols, "X", (rows, cols), 2.5)
     f = inputs.bf16_bits_to_f32(A)
@@ -78,7 +78,7 @@ def test_mx_code_book_bit_exact(rows, cols):
     assert np.array_equal(SF, chunked(Er, cols))
 
 
-@pytest.mark.parametrize("M,N", [(130, 4096), (1000, 5120), (9, 32768), (300, 1056), (5, 32)])
+@pytest.mark.parametrize("M,N", [(130, 4096), (1000, 5120), (9, 32768), (300, 1056), (5, 32), (7, 3072), (3, 8192), (5, 6144), (9, 7168), (5, 2560), (9000, 256)])
 def test_mx_rmsnorm_code_book(M, N):
     """Fused RMSNorm + code book = code book of the device's own BF16 RMSNorm output, bit for bit."""
     H = inputs.normal_bf16(950 + N, "R", (M, N), 1.3)

@@ -47,7 +47,7 @@ def test_scale_bytes():
     assert kx.kx_nvfp4_scale_bytes(129, 80) == 4 * 512 and kx.kx_nvfp4_scale_bytes(-1, 64) < 0
 
 
-@pytest.mark.parametrize("rows,cols", [(1, 16), (5, 80), (300, 2064), (129, 4096), (3, 32768), (700, 1024)])
+@pytest.mark.parametrize("rows,cols", [(1, 16), (5, 80), (300, 2064), (129, 4096), (3, 32768), (700, 1024), (7, 3072), (5, 2560), (9, 7168), (5, 6144), (9000, 256)])
 def test_nvfp4_code_book_bit_exact(rows, cols):
     A = inputs.normal_bf16(1000 + cols, "X", (rows, cols), 2.5)
     f = inputs.bf16_bits_to_f32(A)
@@ -274,7 +274,7 @@ def test_nvfp4_projection_full_sizes_sampled_rows(M, N, K):
 
 
 # ------------------------------------------------------------------ RMSNorm-fused code book, gate/up + SwiGLU
-@pytest.mark.parametrize("M,N", [(130, 4096), (1000, 5120), (9, 32768), (300, 1040)])
+@pytest.mark.parametrize("M,N", [(130, 4096), (1000, 5120), (9, 32768), (300, 1040), (7, 3072), (3, 8192), (5, 6144), (9, 7168), (5, 2560), (9000, 256)])
 def test_nvfp4_rmsnorm_code_book(M, N):
     """Fused RMSNorm + code book = code book of the device's own BF16 RMSNorm output, bit for bit."""
     H = inputs.normal_bf16(1150 + N, "R", (M, N), 1.3)

@@ -24,7 +24,7 @@ def gate_norm(z_bits, ref):
     assert rate <= 0.01, rate
 
 
-@pytest.mark.parametrize("M,N", [(1, 8), (3, 264), (130, 4096), (17, 32768), (1000, 5120), (2500, 2048)])
+@pytest.mark.parametrize("M,N", [(1, 8), (3, 264), (130, 4096), (17, 32768), (1000, 5120), (2500, 2048), (7, 3072), (3, 8192), (5, 6144), (9, 7168), (5, 2560), (9000, 256)])
 @pytest.mark.parametrize("eps", [1e-6, 0.0])
 def test_rmsnorm_matches_oracle(M, N, eps):
     H = inputs.normal_bf16(200 + N, "R", (M, N), 1.0)
