@@ -88,7 +88,10 @@ enum { KX_PATH_AUTO = 0, KX_PATH_TILE = 1, KX_PATH_SWAP = 2, KX_PATH_GEMV = 3, K
  *                 left over after the full waves are split that way and run FIRST, the rest whole
  *                 (the summing of a split tile then overlaps the next tile's main loop)
  *   narrow_tail   tile path: 0 auto, 1 off, 2 = run the tiles left over after the full
- *                 waves as half-width tiles when they then fit in one extra wave
+ *                 waves as half-width tiles when they then fit in one extra wave, 3 = run each
+ *                 of them as two K halves on two CTAs (CTA pairs) at full width instead; the two
+ *                 swap, through the FP32 workspace, the 64-column chunks the other one finishes
+ *                 (needs at most half as many leftover tiles as CTAs / pairs, else KX_ERR_PLAN)
  *   cluster_reduce  swap path: 0 auto, 1 = sum the K splits through the FP32 workspace
  *                 (last CTA to arrive reduces), 2 = the 2..8 splits of a tile form a
  *                 thread-block cluster and the CTA that finishes a row reads the partials of

@@ -355,6 +355,7 @@ struct Plan {
     int cluster_reduce = 0; // swap path: the splits of a tile form a cluster and reduce through DSMEM
     int narrow_tile0 = 0;   // first half-width tail tile id (== units: none)
     int wide_units = 0;     // number of full-width tile positions
+    int khalf_tiles = 0;    // full-width tiles at the end that run as two K halves on two slots (0: none)
     int raster_group = 8;
     int grid = 0, units = 0;
     int tiles_m = 0, tiles_n = 0;   // tile path: tile grid; swap path: m_tiles / n_tiles
@@ -718,8 +719,32 @@ int make_plan_from(long long M, long long N, long long K, const kx_plan_override
         // workspace; 4096 x 4096 on 74 pair slots becomes 3 + 1/2 wave-times instead of 4.
         pl->wide_units = pl->units;
         pl->narrow_tile0 = pl->units;
-        int nt = ov ? ov->narrow_tail : 0;                    // 0 auto, 1 off, 2 on
+        int nt = ov ? ov->narrow_tail : 0;                    // 0 auto, 1 off, 2 on, 3 K halves instead
         const int kcl = (ov && ov->k_cluster) ? ov->k_cluster : auto_kc;
+        // Automatic choice between the two tails (measured, 4096-wide shapes on 74 pair slots): from 64 k-blocks
+        // on the K halves win (K = 4096: 115.5 vs 118.8 us sustained, 100.2 vs 103.3 us in bursts; K = 8192: 222 vs
+        // 242 us), below that their longer exposed epilogue costs more than the narrow MMAs (K = 3072: 94.9 vs 91.7).
+        if (nt == 0 && !pl->stream_k && kcl <= 1 && rem > 0 && full_waves >= 1 && 2 * rem <= slots && nkb >= 64 &&
+            bn >= 128 && static_cast<size_t>(2 * rem) * ctas * 128 * bn * sizeof(float) <= kWorkspaceBytes &&
+            static_cast<long long>(full_waves * slots + 2 * rem) * ctas * 4 <= kMaxCounters)
+            nt = 3;
+        if (nt == 3) {
+            // K-halves tail: each tile left over after the full waves runs as two K halves on two slots at
+            // full tile width (the half-width tiles above pay for their narrower MMAs with more operand
+            // bytes per flop); the two slots swap, through the workspace, the chunks the other one finishes.
+            const size_t ws2 = static_cast<size_t>(2 * rem) * ctas * 128 * bn * sizeof(float);
+            if (pl->stream_k || kcl > 1 || rem == 0 || full_waves < 1 || 2 * rem > slots || nkb < 2 || bn < 128)
+                return KX_ERR_PLAN;
+            if (ws2 > kWorkspaceBytes || static_cast<long long>(full_waves * slots + 2 * rem) * ctas * 4 > kMaxCounters)
+                return KX_ERR_WORKSPACE;
+            pl->khalf_tiles = rem;
+            pl->units = full_waves * slots + 2 * rem;
+            pl->narrow_tile0 = pl->units;
+            pl->sk_tile0 = pl->units;
+            pl->grid = slots * ctas;
+            pl->ws_bytes = ws2;
+            nt = 1;
+        }
         const bool nt_ok = !pl->stream_k && kcl <= 1 && (bn == 256 || bn == 128) && rem > 0 && full_waves >= 1 &&
                            2 * rem <= slots;
         if (nt == 0) nt = nt_ok ? 2 : 1;
@@ -976,6 +1001,7 @@ int run(const void* X, const void* W, const void* bias, const void* R, void* Y, 
         p.sk_tile0 = pl.sk_tile0;
         p.sk_first_tiles = pl.sk_first_tiles;
         p.narrow_tile0 = pl.narrow_tile0;
+        p.khalf_tiles = pl.khalf_tiles;
         p.spin_limit_ns = spin_ns;
         p.status = ctx->status;
         p.ws = ctx->ws;
@@ -1596,6 +1622,7 @@ int run_q8(int kind, const void* Xq, const float* sx, const void* Wq, const floa
     ov.path = KX_PATH_TILE;
     ov.stream_k = 1;          // whole tiles only: unscaled partial accumulators are never added across CTAs
     ov.no_table = 1;
+    ov.narrow_tail = 2;       // half-width tail where it fits (never K halves: they add unscaled partial accumulators too)
     if (swiglu) {
         ov.block_n = 256;     // 128 gate + 128 up accumulator columns = 128 output columns per tile
         ov.narrow_tail = 1;

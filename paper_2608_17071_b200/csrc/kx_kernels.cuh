@@ -173,6 +173,12 @@ struct TileParams {
     int narrow_tile0;             // tile ids >= narrow_tile0 are half-width tiles: id = narrow_tile0 + 2 * j + half
                                   // covers columns [half * BN/2, +BN/2) of full-width position narrow_tile0 + j
                                   // (== num_tiles: none; never combined with stream-K)
+    int khalf_tiles;              // > 0: the last 2 * khalf_tiles tile ids are K halves of khalf_tiles full-width tiles:
+                                  // id = num_tiles - 2 * khalf_tiles + 2 * j + h covers k-blocks [h nkb / 2, (h + 1) nkb / 2)
+                                  // of full-width position num_tiles - 2 * khalf_tiles + j.  The two slots that hold the
+                                  // halves of a tile swap, through the workspace, the 64-column chunks the other one
+                                  // finishes (chunk c goes to half c % 2) and each writes its own chunks of Y
+                                  // (never combined with stream-K, half-width tiles or a K cluster)
     unsigned long long spin_limit_ns;
     unsigned int* status;
     float* ws;                    // stream-K partials: [slot][head|tail][cta rank][chunk][warp][16-byte group][lane]
@@ -229,7 +235,7 @@ __device__ __forceinline__ int sk_slot_of(long long U, int G, long long u) {
 
 // The work of one slot (a CTA or a CTA pair) as a sequence of segments (tile, kb0, kb1).
 struct SegIter {
-    int nkb, t, t_end, tstride, kc_kb0, kc_kb1, sk_base;
+    int nkb, t, t_end, tstride, kc_kb0, kc_kb1, sk_base, kh0;
     bool sk_first;
     long long u, u1;
     // krank / kcluster: position of this CTA in its K cluster (0 / 1 when there is none)
@@ -242,6 +248,7 @@ struct SegIter {
         t = (sk_first ? p.sk_first_tiles : 0) + slot;              // whole tiles: [.., t_end), round-robin
         t_end = sk_first ? p.num_tiles : p.sk_tile0;
         tstride = slots;
+        kh0 = p.num_tiles - 2 * p.khalf_tiles;                     // first K-half id (== num_tiles: none)
         kc_kb0 = static_cast<int>((static_cast<long long>(krank) * nkb_) / kcluster);
         kc_kb1 = static_cast<int>((static_cast<long long>(krank + 1) * nkb_) / kcluster);
         const long long U = static_cast<long long>(sk_tiles) * nkb_;
@@ -253,6 +260,11 @@ struct SegIter {
         tile = t;
         kb0 = kc_kb0;
         kb1 = kc_kb1;
+        if (t >= kh0) {                                            // one K half of a full-width tile
+            const int h = (t - kh0) & 1;
+            kb0 = h ? nkb / 2 : 0;
+            kb1 = h ? nkb : nkb / 2;
+        }
         t += tstride;
         return true;
     }
@@ -348,6 +360,8 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             pos = p.narrow_tile0 + (j >> 1);
             half = j & 1;
         }
+        const int kh0 = p.num_tiles - 2 * p.khalf_tiles;
+        if (p.khalf_tiles > 0 && t >= kh0) pos = kh0 + ((t - kh0) >> 1);
         int tn;
         tile_coords(pos, p.tiles_m, p.tiles_n, p.raster_group, tm, tn);
         col = tn * BN + half * (BN / 2);
@@ -721,10 +735,12 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         auto slab4 = [&](float* part, int c) {
             return reinterpret_cast<float4*>(part) + (static_cast<size_t>(c) * 4 + q) * 16 * 32 + lane;
         };
-        enum { kWhole = 0, kFast = 1, kWriter = 2, kSlow = 3, kNone = 4, kCluster = 5, kExchange = 6 };
+        enum { kWhole = 0, kFast = 1, kWriter = 2, kSlow = 3, kNone = 4, kCluster = 5, kExchange = 6, kHalves = 7 };
+        const int kh0 = p.num_tiles - 2 * p.khalf_tiles;   // first K-half tile id (== num_tiles: none)
         uint32_t scount = 0, rphase = 0;
         bool ok = true;
         int cluster_bars = 0;                              // K-cluster mode: cluster barriers passed so far
+        int halves_in = 0;                                 // K halves: chunks of the partner's share that arrive by bulk copy
         // K-cluster mode: a CTA's partial tile parked at the start of its (idle) operand ring, same
         // float4 order as slab4; `ring` is the shared::cta address of this CTA's copy
         const uint32_t ring = s_stage;
@@ -769,14 +785,18 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             if constexpr (kRowScaled) a_scale = (row0 + lane < p.M) ? __ldg(p.sa + row0 + lane) : 0.f;
             const int nchunks = (narrow || sg) ? C::CHUNKS / 2 : C::CHUNKS;
             const bool whole = (kb0 == 0) && (kb1 == nkb);
+            // K half of a full-width tile: its chunks are dealt to the two halves as in a K cluster of two
+            const bool halves = p.khalf_tiles > 0 && tile >= kh0;
+            const int xk = (kc > 1) ? kc : (halves ? 2 : 1);
+            const int xr = (kc > 1) ? krank : (halves ? ((tile - kh0) & 1) : 0);
             auto chunk_inb = [&](int c) { return (row0 < p.M) && (colbase + c * 64 < p.N); };
-            // chunks this warp writes to Y: all of them, or in K-cluster mode those dealt to this CTA
-            auto chunk_valid = [&](int c) { return chunk_inb(c) && (kc == 1 || (c % kc) == krank); };
+            // chunks this warp writes to Y: all of them, or those dealt to this CTA (K cluster, K halves)
+            auto chunk_valid = [&](int c) { return chunk_inb(c) && (xk == 1 || (c % xk) == xr); };
             // This warp writes `nmine` chunks to Y, numbered i = 0, 1, ...: chunk i of the tile, or in K-cluster
             // mode chunk krank + kc i.  Staging buffers and R requests go by i, so that a CTA's chunks use
             // the buffers in turn whatever their position in the tile.
-            const int nmine = (kc == 1) ? nchunks : (nchunks > krank ? (nchunks - krank + kc - 1) / kc : 0);
-            auto chunk_of = [&](int i) { return (kc == 1) ? i : krank + kc * i; };
+            const int nmine = (xk == 1) ? nchunks : (nchunks > xr ? (nchunks - xr + xk - 1) / xk : 0);
+            auto chunk_of = [&](int i) { return (xk == 1) ? i : xr + xk * i; };
             auto issue_r = [&](int i) {                    // lane 0 only
                 const int c = chunk_of(i);
                 if (chunk_inb(c)) {
@@ -813,7 +833,7 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             int role = kWhole, s_first = 0, s_last = 0;
             unsigned int* ctr = nullptr;
             bool staged = false;   // the partner's partial already sits in the other accumulator buffer
-            if (!whole && kc == 1) {
+            if (!whole && kc == 1 && !halves) {
                 const long long ut = static_cast<long long>(tile - sk_base) * nkb;
                 s_first = sk_slot_of(U, slots, ut);
                 s_last = sk_slot_of(U, slots, ut + nkb - 1);
@@ -854,7 +874,7 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             if (!__all_sync(0xffffffffu, wt.wait(acc_full(b), aph, kWhereAccFull))) { ok = false; break; }
             tc_fence_after();
             if (q == 0 && lane == 0 && leader) KX_TRACE_POINT(p, slot, (scount - 1) * 4 + 2);
-            if (kc > 1 && q == 0 && lane == 0) KX_TRACE_POINT(p, blockIdx.x, 6);
+            if ((kc > 1 || (p.khalf_tiles > 0 && tile >= kh0)) && q == 0 && lane == 0) KX_TRACE_POINT(p, blockIdx.x, 6);
 
             auto release_acc = [&]() {                     // accumulator buffer b is drained
                 tc_fence_before();
@@ -938,6 +958,70 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 cluster_wait();
                 if (q == 0 && lane == 0) KX_TRACE_POINT(p, blockIdx.x, 5);
                 ++cluster_bars;
+            } else if (halves) {
+                // K halves: park the chunks the other half finishes in the workspace, raise this warp's flag,
+                // wait (bounded) for the same warp of the slot that holds the other half, then finish this
+                // half's chunks from the own accumulators plus the partner's parked share.  a + b is
+                // commutative: the bits do not depend on which half finishes a chunk.
+                role = kHalves;
+                float* dst = p.ws + (static_cast<size_t>(tile - kh0) * CTAS + cta_rank) * C::PART_FLOATS;
+#pragma unroll 1
+                for (int c = 0; c < nchunks; ++c) {
+                    if (!chunk_inb(c) || (c & 1) == xr) continue;
+                    uint32_t a[2][32];
+                    tmem_ld_32x32(tbase + c * 64, a[0]);
+                    tmem_ld_32x32(tbase + c * 64 + 32, a[1]);
+                    tmem_ld_wait();
+                    float4* d4 = slab4(dst, c);
+#pragma unroll
+                    for (int i = 0; i < 16; ++i)
+                        d4[i * 32] = make_float4(__uint_as_float(a[i >> 3][(i & 7) * 4 + 0]),
+                                                 __uint_as_float(a[i >> 3][(i & 7) * 4 + 1]),
+                                                 __uint_as_float(a[i >> 3][(i & 7) * 4 + 2]),
+                                                 __uint_as_float(a[i >> 3][(i & 7) * 4 + 3]));
+                }
+                __threadfence();
+                __syncwarp();
+                if (q == 0 && lane == 0) KX_TRACE_POINT(p, blockIdx.x, 4);
+                const int peer_tile = kh0 + ((tile - kh0) ^ 1);
+                unsigned int* const my_flag = p.counters + (static_cast<size_t>(tile) * CTAS + cta_rank) * 4 + q;
+                unsigned int* const peer_flag = p.counters + (static_cast<size_t>(peer_tile) * CTAS + cta_rank) * 4 + q;
+                uint32_t got = 0;
+                if (lane == 0) {
+                    atomicExch(my_flag, 1u);
+                    const unsigned long long t0 = globaltimer_ns();
+                    uint32_t spins = 0;
+                    for (;;) {
+                        if (ld_acquire_gpu_u32(peer_flag) != 0u) { got = 1u; break; }
+                        if ((++spins & 15u) == 0u) {
+                            if (*s_abort != 0) break;
+                            if (globaltimer_ns() - t0 > wt.limit_ns) { wt.raise(kWherePartials); break; }
+                        }
+                    }
+                    if (got) *peer_flag = 0u;              // zero between launches; the partner set it once
+                }
+                got = __shfl_sync(0xffffffffu, got, 0);
+                if (!got) { ok = false; break; }
+                if (q == 0 && lane == 0) KX_TRACE_POINT(p, blockIdx.x, 5);
+                // The partner's share of this warp's chunks: the first chunk is read straight from the workspace
+                // (L2) where it is used; the later ones come by one 8 KB bulk copy each into the operand ring, which
+                // is idle (this is the slot's last segment and its MMAs are done), and land while the first chunk is
+                // being finished (a bulk copy takes about twice as long as the loads, but nothing waits for it).
+                static_assert(((C::CHUNKS + 1) / 2) * 4 * 8192 <= STAGES * C::STAGE_BYTES, "partner share must fit in the ring");
+                for (int i = 1; i < nmine; ++i)
+                    if (chunk_inb(chunk_of(i))) ++halves_in;
+                if (lane == 0 && halves_in > 0) {
+                    const float* src = p.ws + (static_cast<size_t>(peer_tile - kh0) * CTAS + cta_rank) * C::PART_FLOATS;
+                    fence_proxy_async_all();
+                    mbar_arrive_expect_tx(xin_bar(q), static_cast<uint32_t>(halves_in) * 8192u);
+                    for (int i = 1; i < nmine; ++i) {
+                        const int c = chunk_of(i);
+                        if (chunk_inb(c))
+                            bulk_copy_g2s(ring + static_cast<uint32_t>(((c >> 1) * 4 + q) * 8192),
+                                          src + static_cast<size_t>(c * 4 + q) * 2048, 8192u, xin_bar(q));
+                    }
+                }
+                __syncwarp();
             } else if (!whole) {
                 if (staged) {
                     role = kFast;
@@ -1068,6 +1152,46 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         a4[3] = __float_as_uint(__uint_as_float(a4[3]) + t.w);
                     }
                 }
+                if (role == kHalves && ci == 1 && halves_in > 0) {   // the copies behind the first chunk have landed?
+                    if (!__all_sync(0xffffffffu, wt.wait(xin_bar(q), 0u, kWherePartials))) { ok = false; break; }
+                }
+                if (valid && role == kHalves) {
+                    // this slot's accumulators plus the share the other half parked in the workspace
+                    if (ci == 1 && q == 0 && lane == 0) KX_TRACE_POINT(p, blockIdx.x, 12);
+                    tmem_ld_32x32(tbase + c * 64, acc[0]);
+                    tmem_ld_32x32(tbase + c * 64 + 32, acc[1]);
+                    tmem_ld_wait();
+                    if (ci == 1 && q == 0 && lane == 0) KX_TRACE_POINT(p, blockIdx.x, 13);
+                    if (ci == 0) {
+                        const int peer_tile = kh0 + ((tile - kh0) ^ 1);
+                        const float4* s4 = slab4(p.ws + (static_cast<size_t>(peer_tile - kh0) * CTAS + cta_rank) * C::PART_FLOATS, c);
+                        float4 t[16];
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) t[i] = __ldcg(s4 + i * 32);
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            uint32_t* a4 = &acc[i >> 3][(i & 7) * 4];
+                            a4[0] = __float_as_uint(__uint_as_float(a4[0]) + t[i].x);
+                            a4[1] = __float_as_uint(__uint_as_float(a4[1]) + t[i].y);
+                            a4[2] = __float_as_uint(__uint_as_float(a4[2]) + t[i].z);
+                            a4[3] = __float_as_uint(__uint_as_float(a4[3]) + t[i].w);
+                        }
+                    } else {
+                        const uint32_t src = ring + ((((c >> 1) * 4 + q) * 16) * 32 + lane) * 16;
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            float4 t;
+                            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                                         : "=f"(t.x), "=f"(t.y), "=f"(t.z), "=f"(t.w)
+                                         : "r"(src + i * 512));
+                            uint32_t* a4 = &acc[i >> 3][(i & 7) * 4];
+                            a4[0] = __float_as_uint(__uint_as_float(a4[0]) + t.x);
+                            a4[1] = __float_as_uint(__uint_as_float(a4[1]) + t.y);
+                            a4[2] = __float_as_uint(__uint_as_float(a4[2]) + t.z);
+                            a4[3] = __float_as_uint(__uint_as_float(a4[3]) + t.w);
+                        }
+                    }
+                }
                 if (valid && role == kCluster) {
                     // sum the cluster's partials of this chunk in rank order (16 remote 16-byte loads in
                     // flight per rank)
@@ -1126,8 +1250,11 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
                     for (int i = 0; i < 64; ++i) acc[i >> 5][i & 31] = __float_as_uint(sum[i]);
                 }
-                if (ci == nmine - 1 && (role == kWhole || role == kFast || role == kExchange)) release_acc();
-                if (kc > 1 && q == 0 && lane == 0) KX_TRACE_POINT(p, blockIdx.x, 16 + ci * 4 + 0);
+                // (after the slot's last segment nobody waits for the buffer any more, and the releasing arrive
+                // would hold this warp until its outstanding loads have landed)
+                if (ci == nmine - 1 && !last_seg && (role == kWhole || role == kFast || role == kExchange || role == kHalves))
+                    release_acc();
+                if ((kc > 1 || halves) && q == 0 && lane == 0) KX_TRACE_POINT(p, blockIdx.x, 16 + ci * 4 + 0);
                 if (valid) {
                     if (has_r) {
                         if (!__all_sync(0xffffffffu, wt.wait(r_full(q, j), (rphase >> j) & 1u, kWhereRFull))) {
@@ -1136,7 +1263,7 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         }
                         rphase ^= (1u << j);
                     }
-                    if (kc > 1 && q == 0 && lane == 0) KX_TRACE_POINT(p, blockIdx.x, 16 + ci * 4 + 1);
+                    if ((kc > 1 || halves) && q == 0 && lane == 0) KX_TRACE_POINT(p, blockIdx.x, 16 + ci * 4 + 1);
                     // three phases, so that the shared-memory latencies overlap: the residual vectors of this
                     // lane's row are read first (all eight; four at a time in the row-scaled kinds, which have
                     // fewer registers to spare), then the outputs are formed, then written back in place
@@ -1191,7 +1318,7 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     }
                     fence_proxy_async_smem();
                     __syncwarp();
-                    if (kc > 1 && q == 0 && lane == 0) KX_TRACE_POINT(p, blockIdx.x, 16 + ci * 4 + 2);
+                    if ((kc > 1 || halves) && q == 0 && lane == 0) KX_TRACE_POINT(p, blockIdx.x, 16 + ci * 4 + 2);
                     if (lane == 0) {
                         tma_store_2d(&tmY, col0, row0, buf);
                         tma_store_commit();
@@ -1199,7 +1326,7 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         // because the next R slab is requested into the buffer it reads)
                         tma_store_wait_read<(NB > 1) ? 1 : 0>();
                     }
-                    if (kc > 1 && q == 0 && lane == 0) KX_TRACE_POINT(p, blockIdx.x, 16 + ci * 4 + 3);
+                    if ((kc > 1 || halves) && q == 0 && lane == 0) KX_TRACE_POINT(p, blockIdx.x, 16 + ci * 4 + 3);
                 } else if (lane == 0) {
                     tma_store_wait_read<0>();              // nothing stored for this chunk: drain the last store
                 }
@@ -1213,7 +1340,12 @@ kx_tile_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
             if ((role == kFast || role == kSlow) && lane == 0) *ctr = 0u;   // every segment has arrived: reset
             if (q == 0 && lane == 0 && leader) KX_TRACE_POINT(p, slot, (scount - 1) * 4 + 3);
-            if (kc > 1 && q == 0 && lane == 0) KX_TRACE_POINT(p, blockIdx.x, 7);
+            if ((kc > 1 || halves) && q == 0 && lane == 0) KX_TRACE_POINT(p, blockIdx.x, 7);
+        }
+        if (!ok && halves_in > 0) {
+            // gave up with bulk copies into this CTA's shared memory possibly still in flight: let them land
+            uint32_t spins = 0;
+            while (!mbar_try_wait(xin_bar(q), 0u) && ++spins < (1u << 20)) {}
         }
         if (kc > 2) {
             // peers may still be reading this CTA's partial: second barrier; on a give-up path the

@@ -160,6 +160,16 @@ __device__ __forceinline__ void bulk_copy_to_cta(uint32_t dst_cluster, uint32_t 
         "r"(src_cta), "r"(bytes), "r"(bar_cluster)
         : "memory");
 }
+// Untiled bulk copy global -> this CTA's shared memory (both 16-byte aligned, size a multiple of 16 bytes); the
+// bytes are counted on `bar` (a barrier of this CTA).
+__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst_smem, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst_smem),
+                 "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+// Orders this thread's earlier generic-proxy accesses (here: an acquire load that made another CTA's global
+// stores visible) before its later asynchronous-proxy operations.
+__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
 // Ask for a 2-D tile to be brought into L2 (no shared-memory destination, no completion signal).
 // L2 is the coherence point of the device, so a tile prefetched early still reflects any later
 // write made through L2 before it is actually loaded.

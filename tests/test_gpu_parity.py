@@ -158,6 +158,50 @@ def test_stream_k_first_exact_integer_arithmetic(ov, max_ctas, M, N, K):
         kx.kx_plan_query(512, 512, 512, ov=kx.make_override(path=T, block_n=256, cta_pair=1, max_ctas=4, stream_k=3))
 
 
+@pytest.mark.parametrize("ov,max_ctas,M,N,K", [
+    (dict(path=T, block_n=256, cta_pair=2), 12, 640, 1280, 520),     # 15 pair tiles on 6 slots: 3 left over, 6 K halves
+    (dict(path=T, block_n=256, cta_pair=2, stages=3), 12, 640, 1280, 4096),
+    (dict(path=T, block_n=256, cta_pair=1), 10, 640, 1280, 1096),    # 25 tiles on 10 slots: 5 left over, odd k-block count
+    (dict(path=T, block_n=128, cta_pair=2), 12, 700, 520, 264),      # ragged rows and columns
+    (dict(path=T, block_n=192, cta_pair=1, stages=2), 10, 300, 776, 2048),
+    (dict(path=T, block_n=128, cta_pair=1, stages=3), 9, 300, 776, 136),
+    (dict(path=T, block_n=256, cta_pair=2), 0, 4096, 2560, 264),     # full grid: 160 pair tiles on 74 slots, 12 left over
+], ids=["pair256", "pair256-2kb-longk", "single256", "pair128-ragged", "single192-2kb", "single128-2kb", "pair256-fullgrid"])
+def test_k_halves_tail_exact_integer_arithmetic(ov, max_ctas, M, N, K):
+    """Tiles left over after the full waves run as two K halves on two slots, which swap through the workspace the
+    chunks the other one finishes.  Integer-valued data: bit-exact, the same bits in place and on a second run
+    (the flags are back at zero), also without bias and residual."""
+    o = dict(ov, max_ctas=max_ctas, narrow_tail=3)
+    info = kx.kx_plan_query(M, N, K, ov=kx.make_override(**o))
+    assert info.workspace_bytes > 0 and info.narrow_tiles == 0 and info.stream_k == 0
+    X, W, b, R = ternary_case(M, N, K, seed=29)
+    ref = oracle.outproj(X, W, b, R)
+    y = run(X, W, b, R, o)
+    ok, msg = kt.gate_exact(y, ref)
+    assert ok, msg
+    assert np.array_equal(run(X, W, b, R.copy(), o, inplace=True), y)
+    assert np.array_equal(run(X, W, b, R, o), y)
+    ok, msg = kt.gate_exact(run(X, W, None, None, o), oracle.outproj(X, W))
+    assert ok, msg
+    with pytest.raises(kx.KxError):            # nothing is left over
+        kx.kx_plan_query(512, 512, 512, ov=kx.make_override(path=T, block_n=256, cta_pair=1, max_ctas=4, narrow_tail=3))
+
+
+def test_tail_choice_follows_the_reduction_length():
+    """Automatic plans: tiles left over after the full waves run as K halves from 64 k-blocks on, as half-width
+    tiles below, and whole when neither fits; the 8-bit entry points never take K halves."""
+    long_k = kx.kx_plan_query(4096, 4096, 4096)
+    assert long_k.narrow_tiles == 0 and long_k.workspace_bytes > 0 and long_k.stream_k == 0 and long_k.tiles == 290
+    short_k = kx.kx_plan_query(4096, 4096, 2048)
+    assert short_k.narrow_tiles == 68 and short_k.workspace_bytes == 0
+    none = kx.kx_plan_query(8192, 8192, 8192)                  # 1024 tiles on 74 slots: 62 left over, too many to split
+    assert none.narrow_tiles == 0 and none.workspace_bytes == 0 and none.tiles == 1024
+    X, W, b, R = ternary_case(1024, 4096, 4096, seed=31)
+    y = run(X, W, b, R, None, entry="fused")                   # 64 pair tiles: one wave, nothing left over
+    ok, msg = kt.gate_exact(y, oracle.outproj(X, W, b, R))
+    assert ok, msg
+
+
 @pytest.mark.parametrize("group", [1, 3, 16, 64])
 @pytest.mark.parametrize("pair", [1, 2])
 def test_raster_group_exact_integer_arithmetic(group, pair):

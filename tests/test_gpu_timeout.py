@@ -27,9 +27,10 @@ WAIT_FULL = 2   # the MMA issuer's wait for a filled stage
                                 dict(path=S, block_n=128, split_k=2, cluster_reduce=2),
                                 dict(path=S, block_n=32, split_k=4, cluster_reduce=3),
                                 dict(path=T, block_n=256, cta_pair=2, k_cluster=2),
-                                dict(path=T, block_n=128, cta_pair=1, stream_k=3, max_ctas=3)],
+                                dict(path=T, block_n=128, cta_pair=1, stream_k=3, max_ctas=3),
+                                dict(path=T, block_n=128, cta_pair=1, narrow_tail=3, max_ctas=3)],
                          ids=["tile", "pair", "swap-cluster", "pair-streamk", "tile-kcluster", "swap-workspace",
-                              "swap-cluster-pull", "swap-cluster-push", "pair-kcluster", "streamk-first"])
+                              "swap-cluster-pull", "swap-cluster-push", "pair-kcluster", "streamk-first", "k-halves"])
 def test_wait_gives_up_and_context_survives(ov):
     import time
     M, N, K = (128 if ov.get("block_n", 0) >= 128 else 30), 512, 512
