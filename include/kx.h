@@ -163,11 +163,14 @@ typedef struct kx_plan_info {
  * Shared state and concurrency.  Each device has ONE FP32 workspace, one array of tile counters and
  * one status word, shared by every stream and host thread.  Calls whose plan uses the workspace
  * (kx_plan_info.workspace_bytes > 0: split-K through the workspace, i.e. more than 8 splits, a capped
- * grid or cluster_reduce = 1, and stream-K) must not overlap on the GPU with one another: order them
- * on one stream or with events, as for kx_outproj_residual_noalloc's built-in scratch.  The heuristic
- * plans of kx_outproj_residual / kx_gemm_bf16 / _strided / _batched use no workspace (cluster
- * reductions and whole tiles), so those calls may overlap freely; an entry of the built-in measured
- * plan table may name a workspace plan for its shape, and kx_plan_query tells (workspace_bytes).  kx_outproj_residual_host also owns
+ * grid or cluster_reduce = 1, stream-K, and the K-halves tail) must not overlap on the GPU with one
+ * another: order them on one stream or with events, as for kx_outproj_residual_noalloc's built-in
+ * scratch.  The heuristic plans of kx_outproj_residual / kx_gemm_bf16 / _strided / _batched use no
+ * workspace (cluster reductions and whole tiles) with ONE exception: large-M BF16 shapes with K >= 4096
+ * whose tiles do not fill the last wave (at most half of it) take the K-halves tail, which does (the
+ * 4096^3 projection is one).  kx_plan_query tells (workspace_bytes), also for an entry of the built-in
+ * measured plan table; a caller that must overlap such calls passes narrow_tail = 2 (or 1) through
+ * kx_outproj_residual_ex and gets the workspace-free plan.  kx_outproj_residual_host also owns
  * one staging buffer and one set of copy streams per device: its calls must not overlap each other.
  * Host-side entry is thread-safe (the per-device state is built once under a lock; descriptor caches
  * are per thread).
