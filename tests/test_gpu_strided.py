@@ -22,9 +22,10 @@ def wide(bits, ld, pad_value=0x7FC0):
     return buf.view(torch.bfloat16)
 
 
-# small-M path (cluster and workspace split-K), single-CTA tiles, K cluster, CTA pairs with a half-width tail
+# small-M path (cluster and workspace split-K), single-CTA tiles, K cluster, CTA pairs with a half-width tail and
+# (last shape: 110 pair tiles of 192 columns on 74 slots, 64 k-blocks) with a K-halves tail
 @pytest.mark.parametrize("M,N,K", [(1, 520, 1096), (37, 2048, 2048), (200, 1024, 4096), (300, 520, 264), (512, 2048, 2048),
-                                   (1000, 776, 1096), (2381, 4096, 512)])
+                                   (1000, 776, 1096), (2381, 4096, 512), (2560, 2048, 4096)])
 def test_strided_equals_dense(M, N, K):
     d = inputs.make_inputs(inputs.Workload("t", M, N, K, 900 + M, True, True), stress=True)
     Yd = kt.nan_filled(M, N)
