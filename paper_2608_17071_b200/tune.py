@@ -70,6 +70,10 @@ def candidates(M: int, N: int, K: int, kx):
             out.append(dict(path=T, block_n=256, cta_pair=2, raster_group=rg))
         out.append(dict(path=T, block_n=256, cta_pair=2, stages=5))
         out.append(dict(path=T, block_n=256, cta_pair=2, narrow_tail=1))
+        # the two tails for left-over tiles, each forced (the heuristic switches at 64 k-blocks)
+        for bn in (256, 192):
+            out.append(dict(path=T, block_n=bn, cta_pair=2, narrow_tail=3))
+            out.append(dict(path=T, block_n=bn, cta_pair=2, narrow_tail=2))
         out.append(dict(path=T, block_n=256, cta_pair=1, narrow_tail=1))
         for bn in (256, 192, 128):
             for kc in (2, 4):
