@@ -1549,7 +1549,13 @@ bool aligned4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3u) == 0
 // fmt: 0 = INT8 codes, 1 = FP8 E4M3 codes (one scale per row); 2 = FP8 E4M3 codes with one E8M0 scale per 32
 // elements; 3 = E2M1 codes with one E4M3 scale per 16 elements and a tensor scale
 int launch_rowquant(const QuantParams& qp, bool norm, int fmt, cudaStream_t stream, int sm_count) {
-    if (qp.N <= kRowCodeMaxN && !dev_old_rows()) return launch_rowcode(qp, norm, fmt, stream, sm_count);
+    // The short-row kernel takes every fused form it has (it halves their instruction count), the plain code
+    // books of rows up to 3072 elements and those of large matrices (from 64 Mi elements on: 16384 x 4096 INT8
+    // 31.2 vs 32.6 us, 28672 x 4096 52.7 vs 55.2 us); in between the plain rows are HBM-bound in the
+    // one-row-per-CTA kernel below, measured 3-7 % faster there (4096^2: 9.4 vs 10.0 us block-scaled FP8, 10.7 vs
+    // 11.4 us 4-bit).  Both give the same bits: a code book has one correct answer.
+    if (qp.N <= kRowCodeMaxN && (norm || qp.N <= 3072 || qp.M * qp.N >= (64ll << 20)) && !dev_old_rows())
+        return launch_rowcode(qp, norm, fmt, stream, sm_count);
     cudaLaunchConfig_t cfg;
     std::memset(&cfg, 0, sizeof cfg);
     const long long nvec = qp.N / 8;
