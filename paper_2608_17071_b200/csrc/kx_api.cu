@@ -1554,7 +1554,8 @@ int launch_rowquant(const QuantParams& qp, bool norm, int fmt, cudaStream_t stre
     // 31.2 vs 32.6 us, 28672 x 4096 52.7 vs 55.2 us); in between the plain rows are HBM-bound in the
     // one-row-per-CTA kernel below, measured 3-7 % faster there (4096^2: 9.4 vs 10.0 us block-scaled FP8, 10.7 vs
     // 11.4 us 4-bit).  Both give the same bits: a code book has one correct answer.
-    if (qp.N <= kRowCodeMaxN && (norm || qp.N <= 3072 || qp.M * qp.N >= (64ll << 20)) && !dev_old_rows())
+    if (qp.N <= (norm ? kRowCodeMaxN : kRowCodeMaxPlainN) && (norm || qp.N <= 3072 || qp.M * qp.N >= (64ll << 20)) &&
+        !dev_old_rows())
         return launch_rowcode(qp, norm, fmt, stream, sm_count);
     cudaLaunchConfig_t cfg;
     std::memset(&cfg, 0, sizeof cfg);

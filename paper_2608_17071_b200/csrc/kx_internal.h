@@ -50,6 +50,7 @@ struct QuantParams {
 // The kernels for rows of at most kRowCodeMaxN elements (kx_rowcode.cuh).  fmt: 0 INT8 / 1 E4M3 codes with one
 // scale per row, 2 / 3 the block-scaled 8-bit / 4-bit formats, 4 the BF16 RMSNorm itself (qp.Q0 = output).
 constexpr int kRowCodeMaxN = 8192;
+constexpr int kRowCodeMaxPlainN = 16384;   // code books without normalisation
 // rowcode_setup raises the kernels' shared-memory limit once per device.
 int rowcode_setup();
 int launch_rowcode(const QuantParams& qp, bool norm, int fmt, cudaStream_t stream, int sm_count);

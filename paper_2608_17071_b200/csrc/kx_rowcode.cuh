@@ -1,11 +1,12 @@
-// kx_rowcode_kernel: the row kernels of Appendix A, Algorithm 7 for rows of at most 8192 elements -
+// kx_rowcode_kernel: the row kernels of Appendix A, Algorithm 7 for rows of at most 8192 elements (plain code
+// books: 16384, with up to eight vectors per thread) -
 // RMSNorm ("add + RMSNorm" after the projection), the per-row and per-block code books ("activation
 // quantization", "quantize gate/up weights") and the two fused ("fused add + RMSNorm + activation
 // quantization").  Same arithmetic, element by element, as kx_rmsnorm_kernel / kx_rowquant_kernel
 // (which keep the longer rows); what differs is how the work is laid out, because at these row
 // lengths the older kernels are bound by instruction issue, not by HBM:
 //
-//   * G = 128 or 256 threads share a row and a thread owns NV <= 4 16-byte vectors of it (32 elements
+//   * G = 128 or 256 threads share a row and a thread owns NV <= 4 (plain code books: 8) 16-byte vectors of it (32 elements
 //     when the row has 4096), so the fixed per-row work of a thread (two shuffle trees, two group
 //     barriers, the divisions) is spread over twice as many elements; a CTA of 256 threads works on
 //     256 / G neighbouring rows at once, each group with a named barrier of its own;

@@ -75,3 +75,35 @@ def test_row_kernels_random_shapes(chunk):
         assert np.array_equal(Q4.cpu().numpy(), Qr) and np.array_equal(SF4.cpu().numpy(), chunked_nv(Sr, N)), (M, N)
         code, detail = kx.kx_last_device_status()
         assert code == kx.KX_OK
+
+
+@pytest.mark.parametrize("M,N", [(4700, 14336), (6000, 11264), (7000, 9728), (4200, 16384)])
+def test_plain_code_books_of_long_rows_in_large_matrices(M, N):
+    """From 64 Mi elements on, the plain code books of rows up to 16384 elements run in the short-row kernel with
+    five to eight vectors per thread (rows that fill their threads exactly and rows that do not): every format,
+    bit for bit."""
+    assert M * N >= 64 << 20
+    H = inputs.normal_bf16(8100 + N, "R", (M, N), 1.7)
+    Hd = kt.to_dev(H)
+    Q = torch.full((M, N), 77, dtype=torch.int8, device="cuda")
+    S = torch.full((M,), float("nan"), dtype=torch.float32, device="cuda")
+    kx.kx_quantize_rows_int8(Hd, Q, S)
+    Qr, Sr = oracle.quantize_rows(H)
+    assert np.array_equal(S.cpu().numpy(), Sr) and np.array_equal(Q.cpu().numpy(), Qr)
+    del Q
+    Q8 = torch.zeros((M, N), dtype=torch.uint8, device="cuda").view(F8)
+    kx.kx_quantize_rows_fp8(Hd, Q8, S)
+    Qr, Sr = oracle.quantize_rows_fp8(H)
+    assert np.array_equal(host8(Q8), Qr) and np.array_equal(S.cpu().numpy(), Sr)
+    SF = torch.full((kx.kx_mx_scale_bytes(M, N),), 0xEE, dtype=torch.uint8, device="cuda")
+    kx.kx_quantize_rows_mxfp8(Hd, Q8, SF)
+    Qr, Er = oracle.quantize_rows_mx(H)
+    assert np.array_equal(host8(Q8), Qr) and np.array_equal(SF.cpu().numpy(), chunked_mx(Er, N))
+    del Q8
+    gs = 8.0 / 2688.0
+    Q4 = torch.full((M, N // 2), 0x55, dtype=torch.uint8, device="cuda")
+    SF4 = torch.full((kx.kx_nvfp4_scale_bytes(M, N),), 0xEE, dtype=torch.uint8, device="cuda")
+    kx.kx_quantize_rows_nvfp4(Hd, gs, Q4, SF4)
+    Qr, Sr = oracle.quantize_rows_nvfp4(H, gs)
+    assert np.array_equal(Q4.cpu().numpy(), Qr) and np.array_equal(SF4.cpu().numpy(), chunked_nv(Sr, N))
+    assert kx.kx_last_device_status()[0] == kx.KX_OK
